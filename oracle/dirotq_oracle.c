@@ -1,0 +1,241 @@
+/*
+ * DiRotQ rotation-aware W4A4 linear layer -- plain CPU oracle (TEST INFRASTRUCTURE).
+ *
+ * This file is a checker, not a product path: only the tests, the smoke check and
+ * the benchmark's CPU-baseline leg may call it.  It shares no code with the CUDA
+ * library.  Everything is written as the definition reads: fp64 arithmetic,
+ * scalar quantizer, naive triple-loop integer GEMM, no blocking, no fusion.
+ *
+ * Method (paper Sec. 4.2, Eq. 5):  Y ~= [X U_h , Q4(X~_l)] [W~_h ; Q4(W~_l)]
+ *   with  V = [U_h , U_l R]  (called Q here),  W~ = V^T W  folded offline,
+ *   Q4 = symmetric 4-bit per-group quantizer of Eq. 1 with z = 0,
+ *   s = max|.|/q_max, q_max = 2^(4-1)-1 = 7  (Sec. 3), groups along K (Sec. 5.1:
+ *   group size 64, 16-bit scales).
+ *
+ * "Deployed" rounding points (where the product stores a narrow type, the oracle
+ * rounds at the same point; everything in between is fp64):
+ *   - x and the online rotation matrix are bf16 values,
+ *   - the r high-precision coefficients and the r high rows of W~ are bf16,
+ *   - every scale is a bf16 value and the rounded scale is used to divide,
+ *   - the output is bf16.
+ * Readings taken where the paper is silent (listed again in the design notes):
+ *   groups are counted from the first low-precision column; the last group may be
+ *   ragged; rounding is half-to-even; codes are clipped to [-7, 7]; a group whose
+ *   absmax is zero has scale 0 and codes 0; bias is added before the final rounding.
+ *
+ * Parity pins: see tests/test_oracle_*.py (orthogonality, Eq. 4 identity, brute
+ * force nearest-level search, exhaustive integer products, textbook RTN special
+ * case, integer path == dequantized path).  The choices above that no printed
+ * value fixes (group axis/alignment, bf16 scales, tie rule, clip range) are
+ * "parity unpinned" against the authors' implementation.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---------- bf16 <-> double ------------------------------------------------- */
+
+double dq_bf16_to_double(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Round an fp64 value straight to bf16 (8 significant bits), nearest, ties to even. */
+uint16_t dq_double_to_bf16(double v) {
+    if (v != v) return 0x7FC0;
+    uint16_t sign = signbit(v) ? 0x8000 : 0;
+    double a = fabs(v);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return sign | 0x7F80;
+    int e = ilogb(a);                 /* 2^e <= a < 2^(e+1) */
+    if (e < -126) e = -126;           /* subnormal bf16: fixed quantum 2^-133 */
+    double quantum = ldexp(1.0, e - 7);
+    double m = rint(a / quantum);     /* default rounding mode: ties to even */
+    double r = m * quantum;           /* exactly representable in float */
+    float f = (float)r;
+    if (isinf(f) || r > 3.3895313892515355e38) return sign | 0x7F80;
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    return sign | (uint16_t)(u >> 16);
+}
+
+void dq_round_bf16(const double* src, uint16_t* dst, int64_t n) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) dst[i] = dq_double_to_bf16(src[i]);
+}
+
+/* ---------- Eq. 1, symmetric, one group -------------------------------------- */
+
+/* v[0..n): the group's real elements (stride in elements).  Writes the bf16 scale,
+ * the codes, and (if t != NULL) the pre-rounding quotients v/s. */
+void dq_quantize_group(const double* v, int n, int64_t stride, uint16_t* scale_bits, int8_t* codes,
+                       int64_t code_stride, double* t, int64_t t_stride) {
+    double a = 0.0;
+    for (int i = 0; i < n; ++i) {
+        double x = fabs(v[i * stride]);
+        if (x > a) a = x;
+    }
+    uint16_t sb = (a == 0.0) ? 0 : dq_double_to_bf16(a / 7.0);   /* s = max|X| / q_max */
+    double s = dq_bf16_to_double(sb);
+    *scale_bits = sb;
+    for (int i = 0; i < n; ++i) {
+        double q = 0.0, ti = 0.0;
+        if (s != 0.0) {
+            ti = v[i * stride] / s;
+            q = rint(ti);                 /* half to even */
+            if (q > 7.0) q = 7.0;         /* clip to [q_min, q_max] */
+            if (q < -7.0) q = -7.0;
+        }
+        codes[i * code_stride] = (int8_t)q;
+        if (t) t[i * t_stride] = ti;
+    }
+}
+
+/* ---------- offline: fold and weight quantization (Eq. 5, left factor) -------- */
+
+/* Wt[K,N] = Q^T W   (Q[K,K] column j = basis vector j; W[K,N]) */
+void dq_fold(const double* Q, const double* W, double* Wt, int K, int N) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < K; ++i) {
+        double* out = Wt + (int64_t)i * N;
+        for (int n = 0; n < N; ++n) out[n] = 0.0;
+        for (int k = 0; k < K; ++k) {
+            double q = Q[(int64_t)k * K + i];
+            const double* w = W + (int64_t)k * N;
+            for (int n = 0; n < N; ++n) out[n] += q * w[n];
+        }
+    }
+}
+
+/* Rows < r of Wt -> bf16 Wh[r,N].  Rows >= r: per (group, column) scale + codes.
+ * wcodes[K_l,N], wscales[n_g,N], wt (optional) [K_l,N] pre-rounding quotients. */
+void dq_prepare_weights(const double* Wt, int K, int N, int r, int G, uint16_t* Wh, int8_t* wcodes,
+                        uint16_t* wscales, double* wt) {
+    int K_l = K - r;
+    int n_g = (K_l + G - 1) / G;
+    dq_round_bf16(Wt, Wh, (int64_t)r * N);
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int g = 0; g < n_g; ++g) {
+            int j0 = g * G;
+            int len = (j0 + G <= K_l) ? G : (K_l - j0);
+            dq_quantize_group(Wt + (int64_t)(r + j0) * N + n, len, N, wscales + (int64_t)g * N + n,
+                              wcodes + (int64_t)j0 * N + n, N, wt ? wt + (int64_t)j0 * N + n : NULL, N);
+        }
+    }
+}
+
+/* ---------- online step 1: rotation  x~ = x Q_b  (Sec. 4.2) -------------------- */
+
+void dq_rotate(const uint16_t* x_bits, const uint16_t* Qb_bits, double* xt, int M, int K) {
+    double* Qd = (double*)malloc(sizeof(double) * (size_t)K * K);
+    for (int64_t i = 0; i < (int64_t)K * K; ++i) Qd[i] = dq_bf16_to_double(Qb_bits[i]);
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        double* out = xt + (int64_t)m * K;
+        for (int c = 0; c < K; ++c) out[c] = 0.0;
+        for (int k = 0; k < K; ++k) {
+            double xv = dq_bf16_to_double(x_bits[(int64_t)m * K + k]);
+            const double* q = Qd + (int64_t)k * K;
+            for (int c = 0; c < K; ++c) out[c] += xv * q[c];
+        }
+    }
+    free(Qd);
+}
+
+/* ---------- online steps 2-3: split, per-token per-group quantization ---------- */
+
+/* xt[M,K] -> xh bf16 [M,r]; codes [M,K_l]; scales bf16 [M,n_g]; t (optional) [M,K_l] */
+void dq_split_quantize(const double* xt, int M, int K, int r, int G, uint16_t* xh, int8_t* codes,
+                       uint16_t* scales, double* t) {
+    int K_l = K - r;
+    int n_g = (K_l + G - 1) / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const double* row = xt + (int64_t)m * K;
+        for (int i = 0; i < r; ++i) xh[(int64_t)m * r + i] = dq_double_to_bf16(row[i]);
+        for (int g = 0; g < n_g; ++g) {
+            int j0 = g * G;
+            int len = (j0 + G <= K_l) ? G : (K_l - j0);
+            dq_quantize_group(row + r + j0, len, 1, scales + (int64_t)m * n_g + g,
+                              codes + (int64_t)m * K_l + j0, 1, t ? t + (int64_t)m * K_l + j0 : NULL, 1);
+        }
+    }
+}
+
+/* ---------- online step 4: integer GEMM per group ------------------------------ */
+
+/* P[g,m,n] = sum_{j in group g} qx[m,j] * qw[j,n]   (int32, naive triple loop) */
+void dq_int_gemm(const int8_t* qx, const int8_t* qw, int32_t* P, int M, int K_l, int N, int G) {
+    int n_g = (K_l + G - 1) / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int g = 0; g < n_g; ++g) {
+            int j0 = g * G;
+            int j1 = (j0 + G <= K_l) ? j0 + G : K_l;
+            for (int n = 0; n < N; ++n) {
+                int32_t acc = 0;
+                for (int j = j0; j < j1; ++j)
+                    acc += (int32_t)qx[(int64_t)m * K_l + j] * (int32_t)qw[(int64_t)j * N + n];
+                P[((int64_t)g * M + m) * N + n] = acc;
+            }
+        }
+    }
+}
+
+/* ---------- online step 5: dequantize, add the 16-bit branch and the bias ------- */
+
+/* y[m,n] = sum_g sx[m,g] sw[g,n] P[g,m,n] + sum_{i<r} xh[m,i] Wh[i,n] + bias[n]
+ * y64 (optional): value before the final rounding; ybits: bf16 result. */
+void dq_combine(const int32_t* P, const uint16_t* sx, const uint16_t* sw, const uint16_t* xh,
+                const uint16_t* Wh, const uint16_t* bias, int M, int N, int r, int n_g, double* y64,
+                uint16_t* ybits) {
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int g = 0; g < n_g; ++g)
+                acc += dq_bf16_to_double(sx[(int64_t)m * n_g + g]) * dq_bf16_to_double(sw[(int64_t)g * N + n]) *
+                       (double)P[((int64_t)g * M + m) * N + n];
+            double lr = 0.0;
+            for (int i = 0; i < r; ++i)
+                lr += dq_bf16_to_double(xh[(int64_t)m * r + i]) * dq_bf16_to_double(Wh[(int64_t)i * N + n]);
+            double v = acc + lr + (bias ? dq_bf16_to_double(bias[n]) : 0.0);
+            if (y64) y64[(int64_t)m * N + n] = v;
+            ybits[(int64_t)m * N + n] = dq_double_to_bf16(v);
+        }
+    }
+}
+
+/* ---------- plain fp64 product, used by the ideal (nothing quantized) mode ------ */
+
+void dq_matmul(const double* A, const double* B, double* C, int M, int K, int N) {
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        double* out = C + (int64_t)m * N;
+        for (int n = 0; n < N; ++n) out[n] = 0.0;
+        for (int k = 0; k < K; ++k) {
+            double a = A[(int64_t)m * K + k];
+            const double* b = B + (int64_t)k * N;
+            for (int n = 0; n < N; ++n) out[n] += a * b[n];
+        }
+    }
+}
+
+int dq_num_threads(void) {
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp master
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

@@ -1,0 +1,211 @@
+"""ctypes front end of the plain-C DiRotQ oracle (TEST INFRASTRUCTURE, not a product path).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module.  It compiles ``dirotq_oracle.c`` with gcc on first use and exposes
+the steps of the method one by one, in the order of the paper's Eq. 5:
+
+    prepare (offline):  W~ = Q^T W;  rows < r -> bf16;  rows >= r -> INT4 codes + bf16 scales
+    rotate:             x~ = x Q_b           (Q_b = bf16(Q), fp64 accumulation)
+    split/quantize:     x~_h -> bf16;  x~_l -> per token, per group INT4 codes + bf16 scales (Eq. 1, z = 0)
+    int_gemm:           P_g = q_x q_w per group (int32)
+    combine:            y = bf16( sum_g s_x s_w P_g + x~_h W~_h + bias )
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dirotq_oracle.c")
+_LIB = os.path.join(_HERE, "libdirotq_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over rows).  Returns the library path."""
+    with _lock:
+        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+            tmp = _LIB + f".{os.getpid()}.tmp"
+            subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-ffp-contract=off",
+                                   "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.dq_bf16_to_double.restype = ctypes.c_double
+        _lib.dq_bf16_to_double.argtypes = [ctypes.c_uint16]
+        _lib.dq_double_to_bf16.restype = ctypes.c_uint16
+        _lib.dq_double_to_bf16.argtypes = [ctypes.c_double]
+        _lib.dq_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a: np.ndarray | None):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def num_threads() -> int:
+    return int(_load().dq_num_threads())
+
+
+def bf16_round(a) -> np.ndarray:
+    """fp64 -> bf16 bits (uint16), nearest, ties to even."""
+    a = _c(a, np.float64)
+    out = np.empty(a.shape, dtype=np.uint16)
+    _load().dq_round_bf16(_p(a), _p(out), ctypes.c_int64(a.size))
+    return out
+
+
+def bf16_to_f64(bits) -> np.ndarray:
+    bits = np.asarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def quantize_group(v):
+    """Eq. 1 (symmetric, 4 bit) on one group.  Returns (scale_bits, codes, t)."""
+    v = _c(v, np.float64).ravel()
+    n = v.size
+    sb = ctypes.c_uint16(0)
+    codes = np.zeros(n, dtype=np.int8)
+    t = np.zeros(n, dtype=np.float64)
+    _load().dq_quantize_group(_p(v), ctypes.c_int(n), ctypes.c_int64(1), ctypes.byref(sb), _p(codes),
+                              ctypes.c_int64(1), _p(t), ctypes.c_int64(1))
+    return int(sb.value), codes, t
+
+
+def fold(Q, W) -> np.ndarray:
+    """W~ = Q^T W in fp64 (Eq. 5).  Q [K,K] (unrounded), W [K,N]."""
+    Q = _c(Q, np.float64)
+    W = _c(W, np.float64)
+    K, N = W.shape
+    assert Q.shape == (K, K)
+    Wt = np.empty((K, N), dtype=np.float64)
+    _load().dq_fold(_p(Q), _p(W), _p(Wt), ctypes.c_int(K), ctypes.c_int(N))
+    return Wt
+
+
+def prepare_weights(Wt, r: int, G: int, want_t: bool = False):
+    """Split the folded weight at row r; bf16 high rows, INT4 codes + bf16 scales for the rest."""
+    Wt = _c(Wt, np.float64)
+    K, N = Wt.shape
+    K_l = K - r
+    n_g = -(-K_l // G)
+    Wh = np.empty((r, N), dtype=np.uint16)
+    wcodes = np.empty((K_l, N), dtype=np.int8)
+    wscales = np.empty((n_g, N), dtype=np.uint16)
+    wt = np.empty((K_l, N), dtype=np.float64) if want_t else None
+    _load().dq_prepare_weights(_p(Wt), ctypes.c_int(K), ctypes.c_int(N), ctypes.c_int(r), ctypes.c_int(G),
+                               _p(Wh), _p(wcodes), _p(wscales), _p(wt))
+    return {"Wh": Wh, "wcodes": wcodes, "wscales": wscales, "wt": wt}
+
+
+def rotate(x_bits, Qb_bits) -> np.ndarray:
+    """x~ = x Q_b with fp64 accumulation over bf16 inputs."""
+    x_bits = _c(x_bits, np.uint16)
+    Qb_bits = _c(Qb_bits, np.uint16)
+    M, K = x_bits.shape
+    assert Qb_bits.shape == (K, K)
+    xt = np.empty((M, K), dtype=np.float64)
+    _load().dq_rotate(_p(x_bits), _p(Qb_bits), _p(xt), ctypes.c_int(M), ctypes.c_int(K))
+    return xt
+
+
+def split_quantize(xt, r: int, G: int, want_t: bool = True):
+    xt = _c(xt, np.float64)
+    M, K = xt.shape
+    K_l = K - r
+    n_g = -(-K_l // G)
+    xh = np.empty((M, r), dtype=np.uint16)
+    codes = np.empty((M, K_l), dtype=np.int8)
+    scales = np.empty((M, n_g), dtype=np.uint16)
+    t = np.empty((M, K_l), dtype=np.float64) if want_t else None
+    _load().dq_split_quantize(_p(xt), ctypes.c_int(M), ctypes.c_int(K), ctypes.c_int(r), ctypes.c_int(G),
+                              _p(xh), _p(codes), _p(scales), _p(t))
+    return {"xh": xh, "codes": codes, "scales": scales, "t": t}
+
+
+def int_gemm(qx, qw, G: int) -> np.ndarray:
+    """P[g,m,n] = sum over group g of qx[m,j] qw[j,n]  (int32)."""
+    qx = _c(qx, np.int8)
+    qw = _c(qw, np.int8)
+    M, K_l = qx.shape
+    N = qw.shape[1]
+    assert qw.shape[0] == K_l
+    n_g = -(-K_l // G)
+    P = np.empty((n_g, M, N), dtype=np.int32)
+    _load().dq_int_gemm(_p(qx), _p(qw), _p(P), ctypes.c_int(M), ctypes.c_int(K_l), ctypes.c_int(N), ctypes.c_int(G))
+    return P
+
+
+def combine(P, sx, sw, xh, Wh, bias):
+    P = _c(P, np.int32)
+    n_g, M, N = P.shape
+    sx = _c(sx, np.uint16)
+    sw = _c(sw, np.uint16)
+    xh = _c(xh, np.uint16)
+    Wh = _c(Wh, np.uint16)
+    r = xh.shape[1]
+    assert sx.shape == (M, n_g) and sw.shape == (n_g, N) and Wh.shape == (r, N)
+    bias = None if bias is None else _c(bias, np.uint16)
+    y64 = np.empty((M, N), dtype=np.float64)
+    yb = np.empty((M, N), dtype=np.uint16)
+    _load().dq_combine(_p(P), _p(sx), _p(sw), _p(xh), _p(Wh), _p(bias), ctypes.c_int(M), ctypes.c_int(N),
+                       ctypes.c_int(r), ctypes.c_int(n_g), _p(y64), _p(yb))
+    return y64, yb
+
+
+def matmul(A, B) -> np.ndarray:
+    A = _c(A, np.float64)
+    B = _c(B, np.float64)
+    M, K = A.shape
+    N = B.shape[1]
+    C = np.empty((M, N), dtype=np.float64)
+    _load().dq_matmul(_p(A), _p(B), _p(C), ctypes.c_int(M), ctypes.c_int(K), ctypes.c_int(N))
+    return C
+
+
+# ---------------------------------------------------------------------------------------------
+# whole-layer drivers
+
+
+def prepare_layer(W, Q, r: int, G: int, want_t: bool = False):
+    """Offline part: fold with the *unrounded* Q, quantize, and round Q to bf16 for the online GEMM."""
+    Q = _c(Q, np.float64)
+    out = prepare_weights(fold(Q, np.asarray(W, dtype=np.float64)), r, G, want_t=want_t)
+    out["Qb"] = bf16_round(Q)
+    out["r"], out["G"] = r, G
+    return out
+
+
+def linear_deployed(x_bits, layer, bias=None, want_t: bool = True):
+    """Online part on bf16 inputs.  Returns every intermediate the parity tests look at."""
+    r, G = layer["r"], layer["G"]
+    xt = rotate(x_bits, layer["Qb"])
+    sq = split_quantize(xt, r, G, want_t=want_t)
+    P = int_gemm(sq["codes"], layer["wcodes"], G)
+    y64, yb = combine(P, sq["scales"], layer["wscales"], sq["xh"], layer["Wh"], bias)
+    return {"xt": xt, "xh": sq["xh"], "codes": sq["codes"], "scales": sq["scales"], "t": sq["t"],
+            "P": P, "y64": y64, "y": yb}
+
+
+def linear_ideal(x, Q, W, r: int):
+    """Eq. 4 with nothing quantized and nothing rounded: [xU_h, x~_l] [W~_h; W~_l] in fp64."""
+    x = _c(x, np.float64)
+    Q = _c(Q, np.float64)
+    Wt = fold(Q, np.asarray(W, dtype=np.float64))
+    xt = matmul(x, Q)
+    return matmul(xt[:, :r], Wt[:r]) + matmul(xt[:, r:], Wt[r:])
