@@ -1,0 +1,156 @@
+/*
+ * libdirotq -- rotation-aware W4A4 linear layer (DiRotQ) for NVIDIA B200 (sm_100a).
+ *
+ * The layer computes, for activations X [M,K] and a weight W [K,N] (paper Sec. 4.1: Y = XW),
+ *
+ *     Y ~= [ X U_h , Q4(X U_l R) ] [ U_h^T W ; Q4((U_l R)^T W) ]          (paper Eq. 5)
+ *
+ * where V = [U_h, U_l R] is the calibrated orthogonal rotation (Sec. 4.2; here the argument
+ * `Q`, column j = basis vector j, the first r columns = U_h), Q4 is the symmetric 4-bit
+ * quantizer of Eq. 1 with z = 0, s = max|.|/7, applied per group of `group` consecutive
+ * low-precision coefficients (Sec. 5.1: group size 64, 16-bit scales), per token for the
+ * activations and per output column for the weights.  The first r rotated coefficients and the
+ * first r rows of the folded weight stay bf16.
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless the name says `host`.
+ *     The library allocates no device memory.  `stream` is a cudaStream_t passed as void*.
+ *   - Calls enqueue work on `stream` and return without synchronising, unless stated.
+ *   - Argument errors are reported before anything is launched.  A CUDA launch error is
+ *     returned as DIROTQ_ERR_CUDA.  Device-side waits are bounded; when one expires the kernel
+ *     records a code in the workspace status word (see dirotq_workspace_status) and returns.
+ *   - A workspace must be zero-filled once before its first use: its first word is a sticky
+ *     device status (0 = no wait ever expired).
+ *   - Supported shapes: K % 64 == 0, N % 16 == 0, r in {16, 32, 48, ..., 128} with r < K,
+ *     group in {64, 128} with K % group == 0, M >= 1.  Pointers must be 16-byte aligned.
+ *   - Groups are counted from the first low-precision coefficient; the last one may be ragged.
+ *     Rounding is to nearest, ties to even; scales are bf16 values; a group whose absolute
+ *     maximum is zero has scale 0 and codes 0.
+ */
+#ifndef DIROTQ_H_
+#define DIROTQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DIROTQ_API __attribute__((visibility("default")))
+#else
+#define DIROTQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dirotq_layer dirotq_layer_t; /* opaque host-side handle of a prepared layer */
+typedef void* dirotq_stream_t;              /* a cudaStream_t */
+
+typedef enum {
+    DIROTQ_OK = 0,
+    DIROTQ_ERR_INVALID_ARG = 1,
+    DIROTQ_ERR_UNSUPPORTED_SHAPE = 2,
+    DIROTQ_ERR_BUFFER_TOO_SMALL = 3,
+    DIROTQ_ERR_ARCH = 4,           /* device is not sm_100 */
+    DIROTQ_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed */
+    DIROTQ_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait expired */
+} dirotq_status_t;
+
+enum { DIROTQ_DTYPE_F32 = 0, DIROTQ_DTYPE_BF16 = 1, DIROTQ_DTYPE_F64 = 2 };
+enum { DIROTQ_LAYOUT_KN = 0 /* W[k*N + n] */, DIROTQ_LAYOUT_NK = 1 /* W[n*K + k] */ };
+
+/* Human-readable name of a status code (static string, never NULL). */
+DIROTQ_API const char* dirotq_status_string(dirotq_status_t s);
+
+/* Library version (major*10000 + minor*100 + patch). */
+DIROTQ_API int dirotq_version(void);
+
+/* Last CUDA error text recorded by this thread's most recent failing call ("" if none). */
+DIROTQ_API const char* dirotq_last_error(void);
+
+/* ---- sizes (host only, no CUDA call) ------------------------------------------------------ */
+
+/* Bytes of the device blob that holds a prepared layer: the bf16 rotation (K*K*2), the packed
+ * INT4 weight codes ((K-r rounded up to a group) * N / 2), their scales, the bf16 rank-r slice
+ * and the bias. */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes(int K, int N, int r, int group, size_t* bytes);
+
+/* Bytes of the scratch buffer dirotq_prepare_layer needs (the fp64 folded weight, K*N*8). */
+DIROTQ_API dirotq_status_t dirotq_prepare_scratch_bytes(int K, int N, size_t* bytes);
+
+/* Bytes of the workspace one dirotq_linear call on M tokens needs (activation codes, scales,
+ * the bf16 rank-r coefficients, a status word). */
+DIROTQ_API dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_t* bytes);
+
+/* ---- offline: Eq. 5, right factor -------------------------------------------------------- */
+
+/* Folds W~ = Q^T W in fp64 with the unrounded Q, keeps rows < r as bf16, quantizes rows >= r
+ * to INT4 per (group, output column) with round-to-nearest and packs them, rounds Q to bf16
+ * for the online rotation, converts the bias.
+ *   W      device, [K,N] in `w_layout`, dtype `w_dtype` (F32 or BF16)
+ *   Q      device, [K,K] row-major (Q[k*K + j] = component k of basis vector j), F64 or F32
+ *   bias   device bf16 [N], or NULL
+ *   blob   device, dirotq_layer_bytes() bytes, 1024-byte aligned; must outlive the handle
+ *   scratch device, dirotq_prepare_scratch_bytes() bytes; free to reuse once `stream` has
+ *          passed this call
+ * On success *layer_out receives a host handle (free it with dirotq_layer_destroy). */
+DIROTQ_API dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                     const void* bias, int K, int N, int r, int group, void* blob,
+                                     size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                     dirotq_stream_t stream, dirotq_layer_t** layer_out);
+
+/* Frees the host handle (not the blob). */
+DIROTQ_API dirotq_status_t dirotq_layer_destroy(dirotq_layer_t* layer);
+
+/* Shape of a prepared layer.  Any output pointer may be NULL.  K_lp = n_g*group is the padded
+ * width of the activation-code rows in the workspace. */
+DIROTQ_API dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K, int* N, int* r, int* group, int* n_g,
+                                  int* K_lp);
+
+/* ---- online: Eq. 5, the whole right-hand side --------------------------------------------- */
+
+/* y[M,N] (bf16, row-major) = DiRotQ-linear(x[M,K] bf16 row-major).  Two kernels are enqueued:
+ * rotate+split+quantize (x Q_b on the bf16 tensor cores, Eq. 1 in the epilogue), then the
+ * INT4 x INT4 group GEMM on the int8 tensor cores with the per-group rescale, the bf16 rank-r
+ * branch and the bias.  Concurrent calls on one layer need distinct workspaces. */
+DIROTQ_API dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer, void* y, void* workspace,
+                              size_t workspace_bytes, dirotq_stream_t stream);
+
+/* Same computation with HOST input and output (pinned memory recommended): copies x into
+ * x_dev, runs dirotq_linear, copies y_dev into y_host, all on `stream`; x_dev [M,K] and
+ * y_dev [M,N] are device staging buffers of the caller. */
+DIROTQ_API dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer_t* layer, void* y_host,
+                                   void* x_dev, void* y_dev, void* workspace, size_t workspace_bytes,
+                                   dirotq_stream_t stream);
+
+/* Reads the workspace status word.  SYNCHRONISES `stream`.  *device_code is 0 when every wait
+ * completed; otherwise the role that gave up.  Returns DIROTQ_ERR_DEVICE_TIMEOUT in that case. */
+DIROTQ_API dirotq_status_t dirotq_workspace_status(const void* workspace, dirotq_stream_t stream, int* device_code);
+
+/* ---- exports for parity checks ------------------------------------------------------------- */
+
+/* Runs only the first kernel (rotation, split, Eq. 1) and leaves its results in `workspace`.
+ * xrot_f32, if not NULL, receives the fp32 rotated activations [M,K] in the column order of Q. */
+DIROTQ_API dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
+                                       size_t workspace_bytes, float* xrot_f32, dirotq_stream_t stream);
+
+/* Copies the first kernel's results out of the workspace into plain layouts:
+ * xh bf16 [M,r]; codes int8 [M,K-r], one code per byte; scales bf16 [M,n_g]. */
+DIROTQ_API dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
+                                        int8_t* codes, void* scales_bf16, dirotq_stream_t stream);
+
+/* Integer GEMM alone on caller-supplied activation codes (int8, one per byte, [M,K_lp] with
+ * zero codes in columns >= K-r): partials[g][m][n] = sum over group g of q_x q_w, int32. */
+DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const dirotq_layer_t* layer,
+                                      int32_t* partials, void* workspace, size_t workspace_bytes,
+                                      dirotq_stream_t stream);
+
+/* Unpacks a prepared layer: wcodes int8 [K-r,N]; wscales bf16 [n_g,N]; wh bf16 [r,N];
+ * q_bf16 [K,K] in the layout of the Q argument.  Any pointer may be NULL. */
+DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,
+                                    void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIROTQ_H_ */

@@ -1,0 +1,216 @@
+"""ctypes binding of libdirotq: argument marshalling only.
+
+Function names mirror the C ABI in ``include/dirotq.h``.  Tensors are torch tensors used as
+device memory; every step of the layer runs inside the CUDA library.  If the library is not
+built, importing the entry points raises: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdirotq.so")
+
+DIROTQ_OK = 0
+STATUS_NAMES = {0: "ok", 1: "invalid argument", 2: "unsupported shape", 3: "buffer too small",
+                4: "device is not sm_100", 5: "CUDA error", 6: "device-side wait timed out"}
+DTYPE_F32, DTYPE_BF16, DTYPE_F64 = 0, 1, 2
+LAYOUT_KN, LAYOUT_NK = 0, 1
+
+EXPORTED = [
+    "dirotq_status_string", "dirotq_version", "dirotq_last_error", "dirotq_layer_bytes",
+    "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
+    "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
+    "dirotq_rotate_quantize", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
+]
+
+
+class DirotqError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}" + (f" ({detail})" if detail else ""))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdirotq.so (must have been built: ``python -m paper_2605_16732_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: build it with paper_2605_16732_b200.build.build()")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        pi, psz = ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_size_t)
+        L.dirotq_status_string.restype = ctypes.c_char_p
+        L.dirotq_status_string.argtypes = [i]
+        L.dirotq_version.restype = i
+        L.dirotq_last_error.restype = ctypes.c_char_p
+        L.dirotq_layer_bytes.argtypes = [i, i, i, i, psz]
+        L.dirotq_prepare_scratch_bytes.argtypes = [i, i, psz]
+        L.dirotq_workspace_bytes.argtypes = [vp, i, psz]
+        L.dirotq_prepare_layer.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
+        L.dirotq_layer_destroy.argtypes = [vp]
+        L.dirotq_layer_info.argtypes = [vp, pi, pi, pi, pi, pi, pi]
+        L.dirotq_linear.argtypes = [vp, i, vp, vp, vp, sz, vp]
+        L.dirotq_linear_host.argtypes = [vp, i, vp, vp, vp, vp, vp, sz, vp]
+        L.dirotq_workspace_status.argtypes = [vp, vp, pi]
+        L.dirotq_rotate_quantize.argtypes = [vp, i, vp, vp, sz, vp, vp]
+        L.dirotq_workspace_export.argtypes = [vp, i, vp, vp, vp, vp, vp]
+        L.dirotq_int_gemm_debug.argtypes = [vp, i, vp, vp, vp, sz, vp]
+        L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
+        for name in EXPORTED:
+            if name not in ("dirotq_status_string", "dirotq_version", "dirotq_last_error"):
+                getattr(L, name).restype = i
+        _lib = L
+    return _lib
+
+
+def _check(st: int, where: str):
+    if st != DIROTQ_OK:
+        raise DirotqError(st, where, lib().dirotq_last_error().decode())
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def dirotq_layer_bytes(K: int, N: int, r: int, group: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_layer_bytes(K, N, r, group, ctypes.byref(out)), "dirotq_layer_bytes")
+    return out.value
+
+
+def dirotq_prepare_scratch_bytes(K: int, N: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_prepare_scratch_bytes(K, N, ctypes.byref(out)), "dirotq_prepare_scratch_bytes")
+    return out.value
+
+
+class Layer:
+    """Owner of one prepared layer: the device blob (a torch uint8 tensor) and the host handle."""
+
+    def __init__(self, handle: int, blob: torch.Tensor, K: int, N: int, r: int, group: int):
+        self.handle, self.blob = handle, blob
+        self.K, self.N, self.r, self.group = K, N, r, group
+        self.K_l = K - r
+        self.n_g = -(-self.K_l // group)
+        self.K_lp = self.n_g * group
+
+    def close(self):
+        if self.handle:
+            lib().dirotq_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _alloc_bytes(nbytes: int, device, zero: bool = False) -> torch.Tensor:
+    # torch's caching allocator returns 512-byte aligned blocks; over-allocate to align to 1024
+    f = torch.zeros if zero else torch.empty
+    raw = f(nbytes + 1024, dtype=torch.uint8, device=device)
+    off = (-raw.data_ptr()) % 1024
+    return raw[off:off + nbytes]
+
+
+def dirotq_prepare_layer(W: torch.Tensor, Q: torch.Tensor, r: int, group: int, bias: torch.Tensor | None = None,
+                         w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """W: cuda float32/bfloat16 [K,N] (or [N,K] with LAYOUT_NK); Q: cuda float64/float32 [K,K]; bias: cuda bf16 [N]."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    blob = _alloc_bytes(dirotq_layer_bytes(K, N, r, group), W.device)
+    scratch_bytes = dirotq_prepare_scratch_bytes(K, N)
+    scratch = _alloc_bytes(scratch_bytes, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), K, N, r, group,
+                                    blob.data_ptr(), blob.numel(), scratch.data_ptr(), scratch_bytes, _stream(stream),
+                                    ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer")
+    torch.cuda.current_stream().synchronize()  # scratch is released when this function returns
+    return Layer(handle.value, blob, K, N, r, group)
+
+
+def dirotq_workspace_bytes(layer: Layer, M: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_workspace_bytes(layer.handle, M, ctypes.byref(out)), "dirotq_workspace_bytes")
+    return out.value
+
+
+def alloc_workspace(layer: Layer, M: int) -> torch.Tensor:
+    return _alloc_bytes(dirotq_workspace_bytes(layer, M), layer.blob.device, zero=True)
+
+
+def dirotq_linear(x: torch.Tensor, layer: Layer, y: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    M = x.shape[0]
+    _check(lib().dirotq_linear(x.data_ptr(), M, layer.handle, y.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                               _stream(stream)), "dirotq_linear")
+
+
+def dirotq_linear_host(x_host: torch.Tensor, layer: Layer, y_host: torch.Tensor, x_dev: torch.Tensor,
+                       y_dev: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    M = x_host.shape[0]
+    _check(lib().dirotq_linear_host(x_host.data_ptr(), M, layer.handle, y_host.data_ptr(), x_dev.data_ptr(),
+                                    y_dev.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream)),
+           "dirotq_linear_host")
+
+
+def dirotq_workspace_status(workspace: torch.Tensor, stream=None) -> int:
+    code = ctypes.c_int(0)
+    st = lib().dirotq_workspace_status(workspace.data_ptr(), _stream(stream), ctypes.byref(code))
+    if st not in (0, 6):
+        _check(st, "dirotq_workspace_status")
+    return code.value
+
+
+def dirotq_rotate_quantize(x: torch.Tensor, layer: Layer, workspace: torch.Tensor, xrot: torch.Tensor | None = None,
+                           stream=None) -> None:
+    _check(lib().dirotq_rotate_quantize(x.data_ptr(), x.shape[0], layer.handle, workspace.data_ptr(),
+                                        workspace.numel(), _ptr(xrot), _stream(stream)), "dirotq_rotate_quantize")
+
+
+def dirotq_workspace_export(layer: Layer, M: int, workspace: torch.Tensor, stream=None):
+    dev = workspace.device
+    xh = torch.empty((M, layer.r), dtype=torch.bfloat16, device=dev)
+    codes = torch.empty((M, layer.K_l), dtype=torch.int8, device=dev)
+    scales = torch.empty((M, layer.n_g), dtype=torch.bfloat16, device=dev)
+    _check(lib().dirotq_workspace_export(layer.handle, M, workspace.data_ptr(), xh.data_ptr(), codes.data_ptr(),
+                                         scales.data_ptr(), _stream(stream)), "dirotq_workspace_export")
+    return xh, codes, scales
+
+
+def dirotq_int_gemm_debug(act_codes: torch.Tensor, layer: Layer, workspace: torch.Tensor, stream=None) -> torch.Tensor:
+    """act_codes: cuda int8 [M, K_lp] (zero in columns >= K - r).  Returns int32 [n_g, M, N]."""
+    M = act_codes.shape[0]
+    assert act_codes.shape[1] == layer.K_lp and act_codes.is_contiguous()
+    P = torch.empty((layer.n_g, M, layer.N), dtype=torch.int32, device=act_codes.device)
+    _check(lib().dirotq_int_gemm_debug(act_codes.data_ptr(), M, layer.handle, P.data_ptr(), workspace.data_ptr(),
+                                       workspace.numel(), _stream(stream)), "dirotq_int_gemm_debug")
+    return P
+
+
+def dirotq_layer_export(layer: Layer, stream=None):
+    dev = layer.blob.device
+    wcodes = torch.empty((layer.K_l, layer.N), dtype=torch.int8, device=dev)
+    wscales = torch.empty((layer.n_g, layer.N), dtype=torch.bfloat16, device=dev)
+    wh = torch.empty((layer.r, layer.N), dtype=torch.bfloat16, device=dev)
+    qb = torch.empty((layer.K, layer.K), dtype=torch.bfloat16, device=dev)
+    _check(lib().dirotq_layer_export(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(), qb.data_ptr(),
+                                     _stream(stream)), "dirotq_layer_export")
+    return wcodes, wscales, wh, qb

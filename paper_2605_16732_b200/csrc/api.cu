@@ -1,0 +1,310 @@
+// C ABI of libdirotq: argument validation, tensor-map construction, launch sequencing.
+#include "common.h"
+
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+namespace dirotq {
+namespace {
+
+thread_local char g_last_error[256] = "";
+
+void set_error(const char* what, cudaError_t e) {
+    snprintf(g_last_error, sizeof g_last_error, "%s: %s", what, cudaGetErrorString(e));
+}
+void set_error_text(const char* what) { snprintf(g_last_error, sizeof g_last_error, "%s", what); }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is looked up at run time so that the library loads on machines
+// without a driver (build hosts); any call that needs it fails with DIROTQ_ERR_CUDA there.
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres);
+        if (e == cudaSuccess && qres == cudaDriverEntryPointSuccess) fn = reinterpret_cast<EncodeTiledFn>(p);
+        else set_error("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", e);
+    }
+    return fn;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+dirotq_status_t check_shape(int K, int N, int r, int G) {
+    if (K <= 0 || N <= 0 || r <= 0) return DIROTQ_ERR_INVALID_ARG;
+    if (G != 64 && G != 128) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
+    if (K % 64 != 0 || K % G != 0 || N % 16 != 0) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
+    if (r % 16 != 0 || r > 128 || r >= K) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
+    return DIROTQ_OK;
+}
+
+bool valid_layer(const dirotq_layer* L) { return L != nullptr && L->magic == kLayerMagic; }
+
+dirotq_status_t check_device(int* device_out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_error("cudaGetDevice", e); return DIROTQ_ERR_CUDA; }
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { set_error("cudaDeviceGetAttribute", e); return DIROTQ_ERR_CUDA; }
+    if (major != 10) return DIROTQ_ERR_ARCH;
+    *device_out = dev;
+    return DIROTQ_OK;
+}
+
+}  // namespace
+
+int sm_count(int device) {
+    static int cached[64] = {0};
+    if (device < 0 || device >= 64) return 148;
+    if (cached[device] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 148;
+        cached[device] = n;
+    }
+    return cached[device];
+}
+
+dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t elem_bytes, const void* base,
+                               uint64_t dim0, uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1,
+                               CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return DIROTQ_ERR_CUDA;
+    if (!aligned16(base) || stride1_bytes % 16 != 0 || (box0 * elem_bytes) % 16 != 0) return DIROTQ_ERR_INVALID_ARG;
+    cuuint64_t dims[2] = {dim0, dim1};
+    cuuint64_t strides[1] = {stride1_bytes};
+    cuuint32_t box[2] = {box0, box1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_last_error, sizeof g_last_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return DIROTQ_ERR_CUDA;
+    }
+    return DIROTQ_OK;
+}
+
+}  // namespace dirotq
+
+using namespace dirotq;
+
+extern "C" {
+
+const char* dirotq_status_string(dirotq_status_t s) {
+    switch (s) {
+        case DIROTQ_OK: return "ok";
+        case DIROTQ_ERR_INVALID_ARG: return "invalid argument";
+        case DIROTQ_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case DIROTQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case DIROTQ_ERR_ARCH: return "device is not sm_100";
+        case DIROTQ_ERR_CUDA: return "CUDA error";
+        case DIROTQ_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int dirotq_version(void) { return 100; }
+
+const char* dirotq_last_error(void) { return g_last_error; }
+
+dirotq_status_t dirotq_layer_bytes(int K, int N, int r, int group, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, group);
+    if (st != DIROTQ_OK) return st;
+    *bytes = make_blob_layout(make_geometry(K, N, r, group)).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_scratch_bytes(int K, int N, size_t* bytes) {
+    if (!bytes || K <= 0 || N <= 0) return DIROTQ_ERR_INVALID_ARG;
+    *bytes = static_cast<size_t>(K) * N * sizeof(double);
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_t* bytes) {
+    if (!valid_layer(layer) || !bytes || M < 1) return DIROTQ_ERR_INVALID_ARG;
+    *bytes = make_workspace_layout(layer->geo, M).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                     const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                     dirotq_layer_t** layer_out) {
+    if (!W || !Q || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
+    if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
+    if (q_dtype != DIROTQ_DTYPE_F64 && q_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
+    if (w_layout != DIROTQ_LAYOUT_KN && w_layout != DIROTQ_LAYOUT_NK) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, group);
+    if (st != DIROTQ_OK) return st;
+    if (!aligned16(W) || !aligned16(Q) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
+    const Geometry g = make_geometry(K, N, r, group);
+    const BlobLayout lay = make_blob_layout(g);
+    if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (scratch_bytes < static_cast<size_t>(K) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    int dev = 0;
+    st = check_device(&dev);
+    if (st != DIROTQ_OK) return st;
+
+    dirotq_layer* L = new (std::nothrow) dirotq_layer;
+    if (!L) return DIROTQ_ERR_INVALID_ARG;
+    memset(L, 0, sizeof *L);
+    L->magic = kLayerMagic;
+    L->device = dev;
+    L->geo = g;
+    L->lay = lay;
+    L->blob = static_cast<char*>(blob);
+
+    st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                        (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
+                            (uint64_t)g.n_g, (uint64_t)N * 4, 256, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, static_cast<double*>(scratch),
+                            static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) {
+        delete L;
+        return st;
+    }
+    *layer_out = L;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_layer_destroy(dirotq_layer_t* layer) {
+    if (!valid_layer(layer)) return DIROTQ_ERR_INVALID_ARG;
+    layer->magic = 0;
+    delete layer;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K, int* N, int* r, int* group, int* n_g, int* K_lp) {
+    if (!valid_layer(layer)) return DIROTQ_ERR_INVALID_ARG;
+    if (K) *K = layer->geo.K;
+    if (N) *N = layer->geo.N;
+    if (r) *r = layer->geo.r;
+    if (group) *group = layer->geo.G;
+    if (n_g) *n_g = layer->geo.n_g;
+    if (K_lp) *K_lp = layer->geo.K_lp;
+    return DIROTQ_OK;
+}
+
+static dirotq_status_t check_call(const dirotq_layer_t* layer, int M, const void* workspace, size_t workspace_bytes) {
+    if (!valid_layer(layer) || !workspace || M < 1) return DIROTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
+    if (workspace_bytes < make_workspace_layout(layer->geo, M).total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    return DIROTQ_OK;
+}
+
+static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M, char* ws, float* xrot) {
+    const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
+    RotateArgs a;
+    a.x = x; a.M = M;
+    a.codes = reinterpret_cast<int8_t*>(ws + w.off_codes);
+    a.xscale = reinterpret_cast<float*>(ws + w.off_xscale);
+    a.ldm = w.ldm;
+    a.xh = reinterpret_cast<uint16_t*>(ws + w.off_xh);
+    a.xrot = xrot;
+    a.status = reinterpret_cast<int*>(ws + w.off_status);
+    return a;
+}
+
+dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
+                                       size_t workspace_bytes, float* xrot_f32, dirotq_stream_t stream) {
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    if (st != DIROTQ_OK) return st;
+    if (!x || !aligned16(x) || (xrot_f32 && !aligned16(xrot_f32))) return DIROTQ_ERR_INVALID_ARG;
+    return launch_rotate_quantize(layer, rotate_args(layer, x, M, static_cast<char*>(workspace), xrot_f32),
+                                  static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer, void* y, void* workspace,
+                              size_t workspace_bytes, dirotq_stream_t stream) {
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    if (st != DIROTQ_OK) return st;
+    if (!x || !y || !aligned16(x) || !aligned16(y)) return DIROTQ_ERR_INVALID_ARG;
+    char* ws = static_cast<char*>(workspace);
+    const RotateArgs ra = rotate_args(layer, x, M, ws, nullptr);
+    st = launch_rotate_quantize(layer, ra, static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) return st;
+    GemmArgs ga;
+    ga.M = M; ga.codes = ra.codes; ga.xscale = ra.xscale; ga.ldm = ra.ldm; ga.xh = ra.xh;
+    ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr; ga.status = ra.status;
+    return launch_w4a4_gemm(layer, ga, static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer_t* layer, void* y_host, void* x_dev,
+                                   void* y_dev, void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    if (st != DIROTQ_OK) return st;
+    if (!x_host || !y_host || !x_dev || !y_dev) return DIROTQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t xb = static_cast<size_t>(M) * layer->geo.K * 2, yb = static_cast<size_t>(M) * layer->geo.N * 2;
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xb, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) { set_error("cudaMemcpyAsync(H2D)", e); return DIROTQ_ERR_CUDA; }
+    st = dirotq_linear(x_dev, M, layer, y_dev, workspace, workspace_bytes, stream);
+    if (st != DIROTQ_OK) return st;
+    e = cudaMemcpyAsync(y_host, y_dev, yb, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) { set_error("cudaMemcpyAsync(D2H)", e); return DIROTQ_ERR_CUDA; }
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_workspace_status(const void* workspace, dirotq_stream_t stream, int* device_code) {
+    if (!workspace) return DIROTQ_ERR_INVALID_ARG;
+    int code = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&code, workspace, sizeof code, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { set_error("status read", e); return DIROTQ_ERR_CUDA; }
+    if (device_code) *device_code = code;
+    return code == 0 ? DIROTQ_OK : DIROTQ_ERR_DEVICE_TIMEOUT;
+}
+
+dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
+                                        int8_t* codes, void* scales_bf16, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
+    return launch_workspace_export(layer, M, static_cast<const char*>(workspace), static_cast<uint16_t*>(xh_bf16), codes,
+                                   static_cast<uint16_t*>(scales_bf16), static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const dirotq_layer_t* layer, int32_t* partials,
+                                      void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    if (st != DIROTQ_OK) return st;
+    if (!act_codes || !partials || !aligned16(act_codes) || !aligned16(partials)) return DIROTQ_ERR_INVALID_ARG;
+    char* ws = static_cast<char*>(workspace);
+    const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
+    GemmArgs ga;
+    ga.M = M; ga.codes = act_codes;
+    ga.xscale = reinterpret_cast<const float*>(ws + w.off_xscale);
+    ga.ldm = w.ldm;
+    ga.xh = reinterpret_cast<const uint16_t*>(ws + w.off_xh);
+    ga.y = nullptr; ga.partials = partials;
+    ga.status = reinterpret_cast<int*>(ws + w.off_status);
+    return launch_w4a4_gemm(layer, ga, static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16, void* wh_bf16,
+                                    void* q_bf16, dirotq_stream_t stream) {
+    if (!valid_layer(layer)) return DIROTQ_ERR_INVALID_ARG;
+    return launch_layer_export(layer, wcodes, static_cast<uint16_t*>(wscales_bf16), static_cast<uint16_t*>(wh_bf16),
+                               static_cast<uint16_t*>(q_bf16), static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

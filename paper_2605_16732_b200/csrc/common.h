@@ -1,0 +1,142 @@
+// Internal definitions shared by the translation units of libdirotq (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/dirotq.h"
+
+namespace dirotq {
+
+// ------------------------------------------------------------------ geometry of one layer
+//
+// Column order after the online rotation ("permuted" order): the K_l = K - r low-precision
+// coefficients come first, the r high-precision ones last.  Group g of the low block is the
+// permuted columns [g*G, (g+1)*G); when K_l is not a multiple of G the last group is ragged and
+// the slots up to K_lp = n_g*G (which are high columns in this order) carry zero codes.
+struct Geometry {
+    int K, N, r, G;
+    int K_l;    // K - r
+    int n_g;    // ceil(K_l / G)
+    int K_lp;   // n_g * G  (<= K)
+    int r_pad;  // r rounded up to a multiple of 64 (bf16 low-rank operand width)
+};
+
+inline Geometry make_geometry(int K, int N, int r, int G) {
+    Geometry g;
+    g.K = K; g.N = N; g.r = r; g.G = G;
+    g.K_l = K - r;
+    g.n_g = (g.K_l + G - 1) / G;
+    g.K_lp = g.n_g * G;
+    g.r_pad = (r + 63) / 64 * 64;
+    return g;
+}
+
+constexpr size_t kAlign = 1024;
+inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+
+// Sections of the device blob that holds a prepared layer.
+struct BlobLayout {
+    size_t off_qt;       // bf16 [K][K]: row c' = permuted output column, K-major over the input channel
+    size_t off_wpacked;  // u8   [N][K_lp/2]: two INT4 codes per byte, K-major, see prepare.cu for the nibble order
+    size_t off_wscale;   // f32  [n_g][N]: bf16-valued group scales of the weight codes
+    size_t off_wh;       // bf16 [N][r_pad]: high-precision rows of the folded weight, K-major, zero padded
+    size_t off_bias;     // f32  [N]
+    size_t total;
+};
+
+inline BlobLayout make_blob_layout(const Geometry& g) {
+    BlobLayout b;
+    size_t o = 0;
+    b.off_qt = o;      o = align_up(o + (size_t)g.K * g.K * 2);
+    b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K_lp / 2));
+    b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * g.N * 4);
+    b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
+    b.off_bias = o;    o = align_up(o + (size_t)g.N * 4);
+    b.total = o;
+    return b;
+}
+
+// Workspace of one dirotq_linear call (device memory owned by the caller).
+struct WorkspaceLayout {
+    int ldm;            // leading dimension (tokens) of the transposed activation-scale array
+    size_t off_status;  // int32[64]: word 0 = device status
+    size_t off_codes;   // i8  [M][K_lp]: activation codes, one per byte
+    size_t off_xscale;  // f32 [n_g][ldm]: bf16-valued activation scales, group-major
+    size_t off_xh;      // bf16 [M][r_pad]
+    size_t total;
+};
+
+inline WorkspaceLayout make_workspace_layout(const Geometry& g, int M) {
+    WorkspaceLayout w;
+    w.ldm = (M + 63) / 64 * 64;
+    size_t o = 0;
+    w.off_status = o;  o = align_up(o + 256);
+    w.off_codes = o;   o = align_up(o + (size_t)M * g.K_lp);
+    w.off_xscale = o;  o = align_up(o + (size_t)g.n_g * w.ldm * 4);
+    w.off_xh = o;      o = align_up(o + (size_t)M * g.r_pad * 2);
+    w.total = o;
+    return w;
+}
+
+}  // namespace dirotq
+
+// The opaque handle of the C ABI: host-side description of a prepared layer.
+struct dirotq_layer {
+    uint32_t magic;
+    int device;
+    dirotq::Geometry geo;
+    dirotq::BlobLayout lay;
+    char* blob;  // device
+    CUtensorMap tmap_qt;       // bf16 [K][K], box 64 x 256, 128B swizzle
+    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2], box 64 x 256, no swizzle
+    CUtensorMap tmap_wscale;   // f32 [n_g][N], box 256 x (128/G)
+    CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x 256, 128B swizzle
+};
+
+namespace dirotq {
+
+constexpr uint32_t kLayerMagic = 0x44695251u;  // "DiRQ"
+
+// ------------------------------------------------------------------ kernel launch interfaces
+
+struct RotateArgs {
+    const void* x;  // bf16 [M][K]
+    int M;
+    int8_t* codes;
+    float* xscale;
+    int ldm;
+    uint16_t* xh;
+    float* xrot;  // optional fp32 [M][K], columns in the caller's (unpermuted) order
+    int* status;
+};
+
+struct GemmArgs {
+    int M;
+    const int8_t* codes;
+    const float* xscale;
+    int ldm;
+    const uint16_t* xh;
+    uint16_t* y;        // bf16 [M][N]
+    int32_t* partials;  // debug: int32 [n_g][M][N]; when set, y is not written
+    int* status;
+};
+
+// tensor-map factory (api.cu)
+dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t elem_bytes, const void* base,
+                               uint64_t dim0, uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1,
+                               CUtensorMapSwizzle swz);
+
+// launchers (each returns after enqueueing on `stream`)
+dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
+dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream);
+dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
+                               int q_dtype, const void* bias, double* scratch, cudaStream_t stream);
+dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint16_t* wscales, uint16_t* wh,
+                                    uint16_t* qb, cudaStream_t stream);
+dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
+                                        int8_t* codes, uint16_t* scales, cudaStream_t stream);
+int sm_count(int device);
+
+}  // namespace dirotq

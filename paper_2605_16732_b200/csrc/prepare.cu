@@ -1,0 +1,266 @@
+// Offline part (paper Eq. 5, right factor): fold the rotation into the weight, split at row r,
+// quantize the low rows to INT4 per (group, output column) with round-to-nearest, pack, and lay
+// everything out the way the two online kernels read it.  Plain CUDA cores, fp64: this runs once
+// per layer and is not on the timed path.
+//
+// Packed weight-code layout, row n of u8 [N][K_lp/2] (K-major): codes are taken 32 at a time
+// (16 bytes); inside such a piece, byte 4*j + b (j, b in 0..3) holds code 8*j + b in its low
+// nibble and code 8*j + 4 + b in its high nibble (two's complement nibbles).  With this order the
+// online unpack of a 32-bit word is two logic ops per four codes:
+//   (w << 4) & 0xF0F0F0F0  ->  codes 8j..8j+3 as bytes 16*q,      w & 0xF0F0F0F0  ->  codes 8j+4..8j+7.
+#include "common.h"
+
+#include <cuda_bf16.h>
+
+namespace dirotq {
+namespace {
+
+// fp64 -> bf16, nearest, ties to even, with a single rounding: round to odd into fp32 first.
+__device__ __forceinline__ uint16_t f64_to_bf16(double v) {
+    float f = __double2float_rz(v);
+    uint32_t u = __float_as_uint(f);
+    if (static_cast<double>(f) != v && (u & 0x7F800000u) != 0x7F800000u) u |= 1u;  // sticky bit
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0;                             // NaN
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return static_cast<uint16_t>(u >> 16);
+}
+
+__device__ __forceinline__ double bf16_to_f64(uint16_t h) {
+    return static_cast<double>(__uint_as_float(static_cast<uint32_t>(h) << 16));
+}
+
+__device__ __forceinline__ double load_q(const void* Q, int q_dtype, int K, int k, int j) {
+    const size_t i = static_cast<size_t>(k) * K + j;
+    return q_dtype == DIROTQ_DTYPE_F64 ? static_cast<const double*>(Q)[i]
+                                       : static_cast<double>(static_cast<const float*>(Q)[i]);
+}
+
+__device__ __forceinline__ double load_w(const void* W, int w_dtype, int w_layout, int K, int N, int k, int n) {
+    const size_t i = w_layout == DIROTQ_LAYOUT_KN ? static_cast<size_t>(k) * N + n : static_cast<size_t>(n) * K + k;
+    return w_dtype == DIROTQ_DTYPE_F32 ? static_cast<double>(static_cast<const float*>(W)[i])
+                                       : bf16_to_f64(static_cast<const uint16_t*>(W)[i]);
+}
+
+// Wt[i][n] = sum_k Q[k][i] * W[k][n]     (64 x 64 output tile, 4 x 4 per thread, fp64)
+__global__ void __launch_bounds__(256) fold_kernel(const void* Q, int q_dtype, const void* W, int w_dtype, int w_layout,
+                                                   double* Wt, int K, int N) {
+    __shared__ double sq[16][64 + 1];
+    __shared__ double sw[16][64 + 1];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int i0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    double acc[4][4] = {};
+    for (int k0 = 0; k0 < K; k0 += 16) {
+        for (int e = threadIdx.x; e < 16 * 64; e += 256) {
+            const int kk = e >> 6, c = e & 63;
+            sq[kk][c] = (i0 + c < K) ? load_q(Q, q_dtype, K, k0 + kk, i0 + c) : 0.0;
+            sw[kk][c] = (n0 + c < N) ? load_w(W, w_dtype, w_layout, K, N, k0 + kk, n0 + c) : 0.0;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            double a[4], b[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { a[u] = sq[kk][ty * 4 + u]; b[u] = sw[kk][tx * 4 + u]; }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) acc[u][v] = fma(a[u], b[v], acc[u][v]);
+        }
+        __syncthreads();
+    }
+    for (int u = 0; u < 4; ++u)
+        for (int v = 0; v < 4; ++v) {
+            const int i = i0 + ty * 4 + u, n = n0 + tx * 4 + v;
+            if (i < K && n < N) Wt[static_cast<size_t>(i) * N + n] = acc[u][v];
+        }
+}
+
+__host__ __device__ __forceinline__ int packed_byte_index(int k) {  // byte of code k inside its row
+    const int w = k & 31;
+    return (k >> 5) * 16 + (w >> 3) * 4 + (w & 3);
+}
+__host__ __device__ __forceinline__ int packed_is_high(int k) { return (k >> 2) & 1; }
+
+// One thread per (group, output column): Eq. 1 with z = 0, s = bf16(max|w|/7), ties to even.
+__global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, float* wscale, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int grp = blockIdx.y;
+    if (n >= g.N) return;
+    const int j0 = grp * g.G;
+    const int len = min(g.G, g.K_l - j0);
+    const double* col = Wt + static_cast<size_t>(g.r + j0) * g.N + n;
+    double a = 0.0;
+    for (int j = 0; j < len; ++j) a = fmax(a, fabs(col[static_cast<size_t>(j) * g.N]));
+    const uint16_t sb = (a == 0.0) ? 0 : f64_to_bf16(a / 7.0);
+    const double s = bf16_to_f64(sb);
+    wscale[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(s);
+    uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
+    for (int jb = 0; jb < g.G; jb += 8) {
+        // codes j0+jb .. j0+jb+7 share four bytes
+        uint32_t word = 0;
+        for (int t = 0; t < 8; ++t) {
+            const int j = jb + t;
+            int q = 0;
+            if (j < len && s != 0.0) {
+                double qq = rint(col[static_cast<size_t>(j) * g.N] / s);
+                qq = fmin(7.0, fmax(-7.0, qq));
+                q = static_cast<int>(qq);
+            }
+            const uint32_t nib = static_cast<uint32_t>(q) & 0xFu;
+            word |= nib << (8 * (t & 3) + 4 * (t >> 2));
+        }
+        *reinterpret_cast<uint32_t*>(row + packed_byte_index(j0 + jb)) = word;
+    }
+}
+
+// wh[n][i] = bf16(Wt[i][n]) for i < r, zero up to r_pad.
+__global__ void high_rows_kernel(const double* Wt, uint16_t* wh, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= g.N) return;
+    for (int i = 0; i < g.r_pad; ++i)
+        wh[static_cast<size_t>(n) * g.r_pad + i] = i < g.r ? f64_to_bf16(Wt[static_cast<size_t>(i) * g.N + n]) : 0;
+}
+
+// qt[c'][k] = bf16(Q[k][col(c')]) with the low-precision columns first (tiled transpose).
+__global__ void rotation_kernel(const void* Q, int q_dtype, uint16_t* qt, Geometry g) {
+    __shared__ uint16_t tile[32][33];
+    const int k0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    for (int dy = threadIdx.y; dy < 32; dy += blockDim.y) {
+        const int k = k0 + dy, cp = c0 + threadIdx.x;  // read Q[k][col(cp)], coalesced along cp
+        if (k < g.K && cp < g.K) {
+            const int col = cp < g.K_l ? cp + g.r : cp - g.K_l;
+            tile[dy][threadIdx.x] = f64_to_bf16(load_q(Q, q_dtype, g.K, k, col));
+        }
+    }
+    __syncthreads();
+    for (int dy = threadIdx.y; dy < 32; dy += blockDim.y) {
+        const int cp = c0 + dy, k = k0 + threadIdx.x;
+        if (cp < g.K && k < g.K) qt[static_cast<size_t>(cp) * g.K + k] = tile[threadIdx.x][dy];
+    }
+}
+
+__global__ void bias_kernel(const uint16_t* bias, float* out, int N) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n < N) out[n] = bias ? __uint_as_float(static_cast<uint32_t>(bias[n]) << 16) : 0.f;
+}
+
+// ---------------------------------------------------------------- exports (parity checks)
+
+__global__ void export_wcodes_kernel(const uint8_t* wpacked, int8_t* wcodes, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int j = blockIdx.y;
+    if (n >= g.N || j >= g.K_l) return;
+    const uint8_t byte = wpacked[static_cast<size_t>(n) * (g.K_lp / 2) + packed_byte_index(j)];
+    const int nib = packed_is_high(j) ? (byte >> 4) : (byte & 0xF);
+    wcodes[static_cast<size_t>(j) * g.N + n] = static_cast<int8_t>((nib ^ 8) - 8);  // sign-extend 4 bits
+}
+
+__global__ void export_wscales_kernel(const float* wscale, uint16_t* out, size_t count) {
+    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < count) out[i] = static_cast<uint16_t>(__float_as_uint(wscale[i]) >> 16);  // values are bf16-exact
+}
+
+__global__ void export_wh_kernel(const uint16_t* wh, uint16_t* out, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = blockIdx.y;
+    if (n < g.N && i < g.r) out[static_cast<size_t>(i) * g.N + n] = wh[static_cast<size_t>(n) * g.r_pad + i];
+}
+
+__global__ void export_q_kernel(const uint16_t* qt, uint16_t* out, Geometry g) {
+    __shared__ uint16_t tile[32][33];
+    const int k0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    for (int dy = threadIdx.y; dy < 32; dy += blockDim.y) {
+        const int cp = c0 + dy, k = k0 + threadIdx.x;
+        if (cp < g.K && k < g.K) tile[dy][threadIdx.x] = qt[static_cast<size_t>(cp) * g.K + k];
+    }
+    __syncthreads();
+    for (int dy = threadIdx.y; dy < 32; dy += blockDim.y) {
+        const int k = k0 + dy, cp = c0 + threadIdx.x;
+        if (k < g.K && cp < g.K) {
+            const int col = cp < g.K_l ? cp + g.r : cp - g.K_l;
+            out[static_cast<size_t>(k) * g.K + col] = tile[threadIdx.x][dy];
+        }
+    }
+}
+
+__global__ void export_workspace_kernel(const int8_t* codes, const float* xscale, const uint16_t* xh_pad, int M, int ldm,
+                                        Geometry g, uint16_t* xh, int8_t* codes_out, uint16_t* scales) {
+    const int m = blockIdx.y;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < g.K_l; c += gridDim.x * blockDim.x)
+        if (codes_out) codes_out[static_cast<size_t>(m) * g.K_l + c] = codes[static_cast<size_t>(m) * g.K_lp + c];
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < g.r; i += blockDim.x)
+            if (xh) xh[static_cast<size_t>(m) * g.r + i] = xh_pad[static_cast<size_t>(m) * g.r_pad + i];
+        for (int gi = threadIdx.x; gi < g.n_g; gi += blockDim.x)
+            if (scales)
+                scales[static_cast<size_t>(m) * g.n_g + gi] =
+                    static_cast<uint16_t>(__float_as_uint(xscale[static_cast<size_t>(gi) * ldm + m]) >> 16);
+    }
+}
+
+inline bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
+
+}  // namespace
+
+dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
+                               int q_dtype, const void* bias, double* scratch, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    char* blob = L->blob;
+    fold_kernel<<<dim3((g.N + 63) / 64, (g.K + 63) / 64), 256, 0, stream>>>(Q, q_dtype, W, w_dtype, w_layout, scratch,
+                                                                          g.K, g.N);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    // zero the packed codes first: slots of a ragged last group stay zero
+    if (cudaMemsetAsync(blob + L->lay.off_wpacked, 0, static_cast<size_t>(g.N) * (g.K_lp / 2), stream) != cudaSuccess)
+        return DIROTQ_ERR_CUDA;
+    quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
+        Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                       reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint16_t* wscales, uint16_t* wh,
+                                    uint16_t* qb, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const char* blob = L->blob;
+    if (wcodes) {
+        export_wcodes_kernel<<<dim3((g.N + 127) / 128, g.K_l), 128, 0, stream>>>(
+            reinterpret_cast<const uint8_t*>(blob + L->lay.off_wpacked), wcodes, g);
+        if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    }
+    if (wscales) {
+        const size_t count = static_cast<size_t>(g.n_g) * g.N;
+        export_wscales_kernel<<<static_cast<unsigned>((count + 255) / 256), 256, 0, stream>>>(
+            reinterpret_cast<const float*>(blob + L->lay.off_wscale), wscales, count);
+        if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    }
+    if (wh) {
+        export_wh_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(
+            reinterpret_cast<const uint16_t*>(blob + L->lay.off_wh), wh, g);
+        if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    }
+    if (qb) {
+        export_q_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
+            reinterpret_cast<const uint16_t*>(blob + L->lay.off_qt), qb, g);
+        if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    }
+    return DIROTQ_OK;
+}
+
+dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
+                                        int8_t* codes, uint16_t* scales, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const WorkspaceLayout w = make_workspace_layout(g, M);
+    export_workspace_kernel<<<dim3(8, M), 256, 0, stream>>>(
+        reinterpret_cast<const int8_t*>(workspace + w.off_codes), reinterpret_cast<const float*>(workspace + w.off_xscale),
+        reinterpret_cast<const uint16_t*>(workspace + w.off_xh), M, w.ldm, g, xh, codes, scales);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace dirotq

@@ -1,0 +1,298 @@
+// Kernel (a): online rotation, split and activation quantization in one pass.
+//
+//   x~ = x Q_b                      bf16 x bf16 -> fp32 on tcgen05 (kind::f16), operands by TMA
+//   x~_h = bf16(x~[:, high])        the r high-precision coefficients          (paper Sec. 4.2)
+//   per token, per group of G low-precision coefficients:                      (paper Eq. 1, z = 0)
+//       s = bf16(max|x~| / 7),  q = clip(rint(x~ / s), -7, 7)
+//
+// The rotated activations never reach HBM: the fp32 accumulators are read from tensor memory by
+// the epilogue warps, where each thread owns one token row, so the group maximum is a
+// thread-local reduction over the row's G values.
+//
+// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
+// warps 2..5 = epilogue (lane quadrant = warp_id % 4).  Persistent CTAs walk the tile list;
+// two 128x256 fp32 accumulators in TMEM let the epilogue of tile i overlap the MMAs of tile i+1.
+#include "common.h"
+#include "ptx.cuh"
+
+#include <cuda_bf16.h>
+
+namespace dirotq {
+namespace {
+
+constexpr int BM = 128;       // tokens per tile
+constexpr int BN = 256;       // rotated columns per tile
+constexpr int BK = 64;        // bf16 elements per k-block (128-byte rows)
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;  // 16 KB
+constexpr int B_BYTES = BN * BK * 2;  // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct RotKernelParams {
+    int M, K, K_l, K_lp, r, r_pad, ldm;
+    int8_t* codes;
+    float* xscale;
+    uint16_t* xh;
+    float* xrot;
+    int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Quantizes 16 consecutive values with the reciprocal scale and packs them one code per byte.
+__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, bool slow) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float t = slow ? (s != 0.f ? v[4 * i + j] / s : 0.f) : v[4 * i + j] * inv;
+            int q = __float2int_rn(t);  // round to nearest, ties to even
+            q = max(-7, min(7, q));
+            word |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * j);
+        }
+        w[i] = word;
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <int G>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
+                    const RotKernelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+    // barrier map (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + STAGES * STAGE_BYTES + 128);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + STAGES * STAGE_BYTES + 132);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    const int num_m_blocks = (p.M + BM - 1) / BM;
+    const int num_n_blocks = (p.K + BN - 1) / BN;
+    const int num_tiles = num_m_blocks * num_n_blocks;
+    const int num_kb = p.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_x);
+        tma_prefetch_desc(&tmap_qt);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m0 = (tile % num_m_blocks) * BM;
+                const int n0 = (tile / num_m_blocks) * BN;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                    mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+                    const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    tma_load_2d(sa, &tmap_x, full_bar(s), kb * BK, m0);
+                    tma_load_2d(sa + A_BYTES, &tmap_qt, full_bar(s), kb * BK, n0);
+                }
+            }
+            if (!ok) {
+                // leave no bulk copy in flight: wait (bounded) for the loads already issued
+                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1) &&
+                           globaltimer_ns() - t0 < 100000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+                const uint32_t acc = tcount & 1;
+                const uint32_t acc_ph = (tcount >> 1) & 1;
+                if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    const uint64_t adesc = umma_desc_sw128(sa);
+                    const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(tfull_bar(acc));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            const int m0 = (tile % num_m_blocks) * BM;
+            const int n_blk = tile / num_m_blocks;
+            const int n0 = n_blk * BN;
+            const uint32_t acc = tcount & 1;
+            const uint32_t acc_ph = (tcount >> 1) & 1;
+            if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int row = m0 + q * 32 + lane;
+            const bool row_ok = row < p.M;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+
+#pragma unroll 1
+            for (int chunk = 0; chunk < BN / G; ++chunk) {
+                const int col0 = n0 + chunk * G;  // permuted column of v[0]
+                if (col0 >= p.K) break;
+                float v[G];
+#pragma unroll
+                for (int c = 0; c < G / 32; ++c) {
+                    uint32_t raw[32];
+                    tmem_ld_32x32b_x32(taddr + chunk * G + c * 32, raw);
+                    tmem_ld_wait(raw);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[c * 32 + j] = __uint_as_float(raw[j]);
+                }
+                if (p.xrot != nullptr && row_ok) {
+#pragma unroll
+                    for (int b = 0; b < G / 16; ++b) {
+                        const int pc = col0 + 16 * b;
+                        const int oc = pc < p.K_l ? pc + p.r : pc - p.K_l;  // caller's column order
+                        float4* dst = reinterpret_cast<float4*>(p.xrot + static_cast<size_t>(row) * p.K + oc);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            dst[j] = make_float4(v[16 * b + 4 * j], v[16 * b + 4 * j + 1], v[16 * b + 4 * j + 2],
+                                                 v[16 * b + 4 * j + 3]);
+                    }
+                }
+                // number of low-precision values among v[] (a multiple of 16)
+                const int nlow = min(G, max(0, p.K_l - col0));
+                if (nlow > 0) {
+                    float amax = 0.f;
+#pragma unroll
+                    for (int b = 0; b < G / 16; ++b) {
+                        if (16 * b < nlow) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[16 * b + j]));
+                        }
+                    }
+                    const float s = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(amax, 7.0f)));
+                    const bool slow = !(s >= 1e-30f);  // zero or tiny scale: divide instead of multiplying
+                    const float inv = slow ? 0.f : __frcp_rn(s);
+                    if (row_ok) {
+                        p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
+                        int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+#pragma unroll
+                        for (int b = 0; b < G / 16; ++b) {
+                            uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
+                            if (16 * b < nlow) packed = quantize16(v + 16 * b, inv, s, slow);
+                            *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                        }
+                    }
+                }
+                if (nlow < G && row_ok) {
+                    // high-precision coefficients: permuted columns >= K_l
+#pragma unroll
+                    for (int b = 0; b < G / 16; ++b) {
+                        const int pc = col0 + 16 * b;
+                        if (16 * b >= nlow && pc < p.K) {
+                            uint4 lo = make_uint4(pack_bf16x2(v[16 * b + 0], v[16 * b + 1]), pack_bf16x2(v[16 * b + 2], v[16 * b + 3]),
+                                                  pack_bf16x2(v[16 * b + 4], v[16 * b + 5]), pack_bf16x2(v[16 * b + 6], v[16 * b + 7]));
+                            uint4 hi = make_uint4(pack_bf16x2(v[16 * b + 8], v[16 * b + 9]), pack_bf16x2(v[16 * b + 10], v[16 * b + 11]),
+                                                  pack_bf16x2(v[16 * b + 12], v[16 * b + 13]), pack_bf16x2(v[16 * b + 14], v[16 * b + 15]));
+                            uint4* dst = reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + (pc - p.K_l));
+                            dst[0] = lo;
+                            dst[1] = hi;
+                        }
+                    }
+                }
+            }
+            // release the accumulator: every tcgen05.ld of this warp has completed
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
+            if (n_blk == num_n_blocks - 1 && row_ok) {
+                for (int c = p.r; c < p.r_pad; c += 8)
+                    *reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + c) = make_uint4(0, 0, 0, 0);
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace
+
+dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    CUtensorMap tmap_x;
+    dirotq_status_t st = encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M,
+                                        (uint64_t)g.K * 2, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    RotKernelParams p;
+    p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.ldm = a.ldm;
+    p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
+    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.K + BN - 1) / BN);
+    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
+    auto kern = g.G == 64 ? rotate_quant_kernel<64> : rotate_quant_kernel<128>;
+    static bool attr_set[2] = {false, false};
+    const int vi = g.G == 64 ? 0 : 1;
+    if (!attr_set[vi]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return DIROTQ_ERR_CUDA;
+        attr_set[vi] = true;
+    }
+    kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_x, L->tmap_qt, p);
+    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace dirotq

@@ -1,0 +1,436 @@
+// Kernels (b)+(c): W4A4 group GEMM with per-group rescale, bf16 rank-r branch and bias.
+//
+//   y[m,n] = bf16( sum_g s_x[m,g] s_w[g,n] P_g[m,n]  +  sum_{i<r} x~_h[m,i] W~_h[i,n]  +  bias[n] )
+//   P_g[m,n] = sum_{j in group g} q_x[m,j] q_w[j,n]                              (paper Eq. 5)
+//
+// sm_100a has no INT4 MMA.  The weight codes stay packed (two per byte) in HBM and in the TMA
+// staging buffer; two "unpack" warps expand every k-block to one code per byte -- each nibble
+// is moved to the HIGH half of its byte, so the int8 operand is 16*q_w, exact -- into the
+// 128-byte-swizzled layout tcgen05.mma kind::i8 reads.  The activation codes arrive one per byte
+// from kernel (a) and go straight from TMA to the MMA.
+//
+// Every K-group gets its own int32 accumulator tile in tensor memory (two tiles, ping-pong): the
+// MMA warp fills tile g%2 while the epilogue warps drain tile (g-1)%2, convert to fp32 and fold
+// it into per-thread fp32 accumulators with the two group scales.  The bf16 rank-r branch is
+// issued as one more "group" (kind::f16 into the same ping-pong tile) and added unscaled.
+//
+// Roles (384 threads = 3 warpgroups):
+//   warpgroup 0: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-3 INT4->INT8 unpack
+//   warpgroups 1-2: epilogue; warp%4 selects the TMEM lane quadrant (token rows), the warpgroup
+//                   selects the 128-column half of the 256-wide tile.
+#include "common.h"
+#include "ptx.cuh"
+
+#include <cuda_bf16.h>
+
+namespace dirotq {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BKC = 128;  // int8 codes per k-block (128-byte rows)
+constexpr int STAGES = 3;
+constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_h chunk
+constexpr int BU_BYTES = BN * BKC;         // 32 KB  unpacked weight codes / bf16 W~_h chunk
+constexpr int BP_BYTES = BN * BKC / 2;     // 16 KB  packed weight codes (TMA staging)
+constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB
+constexpr int SC_SLOTS = 8;
+constexpr int SC_SW_BYTES = 2 * BN * 4;    // up to two groups per k-block
+constexpr int SC_SX_BYTES = 2 * BM * 4;
+constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 3 KB
+constexpr int NUM_THREADS = 384;
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
+constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024;
+
+struct GemmKernelParams {
+    int M, N, n_g, num_kb, lr_chunks;
+    const float* bias;
+    uint16_t* y;
+    int32_t* partials;
+    int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int G, bool kPartials>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
+                 const __grid_constant__ CUtensorMap tmap_wscale, const __grid_constant__ CUtensorMap tmap_xscale,
+                 const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
+                 const GemmKernelParams p) {
+    constexpr int GPK = BKC / G;       // groups per k-block: 2 (G = 64) or 1 (G = 128)
+    constexpr int MMA_PER_G = G / 32;  // kind::i8 instructions (K = 32) per group
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t sc_base = smem_base + STAGES * STAGE_BYTES;
+    const uint32_t bar_base = smem_base + BAR_OFFSET;
+    // barriers: full[S], unpacked[S], empty[S], sc_full[SC], sc_empty[SC], tmem_full[2], tmem_empty[2]
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto unp_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
+    auto scfull_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + s); };
+    auto scempty_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + SC_SLOTS + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 2 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 400);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 404);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    const int num_m_blocks = (p.M + BM - 1) / BM;
+    const int num_n_blocks = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m_blocks * num_n_blocks;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(unp_bar(s), 2);  // one arrival per unpack warp
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int s = 0; s < SC_SLOTS; ++s) {
+            mbar_init(scfull_bar(s), 1);
+            mbar_init(scempty_bar(s), NUM_EPI_WARPS);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_codes);
+        tma_prefetch_desc(&tmap_wpacked);
+        tma_prefetch_desc(&tmap_wscale);
+        tma_prefetch_desc(&tmap_xscale);
+        tma_prefetch_desc(&tmap_xh);
+        tma_prefetch_desc(&tmap_wh);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        reg_dealloc<72>();
+        if (warp == 0) {
+            // -------------------------------------------------------- TMA producer
+            if (lane == 0) {
+                uint32_t it = 0, sc_it = 0;
+                bool ok = true;
+                for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                    const int m0 = (tile % num_m_blocks) * BM;
+                    const int n0 = (tile / num_m_blocks) * BN;
+                    for (int kb = 0; kb < p.num_kb; ++kb, ++it, ++sc_it) {
+                        const int s = it % STAGES;
+                        if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                        const uint32_t st = smem_base + s * STAGE_BYTES;
+                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
+                        tma_load_2d(st, &tmap_codes, full_bar(s), kb * BKC, m0);
+                        tma_load_2d(st + A_BYTES + BU_BYTES, &tmap_wpacked, full_bar(s), kb * (BKC / 2), n0);
+                        const int slot = sc_it % SC_SLOTS;
+                        if (!mbar_wait(scempty_bar(slot), ((sc_it / SC_SLOTS) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                        const uint32_t sc = sc_base + slot * SC_BYTES;
+                        mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + BM) * 4);
+                        tma_load_2d(sc, &tmap_wscale, scfull_bar(slot), n0, kb * GPK);
+                        tma_load_2d(sc + SC_SW_BYTES, &tmap_xscale, scfull_bar(slot), m0, kb * GPK);
+                    }
+                    if (!ok) break;
+                    for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
+                        const int s = it % STAGES;
+                        if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                        const uint32_t st = smem_base + s * STAGE_BYTES;
+                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BU_BYTES);
+                        tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
+                        tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), lr * 64, n0);
+                    }
+                }
+                if (!ok) {
+                    const uint32_t first = it > STAGES ? it - STAGES : 0;
+                    for (uint32_t j = first; j < it; ++j) {
+                        const unsigned long long t0 = globaltimer_ns();
+                        while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1) &&
+                               globaltimer_ns() - t0 < 100000000ull) {}
+                    }
+                    const uint32_t sfirst = sc_it > SC_SLOTS ? sc_it - SC_SLOTS : 0;
+                    for (uint32_t j = sfirst; j < sc_it; ++j) {
+                        const unsigned long long t0 = globaltimer_ns();
+                        while (!mbar_try_wait(scfull_bar(j % SC_SLOTS), (j / SC_SLOTS) & 1) &&
+                               globaltimer_ns() - t0 < 100000000ull) {}
+                    }
+                }
+            }
+        } else if (warp == 1) {
+            // -------------------------------------------------------- MMA issuer
+            if (lane == 0) {
+                constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);
+                constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
+                uint32_t it = 0, git = 0;
+                bool ok = true;
+                for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                    for (int kb = 0; ok && kb < p.num_kb; ++kb, ++it) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
+                            !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t st = smem_base + s * STAGE_BYTES;
+                        const uint64_t adesc = umma_desc_sw128(st);
+                        const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+                        const int ng_here = min(GPK, p.n_g - kb * GPK);
+                        for (int gi = 0; gi < ng_here; ++gi, ++git) {
+                            const uint32_t b = git & 1;
+                            if (!mbar_wait(tempty_bar(b), ((git >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                            tc_fence_after_sync();
+#pragma unroll
+                            for (int k = 0; k < MMA_PER_G; ++k) {
+                                const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
+                                umma_i8(tmem_base + b * BN, adesc + 2 * kk, bdesc + 2 * kk, idesc_i8, k != 0);
+                            }
+                            umma_commit(tfull_bar(b));
+                        }
+                        umma_commit(empty_bar(s));
+                    }
+                    if (!ok) break;
+                    // rank-r bf16 branch: one more accumulator tile, fp32
+                    const uint32_t b = git & 1;
+                    if (!mbar_wait(tempty_bar(b), ((git >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
+                            !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t st = smem_base + s * STAGE_BYTES;
+                        const uint64_t adesc = umma_desc_sw128(st);
+                        const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16(tmem_base + b * BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, (lr | k) != 0);
+                        umma_commit(empty_bar(s));
+                    }
+                    if (!ok) break;
+                    umma_commit(tfull_bar(b));
+                    ++git;
+                }
+            }
+        } else {
+            // -------------------------------------------------------- INT4 -> INT8 unpack (warps 2, 3)
+            const int u = threadIdx.x - 64;  // 0..63
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int items = p.num_kb + p.lr_chunks;
+                for (int i = 0; i < items; ++i, ++it) {
+                    const int s = it % STAGES;
+                    ok = mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+                    ok = __any_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    if (i < p.num_kb) {
+                        uint8_t* st = smem_gen + s * STAGE_BYTES;
+                        const uint4* src = reinterpret_cast<const uint4*>(st + A_BYTES + BU_BYTES);
+                        uint8_t* dst = st + A_BYTES;
+#pragma unroll 4
+                        for (int j = 0; j < (BN * 4) / 64; ++j) {
+                            const int idx = u + 64 * j;  // 16-byte piece of the packed tile: row = idx/4, piece = idx%4
+                            const int row = idx >> 2;
+                            const int c = idx & 3;
+                            const uint4 pk = src[idx];
+                            // low nibbles of a word are codes k..k+3, high nibbles k+4..k+7 (see prepare.cu)
+                            uint4 o0, o1;
+                            o0.x = (pk.x << 4) & 0xF0F0F0F0u; o0.y = pk.x & 0xF0F0F0F0u;
+                            o0.z = (pk.y << 4) & 0xF0F0F0F0u; o0.w = pk.y & 0xF0F0F0F0u;
+                            o1.x = (pk.z << 4) & 0xF0F0F0F0u; o1.y = pk.z & 0xF0F0F0F0u;
+                            o1.z = (pk.w << 4) & 0xF0F0F0F0u; o1.w = pk.w & 0xF0F0F0F0u;
+                            uint8_t* drow = dst + row * 128;
+                            const int sw = row & 7;  // 128-byte swizzle: 16-byte chunk index ^ (row % 8)
+                            *reinterpret_cast<uint4*>(drow + (((2 * c) ^ sw) << 4)) = o0;
+                            *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ sw) << 4)) = o1;
+                        }
+                        fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(unp_bar(s));
+                }
+            }
+        }
+    } else {
+        reg_alloc<208>();
+        // ------------------------------------------------------------ epilogue (warps 4..11)
+        const int q = warp & 3;
+        const int half = (warp - 4) >> 2;
+        const int row_in_tile = q * 32 + lane;
+        uint32_t git = 0, sc_it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            const int m0 = (tile % num_m_blocks) * BM;
+            const int n0 = (tile / num_m_blocks) * BN;
+            const int row = m0 + row_in_tile;
+            const int colbase = n0 + half * 128;
+            float acc[128];
+#pragma unroll
+            for (int j = 0; j < 128; ++j) acc[j] = 0.f;
+
+            for (int kb = 0; ok && kb < p.num_kb; ++kb, ++sc_it) {
+                const int slot = sc_it % SC_SLOTS;
+                ok = mbar_wait(scfull_bar(slot), (sc_it / SC_SLOTS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+                ok = __any_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const float* s_sw = reinterpret_cast<const float*>(smem_gen + STAGES * STAGE_BYTES + slot * SC_BYTES);
+                const float* s_sx = s_sw + 2 * BN;
+                const int ng_here = min(GPK, p.n_g - kb * GPK);
+                for (int gi = 0; gi < ng_here; ++gi, ++git) {
+                    const uint32_t b = git & 1;
+                    ok = mbar_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+                    ok = __any_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    // operand B carries 16*q_w: fold the 1/16 into the activation scale (exact)
+                    const float sx = s_sx[gi * BM + row_in_tile] * 0.0625f;
+                    const float* swp = s_sw + gi * BN + half * 128;
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t raw[32];
+                        tmem_ld_32x32b_x32(taddr + c * 32, raw);
+                        tmem_ld_wait(raw);
+                        if (c == 3) {
+                            // the whole tile is in registers: hand it back to the MMA warp
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(tempty_bar(b));
+                        }
+                        if constexpr (kPartials) {
+                            if (row < p.M) {
+                                const int g = kb * GPK + gi;
+                                int32_t* dst = p.partials + (static_cast<size_t>(g) * p.M + row) * p.N + colbase + c * 32;
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4) {
+                                    if (colbase + c * 32 + j < p.N)
+                                        *reinterpret_cast<int4*>(dst + j) =
+                                            make_int4(static_cast<int32_t>(raw[j]) >> 4, static_cast<int32_t>(raw[j + 1]) >> 4,
+                                                      static_cast<int32_t>(raw[j + 2]) >> 4, static_cast<int32_t>(raw[j + 3]) >> 4);
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 w = *reinterpret_cast<const float4*>(swp + c * 32 + j);
+                                acc[c * 32 + j + 0] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 0])) * w.x, sx, acc[c * 32 + j + 0]);
+                                acc[c * 32 + j + 1] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 1])) * w.y, sx, acc[c * 32 + j + 1]);
+                                acc[c * 32 + j + 2] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 2])) * w.z, sx, acc[c * 32 + j + 2]);
+                                acc[c * 32 + j + 3] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 3])) * w.w, sx, acc[c * 32 + j + 3]);
+                            }
+                        }
+                    }
+                }
+                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(scempty_bar(slot));
+            }
+            if (!ok) break;
+            // rank-r branch: fp32 tile
+            {
+                const uint32_t b = git & 1;
+                ok = mbar_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+                ok = __any_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t raw[32];
+                    tmem_ld_32x32b_x32(taddr + c * 32, raw);
+                    tmem_ld_wait(raw);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[c * 32 + j] += __uint_as_float(raw[j]);
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(b));
+                ++git;
+            }
+            if constexpr (!kPartials) {
+                if (row < p.M) {
+                    uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + colbase;
+#pragma unroll
+                    for (int j = 0; j < 128; j += 8) {
+                        if (colbase + j < p.N) {
+                            const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + colbase + j));
+                            const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + colbase + j + 4));
+                            uint4 o;
+                            o.x = pack_bf16x2(acc[j + 0] + b0.x, acc[j + 1] + b0.y);
+                            o.y = pack_bf16x2(acc[j + 2] + b0.z, acc[j + 3] + b0.w);
+                            o.z = pack_bf16x2(acc[j + 4] + b1.x, acc[j + 5] + b1.y);
+                            o.w = pack_bf16x2(acc[j + 6] + b1.z, acc[j + 7] + b1.w);
+                            *reinterpret_cast<uint4*>(yrow + j) = o;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace
+
+dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    CUtensorMap tmap_codes, tmap_xscale, tmap_xh;
+    dirotq_status_t st;
+    st = encode_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K_lp, (uint64_t)a.M,
+                        (uint64_t)g.K_lp, BKC, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    st = encode_tmap_2d(&tmap_xscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xscale, (uint64_t)a.ldm, (uint64_t)g.n_g,
+                        (uint64_t)a.ldm * 4, BM, BKC / g.G, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st != DIROTQ_OK) return st;
+    st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,
+                        (uint64_t)g.r_pad * 2, 64, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+
+    GemmKernelParams p;
+    p.M = a.M; p.N = g.N; p.n_g = g.n_g;
+    p.num_kb = (g.K_lp + BKC - 1) / BKC;
+    p.lr_chunks = g.r_pad / 64;
+    p.bias = reinterpret_cast<const float*>(L->blob + L->lay.off_bias);
+    p.y = a.y; p.partials = a.partials; p.status = a.status;
+
+    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
+                              const CUtensorMap, const CUtensorMap, const GemmKernelParams);
+    KernelFn kern;
+    const bool dbg = a.partials != nullptr;
+    if (g.G == 64) kern = dbg ? w4a4_gemm_kernel<64, true> : w4a4_gemm_kernel<64, false>;
+    else           kern = dbg ? w4a4_gemm_kernel<128, true> : w4a4_gemm_kernel<128, false>;
+    static bool attr_set[4] = {false, false, false, false};
+    const int vi = (g.G == 64 ? 0 : 2) + (dbg ? 1 : 0);
+    if (!attr_set[vi]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return DIROTQ_ERR_CUDA;
+        attr_set[vi] = true;
+    }
+    kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, L->tmap_wscale, tmap_xscale, tmap_xh,
+                                                    L->tmap_wh, p);
+    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace dirotq

@@ -1,0 +1,71 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and validates arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2605_16732_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2605_16732_b200 import build
+    build.build()
+    return binding.lib()
+
+
+def test_every_declared_symbol_is_exported(L):
+    header = open(os.path.join(ROOT, "include", "dirotq.h")).read()
+    declared = sorted(set(re.findall(r"DIROTQ_API\s+[\w\s\*]+?\b(dirotq_\w+)\s*\(", header)))
+    assert len(declared) >= 16
+    assert sorted(binding.EXPORTED) == declared
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def test_status_strings(L):
+    assert L.dirotq_status_string(0) == b"ok"
+    assert L.dirotq_status_string(6) == b"device-side wait timed out"
+    assert L.dirotq_version() >= 100
+
+
+def test_layer_bytes_and_shape_validation(L):
+    n = ctypes.c_size_t(0)
+    assert L.dirotq_layer_bytes(1152, 1152, 32, 64, ctypes.byref(n)) == 0
+    K, N, r, G = 1152, 1152, 32, 64
+    n_g = -(-(K - r) // G)
+    floor = K * K * 2 + N * n_g * G // 2 + n_g * N * 4 + N * 64 * 2 + N * 4
+    assert floor <= n.value <= floor + 6 * 1024
+    # unsupported shapes are refused
+    for bad in [(1100, 1152, 32, 64), (1152, 1150, 32, 64), (1152, 1152, 24, 64), (1152, 1152, 32, 32),
+                (1152, 1152, 256, 64), (64, 64, 64, 64), (192, 64, 32, 128)]:
+        assert L.dirotq_layer_bytes(*bad, ctypes.byref(n)) == 2, bad
+    assert L.dirotq_layer_bytes(-1, 64, 32, 64, ctypes.byref(n)) == 1
+    assert L.dirotq_layer_bytes(1152, 1152, 32, 64, None) == 1
+
+
+def test_scratch_bytes(L):
+    n = ctypes.c_size_t(0)
+    assert L.dirotq_prepare_scratch_bytes(3072, 9216, ctypes.byref(n)) == 0
+    assert n.value == 3072 * 9216 * 8
+
+
+def test_null_and_bad_handles_are_rejected(L):
+    n = ctypes.c_size_t(0)
+    assert L.dirotq_workspace_bytes(None, 16, ctypes.byref(n)) == 1
+    assert L.dirotq_layer_destroy(None) == 1
+    assert L.dirotq_linear(None, 1, None, None, None, 0, None) == 1
+    assert L.dirotq_rotate_quantize(None, 1, None, None, 0, None, None) == 1
+    assert L.dirotq_int_gemm_debug(None, 1, None, None, None, 0, None) == 1
+    assert L.dirotq_layer_export(None, None, None, None, None, None) == 1
+    h = ctypes.c_void_p(0)
+    # NULL tensors: refused before any CUDA call
+    assert L.dirotq_prepare_layer(None, 0, 0, None, 2, None, 128, 64, 32, 64, None, 0, None, 0, None,
+                                  ctypes.byref(h)) == 1
+    # a fake handle (wrong magic) is refused too
+    fake = ctypes.create_string_buffer(4096)
+    assert L.dirotq_workspace_bytes(fake, 16, ctypes.byref(n)) == 1
