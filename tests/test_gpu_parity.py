@@ -7,7 +7,7 @@ from oracle import dirotq_oracle as orc
 from paper_2605_16732_b200 import binding as dq
 from paper_2605_16732_b200 import synth
 
-from parity_utils import (bf16_tensor_to_bits, bits_to_bf16_tensor, check_activation_side, check_output,
+from parity_utils import (bf16_tensor_to_bits, bits_to_bf16_tensor, check_activation_side, check_layer_output,
                           check_weight_side)
 
 pytestmark = pytest.mark.gpu
@@ -33,8 +33,9 @@ def _run_case(spec: synth.LayerSpec, M: int, with_bias=True, x_override=None, ch
     dq.dirotq_rotate_quantize(x, layer, ws, xrot)
     assert dq.dirotq_workspace_status(ws) == 0
     xh, codes, scales = dq.dirotq_workspace_export(layer, M, ws)
-    stats = check_activation_side(xrot.cpu().numpy() if check_rot else None, bf16_tensor_to_bits(xh),
-                                  codes.cpu().numpy(), bf16_tensor_to_bits(scales), oo, spec.r, spec.G)
+    xh_b, codes_n, scales_b = bf16_tensor_to_bits(xh), codes.cpu().numpy(), bf16_tensor_to_bits(scales)
+    stats = check_activation_side(xrot.cpu().numpy() if check_rot else None, xh_b, codes_n, scales_b, oo, spec.r,
+                                  spec.G)
 
     # integer GEMM on the oracle's codes: bit exact
     padded = np.zeros((M, layer.K_lp), dtype=np.int8)
@@ -47,7 +48,7 @@ def _run_case(spec: synth.LayerSpec, M: int, with_bias=True, x_override=None, ch
     y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
     dq.dirotq_linear(x, layer, y, ws)
     assert dq.dirotq_workspace_status(ws) == 0
-    stats["y_err_over_rms"] = check_output(bf16_tensor_to_bits(y), oo["y64"])
+    stats.update(check_layer_output(bf16_tensor_to_bits(y), xh_b, codes_n, scales_b, lo, oo, inp["bias"]))
     # a second call on the same workspace gives the same bits (the integer path is deterministic)
     y2 = torch.zeros_like(y)
     dq.dirotq_linear(x, layer, y2, ws)
