@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the DiRotQ W4A4 linear layer on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+One "step" is one pass of the whole hot path (rotate + split + quantize, W4A4 group GEMM,
+rank-r branch, epilogue) over the four FLUX.1-dev-shaped linears at M = 4608 tokens
+(3072->9216, 3072->3072, 3072->12288, 12288->3072; r = 32, group 64).  The metric is effective
+TOPS, sum(2*M*N*K) / time.  Inputs are seeded and synthetic (see paper_2605_16732_b200/synth.py).
+
+With N > 1 (torchrun) every rank runs the same step on its own M tokens (token rows are
+independent: no collective on the data path) and the value is the aggregate over ranks.
+
+``--impl reference`` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FLUX_SHAPES = [("qkv", 3072, 9216), ("out", 3072, 3072), ("mlp_up", 3072, 12288), ("mlp_down", 12288, 3072)]
+M_TOKENS = 4608
+RANK, GROUP = 32, 64
+WORKLOAD = "flux1dev_linears_M4608_r32_g64"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"], "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # median over the samples taken under load (upper half by clock x power is a poor proxy; use power)
+        order = np.argsort(power)
+        load = [sm[i] for i in order[len(order) // 2:]]
+        return {"sm_mhz": float(np.median(load)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": float(max(power))}
+
+
+def _shape_ops(M):
+    return sum(2.0 * M * N * K for _, K, N in FLUX_SHAPES)
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (bounded sample)
+
+
+def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0):
+    """Times the oracle's online steps on `rows` tokens x `cols` output columns of every linear."""
+    from oracle import dirotq_oracle as orc
+    from paper_2605_16732_b200 import synth
+
+    layers = []
+    for name, K, N in FLUX_SHAPES:
+        spec = synth.LayerSpec(K=K, N=N, r=RANK, G=GROUP, model=synth.FLUX, seed=seed)
+        g = np.random.Generator(np.random.Philox(key=[K, N]))
+        # the oracle's run time does not depend on the rotation's values: a seeded Householder
+        # reflection (dense, exactly orthogonal) stands in for the PCA rotation, whose
+        # eigendecomposition takes minutes on a CPU at K = 12288
+        v = g.standard_normal(K)
+        v /= np.linalg.norm(v)
+        Q = np.eye(K) - 2.0 * np.outer(v, v)
+        W = (0.02 * g.standard_normal((K, cols))).astype(np.float32)
+        lo = orc.prepare_layer(W, Q, RANK, GROUP)
+        x = synth.make_tokens(spec, rows, batch_seed=5)
+        layers.append((lo, x, K, cols))
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        for lo, x, K, n in layers:
+            orc.linear_deployed(x, lo, bias=None, want_t=False)
+        times.append(time.perf_counter() - t0)
+    ops = sum(2.0 * rows * n * K for _, _, K, n in layers)
+    t = float(np.mean(times))
+    return {"value": ops / t / 1e12, "unit": "TOPS", "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{rows} token rows x {cols} output columns of each of the 4 linears, online steps only "
+                      f"(rotation, quantize, int GEMM, combine); Householder rotation",
+            "seconds_per_step": t}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, args.steps)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_run(1)
+    res = oracle_sample_run(steps)
+    line = {
+        "impl": "reference", "metric": "dirotq_w4a4_linear_effective_tops", "value": res["value"], "unit": "TOPS",
+        "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4xint4->int32 + bf16",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": res["sample"]},
+        "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": res["value"], "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+
+
+def run_ours(args):
+    import torch
+    from paper_2605_16732_b200 import binding as dq
+    from paper_2605_16732_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    M = M_TOKENS
+    peaks = _peaks()
+
+    def bf(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    layers = []
+    for name, K, N in FLUX_SHAPES:
+        spec = synth.LayerSpec(K=K, N=N, r=RANK, G=GROUP, model=synth.FLUX, seed=100)
+        Q = torch.from_numpy(synth.make_rotation(spec, device=str(dev))).to(dev)
+        W, bias = synth.make_weights(spec)
+        layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
+        del Q
+        x_bits = synth.make_tokens(spec, M, batch_seed=1000 + rank)
+        x = bf(x_bits)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        ws = dq.alloc_workspace(layer, M)
+        layers.append({"name": name, "K": K, "N": N, "layer": layer, "x": x, "y": y, "ws": ws, "x_bits": x_bits})
+    torch.cuda.synchronize()
+
+    def step():
+        for L in layers:
+            dq.dirotq_linear(L["x"], L["layer"], L["y"], L["ws"])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    if rank == 0 and not args.lite:
+        sampler.start()
+        time.sleep(1.0)
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    # ---- headline: K steps, device-timed
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+
+    # ---- per-kernel durations over the same steps (events on the launching stream)
+    evs = []
+    for _ in range(args.steps):
+        for L in layers:
+            a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a.record()
+            dq.dirotq_rotate_quantize(L["x"], L["layer"], L["ws"])
+            b.record()
+            dq.dirotq_w4a4_gemm(M, L["layer"], L["ws"], L["y"])
+            c.record()
+            evs.append((L["name"], a, b, c))
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 and not args.lite else None
+    per = {}
+    for name, a, b, c in evs:
+        d = per.setdefault(name, {"rotate_ms": [], "gemm_ms": []})
+        d["rotate_ms"].append(a.elapsed_time(b))
+        d["gemm_ms"].append(b.elapsed_time(c))
+    for L in layers:
+        assert dq.dirotq_workspace_status(L["ws"]) == 0, "a device-side wait timed out"
+
+    # ---- cuBLAS bf16 comparison on the same shapes (context)
+    cublas = {}
+    for L in ([] if args.lite else layers):
+        Wb = torch.randn((L["K"], L["N"]), device=dev, dtype=torch.bfloat16) * 0.02
+        for _ in range(3):
+            torch.matmul(L["x"], Wb)
+        ts = []
+        for _ in range(10):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); torch.matmul(L["x"], Wb); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        cublas[L["name"]] = float(np.median(ts))
+        del Wb
+
+    # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region)
+    host = []
+    for L in ([] if args.lite else layers):
+        xh = torch.empty((M, L["K"]), dtype=torch.bfloat16).pin_memory()
+        xh.copy_(L["x"].cpu())
+        yh = torch.empty((M, L["N"]), dtype=torch.bfloat16).pin_memory()
+        host.append((xh, yh))
+    e2e_steps = max(1, min(args.steps, 5))
+
+    def e2e_step():
+        for L, (xh, yh) in zip(layers, host):
+            dq.dirotq_linear_host(xh, L["layer"], yh, L["x"], L["y"], L["ws"])
+
+    e2e_ms = float("nan")
+    if not args.lite:
+        e2e_step()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(M * L["K"] * 2 for L in layers)
+    d2h = sum(M * L["N"] * 2 for L in layers)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ops_step = _shape_ops(M)
+    value = world * ops_step / (ms_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel: the rotation GEMM (bf16 tensor cores)
+    rot_ms = {n: float(np.mean(v["rotate_ms"])) for n, v in per.items()}
+    gemm_ms = {n: float(np.mean(v["gemm_ms"])) for n, v in per.items()}
+    rot_total, gemm_total = sum(rot_ms.values()), sum(gemm_ms.values())
+    rot_flops = {n: 2.0 * M * K * K for n, K, _ in FLUX_SHAPES}
+    gemm_ops = {n: 2.0 * M * (K - RANK) * N for n, K, N in FLUX_SHAPES}
+    int8_peak = 2.0 * peaks["bf16_sustained"]  # nominal int8 : bf16 ratio of the part (4.5 : 2.25)
+    if rot_total >= gemm_total:
+        ach = sum(rot_flops.values()) / (rot_total * 1e-3) / 1e12
+        roofline = {"kernel": "rotate_quant_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_sustained"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_sustained"], "traffic": None,
+                    "peak_source": f"{peaks['source']} bf16 sustained"}
+    else:
+        ach = sum(gemm_ops.values()) / (gemm_total * 1e-3) / 1e12
+        roofline = {"kernel": "w4a4_gemm_kernel", "bound": "tensor", "achieved": ach, "peak": int8_peak, "unit": "TOP/s",
+                    "frac": ach / int8_peak, "traffic": None,
+                    "peak_source": f"2 x {peaks['source']} bf16 sustained (nominal int8:bf16 ratio)"}
+    kernels = {}
+    for n, K, N in FLUX_SHAPES:
+        t_roof = (gemm_ops[n] / int8_peak + (rot_flops[n] + 2.0 * M * RANK * N) / peaks["bf16_sustained"]) / 1e12 * 1e3
+        tot = rot_ms[n] + gemm_ms[n]
+        kernels[n] = {
+            "rotate_ms": rot_ms[n], "rotate_tflops": rot_flops[n] / (rot_ms[n] * 1e-3) / 1e12,
+            "rotate_frac_bf16_peak": rot_flops[n] / (rot_ms[n] * 1e-3) / 1e12 / peaks["bf16_sustained"],
+            "gemm_ms": gemm_ms[n], "gemm_tops": gemm_ops[n] / (gemm_ms[n] * 1e-3) / 1e12,
+            "gemm_frac_int8_peak": gemm_ops[n] / (gemm_ms[n] * 1e-3) / 1e12 / int8_peak,
+            "effective_tops": 2.0 * M * N * K / (tot * 1e-3) / 1e12,
+            "frac_of_composite_roofline": t_roof / tot,
+            "cublas_bf16_ms": cublas.get(n), "speedup_vs_cublas_bf16": cublas[n] / tot if n in cublas else None,
+        }
+
+    cpu = oracle_sample_run(1) if not args.lite else {"value": None, "unit": "TOPS", "cores": None, "kind": "oracle",
+                                                      "sample": "skipped (--lite)"}
+    line = {
+        "metric": "dirotq_w4a4_linear_effective_tops", "value": value, "unit": "TOPS", "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int4xint4->int32 + bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK, "group": GROUP,
+                   "l2": "inputs_exceed_l2 (each step streams > 500 MB of rotations, codes and outputs)",
+                   "parallelism": f"token rows x{world}, no collective"},
+        "clocks": clocks,
+        "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "gpu_launches": 2 * len(layers) * args.steps,
+        "roofline": roofline,
+        "kernels": kernels,
+        "frac_int8_peak_effective": value / world / int8_peak,
+        "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--shapes", default="", help="comma-separated subset of qkv,out,mlp_up,mlp_down (profiling runs)")
+    ap.add_argument("--lite", action="store_true", help="skip the cuBLAS, end-to-end and CPU-baseline legs (profiling runs)")
+    args = ap.parse_args()
+    if args.shapes:
+        keep = set(args.shapes.split(","))
+        FLUX_SHAPES[:] = [t for t in FLUX_SHAPES if t[0] in keep]
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

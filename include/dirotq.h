@@ -134,6 +134,14 @@ DIROTQ_API dirotq_status_t dirotq_workspace_status(const void* workspace, dirotq
 DIROTQ_API dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
                                        size_t workspace_bytes, float* xrot_f32, dirotq_stream_t stream);
 
+/* Runs only the second kernel (INT4 group GEMM, rescale, rank-r branch, bias) on a workspace
+ * that dirotq_rotate_quantize filled for the same layer geometry and M.  Together the two calls
+ * equal dirotq_linear; several layers that share one input and one rotation (the paper shares
+ * nothing but allows it: the rotation depends only on the input's calibration statistics,
+ * Sec. 4.2) can reuse a single rotate/quantize pass. */
+DIROTQ_API dirotq_status_t dirotq_w4a4_gemm(int M, const dirotq_layer_t* layer, const void* workspace,
+                                            size_t workspace_bytes, void* y, dirotq_stream_t stream);
+
 /* Copies the first kernel's results out of the workspace into plain layouts:
  * xh bf16 [M,r]; codes int8 [M,K-r], one code per byte; scales bf16 [M,n_g]. */
 DIROTQ_API dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,

@@ -25,7 +25,7 @@ EXPORTED = [
     "dirotq_status_string", "dirotq_version", "dirotq_last_error", "dirotq_layer_bytes",
     "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
-    "dirotq_rotate_quantize", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
+    "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
 ]
 
 
@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_linear_host.argtypes = [vp, i, vp, vp, vp, vp, vp, sz, vp]
         L.dirotq_workspace_status.argtypes = [vp, vp, pi]
         L.dirotq_rotate_quantize.argtypes = [vp, i, vp, vp, sz, vp, vp]
+        L.dirotq_w4a4_gemm.argtypes = [i, vp, vp, sz, vp, vp]
         L.dirotq_workspace_export.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_int_gemm_debug.argtypes = [vp, i, vp, vp, vp, sz, vp]
         L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -183,6 +184,11 @@ def dirotq_rotate_quantize(x: torch.Tensor, layer: Layer, workspace: torch.Tenso
                            stream=None) -> None:
     _check(lib().dirotq_rotate_quantize(x.data_ptr(), x.shape[0], layer.handle, workspace.data_ptr(),
                                         workspace.numel(), _ptr(xrot), _stream(stream)), "dirotq_rotate_quantize")
+
+
+def dirotq_w4a4_gemm(M: int, layer: Layer, workspace: torch.Tensor, y: torch.Tensor, stream=None) -> None:
+    _check(lib().dirotq_w4a4_gemm(M, layer.handle, workspace.data_ptr(), workspace.numel(), y.data_ptr(),
+                                  _stream(stream)), "dirotq_w4a4_gemm")
 
 
 def dirotq_workspace_export(layer: Layer, M: int, workspace: torch.Tensor, stream=None):

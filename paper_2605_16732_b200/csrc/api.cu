@@ -249,6 +249,24 @@ dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer,
     return launch_w4a4_gemm(layer, ga, static_cast<cudaStream_t>(stream));
 }
 
+dirotq_status_t dirotq_w4a4_gemm(int M, const dirotq_layer_t* layer, const void* workspace, size_t workspace_bytes,
+                                 void* y, dirotq_stream_t stream) {
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    if (st != DIROTQ_OK) return st;
+    if (!y || !aligned16(y)) return DIROTQ_ERR_INVALID_ARG;
+    char* ws = const_cast<char*>(static_cast<const char*>(workspace));
+    const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
+    GemmArgs ga;
+    ga.M = M;
+    ga.codes = reinterpret_cast<const int8_t*>(ws + w.off_codes);
+    ga.xscale = reinterpret_cast<const float*>(ws + w.off_xscale);
+    ga.ldm = w.ldm;
+    ga.xh = reinterpret_cast<const uint16_t*>(ws + w.off_xh);
+    ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr;
+    ga.status = reinterpret_cast<int*>(ws + w.off_status);
+    return launch_w4a4_gemm(layer, ga, static_cast<cudaStream_t>(stream));
+}
+
 dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer_t* layer, void* y_host, void* x_dev,
                                    void* y_dev, void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
     dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
