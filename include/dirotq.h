@@ -158,6 +158,16 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,
                                     void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
 
+/* ---- measurement aid (no counterpart in the paper) ------------------------------------------ */
+
+/* Issue-rate probe of the tensor pipe: every SM issues 4*iters back-to-back 128x256 tcgen05.mma
+ * instructions on operands resident in shared memory (kind 0: int8 -> int32, K = 32 per
+ * instruction; kind 1: bf16 -> fp32, K = 16), twice (warm-up + timed).  SYNCHRONISES.
+ * status_word: device int32, zero-filled (receives a code if the bounded completion wait
+ * expires).  *tera_ops_per_s receives 2*M*N*K*instructions / time. */
+DIROTQ_API dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* status_word, float* tera_ops_per_s,
+                                                 dirotq_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

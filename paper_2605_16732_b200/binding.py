@@ -26,6 +26,7 @@ EXPORTED = [
     "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
+    "dirotq_mma_rate_probe",
 ]
 
 
@@ -65,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_workspace_export.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_int_gemm_debug.argtypes = [vp, i, vp, vp, vp, sz, vp]
         L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.dirotq_mma_rate_probe.argtypes = [i, i, vp, ctypes.POINTER(ctypes.c_float), vp]
         for name in EXPORTED:
             if name not in ("dirotq_status_string", "dirotq_version", "dirotq_last_error"):
                 getattr(L, name).restype = i
@@ -220,3 +222,14 @@ def dirotq_layer_export(layer: Layer, stream=None):
     _check(lib().dirotq_layer_export(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(), qb.data_ptr(),
                                      _stream(stream)), "dirotq_layer_export")
     return wcodes, wscales, wh, qb
+
+
+def dirotq_mma_rate_probe(kind: int, iters: int = 20000, stream=None) -> float:
+    """Measured tensor-pipe rate in tera-ops/s.  kind 0: int8 (kind::i8), kind 1: bf16 (kind::f16)."""
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")
+    out = ctypes.c_float(0.0)
+    _check(lib().dirotq_mma_rate_probe(kind, iters, status.data_ptr(), ctypes.byref(out), _stream(stream)),
+           "dirotq_mma_rate_probe")
+    if int(status[0].item()) != 0:
+        raise DirotqError(6, "dirotq_mma_rate_probe")
+    return float(out.value)

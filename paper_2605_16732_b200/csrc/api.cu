@@ -15,7 +15,6 @@ thread_local char g_last_error[256] = "";
 void set_error(const char* what, cudaError_t e) {
     snprintf(g_last_error, sizeof g_last_error, "%s: %s", what, cudaGetErrorString(e));
 }
-void set_error_text(const char* what) { snprintf(g_last_error, sizeof g_last_error, "%s", what); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -169,13 +168,13 @@ dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, c
                         (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
-                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_NONE);
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
-                            (uint64_t)g.n_g, (uint64_t)N * 4, 256, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+                            (uint64_t)g.n_g, (uint64_t)N * 4, kGemmBN, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
-                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, static_cast<double*>(scratch),
                             static_cast<cudaStream_t>(stream));

@@ -90,14 +90,15 @@ struct dirotq_layer {
     dirotq::BlobLayout lay;
     char* blob;  // device
     CUtensorMap tmap_qt;       // bf16 [K][K], box 64 x 256, 128B swizzle
-    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2], box 64 x 256, no swizzle
-    CUtensorMap tmap_wscale;   // f32 [n_g][N], box 256 x (128/G)
-    CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x 256, 128B swizzle
+    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2], box 64 x kGemmBN, no swizzle
+    CUtensorMap tmap_wscale;   // f32 [n_g][N], box kGemmBN x (128/G)
+    CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
 };
 
 namespace dirotq {
 
 constexpr uint32_t kLayerMagic = 0x44695251u;  // "DiRQ"
+constexpr int kGemmBN = 256;  // output columns per tile of the W4A4 kernel (rows of its weight-side TMA boxes)
 
 // ------------------------------------------------------------------ kernel launch interfaces
 

@@ -65,18 +65,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // shared memory, `status` a word in global memory that the host reads.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0;
 #pragma unroll 1
-    for (int i = 0; i < 128; ++i)
+    for (uint32_t spins = 1;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
-#pragma unroll 1
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag != 0) return false;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = code;
-            atomicCAS(status, 0, code);
-            return false;
+        if ((spins & 255u) == 0) {  // the abort flag and the clock are looked at once in a while only
+            if (*abort_flag != 0) return false;
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitNs) {
+                *abort_flag = code;
+                atomicCAS(status, 0, code);
+                return false;
+            }
         }
     }
 }
@@ -195,15 +197,6 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&v)
 
 __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Same wait, with the loaded registers tied to the statement so that no use of them can be
-// scheduled ahead of it.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
-                 :
-                 : "memory");
 }
 
 // ---------------------------------------------------------------- register budget

@@ -191,7 +191,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 for (int c = 0; c < G / 32; ++c) {
                     uint32_t raw[32];
                     tmem_ld_32x32b_x32(taddr + chunk * G + c * 32, raw);
-                    tmem_ld_wait(raw);
+                    tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[c * 32 + j] = __uint_as_float(raw[j]);
                 }

@@ -27,7 +27,7 @@ namespace dirotq {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = 256;
+constexpr int BN = kGemmBN;  // 256
 constexpr int BKC = 128;  // int8 codes per k-block (128-byte rows)
 constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_h chunk
@@ -303,7 +303,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     for (int c = 0; c < 4; ++c) {
                         uint32_t raw[32];
                         tmem_ld_32x32b_x32(taddr + c * 32, raw);
-                        tmem_ld_wait(raw);
+                        tmem_ld_wait();
                         if (c == 3) {
                             // the whole tile is in registers: hand it back to the MMA warp
                             tc_fence_before_sync();
@@ -351,7 +351,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 for (int c = 0; c < 4; ++c) {
                     uint32_t raw[32];
                     tmem_ld_32x32b_x32(taddr + c * 32, raw);
-                    tmem_ld_wait(raw);
+                    tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) acc[c * 32 + j] += __uint_as_float(raw[j]);
                 }
