@@ -309,16 +309,28 @@ def run_ours(args):
     rot_flops = {n: 2.0 * M * K * K for n, K, _ in FLUX_SHAPES}
     gemm_ops = {n: 2.0 * M * (K - RANK) * N for n, K, N in FLUX_SHAPES}
     int8_peak = 2.0 * peaks["bf16_sustained"]  # nominal int8 : bf16 ratio of the part (4.5 : 2.25)
+    # DRAM bytes of one launch of the dominant kernel, from the ncu capture summarised under profiles/
+    # (qkv shape; read + write).  Static: a profiler is never run inside the benchmark.
+    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 68.1e6, "rotate_quant_kernel": 48.5e6}
+    sm_hz = (clocks or {}).get("sm_mhz") or 1850.0
+    elem_steps = sum(M * N * (-(-(K - RANK) // GROUP)) for _, K, N in FLUX_SHAPES)
+    alu_peak = 148 * (128.0 / 3.0) * sm_hz * 1e6  # element-steps/s: 3 thread instructions each, 128 issued per cycle and SM
     if rot_total >= gemm_total:
         ach = sum(rot_flops.values()) / (rot_total * 1e-3) / 1e12
         roofline = {"kernel": "rotate_quant_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_sustained"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_sustained"], "traffic": None,
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_sustained"], "traffic": NCU_TRAFFIC_QKV["rotate_quant_kernel"],
                     "peak_source": f"{peaks['source']} bf16 sustained"}
     else:
         ach = sum(gemm_ops.values()) / (gemm_total * 1e-3) / 1e12
+        ach_alu = elem_steps / (gemm_total * 1e-3)
         roofline = {"kernel": "w4a4_gemm_kernel", "bound": "tensor", "achieved": ach, "peak": int8_peak, "unit": "TOP/s",
-                    "frac": ach / int8_peak, "traffic": None,
-                    "peak_source": f"2 x {peaks['source']} bf16 sustained (nominal int8:bf16 ratio)"}
+                    "frac": ach / int8_peak, "traffic": NCU_TRAFFIC_QKV["w4a4_gemm_kernel"],
+                    "traffic_note": "ncu dram read+write of one qkv-shaped launch (algorithmic bytes of that launch: 117.5e6)",
+                    "peak_source": f"2 x {peaks['source']} bf16 sustained (nominal int8:bf16 ratio)",
+                    "alu": {"bound": "alu", "achieved": ach_alu / 1e9, "peak": alu_peak / 1e9, "unit": "G element-steps/s",
+                            "frac": ach_alu / alu_peak,
+                            "note": "per-group rescale: >= 3 thread instructions per output element and K-group; "
+                                    "148 SMs x 128 issued thread instructions per cycle at the sampled SM clock"}}
     kernels = {}
     for n, K, N in FLUX_SHAPES:
         t_roof = (gemm_ops[n] / int8_peak + (rot_flops[n] + 2.0 * M * RANK * N) / peaks["bf16_sustained"]) / 1e12 * 1e3
