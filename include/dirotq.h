@@ -158,6 +158,25 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,
                                     void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
 
+/* ---- for callers that cannot allocate (no counterpart in the paper) ------------------------- */
+
+/* dirotq_linear without a workspace argument.  Meant for callers that are not allowed to call
+ * cudaMalloc where they run -- a plug-in inside a runtime that owns all device memory, code on a
+ * stream being captured, a fixed-memory real-time loop.  The workspace is a 16 MiB array built
+ * into the library's device image (resident on every GPU that loads the library, until exit);
+ * the call allocates nothing and calls no allocating routine.
+ *   - A call whose workspace (dirotq_workspace_bytes) exceeds 16 MiB returns
+ *     DIROTQ_ERR_BUFFER_TOO_SMALL and prints the two sizes on stderr; roughly M*K <= 16 Mi.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array: calls that may overlap on the GPU (different streams) race.
+ *     Calls on one stream are safe.  The status word is cleared at the start of every call.
+ *   - device_status: optional DEVICE int32 that receives the status word of this call (0 = every
+ *     wait completed), copied on `stream`; NULL to skip.
+ * Same arguments, layouts and results as dirotq_linear otherwise. */
+DIROTQ_API dirotq_status_t dirotq_linear_noalloc(const void* x, int M, const dirotq_layer_t* layer, void* y,
+                                                 int* device_status, dirotq_stream_t stream);
+
 /* ---- measurement aid (no counterpart in the paper) ------------------------------------------ */
 
 /* Issue-rate probe of the tensor pipe: every SM issues 4*iters back-to-back 128x256 tcgen05.mma

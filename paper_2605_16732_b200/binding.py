@@ -26,7 +26,7 @@ EXPORTED = [
     "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
-    "dirotq_mma_rate_probe",
+    "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
 ]
 
 
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_workspace_export.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_int_gemm_debug.argtypes = [vp, i, vp, vp, vp, sz, vp]
         L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.dirotq_linear_noalloc.argtypes = [vp, i, vp, vp, vp, vp]
         L.dirotq_mma_rate_probe.argtypes = [i, i, vp, ctypes.POINTER(ctypes.c_float), vp]
         for name in EXPORTED:
             if name not in ("dirotq_status_string", "dirotq_version", "dirotq_last_error"):
@@ -233,3 +234,12 @@ def dirotq_mma_rate_probe(kind: int, iters: int = 20000, stream=None) -> float:
     if int(status[0].item()) != 0:
         raise DirotqError(6, "dirotq_mma_rate_probe")
     return float(out.value)
+
+
+def dirotq_linear_noalloc(x: torch.Tensor, layer: Layer, y: torch.Tensor, device_status: torch.Tensor | None = None,
+                          stream=None) -> None:
+    """dirotq_linear on the library's built-in 16 MiB workspace: for callers that may not allocate.
+
+    device_status: optional cuda int32 tensor (1 element) that receives this call's device status word."""
+    _check(lib().dirotq_linear_noalloc(x.data_ptr(), x.shape[0], layer.handle, y.data_ptr(), _ptr(device_status),
+                                       _stream(stream)), "dirotq_linear_noalloc")
