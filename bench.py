@@ -165,6 +165,7 @@ def run_ours(args):
     import torch
     from paper_2605_16732_b200 import binding as dq
     from paper_2605_16732_b200 import synth
+    from paper_2605_16732_b200.shard import aggregate_throughput, max_over_ranks
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -221,11 +222,7 @@ def run_ours(args):
         step()
     e1.record()
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dev)
     ms_step = ms_total / args.steps
 
     # ---- per-kernel durations over the same steps (events on the launching stream)
@@ -286,11 +283,7 @@ def run_ours(args):
             e2e_step()
         e1.record()
         barrier()
-        e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, dev)
     h2d = sum(M * L["K"] * 2 for L in layers)
     d2h = sum(M * L["N"] * 2 for L in layers)
 
@@ -300,7 +293,7 @@ def run_ours(args):
         return
 
     ops_step = _shape_ops(M)
-    value = world * ops_step / (ms_step * 1e-3) / 1e12
+    value = aggregate_throughput(ops_step, ms_step, world) / 1e12
 
     # ---- roofline of the dominant kernel: the rotation GEMM (bf16 tensor cores)
     rot_ms = {n: float(np.mean(v["rotate_ms"])) for n, v in per.items()}

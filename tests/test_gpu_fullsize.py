@@ -1,0 +1,119 @@
+"""Parity at the full sizes of the task's configurations, in the launch configuration bench.py times
+(persistent 148-CTA grids, many tiles per CTA), on sampled outputs the oracle can compute one by one.
+
+Token rows are independent (per-token scales, row-wise GEMM) and so are output columns of the weight
+side, hence comparing a seeded sample of rows x columns is exact, not approximate.  Per case:
+  * prepared weights (codes, scales, bf16 rows) of the sampled columns, and the whole bf16 rotation,
+    against the oracle's fold + quantizer;
+  * activation codes / scales / bf16 coefficients of the sampled rows against the oracle's
+    rotation + quantizer (tolerated: +-1 code at a rounding boundary, neighbouring bf16 scale at a
+    boundary, see parity_utils);
+  * int32 group sums of a 128-row slice on the sampled columns, bit exact;
+  * the bf16 output of the sampled rows x columns.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dirotq_oracle as orc
+from paper_2605_16732_b200 import binding as dq
+from paper_2605_16732_b200 import synth
+
+from parity_utils import (bf16_tensor_to_bits, bits_to_bf16_tensor, check_activation_side, check_layer_output)
+
+pytestmark = pytest.mark.gpu
+
+_ROT = {}
+
+
+def _rotation(spec):
+    key = (spec.K, spec.r, spec.model.name, spec.seed)
+    if key not in _ROT:
+        _ROT.clear()  # keep at most one K x K fp64 matrix alive
+        _ROT[key] = synth.make_rotation(spec, device="cuda")
+    return _ROT[key]
+
+
+def _run(M, K, N, r, G, model, n_rows=24, n_cols=96, seed=0):
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=model, seed=seed)
+    Q = _rotation(spec)
+    W, bias = synth.make_weights(spec)
+    x_bits = synth.make_tokens(spec, M, batch_seed=3)
+    g = np.random.default_rng(K * 7 + N)
+    rows = np.sort(g.choice(M, size=min(n_rows, M), replace=False))
+    rows[-1] = M - 1  # always include the last row of the ragged last token block
+    cols = np.sort(g.choice(N, size=n_cols, replace=False))
+    cols[-1] = N - 1
+
+    # ---- oracle on the sample
+    lo = orc.prepare_layer(W[:, cols], Q, r, G, want_t=True)
+    bias_s = bias[cols]
+    oo = orc.linear_deployed(x_bits[rows], lo, bias=bias_s)
+
+    # ---- library on everything
+    Qd = torch.from_numpy(Q).cuda()
+    layer = dq.dirotq_prepare_layer(torch.from_numpy(W).cuda(), Qd, r, G, bias=bits_to_bf16_tensor(bias))
+    del Qd
+    wcodes, wscales, wh, qb = dq.dirotq_layer_export(layer)
+    assert np.array_equal(bf16_tensor_to_bits(qb), lo["Qb"]), "bf16 rotation differs"
+    del qb
+    cols_t = torch.from_numpy(cols).cuda()
+    assert np.array_equal(bf16_tensor_to_bits(wscales[:, cols_t]), lo["wscales"])
+    assert np.array_equal(bf16_tensor_to_bits(wh[:, cols_t]), lo["Wh"])
+    wc = wcodes[:, cols_t].cpu().numpy()
+    bad = wc != lo["wcodes"]
+    assert bad.sum() <= 2 and np.all(np.abs(np.abs(lo["wt"][bad] - np.floor(lo["wt"][bad])) - 0.5) < 1e-9)
+    del wcodes, wscales, wh
+
+    x = bits_to_bf16_tensor(x_bits)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = dq.alloc_workspace(layer, M)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, scales = dq.dirotq_workspace_export(layer, M, ws)
+    rows_t = torch.from_numpy(rows).cuda()
+    xh_b = bf16_tensor_to_bits(xh[rows_t])
+    codes_n = codes[rows_t].cpu().numpy()
+    scales_b = bf16_tensor_to_bits(scales[rows_t])
+    stats = check_activation_side(None, xh_b, codes_n, scales_b, oo, r, G)
+    y_s = bf16_tensor_to_bits(y[rows_t][:, cols_t])
+    stats.update(check_layer_output(y_s, xh_b, codes_n, scales_b, lo, oo, bias_s))
+
+    # ---- int32 group sums, bit exact, on a 128-row slice that spans a token-block boundary
+    m0 = max(0, min(M - 128, (M // 2) - 37))
+    msub = min(128, M)
+    sl = codes[m0:m0 + msub]
+    padded = torch.zeros((msub, layer.K_lp), dtype=torch.int8, device="cuda")
+    padded[:, :layer.K_l] = sl
+    ws2 = dq.alloc_workspace(layer, msub)
+    P = dq.dirotq_int_gemm_debug(padded, layer, ws2)
+    assert dq.dirotq_workspace_status(ws2) == 0
+    P_ref = orc.int_gemm(sl.cpu().numpy(), lo["wcodes"], G)
+    assert np.array_equal(P[:, :, cols_t].cpu().numpy(), P_ref), "int32 group sums differ"
+    layer.close()
+    return stats
+
+
+# config 3: FLUX.1-dev-shaped linears at M = 4608 (the benchmark's workload)
+@pytest.mark.parametrize("K,N", [(3072, 9216), (3072, 3072), (3072, 12288), (12288, 3072)])
+def test_config3_flux_linears(K, N):
+    print(_run(4608, K, N, 32, 64, synth.FLUX))
+
+
+# config 2: PixArt-Sigma-shaped block linears at M = 4096
+@pytest.mark.parametrize("K,N", [(1152, 1152), (1152, 4608), (4608, 1152)])
+def test_config2_pixart_linears(K, N):
+    print(_run(4096, K, N, 32, 64, synth.PIXART))
+
+
+# config 4: batch 4 (M = 18432), rank and group sweep (a subset that covers every r and both G)
+@pytest.mark.parametrize("K,N,r,G", [(3072, 9216, 16, 64), (3072, 9216, 64, 128), (3072, 9216, 128, 64),
+                                     (12288, 3072, 128, 128)])
+def test_config4_rank_group_sweep(K, N, r, G):
+    print(_run(18432, K, N, r, G, synth.FLUX))
+
+
+# config 5: the two single-stream shapes that the other configs do not contain
+@pytest.mark.parametrize("K,N", [(3072, 21504), (15360, 3072)])
+def test_config5_single_stream_shapes(K, N):
+    print(_run(4608, K, N, 32, 64, synth.FLUX))
