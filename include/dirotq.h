@@ -127,6 +127,16 @@ DIROTQ_API dirotq_status_t dirotq_linear_host(const void* x_host, int M, const d
  * completed; otherwise the role that gave up.  Returns DIROTQ_ERR_DEVICE_TIMEOUT in that case. */
 DIROTQ_API dirotq_status_t dirotq_workspace_status(const void* workspace, dirotq_stream_t stream, int* device_code);
 
+/* Diagnostics: the W4A4 kernel sums, per role, the SM cycles spent blocked on each kind of barrier
+ * into 64-bit counters kept next to the status word.  Copies them out (SYNCHRONISES `stream`):
+ * out[0] TMA producer waiting for a free stage, [1] MMA issuer waiting for operands (TMA + unpack),
+ * [2] MMA issuer waiting for a free accumulator tile, [3] unpack warp waiting for TMA data,
+ * [4] first epilogue warp waiting for a finished accumulator tile, [5] same warp waiting for
+ * scales, [6] that warp's total cycles, [7] the MMA role's total cycles; all summed over CTAs
+ * and over the calls since the workspace was last zeroed.  No counterpart in the paper. */
+DIROTQ_API dirotq_status_t dirotq_workspace_wait_counters(const void* workspace, dirotq_stream_t stream,
+                                                          unsigned long long out[8]);
+
 /* ---- exports for parity checks ------------------------------------------------------------- */
 
 /* Runs only the first kernel (rotation, split, Eq. 1) and leaves its results in `workspace`.

@@ -25,7 +25,7 @@ EXPORTED = [
     "dirotq_status_string", "dirotq_version", "dirotq_last_error", "dirotq_layer_bytes",
     "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
-    "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
+    "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_wait_counters", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
 ]
 
@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_workspace_status.argtypes = [vp, vp, pi]
         L.dirotq_rotate_quantize.argtypes = [vp, i, vp, vp, sz, vp, vp]
         L.dirotq_w4a4_gemm.argtypes = [i, vp, vp, sz, vp, vp]
+        L.dirotq_workspace_wait_counters.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_ulonglong)]
         L.dirotq_workspace_export.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_int_gemm_debug.argtypes = [vp, i, vp, vp, vp, sz, vp]
         L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -192,6 +193,18 @@ def dirotq_rotate_quantize(x: torch.Tensor, layer: Layer, workspace: torch.Tenso
 def dirotq_w4a4_gemm(M: int, layer: Layer, workspace: torch.Tensor, y: torch.Tensor, stream=None) -> None:
     _check(lib().dirotq_w4a4_gemm(M, layer.handle, workspace.data_ptr(), workspace.numel(), y.data_ptr(),
                                   _stream(stream)), "dirotq_w4a4_gemm")
+
+
+WAIT_COUNTER_NAMES = ("producer_wait_stage", "mma_wait_operands", "mma_wait_accumulator", "unpack_wait_tma",
+                      "epilogue_wait_accumulator", "epilogue_wait_scales", "epilogue_total", "mma_role_total")
+
+
+def dirotq_workspace_wait_counters(workspace: torch.Tensor, stream=None) -> dict:
+    """Per-role blocked-cycle counters of the W4A4 kernel (summed over CTAs and calls since the workspace was zeroed)."""
+    out = (ctypes.c_ulonglong * 8)()
+    _check(lib().dirotq_workspace_wait_counters(workspace.data_ptr(), _stream(stream), out),
+           "dirotq_workspace_wait_counters")
+    return dict(zip(WAIT_COUNTER_NAMES, [int(v) for v in out]))
 
 
 def dirotq_workspace_export(layer: Layer, M: int, workspace: torch.Tensor, stream=None):

@@ -293,6 +293,16 @@ dirotq_status_t dirotq_workspace_status(const void* workspace, dirotq_stream_t s
     return code == 0 ? DIROTQ_OK : DIROTQ_ERR_DEVICE_TIMEOUT;
 }
 
+dirotq_status_t dirotq_workspace_wait_counters(const void* workspace, dirotq_stream_t stream, unsigned long long out[8]) {
+    if (!workspace || !out) return DIROTQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(out, static_cast<const char*>(workspace) + 8, 8 * sizeof(unsigned long long),
+                                    cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { set_error("wait counter read", e); return DIROTQ_ERR_CUDA; }
+    return DIROTQ_OK;
+}
+
 dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
                                         int8_t* codes, void* scales_bf16, dirotq_stream_t stream) {
     if (!valid_layer(layer) || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;

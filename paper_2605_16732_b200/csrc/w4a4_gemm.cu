@@ -51,6 +51,23 @@ struct GemmKernelParams {
     int* status;
 };
 
+// Wait accounting (diagnostics): cycles a role spends blocked on each kind of barrier are summed into
+// 64-bit counters that follow the status word in the workspace (8-byte slots 1..8, see WaitSlot).
+enum WaitSlot : int { WS_PROD_EMPTY = 1, WS_MMA_OPERANDS = 2, WS_MMA_TEMPTY = 3, WS_UNPACK_FULL = 4, WS_EPI_TFULL = 5,
+                      WS_EPI_SCALES = 6, WS_EPI_TOTAL = 7, WS_KERNEL = 8 };
+
+__device__ __forceinline__ bool timed_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                           long long& acc) {
+    const long long t0 = clock64();
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
+    acc += clock64() - t0;
+    return ok;
+}
+
+__device__ __forceinline__ void flush_wait(int* status, int slot, long long cycles) {
+    atomicAdd(reinterpret_cast<unsigned long long*>(status) + slot, static_cast<unsigned long long>(cycles));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -126,13 +143,14 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             // -------------------------------------------------------- TMA producer
             if (lane == 0) {
                 uint32_t it = 0, sc_it = 0;
+                long long w_empty = 0;
                 bool ok = true;
                 for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                     const int m0 = (tile % num_m_blocks) * BM;
                     const int n0 = (tile / num_m_blocks) * BN;
                     for (int kb = 0; kb < p.num_kb; ++kb, ++it, ++sc_it) {
                         const int s = it % STAGES;
-                        if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                        if (!timed_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER, w_empty)) { ok = false; break; }
                         const uint32_t st = smem_base + s * STAGE_BYTES;
                         mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
                         tma_load_2d(st, &tmap_codes, full_bar(s), kb * BKC, m0);
@@ -154,6 +172,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), lr * 64, n0);
                     }
                 }
+                flush_wait(p.status, WS_PROD_EMPTY, w_empty);
                 if (!ok) {
                     const uint32_t first = it > STAGES ? it - STAGES : 0;
                     for (uint32_t j = first; j < it; ++j) {
@@ -175,13 +194,15 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);
                 constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
                 uint32_t it = 0, git = 0;
+                long long w_ops = 0, w_tempty = 0;
+                const long long t_kernel = clock64();
                 bool ok = true;
                 for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                     for (int kb = 0; ok && kb < p.num_kb; ++kb, ++it) {
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1;
-                        if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
-                            !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                        if (!timed_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops) ||
+                            !timed_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
                         tc_fence_after_sync();
                         const uint32_t st = smem_base + s * STAGE_BYTES;
                         const uint64_t adesc = umma_desc_sw128(st);
@@ -189,7 +210,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         const int ng_here = min(GPK, p.n_g - kb * GPK);
                         for (int gi = 0; gi < ng_here; ++gi, ++git) {
                             const uint32_t b = git & 1;
-                            if (!mbar_wait(tempty_bar(b), ((git >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                            if (!timed_wait(tempty_bar(b), ((git >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA, w_tempty)) { ok = false; break; }
                             tc_fence_after_sync();
 #pragma unroll
                             for (int k = 0; k < MMA_PER_G; ++k) {
@@ -223,39 +244,43 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     umma_commit(tfull_bar(b));
                     ++git;
                 }
+                flush_wait(p.status, WS_MMA_OPERANDS, w_ops);
+                flush_wait(p.status, WS_MMA_TEMPTY, w_tempty);
+                flush_wait(p.status, WS_KERNEL, clock64() - t_kernel);
             }
         } else {
             // -------------------------------------------------------- INT4 -> INT8 unpack (warps 2, 3)
             const int u = threadIdx.x - 64;  // 0..63
             uint32_t it = 0;
+            long long w_full = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 const int items = p.num_kb + p.lr_chunks;
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
-                    ok = mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+                    ok = timed_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK, w_full);
                     ok = __any_sync(0xffffffffu, ok);
                     if (!ok) break;
                     if (i < p.num_kb) {
+                        // 16-byte piece idx = u + 64 j of the packed tile: row = idx/4 = u/4 + 16 j, piece c = u%4.
+                        // The swizzle phase row%8 = (u/4)%8 and the piece do not depend on j, so every address is
+                        // a per-thread base plus a compile-time offset.
                         uint8_t* st = smem_gen + s * STAGE_BYTES;
-                        const uint4* src = reinterpret_cast<const uint4*>(st + A_BYTES + BU_BYTES);
-                        uint8_t* dst = st + A_BYTES;
-#pragma unroll 4
+                        const uint4* src = reinterpret_cast<const uint4*>(st + A_BYTES + BU_BYTES) + u;
+                        const int c = u & 3, sw = (u >> 2) & 7;
+                        uint8_t* d0 = st + A_BYTES + (u >> 2) * 128 + (((2 * c) ^ sw) << 4);
+                        uint8_t* d1 = st + A_BYTES + (u >> 2) * 128 + (((2 * c + 1) ^ sw) << 4);
+#pragma unroll
                         for (int j = 0; j < (BN * 4) / 64; ++j) {
-                            const int idx = u + 64 * j;  // 16-byte piece of the packed tile: row = idx/4, piece = idx%4
-                            const int row = idx >> 2;
-                            const int c = idx & 3;
-                            const uint4 pk = src[idx];
+                            const uint4 pk = src[64 * j];
                             // low nibbles of a word are codes k..k+3, high nibbles k+4..k+7 (see prepare.cu)
                             uint4 o0, o1;
                             o0.x = (pk.x << 4) & 0xF0F0F0F0u; o0.y = pk.x & 0xF0F0F0F0u;
                             o0.z = (pk.y << 4) & 0xF0F0F0F0u; o0.w = pk.y & 0xF0F0F0F0u;
                             o1.x = (pk.z << 4) & 0xF0F0F0F0u; o1.y = pk.z & 0xF0F0F0F0u;
                             o1.z = (pk.w << 4) & 0xF0F0F0F0u; o1.w = pk.w & 0xF0F0F0F0u;
-                            uint8_t* drow = dst + row * 128;
-                            const int sw = row & 7;  // 128-byte swizzle: 16-byte chunk index ^ (row % 8)
-                            *reinterpret_cast<uint4*>(drow + (((2 * c) ^ sw) << 4)) = o0;
-                            *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ sw) << 4)) = o1;
+                            *reinterpret_cast<uint4*>(d0 + j * 2048) = o0;  // 16 rows of 128 bytes further down
+                            *reinterpret_cast<uint4*>(d1 + j * 2048) = o1;
                         }
                         fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core
                     }
@@ -263,6 +288,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     if (lane == 0) mbar_arrive(unp_bar(s));
                 }
             }
+            if (u == 0) flush_wait(p.status, WS_UNPACK_FULL, w_full);
         }
     } else {
         reg_alloc<208>();
@@ -271,6 +297,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         const int half = (warp - 4) >> 2;
         const int row_in_tile = q * 32 + lane;
         uint32_t git = 0, sc_it = 0;
+        long long w_tfull = 0, w_sc = 0;
+        const long long t_epi = clock64();
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             const int m0 = (tile % num_m_blocks) * BM;
@@ -283,7 +311,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
             for (int kb = 0; ok && kb < p.num_kb; ++kb, ++sc_it) {
                 const int slot = sc_it % SC_SLOTS;
-                ok = mbar_wait(scfull_bar(slot), (sc_it / SC_SLOTS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+                ok = timed_wait(scfull_bar(slot), (sc_it / SC_SLOTS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc);
                 ok = __any_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const float* s_sw = reinterpret_cast<const float*>(smem_gen + STAGES * STAGE_BYTES + slot * SC_BYTES);
@@ -291,7 +319,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 const int ng_here = min(GPK, p.n_g - kb * GPK);
                 for (int gi = 0; gi < ng_here; ++gi, ++git) {
                     const uint32_t b = git & 1;
-                    ok = mbar_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+                    ok = timed_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
                     ok = __any_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
@@ -342,7 +370,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             // rank-r branch: fp32 tile
             {
                 const uint32_t b = git & 1;
-                ok = mbar_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+                ok = timed_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
                 ok = __any_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -378,6 +406,11 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                 }
             }
+        }
+        if (warp == 4 && lane == 0) {
+            flush_wait(p.status, WS_EPI_TFULL, w_tfull);
+            flush_wait(p.status, WS_EPI_SCALES, w_sc);
+            flush_wait(p.status, WS_EPI_TOTAL, clock64() - t_epi);
         }
     }
 

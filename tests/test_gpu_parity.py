@@ -126,3 +126,19 @@ def test_argument_errors_on_device():
     assert L.dirotq_linear(x.data_ptr() + 2, 8, layer.handle, y.data_ptr(), ws.data_ptr(), ws.numel(), s) == 1
     assert L.dirotq_linear(x.data_ptr(), 0, layer.handle, y.data_ptr(), ws.data_ptr(), ws.numel(), s) == 1
     torch.cuda.synchronize()
+
+
+def test_wait_counters_are_reported():
+    spec = synth.LayerSpec(K=512, N=1024, r=32, G=64, model=synth.PIXART, seed=12, calib_tokens=512)
+    inp = synth.make_layer_inputs(spec, 700)
+    layer = dq.dirotq_prepare_layer(torch.from_numpy(inp["W"]).cuda(), torch.from_numpy(inp["Q"]).cuda(), spec.r, spec.G)
+    ws = dq.alloc_workspace(layer, 700)
+    x = bits_to_bf16_tensor(inp["x"])
+    y = torch.empty((700, spec.N), dtype=torch.bfloat16, device="cuda")
+    dq.dirotq_linear(x, layer, y, ws)
+    c = dq.dirotq_workspace_wait_counters(ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    assert c["mma_role_total"] > 0 and c["epilogue_total"] > 0
+    assert c["epilogue_wait_accumulator"] <= c["epilogue_total"]
+    assert c["mma_wait_operands"] + c["mma_wait_accumulator"] <= c["mma_role_total"]
+    layer.close()
