@@ -1,0 +1,176 @@
+"""Timing sweep over the task's other configurations (bench.py keeps to its one-line contract).
+
+    python -m paper_2605_16732_b200.suite [--configs 1,2,4,5] [--iters 20]
+
+Prints one JSON line per case: both kernels' device times (CUDA events), effective TOPS
+(2*M*N*K / time), the fraction of the composite roofline
+t_roof = 2*M*(K-r)*N / P_int8 + (2*M*K^2 + 2*M*r*N) / P_bf16, and cuBLAS bf16 (torch.matmul) on the
+same shape.  Config 5 is the chain of all 152 linears of one FLUX.1-dev-shaped denoising step,
+timed device-side end to end against the same chain of bf16 GEMMs.
+
+Run time does not depend on the rotation's values, so a seeded Householder reflection (dense,
+exactly orthogonal) stands in for the PCA rotation here; activations and weights come from the
+same seeded generator as everywhere else.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import binding as dq
+from . import synth
+
+
+def _peaks():
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p.get("bf16_tflops_sustained", p["bf16_tflops"]), p["hbm_gbs"], "measured"
+    return 1400.0, 6650.0, "fallback"
+
+
+def _bf(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _householder(K: int, seed: int) -> torch.Tensor:
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    v = torch.randn(K, dtype=torch.float64, device="cuda", generator=g)
+    v /= v.norm()
+    return torch.eye(K, dtype=torch.float64, device="cuda") - 2.0 * torch.outer(v, v)
+
+
+class Case:
+    def __init__(self, M, K, N, r, G, model):
+        self.M, self.K, self.N, self.r, self.G = M, K, N, r, G
+        spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=model, seed=7)
+        W, bias = synth.make_weights(spec)
+        self.layer = dq.dirotq_prepare_layer(torch.from_numpy(W).cuda(), _householder(K, K + r), r, G, bias=_bf(bias))
+        self.x = _bf(synth.make_tokens(spec, M, batch_seed=11))
+        self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        self.ws = dq.alloc_workspace(self.layer, M)
+        self.Wb = (torch.from_numpy(W).cuda()).to(torch.bfloat16)
+
+    def run(self):
+        dq.dirotq_linear(self.x, self.layer, self.y, self.ws)
+
+    def time_kernels(self, iters):
+        for _ in range(3):
+            self.run()
+        rot, gem = [], []
+        for _ in range(iters):
+            a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a.record()
+            dq.dirotq_rotate_quantize(self.x, self.layer, self.ws)
+            b.record()
+            dq.dirotq_w4a4_gemm(self.M, self.layer, self.ws, self.y)
+            c.record()
+            torch.cuda.synchronize()
+            rot.append(a.elapsed_time(b))
+            gem.append(b.elapsed_time(c))
+        assert dq.dirotq_workspace_status(self.ws) == 0
+        cb = []
+        for _ in range(3):
+            torch.matmul(self.x, self.Wb)
+        for _ in range(iters):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            torch.matmul(self.x, self.Wb)
+            b.record()
+            torch.cuda.synchronize()
+            cb.append(a.elapsed_time(b))
+        return float(np.median(rot)), float(np.median(gem)), float(np.median(cb))
+
+    def report(self, tag, iters, p_bf16, hbm):
+        rot, gem, cb = self.time_kernels(iters)
+        M, K, N, r, G = self.M, self.K, self.N, self.r, self.G
+        K_l = K - r
+        n_g = -(-K_l // G)
+        tot = rot + gem
+        p_i8 = 2.0 * p_bf16
+        t_roof = (2.0 * M * K_l * N / p_i8 + (2.0 * M * K * K + 2.0 * M * r * N) / p_bf16) / 1e12 * 1e3
+        bytes_alg = 2 * M * K + 2 * K * K + n_g * G * N / 2 + 4 * n_g * N + 2 * 64 * N + 2 * (M * n_g * G + 4 * M * n_g + 2 * M * 64) + 2 * M * N
+        line = {"config": tag, "M": M, "K": K, "N": N, "r": r, "group": G, "rotate_ms": rot, "gemm_ms": gem,
+                "effective_tops": 2.0 * M * N * K / (tot * 1e-3) / 1e12,
+                "frac_int8_peak": 2.0 * M * N * K / (tot * 1e-3) / 1e12 / p_i8,
+                "frac_of_composite_roofline": t_roof / tot,
+                "algorithmic_gbs": bytes_alg / (tot * 1e-3) / 1e9, "frac_hbm_peak": bytes_alg / (tot * 1e-3) / 1e9 / hbm,
+                "cublas_bf16_ms": cb, "speedup_vs_cublas_bf16": cb / tot}
+        print(json.dumps(line), flush=True)
+
+    def close(self):
+        self.layer.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="1,2,4,5")
+    ap.add_argument("--iters", type=int, default=20)
+    args = ap.parse_args()
+    todo = set(args.configs.split(","))
+    p_bf16, hbm, src = _peaks()
+    print(json.dumps({"peaks": {"bf16_tflops_sustained": p_bf16, "int8_tops": 2 * p_bf16, "hbm_gbs": hbm, "source": src}}), flush=True)
+
+    if "1" in todo:
+        c = Case(256, 1152, 1152, 32, 64, synth.PIXART)
+        c.report("1: PixArt attention projection, M=256", args.iters, p_bf16, hbm)
+        c.close()
+    if "2" in todo:
+        for K, N in [(1152, 1152), (1152, 4608), (4608, 1152)]:
+            c = Case(4096, K, N, 32, 64, synth.PIXART)
+            c.report("2: PixArt block linear, M=4096", args.iters, p_bf16, hbm)
+            c.close()
+    if "4" in todo:
+        for K, N in [(3072, 9216), (12288, 3072)]:
+            for r in (16, 32, 64, 128):
+                for G in (64, 128):
+                    c = Case(18432, K, N, r, G, synth.FLUX)
+                    c.report("4: FLUX batch 4 (M=18432) rank/group sweep", max(5, args.iters // 2), p_bf16, hbm)
+                    c.close()
+                    torch.cuda.empty_cache()
+    if "5" in todo:
+        M = 4608
+        shapes = {"qkv": (3072, 9216), "out": (3072, 3072), "mlp_up": (3072, 12288), "mlp_down": (12288, 3072),
+                  "single_in": (3072, 21504), "single_out": (15360, 3072)}
+        cases = {n: Case(M, K, N, 32, 64, synth.FLUX) for n, (K, N) in shapes.items()}
+        # 19 double-stream blocks (4 linears, both streams as one M = 4608 batch) + 38 single-stream blocks (2 linears)
+        chain = ["qkv", "out", "mlp_up", "mlp_down"] * 19 + ["single_in", "single_out"] * 38
+        assert len(chain) == 152
+
+        def run_ours():
+            for n in chain:
+                cases[n].run()
+
+        def run_cublas():
+            for n in chain:
+                torch.matmul(cases[n].x, cases[n].Wb)
+
+        res = {}
+        for name, fn in (("dirotq", run_ours), ("cublas_bf16", run_cublas)):
+            fn()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            res[name] = float(np.median(ts))
+        for c in cases.values():
+            assert dq.dirotq_workspace_status(c.ws) == 0
+        ops = sum(2.0 * M * shapes[n][0] * shapes[n][1] for n in chain)
+        print(json.dumps({"config": "5: one FLUX.1-dev-shaped denoising step, 152 linears, M=4608",
+                          "note": "one prepared layer per distinct shape is reused for every block of that shape",
+                          "dirotq_chain_ms": res["dirotq"], "cublas_bf16_chain_ms": res["cublas_bf16"],
+                          "effective_tops": ops / (res["dirotq"] * 1e-3) / 1e12,
+                          "speedup_vs_cublas_bf16": res["cublas_bf16"] / res["dirotq"]}), flush=True)
+
+
+if __name__ == "__main__":
+    main()
