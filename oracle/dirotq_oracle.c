@@ -239,3 +239,157 @@ int dq_num_threads(void) {
 #endif
     return n;
 }
+
+/* =====================================================================================
+ * NVFP4 variant (paper Sec. 5.1: "For 4-bit FP, we use NVFP4, which supports group size 16
+ * with FP8 scaling"; Sec. 3: a 4-bit float with 1 mantissa and 2 exponent bits has q_max = 6).
+ *
+ *   element format E2M1: sign, 2 exponent bits, 1 mantissa bit; magnitudes {0, .5, 1, 1.5, 2, 3, 4, 6}
+ *   block of 16 consecutive low-precision coefficients shares one FP8 E4M3 scale (used unsigned)
+ *   Q(X) = e2m1_rne(X / s) * s,   s = e4m3_rne(max|X| / 6 / 2^e) * 2^e          (Eq. 1 with z = 0)
+ *
+ * Reading where the paper is silent: NVFP4 is a two-level format; the second level here is one
+ * power-of-two scale 2^e per tensor, fixed offline (activations: from the calibration batch;
+ * weights: from the folded weight), chosen so that the largest block scale lands at <= 256 in
+ * E4M3 (max finite 448).  Rounding is to nearest, ties to the even code; the scale saturates at
+ * 448, the element at +-6.  "Parity unpinned" against the authors' implementation.
+ * ===================================================================================== */
+
+/* E4M3 (4 exponent bits, bias 7, 3 mantissa bits, no infinities, max finite 448), unsigned use. */
+double dq_e4m3_to_double(uint8_t b) {
+    int e = (b >> 3) & 0xF, m = b & 7;
+    double v = (e == 0) ? ldexp((double)m, -9) : ldexp(1.0 + m / 8.0, e - 7);
+    return (b & 0x80) ? -v : v;
+}
+
+/* Round a non-negative fp64 value to E4M3, nearest, ties to even, saturating at 448. */
+uint8_t dq_e4m3_round(double v) {
+    if (!(v > 0.0)) return 0;
+    if (v >= 448.0) return 0x7E;                       /* 1111 110 = 448 */
+    int e = ilogb(v);
+    if (e < -6) e = -6;                                /* subnormals: fixed quantum 2^-9 */
+    double quantum = ldexp(1.0, e - 3);
+    double m = rint(v / quantum);                      /* ties to even */
+    double r = m * quantum;
+    if (r >= 448.0) return 0x7E;
+    if (r == 0.0) return 0;
+    int er = ilogb(r);
+    if (er < -6) return (uint8_t)(int)(r / ldexp(1.0, -9));            /* subnormal: mantissa only */
+    int mant = (int)((r / ldexp(1.0, er) - 1.0) * 8.0);
+    return (uint8_t)(((er + 7) << 3) | mant);
+}
+
+static const double kE2M1[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+double dq_e2m1_to_double(uint8_t code) {
+    double v = kE2M1[code & 7];
+    return (code & 8) ? -v : v;
+}
+
+/* Nearest E2M1 value, ties to the even code (mantissa bit 0), saturating at 6. */
+uint8_t dq_e2m1_round(double t) {
+    uint8_t sign = (t < 0.0 || (t == 0.0 && signbit(t))) ? 8 : 0;
+    double a = fabs(t);
+    int best = 0;
+    double bd = fabs(a - kE2M1[0]);
+    for (int c = 1; c < 8; ++c) {
+        double d = fabs(a - kE2M1[c]);
+        if (d < bd || (d == bd && (c & 1) == 0)) { bd = d; best = c; }
+    }
+    return (uint8_t)(sign | best);
+}
+
+/* Exponent of the per-tensor power-of-two scale for a tensor whose absolute maximum is amax. */
+int dq_nvfp4_global_exponent(double amax) {
+    if (!(amax > 0.0)) return 0;
+    return (int)ceil(log2(amax / (6.0 * 256.0)));
+}
+
+/* One block (n <= 16 real elements).  Writes the E4M3 scale byte, the E2M1 codes and, if t != NULL,
+ * the pre-rounding quotients. */
+void dq_nvfp4_quantize_block(const double* v, int n, int64_t stride, int e_global, uint8_t* sf, uint8_t* codes,
+                             int64_t code_stride, double* t, int64_t t_stride) {
+    double a = 0.0;
+    for (int i = 0; i < n; ++i) {
+        double x = fabs(v[i * stride]);
+        if (x > a) a = x;
+    }
+    uint8_t sb = dq_e4m3_round(ldexp(a / 6.0, -e_global));
+    double s = ldexp(dq_e4m3_to_double(sb), e_global);
+    *sf = sb;
+    for (int i = 0; i < n; ++i) {
+        double ti = (s != 0.0) ? v[i * stride] / s : 0.0;
+        codes[i * code_stride] = (s != 0.0) ? dq_e2m1_round(ti) : 0;
+        if (t) t[i * t_stride] = ti;
+    }
+}
+
+/* Weights: rows < r -> bf16 Wh; rows >= r -> blocks of 16 along K per output column.
+ * wcodes[K_l,N] (E2M1 codes 0..15), wsf[ceil(K_l/16),N] (E4M3 bytes); returns the global exponent. */
+int dq_nvfp4_prepare_weights(const double* Wt, int K, int N, int r, uint16_t* Wh, uint8_t* wcodes, uint8_t* wsf,
+                             double* wt) {
+    int K_l = K - r;
+    int nb = (K_l + 15) / 16;
+    dq_round_bf16(Wt, Wh, (int64_t)r * N);
+    double amax = 0.0;
+    for (int64_t i = (int64_t)r * N; i < (int64_t)K * N; ++i) {
+        double x = fabs(Wt[i]);
+        if (x > amax) amax = x;
+    }
+    int e = dq_nvfp4_global_exponent(amax);
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int b = 0; b < nb; ++b) {
+            int j0 = b * 16;
+            int len = (j0 + 16 <= K_l) ? 16 : (K_l - j0);
+            dq_nvfp4_quantize_block(Wt + (int64_t)(r + j0) * N + n, len, N, e, wsf + (int64_t)b * N + n,
+                                    wcodes + (int64_t)j0 * N + n, N, wt ? wt + (int64_t)j0 * N + n : NULL, N);
+        }
+    }
+    return e;
+}
+
+/* Activations: xt[M,K] -> xh bf16 [M,r]; codes [M,K_l]; sf [M,ceil(K_l/16)]; t (optional) [M,K_l]. */
+void dq_nvfp4_split_quantize(const double* xt, int M, int K, int r, int e_global, uint16_t* xh, uint8_t* codes,
+                             uint8_t* sf, double* t) {
+    int K_l = K - r;
+    int nb = (K_l + 15) / 16;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const double* row = xt + (int64_t)m * K;
+        for (int i = 0; i < r; ++i) xh[(int64_t)m * r + i] = dq_double_to_bf16(row[i]);
+        for (int b = 0; b < nb; ++b) {
+            int j0 = b * 16;
+            int len = (j0 + 16 <= K_l) ? 16 : (K_l - j0);
+            dq_nvfp4_quantize_block(row + r + j0, len, 1, e_global, sf + (int64_t)m * nb + b,
+                                    codes + (int64_t)m * K_l + j0, 1, t ? t + (int64_t)m * K_l + j0 : NULL, 1);
+        }
+    }
+}
+
+/* y = sum_k (sfx 2^ex vx)(sfw 2^ew vw) + sum_{i<r} xh Wh + bias, fp64, then bf16. */
+void dq_nvfp4_combine(const uint8_t* xcodes, const uint8_t* xsf, int ex, const uint8_t* wcodes, const uint8_t* wsf,
+                      int ew, const uint16_t* xh, const uint16_t* Wh, const uint16_t* bias, int M, int N, int K_l,
+                      int r, double* y64, uint16_t* ybits) {
+    int nb = (K_l + 15) / 16;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int b = 0; b < nb; ++b) {
+                int j1 = (b * 16 + 16 <= K_l) ? b * 16 + 16 : K_l;
+                double part = 0.0;
+                for (int j = b * 16; j < j1; ++j)
+                    part += dq_e2m1_to_double(xcodes[(int64_t)m * K_l + j]) * dq_e2m1_to_double(wcodes[(int64_t)j * N + n]);
+                acc += part * dq_e4m3_to_double(xsf[(int64_t)m * nb + b]) * dq_e4m3_to_double(wsf[(int64_t)b * N + n]);
+            }
+            acc = ldexp(acc, ex + ew);
+            double lr = 0.0;
+            for (int i = 0; i < r; ++i)
+                lr += dq_bf16_to_double(xh[(int64_t)m * r + i]) * dq_bf16_to_double(Wh[(int64_t)i * N + n]);
+            double v = acc + lr + (bias ? dq_bf16_to_double(bias[n]) : 0.0);
+            if (y64) y64[(int64_t)m * N + n] = v;
+            ybits[(int64_t)m * N + n] = dq_double_to_bf16(v);
+        }
+    }
+}

@@ -47,6 +47,17 @@ def _load():
         _lib.dq_double_to_bf16.restype = ctypes.c_uint16
         _lib.dq_double_to_bf16.argtypes = [ctypes.c_double]
         _lib.dq_num_threads.restype = ctypes.c_int
+        _lib.dq_e4m3_to_double.restype = ctypes.c_double
+        _lib.dq_e4m3_to_double.argtypes = [ctypes.c_uint8]
+        _lib.dq_e4m3_round.restype = ctypes.c_uint8
+        _lib.dq_e4m3_round.argtypes = [ctypes.c_double]
+        _lib.dq_e2m1_to_double.restype = ctypes.c_double
+        _lib.dq_e2m1_to_double.argtypes = [ctypes.c_uint8]
+        _lib.dq_e2m1_round.restype = ctypes.c_uint8
+        _lib.dq_e2m1_round.argtypes = [ctypes.c_double]
+        _lib.dq_nvfp4_global_exponent.restype = ctypes.c_int
+        _lib.dq_nvfp4_global_exponent.argtypes = [ctypes.c_double]
+        _lib.dq_nvfp4_prepare_weights.restype = ctypes.c_int
     return _lib
 
 
@@ -209,3 +220,90 @@ def linear_ideal(x, Q, W, r: int):
     Wt = fold(Q, np.asarray(W, dtype=np.float64))
     xt = matmul(x, Q)
     return matmul(xt[:, :r], Wt[:r]) + matmul(xt[:, r:], Wt[r:])
+
+
+# ---------------------------------------------------------------------------------------------
+# NVFP4 variant (Sec. 5.1): E2M1 elements, blocks of 16 with an E4M3 scale, one power-of-two scale per tensor
+
+E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def e4m3_to_f64(b) -> np.ndarray:
+    b = np.asarray(b, dtype=np.uint8)
+    e = ((b >> 3) & 0xF).astype(np.int64)
+    m = (b & 7).astype(np.float64)
+    v = np.where(e == 0, np.ldexp(m, -9), np.ldexp(1.0 + m / 8.0, e - 7))
+    return np.where(b & 0x80, -v, v)
+
+
+def e2m1_to_f64(c) -> np.ndarray:
+    c = np.asarray(c, dtype=np.uint8)
+    v = E2M1_VALUES[c & 7]
+    return np.where(c & 8, -v, v)
+
+
+def nvfp4_global_exponent(amax: float) -> int:
+    return int(_load().dq_nvfp4_global_exponent(ctypes.c_double(float(amax))))
+
+
+def nvfp4_quantize_block(v, e_global: int):
+    v = _c(v, np.float64).ravel()
+    n = v.size
+    sf = ctypes.c_uint8(0)
+    codes = np.zeros(n, dtype=np.uint8)
+    t = np.zeros(n, dtype=np.float64)
+    _load().dq_nvfp4_quantize_block(_p(v), ctypes.c_int(n), ctypes.c_int64(1), ctypes.c_int(e_global), ctypes.byref(sf),
+                                    _p(codes), ctypes.c_int64(1), _p(t), ctypes.c_int64(1))
+    return int(sf.value), codes, t
+
+
+def nvfp4_prepare_layer(W, Q, r: int, want_t: bool = False):
+    Q = _c(Q, np.float64)
+    Wt = fold(Q, np.asarray(W, dtype=np.float64))
+    K, N = Wt.shape
+    K_l = K - r
+    nb = -(-K_l // 16)
+    Wh = np.empty((r, N), dtype=np.uint16)
+    wcodes = np.empty((K_l, N), dtype=np.uint8)
+    wsf = np.empty((nb, N), dtype=np.uint8)
+    wt = np.empty((K_l, N), dtype=np.float64) if want_t else None
+    ew = _load().dq_nvfp4_prepare_weights(_p(Wt), ctypes.c_int(K), ctypes.c_int(N), ctypes.c_int(r), _p(Wh), _p(wcodes),
+                                          _p(wsf), _p(wt))
+    return {"Wh": Wh, "wcodes": wcodes, "wsf": wsf, "ew": int(ew), "wt": wt, "Qb": bf16_round(Q), "r": r}
+
+
+def nvfp4_split_quantize(xt, r: int, ex: int, want_t: bool = True):
+    xt = _c(xt, np.float64)
+    M, K = xt.shape
+    K_l = K - r
+    nb = -(-K_l // 16)
+    xh = np.empty((M, r), dtype=np.uint16)
+    codes = np.empty((M, K_l), dtype=np.uint8)
+    sf = np.empty((M, nb), dtype=np.uint8)
+    t = np.empty((M, K_l), dtype=np.float64) if want_t else None
+    _load().dq_nvfp4_split_quantize(_p(xt), ctypes.c_int(M), ctypes.c_int(K), ctypes.c_int(r), ctypes.c_int(ex), _p(xh),
+                                    _p(codes), _p(sf), _p(t))
+    return {"xh": xh, "codes": codes, "sf": sf, "t": t}
+
+
+def nvfp4_combine(xcodes, xsf, ex: int, layer, xh, bias):
+    xcodes = _c(xcodes, np.uint8)
+    xsf = _c(xsf, np.uint8)
+    xh = _c(xh, np.uint16)
+    M, K_l = xcodes.shape
+    N = layer["wcodes"].shape[1]
+    r = xh.shape[1]
+    bias = None if bias is None else _c(bias, np.uint16)
+    y64 = np.empty((M, N), dtype=np.float64)
+    yb = np.empty((M, N), dtype=np.uint16)
+    _load().dq_nvfp4_combine(_p(xcodes), _p(xsf), ctypes.c_int(ex), _p(_c(layer["wcodes"], np.uint8)),
+                             _p(_c(layer["wsf"], np.uint8)), ctypes.c_int(layer["ew"]), _p(xh), _p(_c(layer["Wh"], np.uint16)),
+                             _p(bias), ctypes.c_int(M), ctypes.c_int(N), ctypes.c_int(K_l), ctypes.c_int(r), _p(y64), _p(yb))
+    return y64, yb
+
+
+def nvfp4_linear_deployed(x_bits, layer, ex: int, bias=None, want_t: bool = True):
+    xt = rotate(x_bits, layer["Qb"])
+    sq = nvfp4_split_quantize(xt, layer["r"], ex, want_t=want_t)
+    y64, yb = nvfp4_combine(sq["codes"], sq["sf"], ex, layer, sq["xh"], bias)
+    return {"xt": xt, "xh": sq["xh"], "codes": sq["codes"], "sf": sq["sf"], "t": sq["t"], "y64": y64, "y": yb}
