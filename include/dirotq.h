@@ -168,6 +168,39 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,
                                     void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
 
+/* ---- NVFP4 variant (paper Sec. 5.1: "For 4-bit FP, we use NVFP4 ... group size 16 with FP8 scaling") ---- */
+
+/* Same layer with the 4-bit float format instead of INT4: elements are E2M1 (1 sign, 2 exponent,
+ * 1 mantissa bit: q_max = 6, Sec. 3), every block of 16 consecutive low-precision coefficients
+ * shares an FP8 E4M3 scale, and each tensor has one power-of-two scale 2^e (the second level of
+ * the NVFP4 format; the paper does not say how it is chosen):
+ *     Q(X) = e2m1_rne(X / s) * s,   s = e4m3_rne(max|X| / 6 / 2^e) * 2^e.
+ * The weights' exponent is derived inside prepare from the folded weight (largest block scale
+ * <= 256); the activations' exponent `act_scale_log2` is a calibration constant supplied by the
+ * caller (ceil(log2(max|x~_l| / 1536)) over the calibration batch).  Blocks are counted from the
+ * first low-precision coefficient.  The block scales are applied inside the tensor core
+ * (tcgen05.mma kind::mxf4nvf4), so the second kernel has no per-group pass.
+ * dirotq_workspace_bytes, dirotq_linear, dirotq_linear_host, dirotq_linear_noalloc,
+ * dirotq_rotate_quantize, dirotq_w4a4_gemm, dirotq_workspace_status and dirotq_layer_destroy accept
+ * such a layer; the INT4 exports and dirotq_int_gemm_debug do not.  Shapes as for INT4 (group ignored). */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes_nvfp4(int K, int N, int r, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_nvfp4(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                                      const void* bias, int K, int N, int r, int act_scale_log2, void* blob,
+                                                      size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                                      dirotq_stream_t stream, dirotq_layer_t** layer_out);
+
+/* Parity exports of the NVFP4 variant.  codes: one E2M1 code per byte (bit 3 = sign, bits 2..0 index
+ * into {0, .5, 1, 1.5, 2, 3, 4, 6}); scales: E4M3 bytes.  Activations: xh bf16 [M,r], codes [M,K-r],
+ * scales [M,ceil((K-r)/16)].  Weights: wcodes [K-r,N], wscales [ceil((K-r)/16),N], wh bf16 [r,N]
+ * (true values, the internal power-of-two pre-scale undone), q_bf16 [K,K], *weight_scale_log2
+ * (DEVICE int) = exponent of the weights' per-tensor scale.  Any pointer may be NULL. */
+DIROTQ_API dirotq_status_t dirotq_workspace_export_nvfp4(const dirotq_layer_t* layer, int M, const void* workspace,
+                                                         void* xh_bf16, uint8_t* codes, uint8_t* scales_e4m3,
+                                                         dirotq_stream_t stream);
+DIROTQ_API dirotq_status_t dirotq_layer_export_nvfp4(const dirotq_layer_t* layer, uint8_t* wcodes, uint8_t* wscales_e4m3,
+                                                     void* wh_bf16, void* q_bf16, int* weight_scale_log2,
+                                                     dirotq_stream_t stream);
+
 /* ---- for callers that cannot allocate (no counterpart in the paper) ------------------------- */
 
 /* dirotq_linear without a workspace argument.  Meant for callers that are not allowed to call

@@ -27,6 +27,7 @@ EXPORTED = [
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_wait_counters", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
+    "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
 ]
 
 
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
         L.dirotq_linear_noalloc.argtypes = [vp, i, vp, vp, vp, vp]
         L.dirotq_mma_rate_probe.argtypes = [i, i, vp, ctypes.POINTER(ctypes.c_float), vp]
+        L.dirotq_layer_bytes_nvfp4.argtypes = [i, i, i, psz]
+        L.dirotq_prepare_layer_nvfp4.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
+        L.dirotq_workspace_export_nvfp4.argtypes = [vp, i, vp, vp, vp, vp, vp]
+        L.dirotq_layer_export_nvfp4.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         for name in EXPORTED:
             if name not in ("dirotq_status_string", "dirotq_version", "dirotq_last_error"):
                 getattr(L, name).restype = i
@@ -105,9 +110,10 @@ def dirotq_prepare_scratch_bytes(K: int, N: int) -> int:
 class Layer:
     """Owner of one prepared layer: the device blob (a torch uint8 tensor) and the host handle."""
 
-    def __init__(self, handle: int, blob: torch.Tensor, K: int, N: int, r: int, group: int):
+    def __init__(self, handle: int, blob: torch.Tensor, K: int, N: int, r: int, group: int, fmt: str = "int4"):
         self.handle, self.blob = handle, blob
         self.K, self.N, self.r, self.group = K, N, r, group
+        self.fmt = fmt
         self.K_l = K - r
         self.n_g = -(-self.K_l // group)
         self.K_lp = self.n_g * group
@@ -256,3 +262,55 @@ def dirotq_linear_noalloc(x: torch.Tensor, layer: Layer, y: torch.Tensor, device
     device_status: optional cuda int32 tensor (1 element) that receives this call's device status word."""
     _check(lib().dirotq_linear_noalloc(x.data_ptr(), x.shape[0], layer.handle, y.data_ptr(), _ptr(device_status),
                                        _stream(stream)), "dirotq_linear_noalloc")
+
+
+# ------------------------------------------------------------------ NVFP4 variant
+
+def dirotq_layer_bytes_nvfp4(K: int, N: int, r: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_layer_bytes_nvfp4(K, N, r, ctypes.byref(out)), "dirotq_layer_bytes_nvfp4")
+    return out.value
+
+
+def dirotq_prepare_layer_nvfp4(W: torch.Tensor, Q: torch.Tensor, r: int, act_scale_log2: int,
+                               bias: torch.Tensor | None = None, w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """As dirotq_prepare_layer, for the NVFP4 format; act_scale_log2 is the activations' calibrated exponent."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    blob = _alloc_bytes(dirotq_layer_bytes_nvfp4(K, N, r), W.device, zero=True)
+    scratch_bytes = dirotq_prepare_scratch_bytes(K, N)
+    scratch = _alloc_bytes(scratch_bytes, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_nvfp4(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), K, N, r,
+                                          int(act_scale_log2), blob.data_ptr(), blob.numel(), scratch.data_ptr(),
+                                          scratch_bytes, _stream(stream), ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_nvfp4")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, 16, fmt="nvfp4")
+
+
+def dirotq_workspace_export_nvfp4(layer: Layer, M: int, workspace: torch.Tensor, stream=None):
+    dev = workspace.device
+    nb = -(-layer.K_l // 16)
+    xh = torch.empty((M, layer.r), dtype=torch.bfloat16, device=dev)
+    codes = torch.empty((M, layer.K_l), dtype=torch.uint8, device=dev)
+    scales = torch.empty((M, nb), dtype=torch.uint8, device=dev)
+    _check(lib().dirotq_workspace_export_nvfp4(layer.handle, M, workspace.data_ptr(), xh.data_ptr(), codes.data_ptr(),
+                                               scales.data_ptr(), _stream(stream)), "dirotq_workspace_export_nvfp4")
+    return xh, codes, scales
+
+
+def dirotq_layer_export_nvfp4(layer: Layer, stream=None):
+    dev = layer.blob.device
+    nb = -(-layer.K_l // 16)
+    wcodes = torch.empty((layer.K_l, layer.N), dtype=torch.uint8, device=dev)
+    wscales = torch.empty((nb, layer.N), dtype=torch.uint8, device=dev)
+    wh = torch.empty((layer.r, layer.N), dtype=torch.bfloat16, device=dev)
+    qb = torch.empty((layer.K, layer.K), dtype=torch.bfloat16, device=dev)
+    ew = torch.zeros(1, dtype=torch.int32, device=dev)
+    _check(lib().dirotq_layer_export_nvfp4(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(),
+                                           qb.data_ptr(), ew.data_ptr(), _stream(stream)), "dirotq_layer_export_nvfp4")
+    return wcodes, wscales, wh, qb, int(ew.item())

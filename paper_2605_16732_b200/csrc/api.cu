@@ -131,7 +131,7 @@ dirotq_status_t dirotq_prepare_scratch_bytes(int K, int N, size_t* bytes) {
 
 dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_t* bytes) {
     if (!valid_layer(layer) || !bytes || M < 1) return DIROTQ_ERR_INVALID_ARG;
-    *bytes = make_workspace_layout(layer->geo, M).total;
+    *bytes = layer->geo.fmt == 1 ? make_workspace_layout_nvfp4(layer->geo, M).total : make_workspace_layout(layer->geo, M).total;
     return DIROTQ_OK;
 }
 
@@ -207,12 +207,15 @@ dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K, int* N, i
 static dirotq_status_t check_call(const dirotq_layer_t* layer, int M, const void* workspace, size_t workspace_bytes) {
     if (!valid_layer(layer) || !workspace || M < 1) return DIROTQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
-    if (workspace_bytes < make_workspace_layout(layer->geo, M).total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    const size_t need = layer->geo.fmt == 1 ? make_workspace_layout_nvfp4(layer->geo, M).total
+                                            : make_workspace_layout(layer->geo, M).total;
+    if (workspace_bytes < need) return DIROTQ_ERR_BUFFER_TOO_SMALL;
     return DIROTQ_OK;
 }
 
 static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M, char* ws, float* xrot) {
-    const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
+    const bool nv = layer->geo.fmt == 1;
+    const WorkspaceLayout w = nv ? make_workspace_layout_nvfp4(layer->geo, M) : make_workspace_layout(layer->geo, M);
     RotateArgs a;
     a.x = x; a.M = M;
     a.codes = reinterpret_cast<int8_t*>(ws + w.off_codes);
@@ -221,7 +224,21 @@ static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M,
     a.xh = reinterpret_cast<uint16_t*>(ws + w.off_xh);
     a.xrot = xrot;
     a.status = reinterpret_cast<int*>(ws + w.off_status);
+    a.xsf = nv ? reinterpret_cast<uint8_t*>(ws + w.off_xscale) : nullptr;
     return a;
+}
+
+static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateArgs& ra, int M, void* y, cudaStream_t s) {
+    if (layer->geo.fmt == 1) {
+        Nvfp4GemmArgs na;
+        na.M = M; na.codes = reinterpret_cast<const uint8_t*>(ra.codes); na.xsf = ra.xsf; na.xh = ra.xh;
+        na.y = static_cast<uint16_t*>(y); na.status = ra.status;
+        return launch_nvfp4_gemm(layer, na, s);
+    }
+    GemmArgs ga;
+    ga.M = M; ga.codes = ra.codes; ga.xscale = ra.xscale; ga.ldm = ra.ldm; ga.xh = ra.xh;
+    ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr; ga.status = ra.status;
+    return launch_w4a4_gemm(layer, ga, s);
 }
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
@@ -242,10 +259,7 @@ dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer,
     const RotateArgs ra = rotate_args(layer, x, M, ws, nullptr);
     st = launch_rotate_quantize(layer, ra, static_cast<cudaStream_t>(stream));
     if (st != DIROTQ_OK) return st;
-    GemmArgs ga;
-    ga.M = M; ga.codes = ra.codes; ga.xscale = ra.xscale; ga.ldm = ra.ldm; ga.xh = ra.xh;
-    ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr; ga.status = ra.status;
-    return launch_w4a4_gemm(layer, ga, static_cast<cudaStream_t>(stream));
+    return second_kernel(layer, ra, M, y, static_cast<cudaStream_t>(stream));
 }
 
 dirotq_status_t dirotq_w4a4_gemm(int M, const dirotq_layer_t* layer, const void* workspace, size_t workspace_bytes,
@@ -254,16 +268,8 @@ dirotq_status_t dirotq_w4a4_gemm(int M, const dirotq_layer_t* layer, const void*
     if (st != DIROTQ_OK) return st;
     if (!y || !aligned16(y)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = const_cast<char*>(static_cast<const char*>(workspace));
-    const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
-    GemmArgs ga;
-    ga.M = M;
-    ga.codes = reinterpret_cast<const int8_t*>(ws + w.off_codes);
-    ga.xscale = reinterpret_cast<const float*>(ws + w.off_xscale);
-    ga.ldm = w.ldm;
-    ga.xh = reinterpret_cast<const uint16_t*>(ws + w.off_xh);
-    ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr;
-    ga.status = reinterpret_cast<int*>(ws + w.off_status);
-    return launch_w4a4_gemm(layer, ga, static_cast<cudaStream_t>(stream));
+    const RotateArgs ra = rotate_args(layer, nullptr, M, ws, nullptr);
+    return second_kernel(layer, ra, M, y, static_cast<cudaStream_t>(stream));
 }
 
 dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer_t* layer, void* y_host, void* x_dev,
@@ -305,7 +311,7 @@ dirotq_status_t dirotq_workspace_wait_counters(const void* workspace, dirotq_str
 
 dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
                                         int8_t* codes, void* scales_bf16, dirotq_stream_t stream) {
-    if (!valid_layer(layer) || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
+    if (!valid_layer(layer) || layer->geo.fmt != 0 || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
     return launch_workspace_export(layer, M, static_cast<const char*>(workspace), static_cast<uint16_t*>(xh_bf16), codes,
                                    static_cast<uint16_t*>(scales_bf16), static_cast<cudaStream_t>(stream));
 }
@@ -314,6 +320,7 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
                                       void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
     dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
     if (st != DIROTQ_OK) return st;
+    if (layer->geo.fmt != 0) return DIROTQ_ERR_INVALID_ARG;
     if (!act_codes || !partials || !aligned16(act_codes) || !aligned16(partials)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = static_cast<char*>(workspace);
     const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
@@ -329,9 +336,82 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
 
 dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16, void* wh_bf16,
                                     void* q_bf16, dirotq_stream_t stream) {
-    if (!valid_layer(layer)) return DIROTQ_ERR_INVALID_ARG;
+    if (!valid_layer(layer) || layer->geo.fmt != 0) return DIROTQ_ERR_INVALID_ARG;
     return launch_layer_export(layer, wcodes, static_cast<uint16_t*>(wscales_bf16), static_cast<uint16_t*>(wh_bf16),
                                static_cast<uint16_t*>(q_bf16), static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------- NVFP4 variant
+
+dirotq_status_t dirotq_layer_bytes_nvfp4(int K, int N, int r, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, 64);
+    if (st != DIROTQ_OK) return st;
+    *bytes = make_blob_layout_nvfp4(make_geometry(K, N, r, 64)).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_nvfp4(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                           const void* bias, int K, int N, int r, int act_scale_log2, void* blob,
+                                           size_t blob_bytes, void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                           dirotq_layer_t** layer_out) {
+    if (!W || !Q || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
+    if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
+    if (q_dtype != DIROTQ_DTYPE_F64 && q_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
+    if (w_layout != DIROTQ_LAYOUT_KN && w_layout != DIROTQ_LAYOUT_NK) return DIROTQ_ERR_INVALID_ARG;
+    if (act_scale_log2 < -100 || act_scale_log2 > 100) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, 64);
+    if (st != DIROTQ_OK) return st;
+    if (!aligned16(W) || !aligned16(Q) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
+    Geometry g = make_geometry(K, N, r, 64);
+    g.fmt = 1;
+    const BlobLayout lay = make_blob_layout_nvfp4(g);
+    if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (scratch_bytes < static_cast<size_t>(K) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    int dev = 0;
+    st = check_device(&dev);
+    if (st != DIROTQ_OK) return st;
+    dirotq_layer* L = new (std::nothrow) dirotq_layer;
+    if (!L) return DIROTQ_ERR_INVALID_ARG;
+    memset(L, 0, sizeof *L);
+    L->magic = kLayerMagic;
+    L->device = dev;
+    L->geo = g;
+    L->lay = lay;
+    L->blob = static_cast<char*>(blob);
+    L->act_scale_log2 = act_scale_log2;
+    st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                        (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked, (uint64_t)g.K4 / 2,
+                            (uint64_t)N, (uint64_t)g.K4 / 2, 128, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = launch_prepare_nvfp4(L, W, w_dtype, w_layout, Q, q_dtype, bias, static_cast<double*>(scratch),
+                                  static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) {
+        delete L;
+        return st;
+    }
+    *layer_out = L;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_workspace_export_nvfp4(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
+                                              uint8_t* codes, uint8_t* scales_e4m3, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || layer->geo.fmt != 1 || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
+    return launch_workspace_export_nvfp4(layer, M, static_cast<const char*>(workspace), static_cast<uint16_t*>(xh_bf16), codes,
+                                         scales_e4m3, static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_layer_export_nvfp4(const dirotq_layer_t* layer, uint8_t* wcodes, uint8_t* wscales_e4m3, void* wh_bf16,
+                                          void* q_bf16, int* weight_scale_log2, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || layer->geo.fmt != 1) return DIROTQ_ERR_INVALID_ARG;
+    return launch_layer_export_nvfp4(layer, wcodes, wscales_e4m3, static_cast<uint16_t*>(wh_bf16),
+                                     static_cast<uint16_t*>(q_bf16), weight_scale_log2, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -21,6 +21,11 @@ struct Geometry {
     int n_g;    // ceil(K_l / G)
     int K_lp;   // n_g * G  (<= K)
     int r_pad;  // r rounded up to a multiple of 64 (bf16 low-rank operand width)
+    // NVFP4 variant only (fmt == 1): blocks of 16, MMA K = 64, TMA k-blocks of 256 elements
+    int fmt;     // 0 = INT4 groups with bf16 scales, 1 = NVFP4 (E2M1 elements, E4M3 block scales)
+    int K4;      // K_l rounded up to 64 (<= K): width of the packed E2M1 rows
+    int nkb64;   // K4 / 64: scale-factor atoms (128 rows x 4 scales) per row block
+    int nkb64p;  // nkb64 rounded up to 4: one TMA k-block = 256 elements = 4 atoms
 };
 
 inline Geometry make_geometry(int K, int N, int r, int G) {
@@ -30,6 +35,10 @@ inline Geometry make_geometry(int K, int N, int r, int G) {
     g.n_g = (g.K_l + G - 1) / G;
     g.K_lp = g.n_g * G;
     g.r_pad = (r + 63) / 64 * 64;
+    g.fmt = 0;
+    g.K4 = (g.K_l + 63) / 64 * 64;
+    g.nkb64 = g.K4 / 64;
+    g.nkb64p = (g.nkb64 + 3) / 4 * 4;
     return g;
 }
 
@@ -43,6 +52,9 @@ struct BlobLayout {
     size_t off_wscale;   // f32  [n_g][N]: bf16-valued group scales of the weight codes
     size_t off_wh;       // bf16 [N][r_pad]: high-precision rows of the folded weight, K-major, zero padded
     size_t off_bias;     // f32  [N]
+    // NVFP4 variant: off_wpacked = E2M1 codes u8 [N][K4/2] (even k in the low nibble); off_wscale = E4M3 scale
+    // atoms u8 [ceil(N/128)][nkb64p][512]; off_meta = {float out_scale = 2^(ex+ew), int ew, int ex, uint amax bits}
+    size_t off_meta;
     size_t total;
 };
 
@@ -54,6 +66,20 @@ inline BlobLayout make_blob_layout(const Geometry& g) {
     b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * g.N * 4);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
     b.off_bias = o;    o = align_up(o + (size_t)g.N * 4);
+    b.off_meta = o;    o = align_up(o + 64);
+    b.total = o;
+    return b;
+}
+
+inline BlobLayout make_blob_layout_nvfp4(const Geometry& g) {
+    BlobLayout b;
+    size_t o = 0;
+    b.off_qt = o;      o = align_up(o + (size_t)g.K * g.K * 2);
+    b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K4 / 2));
+    b.off_wscale = o;  o = align_up(o + (size_t)((g.N + 127) / 128) * g.nkb64p * 512);
+    b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
+    b.off_bias = o;    o = align_up(o + (size_t)g.N * 4);
+    b.off_meta = o;    o = align_up(o + 64);
     b.total = o;
     return b;
 }
@@ -65,6 +91,7 @@ struct WorkspaceLayout {
     size_t off_codes;   // i8  [M][K_lp]: activation codes, one per byte
     size_t off_xscale;  // f32 [n_g][ldm]: bf16-valued activation scales, group-major
     size_t off_xh;      // bf16 [M][r_pad]
+    // NVFP4 variant: off_codes = E2M1 codes u8 [M][K4/2]; off_xscale = E4M3 scale atoms u8 [ceil(M/128)][nkb64p][512]
     size_t total;
 };
 
@@ -75,6 +102,18 @@ inline WorkspaceLayout make_workspace_layout(const Geometry& g, int M) {
     w.off_status = o;  o = align_up(o + 256);
     w.off_codes = o;   o = align_up(o + (size_t)M * g.K_lp);
     w.off_xscale = o;  o = align_up(o + (size_t)g.n_g * w.ldm * 4);
+    w.off_xh = o;      o = align_up(o + (size_t)M * g.r_pad * 2);
+    w.total = o;
+    return w;
+}
+
+inline WorkspaceLayout make_workspace_layout_nvfp4(const Geometry& g, int M) {
+    WorkspaceLayout w;
+    w.ldm = 0;
+    size_t o = 0;
+    w.off_status = o;  o = align_up(o + 256);
+    w.off_codes = o;   o = align_up(o + (size_t)M * (g.K4 / 2));
+    w.off_xscale = o;  o = align_up(o + (size_t)((M + 127) / 128) * g.nkb64p * 512);
     w.off_xh = o;      o = align_up(o + (size_t)M * g.r_pad * 2);
     w.total = o;
     return w;
@@ -93,12 +132,14 @@ struct dirotq_layer {
     CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2], box 64 x kGemmBN, no swizzle
     CUtensorMap tmap_wscale;   // f32 [n_g][N], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
+    int act_scale_log2;        // NVFP4 variant: exponent of the activations' per-tensor power-of-two scale
 };
 
 namespace dirotq {
 
 constexpr uint32_t kLayerMagic = 0x44695251u;  // "DiRQ"
-constexpr int kGemmBN = 256;  // output columns per tile of the W4A4 kernel (rows of its weight-side TMA boxes)
+constexpr int kGemmBN = 256;
+constexpr int kNvfp4BN = 128;  // output columns per tile of the NVFP4 kernel  // output columns per tile of the W4A4 kernel (rows of its weight-side TMA boxes)
 
 // ------------------------------------------------------------------ kernel launch interfaces
 
@@ -111,6 +152,7 @@ struct RotateArgs {
     uint16_t* xh;
     float* xrot;  // optional fp32 [M][K], columns in the caller's (unpermuted) order
     int* status;
+    uint8_t* xsf = nullptr;  // NVFP4 variant: scale-factor atoms (codes then holds packed E2M1)
 };
 
 struct GemmArgs {
@@ -132,6 +174,21 @@ dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t 
 // launchers (each returns after enqueueing on `stream`)
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
 dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream);
+struct Nvfp4GemmArgs {
+    int M;
+    const uint8_t* codes;  // [M][K4/2]
+    const uint8_t* xsf;    // scale-factor atoms
+    const uint16_t* xh;    // bf16 [M][r_pad]
+    uint16_t* y;           // bf16 [M][N]
+    int* status;
+};
+dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a, cudaStream_t stream);
+dirotq_status_t launch_prepare_nvfp4(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
+                                     int q_dtype, const void* bias, double* scratch, cudaStream_t stream);
+dirotq_status_t launch_layer_export_nvfp4(const dirotq_layer* L, uint8_t* wcodes, uint8_t* wsf, uint16_t* wh, uint16_t* qb,
+                                          int* ew, cudaStream_t stream);
+dirotq_status_t launch_workspace_export_nvfp4(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
+                                              uint8_t* codes, uint8_t* sf, cudaStream_t stream);
 dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
                                int q_dtype, const void* bias, double* scratch, cudaStream_t stream);
 dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint16_t* wscales, uint16_t* wh,

@@ -1,0 +1,316 @@
+// NVFP4 variant of the second kernel (paper Sec. 5.1: 4-bit float elements, blocks of 16, FP8 scales).
+//
+//   y[m,n] = bf16( 2^(ex+ew) * D[m,n] + bias[n] ),
+//   D = sum over blocks of 16:  sf_x[m,blk] * sf_w[n,blk] * sum_{k in blk} v_x[m,k] v_w[n,k]   (E2M1 x E2M1)
+//       + sum_{i<r} x~_h[m,i] * (W~_h[i,n] * 2^-(ex+ew))                                        (bf16 x bf16)
+//
+// The block scales are applied INSIDE the tensor core (tcgen05.mma kind::mxf4nvf4, block16): there is
+// no per-group pass over the accumulator on the CUDA cores, which is what limits the INT4 kernel.
+// The two per-tensor scales are powers of two, so the bf16 rank-r weights can be pre-divided
+// exactly and the rank-r branch accumulates into the same fp32 tile (kind::f16 on the same TMEM
+// columns); the epilogue is one multiply-add per element.
+//
+// Data movement: packed E2M1 operands by TMA (128-byte rows = 256 elements, 128-byte swizzle); the
+// E4M3 scale factors travel as 512-byte atoms (128 rows x 4 scales, row r at (r%32)*16 + (r/32)*4),
+// fetched with cp.async.bulk and copied into tensor memory with tcgen05.cp.32x128b.warpx4 by the MMA
+// thread right before the four MMAs (K = 64 each) that consume them.
+//
+// Roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue.
+// TMEM: two 128-column fp32 accumulators (the epilogue of tile i overlaps the MMAs of tile i+1) and,
+// per pipeline stage, 16 + 16 columns of scale factors.
+#include "common.h"
+#include "ptx.cuh"
+
+#include <cuda_bf16.h>
+
+namespace dirotq {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = kNvfp4BN;  // 128
+constexpr int BKE = 256;      // E2M1 elements per k-block (128-byte rows)
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * 128;      // 16 KB
+constexpr int B_BYTES = BN * 128;      // 16 KB
+constexpr int SF_BYTES = 4 * 512;      // four atoms per operand and k-block
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 2 * SF_BYTES;  // 36 KB
+constexpr int NUM_THREADS = 192;
+constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+constexpr int TMEM_SF_BASE = 2 * BN;   // columns 256.. hold the scale factors: 32 per stage
+
+struct NvKernelParams {
+    int M, N, num_kb, nkb64p, lr_chunks;
+    const uint8_t* xsf;   // activation scale atoms [ceil(M/128)][nkb64p][512]
+    const uint8_t* wsf;   // weight scale atoms [ceil(N/128)][nkb64p][512]
+    const float* bias;
+    const float* out_scale;  // 2^(ex+ew)
+    uint16_t* y;
+    int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 1-D bulk copy global -> shared, completion counted in bytes on `bar` (16-byte aligned, size % 16 == 0).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Shared-memory descriptor of one scale-factor atom for tcgen05.cp: 32 rows of 16 bytes, no swizzle,
+// 8-row core matrices 128 bytes apart.
+__device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
+    d |= static_cast<uint64_t>(128 >> 4) << 16;  // leading byte offset (one 16-byte column only: not stepped over)
+    d |= static_cast<uint64_t>(128 >> 4) << 32;  // stride byte offset: next group of 8 rows
+    d |= static_cast<uint64_t>(1) << 46;         // descriptor version
+    return d;                                    // layout type 0: no swizzle
+}
+
+// 32 lanes x 128 bits from shared memory into 4 TMEM columns, replicated to the four lane quadrants.
+__device__ __forceinline__ void tmem_cp_32x128b_warpx4(uint32_t taddr, uint64_t desc) {
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+}
+
+// Block-scaled instruction descriptor: E2M1 x E2M1 -> fp32, UE4M3 scales, both operands K-major.
+__host__ __device__ constexpr uint32_t nvfp4_idesc(uint32_t M, uint32_t N) {
+    return (1u << 7) /*A: E2M1*/ | (1u << 10) /*B: E2M1*/ | ((N >> 3) << 17) | (0u << 23) /*scale format UE4M3*/ |
+           ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_nvfp4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t tsfa,
+                                           uint32_t tsfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wcodes,
+                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
+                  const NvKernelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t bar_base = smem_base + BAR_OFFSET;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 128);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 132);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_m_blocks = (p.M + BM - 1) / BM;
+    const int num_n_blocks = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m_blocks * num_n_blocks;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_codes);
+        tma_prefetch_desc(&tmap_wcodes);
+        tma_prefetch_desc(&tmap_xh);
+        tma_prefetch_desc(&tmap_wh);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m_blk = tile % num_m_blocks, n_blk = tile / num_m_blocks;
+                const int m0 = m_blk * BM, n0 = n_blk * BN;
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                    const uint32_t st = smem_base + s * STAGE_BYTES;
+                    mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+                    tma_load_2d(st, &tmap_codes, full_bar(s), kb * 128, m0);             // byte coordinates
+                    tma_load_2d(st + A_BYTES, &tmap_wcodes, full_bar(s), kb * 128, n0);
+                    bulk_load(st + A_BYTES + B_BYTES, p.xsf + (static_cast<size_t>(m_blk) * p.nkb64p + kb * 4) * 512, SF_BYTES,
+                              full_bar(s));
+                    bulk_load(st + A_BYTES + B_BYTES + SF_BYTES, p.wsf + (static_cast<size_t>(n_blk) * p.nkb64p + kb * 4) * 512,
+                              SF_BYTES, full_bar(s));
+                }
+                if (!ok) break;
+                for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                    const uint32_t st = smem_base + s * STAGE_BYTES;
+                    mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
+                    tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
+                    tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), lr * 64, n0);
+                }
+            }
+            if (!ok) {
+                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1) && globaltimer_ns() - t0 < 100000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_nv = nvfp4_idesc(BM, BN);
+            constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+                const uint32_t acc = tcount & 1;
+                if (!mbar_wait(tempty_bar(acc), ((tcount >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d = tmem_base + acc * BN;
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t st = smem_base + s * STAGE_BYTES;
+                    const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * 32;
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        tmem_cp_32x128b_warpx4(tsf + 4 * a, sf_desc(st + A_BYTES + B_BYTES + a * 512));
+                        tmem_cp_32x128b_warpx4(tsf + 16 + 4 * a, sf_desc(st + A_BYTES + B_BYTES + SF_BYTES + a * 512));
+                    }
+                    const uint64_t adesc = umma_desc_sw128(st);
+                    const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)  // K = 64 elements = 32 bytes per instruction
+                        umma_nvfp4(d, adesc + 2 * k, bdesc + 2 * k, idesc_nv, tsf + 4 * k, tsf + 16 + 4 * k, (kb | k) != 0);
+                    umma_commit(empty_bar(s));
+                }
+                if (!ok) break;
+                for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t st = smem_base + s * STAGE_BYTES;
+                    const uint64_t adesc = umma_desc_sw128(st);
+                    const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc_bf, 1u);
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(tfull_bar(acc));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;
+        uint32_t tcount = 0;
+        bool ok = true;
+        const float out_scale = __ldg(p.out_scale);
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            const int m0 = (tile % num_m_blocks) * BM;
+            const int n0 = (tile / num_m_blocks) * BN;
+            const uint32_t acc = tcount & 1;
+            ok = mbar_wait(tfull_bar(acc), (tcount >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+            ok = __any_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int row = m0 + q * 32 + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t raw[32];
+                tmem_ld_32x32b_x32(taddr + c * 32, raw);
+                tmem_ld_wait();
+                if (c == BN / 32 - 1) {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(acc));
+                }
+                const int col = n0 + c * 32;
+                if (row < p.M) {
+                    uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + col;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        if (col + j < p.N) {
+                            const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + col + j));
+                            const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + col + j + 4));
+                            uint4 o;
+                            o.x = pack_bf16x2(fmaf(__uint_as_float(raw[j + 0]), out_scale, b0.x), fmaf(__uint_as_float(raw[j + 1]), out_scale, b0.y));
+                            o.y = pack_bf16x2(fmaf(__uint_as_float(raw[j + 2]), out_scale, b0.z), fmaf(__uint_as_float(raw[j + 3]), out_scale, b0.w));
+                            o.z = pack_bf16x2(fmaf(__uint_as_float(raw[j + 4]), out_scale, b1.x), fmaf(__uint_as_float(raw[j + 5]), out_scale, b1.y));
+                            o.w = pack_bf16x2(fmaf(__uint_as_float(raw[j + 6]), out_scale, b1.z), fmaf(__uint_as_float(raw[j + 7]), out_scale, b1.w));
+                            *reinterpret_cast<uint4*>(yrow + j) = o;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace
+
+dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    CUtensorMap tmap_codes, tmap_xh;
+    dirotq_status_t st;
+    st = encode_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K4 / 2, (uint64_t)a.M,
+                        (uint64_t)g.K4 / 2, 128, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,
+                        (uint64_t)g.r_pad * 2, 64, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    NvKernelParams p;
+    p.M = a.M; p.N = g.N;
+    p.num_kb = (g.K4 + BKE - 1) / BKE;
+    p.nkb64p = g.nkb64p;
+    p.lr_chunks = g.r_pad / 64;
+    p.xsf = a.xsf;
+    p.wsf = reinterpret_cast<const uint8_t*>(L->blob + L->lay.off_wscale);
+    p.bias = reinterpret_cast<const float*>(L->blob + L->lay.off_bias);
+    p.out_scale = reinterpret_cast<const float*>(L->blob + L->lay.off_meta);
+    p.y = a.y; p.status = a.status;
+    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(nvfp4_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return DIROTQ_ERR_CUDA;
+        attr_set = true;
+    }
+    nvfp4_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace dirotq

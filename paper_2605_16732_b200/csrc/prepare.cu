@@ -198,6 +198,162 @@ __global__ void export_workspace_kernel(const int8_t* codes, const float* xscale
     }
 }
 
+// ================================================================ NVFP4 variant (paper Sec. 5.1)
+// E2M1 elements, blocks of 16 along K with an E4M3 scale, one power-of-two scale per tensor.
+// Everything offline is done in fp64 so that codes and scales equal the CPU checker's.
+
+// Non-negative fp64 -> E4M3 byte: nearest, ties to even, saturating at 448, subnormals kept.
+__device__ __forceinline__ uint8_t f64_to_e4m3(double v) {
+    if (!(v > 0.0)) return 0;
+    if (v >= 448.0) return 0x7E;
+    int e = ilogb(v);
+    if (e < -6) e = -6;
+    const double quantum = ldexp(1.0, e - 3);
+    const double r = rint(v / quantum) * quantum;
+    if (r >= 448.0) return 0x7E;
+    if (r == 0.0) return 0;
+    const int er = ilogb(r);
+    if (er < -6) return static_cast<uint8_t>(static_cast<int>(r * 512.0));
+    const int mant = static_cast<int>((r / ldexp(1.0, er) - 1.0) * 8.0);
+    return static_cast<uint8_t>(((er + 7) << 3) | mant);
+}
+
+__device__ __forceinline__ double e4m3_to_f64(uint8_t b) {
+    const int e = (b >> 3) & 0xF, m = b & 7;
+    return e == 0 ? ldexp(static_cast<double>(m), -9) : ldexp(1.0 + m / 8.0, e - 7);
+}
+
+// fp64 -> E2M1 code (bit 3 = sign): nearest of {0, .5, 1, 1.5, 2, 3, 4, 6}, ties to the even code, saturating.
+__device__ __forceinline__ uint8_t f64_to_e2m1(double t) {
+    const double vals[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+    const double a = fabs(t);
+    int best = 0;
+    double bd = a;
+    for (int c = 1; c < 8; ++c) {
+        const double d = fabs(a - vals[c]);
+        if (d < bd || (d == bd && (c & 1) == 0)) { bd = d; best = c; }
+    }
+    return static_cast<uint8_t>((t < 0.0 ? 8 : 0) | best);
+}
+
+struct Nvfp4Meta {
+    float out_scale;  // 2^(ex + ew): what the accumulator is multiplied by in the epilogue
+    int ew;           // exponent of the weights' per-tensor scale
+    int ex;           // exponent of the activations' per-tensor scale (argument of prepare)
+    int pad;
+    unsigned long long amax_bits;  // fp64 bit pattern of max |W~_l|
+};
+
+__global__ void nvfp4_amax_kernel(const double* Wt, Geometry g, Nvfp4Meta* meta) {
+    double a = 0.0;
+    const size_t lo = static_cast<size_t>(g.r) * g.N, hi = static_cast<size_t>(g.K) * g.N;
+    for (size_t i = lo + blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < hi;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x)
+        a = fmax(a, fabs(Wt[i]));
+    for (int o = 16; o > 0; o >>= 1) a = fmax(a, __shfl_xor_sync(0xffffffffu, a, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(&meta->amax_bits, static_cast<unsigned long long>(__double_as_longlong(a)));
+}
+
+__global__ void nvfp4_meta_kernel(Nvfp4Meta* meta, int ex) {
+    const double amax = __longlong_as_double(static_cast<long long>(meta->amax_bits));
+    int ew = 0;
+    if (amax > 0.0) {
+        // ceil(log2(amax / 1536)) without a logarithm: x = m 2^e, m in [0.5, 1)
+        int e;
+        const double m = frexp(amax / (6.0 * 256.0), &e);
+        ew = (m == 0.5) ? e - 1 : e;
+    }
+    meta->ew = ew;
+    meta->ex = ex;
+    meta->out_scale = static_cast<float>(ldexp(1.0, ex + ew));
+}
+
+// One thread per (output column n, 64-element slab kb): four blocks of 16.
+__global__ void nvfp4_quantize_weights_kernel(const double* Wt, uint8_t* wcodes, uint8_t* wsf, const Nvfp4Meta* meta,
+                                              Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int kb = blockIdx.y;
+    if (n >= g.N) return;
+    const int ew = meta->ew;
+    uint32_t sfword = 0;
+    uint8_t* crow = wcodes + static_cast<size_t>(n) * (g.K4 / 2) + kb * 32;
+    for (int b = 0; b < 4; ++b) {
+        const int j0 = kb * 64 + b * 16;
+        const int len = min(16, g.K_l - j0);
+        uint8_t codes[16];
+        uint8_t sb = 0;
+        if (len > 0) {
+            const double* col = Wt + static_cast<size_t>(g.r + j0) * g.N + n;
+            double a = 0.0;
+            for (int j = 0; j < len; ++j) a = fmax(a, fabs(col[static_cast<size_t>(j) * g.N]));
+            sb = f64_to_e4m3(ldexp(a / 6.0, -ew));
+            const double s = ldexp(e4m3_to_f64(sb), ew);
+            for (int j = 0; j < 16; ++j)
+                codes[j] = (j < len && s != 0.0) ? f64_to_e2m1(col[static_cast<size_t>(j) * g.N] / s) : 0;
+        } else {
+            for (int j = 0; j < 16; ++j) codes[j] = 0;
+        }
+        sfword |= static_cast<uint32_t>(sb) << (8 * b);
+        for (int j = 0; j < 16; j += 2) crow[b * 8 + j / 2] = static_cast<uint8_t>(codes[j] | (codes[j + 1] << 4));
+    }
+    const int nr = n & 127;
+    *reinterpret_cast<uint32_t*>(wsf + (static_cast<size_t>(n >> 7) * g.nkb64p + kb) * 512 + (nr & 31) * 16 + (nr >> 5) * 4) = sfword;
+}
+
+// wh[n][i] = bf16(Wt[i][n]) * 2^-(ex+ew)  (exact: a power of two), zero padded to r_pad.
+__global__ void nvfp4_high_rows_kernel(const double* Wt, uint16_t* wh, const Nvfp4Meta* meta, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= g.N) return;
+    const int sh = meta->ex + meta->ew;
+    for (int i = 0; i < g.r_pad; ++i) {
+        uint16_t out = 0;
+        if (i < g.r) out = f64_to_bf16(ldexp(bf16_to_f64(f64_to_bf16(Wt[static_cast<size_t>(i) * g.N + n])), -sh));
+        wh[static_cast<size_t>(n) * g.r_pad + i] = out;
+    }
+}
+
+__global__ void nvfp4_export_weights_kernel(const uint8_t* wcodes, const uint8_t* wsf, const uint16_t* wh, const Nvfp4Meta* meta,
+                                            Geometry g, uint8_t* codes_out, uint8_t* sf_out, uint16_t* wh_out, int* ew_out) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int j = blockIdx.y;  // low-precision row
+    if (n == 0 && j == 0 && ew_out) *ew_out = meta->ew;
+    if (n >= g.N) return;
+    if (j < g.K_l && codes_out) {
+        const uint8_t byte = wcodes[static_cast<size_t>(n) * (g.K4 / 2) + j / 2];
+        codes_out[static_cast<size_t>(j) * g.N + n] = (j & 1) ? (byte >> 4) : (byte & 0xF);
+    }
+    const int nb = (g.K_l + 15) / 16;
+    if (j < nb && sf_out) {
+        const int nr = n & 127;
+        sf_out[static_cast<size_t>(j) * g.N + n] =
+            wsf[(static_cast<size_t>(n >> 7) * g.nkb64p + (j >> 2)) * 512 + (nr & 31) * 16 + (nr >> 5) * 4 + (j & 3)];
+    }
+    if (j < g.r && wh_out)
+        wh_out[static_cast<size_t>(j) * g.N + n] =
+            f64_to_bf16(ldexp(bf16_to_f64(wh[static_cast<size_t>(n) * g.r_pad + j]), meta->ex + meta->ew));
+}
+
+__global__ void nvfp4_export_workspace_kernel(const uint8_t* codes, const uint8_t* xsf, const uint16_t* xh_pad, int M, Geometry g,
+                                              uint16_t* xh, uint8_t* codes_out, uint8_t* sf_out) {
+    const int m = blockIdx.y;
+    const int nb = (g.K_l + 15) / 16;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < g.K_l; c += gridDim.x * blockDim.x) {
+        if (codes_out) {
+            const uint8_t byte = codes[static_cast<size_t>(m) * (g.K4 / 2) + c / 2];
+            codes_out[static_cast<size_t>(m) * g.K_l + c] = (c & 1) ? (byte >> 4) : (byte & 0xF);
+        }
+    }
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < g.r; i += blockDim.x)
+            if (xh) xh[static_cast<size_t>(m) * g.r + i] = xh_pad[static_cast<size_t>(m) * g.r_pad + i];
+        const int mr = m & 127;
+        for (int b = threadIdx.x; b < nb; b += blockDim.x)
+            if (sf_out)
+                sf_out[static_cast<size_t>(m) * nb + b] =
+                    xsf[(static_cast<size_t>(m >> 7) * g.nkb64p + (b >> 2)) * 512 + (mr & 31) * 16 + (mr >> 5) * 4 + (b & 3)];
+    }
+}
+
 inline bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
 
 }  // namespace
@@ -260,6 +416,69 @@ dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char
     export_workspace_kernel<<<dim3(8, M), 256, 0, stream>>>(
         reinterpret_cast<const int8_t*>(workspace + w.off_codes), reinterpret_cast<const float*>(workspace + w.off_xscale),
         reinterpret_cast<const uint16_t*>(workspace + w.off_xh), M, w.ldm, g, xh, codes, scales);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace dirotq
+
+namespace dirotq {
+
+dirotq_status_t launch_prepare_nvfp4(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
+                                     int q_dtype, const void* bias, double* scratch, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    char* blob = L->blob;
+    Nvfp4Meta* meta = reinterpret_cast<Nvfp4Meta*>(blob + L->lay.off_meta);
+    fold_kernel<<<dim3((g.N + 63) / 64, (g.K + 63) / 64), 256, 0, stream>>>(Q, q_dtype, W, w_dtype, w_layout, scratch,
+                                                                          g.K, g.N);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    if (cudaMemsetAsync(meta, 0, 64, stream) != cudaSuccess) return DIROTQ_ERR_CUDA;
+    if (cudaMemsetAsync(blob + L->lay.off_wscale, 0, static_cast<size_t>((g.N + 127) / 128) * g.nkb64p * 512, stream) !=
+        cudaSuccess)
+        return DIROTQ_ERR_CUDA;
+    nvfp4_amax_kernel<<<592, 256, 0, stream>>>(scratch, g, meta);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    nvfp4_meta_kernel<<<1, 1, 0, stream>>>(meta, L->act_scale_log2);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    nvfp4_quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.nkb64), 128, 0, stream>>>(
+        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<uint8_t*>(blob + L->lay.off_wscale),
+        meta, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    nvfp4_high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh),
+                                                                  meta, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
+        Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                       reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_layer_export_nvfp4(const dirotq_layer* L, uint8_t* wcodes, uint8_t* wsf, uint16_t* wh, uint16_t* qb,
+                                          int* ew, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const char* blob = L->blob;
+    const int rows = g.K_l > g.r ? g.K_l : g.r;
+    nvfp4_export_weights_kernel<<<dim3((g.N + 127) / 128, rows), 128, 0, stream>>>(
+        reinterpret_cast<const uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<const uint8_t*>(blob + L->lay.off_wscale),
+        reinterpret_cast<const uint16_t*>(blob + L->lay.off_wh), reinterpret_cast<const Nvfp4Meta*>(blob + L->lay.off_meta), g,
+        wcodes, wsf, wh, ew);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    if (qb) {
+        export_q_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
+            reinterpret_cast<const uint16_t*>(blob + L->lay.off_qt), qb, g);
+        if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    }
+    return DIROTQ_OK;
+}
+
+dirotq_status_t launch_workspace_export_nvfp4(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
+                                              uint8_t* codes, uint8_t* sf, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const WorkspaceLayout w = make_workspace_layout_nvfp4(g, M);
+    nvfp4_export_workspace_kernel<<<dim3(8, M), 256, 0, stream>>>(
+        reinterpret_cast<const uint8_t*>(workspace + w.off_codes), reinterpret_cast<const uint8_t*>(workspace + w.off_xscale),
+        reinterpret_cast<const uint16_t*>(workspace + w.off_xh), M, g, xh, codes, sf);
     return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 

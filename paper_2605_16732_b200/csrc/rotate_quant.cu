@@ -37,6 +37,10 @@ struct RotKernelParams {
     uint16_t* xh;
     float* xrot;
     int* status;
+    // NVFP4 variant
+    uint8_t* xsf;     // scale-factor atoms [ceil(M/128)][nkb64p][512]
+    int K4, nkb64p;   // packed row width in elements; atoms per row block
+    int ex;           // exponent of the activations' per-tensor power-of-two scale
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -62,7 +66,52 @@ __device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, 
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int G>
+// ---- NVFP4 (paper Sec. 5.1): E2M1 elements, blocks of 16, E4M3 block scale relative to 2^ex ----------
+
+// Non-negative float -> E4M3 byte, nearest-even, saturating at 448 (hardware conversion).
+__device__ __forceinline__ uint32_t f32_to_e4m3(float v) {
+    uint16_t pair;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(0.0f), "f"(v));  // second operand -> low byte
+    return pair & 0xFFu;
+}
+
+__device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
+    const uint32_t e = (b >> 3) & 0xFu, m = b & 7u;
+    return e == 0 ? static_cast<float>(m) * 0.001953125f : __uint_as_float(((e + 120u) << 23) | (m << 20));
+}
+
+// Two floats -> one byte of two E2M1 codes, nearest-even, saturating at 6: `lo` in bits 0..3, `hi` in bits 4..7.
+__device__ __forceinline__ uint32_t f32x2_to_e2m1x2(float lo, float hi) {
+    uint32_t out;
+    asm("{\n\t"
+        ".reg .b8 t;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n\t"
+        "cvt.u32.u8 %0, t;\n\t"
+        "}\n"
+        : "=r"(out)
+        : "f"(hi), "f"(lo));
+    return out;
+}
+
+// One block of 16 values: returns the E4M3 scale byte and writes the 8 code bytes (two 32-bit words).
+__device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float ex_inv, float ex_scale, uint32_t& w0, uint32_t& w1) {
+    float amax = 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[j]));
+    const uint32_t sb = f32_to_e4m3(__fdiv_rn(amax, 6.0f) * ex_inv);
+    const float s = e4m3_to_f32(sb) * ex_scale;
+    const float inv = s > 0.f ? __frcp_rn(s) : 0.f;
+    w0 = 0;
+    w1 = 0;
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {
+        w0 |= f32x2_to_e2m1x2(v[j] * inv, v[j + 1] * inv) << (4 * j);
+        w1 |= f32x2_to_e2m1x2(v[8 + j] * inv, v[9 + j] * inv) << (4 * j);
+    }
+    return sb;
+}
+
+template <int G, int FMT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
                     const RotKernelParams p) {
@@ -209,7 +258,30 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
                 // number of low-precision values among v[] (a multiple of 16)
                 const int nlow = min(G, max(0, p.K_l - col0));
-                if (nlow > 0) {
+                if constexpr (FMT == 1) {
+                    // NVFP4: four blocks of 16 per 64-column chunk; one 32-bit word of scale bytes per chunk
+                    static_assert(FMT == 0 || G == 64, "the NVFP4 epilogue works on 64-column chunks");
+                    if (col0 < p.K4 && row_ok) {
+                        const float ex_scale = __uint_as_float(static_cast<uint32_t>(127 + p.ex) << 23);
+                        const float ex_inv = __uint_as_float(static_cast<uint32_t>(127 - p.ex) << 23);
+                        uint32_t sfword = 0;
+                        uint8_t* crow = reinterpret_cast<uint8_t*>(p.codes) + static_cast<size_t>(row) * (p.K4 / 2) + col0 / 2;
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            uint32_t w0 = 0, w1 = 0;
+                            if (16 * b < nlow) sfword |= nvfp4_block16(v + 16 * b, ex_inv, ex_scale, w0, w1) << (8 * b);
+                            *reinterpret_cast<uint2*>(crow + 8 * b) = make_uint2(w0, w1);  // zero in the padding slots
+                        }
+                        const int mr = row & 127;
+                        *reinterpret_cast<uint32_t*>(p.xsf + (static_cast<size_t>(row >> 7) * p.nkb64p + (col0 >> 6)) * 512 +
+                                                     (mr & 31) * 16 + (mr >> 5) * 4) = sfword;
+                        // atoms that only pad the last 256-element k-block: scale 0 (never NaN bytes)
+                        if (col0 + 64 >= p.K4)
+                            for (int a = (col0 >> 6) + 1; a < p.nkb64p; ++a)
+                                *reinterpret_cast<uint32_t*>(p.xsf + (static_cast<size_t>(row >> 7) * p.nkb64p + a) * 512 +
+                                                             (mr & 31) * 16 + (mr >> 5) * 4) = 0u;
+                    }
+                } else if (nlow > 0) {
                     float amax = 0.f;
 #pragma unroll
                     for (int b = 0; b < G / 16; ++b) {
@@ -281,11 +353,12 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     RotKernelParams p;
     p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.ldm = a.ldm;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
+    p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
     const int num_tiles = ((a.M + BM - 1) / BM) * ((g.K + BN - 1) / BN);
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
-    auto kern = g.G == 64 ? rotate_quant_kernel<64> : rotate_quant_kernel<128>;
-    static bool attr_set[2] = {false, false};
-    const int vi = g.G == 64 ? 0 : 1;
+    const int vi = g.fmt == 1 ? 2 : (g.G == 64 ? 0 : 1);
+    auto kern = vi == 2 ? rotate_quant_kernel<64, 1> : (vi == 0 ? rotate_quant_kernel<64, 0> : rotate_quant_kernel<128, 0>);
+    static bool attr_set[3] = {false, false, false};
     if (!attr_set[vi]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;

@@ -142,3 +142,112 @@ def check_layer_output(y_bits, xh_bits, codes, scales, layer_orc, out_orc, bias_
     d = np.abs(f64(y_bits) - out_orc["y64"])
     stats["e2e_all_max_err_over_rms"] = float(d.max() / np.sqrt(np.mean(out_orc["y64"] ** 2)))
     return stats
+
+
+# ------------------------------------------------------------------ NVFP4 variant
+#
+# Protocol (same structure as for INT4; E2M1 codes are compared with +0 and -0 identified):
+#   * weights: E4M3 block scales, bf16 rows, rotation and the per-tensor exponent equal the oracle's;
+#     E2M1 codes equal, except at exact ties of the fp64 quotient (|distance to a rounding boundary|
+#     < 1e-9: the fold's summation order differs), at most 4 per layer;
+#   * an activation block scale equals the oracle's or is the neighbouring E4M3 value when the
+#     unrounded absmax/6/2^ex lies within tol_s of the midpoint between the two;
+#   * an activation code equals the oracle quantizer re-run with the library's scale, or is the
+#     neighbouring E2M1 value when the quotient lies within tol_t of the boundary between the two;
+#   * tol_s = 1e-4 relative + 1e-5 ||x~_row|| (fp32 accumulation of the rotation, as for x~_h),
+#     tol_t = 1e-3 + 1e-5 ||x~_row|| / s_block  (blocks of 16 can have scales far below the row norm);
+#   * output: within half a bf16 step + slack * rms of the fp64 combination of the library's own
+#     codes, scales and bf16 coefficients.
+
+_E2M1_BOUNDS = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])
+
+
+def _mag(c):
+    return c & 7
+
+
+def _codes_equal_mod_zero(a, b):
+    return (a == b) | ((_mag(a) == 0) & (_mag(b) == 0))
+
+
+def check_weight_side_nvfp4(export, layer_orc):
+    wcodes, wsf, wh, qb, ew = export
+    assert ew == layer_orc["ew"], "per-tensor weight exponent differs"
+    assert np.array_equal(bf16_tensor_to_bits(qb), layer_orc["Qb"]), "bf16 rotation differs"
+    assert np.array_equal(wsf.cpu().numpy(), layer_orc["wsf"]), "weight block scales differ"
+    assert np.array_equal(bf16_tensor_to_bits(wh), layer_orc["Wh"]), "bf16 high rows differ"
+    got = wcodes.cpu().numpy()
+    bad = ~_codes_equal_mod_zero(got, layer_orc["wcodes"])
+    if bad.any():
+        t = layer_orc["wt"]
+        assert t is not None, f"{bad.sum()} weight codes differ"
+        dist = np.min(np.abs(np.abs(t[bad])[:, None] - _E2M1_BOUNDS[None, :]), axis=1)
+        assert np.all(dist < 1e-9), "a weight code differs away from an exact tie"
+        assert bad.sum() <= 4
+    return {"weight_code_ties": int(bad.sum())}
+
+
+def check_activation_side_nvfp4(xrot, xh, codes, sf, out_orc, r, ex):
+    xt = out_orc["xt"]
+    M, K = xt.shape
+    K_l = K - r
+    nb = -(-K_l // 16)
+    stats = {}
+    norm = np.linalg.norm(xt, axis=1, keepdims=True)
+    if xrot is not None:
+        rel = np.linalg.norm(xrot.astype(np.float64) - xt, axis=1) / np.maximum(norm[:, 0], 1e-300)
+        stats["xrot_rel_max"] = float(rel.max())
+        assert rel.max() <= 2e-3
+    xh_g, xh_o = f64(xh), f64(out_orc["xh"])
+    step = np.maximum(np.abs(xh_o), 2.0 ** -126) * 2.0 ** -7 + 1e-5 * norm
+    assert np.all(np.abs(xh_g - xh_o) <= step), "x~_h differs by more than one bf16 step"
+    # block scales
+    low = np.zeros((M, nb * 16))
+    low[:, :K_l] = xt[:, r:]
+    u = np.abs(low).reshape(M, nb, 16).max(axis=2) / 6.0 * 2.0 ** (-ex)
+    s_g, s_o = orc.e4m3_to_f64(sf), orc.e4m3_to_f64(out_orc["sf"])
+    flip = sf != out_orc["sf"]
+    if flip.any():
+        db = np.abs(sf[flip].astype(np.int64) - out_orc["sf"][flip].astype(np.int64))
+        assert np.all(db == 1), "a block scale is more than one E4M3 step away"
+        mid = 0.5 * (s_g[flip] + s_o[flip])
+        tol = 1e-4 * u[flip] + 1e-5 * np.broadcast_to(norm, u.shape)[flip] / 6.0 * 2.0 ** (-ex)
+        assert np.all(np.abs(u[flip] - mid) <= tol), "block scale differs away from a rounding boundary"
+    stats["scale_flips"] = int(flip.sum())
+    # codes against the quantizer re-run with the library's scale
+    s_use = np.repeat(s_g * 2.0 ** ex, 16, axis=1)[:, :K_l]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(s_use != 0, xt[:, r:] / s_use, 0.0)
+    mag_ref = np.searchsorted(_E2M1_BOUNDS, np.abs(t), side="left").astype(np.uint8)
+    # ties go to the even code: a value exactly on a boundary between codes c and c+1 takes the even one
+    on = np.isin(np.abs(t), _E2M1_BOUNDS)
+    if on.any():
+        lo_code = np.searchsorted(_E2M1_BOUNDS, np.abs(t[on]), side="left").astype(np.uint8)  # the lower neighbour
+        mag_ref[on] = np.where(lo_code % 2 == 0, lo_code, lo_code + 1)
+    q_ref = np.where(t < 0, 8, 0).astype(np.uint8) | mag_ref
+    same_scale = ~np.repeat(flip, 16, axis=1)[:, :K_l]
+    assert np.all(_codes_equal_mod_zero(q_ref, out_orc["codes"])[same_scale]), "the protocol's re-run disagrees with the oracle"
+    bad = ~_codes_equal_mod_zero(codes, q_ref)
+    if bad.any():
+        dm = np.abs(_mag(codes[bad]).astype(int) - _mag(q_ref[bad]).astype(int))
+        sign_ok = ((codes[bad] & 8) == (q_ref[bad] & 8)) | (np.minimum(_mag(codes[bad]), _mag(q_ref[bad])) == 0)
+        assert np.all(dm == 1) and np.all(sign_ok), "a code is off by more than one E2M1 step"
+        dist = np.min(np.abs(np.abs(t[bad])[:, None] - _E2M1_BOUNDS[None, :]), axis=1)
+        with np.errstate(divide="ignore"):
+            tol_t = 1e-3 + 1e-5 * np.broadcast_to(norm, t.shape)[bad] / s_use[bad]
+        assert np.all(dist <= tol_t), "a code differs away from a rounding boundary"
+    stats["code_flips"] = int(bad.sum())
+    return stats
+
+
+def check_layer_output_nvfp4(y_bits, xh_bits, codes, sf, ex, layer_orc, out_orc, bias_bits, slack=3e-4):
+    y_ref, _ = orc.nvfp4_combine(codes, sf, ex, layer_orc, xh_bits, bias_bits)
+    stats = check_output(y_bits, y_ref, slack=slack)
+    clean = (np.all(_codes_equal_mod_zero(codes, out_orc["codes"]), axis=1) & np.all(sf == out_orc["sf"], axis=1)
+             & np.all(xh_bits == out_orc["xh"], axis=1))
+    stats["clean_rows_frac"] = float(np.mean(clean))
+    e2e = check_output(y_bits, out_orc["y64"], rows=clean, slack=slack)
+    stats["e2e_clean_max_err_over_rms"] = e2e.get("max_err_over_rms")
+    d = np.abs(f64(y_bits) - out_orc["y64"])
+    stats["e2e_all_max_err_over_rms"] = float(d.max() / np.sqrt(np.mean(out_orc["y64"] ** 2)))
+    return stats
