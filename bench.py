@@ -189,10 +189,22 @@ def run_ours(args):
         spec = synth.LayerSpec(K=K, N=N, r=RANK, G=GROUP, model=synth.FLUX, seed=100)
         Q = torch.from_numpy(synth.make_rotation(spec, device=str(dev))).to(dev)
         W, bias = synth.make_weights(spec)
-        layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
-        del Q
         x_bits = synth.make_tokens(spec, M, batch_seed=1000 + rank)
         x = bf(x_bits)
+        if args.fmt == "nvfp4":
+            # the activations' power-of-two scale is a calibration constant: taken here from this batch's first
+            # 1024 tokens, rotated by the library itself (a throw-away layer with exponent 0)
+            probe = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, 0, bias=bf(bias))
+            xrot = torch.empty((1024, K), dtype=torch.float32, device=dev)
+            dq.dirotq_rotate_quantize(x[:1024], probe, dq.alloc_workspace(probe, 1024), xrot)
+            amax = float(xrot[:, RANK:].abs().max().item())
+            probe.close()
+            del xrot
+            layer = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, int(np.ceil(np.log2(amax / 1536.0))),
+                                                  bias=bf(bias))
+        else:
+            layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
+        del Q
         y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
         ws = dq.alloc_workspace(layer, M)
         layers.append({"name": name, "K": K, "N": N, "layer": layer, "x": x, "y": y, "ws": ws, "x_bits": x_bits})
@@ -301,13 +313,15 @@ def run_ours(args):
     rot_total, gemm_total = sum(rot_ms.values()), sum(gemm_ms.values())
     rot_flops = {n: 2.0 * M * K * K for n, K, _ in FLUX_SHAPES}
     gemm_ops = {n: 2.0 * M * (K - RANK) * N for n, K, N in FLUX_SHAPES}
-    int8_peak = 2.0 * peaks["bf16_sustained"]  # nominal int8 : bf16 ratio of the part (4.5 : 2.25)
+    nv = args.fmt == "nvfp4"
+    # nominal ratios of the part: 8-bit (int8 / fp8) 2x and fp4 4x the dense bf16 rate (4.5 and 9 : 2.25 PFLOP/s)
+    int8_peak = (4.0 if nv else 2.0) * peaks["bf16_sustained"]
     # DRAM bytes of one launch of the dominant kernel, from the ncu capture summarised under profiles/
     # (qkv shape; read + write).  Static: a profiler is never run inside the benchmark.
-    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 68.1e6, "rotate_quant_kernel": 48.5e6}
+    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 70.2e6, "rotate_quant_kernel": 48.5e6, "nvfp4_gemm_kernel": None}
     sm_hz = (clocks or {}).get("sm_mhz") or 1850.0
     elem_steps = sum(M * N * (-(-(K - RANK) // GROUP)) for _, K, N in FLUX_SHAPES)
-    alu_peak = 148 * (128.0 / 3.0) * sm_hz * 1e6  # element-steps/s: 3 thread instructions each, 128 issued per cycle and SM
+    alu_peak = 148 * (128.0 / 2.0) * sm_hz * 1e6  # element-steps/s: 2 fused multiply-adds each, 128 fp32 lanes per SM
     if rot_total >= gemm_total:
         ach = sum(rot_flops.values()) / (rot_total * 1e-3) / 1e12
         roofline = {"kernel": "rotate_quant_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_sustained"],
@@ -316,14 +330,16 @@ def run_ours(args):
     else:
         ach = sum(gemm_ops.values()) / (gemm_total * 1e-3) / 1e12
         ach_alu = elem_steps / (gemm_total * 1e-3)
-        roofline = {"kernel": "w4a4_gemm_kernel", "bound": "tensor", "achieved": ach, "peak": int8_peak, "unit": "TOP/s",
-                    "frac": ach / int8_peak, "traffic": NCU_TRAFFIC_QKV["w4a4_gemm_kernel"],
+        gname = "nvfp4_gemm_kernel" if nv else "w4a4_gemm_kernel"
+        roofline = {"kernel": gname, "bound": "tensor", "achieved": ach, "peak": int8_peak, "unit": "TOP/s",
+                    "frac": ach / int8_peak, "traffic": NCU_TRAFFIC_QKV[gname],
                     "traffic_note": "ncu dram read+write of one qkv-shaped launch (algorithmic bytes of that launch: 117.5e6)",
-                    "peak_source": f"2 x {peaks['source']} bf16 sustained (nominal int8:bf16 ratio)",
-                    "alu": {"bound": "alu", "achieved": ach_alu / 1e9, "peak": alu_peak / 1e9, "unit": "G element-steps/s",
-                            "frac": ach_alu / alu_peak,
-                            "note": "per-group rescale: >= 3 thread instructions per output element and K-group; "
-                                    "148 SMs x 128 issued thread instructions per cycle at the sampled SM clock"}}
+                    "peak_source": f"{'4' if nv else '2'} x {peaks['source']} bf16 sustained (nominal {'fp4' if nv else '8-bit'}:bf16 ratio)"}
+        if not nv:
+            roofline["alu"] = {"bound": "alu", "achieved": ach_alu / 1e9, "peak": alu_peak / 1e9, "unit": "G element-steps/s",
+                               "frac": ach_alu / alu_peak,
+                               "note": "per-group rescale: 2 fp32 fused multiply-adds per output element and K-group; "
+                                       "148 SMs x 128 fp32 lanes at the sampled SM clock"}
     kernels = {}
     for n, K, N in FLUX_SHAPES:
         t_roof = (gemm_ops[n] / int8_peak + (rot_flops[n] + 2.0 * M * RANK * N) / peaks["bf16_sustained"]) / 1e12 * 1e3
@@ -343,8 +359,11 @@ def run_ours(args):
     line = {
         "metric": "dirotq_w4a4_linear_effective_tops", "value": value, "unit": "TOPS", "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int4xint4->int32 + bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK, "group": GROUP,
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "nvfp4 (e2m1 x e2m1, e4m3 block scales) + bf16" if nv else "int4xint4 (exact group sums on the e4m3 tensor path) + bf16",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
+                   "group": 16 if nv else GROUP, "format": args.fmt,
                    "l2": "inputs_exceed_l2 (each step streams > 500 MB of rotations, codes and outputs)",
                    "parallelism": f"token rows x{world}, no collective"},
         "clocks": clocks,
@@ -368,6 +387,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shapes", default="", help="comma-separated subset of qkv,out,mlp_up,mlp_down (profiling runs)")
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4"],
+                    help="int4: the headline format (groups of 64, bf16 scales); nvfp4: E2M1 blocks of 16 with E4M3 scales")
     ap.add_argument("--lite", action="store_true", help="skip the cuBLAS, end-to-end and CPU-baseline legs (profiling runs)")
     args = ap.parse_args()
     if args.shapes:

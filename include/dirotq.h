@@ -158,7 +158,9 @@ DIROTQ_API dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, 
                                         int8_t* codes, void* scales_bf16, dirotq_stream_t stream);
 
 /* Integer GEMM alone on caller-supplied activation codes (int8, one per byte, [M,K_lp] with
- * zero codes in columns >= K-r): partials[g][m][n] = sum over group g of q_x q_w, int32. */
+ * zero codes in columns >= K-r): partials[g][m][n] = sum over group g of q_x q_w, int32.
+ * The codes are first converted into the workspace (its activation codes and scales are
+ * overwritten), then the production kernel runs with unit scales and stores the group sums. */
 DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const dirotq_layer_t* layer,
                                       int32_t* partials, void* workspace, size_t workspace_bytes,
                                       dirotq_stream_t stream);
@@ -224,7 +226,8 @@ DIROTQ_API dirotq_status_t dirotq_linear_noalloc(const void* x, int M, const dir
 
 /* Issue-rate probe of the tensor pipe: every SM issues 4*iters back-to-back 128x256 tcgen05.mma
  * instructions on operands resident in shared memory (kind 0: int8 -> int32, K = 32 per
- * instruction; kind 1: bf16 -> fp32, K = 16), twice (warm-up + timed).  SYNCHRONISES.
+ * instruction; kind 1: bf16 -> fp32, K = 16; kind 2: E4M3 -> fp32, K = 32, the instruction the
+ * W4A4 kernel computes its exact integer group sums with), twice (warm-up + timed).  SYNCHRONISES.
  * status_word: device int32, zero-filled (receives a code if the bounded completion wait
  * expires).  *tera_ops_per_s receives 2*M*N*K*instructions / time. */
 DIROTQ_API dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* status_word, float* tera_ops_per_s,

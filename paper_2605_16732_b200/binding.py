@@ -245,7 +245,7 @@ def dirotq_layer_export(layer: Layer, stream=None):
 
 
 def dirotq_mma_rate_probe(kind: int, iters: int = 20000, stream=None) -> float:
-    """Measured tensor-pipe rate in tera-ops/s.  kind 0: int8 (kind::i8), kind 1: bf16 (kind::f16)."""
+    """Measured tensor-pipe rate in tera-ops/s.  kind 0: int8 (kind::i8), 1: bf16 (kind::f16), 2: E4M3 (kind::f8f6f4)."""
     status = torch.zeros(64, dtype=torch.int32, device="cuda")
     out = ctypes.c_float(0.0)
     _check(lib().dirotq_mma_rate_probe(kind, iters, status.data_ptr(), ctypes.byref(out), _stream(stream)),

@@ -324,8 +324,10 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
     if (!act_codes || !partials || !aligned16(act_codes) || !aligned16(partials)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = static_cast<char*>(workspace);
     const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
+    st = launch_debug_codes(layer, M, act_codes, ws, static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) return st;
     GemmArgs ga;
-    ga.M = M; ga.codes = act_codes;
+    ga.M = M; ga.codes = reinterpret_cast<const int8_t*>(ws + w.off_codes);
     ga.xscale = reinterpret_cast<const float*>(ws + w.off_xscale);
     ga.ldm = w.ldm;
     ga.xh = reinterpret_cast<const uint16_t*>(ws + w.off_xh);

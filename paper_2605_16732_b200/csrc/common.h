@@ -88,8 +88,9 @@ inline BlobLayout make_blob_layout_nvfp4(const Geometry& g) {
 struct WorkspaceLayout {
     int ldm;            // leading dimension (tokens) of the transposed activation-scale array
     size_t off_status;  // int32[64]: word 0 = device status
-    size_t off_codes;   // i8  [M][K_lp]: activation codes, one per byte
-    size_t off_xscale;  // f32 [n_g][ldm]: bf16-valued activation scales, group-major
+    size_t off_codes;   // u8  [M][K_lp]: activation codes, one per byte, sign-magnitude (bit 7 = sign, bits 2..0 = |q|)
+    size_t off_xscale;  // f32 [2 n_g][ldm]: rows 0..n_g-1 the bf16-valued activation scales s (group-major),
+                        //                   rows n_g..2 n_g-1 the offset corrections -8 * s * sum_k q (see w4a4_gemm.cu)
     size_t off_xh;      // bf16 [M][r_pad]
     // NVFP4 variant: off_codes = E2M1 codes u8 [M][K4/2]; off_xscale = E4M3 scale atoms u8 [ceil(M/128)][nkb64p][512]
     size_t total;
@@ -101,7 +102,7 @@ inline WorkspaceLayout make_workspace_layout(const Geometry& g, int M) {
     size_t o = 0;
     w.off_status = o;  o = align_up(o + 256);
     w.off_codes = o;   o = align_up(o + (size_t)M * g.K_lp);
-    w.off_xscale = o;  o = align_up(o + (size_t)g.n_g * w.ldm * 4);
+    w.off_xscale = o;  o = align_up(o + (size_t)2 * g.n_g * w.ldm * 4);
     w.off_xh = o;      o = align_up(o + (size_t)M * g.r_pad * 2);
     w.total = o;
     return w;
@@ -129,7 +130,7 @@ struct dirotq_layer {
     dirotq::BlobLayout lay;
     char* blob;  // device
     CUtensorMap tmap_qt;       // bf16 [K][K], box 64 x 256, 128B swizzle
-    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2], box 64 x kGemmBN, no swizzle
+    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2] (nibble = q + 8), box 64 x kGemmBN, no swizzle
     CUtensorMap tmap_wscale;   // f32 [n_g][N], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
     int act_scale_log2;        // NVFP4 variant: exponent of the activations' per-tensor power-of-two scale
@@ -195,6 +196,8 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
                                     uint16_t* qb, cudaStream_t stream);
 dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
                                         int8_t* codes, uint16_t* scales, cudaStream_t stream);
+dirotq_status_t launch_debug_codes(const dirotq_layer* L, int M, const int8_t* act_codes, char* workspace,
+                                   cudaStream_t stream);
 int sm_count(int device);
 
 }  // namespace dirotq

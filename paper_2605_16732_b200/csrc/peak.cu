@@ -10,7 +10,8 @@ namespace {
 constexpr int PEAK_THREADS = 128;
 constexpr int PEAK_SMEM = 2 * (16384 + 32768) + 1024 + 64;
 
-// kind: 0 = kind::i8 (s8 x s8 -> s32, K = 32 per instruction), 1 = kind::f16 (bf16 -> f32, K = 16)
+// kind: 0 = kind::i8 (s8 x s8 -> s32, K = 32 per instruction), 1 = kind::f16 (bf16 -> f32, K = 16),
+//       2 = kind::f8f6f4 (E4M3 x E4M3 -> f32, K = 32)
 __global__ void __launch_bounds__(PEAK_THREADS, 1) mma_peak_kernel(int kind, int iters, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -37,7 +38,7 @@ __global__ void __launch_bounds__(PEAK_THREADS, 1) mma_peak_kernel(int kind, int
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 0) {
-        const uint32_t idesc = kind == 0 ? umma_idesc(2, 1, 128, 256) : umma_idesc(1, 1, 128, 256);
+        const uint32_t idesc = kind == 0 ? umma_idesc(2, 1, 128, 256) : (kind == 1 ? umma_idesc(1, 1, 128, 256) : umma_idesc(1, 0, 128, 256));
         for (int i = 0; i < iters; ++i) {
             const uint32_t st = base + (i & 1) * (16384 + 32768);
             const uint64_t adesc = umma_desc_sw128(st);
@@ -46,7 +47,8 @@ __global__ void __launch_bounds__(PEAK_THREADS, 1) mma_peak_kernel(int kind, int
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 if (kind == 0) umma_i8(d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
-                else umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+                else if (kind == 1) umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+                else umma_f8f6f4(d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
             }
         }
         umma_commit(bar);
@@ -67,7 +69,7 @@ using namespace dirotq;
 
 extern "C" dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* status_word, float* tera_ops_per_s,
                                                 dirotq_stream_t stream) {
-    if ((kind != 0 && kind != 1) || iters < 1 || iters > (1 << 20) || !status_word || !tera_ops_per_s)
+    if (kind < 0 || kind > 2 || iters < 1 || iters > (1 << 20) || !status_word || !tera_ops_per_s)
         return DIROTQ_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return DIROTQ_ERR_CUDA;
@@ -94,7 +96,7 @@ extern "C" dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* stat
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     if (e != cudaSuccess || ms <= 0.f) return DIROTQ_ERR_CUDA;
-    const double k_per_instr = kind == 0 ? 32.0 : 16.0;
+    const double k_per_instr = kind == 1 ? 16.0 : 32.0;
     const double ops = 2.0 * 128.0 * 256.0 * k_per_instr * 4.0 * iters * grid;
     *tera_ops_per_s = static_cast<float>(ops / (ms * 1e-3) / 1e12);
     return DIROTQ_OK;

@@ -106,7 +106,8 @@ __global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, floa
                 qq = fmin(7.0, fmax(-7.0, qq));
                 q = static_cast<int>(qq);
             }
-            const uint32_t nib = static_cast<uint32_t>(q) & 0xFu;
+            // stored with an offset of 8: the nibble u = q + 8 in 1..15, read as an E4M3 byte, is u * 2^-9 exactly
+            const uint32_t nib = static_cast<uint32_t>(q + 8) & 0xFu;
             word |= nib << (8 * (t & 3) + 4 * (t >> 2));
         }
         *reinterpret_cast<uint32_t*>(row + packed_byte_index(j0 + jb)) = word;
@@ -152,7 +153,7 @@ __global__ void export_wcodes_kernel(const uint8_t* wpacked, int8_t* wcodes, Geo
     if (n >= g.N || j >= g.K_l) return;
     const uint8_t byte = wpacked[static_cast<size_t>(n) * (g.K_lp / 2) + packed_byte_index(j)];
     const int nib = packed_is_high(j) ? (byte >> 4) : (byte & 0xF);
-    wcodes[static_cast<size_t>(j) * g.N + n] = static_cast<int8_t>((nib ^ 8) - 8);  // sign-extend 4 bits
+    wcodes[static_cast<size_t>(j) * g.N + n] = static_cast<int8_t>(nib - 8);  // stored with an offset of 8
 }
 
 __global__ void export_wscales_kernel(const float* wscale, uint16_t* out, size_t count) {
@@ -187,7 +188,10 @@ __global__ void export_workspace_kernel(const int8_t* codes, const float* xscale
                                         Geometry g, uint16_t* xh, int8_t* codes_out, uint16_t* scales) {
     const int m = blockIdx.y;
     for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < g.K_l; c += gridDim.x * blockDim.x)
-        if (codes_out) codes_out[static_cast<size_t>(m) * g.K_l + c] = codes[static_cast<size_t>(m) * g.K_lp + c];
+        if (codes_out) {
+            const int sm = static_cast<uint8_t>(codes[static_cast<size_t>(m) * g.K_lp + c]);  // sign-magnitude byte
+            codes_out[static_cast<size_t>(m) * g.K_l + c] = static_cast<int8_t>((sm & 0x80) ? -(sm & 7) : (sm & 7));
+        }
     if (blockIdx.x == 0) {
         for (int i = threadIdx.x; i < g.r; i += blockDim.x)
             if (xh) xh[static_cast<size_t>(m) * g.r + i] = xh_pad[static_cast<size_t>(m) * g.r_pad + i];
@@ -196,6 +200,23 @@ __global__ void export_workspace_kernel(const int8_t* codes, const float* xscale
                 scales[static_cast<size_t>(m) * g.n_g + gi] =
                     static_cast<uint16_t>(__float_as_uint(xscale[static_cast<size_t>(gi) * ldm + m]) >> 16);
     }
+}
+
+// Debug entry of the group GEMM: two's-complement codes [M][K_lp] -> the sign-magnitude bytes the kernel reads,
+// unit scales and the offset corrections -8 sum(q) (one thread per token and group).
+__global__ void debug_codes_kernel(const int8_t* in, uint8_t* out, float* xscale, int M, int ldm, Geometry g) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    const int grp = blockIdx.y;
+    if (m >= M) return;
+    int sum = 0;
+    for (int j = 0; j < g.G; ++j) {
+        const size_t idx = static_cast<size_t>(m) * g.K_lp + grp * g.G + j;
+        const int q = in[idx];
+        sum += q;
+        out[idx] = static_cast<uint8_t>((q < 0 ? 0x80 : 0) | (q < 0 ? -q : q));
+    }
+    xscale[static_cast<size_t>(grp) * ldm + m] = 1.0f;
+    xscale[static_cast<size_t>(g.n_g + grp) * ldm + m] = -8.0f * static_cast<float>(sum);
 }
 
 // ================================================================ NVFP4 variant (paper Sec. 5.1)
@@ -407,6 +428,16 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
     }
     return DIROTQ_OK;
+}
+
+dirotq_status_t launch_debug_codes(const dirotq_layer* L, int M, const int8_t* act_codes, char* workspace,
+                                   cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const WorkspaceLayout w = make_workspace_layout(g, M);
+    debug_codes_kernel<<<dim3((M + 127) / 128, g.n_g), 128, 0, stream>>>(
+        act_codes, reinterpret_cast<uint8_t*>(workspace + w.off_codes), reinterpret_cast<float*>(workspace + w.off_xscale), M,
+        w.ldm, g);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,

@@ -3,7 +3,8 @@
 //   x~ = x Q_b                      bf16 x bf16 -> fp32 on tcgen05 (kind::f16), operands by TMA
 //   x~_h = bf16(x~[:, high])        the r high-precision coefficients          (paper Sec. 4.2)
 //   per token, per group of G low-precision coefficients:                      (paper Eq. 1, z = 0)
-//       s = bf16(max|x~| / 7),  q = clip(rint(x~ / s), -7, 7)
+//       s = bf16(max|x~| / 7),  q = clip(rint(x~ / s), -7, 7)   stored as a sign-magnitude byte,
+//       plus the offset correction -8 s sum(q) that the second kernel needs
 //
 // The rotated activations never reach HBM: the fp32 accumulators are read from tensor memory by
 // the epilogue warps, where each thread owns one token row, so the group maximum is a
@@ -31,7 +32,7 @@ constexpr int NUM_THREADS = 192;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct RotKernelParams {
-    int M, K, K_l, K_lp, r, r_pad, ldm;
+    int M, K, K_l, K_lp, r, r_pad, ldm, n_g;
     int8_t* codes;
     float* xscale;
     uint16_t* xh;
@@ -48,20 +49,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Quantizes 16 consecutive values with the reciprocal scale and packs them one code per byte.
-__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, bool slow) {
+// Quantizes 16 consecutive values with the reciprocal scale and packs them one code per byte in
+// sign-magnitude form (bit 7 = sign, bits 2..0 = |q|): read as E4M3 that byte is q * 2^-9 exactly, which
+// is how the second kernel's tensor-core instruction consumes it.  The codes are also added to `sum`.
+__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, bool slow, int& sum) {
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        uint32_t word = 0;
+        uint32_t f[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             float t = slow ? (s != 0.f ? v[4 * i + j] / s : 0.f) : v[4 * i + j] * inv;
-            int q = __float2int_rn(t);  // round to nearest, ties to even
-            q = max(-7, min(7, q));
-            word |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * j);
+            t = fminf(fmaxf(t, -7.0f), 7.0f);
+            // adding 1.5 * 2^23 rounds to the nearest integer, ties to even, and leaves the two's-complement code
+            // in the low byte of the bit pattern
+            f[j] = __float_as_uint(t + 12582912.0f);
         }
-        w[i] = word;
+        const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
+        sum = __dp4a(static_cast<int>(tw), 0x01010101, sum);
+        const uint32_t sg = (tw >> 7) & 0x01010101u;           // 1 where the code is negative
+        const uint32_t mag = (tw ^ (sg * 0xFFu)) + sg;         // |q| per byte (at most 7: no carry between bytes)
+        w[i] = mag | (tw & 0x80808080u);
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
@@ -294,14 +302,18 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const bool slow = !(s >= 1e-30f);  // zero or tiny scale: divide instead of multiplying
                     const float inv = slow ? 0.f : __frcp_rn(s);
                     if (row_ok) {
-                        p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
                         int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+                        int qsum = 0;
 #pragma unroll
                         for (int b = 0; b < G / 16; ++b) {
                             uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
-                            if (16 * b < nlow) packed = quantize16(v + 16 * b, inv, s, slow);
+                            if (16 * b < nlow) packed = quantize16(v + 16 * b, inv, s, slow, qsum);
                             *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
                         }
+                        p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
+                        // the weights reach the tensor core as q_w + 8: -8 s sum(q_x) takes the offset out again
+                        // (exact in fp32: |sum| <= 7 G and s has 8 significant bits)
+                        p.xscale[static_cast<size_t>(p.n_g + col0 / G) * p.ldm + row] = -8.0f * static_cast<float>(qsum) * s;
                     }
                 }
                 if (nlow < G && row_ok) {
@@ -351,7 +363,7 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
                                         (uint64_t)g.K * 2, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != DIROTQ_OK) return st;
     RotKernelParams p;
-    p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.ldm = a.ldm;
+    p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
     const int num_tiles = ((a.M + BM - 1) / BM) * ((g.K + BN - 1) / BN);

@@ -3,19 +3,32 @@
 //   y[m,n] = bf16( sum_g s_x[m,g] s_w[g,n] P_g[m,n]  +  sum_{i<r} x~_h[m,i] W~_h[i,n]  +  bias[n] )
 //   P_g[m,n] = sum_{j in group g} q_x[m,j] q_w[j,n]                              (paper Eq. 5)
 //
-// sm_100a has no INT4 MMA.  The weight codes stay packed (two per byte) in HBM and in the TMA
-// staging buffer; two "unpack" warps expand every k-block to one code per byte -- each nibble
-// is moved to the HIGH half of its byte, so the int8 operand is 16*q_w, exact -- into the
-// 128-byte-swizzled layout tcgen05.mma kind::i8 reads.  The activation codes arrive one per byte
-// from kernel (a) and go straight from TMA to the MMA.
+// sm_100a has no INT4 MMA, and an int32 accumulator costs a conversion per element and group before it
+// can be scaled.  The integer products are therefore computed EXACTLY on the 8-bit float path
+// (tcgen05.mma kind::f8f6f4, E4M3 operands, fp32 accumulation):
+//   * an E4M3 byte 0000mmmm is m * 2^-9 for m = 0..15 (the subnormals 0..7 and the first binade 8..15
+//     lie on one line), and bit 7 is the sign;
+//   * activation codes arrive from kernel (a) one per byte in sign-magnitude form: q_x * 2^-9;
+//   * weight codes stay packed (two per byte) in HBM and in the TMA staging buffer with an offset of 8
+//     (u_w = q_w + 8 in 1..15); two "unpack" warps split every byte into two bytes 0000uuuu = u_w * 2^-9
+//     in the 128-byte-swizzled layout the MMA reads;
+//   * every product is an integer times 2^-18 and a group's sum is below 2^24 in magnitude, so the fp32
+//     accumulator holds S_g = 2^-18 sum_j q_x u_w without rounding, and
+//         P_g = 2^18 S_g - 8 sum_j q_x[m,j];
+//     kernel (a) stores e[m,g] = -8 s_x sum_j q_x (exact in fp32), so that
+//         s_x P_g = fma(S_g, 2^18 s_x, e)        -- one rounding, that of the product s_x P_g itself --
+//     and the group is folded in with two fused multiply-adds per element and no integer conversion.
+// The exactness of the accumulation is a property of the tensor core that the parity tests pin: the
+// group sums exported by the debug entry equal the CPU checker's int32 sums bit for bit, on random
+// codes and on patterns built to lose low bits (long runs of +-49 followed by +-1).
 //
-// Every K-group gets its own int32 accumulator tile in tensor memory (two tiles, ping-pong): the
-// MMA warp fills tile g%2 while the epilogue warps drain tile (g-1)%2, convert to fp32 and fold
-// it into per-thread fp32 accumulators with the two group scales.  The bf16 rank-r branch is
-// issued as one more "group" (kind::f16 into the same ping-pong tile) and added unscaled.
+// Every K-group gets its own accumulator tile in tensor memory (two tiles, ping-pong): the MMA warp
+// fills tile g%2 while the epilogue warps drain tile (g-1)%2 into per-thread fp32 accumulators.  The
+// bf16 rank-r branch is issued as one more "group" (kind::f16 into the same ping-pong tile) and added
+// unscaled.
 //
 // Roles (384 threads = 3 warpgroups):
-//   warpgroup 0: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-3 INT4->INT8 unpack
+//   warpgroup 0: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-3 nibble -> byte unpack
 //   warpgroups 1-2: epilogue; warp%4 selects the TMEM lane quadrant (token rows), the warpgroup
 //                   selects the 128-column half of the 256-wide tile.
 #include "common.h"
@@ -28,7 +41,7 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BN = kGemmBN;  // 256
-constexpr int BKC = 128;  // int8 codes per k-block (128-byte rows)
+constexpr int BKC = 128;  // one-byte codes per k-block (128-byte rows)
 constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_h chunk
 constexpr int BU_BYTES = BN * BKC;         // 32 KB  unpacked weight codes / bf16 W~_h chunk
@@ -36,8 +49,8 @@ constexpr int BP_BYTES = BN * BKC / 2;     // 16 KB  packed weight codes (TMA st
 constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB
 constexpr int SC_SLOTS = 8;
 constexpr int SC_SW_BYTES = 2 * BN * 4;    // up to two groups per k-block
-constexpr int SC_SX_BYTES = 2 * BM * 4;
-constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 3 KB
+constexpr int SC_SX_BYTES = 2 * 2 * BM * 4;  // scales of up to two groups, then their offset corrections
+constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 4 KB
 constexpr int NUM_THREADS = 384;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
@@ -68,6 +81,24 @@ __device__ __forceinline__ void flush_wait(int* status, int slot, long long cycl
     atomicAdd(reinterpret_cast<unsigned long long*>(status) + slot, static_cast<unsigned long long>(cycles));
 }
 
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+// Two independent IEEE fused multiply-adds in one instruction.
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -80,7 +111,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                  const GemmKernelParams p) {
     constexpr int GPK = BKC / G;       // groups per k-block: 2 (G = 64) or 1 (G = 128)
-    constexpr int MMA_PER_G = G / 32;  // kind::i8 instructions (K = 32) per group
+    constexpr int MMA_PER_G = G / 32;  // 8-bit MMA instructions (K = 32) per group
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -158,9 +189,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         const int slot = sc_it % SC_SLOTS;
                         if (!mbar_wait(scempty_bar(slot), ((sc_it / SC_SLOTS) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                         const uint32_t sc = sc_base + slot * SC_BYTES;
-                        mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + BM) * 4);
+                        mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + 2 * BM) * 4);
                         tma_load_2d(sc, &tmap_wscale, scfull_bar(slot), n0, kb * GPK);
                         tma_load_2d(sc + SC_SW_BYTES, &tmap_xscale, scfull_bar(slot), m0, kb * GPK);
+                        tma_load_2d(sc + SC_SW_BYTES + 2 * BM * 4, &tmap_xscale, scfull_bar(slot), m0, p.n_g + kb * GPK);
                     }
                     if (!ok) break;
                     for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
@@ -191,7 +223,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         } else if (warp == 1) {
             // -------------------------------------------------------- MMA issuer
             if (lane == 0) {
-                constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);
+                constexpr uint32_t idesc_f8 = umma_idesc(1 /*f32*/, 0 /*E4M3*/, BM, BN);
                 constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
                 uint32_t it = 0, git = 0;
                 long long w_ops = 0, w_tempty = 0;
@@ -215,7 +247,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
                             for (int k = 0; k < MMA_PER_G; ++k) {
                                 const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
-                                umma_i8(tmem_base + b * BN, adesc + 2 * kk, bdesc + 2 * kk, idesc_i8, k != 0);
+                                umma_f8f6f4(tmem_base + b * BN, adesc + 2 * kk, bdesc + 2 * kk, idesc_f8, k != 0);
                             }
                             umma_commit(tfull_bar(b));
                         }
@@ -249,7 +281,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 flush_wait(p.status, WS_KERNEL, clock64() - t_kernel);
             }
         } else {
-            // -------------------------------------------------------- INT4 -> INT8 unpack (warps 2, 3)
+            // -------------------------------------------------------- nibble -> byte unpack (warps 2, 3)
             const int u = threadIdx.x - 64;  // 0..63
             uint32_t it = 0;
             long long w_full = 0;
@@ -275,10 +307,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                             const uint4 pk = src[64 * j];
                             // low nibbles of a word are codes k..k+3, high nibbles k+4..k+7 (see prepare.cu)
                             uint4 o0, o1;
-                            o0.x = (pk.x << 4) & 0xF0F0F0F0u; o0.y = pk.x & 0xF0F0F0F0u;
-                            o0.z = (pk.y << 4) & 0xF0F0F0F0u; o0.w = pk.y & 0xF0F0F0F0u;
-                            o1.x = (pk.z << 4) & 0xF0F0F0F0u; o1.y = pk.z & 0xF0F0F0F0u;
-                            o1.z = (pk.w << 4) & 0xF0F0F0F0u; o1.w = pk.w & 0xF0F0F0F0u;
+                            o0.x = pk.x & 0x0F0F0F0Fu; o0.y = (pk.x >> 4) & 0x0F0F0F0Fu;
+                            o0.z = pk.y & 0x0F0F0F0Fu; o0.w = (pk.y >> 4) & 0x0F0F0F0Fu;
+                            o1.x = pk.z & 0x0F0F0F0Fu; o1.y = (pk.z >> 4) & 0x0F0F0F0Fu;
+                            o1.z = pk.w & 0x0F0F0F0Fu; o1.w = (pk.w >> 4) & 0x0F0F0F0Fu;
                             *reinterpret_cast<uint4*>(d0 + j * 2048) = o0;  // 16 rows of 128 bytes further down
                             *reinterpret_cast<uint4*>(d1 + j * 2048) = o1;
                         }
@@ -293,9 +325,15 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     } else {
         reg_alloc<208>();
         // ------------------------------------------------------------ epilogue (warps 4..11)
+        // A warp owns 32 token rows (its TMEM lane quadrant) x 128 columns.  The accumulators are read with the
+        // 16x256b shape: a thread then holds 4 rows (l/4 + 8 i) x the column pairs 2 (l%4) + {0, 1} of every block
+        // of 8 columns, so one 8-byte load of weight scales serves four rows (with the 32x32b shape, one row per
+        // thread, every thread would need all 128 column scales of every group and the shared-memory pipe, not the
+        // FMA pipe, would bound the kernel).
         const int q = warp & 3;
         const int half = (warp - 4) >> 2;
-        const int row_in_tile = q * 32 + lane;
+        const int lr4 = lane >> 2;        // row inside a group of 8
+        const int lc2 = (lane & 3) * 2;   // first of this thread's two columns inside a block of 8
         uint32_t git = 0, sc_it = 0;
         long long w_tfull = 0, w_sc = 0;
         const long long t_epi = clock64();
@@ -303,11 +341,11 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
-            const int row = m0 + row_in_tile;
+            const int rbase = m0 + q * 32 + lr4;  // this thread's rows: rbase + 8 i, i = 0..3
             const int colbase = n0 + half * 128;
-            float acc[128];
+            uint64_t acc[64];  // [(chunk c of 16 columns) * 2 + (block cb of 8 columns)] * 4 + row i : one column pair
 #pragma unroll
-            for (int j = 0; j < 128; ++j) acc[j] = 0.f;
+            for (int j = 0; j < 64; ++j) acc[j] = 0ull;
 
             for (int kb = 0; ok && kb < p.num_kb; ++kb, ++sc_it) {
                 const int slot = sc_it % SC_SLOTS;
@@ -323,41 +361,68 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     ok = __any_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    // operand B carries 16*q_w: fold the 1/16 into the activation scale (exact)
-                    const float sx = s_sx[gi * BM + row_in_tile] * 0.0625f;
-                    const float* swp = s_sw + gi * BN + half * 128;
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
+                    // the accumulator holds S = 2^-18 sum q_x (q_w + 8):  s_x P = fma(S, 2^18 s_x, e),  e = -8 s_x sum q_x
+                    uint64_t sx2[4], e2[4];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t raw[32];
-                        tmem_ld_32x32b_x32(taddr + c * 32, raw);
+                    for (int i = 0; i < 4; ++i) {
+                        const float sxs = s_sx[gi * BM + q * 32 + lr4 + 8 * i] * 262144.0f;
+                        const float e = s_sx[(2 + gi) * BM + q * 32 + lr4 + 8 * i];
+                        sx2[i] = pack_f32x2(__float_as_uint(sxs), __float_as_uint(sxs));
+                        e2[i] = pack_f32x2(__float_as_uint(e), __float_as_uint(e));
+                    }
+                    const float* swp = s_sw + gi * BN + half * 128 + lc2;
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
+                    // software pipeline over eight 16-column chunks: the loads of chunk c+1 are in flight while
+                    // chunk c is folded in (tcgen05.wait::ld waits for every outstanding load, hence depth one)
+                    uint32_t raw[2][16];  // [0..7]: TMEM lanes 0..15 of the quadrant (rows i = 0, 1), [8..15]: lanes 16..31
+                    tmem_ld_16x256b_x2(taddr, raw[0]);
+                    tmem_ld_16x256b_x2(taddr + (16u << 16), raw[0] + 8);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t (&cur)[16] = raw[c & 1];
+                        // this chunk's weight scales: requested before the wait so that their latency hides behind it
+                        uint64_t w[2];
+                        if constexpr (!kPartials) {
+                            w[0] = *reinterpret_cast<const uint64_t*>(swp + c * 16);
+                            w[1] = *reinterpret_cast<const uint64_t*>(swp + c * 16 + 8);
+                        }
                         tmem_ld_wait();
-                        if (c == 3) {
+                        tmem_ld_fence(cur);
+                        if (c < 7) {
+                            tmem_ld_16x256b_x2(taddr + (c + 1) * 16, raw[(c + 1) & 1]);
+                            tmem_ld_16x256b_x2(taddr + (16u << 16) + (c + 1) * 16, raw[(c + 1) & 1] + 8);
+                        } else {
                             // the whole tile is in registers: hand it back to the MMA warp
                             tc_fence_before_sync();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(tempty_bar(b));
                         }
-                        if constexpr (kPartials) {
-                            if (row < p.M) {
-                                const int g = kb * GPK + gi;
-                                int32_t* dst = p.partials + (static_cast<size_t>(g) * p.M + row) * p.N + colbase + c * 32;
 #pragma unroll
-                                for (int j = 0; j < 32; j += 4) {
-                                    if (colbase + c * 32 + j < p.N)
-                                        *reinterpret_cast<int4*>(dst + j) =
-                                            make_int4(static_cast<int32_t>(raw[j]) >> 4, static_cast<int32_t>(raw[j + 1]) >> 4,
-                                                      static_cast<int32_t>(raw[j + 2]) >> 4, static_cast<int32_t>(raw[j + 3]) >> 4);
+                        for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                            for (int cb = 0; cb < 2; ++cb) {
+#pragma unroll
+                                for (int rr = 0; rr < 2; ++rr) {
+                                    const int i = 2 * h + rr;
+                                    const int pidx = 8 * h + 4 * cb + 2 * rr;
+                                    if constexpr (kPartials) {
+                                        // unit scales here: fma(S, 2^18, -8 sum q_x) = P, an integer
+                                        float sxs, sxs_, e, e_;
+                                        unpack_f32x2(sx2[i], sxs, sxs_);
+                                        unpack_f32x2(e2[i], e, e_);
+                                        const int row = rbase + 8 * i;
+                                        const int col = colbase + c * 16 + cb * 8 + lc2;
+                                        if (row < p.M && col < p.N) {
+                                            const int g = kb * GPK + gi;
+                                            *reinterpret_cast<int2*>(p.partials + (static_cast<size_t>(g) * p.M + row) * p.N + col) =
+                                                make_int2(__float2int_rn(fmaf(__uint_as_float(cur[pidx]), sxs, e)),
+                                                          __float2int_rn(fmaf(__uint_as_float(cur[pidx + 1]), sxs, e)));
+                                        }
+                                    } else {
+                                        const uint64_t t = ffma2(pack_f32x2(cur[pidx], cur[pidx + 1]), sx2[i], e2[i]);
+                                        acc[(c * 2 + cb) * 4 + i] = ffma2(t, w[cb], acc[(c * 2 + cb) * 4 + i]);
+                                    }
                                 }
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                const float4 w = *reinterpret_cast<const float4*>(swp + c * 32 + j);
-                                acc[c * 32 + j + 0] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 0])) * w.x, sx, acc[c * 32 + j + 0]);
-                                acc[c * 32 + j + 1] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 1])) * w.y, sx, acc[c * 32 + j + 1]);
-                                acc[c * 32 + j + 2] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 2])) * w.z, sx, acc[c * 32 + j + 2]);
-                                acc[c * 32 + j + 3] = fmaf(static_cast<float>(static_cast<int32_t>(raw[j + 3])) * w.w, sx, acc[c * 32 + j + 3]);
                             }
                         }
                     }
@@ -375,13 +440,24 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
+                const uint64_t one2 = pack_f32x2(0x3F800000u, 0x3F800000u);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t raw[32];
-                    tmem_ld_32x32b_x32(taddr + c * 32, raw);
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t raw[16];
+                    tmem_ld_16x256b_x2(taddr + c * 16, raw);
+                    tmem_ld_16x256b_x2(taddr + (16u << 16) + c * 16, raw + 8);
                     tmem_ld_wait();
+                    tmem_ld_fence(raw);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[c * 32 + j] += __uint_as_float(raw[j]);
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int cb = 0; cb < 2; ++cb)
+#pragma unroll
+                            for (int rr = 0; rr < 2; ++rr) {
+                                const int pidx = 8 * h + 4 * cb + 2 * rr;
+                                acc[(c * 2 + cb) * 4 + 2 * h + rr] =
+                                    ffma2(pack_f32x2(raw[pidx], raw[pidx + 1]), one2, acc[(c * 2 + cb) * 4 + 2 * h + rr]);
+                            }
                 }
                 tc_fence_before_sync();
                 __syncwarp();
@@ -389,19 +465,20 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 ++git;
             }
             if constexpr (!kPartials) {
-                if (row < p.M) {
-                    uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + colbase;
 #pragma unroll
-                    for (int j = 0; j < 128; j += 8) {
-                        if (colbase + j < p.N) {
-                            const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + colbase + j));
-                            const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + colbase + j + 4));
-                            uint4 o;
-                            o.x = pack_bf16x2(acc[j + 0] + b0.x, acc[j + 1] + b0.y);
-                            o.y = pack_bf16x2(acc[j + 2] + b0.z, acc[j + 3] + b0.w);
-                            o.z = pack_bf16x2(acc[j + 4] + b1.x, acc[j + 5] + b1.y);
-                            o.w = pack_bf16x2(acc[j + 6] + b1.z, acc[j + 7] + b1.w);
-                            *reinterpret_cast<uint4*>(yrow + j) = o;
+                for (int cc = 0; cc < 16; ++cc) {  // blocks of 8 columns
+                    const int col = colbase + cc * 8 + lc2;
+                    if (col < p.N) {
+                        const float2 bv = __ldg(reinterpret_cast<const float2*>(p.bias + col));
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int row = rbase + 8 * i;
+                            if (row < p.M) {
+                                float a0, a1;
+                                unpack_f32x2(acc[cc * 4 + i], a0, a1);
+                                *reinterpret_cast<uint32_t*>(p.y + static_cast<size_t>(row) * p.N + col) =
+                                    pack_bf16x2(a0 + bv.x, a1 + bv.y);
+                            }
                         }
                     }
                 }
@@ -432,7 +509,7 @@ dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaS
     st = encode_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K_lp, (uint64_t)a.M,
                         (uint64_t)g.K_lp, BKC, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != DIROTQ_OK) return st;
-    st = encode_tmap_2d(&tmap_xscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xscale, (uint64_t)a.ldm, (uint64_t)g.n_g,
+    st = encode_tmap_2d(&tmap_xscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xscale, (uint64_t)a.ldm, (uint64_t)2 * g.n_g,
                         (uint64_t)a.ldm * 4, BM, BKC / g.G, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != DIROTQ_OK) return st;
     st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,

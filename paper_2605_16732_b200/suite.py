@@ -44,13 +44,28 @@ def _householder(K: int, seed: int) -> torch.Tensor:
     return torch.eye(K, dtype=torch.float64, device="cuda") - 2.0 * torch.outer(v, v)
 
 
+FMT = "int4"  # set from --fmt: "int4" (groups of G, bf16 scales) or "nvfp4" (blocks of 16, E4M3 scales)
+
+
 class Case:
     def __init__(self, M, K, N, r, G, model):
         self.M, self.K, self.N, self.r, self.G = M, K, N, r, G
-        spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=model, seed=7)
+        spec = synth.LayerSpec(K=K, N=N, r=r, G=G if FMT == "int4" else 64, model=model, seed=7)
         W, bias = synth.make_weights(spec)
-        self.layer = dq.dirotq_prepare_layer(torch.from_numpy(W).cuda(), _householder(K, K + r), r, G, bias=_bf(bias))
         self.x = _bf(synth.make_tokens(spec, M, batch_seed=11))
+        Wd, Q = torch.from_numpy(W).cuda(), _householder(K, K + r)
+        if FMT == "nvfp4":
+            # calibrate the activations' power-of-two scale on this batch through the library's own rotation
+            probe = dq.dirotq_prepare_layer_nvfp4(Wd, Q, r, 0, bias=_bf(bias))
+            rows = min(M, 1024)
+            xrot = torch.empty((rows, K), dtype=torch.float32, device="cuda")
+            dq.dirotq_rotate_quantize(self.x[:rows], probe, dq.alloc_workspace(probe, rows), xrot)
+            amax = float(xrot[:, r:].abs().max().item())
+            probe.close()
+            ex = int(np.ceil(np.log2(amax / 1536.0)))
+            self.layer = dq.dirotq_prepare_layer_nvfp4(Wd, Q, r, ex, bias=_bf(bias))
+        else:
+            self.layer = dq.dirotq_prepare_layer(Wd, Q, r, G, bias=_bf(bias))
         self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
         self.ws = dq.alloc_workspace(self.layer, M)
         self.Wb = (torch.from_numpy(W).cuda()).to(torch.bfloat16)
@@ -91,12 +106,15 @@ class Case:
         K_l = K - r
         n_g = -(-K_l // G)
         tot = rot + gem
-        p_i8 = 2.0 * p_bf16
+        p_i8 = (4.0 if FMT == "nvfp4" else 2.0) * p_bf16  # nominal ratio of the 4-bit / 8-bit tensor peak to bf16
         t_roof = (2.0 * M * K_l * N / p_i8 + (2.0 * M * K * K + 2.0 * M * r * N) / p_bf16) / 1e12 * 1e3
-        bytes_alg = 2 * M * K + 2 * K * K + n_g * G * N / 2 + 4 * n_g * N + 2 * 64 * N + 2 * (M * n_g * G + 4 * M * n_g + 2 * M * 64) + 2 * M * N
-        line = {"config": tag, "M": M, "K": K, "N": N, "r": r, "group": G, "rotate_ms": rot, "gemm_ms": gem,
+        if FMT == "nvfp4":
+            bytes_alg = 2 * M * K + 2 * K * K + K_l * N / 2 + K_l / 16 * N + 2 * 64 * N + 2 * (M * K_l / 2 + M * K_l / 16 + 2 * M * 64) + 2 * M * N
+        else:
+            bytes_alg = 2 * M * K + 2 * K * K + n_g * G * N / 2 + 4 * n_g * N + 2 * 64 * N + 2 * (M * n_g * G + 4 * M * n_g + 2 * M * 64) + 2 * M * N
+        line = {"config": tag, "fmt": FMT, "M": M, "K": K, "N": N, "r": r, "group": G, "rotate_ms": rot, "gemm_ms": gem,
                 "effective_tops": 2.0 * M * N * K / (tot * 1e-3) / 1e12,
-                "frac_int8_peak": 2.0 * M * N * K / (tot * 1e-3) / 1e12 / p_i8,
+                "frac_low_precision_peak": 2.0 * M * N * K / (tot * 1e-3) / 1e12 / p_i8,
                 "frac_of_composite_roofline": t_roof / tot,
                 "algorithmic_gbs": bytes_alg / (tot * 1e-3) / 1e9, "frac_hbm_peak": bytes_alg / (tot * 1e-3) / 1e9 / hbm,
                 "cublas_bf16_ms": cb, "speedup_vs_cublas_bf16": cb / tot}
@@ -110,10 +128,14 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,4,5")
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4"])
+    ap.add_argument("--ranks", default="16,32,64,128", help="ranks swept by config 4")
     args = ap.parse_args()
+    global FMT
+    FMT = args.fmt
     todo = set(args.configs.split(","))
     p_bf16, hbm, src = _peaks()
-    print(json.dumps({"peaks": {"bf16_tflops_sustained": p_bf16, "int8_tops": 2 * p_bf16, "hbm_gbs": hbm, "source": src}}), flush=True)
+    print(json.dumps({"peaks": {"bf16_tflops_sustained": p_bf16, "int8_tops": 2 * p_bf16, "fp4_tflops_nominal_ratio": 4 * p_bf16, "fmt": FMT, "hbm_gbs": hbm, "source": src}}), flush=True)
 
     if "1" in todo:
         c = Case(256, 1152, 1152, 32, 64, synth.PIXART)
@@ -126,8 +148,8 @@ def main():
             c.close()
     if "4" in todo:
         for K, N in [(3072, 9216), (12288, 3072)]:
-            for r in (16, 32, 64, 128):
-                for G in (64, 128):
+            for r in [int(v) for v in args.ranks.split(",")]:
+                for G in ((64, 128) if FMT == "int4" else (16,)):
                     c = Case(18432, K, N, r, G, synth.FLUX)
                     c.report("4: FLUX batch 4 (M=18432) rank/group sweep", max(5, args.iters // 2), p_bf16, hbm)
                     c.close()

@@ -142,3 +142,41 @@ def test_wait_counters_are_reported():
     assert c["epilogue_wait_accumulator"] <= c["epilogue_total"]
     assert c["mma_wait_operands"] + c["mma_wait_accumulator"] <= c["mma_role_total"]
     layer.close()
+
+
+@pytest.mark.parametrize("G", [64, 128])
+def test_group_sums_exact_on_codes_built_to_lose_low_bits(G):
+    """The group sums come out of a floating-point accumulator (products of small integers, scaled by a power
+    of two): they must still equal the integer sums bit for bit when the sum is as large as it can get and
+    single +-1 products are added to or cancelled against long runs of +-49."""
+    K, N, r, M = 2 * 128 + 128, 256, 128, 128
+    K_l = K - r
+    rng = np.random.default_rng(5)
+    # identity rotation: the folded weight is W itself; every |w| equal in a group -> every weight code is +-7
+    Q = np.eye(K)
+    sign = rng.choice([-1.0, 1.0], size=(K, N))
+    sign[:, :64] = 1.0  # a block of columns with all codes +7
+    W = (0.02 * sign).astype(np.float32)
+    lo = orc.prepare_layer(W, Q, r, G, want_t=True)
+    assert np.all(np.abs(lo["wcodes"]) == 7)
+    layer = dq.dirotq_prepare_layer(torch.from_numpy(W).cuda(), torch.from_numpy(Q).cuda(), r, G)
+    codes = np.zeros((M, K_l), dtype=np.int8)
+    codes[0:16] = 7                                             # largest sum: G * 49
+    codes[16:32] = -7
+    for m in range(32, 64):                                     # a long run of 7s, then 1s
+        codes[m] = 7
+        codes[m, K_l - 1 - (m - 32):] = 1
+    for m in range(64, 96):                                     # cancellation down to a small remainder
+        codes[m, 0::2] = 7
+        codes[m, 1::2] = -7
+        codes[m, 2 * (m - 64)] = 6
+    codes[96:] = rng.integers(-7, 8, size=(M - 96, K_l))
+    ws = dq.alloc_workspace(layer, M)
+    padded = np.zeros((M, layer.K_lp), dtype=np.int8)
+    padded[:, :K_l] = codes
+    P = dq.dirotq_int_gemm_debug(torch.from_numpy(padded).cuda(), layer, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    ref = orc.int_gemm(codes, lo["wcodes"], G)
+    assert int(np.abs(ref).max()) == G * 49
+    assert np.array_equal(P.cpu().numpy(), ref)
+    layer.close()
