@@ -71,6 +71,7 @@ enum WaitSlot : int { WS_PROD_EMPTY = 1, WS_MMA_OPERANDS = 2, WS_MMA_TEMPTY = 3,
 
 __device__ __forceinline__ bool timed_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
                                            long long& acc) {
+    if (mbar_try_wait(bar, parity)) return true;  // the common case costs no clock reads
     const long long t0 = clock64();
     const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
     acc += clock64() - t0;
@@ -302,17 +303,25 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         const int c = u & 3, sw = (u >> 2) & 7;
                         uint8_t* d0 = st + A_BYTES + (u >> 2) * 128 + (((2 * c) ^ sw) << 4);
                         uint8_t* d1 = st + A_BYTES + (u >> 2) * 128 + (((2 * c + 1) ^ sw) << 4);
+                        // The loads of a batch are issued before any of its stores: the compiler cannot prove that the
+                        // staging buffer and the operand tile do not overlap, so a load written after a store would wait
+                        // for it and the whole unpack would run as one dependent chain.
 #pragma unroll
-                        for (int j = 0; j < (BN * 4) / 64; ++j) {
-                            const uint4 pk = src[64 * j];
-                            // low nibbles of a word are codes k..k+3, high nibbles k+4..k+7 (see prepare.cu)
-                            uint4 o0, o1;
-                            o0.x = pk.x & 0x0F0F0F0Fu; o0.y = (pk.x >> 4) & 0x0F0F0F0Fu;
-                            o0.z = pk.y & 0x0F0F0F0Fu; o0.w = (pk.y >> 4) & 0x0F0F0F0Fu;
-                            o1.x = pk.z & 0x0F0F0F0Fu; o1.y = (pk.z >> 4) & 0x0F0F0F0Fu;
-                            o1.z = pk.w & 0x0F0F0F0Fu; o1.w = (pk.w >> 4) & 0x0F0F0F0Fu;
-                            *reinterpret_cast<uint4*>(d0 + j * 2048) = o0;  // 16 rows of 128 bytes further down
-                            *reinterpret_cast<uint4*>(d1 + j * 2048) = o1;
+                        for (int jb = 0; jb < (BN * 4) / 64; jb += 8) {
+                            uint4 pk[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) pk[j] = src[64 * (jb + j)];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                // low nibbles of a word are codes k..k+3, high nibbles k+4..k+7 (see prepare.cu)
+                                uint4 o0, o1;
+                                o0.x = pk[j].x & 0x0F0F0F0Fu; o0.y = (pk[j].x >> 4) & 0x0F0F0F0Fu;
+                                o0.z = pk[j].y & 0x0F0F0F0Fu; o0.w = (pk[j].y >> 4) & 0x0F0F0F0Fu;
+                                o1.x = pk[j].z & 0x0F0F0F0Fu; o1.y = (pk[j].z >> 4) & 0x0F0F0F0Fu;
+                                o1.z = pk[j].w & 0x0F0F0F0Fu; o1.w = (pk[j].w >> 4) & 0x0F0F0F0Fu;
+                                *reinterpret_cast<uint4*>(d0 + (jb + j) * 2048) = o0;  // 16 rows of 128 bytes further down
+                                *reinterpret_cast<uint4*>(d1 + (jb + j) * 2048) = o1;
+                            }
                         }
                         fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core
                     }
@@ -465,21 +474,39 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 ++git;
             }
             if constexpr (!kPartials) {
+                // A lane holds 2 of the 8 columns of every block; four blocks are transposed inside the quad of lanes
+                // (two exchange steps) so that each lane ends up with all 8 columns = 16 bytes of one block and the
+                // warp writes 64 contiguous bytes per row.
+                const int j = lane & 3;
 #pragma unroll
-                for (int cc = 0; cc < 16; ++cc) {  // blocks of 8 columns
-                    const int col = colbase + cc * 8 + lc2;
-                    if (col < p.N) {
-                        const float2 bv = __ldg(reinterpret_cast<const float2*>(p.bias + col));
+                for (int m = 0; m < 4; ++m) {
+                    float2 bv[4];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int row = rbase + 8 * i;
-                            if (row < p.M) {
-                                float a0, a1;
-                                unpack_f32x2(acc[cc * 4 + i], a0, a1);
-                                *reinterpret_cast<uint32_t*>(p.y + static_cast<size_t>(row) * p.N + col) =
-                                    pack_bf16x2(a0 + bv.x, a1 + bv.y);
-                            }
+                    for (int t = 0; t < 4; ++t) {
+                        const int col = colbase + (4 * m + t) * 8 + lc2;
+                        bv[t] = col < p.N ? __ldg(reinterpret_cast<const float2*>(p.bias + col)) : make_float2(0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t v[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            float a0, a1;
+                            unpack_f32x2(acc[(4 * m + t) * 4 + i], a0, a1);
+                            v[t] = pack_bf16x2(a0 + bv[t].x, a1 + bv[t].y);
                         }
+                        const bool odd = (j & 1) != 0, upper = (j & 2) != 0;
+                        const uint32_t r01 = __shfl_xor_sync(0xffffffffu, odd ? v[0] : v[1], 1);
+                        const uint32_t r23 = __shfl_xor_sync(0xffffffffu, odd ? v[2] : v[3], 1);
+                        const uint32_t u0 = odd ? r01 : v[0], u1 = odd ? v[1] : r01;  // block (j & 1), lanes 2 (j / 2) + {0, 1}
+                        const uint32_t p0 = odd ? r23 : v[2], p1 = odd ? v[3] : r23;  // block 2 + (j & 1)
+                        const uint32_t x0 = __shfl_xor_sync(0xffffffffu, upper ? u0 : p0, 2);
+                        const uint32_t x1 = __shfl_xor_sync(0xffffffffu, upper ? u1 : p1, 2);
+                        const uint4 o = upper ? make_uint4(x0, x1, p0, p1) : make_uint4(u0, u1, x0, x1);  // block j
+                        const int row = rbase + 8 * i;
+                        const int col = colbase + (4 * m + j) * 8;
+                        if (row < p.M && col < p.N)
+                            *reinterpret_cast<uint4*>(p.y + static_cast<size_t>(row) * p.N + col) = o;
                     }
                 }
             }
