@@ -104,7 +104,7 @@ def _shape_ops(M):
 # CPU oracle arm (bounded sample)
 
 
-def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0):
+def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0, fmt: str = "int4"):
     """Times the oracle's online steps on `rows` tokens x `cols` output columns of every linear."""
     from oracle import dirotq_oracle as orc
     from paper_2605_16732_b200 import synth
@@ -120,20 +120,27 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
         v /= np.linalg.norm(v)
         Q = np.eye(K) - 2.0 * np.outer(v, v)
         W = (0.02 * g.standard_normal((K, cols))).astype(np.float32)
-        lo = orc.prepare_layer(W, Q, RANK, GROUP)
         x = synth.make_tokens(spec, rows, batch_seed=5)
+        if fmt == "nvfp4":
+            lo = orc.nvfp4_prepare_layer(W, Q, RANK)
+            lo["ex"] = orc.nvfp4_global_exponent(float(np.abs(orc.rotate(x, lo["Qb"])[:, RANK:]).max()))
+        else:
+            lo = orc.prepare_layer(W, Q, RANK, GROUP)
         layers.append((lo, x, K, cols))
     times = []
     for _ in range(steps):
         t0 = time.perf_counter()
         for lo, x, K, n in layers:
-            orc.linear_deployed(x, lo, bias=None, want_t=False)
+            if fmt == "nvfp4":
+                orc.nvfp4_linear_deployed(x, lo, lo["ex"], bias=None, want_t=False)
+            else:
+                orc.linear_deployed(x, lo, bias=None, want_t=False)
         times.append(time.perf_counter() - t0)
     ops = sum(2.0 * rows * n * K for _, _, K, n in layers)
     t = float(np.mean(times))
     return {"value": ops / t / 1e12, "unit": "TOPS", "cores": orc.num_threads(), "kind": "oracle",
             "sample": f"{rows} token rows x {cols} output columns of each of the 4 linears, online steps only "
-                      f"(rotation, quantize, int GEMM, combine); Householder rotation",
+                      f"(rotation, quantize, {'block-scaled products' if fmt == 'nvfp4' else 'int GEMM'}, combine); Householder rotation",
             "seconds_per_step": t}
 
 
@@ -143,13 +150,15 @@ def run_reference(args):
         return
     steps = max(1, args.steps)
     for _ in range(min(args.warmup, 1)):
-        oracle_sample_run(1)
-    res = oracle_sample_run(steps)
+        oracle_sample_run(1, fmt=args.fmt)
+    res = oracle_sample_run(steps, fmt=args.fmt)
     line = {
         "impl": "reference", "metric": "dirotq_w4a4_linear_effective_tops", "value": res["value"], "unit": "TOPS",
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4xint4->int32 + bf16",
-        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": res["sample"]},
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64 (oracle; nvfp4 codes)" if args.fmt == "nvfp4" else "f64 + int32 (oracle; int4 codes)",
+        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else ""), "format": args.fmt,
+                                        "sample": res["sample"]},
         "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": res["value"], "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -354,7 +363,7 @@ def run_ours(args):
             "cublas_bf16_ms": cublas.get(n), "speedup_vs_cublas_bf16": cublas[n] / tot if n in cublas else None,
         }
 
-    cpu = oracle_sample_run(1) if not args.lite else {"value": None, "unit": "TOPS", "cores": None, "kind": "oracle",
+    cpu = oracle_sample_run(1, fmt=args.fmt) if not args.lite else {"value": None, "unit": "TOPS", "cores": None, "kind": "oracle",
                                                       "sample": "skipped (--lite)"}
     line = {
         "metric": "dirotq_w4a4_linear_effective_tops", "value": value, "unit": "TOPS", "n_gpus": world,
