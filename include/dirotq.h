@@ -111,8 +111,8 @@ DIROTQ_API dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K
 
 /* y[M,N] (bf16, row-major) = DiRotQ-linear(x[M,K] bf16 row-major).  Two kernels are enqueued:
  * rotate+split+quantize (x Q_b on the bf16 tensor cores, Eq. 1 in the epilogue), then the
- * INT4 x INT4 group GEMM on the int8 tensor cores with the per-group rescale, the bf16 rank-r
- * branch and the bias.  Concurrent calls on one layer need distinct workspaces. */
+ * INT4 x INT4 group GEMM on the 8-bit tensor-core path (exact integer group sums) with the
+ * per-group rescale, the bf16 rank-r branch and the bias.  Concurrent calls on one layer need distinct workspaces. */
 DIROTQ_API dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer, void* y, void* workspace,
                               size_t workspace_bytes, dirotq_stream_t stream);
 

@@ -1,6 +1,6 @@
 // Tensor-pipe issue-rate probe: every SM issues back-to-back tcgen05.mma instructions on operands
 // that already sit in shared memory (no TMA, no epilogue).  Used by the benchmark to measure the
-// dense int8 and bf16 MMA rates of the part the roofline fractions are quoted against.
+// dense 8-bit (int8, E4M3) and bf16 MMA rates of the part the roofline fractions are quoted against.
 #include "common.h"
 #include "ptx.cuh"
 

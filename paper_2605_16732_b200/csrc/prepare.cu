@@ -5,9 +5,10 @@
 //
 // Packed weight-code layout, row n of u8 [N][K_lp/2] (K-major): codes are taken 32 at a time
 // (16 bytes); inside such a piece, byte 4*j + b (j, b in 0..3) holds code 8*j + b in its low
-// nibble and code 8*j + 4 + b in its high nibble (two's complement nibbles).  With this order the
+// nibble and code 8*j + 4 + b in its high nibble; a nibble holds u = q + 8 (1..15).  With this order the
 // online unpack of a 32-bit word is two logic ops per four codes:
-//   (w << 4) & 0xF0F0F0F0  ->  codes 8j..8j+3 as bytes 16*q,      w & 0xF0F0F0F0  ->  codes 8j+4..8j+7.
+//   w & 0x0F0F0F0F  ->  codes 8j..8j+3 as bytes 0000uuuu,      (w >> 4) & 0x0F0F0F0F  ->  codes 8j+4..8j+7,
+// and a byte 0000uuuu read as E4M3 is u * 2^-9 exactly (see w4a4_gemm.cu).
 #include "common.h"
 
 #include <cuda_bf16.h>
