@@ -117,3 +117,66 @@ def test_config4_rank_group_sweep(K, N, r, G):
 @pytest.mark.parametrize("K,N", [(3072, 21504), (15360, 3072)])
 def test_config5_single_stream_shapes(K, N):
     print(_run(4608, K, N, 32, 64, synth.FLUX))
+
+
+# ------------------------------------------------------------------ NVFP4 variant at the benchmark's sizes
+
+def _run_nvfp4(M, K, N, r, model, n_rows=24, n_cols=96, seed=0):
+    from parity_utils import check_activation_side_nvfp4, check_layer_output_nvfp4, _codes_equal_mod_zero
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=64, model=model, seed=seed)
+    Q = _rotation(spec)
+    W, bias = synth.make_weights(spec)
+    x_bits = synth.make_tokens(spec, M, batch_seed=3)
+    g = np.random.default_rng(K * 7 + N + 1)
+    rows = np.sort(g.choice(M, size=min(n_rows, M), replace=False))
+    rows[-1] = M - 1
+    cols = np.sort(g.choice(N, size=n_cols, replace=False))
+    cols[-1] = N - 1
+
+    # The weights' per-tensor exponent depends on ALL columns (max |W~_l|): the oracle folds the whole weight.
+    lo_full = orc.nvfp4_prepare_layer(W, Q, r, want_t=True)
+    lo = dict(lo_full)
+    lo["wcodes"], lo["wsf"], lo["Wh"] = lo_full["wcodes"][:, cols], lo_full["wsf"][:, cols], lo_full["Wh"][:, cols]
+    bias_s = bias[cols]
+    xt = orc.rotate(x_bits[rows], lo["Qb"])
+    ex = orc.nvfp4_global_exponent(float(np.abs(xt[:, r:]).max()))
+    oo = orc.nvfp4_linear_deployed(x_bits[rows], lo, ex, bias=bias_s)
+
+    Qd = torch.from_numpy(Q).cuda()
+    layer = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).cuda(), Qd, r, ex, bias=bits_to_bf16_tensor(bias))
+    del Qd
+    wcodes, wsf, wh, qb, ew = dq.dirotq_layer_export_nvfp4(layer)
+    assert ew == lo_full["ew"]
+    assert np.array_equal(bf16_tensor_to_bits(qb), lo["Qb"]), "bf16 rotation differs"
+    del qb
+    cols_t = torch.from_numpy(cols).cuda()
+    assert np.array_equal(wsf[:, cols_t].cpu().numpy(), lo["wsf"])
+    assert np.array_equal(bf16_tensor_to_bits(wh[:, cols_t]), lo["Wh"])
+    bad = ~_codes_equal_mod_zero(wcodes[:, cols_t].cpu().numpy(), lo["wcodes"])
+    assert bad.sum() <= 2
+    del wcodes, wsf, wh
+
+    x = bits_to_bf16_tensor(x_bits)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = dq.alloc_workspace(layer, M)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, sf = dq.dirotq_workspace_export_nvfp4(layer, M, ws)
+    rows_t = torch.from_numpy(rows).cuda()
+    xh_b = bf16_tensor_to_bits(xh[rows_t])
+    codes_n = codes[rows_t].cpu().numpy()
+    sf_n = sf[rows_t].cpu().numpy()
+    stats = check_activation_side_nvfp4(None, xh_b, codes_n, sf_n, oo, r, ex)
+    y_s = bf16_tensor_to_bits(y[rows_t][:, cols_t])
+    stats.update(check_layer_output_nvfp4(y_s, xh_b, codes_n, sf_n, ex, lo, oo, bias_s))
+    layer.close()
+    return stats
+
+
+@pytest.mark.parametrize("K,N", [(3072, 9216), (12288, 3072)])
+def test_nvfp4_flux_linears(K, N):
+    print(_run_nvfp4(4608, K, N, 32, synth.FLUX))
+
+
+def test_nvfp4_batch4_rank128():
+    print(_run_nvfp4(18432, 3072, 9216, 128, synth.FLUX))
