@@ -352,9 +352,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             const int n0 = (tile / num_m_blocks) * BN;
             const int rbase = m0 + q * 32 + lr4;  // this thread's rows: rbase + 8 i, i = 0..3
             const int colbase = n0 + half * 128;
-            uint64_t acc[64];  // [(chunk c of 16 columns) * 2 + (block cb of 8 columns)] * 4 + row i : one column pair
+            float accf[128];  // [((chunk c) * 2 + (block cb)) * 4 + row i] * 2 + {0, 1}
 #pragma unroll
-            for (int j = 0; j < 64; ++j) acc[j] = 0ull;
+            for (int j = 0; j < 128; ++j) accf[j] = 0.f;
 
             for (int kb = 0; ok && kb < p.num_kb; ++kb, ++sc_it) {
                 const int slot = sc_it % SC_SLOTS;
@@ -371,13 +371,11 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     if (!ok) break;
                     tc_fence_after_sync();
                     // the accumulator holds S = 2^-18 sum q_x (q_w + 8):  s_x P = fma(S, 2^18 s_x, e),  e = -8 s_x sum q_x
-                    uint64_t sx2[4], e2[4];
+                    float sxv[4], ev[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const float sxs = s_sx[gi * BM + q * 32 + lr4 + 8 * i] * 262144.0f;
-                        const float e = s_sx[(2 + gi) * BM + q * 32 + lr4 + 8 * i];
-                        sx2[i] = pack_f32x2(__float_as_uint(sxs), __float_as_uint(sxs));
-                        e2[i] = pack_f32x2(__float_as_uint(e), __float_as_uint(e));
+                        sxv[i] = s_sx[gi * BM + q * 32 + lr4 + 8 * i] * 262144.0f;
+                        ev[i] = s_sx[(2 + gi) * BM + q * 32 + lr4 + 8 * i];
                     }
                     const float* swp = s_sw + gi * BN + half * 128 + lc2;
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
@@ -390,10 +388,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     for (int c = 0; c < 8; ++c) {
                         uint32_t (&cur)[16] = raw[c & 1];
                         // this chunk's weight scales: requested before the wait so that their latency hides behind it
-                        uint64_t w[2];
+                        float2 w[2];
                         if constexpr (!kPartials) {
-                            w[0] = *reinterpret_cast<const uint64_t*>(swp + c * 16);
-                            w[1] = *reinterpret_cast<const uint64_t*>(swp + c * 16 + 8);
+                            w[0] = *reinterpret_cast<const float2*>(swp + c * 16);
+                            w[1] = *reinterpret_cast<const float2*>(swp + c * 16 + 8);
                         }
                         tmem_ld_wait();
                         tmem_ld_fence(cur);
@@ -416,9 +414,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                     const int pidx = 8 * h + 4 * cb + 2 * rr;
                                     if constexpr (kPartials) {
                                         // unit scales here: fma(S, 2^18, -8 sum q_x) = P, an integer
-                                        float sxs, sxs_, e, e_;
-                                        unpack_f32x2(sx2[i], sxs, sxs_);
-                                        unpack_f32x2(e2[i], e, e_);
+                                        const float sxs = sxv[i], e = ev[i];
                                         const int row = rbase + 8 * i;
                                         const int col = colbase + c * 16 + cb * 8 + lc2;
                                         if (row < p.M && col < p.N) {
@@ -428,8 +424,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                                           __float2int_rn(fmaf(__uint_as_float(cur[pidx + 1]), sxs, e)));
                                         }
                                     } else {
-                                        const uint64_t t = ffma2(pack_f32x2(cur[pidx], cur[pidx + 1]), sx2[i], e2[i]);
-                                        acc[(c * 2 + cb) * 4 + i] = ffma2(t, w[cb], acc[(c * 2 + cb) * 4 + i]);
+                                        const int a = ((c * 2 + cb) * 4 + i) * 2;
+                                        accf[a] = fmaf(fmaf(__uint_as_float(cur[pidx]), sxv[i], ev[i]), w[cb].x, accf[a]);
+                                        accf[a + 1] = fmaf(fmaf(__uint_as_float(cur[pidx + 1]), sxv[i], ev[i]), w[cb].y, accf[a + 1]);
                                     }
                                 }
                             }
@@ -449,7 +446,6 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
-                const uint64_t one2 = pack_f32x2(0x3F800000u, 0x3F800000u);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     uint32_t raw[16];
@@ -464,8 +460,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
                             for (int rr = 0; rr < 2; ++rr) {
                                 const int pidx = 8 * h + 4 * cb + 2 * rr;
-                                acc[(c * 2 + cb) * 4 + 2 * h + rr] =
-                                    ffma2(pack_f32x2(raw[pidx], raw[pidx + 1]), one2, acc[(c * 2 + cb) * 4 + 2 * h + rr]);
+                                const int a = ((c * 2 + cb) * 4 + 2 * h + rr) * 2;
+                                accf[a] += __uint_as_float(raw[pidx]);
+                                accf[a + 1] += __uint_as_float(raw[pidx + 1]);
                             }
                 }
                 tc_fence_before_sync();
@@ -491,9 +488,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         uint32_t v[4];
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
-                            float a0, a1;
-                            unpack_f32x2(acc[(4 * m + t) * 4 + i], a0, a1);
-                            v[t] = pack_bf16x2(a0 + bv[t].x, a1 + bv[t].y);
+                            const int a = ((4 * m + t) * 4 + i) * 2;
+                            v[t] = pack_bf16x2(accf[a] + bv[t].x, accf[a + 1] + bv[t].y);
                         }
                         const bool odd = (j & 1) != 0, upper = (j & 2) != 0;
                         const uint32_t r01 = __shfl_xor_sync(0xffffffffu, odd ? v[0] : v[1], 1);
