@@ -423,13 +423,34 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                                 make_int2(__float2int_rn(fmaf(__uint_as_float(cur[pidx]), sxs, e)),
                                                           __float2int_rn(fmaf(__uint_as_float(cur[pidx + 1]), sxs, e)));
                                         }
-                                    } else {
-                                        const int a = ((c * 2 + cb) * 4 + i) * 2;
-                                        accf[a] = fmaf(fmaf(__uint_as_float(cur[pidx]), sxv[i], ev[i]), w[cb].x, accf[a]);
-                                        accf[a + 1] = fmaf(fmaf(__uint_as_float(cur[pidx + 1]), sxv[i], ev[i]), w[cb].y, accf[a + 1]);
                                     }
                                 }
                             }
+                        }
+                        if constexpr (!kPartials) {
+                            // two passes, each ordered so that consecutive instructions share operands (the token's scale
+                            // and correction in the first, the column's weight scale in the second): shared operands come
+                            // from the operand-reuse latches instead of the register banks
+                            float t[16];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                for (int cb = 0; cb < 2; ++cb)
+#pragma unroll
+                                    for (int bit = 0; bit < 2; ++bit) {
+                                        const int pidx = 8 * (i >> 1) + 4 * cb + 2 * (i & 1) + bit;
+                                        t[pidx] = fmaf(__uint_as_float(cur[pidx]), sxv[i], ev[i]);
+                                    }
+#pragma unroll
+                            for (int cb = 0; cb < 2; ++cb)
+#pragma unroll
+                                for (int bit = 0; bit < 2; ++bit)
+#pragma unroll
+                                    for (int i = 0; i < 4; ++i) {
+                                        const int pidx = 8 * (i >> 1) + 4 * cb + 2 * (i & 1) + bit;
+                                        const int a = ((c * 2 + cb) * 4 + i) * 2 + bit;
+                                        accf[a] = fmaf(t[pidx], bit ? w[cb].y : w[cb].x, accf[a]);
+                                    }
                         }
                     }
                 }
