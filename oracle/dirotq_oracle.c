@@ -213,6 +213,109 @@ void dq_combine(const int32_t* P, const uint16_t* sx, const uint16_t* sw, const 
     }
 }
 
+/* =====================================================================================
+ * Asymmetric activation quantization (paper Sec. 3, Eq. 1 with z = min X,
+ * s = (max X - min X) / (q_max - q_min), q_min = 0, q_max = 2^4 - 1 = 15; Sec. 5.1: the 4-bit INT
+ * setting quantizes activations asymmetrically, weights symmetrically).
+ * Readings: both the scale and the zero-point are kept in 16 bits (bf16) and the ROUNDED values
+ * are the ones that divide and dequantize; the range max - min is taken before any rounding; a
+ * group whose elements are all equal has scale 0 and codes 0 (it dequantizes to z).
+ * "Parity unpinned" against the authors' implementation.
+ * ===================================================================================== */
+
+/* One group: codes u in 0..15 with x ~ s*u + z.  t (optional): pre-rounding quotients (x - z)/s. */
+void dq_quantize_group_asym(const double* v, int n, int64_t stride, uint16_t* scale_bits, uint16_t* zero_bits,
+                            uint8_t* codes, int64_t code_stride, double* t, int64_t t_stride) {
+    double lo = v[0], hi = v[0];
+    for (int i = 1; i < n; ++i) {
+        double x = v[i * stride];
+        if (x < lo) lo = x;
+        if (x > hi) hi = x;
+    }
+    uint16_t zb = dq_double_to_bf16(lo);                          /* z = min X */
+    uint16_t sb = (hi == lo) ? 0 : dq_double_to_bf16((hi - lo) / 15.0);   /* s = (max - min)/(q_max - q_min) */
+    double z = dq_bf16_to_double(zb), s = dq_bf16_to_double(sb);
+    *scale_bits = sb;
+    *zero_bits = zb;
+    for (int i = 0; i < n; ++i) {
+        double q = 0.0, ti = 0.0;
+        if (s != 0.0) {
+            ti = (v[i * stride] - z) / s;
+            q = rint(ti);                  /* half to even */
+            if (q > 15.0) q = 15.0;        /* clip to [q_min, q_max] */
+            if (q < 0.0) q = 0.0;
+        }
+        codes[i * code_stride] = (uint8_t)q;
+        if (t) t[i * t_stride] = ti;
+    }
+}
+
+/* xt[M,K] -> xh bf16 [M,r]; codes u8 [M,K_l]; scales, zeros bf16 [M,n_g]; t (optional) [M,K_l] */
+void dq_split_quantize_asym(const double* xt, int M, int K, int r, int G, uint16_t* xh, uint8_t* codes,
+                            uint16_t* scales, uint16_t* zeros, double* t) {
+    int K_l = K - r;
+    int n_g = (K_l + G - 1) / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const double* row = xt + (int64_t)m * K;
+        for (int i = 0; i < r; ++i) xh[(int64_t)m * r + i] = dq_double_to_bf16(row[i]);
+        for (int g = 0; g < n_g; ++g) {
+            int j0 = g * G;
+            int len = (j0 + G <= K_l) ? G : (K_l - j0);
+            dq_quantize_group_asym(row + r + j0, len, 1, scales + (int64_t)m * n_g + g, zeros + (int64_t)m * n_g + g,
+                                   codes + (int64_t)m * K_l + j0, 1, t ? t + (int64_t)m * K_l + j0 : NULL, 1);
+        }
+    }
+}
+
+/* Integer products with unsigned activation codes: P[g,m,n] = sum_{j in g} u[m,j] qw[j,n]. */
+void dq_int_gemm_u(const uint8_t* ux, const int8_t* qw, int32_t* P, int M, int K_l, int N, int G) {
+    int n_g = (K_l + G - 1) / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int g = 0; g < n_g; ++g) {
+            int j0 = g * G;
+            int j1 = (j0 + G <= K_l) ? j0 + G : K_l;
+            for (int n = 0; n < N; ++n) {
+                int32_t acc = 0;
+                for (int j = j0; j < j1; ++j)
+                    acc += (int32_t)ux[(int64_t)m * K_l + j] * (int32_t)qw[(int64_t)j * N + n];
+                P[((int64_t)g * M + m) * N + n] = acc;
+            }
+        }
+    }
+}
+
+/* y[m,n] = sum_g sw[g,n] ( sx[m,g] P[g,m,n] + zx[m,g] C[g,n] ) + sum_{i<r} xh[m,i] Wh[i,n] + bias[n],
+ * C[g,n] = sum_{j in g} qw[j,n]: the "additional z term" of the asymmetric case -- dequantizing
+ * x^ = s u + z inside the product gives s * (u . qw) + z * (1 . qw) per group. */
+void dq_combine_asym(const int32_t* P, const uint16_t* sx, const uint16_t* zx, const uint16_t* sw, const int8_t* qw,
+                     const uint16_t* xh, const uint16_t* Wh, const uint16_t* bias, int M, int N, int K_l, int r, int G,
+                     double* y64, uint16_t* ybits) {
+    int n_g = (K_l + G - 1) / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int g = 0; g < n_g; ++g) {
+                int j0 = g * G;
+                int j1 = (j0 + G <= K_l) ? j0 + G : K_l;
+                int32_t c = 0;
+                for (int j = j0; j < j1; ++j) c += (int32_t)qw[(int64_t)j * N + n];
+                acc += dq_bf16_to_double(sw[(int64_t)g * N + n]) *
+                       (dq_bf16_to_double(sx[(int64_t)m * n_g + g]) * (double)P[((int64_t)g * M + m) * N + n] +
+                        dq_bf16_to_double(zx[(int64_t)m * n_g + g]) * (double)c);
+            }
+            double lr = 0.0;
+            for (int i = 0; i < r; ++i)
+                lr += dq_bf16_to_double(xh[(int64_t)m * r + i]) * dq_bf16_to_double(Wh[(int64_t)i * N + n]);
+            double v = acc + lr + (bias ? dq_bf16_to_double(bias[n]) : 0.0);
+            if (y64) y64[(int64_t)m * N + n] = v;
+            ybits[(int64_t)m * N + n] = dq_double_to_bf16(v);
+        }
+    }
+}
+
 /* ---------- plain fp64 product, used by the ideal (nothing quantized) mode ------ */
 
 void dq_matmul(const double* A, const double* B, double* C, int M, int K, int N) {

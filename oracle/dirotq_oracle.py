@@ -213,6 +213,72 @@ def linear_deployed(x_bits, layer, bias=None, want_t: bool = True):
             "P": P, "y64": y64, "y": yb}
 
 
+# ---------------------------------------------------------------------------------------------
+# Asymmetric activation quantization (Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the paper's INT4 setting)
+
+def quantize_group_asym(v):
+    v = _c(v, np.float64).ravel()
+    n = v.size
+    sb, zb = ctypes.c_uint16(0), ctypes.c_uint16(0)
+    codes = np.zeros(n, dtype=np.uint8)
+    t = np.zeros(n, dtype=np.float64)
+    _load().dq_quantize_group_asym(_p(v), ctypes.c_int(n), ctypes.c_int64(1), ctypes.byref(sb), ctypes.byref(zb), _p(codes),
+                                   ctypes.c_int64(1), _p(t), ctypes.c_int64(1))
+    return int(sb.value), int(zb.value), codes, t
+
+
+def split_quantize_asym(xt, r: int, G: int, want_t: bool = True):
+    xt = _c(xt, np.float64)
+    M, K = xt.shape
+    K_l = K - r
+    n_g = -(-K_l // G)
+    xh = np.empty((M, r), dtype=np.uint16)
+    codes = np.empty((M, K_l), dtype=np.uint8)
+    scales = np.empty((M, n_g), dtype=np.uint16)
+    zeros = np.empty((M, n_g), dtype=np.uint16)
+    t = np.empty((M, K_l), dtype=np.float64) if want_t else None
+    _load().dq_split_quantize_asym(_p(xt), ctypes.c_int(M), ctypes.c_int(K), ctypes.c_int(r), ctypes.c_int(G), _p(xh),
+                                   _p(codes), _p(scales), _p(zeros), _p(t))
+    return {"xh": xh, "codes": codes, "scales": scales, "zeros": zeros, "t": t}
+
+
+def int_gemm_u(ux, qw, G: int) -> np.ndarray:
+    """P[g,m,n] = sum over group g of u[m,j] qw[j,n] with unsigned activation codes (int32)."""
+    ux = _c(ux, np.uint8)
+    qw = _c(qw, np.int8)
+    M, K_l = ux.shape
+    N = qw.shape[1]
+    n_g = -(-K_l // G)
+    P = np.empty((n_g, M, N), dtype=np.int32)
+    _load().dq_int_gemm_u(_p(ux), _p(qw), _p(P), ctypes.c_int(M), ctypes.c_int(K_l), ctypes.c_int(N), ctypes.c_int(G))
+    return P
+
+
+def combine_asym(P, sx, zx, layer, xh, bias):
+    P = _c(P, np.int32)
+    n_g, M, N = P.shape
+    sx, zx, xh = _c(sx, np.uint16), _c(zx, np.uint16), _c(xh, np.uint16)
+    sw, qw, Wh = _c(layer["wscales"], np.uint16), _c(layer["wcodes"], np.int8), _c(layer["Wh"], np.uint16)
+    bias = None if bias is None else _c(bias, np.uint16)
+    y64 = np.empty((M, N), dtype=np.float64)
+    yb = np.empty((M, N), dtype=np.uint16)
+    _load().dq_combine_asym(_p(P), _p(sx), _p(zx), _p(sw), _p(qw), _p(xh), _p(Wh), _p(bias), ctypes.c_int(M),
+                            ctypes.c_int(N), ctypes.c_int(qw.shape[0]), ctypes.c_int(xh.shape[1]), ctypes.c_int(layer["G"]),
+                            _p(y64), _p(yb))
+    return y64, yb
+
+
+def linear_deployed_asym(x_bits, layer, bias=None, want_t: bool = True):
+    """Online part with asymmetric activation codes (the layer is prepared as for the symmetric case)."""
+    r, G = layer["r"], layer["G"]
+    xt = rotate(x_bits, layer["Qb"])
+    sq = split_quantize_asym(xt, r, G, want_t=want_t)
+    P = int_gemm_u(sq["codes"], layer["wcodes"], G)
+    y64, yb = combine_asym(P, sq["scales"], sq["zeros"], layer, sq["xh"], bias)
+    return {"xt": xt, "xh": sq["xh"], "codes": sq["codes"], "scales": sq["scales"], "zeros": sq["zeros"], "t": sq["t"],
+            "P": P, "y64": y64, "y": yb}
+
+
 def linear_ideal(x, Q, W, r: int):
     """Eq. 4 with nothing quantized and nothing rounded: [xU_h, x~_l] [W~_h; W~_l] in fp64."""
     x = _c(x, np.float64)
