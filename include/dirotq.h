@@ -170,6 +170,31 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,
                                     void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
 
+/* ---- asymmetric activation codes (paper Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the 4-bit INT setting
+ * "using asymmetric activation quantization") ---- */
+
+/* Same layer, but every group of G low-precision coefficients of a token is quantized to unsigned
+ * codes u in 0..15 with a bf16 scale s = (max - min) / 15 and a bf16 zero-point z = min, x^ = s u + z
+ * (weights stay symmetric).  The additional z term of the product, sum_g z[m,g] s_w[g,n] sum_{j in g}
+ * q_w[j,n], is precomputed on the weight side by prepare and evaluated on the bf16 tensor-core
+ * branch together with the rank-r product.  dirotq_workspace_bytes, dirotq_linear, dirotq_linear_host,
+ * dirotq_linear_noalloc, dirotq_rotate_quantize, dirotq_w4a4_gemm, dirotq_layer_export,
+ * dirotq_int_gemm_debug (codes 0..15), dirotq_layer_info and dirotq_layer_destroy accept such a layer;
+ * dirotq_workspace_export does not (use dirotq_workspace_export_asym).  Arguments as for
+ * dirotq_layer_bytes / dirotq_prepare_layer. */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes_asym(int K, int N, int r, int group, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_asym(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                                     const void* bias, int K, int N, int r, int group, void* blob,
+                                                     size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                                     dirotq_stream_t stream, dirotq_layer_t** layer_out);
+/* Parity exports: xh bf16 [M,r]; codes u8 [M,K-r] (0..15); scales, zeros bf16 [M,n_g]; zero_term fp32 [n_g,N]
+ * = s_w[g,n] * sum_{j in g} q_w[j,n] (exact).  Any pointer of the first call may be NULL. */
+DIROTQ_API dirotq_status_t dirotq_workspace_export_asym(const dirotq_layer_t* layer, int M, const void* workspace,
+                                                        void* xh_bf16, uint8_t* codes, void* scales_bf16, void* zeros_bf16,
+                                                        dirotq_stream_t stream);
+DIROTQ_API dirotq_status_t dirotq_layer_export_zero_term(const dirotq_layer_t* layer, float* zero_term,
+                                                         dirotq_stream_t stream);
+
 /* ---- NVFP4 variant (paper Sec. 5.1: "For 4-bit FP, we use NVFP4 ... group size 16 with FP8 scaling") ---- */
 
 /* Same layer with the 4-bit float format instead of INT4: elements are E2M1 (1 sign, 2 exponent,

@@ -28,6 +28,7 @@ EXPORTED = [
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_wait_counters", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
+    "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.dirotq_prepare_layer_nvfp4.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_workspace_export_nvfp4.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_layer_export_nvfp4.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.dirotq_layer_bytes_asym.argtypes = [i, i, i, i, psz]
+        L.dirotq_prepare_layer_asym.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
+        L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
+        L.dirotq_layer_export_zero_term.argtypes = [vp, vp, vp]
         for name in EXPORTED:
             if name not in ("dirotq_status_string", "dirotq_version", "dirotq_last_error"):
                 getattr(L, name).restype = i
@@ -314,3 +319,49 @@ def dirotq_layer_export_nvfp4(layer: Layer, stream=None):
     _check(lib().dirotq_layer_export_nvfp4(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(),
                                            qb.data_ptr(), ew.data_ptr(), _stream(stream)), "dirotq_layer_export_nvfp4")
     return wcodes, wscales, wh, qb, int(ew.item())
+
+
+# ------------------------------------------------------------------ asymmetric activation codes
+
+def dirotq_layer_bytes_asym(K: int, N: int, r: int, group: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_layer_bytes_asym(K, N, r, group, ctypes.byref(out)), "dirotq_layer_bytes_asym")
+    return out.value
+
+
+def dirotq_prepare_layer_asym(W: torch.Tensor, Q: torch.Tensor, r: int, group: int, bias: torch.Tensor | None = None,
+                              w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """As dirotq_prepare_layer, for a layer whose activations are quantized asymmetrically (codes 0..15, zero-point)."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    blob = _alloc_bytes(dirotq_layer_bytes_asym(K, N, r, group), W.device)
+    scratch_bytes = dirotq_prepare_scratch_bytes(K, N)
+    scratch = _alloc_bytes(scratch_bytes, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_asym(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), K, N, r, group,
+                                         blob.data_ptr(), blob.numel(), scratch.data_ptr(), scratch_bytes, _stream(stream),
+                                         ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_asym")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym")
+
+
+def dirotq_workspace_export_asym(layer: Layer, M: int, workspace: torch.Tensor, stream=None):
+    dev = workspace.device
+    xh = torch.empty((M, layer.r), dtype=torch.bfloat16, device=dev)
+    codes = torch.empty((M, layer.K_l), dtype=torch.uint8, device=dev)
+    scales = torch.empty((M, layer.n_g), dtype=torch.bfloat16, device=dev)
+    zeros = torch.empty((M, layer.n_g), dtype=torch.bfloat16, device=dev)
+    _check(lib().dirotq_workspace_export_asym(layer.handle, M, workspace.data_ptr(), xh.data_ptr(), codes.data_ptr(),
+                                              scales.data_ptr(), zeros.data_ptr(), _stream(stream)),
+           "dirotq_workspace_export_asym")
+    return xh, codes, scales, zeros
+
+
+def dirotq_layer_export_zero_term(layer: Layer, stream=None) -> torch.Tensor:
+    d = torch.empty((layer.n_g, layer.N), dtype=torch.float32, device=layer.blob.device)
+    _check(lib().dirotq_layer_export_zero_term(layer.handle, d.data_ptr(), _stream(stream)), "dirotq_layer_export_zero_term")
+    return d

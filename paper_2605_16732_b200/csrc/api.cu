@@ -135,10 +135,10 @@ dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_
     return DIROTQ_OK;
 }
 
-dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
-                                     const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
-                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
-                                     dirotq_layer_t** layer_out) {
+static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                    const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                    void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                    dirotq_layer_t** layer_out) {
     if (!W || !Q || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
     if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
     if (q_dtype != DIROTQ_DTYPE_F64 && q_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
@@ -147,7 +147,8 @@ dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, c
     if (st != DIROTQ_OK) return st;
     if (!aligned16(W) || !aligned16(Q) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
-    const Geometry g = make_geometry(K, N, r, group);
+    Geometry g = make_geometry(K, N, r, group);
+    if (asym) make_asym(g);
     const BlobLayout lay = make_blob_layout(g);
     if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
     if (scratch_bytes < static_cast<size_t>(K) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
@@ -184,6 +185,45 @@ dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, c
     }
     *layer_out = L;
     return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                     const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                     dirotq_layer_t** layer_out) {
+    return prepare_int4(false, W, w_dtype, w_layout, Q, q_dtype, bias, K, N, r, group, blob, blob_bytes, scratch,
+                        scratch_bytes, stream, layer_out);
+}
+
+dirotq_status_t dirotq_layer_bytes_asym(int K, int N, int r, int group, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, group);
+    if (st != DIROTQ_OK) return st;
+    Geometry g = make_geometry(K, N, r, group);
+    make_asym(g);
+    *bytes = make_blob_layout(g).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_asym(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                          const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                          void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                          dirotq_layer_t** layer_out) {
+    return prepare_int4(true, W, w_dtype, w_layout, Q, q_dtype, bias, K, N, r, group, blob, blob_bytes, scratch,
+                        scratch_bytes, stream, layer_out);
+}
+
+dirotq_status_t dirotq_workspace_export_asym(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
+                                             uint8_t* codes, void* scales_bf16, void* zeros_bf16, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || layer->geo.fmt != 2 || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
+    return launch_workspace_export_asym(layer, M, static_cast<const char*>(workspace), static_cast<uint16_t*>(xh_bf16), codes,
+                                        static_cast<uint16_t*>(scales_bf16), static_cast<uint16_t*>(zeros_bf16),
+                                        static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_layer_export_zero_term(const dirotq_layer_t* layer, float* zero_term, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || layer->geo.fmt != 2 || !zero_term) return DIROTQ_ERR_INVALID_ARG;
+    return launch_zero_term_export(layer, zero_term, static_cast<cudaStream_t>(stream));
 }
 
 dirotq_status_t dirotq_layer_destroy(dirotq_layer_t* layer) {
@@ -320,7 +360,7 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
                                       void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
     dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
     if (st != DIROTQ_OK) return st;
-    if (layer->geo.fmt != 0) return DIROTQ_ERR_INVALID_ARG;
+    if (layer->geo.fmt == 1) return DIROTQ_ERR_INVALID_ARG;
     if (!act_codes || !partials || !aligned16(act_codes) || !aligned16(partials)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = static_cast<char*>(workspace);
     const WorkspaceLayout w = make_workspace_layout(layer->geo, M);
@@ -338,7 +378,7 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
 
 dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16, void* wh_bf16,
                                     void* q_bf16, dirotq_stream_t stream) {
-    if (!valid_layer(layer) || layer->geo.fmt != 0) return DIROTQ_ERR_INVALID_ARG;
+    if (!valid_layer(layer) || layer->geo.fmt == 1) return DIROTQ_ERR_INVALID_ARG;
     return launch_layer_export(layer, wcodes, static_cast<uint16_t*>(wscales_bf16), static_cast<uint16_t*>(wh_bf16),
                                static_cast<uint16_t*>(q_bf16), static_cast<cudaStream_t>(stream));
 }

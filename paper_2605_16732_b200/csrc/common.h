@@ -20,9 +20,11 @@ struct Geometry {
     int K_l;    // K - r
     int n_g;    // ceil(K_l / G)
     int K_lp;   // n_g * G  (<= K)
-    int r_pad;  // r rounded up to a multiple of 64 (bf16 low-rank operand width)
+    int r_pad;  // width of the bf16 rank-r operands: r rounded up to 64, plus (fmt 2) the zero-point columns, rounded up to 64
+    int r_pad0; // r rounded up to a multiple of 64: where the zero-point columns of fmt 2 start
     // NVFP4 variant only (fmt == 1): blocks of 16, MMA K = 64, TMA k-blocks of 256 elements
-    int fmt;     // 0 = INT4 groups with bf16 scales, 1 = NVFP4 (E2M1 elements, E4M3 block scales)
+    int fmt;     // 0 = INT4 groups with bf16 scales, 1 = NVFP4 (E2M1 elements, E4M3 block scales),
+                 // 2 = INT4 with asymmetric activation codes (0..15, bf16 scale and zero-point per group)
     int K4;      // K_l rounded up to 64 (<= K): width of the packed E2M1 rows
     int nkb64;   // K4 / 64: scale-factor atoms (128 rows x 4 scales) per row block
     int nkb64p;  // nkb64 rounded up to 4: one TMA k-block = 256 elements = 4 atoms
@@ -35,6 +37,7 @@ inline Geometry make_geometry(int K, int N, int r, int G) {
     g.n_g = (g.K_l + G - 1) / G;
     g.K_lp = g.n_g * G;
     g.r_pad = (r + 63) / 64 * 64;
+    g.r_pad0 = g.r_pad;
     g.fmt = 0;
     g.K4 = (g.K_l + 63) / 64 * 64;
     g.nkb64 = g.K4 / 64;
@@ -46,6 +49,14 @@ constexpr size_t kAlign = 1024;
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
 // Sections of the device blob that holds a prepared layer.
+// Asymmetric activations (fmt 2): x^ = s u + z per group.  The zero-point term sum_g z[m,g] * (s_w[g,n] sum_{j in g} q_w[j,n])
+// is a rank-n_g product; it rides on the bf16 rank-r branch as 3 n_g extra columns: the activation side holds z (bf16,
+// exact) three times, the weight side the three bf16 pieces of s_w * sum q_w (17 significant bits, split exactly).
+inline void make_asym(Geometry& g) {
+    g.fmt = 2;
+    g.r_pad = (g.r_pad0 + 3 * g.n_g + 63) / 64 * 64;
+}
+
 struct BlobLayout {
     size_t off_qt;       // bf16 [K][K]: row c' = permuted output column, K-major over the input channel
     size_t off_wpacked;  // u8   [N][K_lp/2]: two INT4 codes per byte, K-major, see prepare.cu for the nibble order
@@ -196,6 +207,9 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
                                     uint16_t* qb, cudaStream_t stream);
 dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
                                         int8_t* codes, uint16_t* scales, cudaStream_t stream);
+dirotq_status_t launch_workspace_export_asym(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
+                                             uint8_t* codes, uint16_t* scales, uint16_t* zeros, cudaStream_t stream);
+dirotq_status_t launch_zero_term_export(const dirotq_layer* L, float* d, cudaStream_t stream);
 dirotq_status_t launch_debug_codes(const dirotq_layer* L, int M, const int8_t* act_codes, char* workspace,
                                    cudaStream_t stream);
 int sm_count(int device);

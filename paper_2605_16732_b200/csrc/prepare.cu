@@ -83,7 +83,7 @@ __host__ __device__ __forceinline__ int packed_byte_index(int k) {  // byte of c
 __host__ __device__ __forceinline__ int packed_is_high(int k) { return (k >> 2) & 1; }
 
 // One thread per (group, output column): Eq. 1 with z = 0, s = bf16(max|w|/7), ties to even.
-__global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, float* wscale, Geometry g) {
+__global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, float* wscale, uint16_t* wh, Geometry g) {
     const int n = blockIdx.x * blockDim.x + threadIdx.x;
     const int grp = blockIdx.y;
     if (n >= g.N) return;
@@ -96,6 +96,7 @@ __global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, floa
     const double s = bf16_to_f64(sb);
     wscale[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(s);
     uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
+    int csum = 0;
     for (int jb = 0; jb < g.G; jb += 8) {
         // codes j0+jb .. j0+jb+7 share four bytes
         uint32_t word = 0;
@@ -107,11 +108,23 @@ __global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, floa
                 qq = fmin(7.0, fmax(-7.0, qq));
                 q = static_cast<int>(qq);
             }
+            csum += q;
             // stored with an offset of 8: the nibble u = q + 8 in 1..15, read as an E4M3 byte, is u * 2^-9 exactly
             const uint32_t nib = static_cast<uint32_t>(q + 8) & 0xFu;
             word |= nib << (8 * (t & 3) + 4 * (t >> 2));
         }
         *reinterpret_cast<uint32_t*>(row + packed_byte_index(j0 + jb)) = word;
+    }
+    if (g.fmt == 2) {
+        // zero-point term of asymmetric activations: d = s_w * sum(q_w) (at most 17 significant bits), stored as three
+        // bf16 pieces that add up to it exactly, in the extra columns of the rank-r weight operand
+        double rem = s * static_cast<double>(csum);
+        uint16_t* ext = wh + static_cast<size_t>(n) * g.r_pad + g.r_pad0;
+        for (int piece = 0; piece < 3; ++piece) {
+            const uint16_t pb = f64_to_bf16(rem);
+            ext[piece * g.n_g + grp] = pb;
+            rem -= bf16_to_f64(pb);
+        }
     }
 }
 
@@ -201,6 +214,34 @@ __global__ void export_workspace_kernel(const int8_t* codes, const float* xscale
                 scales[static_cast<size_t>(m) * g.n_g + gi] =
                     static_cast<uint16_t>(__float_as_uint(xscale[static_cast<size_t>(gi) * ldm + m]) >> 16);
     }
+}
+
+// fmt 2: codes are plain bytes 0..15; the zero-points sit in the extra columns of x~_h.
+__global__ void export_workspace_asym_kernel(const uint8_t* codes, const float* xscale, const uint16_t* xh_pad, int M, int ldm,
+                                             Geometry g, uint16_t* xh, uint8_t* codes_out, uint16_t* scales, uint16_t* zeros) {
+    const int m = blockIdx.y;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < g.K_l; c += gridDim.x * blockDim.x)
+        if (codes_out) codes_out[static_cast<size_t>(m) * g.K_l + c] = codes[static_cast<size_t>(m) * g.K_lp + c];
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < g.r; i += blockDim.x)
+            if (xh) xh[static_cast<size_t>(m) * g.r + i] = xh_pad[static_cast<size_t>(m) * g.r_pad + i];
+        for (int gi = threadIdx.x; gi < g.n_g; gi += blockDim.x) {
+            if (scales)
+                scales[static_cast<size_t>(m) * g.n_g + gi] =
+                    static_cast<uint16_t>(__float_as_uint(xscale[static_cast<size_t>(gi) * ldm + m]) >> 16);
+            if (zeros) zeros[static_cast<size_t>(m) * g.n_g + gi] = xh_pad[static_cast<size_t>(m) * g.r_pad + g.r_pad0 + gi];
+        }
+    }
+}
+
+__global__ void export_zero_term_kernel(const uint16_t* wh, float* d, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int grp = blockIdx.y;
+    if (n >= g.N) return;
+    const uint16_t* ext = wh + static_cast<size_t>(n) * g.r_pad + g.r_pad0;
+    double v = 0.0;
+    for (int piece = 2; piece >= 0; --piece) v += bf16_to_f64(ext[piece * g.n_g + grp]);
+    d[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(v);  // 17 significant bits: exact
 }
 
 // Debug entry of the group GEMM: two's-complement codes [M][K_lp] -> the sign-magnitude bytes the kernel reads,
@@ -390,10 +431,12 @@ dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype
     // zero the packed codes first: slots of a ragged last group stay zero
     if (cudaMemsetAsync(blob + L->lay.off_wpacked, 0, static_cast<size_t>(g.N) * (g.K_lp / 2), stream) != cudaSuccess)
         return DIROTQ_ERR_CUDA;
-    quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
-        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale), g);
-    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    // the rank-r rows first (zero padded to r_pad), then the quantizer, which for fmt 2 fills its extra columns
     high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale),
+        reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
         Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
@@ -429,6 +472,23 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
     }
     return DIROTQ_OK;
+}
+
+dirotq_status_t launch_workspace_export_asym(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
+                                             uint8_t* codes, uint16_t* scales, uint16_t* zeros, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const WorkspaceLayout w = make_workspace_layout(g, M);
+    export_workspace_asym_kernel<<<dim3(8, M), 256, 0, stream>>>(
+        reinterpret_cast<const uint8_t*>(workspace + w.off_codes), reinterpret_cast<const float*>(workspace + w.off_xscale),
+        reinterpret_cast<const uint16_t*>(workspace + w.off_xh), M, w.ldm, g, xh, codes, scales, zeros);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_zero_term_export(const dirotq_layer* L, float* d, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    export_zero_term_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+        reinterpret_cast<const uint16_t*>(L->blob + L->lay.off_wh), d, g);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 dirotq_status_t launch_debug_codes(const dirotq_layer* L, int M, const int8_t* act_codes, char* workspace,

@@ -32,7 +32,7 @@ constexpr int NUM_THREADS = 192;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct RotKernelParams {
-    int M, K, K_l, K_lp, r, r_pad, ldm, n_g;
+    int M, K, K_l, K_lp, r, r_pad, r_pad0, ldm, n_g;
     int8_t* codes;
     float* xscale;
     uint16_t* xh;
@@ -70,6 +70,27 @@ __device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, 
         const uint32_t sg = (tw >> 7) & 0x01010101u;           // 1 where the code is negative
         const uint32_t mag = (tw ^ (sg * 0xFFu)) + sg;         // |q| per byte (at most 7: no carry between bytes)
         w[i] = mag | (tw & 0x80808080u);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Asymmetric variant (Eq. 1 with z = min X): 16 values -> 16 bytes u = clip(rint((v - z) / s), 0, 15); as E4M3 the byte
+// 0000uuuu is u * 2^-9 exactly.  The codes are also added to `sum`.
+__device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float inv, float s, bool slow, int& sum) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t f[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float d = v[4 * i + j] - z;
+            float t = slow ? (s != 0.f ? d / s : 0.f) : d * inv;
+            t = fminf(fmaxf(t, 0.0f), 15.0f);
+            f[j] = __float_as_uint(t + 12582912.0f);  // nearest integer, ties to even, in the low byte
+        }
+        const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
+        sum = __dp4a(tw, 0x01010101u, static_cast<unsigned>(sum));
+        w[i] = tw;
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
@@ -289,6 +310,43 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                                 *reinterpret_cast<uint32_t*>(p.xsf + (static_cast<size_t>(row >> 7) * p.nkb64p + a) * 512 +
                                                              (mr & 31) * 16 + (mr >> 5) * 4) = 0u;
                     }
+                } else if constexpr (FMT == 2) {
+                    if (nlow > 0 && row_ok) {
+                        // asymmetric: z = bf16(min), s = bf16((max - min) / 15) over the group's real elements
+                        float lo = v[0], hi = v[0];
+#pragma unroll
+                        for (int b = 0; b < G / 16; ++b) {
+                            if (16 * b < nlow) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    lo = fminf(lo, v[16 * b + j]);
+                                    hi = fmaxf(hi, v[16 * b + j]);
+                                }
+                            }
+                        }
+                        const __nv_bfloat16 zb = __float2bfloat16_rn(lo);
+                        const float z = __bfloat162float(zb);
+                        const float s = hi > lo ? __bfloat162float(__float2bfloat16_rn(__fdiv_rn(hi - lo, 15.0f))) : 0.f;
+                        const bool slow = !(s >= 1e-30f);
+                        const float inv = slow ? 0.f : __frcp_rn(s);
+                        int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+                        int usum = 0;
+#pragma unroll
+                        for (int b = 0; b < G / 16; ++b) {
+                            uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
+                            if (16 * b < nlow) packed = quantize16_asym(v + 16 * b, z, inv, s, slow, usum);
+                            *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                        }
+                        const int grp = col0 / G;
+                        p.xscale[static_cast<size_t>(grp) * p.ldm + row] = s;
+                        p.xscale[static_cast<size_t>(p.n_g + grp) * p.ldm + row] = -8.0f * static_cast<float>(usum) * s;
+                        // the zero-point, three times, in the extra columns of the bf16 rank-r operand
+                        uint16_t* zrow = p.xh + static_cast<size_t>(row) * p.r_pad + p.r_pad0 + grp;
+                        const uint16_t zbits = *reinterpret_cast<const uint16_t*>(&zb);
+                        zrow[0] = zbits;
+                        zrow[p.n_g] = zbits;
+                        zrow[2 * p.n_g] = zbits;
+                    }
                 } else if (nlow > 0) {
                     float amax = 0.f;
 #pragma unroll
@@ -339,8 +397,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
             if (n_blk == num_n_blocks - 1 && row_ok) {
-                for (int c = p.r; c < p.r_pad; c += 8)
+                for (int c = p.r; c < p.r_pad0; c += 8)
                     *reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + c) = make_uint4(0, 0, 0, 0);
+                if constexpr (FMT == 2) {  // behind the 3 n_g zero-point columns
+                    for (int c = p.r_pad0 + 3 * p.n_g; c < p.r_pad; ++c) p.xh[static_cast<size_t>(row) * p.r_pad + c] = 0;
+                }
             }
         }
     }
@@ -363,14 +424,17 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
                                         (uint64_t)g.K * 2, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != DIROTQ_OK) return st;
     RotKernelParams p;
-    p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.ldm = a.ldm; p.n_g = g.n_g;
+    p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
     const int num_tiles = ((a.M + BM - 1) / BM) * ((g.K + BN - 1) / BN);
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
-    const int vi = g.fmt == 1 ? 2 : (g.G == 64 ? 0 : 1);
-    auto kern = vi == 2 ? rotate_quant_kernel<64, 1> : (vi == 0 ? rotate_quant_kernel<64, 0> : rotate_quant_kernel<128, 0>);
-    static bool attr_set[3] = {false, false, false};
+    const int vi = g.fmt == 1 ? 2 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
+    auto kern = vi == 2 ? rotate_quant_kernel<64, 1>
+              : vi == 3 ? rotate_quant_kernel<64, 2>
+              : vi == 4 ? rotate_quant_kernel<128, 2>
+              : vi == 0 ? rotate_quant_kernel<64, 0> : rotate_quant_kernel<128, 0>;
+    static bool attr_set[5] = {false, false, false, false, false};
     if (!attr_set[vi]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;

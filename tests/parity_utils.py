@@ -251,3 +251,80 @@ def check_layer_output_nvfp4(y_bits, xh_bits, codes, sf, ex, layer_orc, out_orc,
     d = np.abs(f64(y_bits) - out_orc["y64"])
     stats["e2e_all_max_err_over_rms"] = float(d.max() / np.sqrt(np.mean(out_orc["y64"] ** 2)))
     return stats
+
+
+# ------------------------------------------------------------------ asymmetric activation codes
+#
+# Same protocol as the symmetric case with a zero-point per group: the zero-point equals the oracle's or is the
+# neighbouring bf16 value when the unrounded minimum lies within 1e-4 (relative) + 1e-5 ||x~_row|| of the midpoint; the
+# scale likewise for (max - min)/15; codes are checked against the quantizer re-run with the library's scale and
+# zero-point (+-1 within 1e-3 + 1e-5 ||x~_row|| / s of a rounding boundary); the output against the fp64
+# combination (integer sums, scales, zero-point term, rank-r branch, bias) of the library's own intermediates.
+
+def check_activation_side_asym(xrot, xh, codes, scales, zeros, out_orc, r, G):
+    xt = out_orc["xt"]
+    M, K = xt.shape
+    K_l = K - r
+    n_g = -(-K_l // G)
+    stats = {}
+    norm = np.linalg.norm(xt, axis=1, keepdims=True)
+    if xrot is not None:
+        rel = np.linalg.norm(xrot.astype(np.float64) - xt, axis=1) / np.maximum(norm[:, 0], 1e-300)
+        stats["xrot_rel_max"] = float(rel.max())
+        assert rel.max() <= 2e-3
+    xh_g, xh_o = f64(xh), f64(out_orc["xh"])
+    step = np.maximum(np.abs(xh_o), 2.0 ** -126) * 2.0 ** -7 + 1e-5 * norm
+    assert np.all(np.abs(xh_g - xh_o) <= step), "x~_h differs by more than one bf16 step"
+    # group minima / ranges of the oracle's fp64 rotation (padding slots excluded)
+    lo = np.full((M, n_g), np.inf)
+    hi = np.full((M, n_g), -np.inf)
+    for g in range(n_g):
+        seg = xt[:, r + g * G: r + min((g + 1) * G, K_l)]
+        lo[:, g], hi[:, g] = seg.min(axis=1), seg.max(axis=1)
+    normb = np.broadcast_to(norm, lo.shape)
+    z_g, z_o = f64(zeros), f64(out_orc["zeros"])
+    zflip = zeros != out_orc["zeros"]
+    if zflip.any():
+        assert np.all(np.abs(z_g[zflip] - z_o[zflip]) <= np.maximum(np.abs(z_o[zflip]), 2.0 ** -126) * 2.0 ** -7), \
+            "a zero-point is more than one bf16 step away"
+        mid = 0.5 * (z_g[zflip] + z_o[zflip])
+        assert np.all(np.abs(lo[zflip] - mid) <= 1e-4 * np.abs(lo[zflip]) + 1e-5 * normb[zflip]), \
+            "zero-point differs away from a rounding boundary"
+    s_g, s_o = f64(scales), f64(out_orc["scales"])
+    u = (hi - lo) / 15.0
+    sflip = scales != out_orc["scales"]
+    if sflip.any():
+        db = np.abs(scales[sflip].astype(np.int64) - out_orc["scales"][sflip].astype(np.int64))
+        assert np.all(db == 1), "a scale is more than one bf16 step away"
+        mid = 0.5 * (s_g[sflip] + s_o[sflip])
+        assert np.all(np.abs(u[sflip] - mid) <= 1e-4 * u[sflip] + 2e-5 * normb[sflip] / 15.0), \
+            "scale differs away from a rounding boundary"
+    stats["scale_flips"], stats["zero_flips"] = int(sflip.sum()), int(zflip.sum())
+    s_use = np.repeat(s_g, G, axis=1)[:, :K_l]
+    z_use = np.repeat(z_g, G, axis=1)[:, :K_l]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(s_use != 0, (xt[:, r:] - z_use) / s_use, 0.0)
+    q_ref = np.clip(np.rint(t), 0, 15).astype(np.uint8)
+    same = ~np.repeat(sflip | zflip, G, axis=1)[:, :K_l]
+    assert np.array_equal(q_ref[same], out_orc["codes"][same])
+    bad = codes != q_ref
+    if bad.any():
+        assert np.all(np.abs(codes[bad].astype(int) - q_ref[bad].astype(int)) == 1), "a code is off by more than 1"
+        dist = np.abs(np.abs(t[bad] - np.floor(t[bad])) - 0.5)
+        with np.errstate(divide="ignore"):
+            tol = 1e-3 + 1e-5 * np.broadcast_to(norm, t.shape)[bad] / s_use[bad]
+        assert np.all(dist <= tol), "a code differs away from a rounding boundary"
+    stats["code_flips"] = int(bad.sum())
+    return stats
+
+
+def check_layer_output_asym(y_bits, xh_bits, codes, scales, zeros, layer_orc, out_orc, bias_bits, slack=3e-4):
+    P = orc.int_gemm_u(codes, layer_orc["wcodes"], layer_orc["G"])
+    y_ref, _ = orc.combine_asym(P, scales, zeros, layer_orc, xh_bits, bias_bits)
+    stats = check_output(y_bits, y_ref, slack=slack)
+    clean = (np.all(codes == out_orc["codes"], axis=1) & np.all(scales == out_orc["scales"], axis=1)
+             & np.all(zeros == out_orc["zeros"], axis=1) & np.all(xh_bits == out_orc["xh"], axis=1))
+    stats["clean_rows_frac"] = float(np.mean(clean))
+    e2e = check_output(y_bits, out_orc["y64"], rows=clean, slack=slack)
+    stats["e2e_clean_max_err_over_rms"] = e2e.get("max_err_over_rms")
+    return stats
