@@ -133,6 +133,8 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
         for lo, x, K, n in layers:
             if fmt == "nvfp4":
                 orc.nvfp4_linear_deployed(x, lo, lo["ex"], bias=None, want_t=False)
+            elif fmt == "int4_asym":
+                orc.linear_deployed_asym(x, lo, bias=None, want_t=False)
             else:
                 orc.linear_deployed(x, lo, bias=None, want_t=False)
         times.append(time.perf_counter() - t0)
@@ -157,7 +159,8 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64 (oracle; nvfp4 codes)" if args.fmt == "nvfp4" else "f64 + int32 (oracle; int4 codes)",
-        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else ""), "format": args.fmt,
+        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else "_asym" if args.fmt == "int4_asym" else ""),
+                                        "format": args.fmt,
                                         "sample": res["sample"]},
         "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": res["value"], "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -211,6 +214,8 @@ def run_ours(args):
             del xrot
             layer = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, int(np.ceil(np.log2(amax / 1536.0))),
                                                   bias=bf(bias))
+        elif args.fmt == "int4_asym":
+            layer = dq.dirotq_prepare_layer_asym(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         else:
             layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         del Q
@@ -371,7 +376,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None,
         "dtype": "nvfp4 (e2m1 x e2m1, e4m3 block scales) + bf16" if nv else "int4xint4 (exact group sums on the e4m3 tensor path) + bf16",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
+        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else "_asym" if args.fmt == "int4_asym" else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
                    "group": 16 if nv else GROUP, "format": args.fmt,
                    "l2": "inputs_exceed_l2 (each step streams > 500 MB of rotations, codes and outputs)",
                    "parallelism": f"token rows x{world}, no collective"},
@@ -396,8 +401,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shapes", default="", help="comma-separated subset of qkv,out,mlp_up,mlp_down (profiling runs)")
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4"],
-                    help="int4: the headline format (groups of 64, bf16 scales); nvfp4: E2M1 blocks of 16 with E4M3 scales")
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym"],
+                    help="int4: the headline format (groups of 64, bf16 scales, symmetric); nvfp4: E2M1 blocks of 16 with E4M3 "
+                         "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group)")
     ap.add_argument("--lite", action="store_true", help="skip the cuBLAS, end-to-end and CPU-baseline legs (profiling runs)")
     args = ap.parse_args()
     if args.shapes:

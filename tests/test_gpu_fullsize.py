@@ -180,3 +180,62 @@ def test_nvfp4_flux_linears(K, N):
 
 def test_nvfp4_batch4_rank128():
     print(_run_nvfp4(18432, 3072, 9216, 128, synth.FLUX))
+
+
+# ------------------------------------------------------------------ asymmetric activation codes at the benchmark's sizes
+
+def _run_asym(M, K, N, r, G, model, n_rows=24, n_cols=96, seed=0):
+    from parity_utils import check_activation_side_asym, check_layer_output_asym
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=model, seed=seed)
+    Q = _rotation(spec)
+    W, bias = synth.make_weights(spec)
+    x_bits = synth.make_tokens(spec, M, batch_seed=3)
+    g = np.random.default_rng(K * 7 + N + 2)
+    rows = np.sort(g.choice(M, size=min(n_rows, M), replace=False))
+    rows[-1] = M - 1
+    cols = np.sort(g.choice(N, size=n_cols, replace=False))
+    cols[-1] = N - 1
+    lo = orc.prepare_layer(W[:, cols], Q, r, G, want_t=True)
+    bias_s = bias[cols]
+    oo = orc.linear_deployed_asym(x_bits[rows], lo, bias=bias_s)
+
+    Qd = torch.from_numpy(Q).cuda()
+    layer = dq.dirotq_prepare_layer_asym(torch.from_numpy(W).cuda(), Qd, r, G, bias=bits_to_bf16_tensor(bias))
+    del Qd
+    cols_t = torch.from_numpy(cols).cuda()
+    n_g = layer.n_g
+    csum = np.stack([lo["wcodes"][gi * G:(gi + 1) * G].astype(np.int64).sum(axis=0) for gi in range(n_g)])
+    d_ref = (orc.bf16_to_f64(lo["wscales"]) * csum).astype(np.float32)
+    d = dq.dirotq_layer_export_zero_term(layer)[:, cols_t].cpu().numpy()
+    # a weight code may differ from the oracle's at an exact tie of the fp64 quotient (different summation order in
+    # the fold): compare the zero-point term on the columns whose codes all agree
+    wc = dq.dirotq_layer_export(layer)[0][:, cols_t].cpu().numpy()
+    agree = np.all(wc == lo["wcodes"], axis=0)
+    assert agree.sum() >= n_cols - 2 and np.array_equal(d[:, agree], d_ref[:, agree]), "zero-point term differs"
+
+    x = bits_to_bf16_tensor(x_bits)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = dq.alloc_workspace(layer, M)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, scales, zeros = dq.dirotq_workspace_export_asym(layer, M, ws)
+    rows_t = torch.from_numpy(rows).cuda()
+    xh_b = bf16_tensor_to_bits(xh[rows_t])
+    codes_n = codes[rows_t].cpu().numpy()
+    scales_b, zeros_b = bf16_tensor_to_bits(scales[rows_t]), bf16_tensor_to_bits(zeros[rows_t])
+    stats = check_activation_side_asym(None, xh_b, codes_n, scales_b, zeros_b, oo, r, G)
+    lo_lib = dict(lo)
+    lo_lib["wcodes"] = wc  # the output check uses the library's own weight codes
+    y_s = bf16_tensor_to_bits(y[rows_t][:, cols_t])
+    stats.update(check_layer_output_asym(y_s, xh_b, codes_n, scales_b, zeros_b, lo_lib, oo, bias_s))
+    layer.close()
+    return stats
+
+
+@pytest.mark.parametrize("K,N", [(3072, 9216), (12288, 3072)])
+def test_asym_flux_linears(K, N):
+    print(_run_asym(4608, K, N, 32, 64, synth.FLUX))
+
+
+def test_asym_batch4_rank64_group128():
+    print(_run_asym(18432, 3072, 9216, 64, 128, synth.FLUX))
