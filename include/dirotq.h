@@ -116,9 +116,13 @@ DIROTQ_API dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K
 DIROTQ_API dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer, void* y, void* workspace,
                               size_t workspace_bytes, dirotq_stream_t stream);
 
-/* Same computation with HOST input and output (pinned memory recommended): copies x into
- * x_dev, runs dirotq_linear, copies y_dev into y_host, all on `stream`; x_dev [M,K] and
- * y_dev [M,N] are device staging buffers of the caller. */
+/* Same computation with HOST input and output (pinned memory, or the copies do not overlap):
+ * copies x into x_dev, runs dirotq_linear, copies y_dev into y_host; x_dev [M,K] and y_dev [M,N]
+ * are device staging buffers of the caller.  For M >= 2048 the call is cut into up to 8 row chunks
+ * (token rows are independent) whose two copies run on two copy streams the library creates once
+ * per device, overlapping each other and the kernels on `stream`; everything is ordered after the
+ * work already on `stream`, and later work on `stream` (or a synchronisation of it) is ordered
+ * after the last copy into y_host.  Not for use during stream capture. */
 DIROTQ_API dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer_t* layer, void* y_host,
                                    void* x_dev, void* y_dev, void* workspace, size_t workspace_bytes,
                                    dirotq_stream_t stream);

@@ -1,6 +1,8 @@
 // C ABI of libdirotq: argument validation, tensor-map construction, launch sequencing.
 #include "common.h"
 
+#include <mutex>
+
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
@@ -312,19 +314,87 @@ dirotq_status_t dirotq_w4a4_gemm(int M, const dirotq_layer_t* layer, const void*
     return second_kernel(layer, ra, M, y, static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+// Copy streams and events of dirotq_linear_host, created once per device (no device memory involved).
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    static constexpr int kMaxChunks = 8;
+    cudaEvent_t start = nullptr, done = nullptr, copied[kMaxChunks] = {}, computed[kMaxChunks] = {};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipe[64];
+
+dirotq_status_t host_pipe(int dev, HostPipe** out) {
+    if (dev < 0 || dev >= 64) return DIROTQ_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe& p = g_pipe[dev];
+    if (!p.ready) {
+        cudaError_t e = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p.done, cudaEventDisableTiming);
+        for (int i = 0; i < HostPipe::kMaxChunks && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&p.copied[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p.computed[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) { set_error("host pipeline set-up", e); return DIROTQ_ERR_CUDA; }
+        p.ready = true;
+    }
+    *out = &p;
+    return DIROTQ_OK;
+}
+
+}  // namespace
+
 dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer_t* layer, void* y_host, void* x_dev,
                                    void* y_dev, void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
     dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
     if (st != DIROTQ_OK) return st;
     if (!x_host || !y_host || !x_dev || !y_dev) return DIROTQ_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t xb = static_cast<size_t>(M) * layer->geo.K * 2, yb = static_cast<size_t>(M) * layer->geo.N * 2;
-    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xb, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) { set_error("cudaMemcpyAsync(H2D)", e); return DIROTQ_ERR_CUDA; }
-    st = dirotq_linear(x_dev, M, layer, y_dev, workspace, workspace_bytes, stream);
+    const size_t xrow = static_cast<size_t>(layer->geo.K) * 2, yrow = static_cast<size_t>(layer->geo.N) * 2;
+    // Token rows are independent: the call is cut into row chunks whose host-to-device copy, computation and
+    // device-to-host copy overlap (copy engines in both directions + SMs).  The chunks' kernels run one after another on
+    // `stream`, so they can share the workspace.
+    int chunks = M / 1024;
+    if (chunks > HostPipe::kMaxChunks) chunks = HostPipe::kMaxChunks;
+    if (chunks <= 1) {
+        cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xrow * M, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) { set_error("cudaMemcpyAsync(H2D)", e); return DIROTQ_ERR_CUDA; }
+        st = dirotq_linear(x_dev, M, layer, y_dev, workspace, workspace_bytes, stream);
+        if (st != DIROTQ_OK) return st;
+        e = cudaMemcpyAsync(y_host, y_dev, yrow * M, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) { set_error("cudaMemcpyAsync(D2H)", e); return DIROTQ_ERR_CUDA; }
+        return DIROTQ_OK;
+    }
+    HostPipe* p = nullptr;
+    st = host_pipe(layer->device, &p);
     if (st != DIROTQ_OK) return st;
-    e = cudaMemcpyAsync(y_host, y_dev, yb, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) { set_error("cudaMemcpyAsync(D2H)", e); return DIROTQ_ERR_CUDA; }
+    const int rows_per_chunk = ((M + chunks - 1) / chunks + 127) / 128 * 128;
+    cudaError_t e = cudaEventRecord(p->start, s);  // the staging buffers may still be in use by earlier work on `stream`
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(p->h2d, p->start, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(p->d2h, p->start, 0);
+    int c = 0;
+    for (int m0 = 0; m0 < M && e == cudaSuccess; m0 += rows_per_chunk, ++c) {
+        const int mc = M - m0 < rows_per_chunk ? M - m0 : rows_per_chunk;
+        char* xd = static_cast<char*>(x_dev) + xrow * m0;
+        char* yd = static_cast<char*>(y_dev) + yrow * m0;
+        e = cudaMemcpyAsync(xd, static_cast<const char*>(x_host) + xrow * m0, xrow * mc, cudaMemcpyHostToDevice, p->h2d);
+        if (e == cudaSuccess) e = cudaEventRecord(p->copied[c], p->h2d);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, p->copied[c], 0);
+        if (e != cudaSuccess) break;
+        st = dirotq_linear(xd, mc, layer, yd, workspace, workspace_bytes, stream);
+        if (st != DIROTQ_OK) return st;
+        e = cudaEventRecord(p->computed[c], s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(p->d2h, p->computed[c], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(static_cast<char*>(y_host) + yrow * m0, yd, yrow * mc, cudaMemcpyDeviceToHost, p->d2h);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(p->done, p->d2h);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, p->done, 0);  // later work on `stream` (and its synchronisation) sees y_host
+    if (e != cudaSuccess) { set_error("host pipeline", e); return DIROTQ_ERR_CUDA; }
     return DIROTQ_OK;
 }
 

@@ -180,3 +180,28 @@ def test_group_sums_exact_on_codes_built_to_lose_low_bits(G):
     assert int(np.abs(ref).max()) == G * 49
     assert np.array_equal(P.cpu().numpy(), ref)
     layer.close()
+
+
+@pytest.mark.parametrize("M", [300, 2500, 4608])
+def test_host_entry_point_equals_device_entry_point(M):
+    """dirotq_linear_host (pinned host buffers; row chunks pipelined over copy streams for large M) gives the same
+    bits as dirotq_linear on device buffers, twice in a row (re-use of the staging buffers and events)."""
+    spec = synth.LayerSpec(K=512, N=384, r=32, G=64, model=synth.PIXART, seed=9, calib_tokens=1024)
+    inp = synth.make_layer_inputs(spec, M)
+    layer = dq.dirotq_prepare_layer(torch.from_numpy(inp["W"]).cuda(), torch.from_numpy(inp["Q"]).cuda(), spec.r, spec.G,
+                                    bias=bits_to_bf16_tensor(inp["bias"]))
+    x = bits_to_bf16_tensor(inp["x"])
+    ws = dq.alloc_workspace(layer, M)
+    y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device="cuda")
+    dq.dirotq_linear(x, layer, y, ws)
+    torch.cuda.synchronize()
+    xh = x.cpu().pin_memory()
+    yh = torch.zeros((M, spec.N), dtype=torch.bfloat16).pin_memory()
+    x_dev, y_dev = torch.empty_like(x), torch.empty_like(y)
+    for _ in range(2):
+        yh.zero_()
+        dq.dirotq_linear_host(xh, layer, yh, x_dev, y_dev, ws)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(yh.view(torch.int16), y.cpu().view(torch.int16))
+    assert dq.dirotq_workspace_status(ws) == 0
+    layer.close()
