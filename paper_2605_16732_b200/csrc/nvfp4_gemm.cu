@@ -29,7 +29,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BN = kNvfp4BN;  // 128
 constexpr int BKE = 256;      // E2M1 elements per k-block (128-byte rows)
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * 128;      // 16 KB
 constexpr int B_BYTES = BN * 128;      // 16 KB
 constexpr int SF_BYTES = 4 * 512;      // four atoms per operand and k-block

@@ -148,6 +148,32 @@ def main():
             c = Case(4096, K, N, 32, 64, synth.PIXART)
             c.report("2: PixArt block linear, M=4096", args.iters, p_bf16, hbm)
             c.close()
+    if "2" in todo and FMT == "int4":
+        # q, k, v of a PixArt block read the same activations: one rotate/quantize pass, three second-kernel launches
+        cs = [Case(4096, 1152, 1152, 32, 64, synth.PIXART) for _ in range(3)]
+        def shared():
+            dq.dirotq_rotate_quantize(cs[0].x, cs[0].layer, cs[0].ws)
+            for c in cs:
+                dq.dirotq_w4a4_gemm(c.M, c.layer, cs[0].ws, c.y)
+        def separate():
+            for c in cs:
+                dq.dirotq_linear(cs[0].x, c.layer, c.y, c.ws)
+        res = {}
+        for name, fn in (("shared_rotation", shared), ("separate", separate)):
+            for _ in range(3):
+                fn()
+            ts = []
+            for _ in range(args.iters):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            res[name] = float(np.median(ts))
+        print(json.dumps({"config": "2: PixArt q/k/v projections (3 x 1152 -> 1152, M=4096) on one shared rotation",
+                          "shared_rotation_ms": res["shared_rotation"], "separate_ms": res["separate"],
+                          "speedup": res["separate"] / res["shared_rotation"]}), flush=True)
+        for c in cs:
+            c.close()
     if "4" in todo:
         for K, N in [(3072, 9216), (12288, 3072)]:
             for r in [int(v) for v in args.ranks.split(",")]:

@@ -205,3 +205,34 @@ def test_host_entry_point_equals_device_entry_point(M):
         assert torch.equal(yh.view(torch.int16), y.cpu().view(torch.int16))
     assert dq.dirotq_workspace_status(ws) == 0
     layer.close()
+
+
+def test_shared_rotation_across_linears_with_the_same_input():
+    """Linears that read the same activations and were calibrated on them have the same rotation (Sec. 4.2: the basis
+    depends only on the input's statistics), so one rotate/quantize pass serves them all: dirotq_rotate_quantize once,
+    then dirotq_w4a4_gemm per layer on the same workspace.  Must equal each layer's own dirotq_linear bit for bit."""
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=11)
+    M = 520
+    inp = synth.make_layer_inputs(spec, M)
+    Q = torch.from_numpy(inp["Q"]).cuda()
+    x = bits_to_bf16_tensor(inp["x"])
+    rng = np.random.default_rng(3)
+    layers, own = [], []
+    for i in range(3):  # q, k, v projections: same input, different weights
+        W = (0.02 * rng.standard_normal((spec.K, spec.N))).astype(np.float32)
+        layer = dq.dirotq_prepare_layer(torch.from_numpy(W).cuda(), Q, spec.r, spec.G)
+        ws = dq.alloc_workspace(layer, M)
+        y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device="cuda")
+        dq.dirotq_linear(x, layer, y, ws)
+        layers.append(layer)
+        own.append(y)
+    ws = dq.alloc_workspace(layers[0], M)
+    dq.dirotq_rotate_quantize(x, layers[0], ws)
+    for layer, y_own in zip(layers, own):
+        y = torch.zeros_like(y_own)
+        dq.dirotq_w4a4_gemm(M, layer, ws, y)
+        torch.cuda.synchronize()
+        assert torch.equal(y.view(torch.int16), y_own.view(torch.int16))
+    assert dq.dirotq_workspace_status(ws) == 0
+    for layer in layers:
+        layer.close()
