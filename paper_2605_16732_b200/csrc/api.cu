@@ -326,9 +326,9 @@ struct HostPipe {
 std::mutex g_pipe_mutex;
 HostPipe g_pipe[64];
 
+// Caller holds g_pipe_mutex (also while it enqueues on the pipe: its events are shared by all calls on the device).
 dirotq_status_t host_pipe(int dev, HostPipe** out) {
     if (dev < 0 || dev >= 64) return DIROTQ_ERR_INVALID_ARG;
-    std::lock_guard<std::mutex> lock(g_pipe_mutex);
     HostPipe& p = g_pipe[dev];
     if (!p.ready) {
         cudaError_t e = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking);
@@ -369,6 +369,7 @@ dirotq_status_t dirotq_linear_host(const void* x_host, int M, const dirotq_layer
         if (e != cudaSuccess) { set_error("cudaMemcpyAsync(D2H)", e); return DIROTQ_ERR_CUDA; }
         return DIROTQ_OK;
     }
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
     HostPipe* p = nullptr;
     st = host_pipe(layer->device, &p);
     if (st != DIROTQ_OK) return st;
