@@ -332,7 +332,7 @@ def run_ours(args):
     int8_peak = (4.0 if nv else 2.0) * peaks["bf16_sustained"]
     # DRAM bytes of one launch of the dominant kernel, from the ncu capture summarised under profiles/
     # (qkv shape; read + write).  Static: a profiler is never run inside the benchmark.
-    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 70.2e6, "rotate_quant_kernel": 48.5e6, "nvfp4_gemm_kernel": None}
+    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 75.5e6, "rotate_quant_kernel": 48.5e6, "nvfp4_gemm_kernel": 60.5e6}
     sm_hz = (clocks or {}).get("sm_mhz") or 1850.0
     elem_steps = sum(M * N * (-(-(K - RANK) // GROUP)) for _, K, N in FLUX_SHAPES)
     alu_peak = 148 * (128.0 / 2.0) * sm_hz * 1e6  # element-steps/s: 2 fused multiply-adds each, 128 fp32 lanes per SM

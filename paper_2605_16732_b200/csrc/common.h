@@ -150,8 +150,8 @@ struct dirotq_layer {
 namespace dirotq {
 
 constexpr uint32_t kLayerMagic = 0x44695251u;  // "DiRQ"
-constexpr int kGemmBN = 256;
-constexpr int kNvfp4BN = 128;  // output columns per tile of the NVFP4 kernel  // output columns per tile of the W4A4 kernel (rows of its weight-side TMA boxes)
+constexpr int kGemmBN = 256;   // output columns per tile of the W4A4 kernel (rows of its weight-side TMA boxes)
+constexpr int kNvfp4BN = 128;  // output columns per tile of the NVFP4 kernel
 
 // ------------------------------------------------------------------ kernel launch interfaces
 
