@@ -316,6 +316,45 @@ void dq_combine_asym(const int32_t* P, const uint16_t* sx, const uint16_t* zx, c
     }
 }
 
+/* =====================================================================================
+ * W4A8 (paper Sec. 5.1, "INT W4A8" rows of Table 1): 8-bit activations with one dynamic scale per
+ * token, 4-bit weights with one static scale per output channel ("per-token dynamic activation
+ * quantization and per-channel static weight quantization for 8-bit settings").
+ * Readings: symmetric on both sides (Eq. 1 with z = 0, q_max = 2^7 - 1 = 127 for the activations);
+ * the token's scale covers its K - r low-precision coefficients and is kept as bf16, the rounded
+ * value dividing and dequantizing; the weight side is Eq. 1 with one group spanning the whole
+ * column, i.e. dq_prepare_weights with G = K - r.  "Parity unpinned" against the authors' code.
+ * ===================================================================================== */
+
+/* xt[M,K] -> xh bf16 [M,r]; codes int8 [M,K_l]; scales bf16 [M]; t (optional) [M,K_l] */
+void dq_split_quantize_a8(const double* xt, int M, int K, int r, uint16_t* xh, int8_t* codes, uint16_t* scales, double* t) {
+    int K_l = K - r;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const double* row = xt + (int64_t)m * K;
+        for (int i = 0; i < r; ++i) xh[(int64_t)m * r + i] = dq_double_to_bf16(row[i]);
+        double a = 0.0;
+        for (int j = 0; j < K_l; ++j) {
+            double x = fabs(row[r + j]);
+            if (x > a) a = x;
+        }
+        uint16_t sb = (a == 0.0) ? 0 : dq_double_to_bf16(a / 127.0);      /* s = max|X| / q_max */
+        double s = dq_bf16_to_double(sb);
+        scales[m] = sb;
+        for (int j = 0; j < K_l; ++j) {
+            double q = 0.0, tj = 0.0;
+            if (s != 0.0) {
+                tj = row[r + j] / s;
+                q = rint(tj);
+                if (q > 127.0) q = 127.0;
+                if (q < -127.0) q = -127.0;
+            }
+            codes[(int64_t)m * K_l + j] = (int8_t)q;
+            if (t) t[(int64_t)m * K_l + j] = tj;
+        }
+    }
+}
+
 /* ---------- plain fp64 product, used by the ideal (nothing quantized) mode ------ */
 
 void dq_matmul(const double* A, const double* B, double* C, int M, int K, int N) {

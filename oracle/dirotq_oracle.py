@@ -279,6 +279,39 @@ def linear_deployed_asym(x_bits, layer, bias=None, want_t: bool = True):
             "P": P, "y64": y64, "y": yb}
 
 
+# ---------------------------------------------------------------------------------------------
+# W4A8 (Sec. 5.1): per-token INT8 activations, per-output-channel INT4 weights
+
+def prepare_layer_w4a8(W, Q, r: int, want_t: bool = False):
+    """The weight side is Eq. 1 with a single group spanning the column: prepare_layer with G = K - r."""
+    K = np.asarray(Q).shape[0]
+    return prepare_layer(W, Q, r, K - r, want_t=want_t)
+
+
+def split_quantize_a8(xt, r: int, want_t: bool = True):
+    xt = _c(xt, np.float64)
+    M, K = xt.shape
+    K_l = K - r
+    xh = np.empty((M, r), dtype=np.uint16)
+    codes = np.empty((M, K_l), dtype=np.int8)
+    scales = np.empty((M,), dtype=np.uint16)
+    t = np.empty((M, K_l), dtype=np.float64) if want_t else None
+    _load().dq_split_quantize_a8(_p(xt), ctypes.c_int(M), ctypes.c_int(K), ctypes.c_int(r), _p(xh), _p(codes), _p(scales),
+                                 _p(t))
+    return {"xh": xh, "codes": codes, "scales": scales, "t": t}
+
+
+def linear_deployed_w4a8(x_bits, layer, bias=None, want_t: bool = True):
+    r = layer["r"]
+    xt = rotate(x_bits, layer["Qb"])
+    sq = split_quantize_a8(xt, r, want_t=want_t)
+    K_l = xt.shape[1] - r
+    P = int_gemm(sq["codes"], layer["wcodes"], K_l)                      # one "group": the whole row
+    y64, yb = combine(P, sq["scales"].reshape(-1, 1), layer["wscales"], sq["xh"], layer["Wh"], bias)
+    return {"xt": xt, "xh": sq["xh"], "codes": sq["codes"], "scales": sq["scales"], "t": sq["t"], "P": P[0], "y64": y64,
+            "y": yb}
+
+
 def linear_ideal(x, Q, W, r: int):
     """Eq. 4 with nothing quantized and nothing rounded: [xU_h, x~_l] [W~_h; W~_l] in fp64."""
     x = _c(x, np.float64)
