@@ -199,6 +199,30 @@ DIROTQ_API dirotq_status_t dirotq_workspace_export_asym(const dirotq_layer_t* la
 DIROTQ_API dirotq_status_t dirotq_layer_export_zero_term(const dirotq_layer_t* layer, float* zero_term,
                                                          dirotq_stream_t stream);
 
+/* ---- W4A8 (paper Sec. 5.1 and the "INT W4A8" rows of Table 1: "per-token dynamic activation
+ * quantization and per-channel static weight quantization for 8-bit settings") ---- */
+
+/* Same layer with 8-bit activations and per-channel 4-bit weights, both symmetric (Eq. 1, z = 0): every
+ * token's K - r low-precision coefficients share one bf16 scale s_x[m] = max|x~| / 127 and are rounded to
+ * int8 codes in [-127, 127]; every output column of the folded weight has one bf16 scale
+ * s_w[n] = max|W~_l[:,n]| / 7 and int4 codes.  y = s_x s_w (q_x . q_w) + x~_h W~_h + bias, the integer
+ * product accumulated exactly in int32 over the whole of K (tcgen05.mma kind::i8).  A token's scale needs
+ * its whole rotated row, so the first stage is two kernels here (rotation writing fp32 coefficients and row
+ * maxima into the workspace, then the quantizer); the workspace is correspondingly larger
+ * (dirotq_workspace_bytes).  dirotq_linear, dirotq_linear_host, dirotq_linear_noalloc,
+ * dirotq_rotate_quantize, dirotq_w4a4_gemm (the second kernel, whatever the format), dirotq_layer_export
+ * (wscales then [1,N]), dirotq_int_gemm_debug (partials then [M,N], codes int8 [M,K_lp] read in place,
+ * K_lp = K - r rounded up to 128) and dirotq_layer_destroy accept such a layer. */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes_w4a8(int K, int N, int r, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_w4a8(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                                     const void* bias, int K, int N, int r, void* blob, size_t blob_bytes,
+                                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                                     dirotq_layer_t** layer_out);
+/* Parity export: xh bf16 [M,r]; codes int8 [M,K-r]; scales bf16 [M].  Any pointer may be NULL. */
+DIROTQ_API dirotq_status_t dirotq_workspace_export_w4a8(const dirotq_layer_t* layer, int M, const void* workspace,
+                                                        void* xh_bf16, int8_t* codes, void* scales_bf16,
+                                                        dirotq_stream_t stream);
+
 /* ---- NVFP4 variant (paper Sec. 5.1: "For 4-bit FP, we use NVFP4 ... group size 16 with FP8 scaling") ---- */
 
 /* Same layer with the 4-bit float format instead of INT4: elements are E2M1 (1 sign, 2 exponent,

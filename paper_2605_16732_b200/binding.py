@@ -28,6 +28,7 @@ EXPORTED = [
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_wait_counters", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
+    "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
     "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
@@ -75,6 +76,9 @@ def lib() -> ctypes.CDLL:
         L.dirotq_prepare_layer_nvfp4.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_workspace_export_nvfp4.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_layer_export_nvfp4.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.dirotq_layer_bytes_w4a8.argtypes = [i, i, i, psz]
+        L.dirotq_prepare_layer_w4a8.argtypes = [vp, i, i, vp, i, vp, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
+        L.dirotq_workspace_export_w4a8.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_layer_bytes_asym.argtypes = [i, i, i, i, psz]
         L.dirotq_prepare_layer_asym.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -232,7 +236,7 @@ def dirotq_int_gemm_debug(act_codes: torch.Tensor, layer: Layer, workspace: torc
     """act_codes: cuda int8 [M, K_lp] (zero in columns >= K - r).  Returns int32 [n_g, M, N]."""
     M = act_codes.shape[0]
     assert act_codes.shape[1] == layer.K_lp and act_codes.is_contiguous()
-    P = torch.empty((layer.n_g, M, layer.N), dtype=torch.int32, device=act_codes.device)
+    P = torch.empty((1 if layer.fmt == "w4a8" else layer.n_g, M, layer.N), dtype=torch.int32, device=act_codes.device)
     _check(lib().dirotq_int_gemm_debug(act_codes.data_ptr(), M, layer.handle, P.data_ptr(), workspace.data_ptr(),
                                        workspace.numel(), _stream(stream)), "dirotq_int_gemm_debug")
     return P
@@ -241,7 +245,7 @@ def dirotq_int_gemm_debug(act_codes: torch.Tensor, layer: Layer, workspace: torc
 def dirotq_layer_export(layer: Layer, stream=None):
     dev = layer.blob.device
     wcodes = torch.empty((layer.K_l, layer.N), dtype=torch.int8, device=dev)
-    wscales = torch.empty((layer.n_g, layer.N), dtype=torch.bfloat16, device=dev)
+    wscales = torch.empty((1 if layer.fmt == "w4a8" else layer.n_g, layer.N), dtype=torch.bfloat16, device=dev)
     wh = torch.empty((layer.r, layer.N), dtype=torch.bfloat16, device=dev)
     qb = torch.empty((layer.K, layer.K), dtype=torch.bfloat16, device=dev)
     _check(lib().dirotq_layer_export(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(), qb.data_ptr(),
@@ -365,3 +369,41 @@ def dirotq_layer_export_zero_term(layer: Layer, stream=None) -> torch.Tensor:
     d = torch.empty((layer.n_g, layer.N), dtype=torch.float32, device=layer.blob.device)
     _check(lib().dirotq_layer_export_zero_term(layer.handle, d.data_ptr(), _stream(stream)), "dirotq_layer_export_zero_term")
     return d
+
+
+# ------------------------------------------------------------------ W4A8
+
+def dirotq_layer_bytes_w4a8(K: int, N: int, r: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_layer_bytes_w4a8(K, N, r, ctypes.byref(out)), "dirotq_layer_bytes_w4a8")
+    return out.value
+
+
+def dirotq_prepare_layer_w4a8(W: torch.Tensor, Q: torch.Tensor, r: int, bias: torch.Tensor | None = None,
+                              w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """Per-token INT8 activations, per-channel INT4 weights (Layer.group is the packing granularity, 128)."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    blob = _alloc_bytes(dirotq_layer_bytes_w4a8(K, N, r), W.device)
+    scratch_bytes = dirotq_prepare_scratch_bytes(K, N)
+    scratch = _alloc_bytes(scratch_bytes, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_w4a8(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), K, N, r, blob.data_ptr(),
+                                         blob.numel(), scratch.data_ptr(), scratch_bytes, _stream(stream),
+                                         ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_w4a8")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, 128, fmt="w4a8")
+
+
+def dirotq_workspace_export_w4a8(layer: Layer, M: int, workspace: torch.Tensor, stream=None):
+    dev = workspace.device
+    xh = torch.empty((M, layer.r), dtype=torch.bfloat16, device=dev)
+    codes = torch.empty((M, layer.K_l), dtype=torch.int8, device=dev)
+    scales = torch.empty((M,), dtype=torch.bfloat16, device=dev)
+    _check(lib().dirotq_workspace_export_w4a8(layer.handle, M, workspace.data_ptr(), xh.data_ptr(), codes.data_ptr(),
+                                              scales.data_ptr(), _stream(stream)), "dirotq_workspace_export_w4a8")
+    return xh, codes, scales

@@ -131,9 +131,17 @@ dirotq_status_t dirotq_prepare_scratch_bytes(int K, int N, size_t* bytes) {
     return DIROTQ_OK;
 }
 
+static size_t workspace_need(const dirotq_layer_t* layer, int M) {
+    switch (layer->geo.fmt) {
+        case 1: return make_workspace_layout_nvfp4(layer->geo, M).total;
+        case 3: return make_workspace_layout_w4a8(layer->geo, M).total;
+        default: return make_workspace_layout(layer->geo, M).total;
+    }
+}
+
 dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_t* bytes) {
     if (!valid_layer(layer) || !bytes || M < 1) return DIROTQ_ERR_INVALID_ARG;
-    *bytes = layer->geo.fmt == 1 ? make_workspace_layout_nvfp4(layer->geo, M).total : make_workspace_layout(layer->geo, M).total;
+    *bytes = workspace_need(layer, M);
     return DIROTQ_OK;
 }
 
@@ -215,6 +223,69 @@ dirotq_status_t dirotq_prepare_layer_asym(const void* W, int w_dtype, int w_layo
                         scratch_bytes, stream, layer_out);
 }
 
+dirotq_status_t dirotq_layer_bytes_w4a8(int K, int N, int r, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, 64);
+    if (st != DIROTQ_OK) return st;
+    Geometry g = make_geometry(K, N, r, 128);
+    g.fmt = 3;
+    *bytes = make_blob_layout(g).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_w4a8(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                          const void* bias, int K, int N, int r, void* blob, size_t blob_bytes, void* scratch,
+                                          size_t scratch_bytes, dirotq_stream_t stream, dirotq_layer_t** layer_out) {
+    if (!W || !Q || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
+    if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
+    if (q_dtype != DIROTQ_DTYPE_F64 && q_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
+    if (w_layout != DIROTQ_LAYOUT_KN && w_layout != DIROTQ_LAYOUT_NK) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, 64);
+    if (st != DIROTQ_OK) return st;
+    if (!aligned16(W) || !aligned16(Q) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
+    Geometry g = make_geometry(K, N, r, 128);  // 128: packing granularity of the codes only
+    g.fmt = 3;
+    const BlobLayout lay = make_blob_layout(g);
+    if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (scratch_bytes < static_cast<size_t>(K) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    int dev = 0;
+    st = check_device(&dev);
+    if (st != DIROTQ_OK) return st;
+    dirotq_layer* L = new (std::nothrow) dirotq_layer;
+    if (!L) return DIROTQ_ERR_INVALID_ARG;
+    memset(L, 0, sizeof *L);
+    L->magic = kLayerMagic;
+    L->device = dev;
+    L->geo = g;
+    L->lay = lay;
+    L->blob = static_cast<char*>(blob);
+    st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                        (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = launch_prepare_w4a8(L, W, w_dtype, w_layout, Q, q_dtype, bias, static_cast<double*>(scratch),
+                                 static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) {
+        delete L;
+        return st;
+    }
+    *layer_out = L;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_workspace_export_w4a8(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
+                                             int8_t* codes, void* scales_bf16, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || layer->geo.fmt != 3 || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
+    return launch_workspace_export_w4a8(layer, M, static_cast<const char*>(workspace), static_cast<uint16_t*>(xh_bf16), codes,
+                                        static_cast<uint16_t*>(scales_bf16), static_cast<cudaStream_t>(stream));
+}
+
 dirotq_status_t dirotq_workspace_export_asym(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
                                              uint8_t* codes, void* scales_bf16, void* zeros_bf16, dirotq_stream_t stream) {
     if (!valid_layer(layer) || layer->geo.fmt != 2 || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
@@ -249,13 +320,25 @@ dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K, int* N, i
 static dirotq_status_t check_call(const dirotq_layer_t* layer, int M, const void* workspace, size_t workspace_bytes) {
     if (!valid_layer(layer) || !workspace || M < 1) return DIROTQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
-    const size_t need = layer->geo.fmt == 1 ? make_workspace_layout_nvfp4(layer->geo, M).total
-                                            : make_workspace_layout(layer->geo, M).total;
-    if (workspace_bytes < need) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (workspace_bytes < workspace_need(layer, M)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
     return DIROTQ_OK;
 }
 
 static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M, char* ws, float* xrot) {
+    if (layer->geo.fmt == 3) {
+        const WorkspaceLayoutA8 w = make_workspace_layout_w4a8(layer->geo, M);
+        RotateArgs a;
+        a.x = x; a.M = M;
+        a.codes = reinterpret_cast<int8_t*>(ws + w.off_codes);
+        a.xscale = reinterpret_cast<float*>(ws + w.off_xscale);
+        a.ldm = 0;
+        a.xh = reinterpret_cast<uint16_t*>(ws + w.off_xh);
+        a.xrot = xrot;
+        a.status = reinterpret_cast<int*>(ws + w.off_status);
+        a.xtilde = reinterpret_cast<float*>(ws + w.off_xtilde);
+        a.rowmax = reinterpret_cast<unsigned int*>(ws + w.off_rowmax);
+        return a;
+    }
     const bool nv = layer->geo.fmt == 1;
     const WorkspaceLayout w = nv ? make_workspace_layout_nvfp4(layer->geo, M) : make_workspace_layout(layer->geo, M);
     RotateArgs a;
@@ -270,7 +353,25 @@ static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M,
     return a;
 }
 
+// First kernel(s): rotation + split + quantization.  W4A8 needs the token's whole row before it can quantize: the rotation
+// kernel writes fp32 coefficients and the row maxima, a second small kernel quantizes.
+static dirotq_status_t first_kernel(const dirotq_layer_t* layer, const RotateArgs& ra, int M, cudaStream_t s) {
+    if (layer->geo.fmt == 3) {
+        if (cudaMemsetAsync(ra.rowmax, 0, static_cast<size_t>(M) * 4, s) != cudaSuccess) return DIROTQ_ERR_CUDA;
+        dirotq_status_t st = launch_rotate_quantize(layer, ra, s);
+        if (st != DIROTQ_OK) return st;
+        return launch_a8_quantize(layer, M, ra.xtilde, ra.rowmax, ra.codes, ra.xscale, s);
+    }
+    return launch_rotate_quantize(layer, ra, s);
+}
+
 static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateArgs& ra, int M, void* y, cudaStream_t s) {
+    if (layer->geo.fmt == 3) {
+        A8GemmArgs ga;
+        ga.M = M; ga.codes = ra.codes; ga.xscale = ra.xscale; ga.xh = ra.xh;
+        ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr; ga.status = ra.status;
+        return launch_w4a8_gemm(layer, ga, s);
+    }
     if (layer->geo.fmt == 1) {
         Nvfp4GemmArgs na;
         na.M = M; na.codes = reinterpret_cast<const uint8_t*>(ra.codes); na.xsf = ra.xsf; na.xh = ra.xh;
@@ -288,8 +389,8 @@ dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_
     dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
     if (st != DIROTQ_OK) return st;
     if (!x || !aligned16(x) || (xrot_f32 && !aligned16(xrot_f32))) return DIROTQ_ERR_INVALID_ARG;
-    return launch_rotate_quantize(layer, rotate_args(layer, x, M, static_cast<char*>(workspace), xrot_f32),
-                                  static_cast<cudaStream_t>(stream));
+    return first_kernel(layer, rotate_args(layer, x, M, static_cast<char*>(workspace), xrot_f32), M,
+                        static_cast<cudaStream_t>(stream));
 }
 
 dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer, void* y, void* workspace,
@@ -299,7 +400,7 @@ dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer,
     if (!x || !y || !aligned16(x) || !aligned16(y)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = static_cast<char*>(workspace);
     const RotateArgs ra = rotate_args(layer, x, M, ws, nullptr);
-    st = launch_rotate_quantize(layer, ra, static_cast<cudaStream_t>(stream));
+    st = first_kernel(layer, ra, M, static_cast<cudaStream_t>(stream));
     if (st != DIROTQ_OK) return st;
     return second_kernel(layer, ra, M, y, static_cast<cudaStream_t>(stream));
 }
@@ -432,6 +533,16 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
     dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
     if (st != DIROTQ_OK) return st;
     if (layer->geo.fmt == 1) return DIROTQ_ERR_INVALID_ARG;
+    if (layer->geo.fmt == 3) {  // one sum per output: partials [M][N]; the caller's codes are read in place
+        if (!act_codes || !partials || !aligned16(act_codes) || !aligned16(partials)) return DIROTQ_ERR_INVALID_ARG;
+        const WorkspaceLayoutA8 w8 = make_workspace_layout_w4a8(layer->geo, M);
+        char* ws8 = static_cast<char*>(workspace);
+        A8GemmArgs ga;
+        ga.M = M; ga.codes = act_codes; ga.xscale = reinterpret_cast<const float*>(ws8 + w8.off_xscale);
+        ga.xh = reinterpret_cast<const uint16_t*>(ws8 + w8.off_xh);
+        ga.y = nullptr; ga.partials = partials; ga.status = reinterpret_cast<int*>(ws8 + w8.off_status);
+        return launch_w4a8_gemm(layer, ga, static_cast<cudaStream_t>(stream));
+    }
     if (!act_codes || !partials || !aligned16(act_codes) || !aligned16(partials)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = static_cast<char*>(workspace);
     const WorkspaceLayout w = make_workspace_layout(layer->geo, M);

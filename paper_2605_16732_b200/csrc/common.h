@@ -24,7 +24,9 @@ struct Geometry {
     int r_pad0; // r rounded up to a multiple of 64: where the zero-point columns of fmt 2 start
     // NVFP4 variant only (fmt == 1): blocks of 16, MMA K = 64, TMA k-blocks of 256 elements
     int fmt;     // 0 = INT4 groups with bf16 scales, 1 = NVFP4 (E2M1 elements, E4M3 block scales),
-                 // 2 = INT4 with asymmetric activation codes (0..15, bf16 scale and zero-point per group)
+                 // 2 = INT4 with asymmetric activation codes (0..15, bf16 scale and zero-point per group),
+                 // 3 = W4A8: INT8 activations with one scale per token, INT4 weights with one scale per output column
+                 //     (G = 128 is then only the packing granularity: K_lp = K_l rounded up to 128, n_g = K_lp / 128)
     int K4;      // K_l rounded up to 64 (<= K): width of the packed E2M1 rows
     int nkb64;   // K4 / 64: scale-factor atoms (128 rows x 4 scales) per row block
     int nkb64p;  // nkb64 rounded up to 4: one TMA k-block = 256 elements = 4 atoms
@@ -119,6 +121,24 @@ inline WorkspaceLayout make_workspace_layout(const Geometry& g, int M) {
     return w;
 }
 
+// W4A8 (fmt 3): off_codes = int8 [M][K_lp]; off_xscale = f32 [M] token scales; off_xtilde = f32 [M][K_lp] rotated
+// low-precision coefficients (first pass); off_rowmax = u32 [M] bit patterns of the tokens' max |x~| (atomic max).
+struct WorkspaceLayoutA8 {
+    size_t off_status, off_codes, off_xscale, off_rowmax, off_xh, off_xtilde, total;
+};
+inline WorkspaceLayoutA8 make_workspace_layout_w4a8(const Geometry& g, int M) {
+    WorkspaceLayoutA8 w;
+    size_t o = 0;
+    w.off_status = o;  o = align_up(o + 256);
+    w.off_codes = o;   o = align_up(o + (size_t)M * g.K_lp);
+    w.off_xscale = o;  o = align_up(o + (size_t)M * 4);
+    w.off_rowmax = o;  o = align_up(o + (size_t)M * 4);
+    w.off_xh = o;      o = align_up(o + (size_t)M * g.r_pad * 2);
+    w.off_xtilde = o;  o = align_up(o + (size_t)M * g.K_lp * 4);
+    w.total = o;
+    return w;
+}
+
 inline WorkspaceLayout make_workspace_layout_nvfp4(const Geometry& g, int M) {
     WorkspaceLayout w;
     w.ldm = 0;
@@ -165,6 +185,18 @@ struct RotateArgs {
     float* xrot;  // optional fp32 [M][K], columns in the caller's (unpermuted) order
     int* status;
     uint8_t* xsf = nullptr;  // NVFP4 variant: scale-factor atoms (codes then holds packed E2M1)
+    float* xtilde = nullptr;       // W4A8: fp32 [M][K_lp] rotated low-precision coefficients
+    unsigned int* rowmax = nullptr;  // W4A8: bit patterns of the tokens' max |x~| (zeroed before the launch)
+};
+
+struct A8GemmArgs {
+    int M;
+    const int8_t* codes;   // [M][K_lp]
+    const float* xscale;   // [M]
+    const uint16_t* xh;    // bf16 [M][r_pad]
+    uint16_t* y;           // bf16 [M][N]
+    int32_t* partials;     // debug: int32 [M][N]; when set, y is not written
+    int* status;
 };
 
 struct GemmArgs {
@@ -210,6 +242,13 @@ dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char
 dirotq_status_t launch_workspace_export_asym(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
                                              uint8_t* codes, uint16_t* scales, uint16_t* zeros, cudaStream_t stream);
 dirotq_status_t launch_zero_term_export(const dirotq_layer* L, float* d, cudaStream_t stream);
+dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cudaStream_t stream);
+dirotq_status_t launch_a8_quantize(const dirotq_layer* L, int M, const float* xtilde, const unsigned int* rowmax, int8_t* codes,
+                                   float* xscale, cudaStream_t stream);
+dirotq_status_t launch_prepare_w4a8(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
+                                    int q_dtype, const void* bias, double* scratch, cudaStream_t stream);
+dirotq_status_t launch_workspace_export_w4a8(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh, int8_t* codes,
+                                             uint16_t* scales, cudaStream_t stream);
 dirotq_status_t launch_debug_codes(const dirotq_layer* L, int M, const int8_t* act_codes, char* workspace,
                                    cudaStream_t stream);
 int sm_count(int device);

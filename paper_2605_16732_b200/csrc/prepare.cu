@@ -261,6 +261,77 @@ __global__ void debug_codes_kernel(const int8_t* in, uint8_t* out, float* xscale
     xscale[static_cast<size_t>(g.n_g + grp) * ldm + m] = -8.0f * static_cast<float>(sum);
 }
 
+// ================================================================ W4A8 (paper Sec. 5.1: per-channel 4-bit weights, per-token 8-bit activations)
+
+// One thread per output column: Eq. 1 with z = 0 over the whole column (one scale per channel), codes packed like
+// the grouped format (nibble = q + 8).
+__global__ void w4a8_quantize_weights_kernel(const double* Wt, uint8_t* wpacked, float* wscale, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= g.N) return;
+    const double* col = Wt + static_cast<size_t>(g.r) * g.N + n;
+    double a = 0.0;
+    for (int j = 0; j < g.K_l; ++j) a = fmax(a, fabs(col[static_cast<size_t>(j) * g.N]));
+    const uint16_t sb = (a == 0.0) ? 0 : f64_to_bf16(a / 7.0);
+    const double s = bf16_to_f64(sb);
+    wscale[n] = static_cast<float>(s);
+    uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
+    for (int jb = 0; jb < g.K_lp; jb += 8) {
+        uint32_t word = 0;
+        for (int t = 0; t < 8; ++t) {
+            const int j = jb + t;
+            int q = 0;
+            if (j < g.K_l && s != 0.0) {
+                double qq = rint(col[static_cast<size_t>(j) * g.N] / s);
+                qq = fmin(7.0, fmax(-7.0, qq));
+                q = static_cast<int>(qq);
+            }
+            word |= (static_cast<uint32_t>(q + 8) & 0xFu) << (8 * (t & 3) + 4 * (t >> 2));
+        }
+        *reinterpret_cast<uint32_t*>(row + packed_byte_index(jb)) = word;
+    }
+}
+
+// Second pass of the W4A8 activation side, one warp per token: s = bf16(max|x~| / 127), q = clip(rint(x~ / s), -127, 127).
+__global__ void a8_quantize_kernel(const float* xtilde, const unsigned int* rowmax, int8_t* codes, float* xscale, int M,
+                                   Geometry g) {
+    const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (m >= M) return;
+    const float amax = __uint_as_float(rowmax[m]);
+    const float s = amax > 0.f ? __bfloat162float(__float2bfloat16_rn(__fdiv_rn(amax, 127.0f))) : 0.f;
+    const bool slow = !(s >= 1e-30f);
+    const float inv = slow ? 0.f : __frcp_rn(s);
+    if (lane == 0) xscale[m] = s;
+    const float* xr = xtilde + static_cast<size_t>(m) * g.K_lp;
+    int8_t* cr = codes + static_cast<size_t>(m) * g.K_lp;
+    for (int j = lane * 4; j < g.K_lp; j += 128) {
+        uint32_t word = 0;
+        if (j < g.K_l) {  // K_l is a multiple of 16: the four values are all real or all padding
+            const float4 v = *reinterpret_cast<const float4*>(xr + j);
+            const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                float q = slow ? (s != 0.f ? vv[t] / s : 0.f) : vv[t] * inv;
+                q = fminf(fmaxf(q, -127.0f), 127.0f);
+                word |= (static_cast<uint32_t>(__float2int_rn(q)) & 0xFFu) << (8 * t);
+            }
+        }
+        *reinterpret_cast<uint32_t*>(cr + j) = word;
+    }
+}
+
+__global__ void export_workspace_w4a8_kernel(const int8_t* codes, const float* xscale, const uint16_t* xh_pad, int M, Geometry g,
+                                             uint16_t* xh, int8_t* codes_out, uint16_t* scales) {
+    const int m = blockIdx.y;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < g.K_l; c += gridDim.x * blockDim.x)
+        if (codes_out) codes_out[static_cast<size_t>(m) * g.K_l + c] = codes[static_cast<size_t>(m) * g.K_lp + c];
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < g.r; i += blockDim.x)
+            if (xh) xh[static_cast<size_t>(m) * g.r + i] = xh_pad[static_cast<size_t>(m) * g.r_pad + i];
+        if (threadIdx.x == 0 && scales) scales[m] = static_cast<uint16_t>(__float_as_uint(xscale[m]) >> 16);
+    }
+}
+
 // ================================================================ NVFP4 variant (paper Sec. 5.1)
 // E2M1 elements, blocks of 16 along K with an E4M3 scale, one power-of-two scale per tensor.
 // Everything offline is done in fp64 so that codes and scales equal the CPU checker's.
@@ -456,7 +527,7 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
     }
     if (wscales) {
-        const size_t count = static_cast<size_t>(g.n_g) * g.N;
+        const size_t count = static_cast<size_t>(g.fmt == 3 ? 1 : g.n_g) * g.N;  // W4A8: one scale per output column
         export_wscales_kernel<<<static_cast<unsigned>((count + 255) / 256), 256, 0, stream>>>(
             reinterpret_cast<const float*>(blob + L->lay.off_wscale), wscales, count);
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
@@ -472,6 +543,42 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
     }
     return DIROTQ_OK;
+}
+
+dirotq_status_t launch_prepare_w4a8(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
+                                    int q_dtype, const void* bias, double* scratch, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    char* blob = L->blob;
+    fold_kernel<<<dim3((g.N + 63) / 64, (g.K + 63) / 64), 256, 0, stream>>>(Q, q_dtype, W, w_dtype, w_layout, scratch,
+                                                                          g.K, g.N);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    w4a8_quantize_weights_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(
+        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
+        Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                       reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_a8_quantize(const dirotq_layer* L, int M, const float* xtilde, const unsigned int* rowmax, int8_t* codes,
+                                   float* xscale, cudaStream_t stream) {
+    a8_quantize_kernel<<<(M + 7) / 8, 256, 0, stream>>>(xtilde, rowmax, codes, xscale, M, L->geo);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_workspace_export_w4a8(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh, int8_t* codes,
+                                             uint16_t* scales, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    const WorkspaceLayoutA8 w = make_workspace_layout_w4a8(g, M);
+    export_workspace_w4a8_kernel<<<dim3(8, M), 256, 0, stream>>>(
+        reinterpret_cast<const int8_t*>(workspace + w.off_codes), reinterpret_cast<const float*>(workspace + w.off_xscale),
+        reinterpret_cast<const uint16_t*>(workspace + w.off_xh), M, g, xh, codes, scales);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 dirotq_status_t launch_workspace_export_asym(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,

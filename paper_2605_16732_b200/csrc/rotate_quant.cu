@@ -42,6 +42,9 @@ struct RotKernelParams {
     uint8_t* xsf;     // scale-factor atoms [ceil(M/128)][nkb64p][512]
     int K4, nkb64p;   // packed row width in elements; atoms per row block
     int ex;           // exponent of the activations' per-tensor power-of-two scale
+    // W4A8 variant: first pass only (the token's scale needs its whole row)
+    float* xtilde;          // fp32 [M][K_lp]
+    unsigned int* rowmax;   // per-token max |x~_l| as a bit pattern, atomic max (zeroed by the host before the launch)
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -260,6 +263,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const bool row_ok = row < p.M;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
 
+            float tile_amax = 0.f;  // W4A8: this thread's row, this tile's columns
 #pragma unroll 1
             for (int chunk = 0; chunk < BN / G; ++chunk) {
                 const int col0 = n0 + chunk * G;  // permuted column of v[0]
@@ -309,6 +313,24 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                             for (int a = (col0 >> 6) + 1; a < p.nkb64p; ++a)
                                 *reinterpret_cast<uint32_t*>(p.xsf + (static_cast<size_t>(row >> 7) * p.nkb64p + a) * 512 +
                                                              (mr & 31) * 16 + (mr >> 5) * 4) = 0u;
+                    }
+                } else if constexpr (FMT == 3) {
+                    // W4A8, first pass: the rotated low-precision coefficients go out as fp32 and the token's maximum is
+                    // gathered with an atomic max (non-negative floats order like their bit patterns)
+                    if (nlow > 0 && row_ok) {
+                        float4* dst = reinterpret_cast<float4*>(p.xtilde + static_cast<size_t>(row) * p.K_lp + col0);
+#pragma unroll
+                        for (int b = 0; b < G / 16; ++b) {
+                            if (16 * b < nlow) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const float4 q4 = make_float4(v[16 * b + 4 * j], v[16 * b + 4 * j + 1], v[16 * b + 4 * j + 2],
+                                                                  v[16 * b + 4 * j + 3]);
+                                    dst[4 * b + j] = q4;
+                                    tile_amax = fmaxf(tile_amax, fmaxf(fmaxf(fabsf(q4.x), fabsf(q4.y)), fmaxf(fabsf(q4.z), fabsf(q4.w))));
+                                }
+                            }
+                        }
                     }
                 } else if constexpr (FMT == 2) {
                     if (nlow > 0 && row_ok) {
@@ -391,6 +413,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
             }
+            if constexpr (FMT == 3) {
+                if (row_ok && tile_amax > 0.f) atomicMax(p.rowmax + row, __float_as_uint(tile_amax));
+            }
             // release the accumulator: every tcgen05.ld of this warp has completed
             tc_fence_before_sync();
             __syncwarp();
@@ -429,12 +454,14 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
     const int num_tiles = ((a.M + BM - 1) / BM) * ((g.K + BN - 1) / BN);
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
-    const int vi = g.fmt == 1 ? 2 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
+    p.xtilde = a.xtilde; p.rowmax = a.rowmax;
+    const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
     auto kern = vi == 2 ? rotate_quant_kernel<64, 1>
+              : vi == 5 ? rotate_quant_kernel<64, 3>
               : vi == 3 ? rotate_quant_kernel<64, 2>
               : vi == 4 ? rotate_quant_kernel<128, 2>
               : vi == 0 ? rotate_quant_kernel<64, 0> : rotate_quant_kernel<128, 0>;
-    static bool attr_set[5] = {false, false, false, false, false};
+    static bool attr_set[6] = {false, false, false, false, false, false};
     if (!attr_set[vi]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;

@@ -1,0 +1,320 @@
+// W4A8 variant of the second kernel (paper Sec. 5.1, "INT W4A8": 8-bit activations with one scale per
+// token, 4-bit weights with one scale per output column).
+//
+//   y[m,n] = bf16( s_x[m] s_w[n] P[m,n]  +  sum_{i<r} x~_h[m,i] W~_h[i,n]  +  bias[n] ),
+//   P[m,n] = sum_j q_x[m,j] q_w[j,n]                  (int8 x int4, exact in int32)
+//
+// With one scale per row and per column there is no rescale inside K: the whole contraction runs on
+// tcgen05.mma kind::i8 into one int32 accumulator tile and the CUDA cores touch every output once.
+// The weight codes stay packed (two per byte, nibble = q + 8) in HBM and in the TMA staging buffer;
+// four unpack warps turn every nibble into the byte 16 q (shift the nibble into the high half, flip
+// bit 7: 16 (q + 8) - 128), so the accumulator holds 16 P and the epilogue shifts it back.
+//
+// Roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 unpack,
+// warps 6..9 epilogue (one token row per thread).  TMEM: columns 0..255 the int32 tile, 256..511 the
+// fp32 tile of the bf16 rank-r branch (kind::f16 cannot accumulate into the integer tile); single
+// buffered, so the epilogue of a tile (one pass) is not overlapped with the next tile's MMAs.
+#include "common.h"
+#include "ptx.cuh"
+
+#include <cuda_bf16.h>
+
+namespace dirotq {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = kGemmBN;  // 256
+constexpr int BKC = 128;     // one-byte codes per k-block (128-byte rows)
+constexpr int STAGES = 3;
+constexpr int A_BYTES = BM * BKC;       // 16 KB activation codes / bf16 x~_h chunk
+constexpr int BU_BYTES = BN * BKC;      // 32 KB unpacked weight codes / bf16 W~_h chunk
+constexpr int BP_BYTES = BN * BKC / 2;  // 16 KB packed weight codes (TMA staging)
+constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;
+constexpr int NUM_THREADS = 320;
+constexpr int NUM_UNPACK_WARPS = 4;
+constexpr int NUM_EPI_WARPS = 4;
+constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+
+struct A8KernelParams {
+    int M, N, num_kb, lr_chunks;
+    const float* xscale;  // [M]
+    const float* wscale;  // [N]
+    const float* bias;    // [N]
+    uint16_t* y;
+    int32_t* partials;
+    int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ void tmem_ld_fence32(uint32_t (&v)[32]) {
+    asm volatile("" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                      "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                      "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                      "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+                 :: "memory");
+}
+
+template <bool kPartials>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
+                 const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
+                 const A8KernelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t bar_base = smem_base + BAR_OFFSET;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto unp_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
+    const uint32_t tfull_bar = bar_base + 8u * (3 * STAGES);
+    const uint32_t tempty_bar = bar_base + 8u * (3 * STAGES + 1);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 128);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 132);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_m_blocks = (p.M + BM - 1) / BM;
+    const int num_n_blocks = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m_blocks * num_n_blocks;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(unp_bar(s), NUM_UNPACK_WARPS);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(tfull_bar, 1);
+        mbar_init(tempty_bar, NUM_EPI_WARPS);
+        *abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_codes);
+        tma_prefetch_desc(&tmap_wpacked);
+        tma_prefetch_desc(&tmap_xh);
+        tma_prefetch_desc(&tmap_wh);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const int items = p.num_kb + p.lr_chunks;  // pipeline items per tile
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m0 = (tile % num_m_blocks) * BM;
+                const int n0 = (tile / num_m_blocks) * BN;
+                for (int i = 0; i < items; ++i, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                    const uint32_t st = smem_base + s * STAGE_BYTES;
+                    if (i < p.num_kb) {
+                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
+                        tma_load_2d(st, &tmap_codes, full_bar(s), i * BKC, m0);
+                        tma_load_2d(st + A_BYTES + BU_BYTES, &tmap_wpacked, full_bar(s), i * (BKC / 2), n0);
+                    } else {
+                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BU_BYTES);
+                        tma_load_2d(st, &tmap_xh, full_bar(s), (i - p.num_kb) * 64, m0);
+                        tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), (i - p.num_kb) * 64, n0);
+                    }
+                }
+            }
+            if (!ok) {  // let the copies in flight land before the CTA's shared memory goes away
+                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1) && globaltimer_ns() - t0 < 100000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);
+            constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+                if (!mbar_wait(tempty_bar, (tcount & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                tc_fence_after_sync();
+                for (int i = 0; i < items; ++i, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
+                        !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t st = smem_base + s * STAGE_BYTES;
+                    const uint64_t adesc = umma_desc_sw128(st);
+                    const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+                    if (i < p.num_kb) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_i8(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16(tmem_base + BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, ((i - p.num_kb) | k) != 0);
+                    }
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(tfull_bar);
+            }
+        }
+    } else if (warp < 2 + NUM_UNPACK_WARPS) {
+        // ------------------------------------------------------------ nibble -> byte unpack (warps 2..5)
+        const int u = threadIdx.x - 64;  // 0..127
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int i = 0; i < items; ++i, ++it) {
+                const int s = it % STAGES;
+                ok = mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+                ok = __any_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (i < p.num_kb) {
+                    // 16-byte piece idx = u + 128 j of the packed tile: row = idx / 4 = u / 4 + 32 j, piece c = u % 4; the
+                    // swizzle phase row % 8 and the piece do not depend on j
+                    uint8_t* st = smem_gen + s * STAGE_BYTES;
+                    const uint4* src = reinterpret_cast<const uint4*>(st + A_BYTES + BU_BYTES) + u;
+                    const int c = u & 3, sw = (u >> 2) & 7;
+                    uint8_t* d0 = st + A_BYTES + (u >> 2) * 128 + (((2 * c) ^ sw) << 4);
+                    uint8_t* d1 = st + A_BYTES + (u >> 2) * 128 + (((2 * c + 1) ^ sw) << 4);
+                    uint4 pk[8];  // loads before stores: the compiler cannot prove the two buffers disjoint
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) pk[j] = src[128 * j];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        // nibble q + 8 -> byte 16 q: into the high half, then flip bit 7 (16 (q + 8) - 128)
+                        uint4 o0, o1;
+                        o0.x = ((pk[j].x << 4) & 0xF0F0F0F0u) ^ 0x80808080u; o0.y = (pk[j].x & 0xF0F0F0F0u) ^ 0x80808080u;
+                        o0.z = ((pk[j].y << 4) & 0xF0F0F0F0u) ^ 0x80808080u; o0.w = (pk[j].y & 0xF0F0F0F0u) ^ 0x80808080u;
+                        o1.x = ((pk[j].z << 4) & 0xF0F0F0F0u) ^ 0x80808080u; o1.y = (pk[j].z & 0xF0F0F0F0u) ^ 0x80808080u;
+                        o1.z = ((pk[j].w << 4) & 0xF0F0F0F0u) ^ 0x80808080u; o1.w = (pk[j].w & 0xF0F0F0F0u) ^ 0x80808080u;
+                        *reinterpret_cast<uint4*>(d0 + j * 4096) = o0;  // 32 rows of 128 bytes further down
+                        *reinterpret_cast<uint4*>(d1 + j * 4096) = o1;
+                    }
+                    fence_proxy_async_smem();
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(unp_bar(s));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 6..9)
+        const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            const int m0 = (tile % num_m_blocks) * BM;
+            const int n0 = (tile / num_m_blocks) * BN;
+            ok = mbar_wait(tfull_bar, tcount & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+            ok = __any_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int row = m0 + q * 32 + lane;
+            const float sx = row < p.M ? __ldg(p.xscale + row) : 0.f;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t acc[32], lr[32];
+                tmem_ld_32x32b_x32(taddr + c * 32, acc);
+                tmem_ld_32x32b_x32(taddr + BN + c * 32, lr);
+                tmem_ld_wait();
+                tmem_ld_fence32(acc);
+                tmem_ld_fence32(lr);
+                if (c == BN / 32 - 1) {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar);
+                }
+                const int col = n0 + c * 32;
+                if (row < p.M) {
+                    if constexpr (kPartials) {
+                        int32_t* dst = p.partials + static_cast<size_t>(row) * p.N + col;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (col + j < p.N)
+                                *reinterpret_cast<int4*>(dst + j) =
+                                    make_int4(static_cast<int32_t>(acc[j]) >> 4, static_cast<int32_t>(acc[j + 1]) >> 4,
+                                              static_cast<int32_t>(acc[j + 2]) >> 4, static_cast<int32_t>(acc[j + 3]) >> 4);
+                    } else {
+                        uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + col;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            if (col + j < p.N) {
+                                float o[8];
+#pragma unroll
+                                for (int t = 0; t < 8; t += 4) {
+                                    const float4 sw = __ldg(reinterpret_cast<const float4*>(p.wscale + col + j + t));
+                                    const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col + j + t));
+                                    const float sws[4] = {sw.x, sw.y, sw.z, sw.w}, bs[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        // the accumulator holds 16 P (exact); |P| < 2^24, so the conversion is exact too
+                                        const float pf = static_cast<float>(static_cast<int32_t>(acc[j + t + e]) >> 4);
+                                        o[t + e] = fmaf(pf * sx, sws[e], __uint_as_float(lr[j + t + e])) + bs[e];
+                                    }
+                                }
+                                *reinterpret_cast<uint4*>(yrow + j) = make_uint4(pack_bf16x2(o[0], o[1]), pack_bf16x2(o[2], o[3]),
+                                                                                 pack_bf16x2(o[4], o[5]), pack_bf16x2(o[6], o[7]));
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace
+
+dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    CUtensorMap tmap_codes, tmap_xh;
+    dirotq_status_t st;
+    st = encode_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K_lp, (uint64_t)a.M,
+                        (uint64_t)g.K_lp, BKC, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,
+                        (uint64_t)g.r_pad * 2, 64, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    A8KernelParams p;
+    p.M = a.M; p.N = g.N;
+    p.num_kb = g.K_lp / BKC;
+    p.lr_chunks = g.r_pad / 64;
+    p.xscale = a.xscale;
+    p.wscale = reinterpret_cast<const float*>(L->blob + L->lay.off_wscale);
+    p.bias = reinterpret_cast<const float*>(L->blob + L->lay.off_bias);
+    p.y = a.y; p.partials = a.partials; p.status = a.status;
+    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
+    const bool dbg = a.partials != nullptr;
+    auto kern = dbg ? w4a8_gemm_kernel<true> : w4a8_gemm_kernel<false>;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[dbg]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return DIROTQ_ERR_CUDA;
+        attr_set[dbg] = true;
+    }
+    kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace dirotq

@@ -328,3 +328,59 @@ def check_layer_output_asym(y_bits, xh_bits, codes, scales, zeros, layer_orc, ou
     e2e = check_output(y_bits, out_orc["y64"], rows=clean, slack=slack)
     stats["e2e_clean_max_err_over_rms"] = e2e.get("max_err_over_rms")
     return stats
+
+
+# ------------------------------------------------------------------ W4A8 (per-token INT8 activations, per-channel INT4 weights)
+#
+# Protocol: weights as in the grouped case (one "group" per column); the token scale equals the oracle's or is the
+# neighbouring bf16 value when the unrounded max|x~|/127 lies within 1e-4 (relative) + 1e-5 ||x~_row|| / 127 of the
+# midpoint; codes against the quantizer re-run with the library's scale (+-1 within 1e-3 + 1e-5 ||x~_row|| / s of a
+# rounding boundary); int32 sums bit for bit; output within half a bf16 step + slack * rms of the fp64 combination of
+# the library's own intermediates.
+
+def check_activation_side_w4a8(xrot, xh, codes, scales, out_orc, r):
+    xt = out_orc["xt"]
+    M, K = xt.shape
+    stats = {}
+    norm = np.linalg.norm(xt, axis=1)
+    if xrot is not None:
+        rel = np.linalg.norm(xrot.astype(np.float64) - xt, axis=1) / np.maximum(norm, 1e-300)
+        stats["xrot_rel_max"] = float(rel.max())
+        assert rel.max() <= 2e-3
+    xh_g, xh_o = f64(xh), f64(out_orc["xh"])
+    step = np.maximum(np.abs(xh_o), 2.0 ** -126) * 2.0 ** -7 + 1e-5 * norm[:, None]
+    assert np.all(np.abs(xh_g - xh_o) <= step), "x~_h differs by more than one bf16 step"
+    s_g, s_o = f64(scales), f64(out_orc["scales"])
+    u = np.abs(xt[:, r:]).max(axis=1) / 127.0
+    flip = scales != out_orc["scales"]
+    if flip.any():
+        db = np.abs(scales[flip].astype(np.int64) - out_orc["scales"][flip].astype(np.int64))
+        assert np.all(db == 1), "a token scale is more than one bf16 step away"
+        mid = 0.5 * (s_g[flip] + s_o[flip])
+        assert np.all(np.abs(u[flip] - mid) <= 1e-4 * u[flip] + 1e-5 * norm[flip] / 127.0)
+    stats["scale_flips"] = int(flip.sum())
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(s_g[:, None] != 0, xt[:, r:] / s_g[:, None], 0.0)
+    q_ref = np.clip(np.rint(t), -127, 127).astype(np.int8)
+    assert np.array_equal(q_ref[~flip], out_orc["codes"][~flip])
+    bad = codes != q_ref
+    if bad.any():
+        assert np.all(np.abs(codes[bad].astype(int) - q_ref[bad].astype(int)) == 1), "a code is off by more than 1"
+        dist = np.abs(np.abs(t[bad] - np.floor(t[bad])) - 0.5)
+        with np.errstate(divide="ignore"):
+            tol = 1e-3 + 1e-5 * np.broadcast_to(norm[:, None], t.shape)[bad] / np.broadcast_to(s_g[:, None], t.shape)[bad]
+        assert np.all(dist <= tol), "a code differs away from a rounding boundary"
+    stats["code_flips"] = int(bad.sum())
+    return stats
+
+
+def check_layer_output_w4a8(y_bits, xh_bits, codes, scales, layer_orc, out_orc, bias_bits, slack=3e-4):
+    K_l = codes.shape[1]
+    P = orc.int_gemm(codes, layer_orc["wcodes"], K_l)
+    y_ref, _ = orc.combine(P, scales.reshape(-1, 1), layer_orc["wscales"], xh_bits, layer_orc["Wh"], bias_bits)
+    stats = check_output(y_bits, y_ref, slack=slack)
+    clean = (np.all(codes == out_orc["codes"], axis=1) & (scales == out_orc["scales"]) & np.all(xh_bits == out_orc["xh"], axis=1))
+    stats["clean_rows_frac"] = float(np.mean(clean))
+    e2e = check_output(y_bits, out_orc["y64"], rows=clean, slack=slack)
+    stats["e2e_clean_max_err_over_rms"] = e2e.get("max_err_over_rms")
+    return stats
