@@ -121,7 +121,9 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
         Q = np.eye(K) - 2.0 * np.outer(v, v)
         W = (0.02 * g.standard_normal((K, cols))).astype(np.float32)
         x = synth.make_tokens(spec, rows, batch_seed=5)
-        if fmt == "nvfp4":
+        if fmt == "w4a8":
+            lo = orc.prepare_layer_w4a8(W, Q, RANK)
+        elif fmt == "nvfp4":
             lo = orc.nvfp4_prepare_layer(W, Q, RANK)
             lo["ex"] = orc.nvfp4_global_exponent(float(np.abs(orc.rotate(x, lo["Qb"])[:, RANK:]).max()))
         else:
@@ -135,6 +137,8 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
                 orc.nvfp4_linear_deployed(x, lo, lo["ex"], bias=None, want_t=False)
             elif fmt == "int4_asym":
                 orc.linear_deployed_asym(x, lo, bias=None, want_t=False)
+            elif fmt == "w4a8":
+                orc.linear_deployed_w4a8(x, lo, bias=None, want_t=False)
             else:
                 orc.linear_deployed(x, lo, bias=None, want_t=False)
         times.append(time.perf_counter() - t0)
@@ -159,7 +163,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64 (oracle; nvfp4 codes)" if args.fmt == "nvfp4" else "f64 + int32 (oracle; int4 codes)",
-        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else "_asym" if args.fmt == "int4_asym" else ""),
+        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else ""),
                                         "format": args.fmt,
                                         "sample": res["sample"]},
         "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
@@ -214,6 +218,8 @@ def run_ours(args):
             del xrot
             layer = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, int(np.ceil(np.log2(amax / 1536.0))),
                                                   bias=bf(bias))
+        elif args.fmt == "w4a8":
+            layer = dq.dirotq_prepare_layer_w4a8(torch.from_numpy(W).to(dev), Q, RANK, bias=bf(bias))
         elif args.fmt == "int4_asym":
             layer = dq.dirotq_prepare_layer_asym(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         else:
@@ -344,12 +350,12 @@ def run_ours(args):
     else:
         ach = sum(gemm_ops.values()) / (gemm_total * 1e-3) / 1e12
         ach_alu = elem_steps / (gemm_total * 1e-3)
-        gname = "nvfp4_gemm_kernel" if nv else "w4a4_gemm_kernel"
+        gname = "nvfp4_gemm_kernel" if nv else "w4a8_gemm_kernel" if args.fmt == "w4a8" else "w4a4_gemm_kernel"
         roofline = {"kernel": gname, "bound": "tensor", "achieved": ach, "peak": int8_peak, "unit": "TOP/s",
-                    "frac": ach / int8_peak, "traffic": NCU_TRAFFIC_QKV[gname],
+                    "frac": ach / int8_peak, "traffic": NCU_TRAFFIC_QKV.get(gname),
                     "traffic_note": "ncu dram read+write of one qkv-shaped launch (algorithmic bytes of that launch: 117.5e6)",
                     "peak_source": f"{'4' if nv else '2'} x {peaks['source']} bf16 sustained (nominal {'fp4' if nv else '8-bit'}:bf16 ratio)"}
-        if not nv:
+        if args.fmt in ("int4", "int4_asym"):
             roofline["alu"] = {"bound": "alu", "achieved": ach_alu / 1e9, "peak": alu_peak / 1e9, "unit": "G element-steps/s",
                                "frac": ach_alu / alu_peak,
                                "note": "per-group rescale: 2 fp32 fused multiply-adds per output element and K-group; "
@@ -374,16 +380,17 @@ def run_ours(args):
         "metric": "dirotq_w4a4_linear_effective_tops", "value": value, "unit": "TOPS", "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
-        "dtype": "nvfp4 (e2m1 x e2m1, e4m3 block scales) + bf16" if nv else "int4xint4 (exact group sums on the e4m3 tensor path) + bf16",
+        "dtype": ("nvfp4 (e2m1 x e2m1, e4m3 block scales) + bf16" if nv else "int8xint4->int32 + bf16" if args.fmt == "w4a8"
+                  else "int4xint4 (exact group sums on the e4m3 tensor path) + bf16"),
         "data": "synthetic",
-        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else "_asym" if args.fmt == "int4_asym" else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
-                   "group": 16 if nv else GROUP, "format": args.fmt,
+        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
+                   "group": 16 if nv else ("per-token / per-channel" if args.fmt == "w4a8" else GROUP), "format": args.fmt,
                    "l2": "inputs_exceed_l2 (each step streams > 500 MB of rotations, codes and outputs)",
                    "parallelism": f"token rows x{world}, no collective"},
         "clocks": clocks,
         "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-        "gpu_launches": 2 * len(layers) * args.steps,
+        "gpu_launches": (3 if args.fmt == "w4a8" else 2) * len(layers) * args.steps,
         "roofline": roofline,
         "kernels": kernels,
         "frac_int8_peak_effective": value / world / int8_peak,
@@ -401,9 +408,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shapes", default="", help="comma-separated subset of qkv,out,mlp_up,mlp_down (profiling runs)")
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym"],
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8"],
                     help="int4: the headline format (groups of 64, bf16 scales, symmetric); nvfp4: E2M1 blocks of 16 with E4M3 "
-                         "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group)")
+                         "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group); w4a8: per-token int8 "
+                         "activations, per-channel int4 weights")
     ap.add_argument("--lite", action="store_true", help="skip the cuBLAS, end-to-end and CPU-baseline legs (profiling runs)")
     args = ap.parse_args()
     if args.shapes:

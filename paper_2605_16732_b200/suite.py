@@ -50,7 +50,7 @@ FMT = "int4"  # set from --fmt: "int4" (groups of G, bf16 scales) or "nvfp4" (bl
 class Case:
     def __init__(self, M, K, N, r, G, model):
         self.M, self.K, self.N, self.r, self.G = M, K, N, r, G
-        spec = synth.LayerSpec(K=K, N=N, r=r, G=G if FMT != "nvfp4" else 64, model=model, seed=7)
+        spec = synth.LayerSpec(K=K, N=N, r=r, G=G if FMT in ("int4", "int4_asym") else 64, model=model, seed=7)
         W, bias = synth.make_weights(spec)
         self.x = _bf(synth.make_tokens(spec, M, batch_seed=11))
         Wd, Q = torch.from_numpy(W).cuda(), _householder(K, K + r)
@@ -64,6 +64,8 @@ class Case:
             probe.close()
             ex = int(np.ceil(np.log2(amax / 1536.0)))
             self.layer = dq.dirotq_prepare_layer_nvfp4(Wd, Q, r, ex, bias=_bf(bias))
+        elif FMT == "w4a8":
+            self.layer = dq.dirotq_prepare_layer_w4a8(Wd, Q, r, bias=_bf(bias))
         elif FMT == "int4_asym":
             self.layer = dq.dirotq_prepare_layer_asym(Wd, Q, r, G, bias=_bf(bias))
         else:
@@ -106,11 +108,13 @@ class Case:
         rot, gem, cb = self.time_kernels(iters)
         M, K, N, r, G = self.M, self.K, self.N, self.r, self.G
         K_l = K - r
-        n_g = -(-K_l // G)
+        n_g = -(-K_l // G) if G else 1
         tot = rot + gem
         p_i8 = (4.0 if FMT == "nvfp4" else 2.0) * p_bf16  # nominal ratio of the 4-bit / 8-bit tensor peak to bf16
         t_roof = (2.0 * M * K_l * N / p_i8 + (2.0 * M * K * K + 2.0 * M * r * N) / p_bf16) / 1e12 * 1e3
-        if FMT == "nvfp4":
+        if FMT == "w4a8":
+            bytes_alg = 2 * M * K + 2 * K * K + K_l * N / 2 + 4 * N + 2 * 64 * N + 2 * (M * K_l * 5 + 8 * M + 2 * M * 64) + 2 * M * N
+        elif FMT == "nvfp4":
             bytes_alg = 2 * M * K + 2 * K * K + K_l * N / 2 + K_l / 16 * N + 2 * 64 * N + 2 * (M * K_l / 2 + M * K_l / 16 + 2 * M * 64) + 2 * M * N
         else:
             bytes_alg = 2 * M * K + 2 * K * K + n_g * G * N / 2 + 4 * n_g * N + 2 * 64 * N + 2 * (M * n_g * G + 4 * M * n_g + 2 * M * 64) + 2 * M * N
@@ -130,7 +134,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,4,5")
     ap.add_argument("--iters", type=int, default=20)
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym"])
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8"])
     ap.add_argument("--ranks", default="16,32,64,128", help="ranks swept by config 4")
     args = ap.parse_args()
     global FMT
@@ -177,7 +181,7 @@ def main():
     if "4" in todo:
         for K, N in [(3072, 9216), (12288, 3072)]:
             for r in [int(v) for v in args.ranks.split(",")]:
-                for G in ((64, 128) if FMT != "nvfp4" else (16,)):
+                for G in ((64, 128) if FMT in ("int4", "int4_asym") else (16,) if FMT == "nvfp4" else (0,)):
                     c = Case(18432, K, N, r, G, synth.FLUX)
                     c.report("4: FLUX batch 4 (M=18432) rank/group sweep", max(5, args.iters // 2), p_bf16, hbm)
                     c.close()

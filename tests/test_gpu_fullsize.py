@@ -239,3 +239,58 @@ def test_asym_flux_linears(K, N):
 
 def test_asym_batch4_rank64_group128():
     print(_run_asym(18432, 3072, 9216, 64, 128, synth.FLUX))
+
+
+# ------------------------------------------------------------------ W4A8 at the benchmark's sizes
+
+def _run_w4a8(M, K, N, r, model, n_rows=24, n_cols=96, seed=0):
+    from parity_utils import check_activation_side_w4a8, check_layer_output_w4a8
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=64, model=model, seed=seed)
+    Q = _rotation(spec)
+    W, bias = synth.make_weights(spec)
+    x_bits = synth.make_tokens(spec, M, batch_seed=3)
+    g = np.random.default_rng(K * 7 + N + 3)
+    rows = np.sort(g.choice(M, size=min(n_rows, M), replace=False))
+    rows[-1] = M - 1
+    cols = np.sort(g.choice(N, size=n_cols, replace=False))
+    cols[-1] = N - 1
+    lo = orc.prepare_layer_w4a8(W[:, cols], Q, r, want_t=True)   # one scale per column: columns are independent
+    bias_s = bias[cols]
+    oo = orc.linear_deployed_w4a8(x_bits[rows], lo, bias=bias_s)
+
+    Qd = torch.from_numpy(Q).cuda()
+    layer = dq.dirotq_prepare_layer_w4a8(torch.from_numpy(W).cuda(), Qd, r, bias=bits_to_bf16_tensor(bias))
+    del Qd
+    wcodes, wscales, wh, qb = dq.dirotq_layer_export(layer)
+    assert np.array_equal(bf16_tensor_to_bits(qb), lo["Qb"]), "bf16 rotation differs"
+    del qb
+    cols_t = torch.from_numpy(cols).cuda()
+    assert np.array_equal(bf16_tensor_to_bits(wscales[:, cols_t]), lo["wscales"])
+    assert np.array_equal(bf16_tensor_to_bits(wh[:, cols_t]), lo["Wh"])
+    wc = wcodes[:, cols_t].cpu().numpy()
+    bad = wc != lo["wcodes"]
+    assert bad.sum() <= 2 and np.all(np.abs(np.abs(lo["wt"][bad] - np.floor(lo["wt"][bad])) - 0.5) < 1e-9)
+    del wcodes, wscales, wh
+
+    x = bits_to_bf16_tensor(x_bits)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = dq.alloc_workspace(layer, M)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, scales = dq.dirotq_workspace_export_w4a8(layer, M, ws)
+    rows_t = torch.from_numpy(rows).cuda()
+    xh_b = bf16_tensor_to_bits(xh[rows_t])
+    codes_n = codes[rows_t].cpu().numpy()
+    scales_b = bf16_tensor_to_bits(scales[rows_t])
+    stats = check_activation_side_w4a8(None, xh_b, codes_n, scales_b, oo, r)
+    lo_lib = dict(lo)
+    lo_lib["wcodes"] = wc
+    y_s = bf16_tensor_to_bits(y[rows_t][:, cols_t])
+    stats.update(check_layer_output_w4a8(y_s, xh_b, codes_n, scales_b, lo_lib, oo, bias_s))
+    layer.close()
+    return stats
+
+
+@pytest.mark.parametrize("K,N", [(3072, 9216), (12288, 3072)])
+def test_w4a8_flux_linears(K, N):
+    print(_run_w4a8(4608, K, N, 32, synth.FLUX))
