@@ -6,8 +6,8 @@
 //
 // With one scale per row and per column there is no rescale inside K: the whole contraction runs on
 // tcgen05.mma kind::i8 into one int32 accumulator tile and the CUDA cores touch every output once.
-// The weight codes stay packed (two per byte, nibble = q + 8) in HBM and in the TMA staging buffer;
-// four unpack warps turn every nibble into the byte 16 q (shift the nibble into the high half, flip
+// The weight codes stay packed (two per byte, nibble = q + 8) in HBM; TMA lands them in the upper half of
+// the operand buffer and four unpack warps expand them in place, turning every nibble into the byte 16 q (shift the nibble into the high half, flip
 // bit 7: 16 (q + 8) - 128), so the accumulator holds 16 P and the epilogue shifts it back.
 //
 // Roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 unpack,
@@ -25,16 +25,19 @@ namespace {
 constexpr int BM = 128;
 constexpr int BN = kGemmBN;  // 256
 constexpr int BKC = 128;     // one-byte codes per k-block (128-byte rows)
-constexpr int STAGES = 3;
+constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BKC;       // 16 KB activation codes / bf16 x~_h chunk
 constexpr int BU_BYTES = BN * BKC;      // 32 KB unpacked weight codes / bf16 W~_h chunk
-constexpr int BP_BYTES = BN * BKC / 2;  // 16 KB packed weight codes (TMA staging)
-constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;
+constexpr int BP_BYTES = BN * BKC / 2;  // 16 KB packed weight codes: TMA puts them into the UPPER HALF of the 32 KB
+constexpr int BP_OFFSET = A_BYTES + BU_BYTES - BP_BYTES;  // operand buffer and the unpack expands them in place
+constexpr int STAGE_BYTES = A_BYTES + BU_BYTES;           // 48 KB: four stages fit
 constexpr int NUM_THREADS = 320;
 constexpr int NUM_UNPACK_WARPS = 4;
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+constexpr int SCALE_OFFSET = BAR_OFFSET + 256;      // two buffers of {weight scales, bias} for a tile's 256 columns
+constexpr int SCALE_BYTES = 2 * 2 * BN * 4;
+constexpr int SMEM_BYTES = SCALE_OFFSET + SCALE_BYTES + 1024;
 
 struct A8KernelParams {
     int M, N, num_kb, lr_chunks;
@@ -122,7 +125,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     if (i < p.num_kb) {
                         mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
                         tma_load_2d(st, &tmap_codes, full_bar(s), i * BKC, m0);
-                        tma_load_2d(st + A_BYTES + BU_BYTES, &tmap_wpacked, full_bar(s), i * (BKC / 2), n0);
+                        tma_load_2d(st + BP_OFFSET, &tmap_wpacked, full_bar(s), i * (BKC / 2), n0);
                     } else {
                         mbar_arrive_expect_tx(full_bar(s), A_BYTES + BU_BYTES);
                         tma_load_2d(st, &tmap_xh, full_bar(s), (i - p.num_kb) * 64, m0);
@@ -178,20 +181,37 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int i = 0; i < items; ++i, ++it) {
                 const int s = it % STAGES;
-                ok = mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
-                ok = __any_sync(0xffffffffu, ok);
+                // The four unpack warps meet at a hardware barrier below, which has no time limit: they must all go on or
+                // all give up.  Every thread reaches this reducing barrier once per item whatever its wait returned.
+                const bool mine = mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+                uint32_t any_failed;
+                asm volatile(
+                    "{\n\t"
+                    ".reg .pred pin, pout;\n\t"
+                    "setp.eq.u32 pin, %1, 0;\n\t"
+                    "bar.red.or.pred pout, 1, %2, pin;\n\t"
+                    "selp.u32 %0, 1, 0, pout;\n\t"
+                    "}\n"
+                    : "=r"(any_failed)
+                    : "r"(static_cast<uint32_t>(mine)), "n"(NUM_UNPACK_WARPS * 32)
+                    : "memory");
+                ok = any_failed == 0;
                 if (!ok) break;
                 if (i < p.num_kb) {
                     // 16-byte piece idx = u + 128 j of the packed tile: row = idx / 4 = u / 4 + 32 j, piece c = u % 4; the
                     // swizzle phase row % 8 and the piece do not depend on j
                     uint8_t* st = smem_gen + s * STAGE_BYTES;
-                    const uint4* src = reinterpret_cast<const uint4*>(st + A_BYTES + BU_BYTES) + u;
+                    const uint4* src = reinterpret_cast<const uint4*>(st + BP_OFFSET) + u;
                     const int c = u & 3, sw = (u >> 2) & 7;
                     uint8_t* d0 = st + A_BYTES + (u >> 2) * 128 + (((2 * c) ^ sw) << 4);
                     uint8_t* d1 = st + A_BYTES + (u >> 2) * 128 + (((2 * c + 1) ^ sw) << 4);
-                    uint4 pk[8];  // loads before stores: the compiler cannot prove the two buffers disjoint
+                    // The packed codes sit in the upper half of the buffer they are expanded into: every unpack thread
+                    // takes its eight pieces into registers, the four warps meet at a named barrier, and only then is
+                    // anything stored.
+                    uint4 pk[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) pk[j] = src[128 * j];
+                    asm volatile("bar.sync 2, %0;" ::"n"(NUM_UNPACK_WARPS * 32) : "memory");  // reached by all four warps (see above)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         // nibble q + 8 -> byte 16 q: into the high half, then flip bit 7 (16 (q + 8) - 128)
@@ -217,8 +237,35 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
-            ok = mbar_wait(tfull_bar, tcount & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
-            ok = __any_sync(0xffffffffu, ok);
+            // This tile's column scales and bias go to shared memory while the MMAs are still running (two buffers: a warp
+            // can be one tile ahead of the others).  The reducing barrier orders these stores before the reads below and
+            // makes the four warps agree on whether to go on: a plain barrier behind a bounded wait could strand a warp.
+            float* s_sw = reinterpret_cast<float*>(smem_gen + SCALE_OFFSET) + (tcount & 1) * 2 * BN;
+            float* s_b = s_sw + BN;
+            {
+                const int e = threadIdx.x - (2 + NUM_UNPACK_WARPS) * 32;  // 0..127
+                const int col = n0 + 2 * e;
+                float2 w2 = make_float2(0.f, 0.f), b2 = make_float2(0.f, 0.f);
+                if (col < p.N) {
+                    w2 = __ldg(reinterpret_cast<const float2*>(p.wscale + col));
+                    b2 = __ldg(reinterpret_cast<const float2*>(p.bias + col));
+                }
+                *reinterpret_cast<float2*>(s_sw + 2 * e) = w2;
+                *reinterpret_cast<float2*>(s_b + 2 * e) = b2;
+            }
+            const bool mine = mbar_wait(tfull_bar, tcount & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+            uint32_t any_failed;
+            asm volatile(
+                "{\n\t"
+                ".reg .pred pin, pout;\n\t"
+                "setp.eq.u32 pin, %1, 0;\n\t"
+                "bar.red.or.pred pout, 3, %2, pin;\n\t"
+                "selp.u32 %0, 1, 0, pout;\n\t"
+                "}\n"
+                : "=r"(any_failed)
+                : "r"(static_cast<uint32_t>(mine)), "n"(NUM_EPI_WARPS * 32)
+                : "memory");
+            ok = any_failed == 0;
             if (!ok) break;
             tc_fence_after_sync();
             const int row = m0 + q * 32 + lane;
@@ -255,8 +302,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                 float o[8];
 #pragma unroll
                                 for (int t = 0; t < 8; t += 4) {
-                                    const float4 sw = __ldg(reinterpret_cast<const float4*>(p.wscale + col + j + t));
-                                    const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col + j + t));
+                                    const float4 sw = *reinterpret_cast<const float4*>(s_sw + c * 32 + j + t);
+                                    const float4 b = *reinterpret_cast<const float4*>(s_b + c * 32 + j + t);
                                     const float sws[4] = {sw.x, sw.y, sw.z, sw.w}, bs[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
                                     for (int e = 0; e < 4; ++e) {
