@@ -36,7 +36,8 @@ constexpr int SF_BYTES = 4 * 512;      // four atoms per operand and k-block
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 2 * SF_BYTES;  // 36 KB
 constexpr int NUM_THREADS = 192;
 constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+constexpr int BIAS_OFFSET = BAR_OFFSET + 256;  // two buffers of a tile's 128 bias values
+constexpr int SMEM_BYTES = BIAS_OFFSET + 2 * BN * 4 + 1024;
 constexpr int TMEM_SF_BASE = 2 * BN;   // columns 256.. hold the scale factors: 32 per stage
 
 struct NvKernelParams {
@@ -234,8 +235,27 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
             const uint32_t acc = tcount & 1;
-            ok = mbar_wait(tfull_bar(acc), (tcount >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
-            ok = __any_sync(0xffffffffu, ok);
+            // The tile's bias goes to shared memory while its MMAs are still running (two buffers: a warp can be one tile
+            // ahead of the others).  The reducing barrier orders the stores before the reads below and makes the four
+            // warps agree on whether to go on: a plain barrier behind a bounded wait could strand a warp.
+            float* s_b = reinterpret_cast<float*>(smem_gen + BIAS_OFFSET) + (tcount & 1) * BN;
+            {
+                const int e = threadIdx.x - 64;  // 0..127
+                s_b[e] = n0 + e < p.N ? __ldg(p.bias + n0 + e) : 0.f;
+            }
+            const bool mine = mbar_wait(tfull_bar(acc), (tcount >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+            uint32_t any_failed;
+            asm volatile(
+                "{\n\t"
+                ".reg .pred pin, pout;\n\t"
+                "setp.eq.u32 pin, %1, 0;\n\t"
+                "bar.red.or.pred pout, 1, 128, pin;\n\t"
+                "selp.u32 %0, 1, 0, pout;\n\t"
+                "}\n"
+                : "=r"(any_failed)
+                : "r"(static_cast<uint32_t>(mine))
+                : "memory");
+            ok = any_failed == 0;
             if (!ok) break;
             tc_fence_after_sync();
             const int row = m0 + q * 32 + lane;
@@ -256,8 +276,8 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
                         if (col + j < p.N) {
-                            const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + col + j));
-                            const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + col + j + 4));
+                            const float4 b0 = *reinterpret_cast<const float4*>(s_b + c * 32 + j);
+                            const float4 b1 = *reinterpret_cast<const float4*>(s_b + c * 32 + j + 4);
                             uint4 o;
                             o.x = pack_bf16x2(fmaf(__uint_as_float(raw[j + 0]), out_scale, b0.x), fmaf(__uint_as_float(raw[j + 1]), out_scale, b0.y));
                             o.y = pack_bf16x2(fmaf(__uint_as_float(raw[j + 2]), out_scale, b0.z), fmaf(__uint_as_float(raw[j + 3]), out_scale, b0.w));
