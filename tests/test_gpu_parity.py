@@ -236,3 +236,34 @@ def test_shared_rotation_across_linears_with_the_same_input():
     assert dq.dirotq_workspace_status(ws) == 0
     for layer in layers:
         layer.close()
+
+
+def test_host_entry_point_on_concurrent_streams():
+    """Two independent layers through dirotq_linear_host on two streams at once (the library's copy streams and events
+    are shared by all calls on a device): both results equal the device entry point's."""
+    M = 3000
+    cases = []
+    for seed, (K, N) in enumerate([(512, 384), (384, 640)]):
+        spec = synth.LayerSpec(K=K, N=N, r=32, G=64, model=synth.PIXART, seed=20 + seed, calib_tokens=1024)
+        inp = synth.make_layer_inputs(spec, M)
+        layer = dq.dirotq_prepare_layer(torch.from_numpy(inp["W"]).cuda(), torch.from_numpy(inp["Q"]).cuda(), spec.r, spec.G,
+                                        bias=bits_to_bf16_tensor(inp["bias"]))
+        x = bits_to_bf16_tensor(inp["x"])
+        ws = dq.alloc_workspace(layer, M)
+        y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+        dq.dirotq_linear(x, layer, y, ws)
+        cases.append({"layer": layer, "ws": ws, "y": y, "xh": x.cpu().pin_memory(),
+                      "yh": torch.zeros((M, N), dtype=torch.bfloat16).pin_memory(), "x_dev": torch.empty_like(x),
+                      "y_dev": torch.empty_like(y), "stream": torch.cuda.Stream()})
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for c in cases:
+            c["yh"].zero_()
+        for c in cases:
+            dq.dirotq_linear_host(c["xh"], c["layer"], c["yh"], c["x_dev"], c["y_dev"], c["ws"], stream=c["stream"])
+        for c in cases:
+            c["stream"].synchronize()
+            assert torch.equal(c["yh"].view(torch.int16), c["y"].cpu().view(torch.int16))
+    for c in cases:
+        assert dq.dirotq_workspace_status(c["ws"]) == 0
+        c["layer"].close()
