@@ -178,6 +178,9 @@ static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w
     st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
                         (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                            (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
@@ -262,6 +265,9 @@ dirotq_status_t dirotq_prepare_layer_w4a8(const void* W, int w_dtype, int w_layo
     L->blob = static_cast<char*>(blob);
     st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
                         (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                            (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -607,6 +613,9 @@ dirotq_status_t dirotq_prepare_layer_nvfp4(const void* W, int w_dtype, int w_lay
     L->act_scale_log2 = act_scale_log2;
     st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
                         (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                            (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked, (uint64_t)g.K4 / 2,
                             (uint64_t)N, (uint64_t)g.K4 / 2, 128, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);

@@ -161,6 +161,7 @@ struct dirotq_layer {
     dirotq::BlobLayout lay;
     char* blob;  // device
     CUtensorMap tmap_qt;       // bf16 [K][K], box 64 x 256, 128B swizzle
+    CUtensorMap tmap_qt128;    // the same tensor with box 64 x 128 (narrow tiles of the rotation kernel)
     CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2] (nibble = q + 8), box 64 x kGemmBN, no swizzle
     CUtensorMap tmap_wscale;   // f32 [n_g][N], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle

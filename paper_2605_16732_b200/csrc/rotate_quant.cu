@@ -22,11 +22,11 @@ namespace dirotq {
 namespace {
 
 constexpr int BM = 128;       // tokens per tile
-constexpr int BN = 256;       // rotated columns per tile
+constexpr int BN_MAX = 256;   // rotated columns per tile: 256, or 128 when there are few tiles (template parameter BN)
 constexpr int BK = 64;        // bf16 elements per k-block (128-byte rows)
 constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;  // 16 KB
-constexpr int B_BYTES = BN * BK * 2;  // 32 KB
+constexpr int B_BYTES = BN_MAX * BK * 2;  // 32 KB (a 128-column tile uses half of it)
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_THREADS = 192;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -143,7 +143,7 @@ __device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float ex_inv, 
     return sb;
 }
 
-template <int G, int FMT>
+template <int G, int FMT, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
                     const RotKernelParams p) {
@@ -202,7 +202,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+                    mbar_arrive_expect_tx(full_bar(s), A_BYTES + BN * BK * 2);
                     const uint32_t sa = smem_base + s * STAGE_BYTES;
                     tma_load_2d(sa, &tmap_x, full_bar(s), kb * BK, m0);
                     tma_load_2d(sa + A_BYTES, &tmap_qt, full_bar(s), kb * BK, n0);
@@ -452,20 +452,32 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
-    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.K + BN - 1) / BN);
-    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
     p.xtilde = a.xtilde; p.rowmax = a.rowmax;
+    // 256-column tiles, or 128-column ones when the wide tiles would not give every SM about two of them (few, large
+    // tiles leave a nearly empty last wave: 160 tiles on 148 SMs take as long as 296)
+    const int sms = sm_count(L->device);
+    const int m_blocks = (a.M + BM - 1) / BM;
+    const bool narrow = m_blocks * ((g.K + 255) / 256) < 2 * sms;
+    const int bn = narrow ? 128 : 256;
+    const int num_tiles = m_blocks * ((g.K + bn - 1) / bn);
+    const int grid = num_tiles < sms ? num_tiles : sms;
     const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
-    auto kern = vi == 2 ? rotate_quant_kernel<64, 1>
-              : vi == 5 ? rotate_quant_kernel<64, 3>
-              : vi == 3 ? rotate_quant_kernel<64, 2>
-              : vi == 4 ? rotate_quant_kernel<128, 2>
-              : vi == 0 ? rotate_quant_kernel<64, 0> : rotate_quant_kernel<128, 0>;
-    static bool attr_set[6] = {false, false, false, false, false, false};
-    if (!attr_set[vi]) {
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const RotKernelParams);
+    static const KernelFn table[2][6] = {
+        {rotate_quant_kernel<64, 0, 256>, rotate_quant_kernel<128, 0, 256>, rotate_quant_kernel<64, 1, 256>,
+         rotate_quant_kernel<64, 2, 256>, rotate_quant_kernel<128, 2, 256>, rotate_quant_kernel<64, 3, 256>},
+        {rotate_quant_kernel<64, 0, 128>, rotate_quant_kernel<128, 0, 128>, rotate_quant_kernel<64, 1, 128>,
+         rotate_quant_kernel<64, 2, 128>, rotate_quant_kernel<128, 2, 128>, rotate_quant_kernel<64, 3, 128>}};
+    const KernelFn kern = table[narrow ? 1 : 0][vi];
+    static bool attr_set[2][6] = {};
+    if (!attr_set[narrow ? 1 : 0][vi]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
-        attr_set[vi] = true;
+        attr_set[narrow ? 1 : 0][vi] = true;
+    }
+    if (narrow) {
+        kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_x, L->tmap_qt128, p);
+        return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
     }
     kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_x, L->tmap_qt, p);
     return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
