@@ -175,7 +175,7 @@ DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8
                                     void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
 
 /* ---- asymmetric activation codes (paper Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the 4-bit INT setting
- * "using asymmetric activation quantization") ---- */
+ * quantizes the activations asymmetrically) ---- */
 
 /* Same layer, but every group of G low-precision coefficients of a token is quantized to unsigned
  * codes u in 0..15 with a bf16 scale s = (max - min) / 15 and a bf16 zero-point z = min, x^ = s u + z
@@ -199,8 +199,8 @@ DIROTQ_API dirotq_status_t dirotq_workspace_export_asym(const dirotq_layer_t* la
 DIROTQ_API dirotq_status_t dirotq_layer_export_zero_term(const dirotq_layer_t* layer, float* zero_term,
                                                          dirotq_stream_t stream);
 
-/* ---- W4A8 (paper Sec. 5.1 and the "INT W4A8" rows of Table 1: "per-token dynamic activation
- * quantization and per-channel static weight quantization for 8-bit settings") ---- */
+/* ---- W4A8 (paper Sec. 5.1 and the "INT W4A8" rows of Table 1: for 8-bit settings the activations get
+ * one dynamic scale per token and the weights one static scale per output channel) ---- */
 
 /* Same layer with 8-bit activations and per-channel 4-bit weights, both symmetric (Eq. 1, z = 0): every
  * token's K - r low-precision coefficients share one bf16 scale s_x[m] = max|x~| / 127 and are rounded to
@@ -223,7 +223,7 @@ DIROTQ_API dirotq_status_t dirotq_workspace_export_w4a8(const dirotq_layer_t* la
                                                         void* xh_bf16, int8_t* codes, void* scales_bf16,
                                                         dirotq_stream_t stream);
 
-/* ---- NVFP4 variant (paper Sec. 5.1: "For 4-bit FP, we use NVFP4 ... group size 16 with FP8 scaling") ---- */
+/* ---- NVFP4 variant (paper Sec. 5.1: the 4-bit float setting is NVFP4, blocks of 16 with an FP8 scale) ---- */
 
 /* Same layer with the 4-bit float format instead of INT4: elements are E2M1 (1 sign, 2 exponent,
  * 1 mantissa bit: q_max = 6, Sec. 3), every block of 16 consecutive low-precision coefficients

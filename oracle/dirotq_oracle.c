@@ -318,8 +318,8 @@ void dq_combine_asym(const int32_t* P, const uint16_t* sx, const uint16_t* zx, c
 
 /* =====================================================================================
  * W4A8 (paper Sec. 5.1, "INT W4A8" rows of Table 1): 8-bit activations with one dynamic scale per
- * token, 4-bit weights with one static scale per output channel ("per-token dynamic activation
- * quantization and per-channel static weight quantization for 8-bit settings").
+ * token, 4-bit weights with one static scale per output channel (Sec. 5.1 gives these two granularities
+ * for its 8-bit settings).
  * Readings: symmetric on both sides (Eq. 1 with z = 0, q_max = 2^7 - 1 = 127 for the activations);
  * the token's scale covers its K - r low-precision coefficients and is kept as bf16, the rounded
  * value dividing and dequantizing; the weight side is Eq. 1 with one group spanning the whole
@@ -383,8 +383,8 @@ int dq_num_threads(void) {
 }
 
 /* =====================================================================================
- * NVFP4 variant (paper Sec. 5.1: "For 4-bit FP, we use NVFP4, which supports group size 16
- * with FP8 scaling"; Sec. 3: a 4-bit float with 1 mantissa and 2 exponent bits has q_max = 6).
+ * NVFP4 variant (paper Sec. 5.1: the 4-bit float setting is NVFP4, blocks of 16 with an FP8 scale each;
+ * Sec. 3: a 4-bit float with 1 mantissa and 2 exponent bits has q_max = 6).
  *
  *   element format E2M1: sign, 2 exponent bits, 1 mantissa bit; magnitudes {0, .5, 1, 1.5, 2, 3, 4, 6}
  *   block of 16 consecutive low-precision coefficients shares one FP8 E4M3 scale (used unsigned)
