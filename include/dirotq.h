@@ -174,6 +174,21 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,
                                     void* wh_bf16, void* q_bf16, dirotq_stream_t stream);
 
+/* ---- residual weights rounded by the caller (paper Sec. 4.1 and App. F.1: the residual weight is rounded with
+ * GPTQ, which minimises the activation-weighted output error instead of rounding each value to nearest) ----
+ *
+ * As dirotq_prepare_layer (asym == 0) or dirotq_prepare_layer_asym (asym != 0), except that the INT4 codes and
+ * scales of the folded rows r..K-1 are the caller's: wcodes int8 [K-r,N] (row j = rotated column r+j; values
+ * outside -7..7 are clamped) and wscales bf16 [n_g,N], both DEVICE, row-major, read during the call only.
+ * W and Q are still needed: the rows below r of Q^T W are kept in bf16 and Q is rounded for the online GEMM.
+ * Any offline rounding (GPTQ on a calibration Hessian, a search over clipping ratios, ...) can be deployed
+ * this way; the online path is the same. */
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_codes(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                                      const void* bias, const int8_t* wcodes, const void* wscales_bf16,
+                                                      int asym, int K, int N, int r, int group, void* blob,
+                                                      size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                                      dirotq_stream_t stream, dirotq_layer_t** layer_out);
+
 /* ---- asymmetric activation codes (paper Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the 4-bit INT setting
  * quantizes the activations asymmetrically) ---- */
 

@@ -214,6 +214,79 @@ def linear_deployed(x_bits, layer, bias=None, want_t: bool = True):
 
 
 # ---------------------------------------------------------------------------------------------
+# GPTQ rounding of the residual weight (Sec. 4.1: the rounding minimises ||X W - X W^||_F^2 rather than the
+# layer-wise surrogate; App. F.1: damping 0.01, block size 128).  The steps are those of the published GPTQ
+# algorithm, on the residual weight W~_l whose rows are the rotated low columns: the Hessian is
+# H = X~_l^T X~_l of the calibration tokens, rows are rounded in order, and the rounding error of each row is
+# spread over the rows not yet rounded, weighted by the upper Cholesky factor of H^-1.
+
+def gptq_hessian(xt_low) -> np.ndarray:
+    """H = X~_l^T X~_l  [K_l, K_l] in fp64 for calibration tokens X~_l [T, K_l] (already rotated and split)."""
+    xt_low = _c(xt_low, np.float64)
+    return matmul(np.ascontiguousarray(xt_low.T), xt_low)
+
+
+def gptq_quantize(Wt_low, H, G: int, damp: float = 0.01, block: int = 128, lazy: bool = True):
+    """INT4 codes [K_l, N] and bf16 scale bits [n_g, N] for the residual weight Wt_low [K_l, N].
+
+    Group scales are those of Eq. 1 (bf16(absmax/7) per group of G rows and output column), taken from the
+    rows as they stand when the group starts, i.e. after the feedback of every earlier row.  `lazy` applies
+    the feedback beyond the current block once per block (the published blocked form); lazy=False applies it
+    row by row.  Both are the same arithmetic up to rounding order.
+    """
+    W = np.array(Wt_low, dtype=np.float64, copy=True)
+    H = np.array(H, dtype=np.float64, copy=True)
+    K_l, N = W.shape
+    assert H.shape == (K_l, K_l) and block % G == 0
+    n_g = -(-K_l // G)
+    dead = np.diag(H) == 0.0                       # a column no calibration token excites
+    H[dead, dead] = 1.0
+    W[dead, :] = 0.0
+    H[np.diag_indices(K_l)] += damp * np.mean(np.diag(H))
+    Hinv = np.linalg.inv(H)
+    Hinv = 0.5 * (Hinv + Hinv.T)
+    U = np.linalg.cholesky(Hinv).T                 # upper, H^-1 = U^T U
+    codes = np.zeros((K_l, N), dtype=np.int8)
+    scales = np.zeros((n_g, N), dtype=np.uint16)
+    s = np.zeros(N, dtype=np.float64)
+    for b0 in range(0, K_l, block):
+        b1 = min(b0 + block, K_l)
+        E = np.zeros((b1 - b0, N), dtype=np.float64)
+        for j in range(b0, b1):
+            if j % G == 0:
+                g1 = min(j + G, K_l)
+                sb = bf16_round(np.max(np.abs(W[j:g1, :]), axis=0) / 7.0)
+                scales[j // G, :] = sb
+                s = bf16_to_f64(sb)
+            safe = np.where(s > 0.0, s, 1.0)
+            q = np.where(s > 0.0, np.clip(np.rint(W[j, :] / safe), -7.0, 7.0), 0.0)
+            codes[j, :] = q.astype(np.int8)
+            err = (W[j, :] - s * q) / U[j, j]
+            end = b1 if lazy else K_l
+            W[j + 1:end, :] -= np.outer(U[j, j + 1:end], err)
+            E[j - b0, :] = err
+        if lazy and b1 < K_l:
+            W[b1:, :] -= U[b0:b1, b1:].T @ E
+    return codes, scales
+
+
+def prepare_layer_gptq(W, Q, calib_bits, r: int, G: int, damp: float = 0.01, block: int = 128):
+    """Offline part with GPTQ rounding: like prepare_layer, but the residual codes and scales come from
+    gptq_quantize with the Hessian of the rotated calibration tokens (bf16 bits [T, K])."""
+    Q = _c(Q, np.float64)
+    Wt = fold(Q, np.asarray(W, dtype=np.float64))
+    out = prepare_weights(Wt, r, G, want_t=False)
+    out["Qb"] = bf16_round(Q)
+    out["r"], out["G"] = r, G
+    xt = rotate(calib_bits, out["Qb"])
+    H = gptq_hessian(xt[:, r:])
+    out["wcodes_rtn"], out["wscales_rtn"] = out["wcodes"], out["wscales"]
+    out["wcodes"], out["wscales"] = gptq_quantize(Wt[r:, :], H, G, damp=damp, block=block)
+    out["H"], out["Wt_low"] = H, Wt[r:, :]
+    return out
+
+
+# ---------------------------------------------------------------------------------------------
 # Asymmetric activation quantization (Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the paper's INT4 setting)
 
 def quantize_group_asym(v):

@@ -29,7 +29,7 @@ EXPORTED = [
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
-    "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_prepare_layer_codes", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.dirotq_workspace_export_w4a8.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_layer_bytes_asym.argtypes = [i, i, i, i, psz]
         L.dirotq_prepare_layer_asym.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
+        L.dirotq_prepare_layer_codes.argtypes = [vp, i, i, vp, i, vp, vp, vp, i, i, i, i, i, vp, sz, vp, sz, vp,
+                                                 ctypes.POINTER(vp)]
         L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
         L.dirotq_layer_export_zero_term.argtypes = [vp, vp, vp]
         for name in EXPORTED:
@@ -351,6 +353,31 @@ def dirotq_prepare_layer_asym(W: torch.Tensor, Q: torch.Tensor, r: int, group: i
     _check(st, "dirotq_prepare_layer_asym")
     torch.cuda.current_stream().synchronize()
     return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym")
+
+
+def dirotq_prepare_layer_codes(W: torch.Tensor, Q: torch.Tensor, wcodes: torch.Tensor, wscales: torch.Tensor, r: int,
+                               group: int, bias: torch.Tensor | None = None, asym: bool = False,
+                               w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """As dirotq_prepare_layer(_asym), with the residual codes int8 [K-r,N] and bf16 scales [n_g,N] given by the caller."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    n_g = -(-(K - r) // group)
+    assert wcodes.is_cuda and wcodes.is_contiguous() and wcodes.dtype == torch.int8 and tuple(wcodes.shape) == (K - r, N)
+    assert wscales.is_cuda and wscales.is_contiguous() and wscales.dtype == torch.bfloat16 and tuple(wscales.shape) == (n_g, N)
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    nbytes = dirotq_layer_bytes_asym(K, N, r, group) if asym else dirotq_layer_bytes(K, N, r, group)
+    blob = _alloc_bytes(nbytes, W.device)
+    scratch_bytes = dirotq_prepare_scratch_bytes(K, N)
+    scratch = _alloc_bytes(scratch_bytes, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_codes(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), wcodes.data_ptr(),
+                                          wscales.data_ptr(), int(asym), K, N, r, group, blob.data_ptr(), blob.numel(),
+                                          scratch.data_ptr(), scratch_bytes, _stream(stream), ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_codes")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym" if asym else "int4")
 
 
 def dirotq_workspace_export_asym(layer: Layer, M: int, workspace: torch.Tensor, stream=None):

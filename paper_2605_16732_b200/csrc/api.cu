@@ -146,7 +146,8 @@ dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_
 }
 
 static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
-                                    const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                    const void* bias, const int8_t* wcodes, const void* wscales, int K, int N, int r,
+                                    int group, void* blob, size_t blob_bytes,
                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
                                     dirotq_layer_t** layer_out) {
     if (!W || !Q || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
@@ -156,6 +157,7 @@ static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w
     dirotq_status_t st = check_shape(K, N, r, group);
     if (st != DIROTQ_OK) return st;
     if (!aligned16(W) || !aligned16(Q) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
+    if ((wcodes == nullptr) != (wscales == nullptr)) return DIROTQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
     Geometry g = make_geometry(K, N, r, group);
     if (asym) make_asym(g);
@@ -190,7 +192,7 @@ static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w
         st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
-        st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, static_cast<double*>(scratch),
+        st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, static_cast<double*>(scratch),
                             static_cast<cudaStream_t>(stream));
     if (st != DIROTQ_OK) {
         delete L;
@@ -204,8 +206,17 @@ dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, c
                                      const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
                                      void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
                                      dirotq_layer_t** layer_out) {
-    return prepare_int4(false, W, w_dtype, w_layout, Q, q_dtype, bias, K, N, r, group, blob, blob_bytes, scratch,
-                        scratch_bytes, stream, layer_out);
+    return prepare_int4(false, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob, blob_bytes,
+                        scratch, scratch_bytes, stream, layer_out);
+}
+
+dirotq_status_t dirotq_prepare_layer_codes(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                           const void* bias, const int8_t* wcodes, const void* wscales, int asym, int K,
+                                           int N, int r, int group, void* blob, size_t blob_bytes, void* scratch,
+                                           size_t scratch_bytes, dirotq_stream_t stream, dirotq_layer_t** layer_out) {
+    if (!wcodes || !wscales) return DIROTQ_ERR_INVALID_ARG;
+    return prepare_int4(asym != 0, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, K, N, r, group, blob,
+                        blob_bytes, scratch, scratch_bytes, stream, layer_out);
 }
 
 dirotq_status_t dirotq_layer_bytes_asym(int K, int N, int r, int group, size_t* bytes) {
@@ -222,8 +233,8 @@ dirotq_status_t dirotq_prepare_layer_asym(const void* W, int w_dtype, int w_layo
                                           const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
                                           void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
                                           dirotq_layer_t** layer_out) {
-    return prepare_int4(true, W, w_dtype, w_layout, Q, q_dtype, bias, K, N, r, group, blob, blob_bytes, scratch,
-                        scratch_bytes, stream, layer_out);
+    return prepare_int4(true, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob, blob_bytes,
+                        scratch, scratch_bytes, stream, layer_out);
 }
 
 dirotq_status_t dirotq_layer_bytes_w4a8(int K, int N, int r, size_t* bytes) {

@@ -235,7 +235,8 @@ dirotq_status_t launch_layer_export_nvfp4(const dirotq_layer* L, uint8_t* wcodes
 dirotq_status_t launch_workspace_export_nvfp4(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,
                                               uint8_t* codes, uint8_t* sf, cudaStream_t stream);
 dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
-                               int q_dtype, const void* bias, double* scratch, cudaStream_t stream);
+                               int q_dtype, const void* bias, const int8_t* wcodes, const void* wscales, double* scratch,
+                               cudaStream_t stream);
 dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint16_t* wscales, uint16_t* wh,
                                     uint16_t* qb, cudaStream_t stream);
 dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,

@@ -128,6 +128,41 @@ __global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, floa
     }
 }
 
+// Residual weights rounded by the caller (GPTQ or any other offline rounding): codes [K_l][N] int8 and bf16 scales
+// [n_g][N] go into the same packed layout as the library's own round-to-nearest codes.
+__global__ void pack_codes_kernel(const int8_t* codes, const uint16_t* scales, uint8_t* wpacked, float* wscale,
+                                  uint16_t* wh, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int grp = blockIdx.y;
+    if (n >= g.N) return;
+    const int j0 = grp * g.G;
+    const int len = min(g.G, g.K_l - j0);
+    const double s = bf16_to_f64(scales[static_cast<size_t>(grp) * g.N + n]);
+    wscale[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(s);
+    const int8_t* col = codes + static_cast<size_t>(j0) * g.N + n;
+    uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
+    int csum = 0;
+    for (int jb = 0; jb < g.G; jb += 8) {
+        uint32_t word = 0;
+        for (int t = 0; t < 8; ++t) {
+            const int j = jb + t;
+            const int q = j < len ? max(-7, min(7, static_cast<int>(col[static_cast<size_t>(j) * g.N]))) : 0;
+            csum += q;
+            word |= (static_cast<uint32_t>(q + 8) & 0xFu) << (8 * (t & 3) + 4 * (t >> 2));
+        }
+        *reinterpret_cast<uint32_t*>(row + packed_byte_index(j0 + jb)) = word;
+    }
+    if (g.fmt == 2) {
+        double rem = s * static_cast<double>(csum);
+        uint16_t* ext = wh + static_cast<size_t>(n) * g.r_pad + g.r_pad0;
+        for (int piece = 0; piece < 3; ++piece) {
+            const uint16_t pb = f64_to_bf16(rem);
+            ext[piece * g.n_g + grp] = pb;
+            rem -= bf16_to_f64(pb);
+        }
+    }
+}
+
 // wh[n][i] = bf16(Wt[i][n]) for i < r, zero up to r_pad.
 __global__ void high_rows_kernel(const double* Wt, uint16_t* wh, Geometry g) {
     const int n = blockIdx.x * blockDim.x + threadIdx.x;
@@ -493,7 +528,8 @@ inline bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
 }  // namespace
 
 dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
-                               int q_dtype, const void* bias, double* scratch, cudaStream_t stream) {
+                               int q_dtype, const void* bias, const int8_t* wcodes, const void* wscales, double* scratch,
+                               cudaStream_t stream) {
     const Geometry& g = L->geo;
     char* blob = L->blob;
     fold_kernel<<<dim3((g.N + 63) / 64, (g.K + 63) / 64), 256, 0, stream>>>(Q, q_dtype, W, w_dtype, w_layout, scratch,
@@ -505,9 +541,14 @@ dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype
     // the rank-r rows first (zero padded to r_pad), then the quantizer, which for fmt 2 fills its extra columns
     high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
-    quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
-        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale),
-        reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    if (wcodes)
+        pack_codes_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+            wcodes, static_cast<const uint16_t*>(wscales), reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked),
+            reinterpret_cast<float*>(blob + L->lay.off_wscale), reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    else
+        quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+            scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked),
+            reinterpret_cast<float*>(blob + L->lay.off_wscale), reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
         Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
