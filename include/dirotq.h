@@ -169,6 +169,12 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
                                       int32_t* partials, void* workspace, size_t workspace_bytes,
                                       dirotq_stream_t stream);
 
+/* Tuning knob of the INT4 second kernel (symmetric and asymmetric layers): output columns per tile.  0 (default):
+ * chosen per call from M, N and the number of SMs (128-column tiles when 256-column ones would leave the last wave
+ * of tiles nearly empty or use fewer tiles than SMs); 128 or 256: forced.  Process-wide; results do not depend on
+ * it (each output element is accumulated in the same order).  Other values: DIROTQ_ERR_INVALID_ARG. */
+DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
+
 /* Unpacks a prepared layer: wcodes int8 [K-r,N]; wscales bf16 [n_g,N]; wh bf16 [r,N];
  * q_bf16 [K,K] in the layout of the Q argument.  Any pointer may be NULL. */
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,

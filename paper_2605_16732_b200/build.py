@@ -52,7 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + f".{os.getpid()}.tmp"
-    subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-cudart", "static", "-Xlinker", "--no-undefined",
+    subprocess.check_call([_nvcc(), "-Wno-deprecated-gpu-targets", "-shared", "-o", tmp, *objs, "-cudart", "static", "-Xlinker", "--no-undefined",
                            "-lpthread", "-ldl", "-lrt"])
     os.replace(tmp, LIB)
     return LIB

@@ -192,6 +192,15 @@ static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w
         st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked128, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wscale128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
+                            (uint64_t)g.n_g, (uint64_t)N * 4, 128, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
         st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, static_cast<double*>(scratch),
                             static_cast<cudaStream_t>(stream));
     if (st != DIROTQ_OK) {
@@ -400,6 +409,8 @@ static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateAr
     ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr; ga.status = ra.status;
     return launch_w4a4_gemm(layer, ga, s);
 }
+
+dirotq_status_t dirotq_set_gemm_tile(int columns) { return set_w4a4_tile_columns(columns); }
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
                                        size_t workspace_bytes, float* xrot_f32, dirotq_stream_t stream) {

@@ -165,6 +165,7 @@ struct dirotq_layer {
     CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2] (nibble = q + 8), box 64 x kGemmBN, no swizzle
     CUtensorMap tmap_wscale;   // f32 [n_g][N], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
+    CUtensorMap tmap_wpacked128, tmap_wscale128, tmap_wh128;  // the same three with 128-row boxes (narrow W4A4 tiles)
     int act_scale_log2;        // NVFP4 variant: exponent of the activations' per-tensor power-of-two scale
 };
 
@@ -219,6 +220,7 @@ dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t 
 // launchers (each returns after enqueueing on `stream`)
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
 dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream);
+dirotq_status_t set_w4a4_tile_columns(int columns);
 struct Nvfp4GemmArgs {
     int M;
     const uint8_t* codes;  // [M][K4/2]

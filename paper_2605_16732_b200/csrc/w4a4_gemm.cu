@@ -30,31 +30,40 @@
 // Roles (384 threads = 3 warpgroups):
 //   warpgroup 0: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-3 nibble -> byte unpack
 //   warpgroups 1-2: epilogue; warp%4 selects the TMEM lane quadrant (token rows), the warpgroup
-//                   selects the 128-column half of the 256-wide tile.
+//                   selects the half of the tile's columns.
 #include "common.h"
 #include "ptx.cuh"
 
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 namespace dirotq {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = kGemmBN;  // 256
 constexpr int BKC = 128;  // one-byte codes per k-block (128-byte rows)
-constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_h chunk
-constexpr int BU_BYTES = BN * BKC;         // 32 KB  unpacked weight codes / bf16 W~_h chunk
-constexpr int BP_BYTES = BN * BKC / 2;     // 16 KB  packed weight codes (TMA staging)
-constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB
 constexpr int SC_SLOTS = 8;
-constexpr int SC_SW_BYTES = 2 * BN * 4;    // up to two groups per k-block
-constexpr int SC_SX_BYTES = 2 * 2 * BM * 4;  // scales of up to two groups, then their offset corrections
-constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 4 KB
 constexpr int NUM_THREADS = 384;
 constexpr int NUM_EPI_WARPS = 8;
-constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
-constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024;
+
+// Shared-memory plan for tiles of BN output columns.  256 columns is the default; 128-column tiles (with more
+// pipeline stages) are used when the wide ones would leave most SMs idle in the last wave, see the launcher.
+template <int BN>
+struct Plan {
+    static constexpr int STAGES = BN == 256 ? 3 : 5;
+    static constexpr int BU_BYTES = BN * BKC;         // unpacked weight codes / bf16 W~_h chunk (32 KB at BN = 256)
+    static constexpr int BP_BYTES = BN * BKC / 2;     // packed weight codes (TMA staging)
+    static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB / 40 KB
+    static constexpr int SC_SW_BYTES = 2 * BN * 4;    // up to two groups per k-block
+    static constexpr int SC_SX_BYTES = 2 * 2 * BM * 4;  // scales of up to two groups, then their offset corrections
+    static constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 4 KB / 3 KB
+    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
+    static constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024;
+};
+static_assert(Plan<256>::SMEM_BYTES <= 232448 && Plan<128>::SMEM_BYTES <= 232448, "shared memory plan too large");
+static_assert(Plan<128>::STAGE_BYTES % 1024 == 0 && Plan<128>::SC_BYTES % 128 == 0, "tile alignment");
 
 struct GemmKernelParams {
     int M, N, n_g, num_kb, lr_chunks;
@@ -87,12 +96,17 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int G, bool kPartials>
+template <int G, bool kPartials, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
                  const __grid_constant__ CUtensorMap tmap_wscale, const __grid_constant__ CUtensorMap tmap_xscale,
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                  const GemmKernelParams p) {
+    using P = Plan<BN>;
+    constexpr int STAGES = P::STAGES, STAGE_BYTES = P::STAGE_BYTES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES;
+    constexpr int SC_SW_BYTES = P::SC_SW_BYTES, SC_BYTES = P::SC_BYTES, BAR_OFFSET = P::BAR_OFFSET;
+    constexpr int HB = BN / 2;         // columns per epilogue warp: the warpgroup selects the half of the tile
+    constexpr int CHUNKS = HB / 16;    // 16-column chunks per epilogue warp and accumulator tile
     constexpr int GPK = BKC / G;       // groups per k-block: 2 (G = 64) or 1 (G = 128)
     constexpr int MMA_PER_G = G / 32;  // 8-bit MMA instructions (K = 32) per group
 
@@ -316,7 +330,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     } else {
         reg_alloc<208>();
         // ------------------------------------------------------------ epilogue (warps 4..11)
-        // A warp owns 32 token rows (its TMEM lane quadrant) x 128 columns.  The accumulators are read with the
+        // A warp owns 32 token rows (its TMEM lane quadrant) x BN/2 columns.  The accumulators are read with the
         // 16x256b shape: a thread then holds 4 rows (l/4 + 8 i) x the column pairs 2 (l%4) + {0, 1} of every block
         // of 8 columns, so one 8-byte load of weight scales serves four rows (with the 32x32b shape, one row per
         // thread, every thread would need all 128 column scales of every group and the shared-memory pipe, not the
@@ -333,10 +347,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
             const int rbase = m0 + q * 32 + lr4;  // this thread's rows: rbase + 8 i, i = 0..3
-            const int colbase = n0 + half * 128;
-            float accf[128];  // [((chunk c) * 2 + (block cb)) * 4 + row i] * 2 + {0, 1}
+            const int colbase = n0 + half * HB;
+            float accf[HB];  // [((chunk c) * 2 + (block cb)) * 4 + row i] * 2 + {0, 1}
 #pragma unroll
-            for (int j = 0; j < 128; ++j) accf[j] = 0.f;
+            for (int j = 0; j < HB; ++j) accf[j] = 0.f;
 
             for (int kb = 0; ok && kb < p.num_kb; ++kb, ++sc_it) {
                 const int slot = sc_it % SC_SLOTS;
@@ -359,15 +373,15 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         sxv[i] = s_sx[gi * BM + q * 32 + lr4 + 8 * i] * 262144.0f;
                         ev[i] = s_sx[(2 + gi) * BM + q * 32 + lr4 + 8 * i];
                     }
-                    const float* swp = s_sw + gi * BN + half * 128 + lc2;
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
-                    // software pipeline over eight 16-column chunks: the loads of chunk c+1 are in flight while
+                    const float* swp = s_sw + gi * BN + half * HB + lc2;
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * HB;
+                    // software pipeline over the 16-column chunks: the loads of chunk c+1 are in flight while
                     // chunk c is folded in (tcgen05.wait::ld waits for every outstanding load, hence depth one)
                     uint32_t raw[2][16];  // [0..7]: TMEM lanes 0..15 of the quadrant (rows i = 0, 1), [8..15]: lanes 16..31
                     tmem_ld_16x256b_x2(taddr, raw[0]);
                     tmem_ld_16x256b_x2(taddr + (16u << 16), raw[0] + 8);
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
+                    for (int c = 0; c < CHUNKS; ++c) {
                         uint32_t (&cur)[16] = raw[c & 1];
                         // this chunk's weight scales: requested before the wait so that their latency hides behind it
                         float2 w[2];
@@ -377,7 +391,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         }
                         tmem_ld_wait();
                         tmem_ld_fence(cur);
-                        if (c < 7) {
+                        if (c < CHUNKS - 1) {
                             tmem_ld_16x256b_x2(taddr + (c + 1) * 16, raw[(c + 1) & 1]);
                             tmem_ld_16x256b_x2(taddr + (16u << 16) + (c + 1) * 16, raw[(c + 1) & 1] + 8);
                         } else {
@@ -448,9 +462,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 ok = __any_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * 128;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * HB;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int c = 0; c < CHUNKS; ++c) {
                     uint32_t raw[16];
                     tmem_ld_16x256b_x2(taddr + c * 16, raw);
                     tmem_ld_16x256b_x2(taddr + (16u << 16) + c * 16, raw + 8);
@@ -479,7 +493,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 // warp writes 64 contiguous bytes per row.
                 const int j = lane & 3;
 #pragma unroll
-                for (int m = 0; m < 4; ++m) {
+                for (int m = 0; m < CHUNKS / 2; ++m) {
                     float2 bv[4];
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
@@ -526,9 +540,20 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     }
 }
 
-}  // namespace
+// A 128-column tile takes 0.70-0.76 of the time of a 256-column one (measured: the activation tile, the rank-r
+// branch, the pipeline fill and the per-group hand-over are paid per tile whatever its width), so narrow tiles are
+// chosen only when they shorten the schedule by more than that: when the wide tiles' last wave would be nearly
+// empty (PixArt-sized layers, N = 1152: 160 wide tiles on 148 SMs) or when there are fewer wide tiles than SMs.
+static bool narrow_tiles_pay(int M, int N, int sms) {
+    const long m_blocks = (M + BM - 1) / BM;
+    const long wide = m_blocks * ((N + 255) / 256), narrow = m_blocks * ((N + 127) / 128);
+    const double cost_wide = static_cast<double>((wide + sms - 1) / sms);
+    const double cost_narrow = 0.73 * static_cast<double>((narrow + sms - 1) / sms);
+    return cost_narrow < 0.98 * cost_wide;
+}
 
-dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
+template <int BN>
+static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     CUtensorMap tmap_codes, tmap_xscale, tmap_xh;
     dirotq_status_t st;
@@ -555,18 +580,36 @@ dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaS
                               const CUtensorMap, const CUtensorMap, const GemmKernelParams);
     KernelFn kern;
     const bool dbg = a.partials != nullptr;
-    if (g.G == 64) kern = dbg ? w4a4_gemm_kernel<64, true> : w4a4_gemm_kernel<64, false>;
-    else           kern = dbg ? w4a4_gemm_kernel<128, true> : w4a4_gemm_kernel<128, false>;
+    if (g.G == 64) kern = dbg ? w4a4_gemm_kernel<64, true, BN> : w4a4_gemm_kernel<64, false, BN>;
+    else           kern = dbg ? w4a4_gemm_kernel<128, true, BN> : w4a4_gemm_kernel<128, false, BN>;
     static bool attr_set[4] = {false, false, false, false};
     const int vi = (g.G == 64 ? 0 : 2) + (dbg ? 1 : 0);
     if (!attr_set[vi]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<BN>::SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
         attr_set[vi] = true;
     }
-    kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, L->tmap_wscale, tmap_xscale, tmap_xh,
-                                                    L->tmap_wh, p);
+    const bool narrow = BN == 128;
+    kern<<<grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream>>>(tmap_codes, narrow ? L->tmap_wpacked128 : L->tmap_wpacked,
+                                                              narrow ? L->tmap_wscale128 : L->tmap_wscale, tmap_xscale,
+                                                              tmap_xh, narrow ? L->tmap_wh128 : L->tmap_wh, p);
     return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+}  // namespace
+
+static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 128 / 256: forced
+
+dirotq_status_t set_w4a4_tile_columns(int columns) {
+    if (columns != 0 && columns != 128 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+    g_tile_columns.store(columns);
+    return DIROTQ_OK;
+}
+
+dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
+    const int forced = g_tile_columns.load();
+    const bool narrow = forced ? forced == 128 : narrow_tiles_pay(a.M, L->geo.N, sm_count(L->device));
+    return narrow ? launch_w4a4_gemm_bn<128>(L, a, stream) : launch_w4a4_gemm_bn<256>(L, a, stream);
 }
 
 }  // namespace dirotq

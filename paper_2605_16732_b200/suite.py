@@ -104,7 +104,31 @@ class Case:
             cb.append(a.elapsed_time(b))
         return float(np.median(rot)), float(np.median(gem)), float(np.median(cb))
 
-    def report(self, tag, iters, p_bf16, hbm):
+    def graph_ms(self, fn, calls=10, iters=20):
+        """Per-call device time of fn replayed from a CUDA graph of `calls` back-to-back calls: what a launch-bound
+        small layer costs once the host is out of the way (inputs of these small shapes stay in L2 between calls)."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                fn()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(calls):
+                    fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(iters):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            graph.replay()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / calls)
+        return float(np.median(ts))
+
+    def report(self, tag, iters, p_bf16, hbm, graphs=False):
         rot, gem, cb = self.time_kernels(iters)
         M, K, N, r, G = self.M, self.K, self.N, self.r, self.G
         K_l = K - r
@@ -124,6 +148,10 @@ class Case:
                 "frac_of_composite_roofline": t_roof / tot,
                 "algorithmic_gbs": bytes_alg / (tot * 1e-3) / 1e9, "frac_hbm_peak": bytes_alg / (tot * 1e-3) / 1e9 / hbm,
                 "cublas_bf16_ms": cb, "speedup_vs_cublas_bf16": cb / tot}
+        if graphs:
+            line["linear_graph_ms"] = self.graph_ms(self.run)
+            line["cublas_bf16_graph_ms"] = self.graph_ms(lambda: torch.matmul(self.x, self.Wb))
+            assert dq.dirotq_workspace_status(self.ws) == 0
         print(json.dumps(line), flush=True)
 
     def close(self):
@@ -145,12 +173,12 @@ def main():
 
     if "1" in todo:
         c = Case(256, 1152, 1152, 32, 64, synth.PIXART)
-        c.report("1: PixArt attention projection, M=256", args.iters, p_bf16, hbm)
+        c.report("1: PixArt attention projection, M=256", args.iters, p_bf16, hbm, graphs=True)
         c.close()
     if "2" in todo:
         for K, N in [(1152, 1152), (1152, 4608), (4608, 1152)]:
             c = Case(4096, K, N, 32, 64, synth.PIXART)
-            c.report("2: PixArt block linear, M=4096", args.iters, p_bf16, hbm)
+            c.report("2: PixArt block linear, M=4096", args.iters, p_bf16, hbm, graphs=True)
             c.close()
     if "2" in todo and FMT == "int4":
         # q, k, v of a PixArt block read the same activations: one rotate/quantize pass, three second-kernel launches

@@ -267,3 +267,48 @@ def test_host_entry_point_on_concurrent_streams():
     for c in cases:
         assert dq.dirotq_workspace_status(c["ws"]) == 0
         c["layer"].close()
+
+
+def test_layer_chain_replayed_from_a_cuda_graph_gives_the_same_bits():
+    # the entry points only enqueue work on the caller's stream (no allocation, no synchronisation), so a chain of
+    # layers can be captured once and replayed; small layers are launch-bound without this
+    specs = [synth.LayerSpec(K=256, N=512, r=32, G=64, model=synth.PIXART, seed=41, calib_tokens=512),
+             synth.LayerSpec(K=512, N=384, r=16, G=128, model=synth.PIXART, seed=42, calib_tokens=512),
+             synth.LayerSpec(K=384, N=256, r=32, G=64, model=synth.PIXART, seed=43, calib_tokens=512)]
+    M, dev = 200, "cuda"
+    layers, bufs = [], []
+    for spec in specs:
+        inp = synth.make_layer_inputs(spec, M, with_bias=True)
+        layers.append(dq.dirotq_prepare_layer(torch.from_numpy(inp["W"]).to(dev), torch.from_numpy(inp["Q"]).to(dev),
+                                              spec.r, spec.G, bias=bits_to_bf16_tensor(inp["bias"])))
+        bufs.append(torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev))
+    x0 = bits_to_bf16_tensor(synth.make_layer_inputs(specs[0], M)["x"])
+    wss = [dq.alloc_workspace(l, M) for l in layers]
+
+    def chain():
+        cur = x0
+        for l, y, ws in zip(layers, bufs, wss):
+            dq.dirotq_linear(cur, l, y, ws)
+            cur = y
+
+    chain()
+    torch.cuda.synchronize()
+    eager = [b.view(torch.int16).clone() for b in bufs]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            chain()
+    torch.cuda.current_stream().wait_stream(side)
+    for b in bufs:
+        b.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    for ws in wss:
+        assert dq.dirotq_workspace_status(ws) == 0
+    for b, e in zip(bufs, eager):
+        assert torch.equal(b.view(torch.int16), e)
+    for l in layers:
+        l.close()
