@@ -12,10 +12,11 @@
 //
 // Data movement: packed E2M1 operands by TMA (128-byte rows = 256 elements, 128-byte swizzle); the
 // E4M3 scale factors travel as 512-byte atoms (128 rows x 4 scales, row r at (r%32)*16 + (r/32)*4),
-// fetched with cp.async.bulk and copied into tensor memory with tcgen05.cp.32x128b.warpx4 by the MMA
-// thread right before the four MMAs (K = 64 each) that consume them.
+// fetched with cp.async.bulk and copied into tensor memory with tcgen05.cp.32x128b.warpx4 by two copier
+// threads, which hand the stage to the MMA thread through an mbarrier (tcgen05.commit).
 //
-// Roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue.
+// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue, warps 6..7 copy the
+// scale factors of each stage from shared to tensor memory (activation side / weight side).
 // TMEM: two 128-column fp32 accumulators (the epilogue of tile i overlaps the MMAs of tile i+1) and,
 // per pipeline stage, 16 + 16 columns of scale factors.
 #include "common.h"
@@ -34,7 +35,7 @@ constexpr int A_BYTES = BM * 128;      // 16 KB
 constexpr int B_BYTES = BN * 128;      // 16 KB
 constexpr int SF_BYTES = 4 * 512;      // four atoms per operand and k-block
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 2 * SF_BYTES;  // 36 KB
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 256;
 constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
 constexpr int BIAS_OFFSET = BAR_OFFSET + 256;  // two buffers of a tile's 128 bias values
 constexpr int SMEM_BYTES = BIAS_OFFSET + 2 * BN * 4 + 1024;
@@ -108,8 +109,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 128);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 132);
+    auto sfready_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + 4 + s); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 196);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -121,6 +123,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
+            mbar_init(sfready_bar(s), 2);  // one arrival per copier warp
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
@@ -198,11 +201,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     tc_fence_after_sync();
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * 32;
-#pragma unroll
-                    for (int a = 0; a < 4; ++a) {
-                        tmem_cp_32x128b_warpx4(tsf + 4 * a, sf_desc(st + A_BYTES + B_BYTES + a * 512));
-                        tmem_cp_32x128b_warpx4(tsf + 16 + 4 * a, sf_desc(st + A_BYTES + B_BYTES + SF_BYTES + a * 512));
-                    }
+                    // the scale factors of this stage are copied into tensor memory by the copier warp
+                    if (!mbar_wait(sfready_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    tc_fence_after_sync();
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
 #pragma unroll
@@ -213,7 +214,8 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                 if (!ok) break;
                 for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
                     const int s = it % STAGES;
-                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
+                        !mbar_wait(sfready_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     const uint64_t adesc = umma_desc_sw128(st);
@@ -223,6 +225,35 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     umma_commit(empty_bar(s));
                 }
                 if (ok) umma_commit(tfull_bar(acc));
+            }
+        }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ scale-factor copier
+        // A tcgen05.cp occupies the issuing thread for roughly a hundred cycles.  With the eight copies of a k-block on
+        // the MMA thread, that thread bounded the kernel (0.137 ms on the 4608 x 3072 -> 9216 layer; 0.112 ms with one
+        // copier thread, itself the bound; 0.093 ms with two).  Each copier hands its half of a stage over through an
+        // mbarrier that tcgen05.commit arrives on once the copies have landed in tensor memory.
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int items = p.num_kb + p.lr_chunks;
+                for (int i = 0; i < items; ++i, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK)) { ok = false; break; }
+                    if (i < p.num_kb) {
+                        tc_fence_after_sync();
+                        const uint32_t sf = smem_base + s * STAGE_BYTES + A_BYTES + B_BYTES;
+                        const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * 32;
+                        const uint32_t half = warp - 6;  // warp 6: activation scales, warp 7: weight scales
+#pragma unroll
+                        for (int a = 0; a < 4; ++a)
+                            tmem_cp_32x128b_warpx4(tsf + 16 * half + 4 * a, sf_desc(sf + half * SF_BYTES + a * 512));
+                        umma_commit(sfready_bar(s));
+                    } else {
+                        mbar_arrive(sfready_bar(s));  // a rank-r chunk: nothing to copy
+                    }
+                }
             }
         }
     } else {
