@@ -423,6 +423,8 @@ def main():
                     help="int4: the headline format (groups of 64, bf16 scales, symmetric); nvfp4: E2M1 blocks of 16 with E4M3 "
                          "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group); w4a8: per-token int8 "
                          "activations, per-channel int4 weights")
+    ap.add_argument("--gemm-tile", type=int, default=0, choices=[0, 128, 256],
+                    help="output columns per tile of the second kernel (int4 / int4_asym / nvfp4): 0 = chosen per call")
     ap.add_argument("--lite", action="store_true", help="skip the cuBLAS, end-to-end and CPU-baseline legs (profiling runs)")
     args = ap.parse_args()
     if args.shapes:
@@ -431,6 +433,9 @@ def main():
     if args.impl == "reference":
         run_reference(args)
     else:
+        if args.gemm_tile:
+            from paper_2605_16732_b200 import binding as _dq
+            _dq.dirotq_set_gemm_tile(args.gemm_tile)
         run_ours(args)
 
 

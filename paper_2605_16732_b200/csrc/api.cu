@@ -410,7 +410,10 @@ static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateAr
     return launch_w4a4_gemm(layer, ga, s);
 }
 
-dirotq_status_t dirotq_set_gemm_tile(int columns) { return set_w4a4_tile_columns(columns); }
+dirotq_status_t dirotq_set_gemm_tile(int columns) {
+    const dirotq_status_t st = set_w4a4_tile_columns(columns);
+    return st != DIROTQ_OK ? st : set_nvfp4_tile_columns(columns);
+}
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
                                        size_t workspace_bytes, float* xrot_f32, dirotq_stream_t stream) {

@@ -221,6 +221,7 @@ dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t 
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
 dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream);
 dirotq_status_t set_w4a4_tile_columns(int columns);
+dirotq_status_t set_nvfp4_tile_columns(int columns);
 struct Nvfp4GemmArgs {
     int M;
     const uint8_t* codes;  // [M][K4/2]

@@ -15,31 +15,48 @@
 // fetched with cp.async.bulk and copied into tensor memory with tcgen05.cp.32x128b.warpx4 by two copier
 // threads, which hand the stage to the MMA thread through an mbarrier (tcgen05.commit).
 //
-// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue, warps 6..7 copy the
-// scale factors of each stage from shared to tensor memory (activation side / weight side).
-// TMEM: two 128-column fp32 accumulators (the epilogue of tile i overlaps the MMAs of tile i+1) and,
-// per pipeline stage, 16 + 16 columns of scale factors.
+// Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..3 copy the scale factors of
+// each stage from shared to tensor memory (activation side / weight side), warps 4..11 epilogue.
+// TMEM: one 256-column fp32 accumulator (or two of 128 columns, see Plan) and, per pipeline stage, 16 columns of
+// scale factors for the tokens and 16 per 128 output columns.
 #include "common.h"
 #include "ptx.cuh"
 
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 namespace dirotq {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = kNvfp4BN;  // 128
 constexpr int BKE = 256;      // E2M1 elements per k-block (128-byte rows)
-constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * 128;      // 16 KB
-constexpr int B_BYTES = BN * 128;      // 16 KB
-constexpr int SF_BYTES = 4 * 512;      // four atoms per operand and k-block
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 2 * SF_BYTES;  // 36 KB
-constexpr int NUM_THREADS = 256;
-constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-constexpr int BIAS_OFFSET = BAR_OFFSET + 256;  // two buffers of a tile's 128 bias values
-constexpr int SMEM_BYTES = BIAS_OFFSET + 2 * BN * 4 + 1024;
-constexpr int TMEM_SF_BASE = 2 * BN;   // columns 256.. hold the scale factors: 32 per stage
+constexpr int SF_BYTES = 4 * 512;      // four atoms per 128 rows (tokens or output columns) and k-block
+constexpr int NUM_THREADS = 384;
+constexpr int NUM_EPI_WARPS = 8;
+
+// Tile plans.  Both kernels are bound by the stream of operands from L2 into shared memory, so the wider tile (a
+// quarter less traffic per flop) is the default; the 128-column plan double-buffers the accumulator and serves
+// layers with few tiles.  With 256 columns one accumulator (256 of the 512 tensor-memory columns) is all that fits
+// beside the scale factors: the epilogue of a tile then does not overlap the MMAs of the next, but the producer keeps
+// filling the stages meanwhile, and the MMAs catch up on a full pipeline.
+template <int BN>
+struct Plan {
+    static constexpr int NB = BN / 128;               // 128-column blocks per tile
+    static constexpr int STAGES = BN == 128 ? 6 : 4;
+    static constexpr int ACC_BUFS = BN == 128 ? 2 : 1;
+    static constexpr int B_BYTES = BN * 128;          // 16 / 32 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + (1 + NB) * SF_BYTES;  // 36 / 54 KB
+    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int BIAS_OFFSET = BAR_OFFSET + 256;  // two buffers of a tile's bias values
+    static constexpr int SMEM_BYTES = BIAS_OFFSET + 2 * BN * 4 + 1024;
+    static constexpr int TMEM_SF_BASE = ACC_BUFS * BN;    // columns 256.. hold the scale factors
+    static constexpr int SF_COLS = 16 * (1 + NB);         // per stage: 16 columns for the tokens, 16 per 128 output columns
+    static_assert(TMEM_SF_BASE + STAGES * SF_COLS <= 512, "tensor memory plan");
+    static_assert(SMEM_BYTES <= 232448, "shared memory plan");
+    static_assert(STAGE_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+};
 
 struct NvKernelParams {
     int M, N, num_kb, nkb64p, lr_chunks;
@@ -97,10 +114,15 @@ __device__ __forceinline__ void umma_nvfp4(uint32_t d_tmem, uint64_t adesc, uint
         : "memory");
 }
 
+template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wcodes,
                   const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                   const NvKernelParams p) {
+    using P = Plan<BN>;
+    constexpr int NB = P::NB, STAGES = P::STAGES, ACC_BUFS = P::ACC_BUFS, B_BYTES = P::B_BYTES;
+    constexpr int STAGE_BYTES = P::STAGE_BYTES, BAR_OFFSET = P::BAR_OFFSET, BIAS_OFFSET = P::BIAS_OFFSET;
+    constexpr int TMEM_SF_BASE = P::TMEM_SF_BASE, SF_COLS = P::SF_COLS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -127,7 +149,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 4);
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -153,17 +175,23 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 const int m_blk = tile % num_m_blocks, n_blk = tile / num_m_blocks;
                 const int m0 = m_blk * BM, n0 = n_blk * BN;
+                // 128-column blocks of this tile that exist (the scale atoms of a missing one are not fetched; its
+                // outputs are never stored)
+                const int nb_here = min(NB, (p.N + 127) / 128 - n_blk * NB);
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t st = smem_base + s * STAGE_BYTES;
-                    mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+                    mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES + (1 + nb_here) * SF_BYTES);
                     tma_load_2d(st, &tmap_codes, full_bar(s), kb * 128, m0);             // byte coordinates
-                    tma_load_2d(st + A_BYTES, &tmap_wcodes, full_bar(s), kb * 128, n0);
+#pragma unroll
+                    for (int b = 0; b < NB; ++b)  // rows past N are filled with zeros (and still counted)
+                        tma_load_2d(st + A_BYTES + b * 16384, &tmap_wcodes, full_bar(s), kb * 128, n0 + b * 128);
                     bulk_load(st + A_BYTES + B_BYTES, p.xsf + (static_cast<size_t>(m_blk) * p.nkb64p + kb * 4) * 512, SF_BYTES,
                               full_bar(s));
-                    bulk_load(st + A_BYTES + B_BYTES + SF_BYTES, p.wsf + (static_cast<size_t>(n_blk) * p.nkb64p + kb * 4) * 512,
-                              SF_BYTES, full_bar(s));
+                    for (int b = 0; b < nb_here; ++b)
+                        bulk_load(st + A_BYTES + B_BYTES + (1 + b) * SF_BYTES,
+                                  p.wsf + (static_cast<size_t>(n_blk * NB + b) * p.nkb64p + kb * 4) * 512, SF_BYTES, full_bar(s));
                 }
                 if (!ok) break;
                 for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
@@ -172,7 +200,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
                     tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
-                    tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), lr * 64, n0);
+#pragma unroll
+                    for (int b = 0; b < NB; ++b)
+                        tma_load_2d(st + A_BYTES + b * 16384, &tmap_wh, full_bar(s), lr * 64, n0 + b * 128);
                 }
             }
             if (!ok) {
@@ -191,8 +221,8 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-                const uint32_t acc = tcount & 1;
-                if (!mbar_wait(tempty_bar(acc), ((tcount >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                const uint32_t acc = tcount % ACC_BUFS;
+                if (!mbar_wait(tempty_bar(acc), ((tcount / ACC_BUFS) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + acc * BN;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
@@ -200,7 +230,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t st = smem_base + s * STAGE_BYTES;
-                    const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * 32;
+                    const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * SF_COLS;
                     // the scale factors of this stage are copied into tensor memory by the copier warp
                     if (!mbar_wait(sfready_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
@@ -208,7 +238,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)  // K = 64 elements = 32 bytes per instruction
-                        umma_nvfp4(d, adesc + 2 * k, bdesc + 2 * k, idesc_nv, tsf + 4 * k, tsf + 16 + 4 * k, (kb | k) != 0);
+                        umma_nvfp4(d, adesc + 2 * k, bdesc + 2 * k, idesc_nv, tsf + 4 * k, tsf + 16 + 4 * NB * k, (kb | k) != 0);
                     umma_commit(empty_bar(s));
                 }
                 if (!ok) break;
@@ -227,7 +257,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                 if (ok) umma_commit(tfull_bar(acc));
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp < 4) {
         // ------------------------------------------------------------ scale-factor copier
         // A tcgen05.cp occupies the issuing thread for roughly a hundred cycles.  With the eight copies of a k-block on
         // the MMA thread, that thread bounded the kernel (0.137 ms on the 4608 x 3072 -> 9216 layer; 0.112 ms with one
@@ -244,11 +274,19 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     if (i < p.num_kb) {
                         tc_fence_after_sync();
                         const uint32_t sf = smem_base + s * STAGE_BYTES + A_BYTES + B_BYTES;
-                        const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * 32;
-                        const uint32_t half = warp - 6;  // warp 6: activation scales, warp 7: weight scales
+                        const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * SF_COLS;
+                        if (warp == 2) {
+                            // activation scales: the four K = 64 steps of the k-block, 4 columns each
 #pragma unroll
-                        for (int a = 0; a < 4; ++a)
-                            tmem_cp_32x128b_warpx4(tsf + 16 * half + 4 * a, sf_desc(sf + half * SF_BYTES + a * 512));
+                            for (int a = 0; a < 4; ++a) tmem_cp_32x128b_warpx4(tsf + 4 * a, sf_desc(sf + a * 512));
+                        } else {
+                            // weight scales: per K step, the tile's 128-column blocks side by side (4 columns each)
+#pragma unroll
+                            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                                for (int b = 0; b < NB; ++b)
+                                    tmem_cp_32x128b_warpx4(tsf + 16 + 4 * NB * a + 4 * b, sf_desc(sf + (1 + b) * SF_BYTES + a * 512));
+                        }
                         umma_commit(sfready_bar(s));
                     } else {
                         mbar_arrive(sfready_bar(s));  // a rank-r chunk: nothing to copy
@@ -257,30 +295,35 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------ epilogue (warps 4..11)
+        // warp % 4 selects the TMEM lane quadrant (32 token rows), the warpgroup the half of the tile's columns.  The
+        // whole slice of the accumulator is read into registers first and the accumulator handed back at once, so that
+        // the conversion and the stores overlap the next tile's MMAs even where there is a single accumulator.
+        constexpr int HB = BN / 2;
         const int q = warp & 3;
+        const int half = (warp - 4) >> 2;
         uint32_t tcount = 0;
         bool ok = true;
         const float out_scale = __ldg(p.out_scale);
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
-            const uint32_t acc = tcount & 1;
+            const uint32_t acc = tcount % ACC_BUFS;
             // The tile's bias goes to shared memory while its MMAs are still running (two buffers: a warp can be one tile
-            // ahead of the others).  The reducing barrier orders the stores before the reads below and makes the four
+            // ahead of the others).  The reducing barrier orders the stores before the reads below and makes the eight
             // warps agree on whether to go on: a plain barrier behind a bounded wait could strand a warp.
             float* s_b = reinterpret_cast<float*>(smem_gen + BIAS_OFFSET) + (tcount & 1) * BN;
             {
-                const int e = threadIdx.x - 64;  // 0..127
-                s_b[e] = n0 + e < p.N ? __ldg(p.bias + n0 + e) : 0.f;
+                const int e = threadIdx.x - 128;  // 0..255
+                if (e < BN) s_b[e] = n0 + e < p.N ? __ldg(p.bias + n0 + e) : 0.f;
             }
-            const bool mine = mbar_wait(tfull_bar(acc), (tcount >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+            const bool mine = mbar_wait(tfull_bar(acc), (tcount / ACC_BUFS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
             uint32_t any_failed;
             asm volatile(
                 "{\n\t"
                 ".reg .pred pin, pout;\n\t"
                 "setp.eq.u32 pin, %1, 0;\n\t"
-                "bar.red.or.pred pout, 1, 128, pin;\n\t"
+                "bar.red.or.pred pout, 1, 256, pin;\n\t"
                 "selp.u32 %0, 1, 0, pout;\n\t"
                 "}\n"
                 : "=r"(any_failed)
@@ -290,31 +333,30 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             if (!ok) break;
             tc_fence_after_sync();
             const int row = m0 + q * 32 + lane;
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t raw[32];
-                tmem_ld_32x32b_x32(taddr + c * 32, raw);
-                tmem_ld_wait();
-                if (c == BN / 32 - 1) {
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar(acc));
-                }
-                const int col = n0 + c * 32;
-                if (row < p.M) {
-                    uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + col;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + half * HB;
+            uint32_t raw[HB / 32][32];
+#pragma unroll
+            for (int c = 0; c < HB / 32; ++c) tmem_ld_32x32b_x32(taddr + c * 32, raw[c]);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (row < p.M) {
+                const float* bq = s_b + half * HB;
+                uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + n0 + half * HB;
+#pragma unroll
+                for (int c = 0; c < HB / 32; ++c) {
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
-                        if (col + j < p.N) {
-                            const float4 b0 = *reinterpret_cast<const float4*>(s_b + c * 32 + j);
-                            const float4 b1 = *reinterpret_cast<const float4*>(s_b + c * 32 + j + 4);
+                        if (n0 + half * HB + c * 32 + j < p.N) {
+                            const float4 b0 = *reinterpret_cast<const float4*>(bq + c * 32 + j);
+                            const float4 b1 = *reinterpret_cast<const float4*>(bq + c * 32 + j + 4);
                             uint4 o;
-                            o.x = pack_bf16x2(fmaf(__uint_as_float(raw[j + 0]), out_scale, b0.x), fmaf(__uint_as_float(raw[j + 1]), out_scale, b0.y));
-                            o.y = pack_bf16x2(fmaf(__uint_as_float(raw[j + 2]), out_scale, b0.z), fmaf(__uint_as_float(raw[j + 3]), out_scale, b0.w));
-                            o.z = pack_bf16x2(fmaf(__uint_as_float(raw[j + 4]), out_scale, b1.x), fmaf(__uint_as_float(raw[j + 5]), out_scale, b1.y));
-                            o.w = pack_bf16x2(fmaf(__uint_as_float(raw[j + 6]), out_scale, b1.z), fmaf(__uint_as_float(raw[j + 7]), out_scale, b1.w));
-                            *reinterpret_cast<uint4*>(yrow + j) = o;
+                            o.x = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 0]), out_scale, b0.x), fmaf(__uint_as_float(raw[c][j + 1]), out_scale, b0.y));
+                            o.y = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 2]), out_scale, b0.z), fmaf(__uint_as_float(raw[c][j + 3]), out_scale, b0.w));
+                            o.z = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 4]), out_scale, b1.x), fmaf(__uint_as_float(raw[c][j + 5]), out_scale, b1.y));
+                            o.w = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 6]), out_scale, b1.z), fmaf(__uint_as_float(raw[c][j + 7]), out_scale, b1.w));
+                            *reinterpret_cast<uint4*>(yrow + c * 32 + j) = o;
                         }
                     }
                 }
@@ -330,9 +372,8 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
     }
 }
 
-}  // namespace
-
-dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a, cudaStream_t stream) {
+template <int BN>
+static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4GemmArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     CUtensorMap tmap_codes, tmap_xh;
     dirotq_status_t st;
@@ -356,12 +397,37 @@ dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a,
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(nvfp4_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(nvfp4_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<BN>::SMEM_BYTES) !=
+            cudaSuccess)
             return DIROTQ_ERR_CUDA;
         attr_set = true;
     }
-    nvfp4_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand
+    nvfp4_gemm_kernel<BN><<<grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, tmap_xh,
+                                                                             L->tmap_wh, p);
     return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+static std::atomic<int> g_nv_tile_columns{0};  // 0: chosen per call; 128 / 256: forced
+
+}  // namespace
+
+dirotq_status_t set_nvfp4_tile_columns(int columns) {
+    if (columns != 0 && columns != 128 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+    g_nv_tile_columns.store(columns);
+    return DIROTQ_OK;
+}
+
+dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a, cudaStream_t stream) {
+    // A 128-column tile takes about 0.6 of the time of a 256-column one (measured), so the narrow plan is chosen only
+    // when it fills the SMs so much better that it wins anyway (few tiles, or a nearly empty last wave).
+    const int forced = g_nv_tile_columns.load();
+    const int sms = sm_count(L->device);
+    const long m_blocks = (a.M + BM - 1) / BM;
+    const long t_wide = m_blocks * ((L->geo.N + 255) / 256), t_narrow = m_blocks * ((L->geo.N + 127) / 128);
+    const bool narrow_pays = 0.6 * static_cast<double>((t_narrow + sms - 1) / sms) < 0.98 * static_cast<double>((t_wide + sms - 1) / sms);
+    const bool wide = forced ? forced == 256 : !narrow_pays;
+    return wide ? launch_nvfp4_gemm_bn<256>(L, a, stream) : launch_nvfp4_gemm_bn<128>(L, a, stream);
 }
 
 }  // namespace dirotq

@@ -74,3 +74,59 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
     finally:
         dq.dirotq_set_gemm_tile(0)
     layer.close()
+
+
+# ------------------------------------------------------------------ NVFP4 second kernel: 128- and 256-column tiles
+
+import test_gpu_nvfp4
+
+
+@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+def test_nvfp4_ragged_columns_two_blocks_in_last_tile(tile):
+    # N = 400: four 128-column blocks, the last one ragged
+    spec = synth.LayerSpec(K=512, N=400, r=16, G=64, model=synth.FLUX, seed=51, calib_tokens=1024)
+    print(tile, test_gpu_nvfp4._run_case(spec, M=300))
+
+
+@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+def test_nvfp4_odd_number_of_column_blocks(tile):
+    # N = 384: three 128-column blocks, so the second 256-column tile has no second block (its scale atoms do not exist)
+    spec = synth.LayerSpec(K=768, N=384, r=32, G=64, model=synth.PIXART, seed=52, calib_tokens=1024)
+    print(tile, test_gpu_nvfp4._run_case(spec, M=257, with_bias=False))
+
+
+@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+def test_nvfp4_single_column_block_and_two_rank_chunks(tile):
+    spec = synth.LayerSpec(K=640, N=128, r=128, G=64, model=synth.FLUX, seed=53, calib_tokens=1024)
+    print(tile, test_gpu_nvfp4._run_case(spec, M=130))
+
+
+def test_nvfp4_both_widths_give_the_same_bits():
+    from oracle import dirotq_oracle as orc
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=54)
+    M = 4096 + 77
+    inp = synth.make_layer_inputs(spec, M, with_bias=True)
+    dev = "cuda"
+    W, Q = torch.from_numpy(inp["W"]).to(dev), torch.from_numpy(inp["Q"]).to(dev)
+    x = bits_to_bf16_tensor(inp["x"])
+    probe = dq.dirotq_prepare_layer_nvfp4(W, Q, spec.r, 0)
+    xrot = torch.empty((256, spec.K), dtype=torch.float32, device=dev)
+    dq.dirotq_rotate_quantize(x[:256], probe, dq.alloc_workspace(probe, 256), xrot)
+    ex = orc.nvfp4_global_exponent(float(xrot[:, spec.r:].abs().max().item()))
+    probe.close()
+    layer = dq.dirotq_prepare_layer_nvfp4(W, Q, spec.r, ex, bias=bits_to_bf16_tensor(inp["bias"]))
+    ws = dq.alloc_workspace(layer, M)
+    outs = {}
+    try:
+        for cols in (0, 128, 256):
+            dq.dirotq_set_gemm_tile(cols)
+            y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
+            dq.dirotq_linear(x, layer, y, ws)
+            torch.cuda.synchronize()
+            assert dq.dirotq_workspace_status(ws) == 0
+            outs[cols] = y.view(torch.int16).clone()
+        # the accumulation order inside the tensor core does not depend on the tile width: same bits
+        assert torch.equal(outs[128], outs[256]) and torch.equal(outs[0], outs[128])
+    finally:
+        dq.dirotq_set_gemm_tile(0)
+    layer.close()
