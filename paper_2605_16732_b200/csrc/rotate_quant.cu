@@ -10,9 +10,16 @@
 // the epilogue warps, where each thread owns one token row, so the group maximum is a
 // thread-local reduction over the row's G values.
 //
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
-// warps 2..5 = epilogue (lane quadrant = warp_id % 4).  Persistent CTAs walk the tile list;
-// two 128x256 fp32 accumulators in TMEM let the epilogue of tile i overlap the MMAs of tile i+1.
+// Roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
+// warps 2..9 = epilogue (lane quadrant = warp_id % 4; the two warps of a quadrant take half of the
+// tile's column groups each).  Persistent CTAs walk the tile list; two 128x256 fp32 accumulators in
+// TMEM let the epilogue of tile i overlap the MMAs of tile i+1.
+//
+// What bounds it (timing runs with one kind of work switched off, 4608 x 3072 x 3072): the operand stream
+// alone takes 0.050 ms (1.0 GB from L2 at 20 TB/s with 4 x 48 KB in flight per SM; 0.056 ms with three
+// stages, so the ring depth, i.e. the latency of a loaded L2, sets the rate), with the MMAs 0.064 ms (a
+// stage is only refilled once its MMAs have completed, which adds their time to each slot's cycle), with
+// the epilogue 0.069 ms (0.074 ms with four epilogue warps).  All 227 KB of shared memory are in use.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -28,7 +35,7 @@ constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;  // 16 KB
 constexpr int B_BYTES = BN_MAX * BK * 2;  // 32 KB (a 128-column tile uses half of it)
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, eight epilogue warps
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct RotKernelParams {
@@ -174,7 +181,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+            mbar_init(tempty_bar(a), 8);  // one arrival per epilogue warp
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -249,6 +256,8 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     } else {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;  // two warps per quadrant share a tile's column chunks
+        constexpr int CHUNKS = BN / G, CPH = CHUNKS > 1 ? CHUNKS / 2 : 1;
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
@@ -265,7 +274,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
             float tile_amax = 0.f;  // W4A8: this thread's row, this tile's columns
 #pragma unroll 1
-            for (int chunk = 0; chunk < BN / G; ++chunk) {
+            for (int chunk = half * CPH; chunk < min(CHUNKS, (half + 1) * CPH); ++chunk) {
                 const int col0 = n0 + chunk * G;  // permuted column of v[0]
                 if (col0 >= p.K) break;
                 float v[G];
@@ -421,7 +430,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
-            if (n_blk == num_n_blocks - 1 && row_ok) {
+            if (n_blk == num_n_blocks - 1 && row_ok && half == 0) {
                 for (int c = p.r; c < p.r_pad0; c += 8)
                     *reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + c) = make_uint4(0, 0, 0, 0);
                 if constexpr (FMT == 2) {  // behind the 3 n_g zero-point columns
