@@ -357,7 +357,7 @@ def dirotq_prepare_layer_asym(W: torch.Tensor, Q: torch.Tensor, r: int, group: i
 
 
 def dirotq_set_gemm_tile(columns: int) -> None:
-    """Output columns per tile of the INT4 second kernel: 0 automatic, 128 or 256 forced (process-wide)."""
+    """Output columns per tile of the INT4 and NVFP4 second kernels: 0 automatic, 128 or 256 forced (process-wide)."""
     _check(lib().dirotq_set_gemm_tile(int(columns)), "dirotq_set_gemm_tile")
 
 
