@@ -176,6 +176,13 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
  * order).  W4A8 layers ignore it.  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
 
+/* The second kernel of a layer is launched as a programmatic dependent launch: it may be scheduled onto SMs that
+ * the first kernel's thread blocks have left and runs its set-up there, then waits (griddepcontrol.wait) for the
+ * whole first kernel before it reads anything.  Results are unaffected; the launch gap between the two kernels
+ * shrinks, which matters for small layers.  enabled == 0 switches this off process-wide (plain stream order),
+ * anything else on (default).  Works in stream capture. */
+DIROTQ_API dirotq_status_t dirotq_set_dependent_launch(int enabled);
+
 /* Unpacks a prepared layer: wcodes int8 [K-r,N]; wscales bf16 [n_g,N]; wh bf16 [r,N];
  * q_bf16 [K,K] in the layout of the Q argument.  Any pointer may be NULL. */
 DIROTQ_API dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16,

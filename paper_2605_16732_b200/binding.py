@@ -29,7 +29,7 @@ EXPORTED = [
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
-    "dirotq_prepare_layer_codes", "dirotq_set_gemm_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_prepare_layer_codes", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_layer_bytes_asym.argtypes = [i, i, i, i, psz]
         L.dirotq_prepare_layer_asym.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_set_gemm_tile.argtypes = [i]
+        L.dirotq_set_dependent_launch.argtypes = [i]
         L.dirotq_prepare_layer_codes.argtypes = [vp, i, i, vp, i, vp, vp, vp, i, i, i, i, i, vp, sz, vp, sz, vp,
                                                  ctypes.POINTER(vp)]
         L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -359,6 +360,11 @@ def dirotq_prepare_layer_asym(W: torch.Tensor, Q: torch.Tensor, r: int, group: i
 def dirotq_set_gemm_tile(columns: int) -> None:
     """Output columns per tile of the INT4 and NVFP4 second kernels: 0 automatic, 128 or 256 forced (process-wide)."""
     _check(lib().dirotq_set_gemm_tile(int(columns)), "dirotq_set_gemm_tile")
+
+
+def dirotq_set_dependent_launch(enabled: bool) -> None:
+    """Programmatic dependent launch of each layer's second kernel: on (default) or off, process-wide."""
+    _check(lib().dirotq_set_dependent_launch(int(bool(enabled))), "dirotq_set_dependent_launch")
 
 
 def dirotq_prepare_layer_codes(W: torch.Tensor, Q: torch.Tensor, wcodes: torch.Tensor, wscales: torch.Tensor, r: int,

@@ -1,6 +1,8 @@
 // C ABI of libdirotq: argument validation, tensor-map construction, launch sequencing.
 #include "common.h"
 
+#include <atomic>
+
 #include <mutex>
 
 #include <stdio.h>
@@ -93,6 +95,10 @@ dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t 
     }
     return DIROTQ_OK;
 }
+
+static std::atomic<bool> g_dependent_launch{true};
+bool dependent_launch_enabled() { return g_dependent_launch.load(); }
+void set_dependent_launch(bool on) { g_dependent_launch.store(on); }
 
 }  // namespace dirotq
 
@@ -408,6 +414,11 @@ static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateAr
     ga.M = M; ga.codes = ra.codes; ga.xscale = ra.xscale; ga.ldm = ra.ldm; ga.xh = ra.xh;
     ga.y = static_cast<uint16_t*>(y); ga.partials = nullptr; ga.status = ra.status;
     return launch_w4a4_gemm(layer, ga, s);
+}
+
+dirotq_status_t dirotq_set_dependent_launch(int enabled) {
+    dirotq::set_dependent_launch(enabled != 0);
+    return DIROTQ_OK;
 }
 
 dirotq_status_t dirotq_set_gemm_tile(int columns) {

@@ -2,6 +2,8 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
+
+#include <utility>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -221,6 +223,28 @@ dirotq_status_t encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t 
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
 dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream);
 dirotq_status_t set_w4a4_tile_columns(int columns);
+// Launches `kern`; with `dependent` (and unless switched off process-wide) as a programmatic dependent launch: the
+// kernel may be scheduled while the previous kernel of the stream drains, and orders itself with
+// grid_dependency_wait().
+bool dependent_launch_enabled();
+void set_dependent_launch(bool on);
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, bool dependent,
+                                 Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    const bool pdl = dependent && dependent_launch_enabled();
+    cfg.attrs = pdl ? attr : nullptr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 dirotq_status_t set_nvfp4_tile_columns(int columns);
 struct Nvfp4GemmArgs {
     int M;

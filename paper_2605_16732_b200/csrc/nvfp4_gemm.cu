@@ -166,6 +166,10 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
+    grid_dependency_wait();
+    // the next layer's first kernel may be scheduled as this grid's CTAs leave their SMs (it waits for this whole grid)
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -403,9 +407,9 @@ static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4Ge
         attr_set = true;
     }
     // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand
-    nvfp4_gemm_kernel<BN><<<grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, tmap_xh,
-                                                                             L->tmap_wh, p);
-    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+    const cudaError_t err = launch_kernel(nvfp4_gemm_kernel<BN>, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true,
+                                          tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 static std::atomic<int> g_nv_tile_columns{0};  // 0: chosen per call; 128 / 256: forced

@@ -191,6 +191,15 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start before the previous kernel of
+// the stream has finished; it must execute grid_dependency_wait() before it touches anything that kernel wrote (or
+// writes anything that kernel reads).  The wait returns at once in a kernel launched without the attribute.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream (if launched with the attribute) be scheduled once every CTA of this grid has
+// executed this or exited.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- TMEM -> registers
 
 // 32 lanes x 32 columns of 32-bit: thread i of the warp receives lane (base_lane + i),

@@ -196,6 +196,10 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dependency_wait();
+    // the second kernel of the layer may be scheduled onto SMs as this grid's CTAs leave them (it waits for the whole
+    // grid before it reads anything)
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -478,6 +482,8 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         {rotate_quant_kernel<64, 0, 128>, rotate_quant_kernel<128, 0, 128>, rotate_quant_kernel<64, 1, 128>,
          rotate_quant_kernel<64, 2, 128>, rotate_quant_kernel<128, 2, 128>, rotate_quant_kernel<64, 3, 128>}};
     const KernelFn kern = table[narrow ? 1 : 0][vi];
+    // a dependent launch needs a kernel as the previous operation of the stream: the W4A8 path puts a memset there
+    const bool dependent = g.fmt != 3;
     static bool attr_set[2][6] = {};
     if (!attr_set[narrow ? 1 : 0][vi]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
@@ -485,11 +491,11 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         attr_set[narrow ? 1 : 0][vi] = true;
     }
     if (narrow) {
-        kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_x, L->tmap_qt128, p);
-        return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+        return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, L->tmap_qt128, p) == cudaSuccess
+                   ? DIROTQ_OK : DIROTQ_ERR_CUDA;
     }
-    kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_x, L->tmap_qt, p);
-    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, L->tmap_qt, p) == cudaSuccess
+               ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 }  // namespace dirotq

@@ -164,6 +164,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
+    grid_dependency_wait();
+    // the next layer's first kernel may be scheduled as this grid's CTAs leave their SMs (it waits for this whole grid)
+    grid_launch_dependents();
 
     if (warp < 4) {
         reg_dealloc<72>();
@@ -590,10 +594,11 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
         attr_set[vi] = true;
     }
     const bool narrow = BN == 128;
-    kern<<<grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream>>>(tmap_codes, narrow ? L->tmap_wpacked128 : L->tmap_wpacked,
-                                                              narrow ? L->tmap_wscale128 : L->tmap_wscale, tmap_xscale,
-                                                              tmap_xh, narrow ? L->tmap_wh128 : L->tmap_wh, p);
-    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+    const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
+                                          narrow ? L->tmap_wpacked128 : L->tmap_wpacked,
+                                          narrow ? L->tmap_wscale128 : L->tmap_wscale, tmap_xscale, tmap_xh,
+                                          narrow ? L->tmap_wh128 : L->tmap_wh, p);
+    return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 }  // namespace

@@ -108,6 +108,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
+    grid_dependency_wait();
+    // the next layer's first kernel may be scheduled as this grid's CTAs leave their SMs (it waits for this whole grid)
+    grid_launch_dependents();
     const int items = p.num_kb + p.lr_chunks;  // pipeline items per tile
 
     if (warp == 0) {
@@ -360,8 +364,9 @@ dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cud
             return DIROTQ_ERR_CUDA;
         attr_set[dbg] = true;
     }
-    kern<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
-    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+    const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, true, tmap_codes, L->tmap_wpacked,
+                                          tmap_xh, L->tmap_wh, p);
+    return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 }  // namespace dirotq

@@ -312,3 +312,37 @@ def test_layer_chain_replayed_from_a_cuda_graph_gives_the_same_bits():
         assert torch.equal(b.view(torch.int16), e)
     for l in layers:
         l.close()
+
+
+def test_dependent_launch_on_and_off_give_the_same_bits():
+    # the second kernel of a layer (and the first kernel of the next) is scheduled early and orders itself with
+    # griddepcontrol.wait; a chain on ONE workspace is the case where an early writer would be caught
+    specs = [synth.LayerSpec(K=512, N=512, r=32, G=64, model=synth.PIXART, seed=61, calib_tokens=512),
+             synth.LayerSpec(K=512, N=512, r=16, G=128, model=synth.PIXART, seed=62, calib_tokens=512)]
+    M, dev = 700, "cuda"
+    layers = []
+    for spec in specs:
+        inp = synth.make_layer_inputs(spec, M, with_bias=True)
+        layers.append(dq.dirotq_prepare_layer(torch.from_numpy(inp["W"]).to(dev), torch.from_numpy(inp["Q"]).to(dev),
+                                              spec.r, spec.G, bias=bits_to_bf16_tensor(inp["bias"])))
+    x0 = bits_to_bf16_tensor(synth.make_layer_inputs(specs[0], M)["x"])
+    ws = dq.alloc_workspace(layers[0], M)
+    assert ws.numel() >= dq.alloc_workspace(layers[1], M).numel()
+    bufs = [torch.zeros((M, 512), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    outs = {}
+    try:
+        for on in (False, True):
+            dq.dirotq_set_dependent_launch(on)
+            for b in bufs:
+                b.zero_()
+            for _ in range(4):      # ping-pong through both layers, same workspace throughout
+                dq.dirotq_linear(x0, layers[0], bufs[0], ws)
+                dq.dirotq_linear(bufs[0], layers[1], bufs[1], ws)
+            torch.cuda.synchronize()
+            assert dq.dirotq_workspace_status(ws) == 0
+            outs[on] = [b.view(torch.int16).clone() for b in bufs]
+        assert all(torch.equal(a, b) for a, b in zip(outs[False], outs[True]))
+    finally:
+        dq.dirotq_set_dependent_launch(True)
+    for l in layers:
+        l.close()
