@@ -31,12 +31,12 @@ namespace {
 constexpr int BM = 128;       // tokens per tile
 constexpr int BN_MAX = 256;   // rotated columns per tile: 256, or 128 when there are few tiles (template parameter BN)
 constexpr int BK = 64;        // bf16 elements per k-block (128-byte rows)
-constexpr int STAGES = 4;
+constexpr int STAGES_WIDE = 4;  // 256-column tiles: 4 x 48 KB; 128-column tiles: 6 x 32 KB (same bytes in flight)
 constexpr int A_BYTES = BM * BK * 2;  // 16 KB
 constexpr int B_BYTES = BN_MAX * BK * 2;  // 32 KB (a 128-column tile uses half of it)
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int STAGE_BYTES_WIDE = A_BYTES + B_BYTES;
 constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, eight epilogue warps
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = STAGES_WIDE * STAGE_BYTES_WIDE + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct RotKernelParams {
     int M, K, K_l, K_lp, r, r_pad, r_pad0, ldm, n_g;
@@ -156,6 +156,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const RotKernelParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    // The ring holds 192 KB either way; with narrow tiles it is cut into more, smaller stages: the operand stream is
+    // paced by (L2 latency + MMA time of a stage) / number of stages.
+    constexpr int STAGES = BN == 256 ? STAGES_WIDE : 6;
+    constexpr int STAGE_BYTES = A_BYTES + BN * BK * 2;
+    static_assert(STAGES * STAGE_BYTES == STAGES_WIDE * STAGE_BYTES_WIDE && STAGE_BYTES % 1024 == 0, "ring layout");
     const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
     // barrier map (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
