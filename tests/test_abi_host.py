@@ -69,3 +69,19 @@ def test_null_and_bad_handles_are_rejected(L):
     # a fake handle (wrong magic) is refused too
     fake = ctypes.create_string_buffer(4096)
     assert L.dirotq_workspace_bytes(fake, 16, ctypes.byref(n)) == 1
+
+
+def test_knobs_validate_their_argument_without_a_gpu(L):
+    for ok in (0, 128, 256, 0):
+        assert L.dirotq_set_gemm_tile(ok) == 0
+    for bad in (-1, 64, 192, 512):
+        assert L.dirotq_set_gemm_tile(bad) == 1
+    assert L.dirotq_set_dependent_launch(0) == 0 and L.dirotq_set_dependent_launch(1) == 0
+
+
+def test_prepare_from_codes_rejects_null_arguments(L):
+    h = ctypes.c_void_p(0)
+    # codes without scales (or neither) are refused before any CUDA call
+    assert L.dirotq_prepare_layer_codes(None, 0, 0, None, 2, None, None, None, 0, 128, 64, 32, 64, None, 0, None, 0, None,
+                                        ctypes.byref(h)) == 1
+    assert not h.value
