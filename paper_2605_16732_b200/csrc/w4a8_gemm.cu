@@ -10,8 +10,8 @@
 // the operand buffer and four unpack warps expand them in place, turning every nibble into the byte 16 q (shift the nibble into the high half, flip
 // bit 7: 16 (q + 8) - 128), so the accumulator holds 16 P and the epilogue shifts it back.
 //
-// Roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 unpack,
-// warps 6..9 epilogue (one token row per thread).  TMEM: columns 0..255 the int32 tile, 256..511 the
+// Roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 unpack,
+// warps 6..13 epilogue (one token row per thread, two warps per lane quadrant).  TMEM: columns 0..255 the int32 tile, 256..511 the
 // fp32 tile of the bf16 rank-r branch (kind::f16 cannot accumulate into the integer tile); single
 // buffered, so the epilogue of a tile (one pass) is not overlapped with the next tile's MMAs.
 #include "common.h"
@@ -31,9 +31,9 @@ constexpr int BU_BYTES = BN * BKC;      // 32 KB unpacked weight codes / bf16 W~
 constexpr int BP_BYTES = BN * BKC / 2;  // 16 KB packed weight codes: TMA puts them into the UPPER HALF of the 32 KB
 constexpr int BP_OFFSET = A_BYTES + BU_BYTES - BP_BYTES;  // operand buffer and the unpack expands them in place
 constexpr int STAGE_BYTES = A_BYTES + BU_BYTES;           // 48 KB: four stages fit
-constexpr int NUM_THREADS = 320;
+constexpr int NUM_THREADS = 448;
 constexpr int NUM_UNPACK_WARPS = 4;
-constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_EPI_WARPS = 8;  // two per TMEM lane quadrant, half of the tile's columns each
 constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
 constexpr int SCALE_OFFSET = BAR_OFFSET + 256;      // two buffers of {weight scales, bias} for a tile's 256 columns
 constexpr int SCALE_BYTES = 2 * 2 * BN * 4;
@@ -234,8 +234,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 6..9)
+        // ------------------------------------------------------------ epilogue (warps 6..13)
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        const int half = (warp - (2 + NUM_UNPACK_WARPS)) >> 2;
+        constexpr int CPH = BN / 32 / 2;  // 32-column chunks per warp
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
@@ -247,15 +249,17 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             float* s_sw = reinterpret_cast<float*>(smem_gen + SCALE_OFFSET) + (tcount & 1) * 2 * BN;
             float* s_b = s_sw + BN;
             {
-                const int e = threadIdx.x - (2 + NUM_UNPACK_WARPS) * 32;  // 0..127
-                const int col = n0 + 2 * e;
-                float2 w2 = make_float2(0.f, 0.f), b2 = make_float2(0.f, 0.f);
-                if (col < p.N) {
-                    w2 = __ldg(reinterpret_cast<const float2*>(p.wscale + col));
-                    b2 = __ldg(reinterpret_cast<const float2*>(p.bias + col));
+                const int e = threadIdx.x - (2 + NUM_UNPACK_WARPS) * 32;  // 0..255; the first 128 stage two columns each
+                if (e < BN / 2) {
+                    const int col = n0 + 2 * e;
+                    float2 w2 = make_float2(0.f, 0.f), b2 = make_float2(0.f, 0.f);
+                    if (col < p.N) {
+                        w2 = __ldg(reinterpret_cast<const float2*>(p.wscale + col));
+                        b2 = __ldg(reinterpret_cast<const float2*>(p.bias + col));
+                    }
+                    *reinterpret_cast<float2*>(s_sw + 2 * e) = w2;
+                    *reinterpret_cast<float2*>(s_b + 2 * e) = b2;
                 }
-                *reinterpret_cast<float2*>(s_sw + 2 * e) = w2;
-                *reinterpret_cast<float2*>(s_b + 2 * e) = b2;
             }
             const bool mine = mbar_wait(tfull_bar, tcount & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
             uint32_t any_failed;
@@ -276,14 +280,14 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             const float sx = row < p.M ? __ldg(p.xscale + row) : 0.f;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = half * CPH; c < (half + 1) * CPH; ++c) {
                 uint32_t acc[32], lr[32];
                 tmem_ld_32x32b_x32(taddr + c * 32, acc);
                 tmem_ld_32x32b_x32(taddr + BN + c * 32, lr);
                 tmem_ld_wait();
                 tmem_ld_fence32(acc);
                 tmem_ld_fence32(lr);
-                if (c == BN / 32 - 1) {
+                if (c == (half + 1) * CPH - 1) {
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar);
