@@ -21,7 +21,8 @@
  *     records a code in the workspace status word (see dirotq_workspace_status) and returns.
  *   - A workspace must be zero-filled once before its first use: its first word is a sticky
  *     device status (0 = no wait ever expired).
- *   - Supported shapes: K % 64 == 0, N % 16 == 0, r in {16, 32, 48, ..., 128} with r < K,
+ *   - Supported shapes: K % 64 == 0, N % 16 == 0, r a multiple of 16 with r < K and r <= 4096 (the paper keeps
+ *     about a tenth of the coefficients in 16 bits: r = 112..128 for K = 1152, 304..320 for K = 3072),
  *     group in {64, 128} with K % group == 0, M >= 1.  Pointers must be 16-byte aligned.
  *   - Groups are counted from the first low-precision coefficient; the last one may be ragged.
  *     Rounding is to nearest, ties to even; scales are bf16 values; a group whose absolute

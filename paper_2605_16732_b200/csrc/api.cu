@@ -46,7 +46,7 @@ dirotq_status_t check_shape(int K, int N, int r, int G) {
     if (K <= 0 || N <= 0 || r <= 0) return DIROTQ_ERR_INVALID_ARG;
     if (G != 64 && G != 128) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
     if (K % 64 != 0 || K % G != 0 || N % 16 != 0) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
-    if (r % 16 != 0 || r > 128 || r >= K) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
+    if (r % 16 != 0 || r > 4096 || r >= K) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
     return DIROTQ_OK;
 }
 

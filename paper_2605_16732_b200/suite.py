@@ -160,7 +160,7 @@ class Case:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", default="1,2,4,5")
+    ap.add_argument("--configs", default="1,2,4,5", help="comma-separated subset of 1,2,3p,4,5")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8"])
     ap.add_argument("--ranks", default="16,32,64,128", help="ranks swept by config 4")
@@ -205,6 +205,12 @@ def main():
                           "shared_rotation_ms": res["shared_rotation"], "separate_ms": res["separate"],
                           "speedup": res["separate"] / res["shared_rotation"]}), flush=True)
         for c in cs:
+            c.close()
+    if "3p" in todo:
+        # the FLUX linears at the paper's own rank, about a tenth of K kept in 16 bits (Sec. 4.2), instead of r = 32
+        for K, N, r in [(3072, 9216, 320), (3072, 3072, 320), (3072, 12288, 320), (12288, 3072, 1232)]:
+            c = Case(4608, K, N, r, 64, synth.FLUX)
+            c.report("3p: FLUX linear, M=4608, r = 10 % of K", args.iters, p_bf16, hbm)
             c.close()
     if "4" in todo:
         for K, N in [(3072, 9216), (12288, 3072)]:

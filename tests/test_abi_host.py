@@ -42,7 +42,7 @@ def test_layer_bytes_and_shape_validation(L):
     assert floor <= n.value <= floor + 6 * 1024
     # unsupported shapes are refused
     for bad in [(1100, 1152, 32, 64), (1152, 1150, 32, 64), (1152, 1152, 24, 64), (1152, 1152, 32, 32),
-                (1152, 1152, 256, 64), (64, 64, 64, 64), (192, 64, 32, 128)]:
+                (12288, 1152, 4112, 64), (64, 64, 64, 64), (192, 64, 32, 128)]:
         assert L.dirotq_layer_bytes(*bad, ctypes.byref(n)) == 2, bad
     assert L.dirotq_layer_bytes(-1, 64, 32, 64, ctypes.byref(n)) == 1
     assert L.dirotq_layer_bytes(1152, 1152, 32, 64, None) == 1

@@ -113,6 +113,12 @@ def test_config4_rank_group_sweep(K, N, r, G):
     print(_run(18432, K, N, r, G, synth.FLUX))
 
 
+# the paper's own rank (about a tenth of K kept in 16 bits, Sec. 4.2) on two FLUX linears at M = 4608
+@pytest.mark.parametrize("K,N,r", [(3072, 9216, 320), (12288, 3072, 1232)])
+def test_flux_linears_at_ten_percent_rank(K, N, r):
+    print(_run(4608, K, N, r, 64, synth.FLUX))
+
+
 # config 5: the two single-stream shapes that the other configs do not contain
 @pytest.mark.parametrize("K,N", [(3072, 21504), (15360, 3072)])
 def test_config5_single_stream_shapes(K, N):
