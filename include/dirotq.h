@@ -170,11 +170,11 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
                                       int32_t* partials, void* workspace, size_t workspace_bytes,
                                       dirotq_stream_t stream);
 
-/* Tuning knob of the INT4 (symmetric and asymmetric layers) and NVFP4 second kernels: output columns per tile.
+/* Tuning knob of the second kernels (all four formats): output columns per tile.
  * 0 (default): chosen per call from M, N and the number of SMs (INT4: 256 columns unless 128-column tiles fill the
  * SMs so much better that they win although a narrow tile costs about 0.73 of a wide one; NVFP4 likewise with 0.6);
  * 128 or 256: forced.  Process-wide; results do not depend on it (each output element is accumulated in the same
- * order).  W4A8 layers ignore it.  Other values: DIROTQ_ERR_INVALID_ARG. */
+ * order).  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
 
 /* The second kernel of a layer is launched as a programmatic dependent launch: it may be scheduled onto SMs that

@@ -301,6 +301,12 @@ dirotq_status_t dirotq_prepare_layer_w4a8(const void* W, int w_dtype, int w_layo
         st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked128, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
         st = launch_prepare_w4a8(L, W, w_dtype, w_layout, Q, q_dtype, bias, static_cast<double*>(scratch),
                                  static_cast<cudaStream_t>(stream));
     if (st != DIROTQ_OK) {
@@ -422,8 +428,9 @@ dirotq_status_t dirotq_set_dependent_launch(int enabled) {
 }
 
 dirotq_status_t dirotq_set_gemm_tile(int columns) {
-    const dirotq_status_t st = set_w4a4_tile_columns(columns);
-    return st != DIROTQ_OK ? st : set_nvfp4_tile_columns(columns);
+    dirotq_status_t st = set_w4a4_tile_columns(columns);
+    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(columns);
+    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(columns);
 }
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,

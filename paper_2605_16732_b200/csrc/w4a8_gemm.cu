@@ -19,25 +19,33 @@
 
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 namespace dirotq {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = kGemmBN;  // 256
 constexpr int BKC = 128;     // one-byte codes per k-block (128-byte rows)
-constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BKC;       // 16 KB activation codes / bf16 x~_h chunk
-constexpr int BU_BYTES = BN * BKC;      // 32 KB unpacked weight codes / bf16 W~_h chunk
-constexpr int BP_BYTES = BN * BKC / 2;  // 16 KB packed weight codes: TMA puts them into the UPPER HALF of the 32 KB
-constexpr int BP_OFFSET = A_BYTES + BU_BYTES - BP_BYTES;  // operand buffer and the unpack expands them in place
-constexpr int STAGE_BYTES = A_BYTES + BU_BYTES;           // 48 KB: four stages fit
 constexpr int NUM_THREADS = 448;
 constexpr int NUM_UNPACK_WARPS = 4;
 constexpr int NUM_EPI_WARPS = 8;  // two per TMEM lane quadrant, half of the tile's columns each
-constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-constexpr int SCALE_OFFSET = BAR_OFFSET + 256;      // two buffers of {weight scales, bias} for a tile's 256 columns
-constexpr int SCALE_BYTES = 2 * 2 * BN * 4;
-constexpr int SMEM_BYTES = SCALE_OFFSET + SCALE_BYTES + 1024;
+
+// Shared-memory plan for tiles of BN output columns (256, or 128 where wide tiles would leave SMs idle).
+template <int BN>
+struct Plan {
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int BU_BYTES = BN * BKC;      // unpacked weight codes / bf16 W~_h chunk (32 KB at BN = 256)
+    static constexpr int BP_BYTES = BN * BKC / 2;  // packed weight codes: TMA puts them into the UPPER HALF of the
+    static constexpr int BP_OFFSET = A_BYTES + BU_BYTES - BP_BYTES;  // operand buffer and the unpack expands them in place
+    static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES;           // 48 KB x 4 or 32 KB x 6
+    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int SCALE_OFFSET = BAR_OFFSET + 256;  // two buffers of {weight scales, bias} for a tile's columns
+    static constexpr int SCALE_BYTES = 2 * 2 * BN * 4;
+    static constexpr int SMEM_BYTES = SCALE_OFFSET + SCALE_BYTES + 1024;
+    static_assert(8 * (3 * STAGES + 2) <= 192, "barriers must end below the two words at +192");
+    static_assert(SMEM_BYTES <= 232448 && STAGE_BYTES % 1024 == 0, "shared memory plan");
+};
 
 struct A8KernelParams {
     int M, N, num_kb, lr_chunks;
@@ -62,11 +70,15 @@ __device__ __forceinline__ void tmem_ld_fence32(uint32_t (&v)[32]) {
                  :: "memory");
 }
 
-template <bool kPartials>
+template <bool kPartials, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                  const A8KernelParams p) {
+    using P = Plan<BN>;
+    constexpr int STAGES = P::STAGES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES, BP_OFFSET = P::BP_OFFSET;
+    constexpr int STAGE_BYTES = P::STAGE_BYTES, BAR_OFFSET = P::BAR_OFFSET, SCALE_OFFSET = P::SCALE_OFFSET;
+    constexpr int PIECES = BN * 4 / (NUM_UNPACK_WARPS * 32);  // 16-byte pieces of the packed tile per unpack thread
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -76,8 +88,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     auto empty_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
     const uint32_t tfull_bar = bar_base + 8u * (3 * STAGES);
     const uint32_t tempty_bar = bar_base + 8u * (3 * STAGES + 1);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 128);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 132);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 196);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -210,14 +222,14 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     uint8_t* d0 = st + A_BYTES + (u >> 2) * 128 + (((2 * c) ^ sw) << 4);
                     uint8_t* d1 = st + A_BYTES + (u >> 2) * 128 + (((2 * c + 1) ^ sw) << 4);
                     // The packed codes sit in the upper half of the buffer they are expanded into: every unpack thread
-                    // takes its eight pieces into registers, the four warps meet at a named barrier, and only then is
+                    // takes its pieces into registers, the four warps meet at a named barrier, and only then is
                     // anything stored.
-                    uint4 pk[8];
+                    uint4 pk[PIECES];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) pk[j] = src[128 * j];
+                    for (int j = 0; j < PIECES; ++j) pk[j] = src[128 * j];
                     asm volatile("bar.sync 2, %0;" ::"n"(NUM_UNPACK_WARPS * 32) : "memory");  // reached by all four warps (see above)
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
+                    for (int j = 0; j < PIECES; ++j) {
                         // nibble q + 8 -> byte 16 q: into the high half, then flip bit 7 (16 (q + 8) - 128)
                         uint4 o0, o1;
                         o0.x = ((pk[j].x << 4) & 0xF0F0F0F0u) ^ 0x80808080u; o0.y = (pk[j].x & 0xF0F0F0F0u) ^ 0x80808080u;
@@ -338,9 +350,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     }
 }
 
-}  // namespace
-
-dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cudaStream_t stream) {
+template <int BN>
+static dirotq_status_t launch_w4a8_gemm_bn(const dirotq_layer* L, const A8GemmArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     CUtensorMap tmap_codes, tmap_xh;
     dirotq_status_t st;
@@ -361,16 +372,41 @@ dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cud
     const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
     const bool dbg = a.partials != nullptr;
-    auto kern = dbg ? w4a8_gemm_kernel<true> : w4a8_gemm_kernel<false>;
+    auto kern = dbg ? w4a8_gemm_kernel<true, BN> : w4a8_gemm_kernel<false, BN>;
     static bool attr_set[2] = {false, false};
     if (!attr_set[dbg]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<BN>::SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
         attr_set[dbg] = true;
     }
-    const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, true, tmap_codes, L->tmap_wpacked,
-                                          tmap_xh, L->tmap_wh, p);
+    const bool narrow = BN == 128;
+    const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
+                                          narrow ? L->tmap_wpacked128 : L->tmap_wpacked, tmap_xh,
+                                          narrow ? L->tmap_wh128 : L->tmap_wh, p);
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+static std::atomic<int> g_a8_tile_columns{0};  // 0: chosen per call; 128 / 256: forced
+
+}  // namespace
+
+dirotq_status_t set_w4a8_tile_columns(int columns) {
+    if (columns != 0 && columns != 128 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+    g_a8_tile_columns.store(columns);
+    return DIROTQ_OK;
+}
+
+dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cudaStream_t stream) {
+    // narrow tiles only where the wide ones leave SMs idle: a 128-column tile costs about NARROW_COST of a 256-column one
+    constexpr double NARROW_COST = 0.68;  // measured: 0.220 against 0.162 ms with twice as many tiles (4608 x 3072 -> 9216)
+    const int forced = g_a8_tile_columns.load();
+    const int sms = sm_count(L->device);
+    const long m_blocks = (a.M + BM - 1) / BM;
+    const long t_wide = m_blocks * ((L->geo.N + 255) / 256), t_narrow = m_blocks * ((L->geo.N + 127) / 128);
+    const bool narrow_pays =
+        NARROW_COST * static_cast<double>((t_narrow + sms - 1) / sms) < 0.98 * static_cast<double>((t_wide + sms - 1) / sms);
+    const bool narrow = forced ? forced == 128 : narrow_pays;
+    return narrow ? launch_w4a8_gemm_bn<128>(L, a, stream) : launch_w4a8_gemm_bn<256>(L, a, stream);
 }
 
 }  // namespace dirotq

@@ -130,3 +130,20 @@ def test_nvfp4_both_widths_give_the_same_bits():
     finally:
         dq.dirotq_set_gemm_tile(0)
     layer.close()
+
+
+# ------------------------------------------------------------------ W4A8 second kernel: 128- and 256-column tiles
+
+import test_gpu_w4a8
+
+
+@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+def test_w4a8_ragged_rows_and_columns(tile):
+    spec = synth.LayerSpec(K=768, N=400, r=32, G=64, model=synth.FLUX, seed=81, calib_tokens=1024)
+    print(tile, test_gpu_w4a8._run_case(spec, M=300))
+
+
+@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+def test_w4a8_pixart_projection_many_tiles(tile):
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=82)
+    print(tile, test_gpu_w4a8._run_case(spec, M=1024, check_rot=False))
