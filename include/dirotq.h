@@ -177,6 +177,12 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
  * order).  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
 
+/* Tuning knob of the first kernel (rotation): tile plan.  0 (default): chosen per call from M, K and the number of
+ * SMs; 1: 128 tokens x 128 rotated columns; 2: 128 x 256; 3: 256 x 256 (two MMAs share one tile of the rotation: a
+ * third fewer operand bytes per flop, no overlap of the epilogue; pays where a layer has many tiles per SM, e.g.
+ * K = 12288 at M = 4608).  Process-wide; results do not depend on it.  Other values: DIROTQ_ERR_INVALID_ARG. */
+DIROTQ_API dirotq_status_t dirotq_set_rotation_tile(int plan);
+
 /* The second kernel of a layer is launched as a programmatic dependent launch: it may be scheduled onto SMs that
  * the first kernel's thread blocks have left and runs its set-up there, then waits (griddepcontrol.wait) for the
  * whole first kernel before it reads anything.  Results are unaffected; the launch gap between the two kernels

@@ -29,7 +29,7 @@ EXPORTED = [
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
-    "dirotq_prepare_layer_codes", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_prepare_layer_codes", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_prepare_layer_asym.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_set_gemm_tile.argtypes = [i]
         L.dirotq_set_dependent_launch.argtypes = [i]
+        L.dirotq_set_rotation_tile.argtypes = [i]
         L.dirotq_prepare_layer_codes.argtypes = [vp, i, i, vp, i, vp, vp, vp, i, i, i, i, i, vp, sz, vp, sz, vp,
                                                  ctypes.POINTER(vp)]
         L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -360,6 +361,11 @@ def dirotq_prepare_layer_asym(W: torch.Tensor, Q: torch.Tensor, r: int, group: i
 def dirotq_set_gemm_tile(columns: int) -> None:
     """Output columns per tile of the INT4 and NVFP4 second kernels: 0 automatic, 128 or 256 forced (process-wide)."""
     _check(lib().dirotq_set_gemm_tile(int(columns)), "dirotq_set_gemm_tile")
+
+
+def dirotq_set_rotation_tile(plan: int) -> None:
+    """Tile plan of the rotation kernel: 0 automatic, 1 = 128x128, 2 = 128x256, 3 = 256x256 (process-wide)."""
+    _check(lib().dirotq_set_rotation_tile(int(plan)), "dirotq_set_rotation_tile")
 
 
 def dirotq_set_dependent_launch(enabled: bool) -> None:

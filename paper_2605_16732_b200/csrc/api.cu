@@ -422,6 +422,8 @@ static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateAr
     return launch_w4a4_gemm(layer, ga, s);
 }
 
+dirotq_status_t dirotq_set_rotation_tile(int plan) { return set_rotation_plan(plan); }
+
 dirotq_status_t dirotq_set_dependent_launch(int enabled) {
     dirotq::set_dependent_launch(enabled != 0);
     return DIROTQ_OK;

@@ -247,6 +247,7 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
 
 dirotq_status_t set_nvfp4_tile_columns(int columns);
 dirotq_status_t set_w4a8_tile_columns(int columns);
+dirotq_status_t set_rotation_plan(int plan);
 struct Nvfp4GemmArgs {
     int M;
     const uint8_t* codes;  // [M][K4/2]

@@ -25,16 +25,18 @@
 
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 namespace dirotq {
 namespace {
 
-constexpr int BM = 128;       // tokens per tile
+constexpr int BM_MMA = 128;   // token rows of one MMA; a tile has BM = 128 or 256 rows (template parameter)
 constexpr int BN_MAX = 256;   // rotated columns per tile: 256, or 128 when there are few tiles (template parameter BN)
 constexpr int BK = 64;        // bf16 elements per k-block (128-byte rows)
 constexpr int STAGES_WIDE = 4;  // 256-column tiles: 4 x 48 KB; 128-column tiles: 6 x 32 KB (same bytes in flight)
-constexpr int A_BYTES = BM * BK * 2;  // 16 KB
+constexpr int A_BYTES_128 = BM_MMA * BK * 2;  // 16 KB per 128 token rows
 constexpr int B_BYTES = BN_MAX * BK * 2;  // 32 KB (a 128-column tile uses half of it)
-constexpr int STAGE_BYTES_WIDE = A_BYTES + B_BYTES;
+constexpr int STAGE_BYTES_WIDE = A_BYTES_128 + B_BYTES;
 constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, eight epilogue warps
 constexpr int SMEM_BYTES = STAGES_WIDE * STAGE_BYTES_WIDE + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
@@ -150,7 +152,7 @@ __device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float ex_inv, 
     return sb;
 }
 
-template <int G, int FMT, int BN>
+template <int G, int FMT, int BN, int BM>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
                     const RotKernelParams p) {
@@ -158,8 +160,14 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     // The ring holds 192 KB either way; with narrow tiles it is cut into more, smaller stages: the operand stream is
     // paced by (L2 latency + MMA time of a stage) / number of stages.
-    constexpr int STAGES = BN == 256 ? STAGES_WIDE : 6;
+    // A 256 x 256 tile (two MMAs of 128 rows on one Qt tile: a third fewer operand bytes per flop) takes three 64 KB
+    // stages and all 512 tensor-memory columns, so its epilogue does not overlap the next tile's MMAs; it is used
+    // where a tile's main loop is long and there are many tiles per SM.
+    static_assert(BM == 128 || (BM == 256 && BN == 256), "256-row tiles are 256 columns wide");
+    constexpr int A_BYTES = BM * BK * 2;
+    constexpr int STAGES = BM == 256 ? 3 : (BN == 256 ? STAGES_WIDE : 6);
     constexpr int STAGE_BYTES = A_BYTES + BN * BK * 2;
+    constexpr int ACC_BUFS = BM == 256 ? 1 : 2;
     static_assert(STAGES * STAGE_BYTES == STAGES_WIDE * STAGE_BYTES_WIDE && STAGE_BYTES % 1024 == 0, "ring layout");
     const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
     // barrier map (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
@@ -237,12 +245,12 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
+            constexpr uint32_t idesc = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM_MMA, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-                const uint32_t acc = tcount & 1;
-                const uint32_t acc_ph = (tcount >> 1) & 1;
+                const uint32_t acc = tcount % ACC_BUFS;
+                const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
                 if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + acc * BN;
@@ -255,8 +263,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint64_t adesc = umma_desc_sw128(sa);
                     const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
+                    for (int k = 0; k < BK / 16; ++k) {
                         umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        if constexpr (BM == 256)  // token rows 128..255: next 16 KB of the x tile, columns 256..511 of TMEM
+                            umma_bf16(d + 256, adesc + (A_BYTES_128 >> 4) + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    }
                     umma_commit(empty_bar(s));
                 }
                 if (ok) umma_commit(tfull_bar(acc));
@@ -265,25 +276,27 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     } else {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
-        const int half = (warp - 2) >> 2;  // two warps per quadrant share a tile's column chunks
-        constexpr int CHUNKS = BN / G, CPH = CHUNKS > 1 ? CHUNKS / 2 : 1;
+        // two warps per quadrant: with 128-row tiles they share the tile's column chunks, with 256-row tiles each
+        // takes all chunks of one 128-row block
+        const int half = (warp - 2) >> 2;
+        constexpr int CHUNKS = BN / G, CPH = BM == 256 ? CHUNKS : (CHUNKS > 1 ? CHUNKS / 2 : 1);
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
             const int m0 = (tile % num_m_blocks) * BM;
             const int n_blk = tile / num_m_blocks;
             const int n0 = n_blk * BN;
-            const uint32_t acc = tcount & 1;
-            const uint32_t acc_ph = (tcount >> 1) & 1;
+            const uint32_t acc = tcount % ACC_BUFS;
+            const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
             tc_fence_after_sync();
-            const int row = m0 + q * 32 + lane;
+            const int row = m0 + (BM == 256 ? half * 128 : 0) + q * 32 + lane;
             const bool row_ok = row < p.M;
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (BM == 256 ? half * 256 : acc * BN);
 
             float tile_amax = 0.f;  // W4A8: this thread's row, this tile's columns
 #pragma unroll 1
-            for (int chunk = half * CPH; chunk < min(CHUNKS, (half + 1) * CPH); ++chunk) {
+            for (int chunk = (BM == 256 ? 0 : half * CPH); chunk < min(CHUNKS, (BM == 256 ? 1 : half + 1) * CPH); ++chunk) {
                 const int col0 = n0 + chunk * G;  // permuted column of v[0]
                 if (col0 >= p.K) break;
                 float v[G];
@@ -439,7 +452,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
-            if (n_blk == num_n_blocks - 1 && row_ok && half == 0) {
+            if (n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
                 for (int c = p.r; c < p.r_pad0; c += 8)
                     *reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + c) = make_uint4(0, 0, 0, 0);
                 if constexpr (FMT == 2) {  // behind the 3 n_g zero-point columns
@@ -458,49 +471,68 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     }
 }
 
+static std::atomic<int> g_rotation_plan{0};  // 0: chosen per call; 1: 128 x 128, 2: 128 x 256, 3: 256 x 256 tiles
+
 }  // namespace
+
+dirotq_status_t set_rotation_plan(int plan) {
+    if (plan < 0 || plan > 3) return DIROTQ_ERR_INVALID_ARG;
+    g_rotation_plan.store(plan);
+    return DIROTQ_OK;
+}
 
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
-    CUtensorMap tmap_x;
-    dirotq_status_t st = encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M,
-                                        (uint64_t)g.K * 2, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (st != DIROTQ_OK) return st;
     RotKernelParams p;
     p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
     p.xtilde = a.xtilde; p.rowmax = a.rowmax;
-    // 256-column tiles, or 128-column ones when the wide tiles would not give every SM about two of them (few, large
-    // tiles leave a nearly empty last wave: 160 tiles on 148 SMs take as long as 296)
+    // Tile plan.  128 x 256 is the default.  128 x 128 when the wide tiles would not give every SM about two of them
+    // (few, large tiles leave a nearly empty last wave: 160 tiles on 148 SMs take as long as 296).  256 x 256 (a third
+    // fewer operand bytes per flop, but the epilogue, about 11 k-blocks' worth, is not overlapped) for long main
+    // loops only: measured 0.99 -> 0.92 ms at M = 4608, K = 12288 and 1.54 -> 1.48 ms at K = 15360, but 0.125 ->
+    // 0.141 ms at M = 9216, K = 3072.
     const int sms = sm_count(L->device);
-    const int m_blocks = (a.M + BM - 1) / BM;
-    const bool narrow = m_blocks * ((g.K + 255) / 256) < 2 * sms;
-    const int bn = narrow ? 128 : 256;
-    const int num_tiles = m_blocks * ((g.K + bn - 1) / bn);
-    const int grid = num_tiles < sms ? num_tiles : sms;
+    const long mb128 = (a.M + 127) / 128, mb256 = (a.M + 255) / 256, nb256 = (g.K + 255) / 256;
+    int plan = g_rotation_plan.load();
+    if (plan == 0) {
+        const long waves128 = (mb128 * nb256 + sms - 1) / sms, waves256 = (mb256 * nb256 + sms - 1) / sms;
+        const double kb = static_cast<double>(g.K / BK);
+        const double cost256 = 1.86 + 11.0 / kb;  // a 256-row tile in units of a 128-row tile
+        if (mb128 * nb256 < 2 * sms) plan = 1;
+        else if (g.K >= 8192 && cost256 * static_cast<double>(waves256) < 0.98 * static_cast<double>(waves128)) plan = 3;
+        else plan = 2;
+    }
+    const int bm = plan == 3 ? 256 : 128, bn = plan == 1 ? 128 : 256;
+    CUtensorMap tmap_x;
+    dirotq_status_t st = encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M,
+                                        (uint64_t)g.K * 2, BK, bm, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
+    const long num_tiles = ((a.M + bm - 1) / bm) * ((g.K + bn - 1) / bn);
+    const int grid = num_tiles < sms ? static_cast<int>(num_tiles) : sms;
     const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const RotKernelParams);
-    static const KernelFn table[2][6] = {
-        {rotate_quant_kernel<64, 0, 256>, rotate_quant_kernel<128, 0, 256>, rotate_quant_kernel<64, 1, 256>,
-         rotate_quant_kernel<64, 2, 256>, rotate_quant_kernel<128, 2, 256>, rotate_quant_kernel<64, 3, 256>},
-        {rotate_quant_kernel<64, 0, 128>, rotate_quant_kernel<128, 0, 128>, rotate_quant_kernel<64, 1, 128>,
-         rotate_quant_kernel<64, 2, 128>, rotate_quant_kernel<128, 2, 128>, rotate_quant_kernel<64, 3, 128>}};
-    const KernelFn kern = table[narrow ? 1 : 0][vi];
+    static const KernelFn table[3][6] = {
+        {rotate_quant_kernel<64, 0, 128, 128>, rotate_quant_kernel<128, 0, 128, 128>, rotate_quant_kernel<64, 1, 128, 128>,
+         rotate_quant_kernel<64, 2, 128, 128>, rotate_quant_kernel<128, 2, 128, 128>, rotate_quant_kernel<64, 3, 128, 128>},
+        {rotate_quant_kernel<64, 0, 256, 128>, rotate_quant_kernel<128, 0, 256, 128>, rotate_quant_kernel<64, 1, 256, 128>,
+         rotate_quant_kernel<64, 2, 256, 128>, rotate_quant_kernel<128, 2, 256, 128>, rotate_quant_kernel<64, 3, 256, 128>},
+        {rotate_quant_kernel<64, 0, 256, 256>, rotate_quant_kernel<128, 0, 256, 256>, rotate_quant_kernel<64, 1, 256, 256>,
+         rotate_quant_kernel<64, 2, 256, 256>, rotate_quant_kernel<128, 2, 256, 256>, rotate_quant_kernel<64, 3, 256, 256>}};
+    const KernelFn kern = table[plan - 1][vi];
     // a dependent launch needs a kernel as the previous operation of the stream: the W4A8 path puts a memset there
     const bool dependent = g.fmt != 3;
-    static bool attr_set[2][6] = {};
-    if (!attr_set[narrow ? 1 : 0][vi]) {
+    static bool attr_set[3][6] = {};
+    if (!attr_set[plan - 1][vi]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
-        attr_set[narrow ? 1 : 0][vi] = true;
+        attr_set[plan - 1][vi] = true;
     }
-    if (narrow) {
-        return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, L->tmap_qt128, p) == cudaSuccess
-                   ? DIROTQ_OK : DIROTQ_ERR_CUDA;
-    }
-    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, L->tmap_qt, p) == cudaSuccess
-               ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, plan == 1 ? L->tmap_qt128 : L->tmap_qt,
+                         p) == cudaSuccess
+               ? DIROTQ_OK
+               : DIROTQ_ERR_CUDA;
 }
 
 }  // namespace dirotq
