@@ -210,6 +210,20 @@ DIROTQ_API dirotq_status_t dirotq_prepare_layer_codes(const void* W, int w_dtype
                                                       size_t blob_bytes, void* scratch, size_t scratch_bytes,
                                                       dirotq_stream_t stream, dirotq_layer_t** layer_out);
 
+/* ---- layers that share one rotation (paper Sec. 4.2: the rotation belongs to a layer's INPUT, so linears that read
+ * the same activations, e.g. the q, k and v projections of a block, are rotated by the same Q) ----
+ *
+ * A sibling layer is prepared like dirotq_prepare_layer (asym == 0) or dirotq_prepare_layer_asym (asym != 0) with the
+ * SAME Q, r and group as the layer that owns the rotation, but its blob holds no copy of Q (K*K*2 bytes less).  It is
+ * used through dirotq_w4a4_gemm on a workspace filled by dirotq_rotate_quantize of the owning layer; dirotq_linear,
+ * dirotq_linear_host, dirotq_linear_noalloc, dirotq_rotate_quantize and the q_bf16 output of dirotq_layer_export
+ * refuse it with DIROTQ_ERR_INVALID_ARG.  Q is still an argument: the weights are folded with it. */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes_sibling(int K, int N, int r, int group, int asym, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_sibling(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                                        const void* bias, int asym, int K, int N, int r, int group,
+                                                        void* blob, size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                                        dirotq_stream_t stream, dirotq_layer_t** layer_out);
+
 /* ---- asymmetric activation codes (paper Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the 4-bit INT setting
  * quantizes the activations asymmetrically) ---- */
 

@@ -29,7 +29,7 @@ EXPORTED = [
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
-    "dirotq_prepare_layer_codes", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_prepare_layer_codes", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.dirotq_workspace_export_w4a8.argtypes = [vp, i, vp, vp, vp, vp, vp]
         L.dirotq_layer_bytes_asym.argtypes = [i, i, i, i, psz]
         L.dirotq_prepare_layer_asym.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
+        L.dirotq_layer_bytes_sibling.argtypes = [i, i, i, i, i, ctypes.POINTER(sz)]
+        L.dirotq_prepare_layer_sibling.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_set_gemm_tile.argtypes = [i]
         L.dirotq_set_dependent_launch.argtypes = [i]
         L.dirotq_set_rotation_tile.argtypes = [i]
@@ -356,6 +358,32 @@ def dirotq_prepare_layer_asym(W: torch.Tensor, Q: torch.Tensor, r: int, group: i
     _check(st, "dirotq_prepare_layer_asym")
     torch.cuda.current_stream().synchronize()
     return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym")
+
+
+def dirotq_layer_bytes_sibling(K: int, N: int, r: int, group: int, asym: bool = False) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().dirotq_layer_bytes_sibling(K, N, r, group, int(asym), ctypes.byref(out)), "dirotq_layer_bytes_sibling")
+    return out.value
+
+
+def dirotq_prepare_layer_sibling(W: torch.Tensor, Q: torch.Tensor, r: int, group: int, bias: torch.Tensor | None = None,
+                                 asym: bool = False, w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """A layer without its own copy of the rotation: used through dirotq_w4a4_gemm on a sibling's rotated workspace."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    blob = _alloc_bytes(dirotq_layer_bytes_sibling(K, N, r, group, asym), W.device)
+    scratch_bytes = dirotq_prepare_scratch_bytes(K, N)
+    scratch = _alloc_bytes(scratch_bytes, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_sibling(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), int(asym), K, N, r, group,
+                                            blob.data_ptr(), blob.numel(), scratch.data_ptr(), scratch_bytes, _stream(stream),
+                                            ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_sibling")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym" if asym else "int4")
 
 
 def dirotq_set_gemm_tile(columns: int) -> None:

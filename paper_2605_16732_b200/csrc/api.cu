@@ -151,7 +151,7 @@ dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_
     return DIROTQ_OK;
 }
 
-static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
                                     const void* bias, const int8_t* wcodes, const void* wscales, int K, int N, int r,
                                     int group, void* blob, size_t blob_bytes,
                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
@@ -167,6 +167,7 @@ static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w
     if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
     Geometry g = make_geometry(K, N, r, group);
     if (asym) make_asym(g);
+    g.no_rot = sibling ? 1 : 0;
     const BlobLayout lay = make_blob_layout(g);
     if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
     if (scratch_bytes < static_cast<size_t>(K) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
@@ -183,11 +184,14 @@ static dirotq_status_t prepare_int4(bool asym, const void* W, int w_dtype, int w
     L->lay = lay;
     L->blob = static_cast<char*>(blob);
 
-    st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
-                        (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (st == DIROTQ_OK)
-        st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
-                            (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    st = DIROTQ_OK;
+    if (!sibling) {
+        st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                            (uint64_t)K * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (st == DIROTQ_OK)
+            st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K,
+                                (uint64_t)K, (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    }
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -221,7 +225,7 @@ dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, c
                                      const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
                                      void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
                                      dirotq_layer_t** layer_out) {
-    return prepare_int4(false, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob, blob_bytes,
+    return prepare_int4(false, false, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob, blob_bytes,
                         scratch, scratch_bytes, stream, layer_out);
 }
 
@@ -230,7 +234,7 @@ dirotq_status_t dirotq_prepare_layer_codes(const void* W, int w_dtype, int w_lay
                                            int N, int r, int group, void* blob, size_t blob_bytes, void* scratch,
                                            size_t scratch_bytes, dirotq_stream_t stream, dirotq_layer_t** layer_out) {
     if (!wcodes || !wscales) return DIROTQ_ERR_INVALID_ARG;
-    return prepare_int4(asym != 0, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, K, N, r, group, blob,
+    return prepare_int4(asym != 0, false, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, K, N, r, group, blob,
                         blob_bytes, scratch, scratch_bytes, stream, layer_out);
 }
 
@@ -248,8 +252,27 @@ dirotq_status_t dirotq_prepare_layer_asym(const void* W, int w_dtype, int w_layo
                                           const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
                                           void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
                                           dirotq_layer_t** layer_out) {
-    return prepare_int4(true, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob, blob_bytes,
+    return prepare_int4(true, false, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob, blob_bytes,
                         scratch, scratch_bytes, stream, layer_out);
+}
+
+dirotq_status_t dirotq_layer_bytes_sibling(int K, int N, int r, int group, int asym, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, group);
+    if (st != DIROTQ_OK) return st;
+    Geometry g = make_geometry(K, N, r, group);
+    if (asym) make_asym(g);
+    g.no_rot = 1;
+    *bytes = make_blob_layout(g).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_sibling(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                             const void* bias, int asym, int K, int N, int r, int group, void* blob,
+                                             size_t blob_bytes, void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                             dirotq_layer_t** layer_out) {
+    return prepare_int4(asym != 0, true, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob,
+                        blob_bytes, scratch, scratch_bytes, stream, layer_out);
 }
 
 dirotq_status_t dirotq_layer_bytes_w4a8(int K, int N, int r, size_t* bytes) {
@@ -355,8 +378,10 @@ dirotq_status_t dirotq_layer_info(const dirotq_layer_t* layer, int* K, int* N, i
     return DIROTQ_OK;
 }
 
-static dirotq_status_t check_call(const dirotq_layer_t* layer, int M, const void* workspace, size_t workspace_bytes) {
+static dirotq_status_t check_call(const dirotq_layer_t* layer, int M, const void* workspace, size_t workspace_bytes,
+                                  bool rotates = true) {
     if (!valid_layer(layer) || !workspace || M < 1) return DIROTQ_ERR_INVALID_ARG;
+    if (rotates && layer->geo.no_rot) return DIROTQ_ERR_INVALID_ARG;  // a sibling layer holds no rotation
     if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
     if (workspace_bytes < workspace_need(layer, M)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
     return DIROTQ_OK;
@@ -458,7 +483,7 @@ dirotq_status_t dirotq_linear(const void* x, int M, const dirotq_layer_t* layer,
 
 dirotq_status_t dirotq_w4a4_gemm(int M, const dirotq_layer_t* layer, const void* workspace, size_t workspace_bytes,
                                  void* y, dirotq_stream_t stream) {
-    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes, false);
     if (st != DIROTQ_OK) return st;
     if (!y || !aligned16(y)) return DIROTQ_ERR_INVALID_ARG;
     char* ws = const_cast<char*>(static_cast<const char*>(workspace));
@@ -581,7 +606,7 @@ dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, cons
 
 dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const dirotq_layer_t* layer, int32_t* partials,
                                       void* workspace, size_t workspace_bytes, dirotq_stream_t stream) {
-    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes);
+    dirotq_status_t st = check_call(layer, M, workspace, workspace_bytes, false);
     if (st != DIROTQ_OK) return st;
     if (layer->geo.fmt == 1) return DIROTQ_ERR_INVALID_ARG;
     if (layer->geo.fmt == 3) {  // one sum per output: partials [M][N]; the caller's codes are read in place
@@ -612,6 +637,7 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
 dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16, void* wh_bf16,
                                     void* q_bf16, dirotq_stream_t stream) {
     if (!valid_layer(layer) || layer->geo.fmt == 1) return DIROTQ_ERR_INVALID_ARG;
+    if (q_bf16 && layer->geo.no_rot) return DIROTQ_ERR_INVALID_ARG;  // a sibling layer holds no rotation
     return launch_layer_export(layer, wcodes, static_cast<uint16_t*>(wscales_bf16), static_cast<uint16_t*>(wh_bf16),
                                static_cast<uint16_t*>(q_bf16), static_cast<cudaStream_t>(stream));
 }

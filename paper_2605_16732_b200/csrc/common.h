@@ -32,6 +32,7 @@ struct Geometry {
     int K4;      // K_l rounded up to 64 (<= K): width of the packed E2M1 rows
     int nkb64;   // K4 / 64: scale-factor atoms (128 rows x 4 scales) per row block
     int nkb64p;  // nkb64 rounded up to 4: one TMA k-block = 256 elements = 4 atoms
+    int no_rot;  // 1: the blob holds no rotation (a layer that only consumes a workspace rotated through a sibling layer)
 };
 
 inline Geometry make_geometry(int K, int N, int r, int G) {
@@ -46,6 +47,7 @@ inline Geometry make_geometry(int K, int N, int r, int G) {
     g.K4 = (g.K_l + 63) / 64 * 64;
     g.nkb64 = g.K4 / 64;
     g.nkb64p = (g.nkb64 + 3) / 4 * 4;
+    g.no_rot = 0;
     return g;
 }
 
@@ -76,7 +78,7 @@ struct BlobLayout {
 inline BlobLayout make_blob_layout(const Geometry& g) {
     BlobLayout b;
     size_t o = 0;
-    b.off_qt = o;      o = align_up(o + (size_t)g.K * g.K * 2);
+    b.off_qt = o;      o = align_up(o + (g.no_rot ? 0 : (size_t)g.K * g.K * 2));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K_lp / 2));
     b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * g.N * 4);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);

@@ -49,7 +49,7 @@ using namespace dirotq;
 
 extern "C" dirotq_status_t dirotq_linear_noalloc(const void* x, int M, const dirotq_layer_t* layer, void* y,
                                                  int* device_status, dirotq_stream_t stream) {
-    if (layer == nullptr || layer->magic != kLayerMagic || x == nullptr || y == nullptr || M < 1)
+    if (layer == nullptr || layer->magic != kLayerMagic || x == nullptr || y == nullptr || M < 1 || layer->geo.no_rot)
         return DIROTQ_ERR_INVALID_ARG;
     size_t need = 0;
     dirotq_status_t st = dirotq_workspace_bytes(layer, M, &need);

@@ -550,9 +550,11 @@ dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype
             scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked),
             reinterpret_cast<float*>(blob + L->lay.off_wscale), reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
-    rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
-        Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
-    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    if (!g.no_rot) {
+        rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
+            Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
+        if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    }
     bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
                                                        reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);
     return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;

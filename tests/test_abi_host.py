@@ -85,3 +85,13 @@ def test_prepare_from_codes_rejects_null_arguments(L):
     assert L.dirotq_prepare_layer_codes(None, 0, 0, None, 2, None, None, None, 0, 128, 64, 32, 64, None, 0, None, 0, None,
                                         ctypes.byref(h)) == 1
     assert not h.value
+
+
+def test_sibling_layer_is_smaller_by_the_rotation(L):
+    full, sib = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    for K, N, r, G, asym in [(1152, 1152, 32, 64, 0), (3072, 9216, 320, 128, 0), (1152, 4608, 112, 64, 1)]:
+        fn = L.dirotq_layer_bytes_asym if asym else L.dirotq_layer_bytes
+        assert fn(K, N, r, G, ctypes.byref(full)) == 0
+        assert L.dirotq_layer_bytes_sibling(K, N, r, G, asym, ctypes.byref(sib)) == 0
+        assert 0 <= full.value - sib.value - 2 * K * K <= 1024          # the bf16 rotation, up to the section alignment
+    assert L.dirotq_layer_bytes_sibling(1100, 1152, 32, 64, 0, ctypes.byref(sib)) == 2

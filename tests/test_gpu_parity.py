@@ -346,3 +346,40 @@ def test_dependent_launch_on_and_off_give_the_same_bits():
         dq.dirotq_set_dependent_launch(True)
     for l in layers:
         l.close()
+
+
+def test_sibling_layers_without_their_own_rotation():
+    # q / k / v-style group: one layer owns the rotation, the others are prepared without a copy of it and consume
+    # the owner's rotated workspace; they must give the bits of fully prepared layers
+    spec = synth.LayerSpec(K=512, N=384, r=32, G=64, model=synth.PIXART, seed=95, calib_tokens=1024)
+    M, dev = 333, "cuda"
+    base = synth.make_layer_inputs(spec, M, with_bias=True)
+    Q = torch.from_numpy(base["Q"]).to(dev)
+    x = bits_to_bf16_tensor(base["x"])
+    rng = np.random.default_rng(5)
+    Ws = [torch.from_numpy((rng.standard_normal((spec.K, spec.N)) * 0.02).astype(np.float32)).to(dev) for _ in range(3)]
+    bias = bits_to_bf16_tensor(base["bias"])
+    for asym in (False, True):
+        prep = dq.dirotq_prepare_layer_asym if asym else dq.dirotq_prepare_layer
+        full = [prep(W, Q, spec.r, spec.G, bias=bias) for W in Ws]
+        sibs = [dq.dirotq_prepare_layer_sibling(W, Q, spec.r, spec.G, bias=bias, asym=asym) for W in Ws[1:]]
+        assert all(s.blob.numel() <= f.blob.numel() - 2 * spec.K * spec.K for s, f in zip(sibs, full[1:]))
+        ws = dq.alloc_workspace(full[0], M)
+        dq.dirotq_rotate_quantize(x, full[0], ws)
+        for i, sib in enumerate(sibs, start=1):
+            y_ref = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
+            dq.dirotq_linear(x, full[i], y_ref, dq.alloc_workspace(full[i], M))
+            y = torch.zeros_like(y_ref)
+            dq.dirotq_w4a4_gemm(M, sib, ws, y)
+            torch.cuda.synchronize()
+            assert dq.dirotq_workspace_status(ws) == 0
+            assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16))
+            # what a sibling cannot do is refused before any launch
+            with pytest.raises(dq.DirotqError):
+                dq.dirotq_linear(x, sib, y, ws)
+            with pytest.raises(dq.DirotqError):
+                dq.dirotq_rotate_quantize(x, sib, ws)
+            with pytest.raises(dq.DirotqError):
+                dq.dirotq_layer_export(sib)
+        for l in full + sibs:
+            l.close()
