@@ -33,13 +33,17 @@ def _one(rng, big):
         G = 64
     tile = rng.choice([0, 0, 128, 256])
     pdl = rng.choice([True, True, False])
+    plan = rng.choice([0, 0, 1, 2, 3])     # tile plan of the rotation kernel
+    if not big and rng.random() < 0.3:
+        r = 16 * rng.randint(1, max(1, K // 32))      # up to half of K in 16 bits
     bias = rng.random() < 0.7
     model = rng.choice([synth.PIXART, synth.FLUX])
     spec = synth.LayerSpec(K=K, N=N, r=r, G=G if fmt in ("int4", "asym") else 64, model=model, seed=rng.randint(1, 10 ** 6),
                            calib_tokens=max(512, 2 * K))
-    desc = dict(fmt=fmt, M=M, K=K, N=N, r=r, G=spec.G, tile=tile, pdl=pdl, bias=bias)
+    desc = dict(fmt=fmt, M=M, K=K, N=N, r=r, G=spec.G, tile=tile, pdl=pdl, bias=bias, plan=plan)
     dq.dirotq_set_gemm_tile(tile)
     dq.dirotq_set_dependent_launch(pdl)
+    dq.dirotq_set_rotation_tile(plan)
     try:
         if fmt == "int4":
             test_gpu_parity._run_case(spec, M=M, with_bias=bias, check_rot=not big)
@@ -54,6 +58,7 @@ def _one(rng, big):
     finally:
         dq.dirotq_set_gemm_tile(0)
         dq.dirotq_set_dependent_launch(True)
+        dq.dirotq_set_rotation_tile(0)
 
 
 def test_random_small_shapes():
