@@ -158,13 +158,33 @@ class Case:
         self.layer.close()
 
 
+def memory_report():
+    """Bytes of a prepared layer (`dirotq_layer_bytes*`, no GPU needed) against its bf16 weights, for the layer shapes of
+    the configurations, at the benchmark's rank and at about a tenth of K."""
+    shapes = {"pixart qkv/o": (1152, 1152), "pixart fc1": (1152, 4608), "pixart fc2": (4608, 1152),
+              "flux qkv": (3072, 9216), "flux out": (3072, 3072), "flux mlp_up": (3072, 12288), "flux mlp_down": (12288, 3072),
+              "flux single_in": (3072, 21504), "flux single_out": (15360, 3072)}
+    for name, (K, N) in shapes.items():
+        for r in (32, int(round(0.1 * K / 16)) * 16):
+            full = dq.dirotq_layer_bytes(K, N, r, 64)
+            sib = dq.dirotq_layer_bytes_sibling(K, N, r, 64)
+            print(json.dumps({"layer": name, "K": K, "N": N, "r": r, "group": 64, "bf16_weight_bytes": 2 * K * N,
+                              "layer_bytes": full, "layer_bytes_without_rotation": sib,
+                              "x_smaller_than_bf16": 2.0 * K * N / full,
+                              "x_smaller_than_bf16_without_rotation": 2.0 * K * N / sib}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--memory", action="store_true", help="print the layer sizes (no GPU needed) and exit")
     ap.add_argument("--configs", default="1,2,4,5", help="comma-separated subset of 1,2,3p,4,5")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8"])
     ap.add_argument("--ranks", default="16,32,64,128", help="ranks swept by config 4")
     args = ap.parse_args()
+    if args.memory:
+        memory_report()
+        return
     global FMT
     FMT = args.fmt
     todo = set(args.configs.split(","))

@@ -95,3 +95,14 @@ def test_sibling_layer_is_smaller_by_the_rotation(L):
         assert L.dirotq_layer_bytes_sibling(K, N, r, G, asym, ctypes.byref(sib)) == 0
         assert 0 <= full.value - sib.value - 2 * K * K <= 1024          # the bf16 rotation, up to the section alignment
     assert L.dirotq_layer_bytes_sibling(1100, 1152, 32, 64, 0, ctypes.byref(sib)) == 2
+
+
+def test_memory_report_runs_without_a_gpu(capsys):
+    import json
+    from paper_2605_16732_b200 import suite
+    suite.memory_report()
+    rows = [json.loads(l) for l in capsys.readouterr().out.splitlines()]
+    assert len(rows) == 18
+    for row in rows:
+        assert row["layer_bytes"] - row["layer_bytes_without_rotation"] >= 2 * row["K"] ** 2
+        assert 2.5 < row["x_smaller_than_bf16_without_rotation"] < 3.6
