@@ -499,9 +499,12 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     if (plan == 0) {
         const long waves128 = (mb128 * nb256 + sms - 1) / sms, waves256 = (mb256 * nb256 + sms - 1) / sms;
         const double kb = static_cast<double>(g.K / BK);
-        const double cost256 = 1.86 + 11.0 / kb;  // a 256-row tile in units of a 128-row tile
+        // a 256-row tile in units of a 128-row tile; once x no longer fits the L2 beside the rotation the 128-row plan
+        // re-reads it from HBM and the ratio falls to 1.9 (measured at M = 18432, K = 3072: 0.304 -> 0.288 ms)
+        const bool x_exceeds_l2 = static_cast<double>(a.M) * g.K * 2.0 > 96e6;
+        const double cost256 = x_exceeds_l2 ? 1.9 : 1.86 + 11.0 / kb;
         if (mb128 * nb256 < 2 * sms) plan = 1;
-        else if (g.K >= 8192 && cost256 * static_cast<double>(waves256) < 0.98 * static_cast<double>(waves128)) plan = 3;
+        else if ((g.K >= 8192 || x_exceeds_l2) && cost256 * static_cast<double>(waves256) < 0.98 * static_cast<double>(waves128)) plan = 3;
         else plan = 2;
     }
     const int bm = plan == 3 ? 256 : 128, bn = plan == 1 ? 128 : 256;
