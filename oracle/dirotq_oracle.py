@@ -214,6 +214,69 @@ def linear_deployed(x_bits, layer, bias=None, want_t: bool = True):
 
 
 # ---------------------------------------------------------------------------------------------
+# Projection form with a structured rotation: NOT the paper's Eq. 5 but the cheaper formulation its remarks on the cost
+# of the online rotation point towards (Sec. 4.2 keeps only the top-r directions in 16 bits; App. E notes that the
+# rotation's cost and memory grow with the layer width).  Only U_h is applied densely:
+#     x~_h = bf16(x U_hb),   d = x - x~_h U_hb^T,   x~_l = d H,   y = x~_h (U_hb^T W) + Q4(x~_l) Q4(H^T W) + bias
+# with U_hb = bf16(U_h) and H block-diagonal, one orthonormal Hadamard block per quantization group.  Because d is the
+# residual of the ROUNDED projection, x = x~_h U_hb^T + d holds exactly, so the layer equals x W when nothing is
+# quantized, for any U_h.  No CUDA path computes this form yet; these functions are the reference it will be held to.
+
+def hadamard(n: int) -> np.ndarray:
+    """Orthonormal Sylvester-Hadamard matrix of order n (a power of two): entries +-1/sqrt(n), symmetric."""
+    assert n >= 1 and n & (n - 1) == 0
+    H = np.ones((1, 1), dtype=np.float64)
+    while H.shape[0] < n:
+        H = np.block([[H, H], [H, -H]])
+    return H / np.sqrt(float(n))
+
+
+def block_hadamard_rows(A, G: int) -> np.ndarray:
+    """H^T A for the block-diagonal H with blocks of order G: every group of G consecutive ROWS of A is transformed."""
+    A = _c(A, np.float64)
+    K = A.shape[0]
+    assert K % G == 0
+    H = hadamard(G)
+    return (H.T @ A.reshape(K // G, G, -1)).reshape(A.shape)
+
+
+def block_hadamard_cols(A, G: int) -> np.ndarray:
+    """A H: every group of G consecutive COLUMNS of A is transformed."""
+    A = _c(A, np.float64)
+    return block_hadamard_rows(np.ascontiguousarray(A.T), G).T.copy()
+
+
+def prepare_layer_ph(W, Uh, G: int):
+    """Offline part of the projection form.  W [K, N]; Uh [K, r] (the leading principal directions, unrounded)."""
+    W = _c(W, np.float64)
+    Uh = _c(Uh, np.float64)
+    K, N = W.shape
+    r = Uh.shape[1]
+    assert Uh.shape[0] == K and K % G == 0
+    Uhb = bf16_round(Uh)                                        # the projection that runs online
+    Wt = np.concatenate([matmul(np.ascontiguousarray(bf16_to_f64(Uhb).T), W), block_hadamard_rows(W, G)], axis=0)
+    out = prepare_weights(Wt, r, G, want_t=True)               # rows < r -> bf16, the K transformed rows -> INT4 groups
+    out["Uhb"] = Uhb
+    out["r"], out["G"], out["K"] = r, G, K
+    return out
+
+
+def linear_deployed_ph(x_bits, layer, bias=None, want_t: bool = True):
+    """Online part of the projection form on bf16 inputs; every intermediate is returned."""
+    r, G, K = layer["r"], layer["G"], layer["K"]
+    x = bf16_to_f64(_c(x_bits, np.uint16))
+    Uhb = bf16_to_f64(layer["Uhb"])
+    xh_bits = bf16_round(matmul(x, Uhb))
+    d = x - matmul(bf16_to_f64(xh_bits), np.ascontiguousarray(Uhb.T))
+    xl = block_hadamard_cols(d, G)
+    sq = split_quantize(np.concatenate([np.zeros((x.shape[0], 0)), xl], axis=1), 0, G, want_t=want_t)
+    P = int_gemm(sq["codes"], layer["wcodes"], G)
+    y64, yb = combine(P, sq["scales"], layer["wscales"], xh_bits, layer["Wh"], bias)
+    return {"xh": xh_bits, "d": d, "xl": xl, "codes": sq["codes"], "scales": sq["scales"], "t": sq["t"], "P": P,
+            "y64": y64, "y": yb}
+
+
+# ---------------------------------------------------------------------------------------------
 # GPTQ rounding of the residual weight (Sec. 4.1: the rounding minimises ||X W - X W^||_F^2 rather than the
 # layer-wise surrogate; App. F.1: damping 0.01, block size 128).  The steps are those of the published GPTQ
 # algorithm, on the residual weight W~_l whose rows are the rotated low columns: the Hessian is

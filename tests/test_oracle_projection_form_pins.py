@@ -1,0 +1,94 @@
+"""Pins of the oracle's projection form (only U_h applied densely, the residual rotated by a block Hadamard): the
+reference for a cheaper first stage that no CUDA kernel computes yet.  What the construction fixes: the Hadamard blocks
+are orthonormal; the decomposition x = x~_h U_hb^T + d is exact for ANY U_h because d is the residual of the rounded
+projection, so without quantization the layer is x W; the integer path equals dequantize-then-multiply; with no
+projection it reduces to group-wise rounding of the Hadamard-rotated operands; and on activations with outlier
+directions the projection is what keeps the error down."""
+import numpy as np
+
+from oracle import dirotq_oracle as orc
+from paper_2605_16732_b200 import synth
+
+
+def _bf(bits):
+    return orc.bf16_to_f64(np.asarray(bits, dtype=np.uint16))
+
+
+def test_hadamard_blocks_are_orthonormal_and_the_two_transforms_cancel():
+    for n in (1, 2, 8, 64, 128):
+        H = orc.hadamard(n)
+        assert np.allclose(H @ H.T, np.eye(n), atol=1e-12) and np.array_equal(H, H.T)
+        assert set(np.unique(np.round(np.abs(H) * np.sqrt(n), 12))) == {1.0}
+    rng = np.random.default_rng(0)
+    A, B = rng.standard_normal((7, 192)), rng.standard_normal((192, 5))
+    assert np.allclose(orc.block_hadamard_cols(A, 64) @ orc.block_hadamard_rows(B, 64), A @ B, atol=1e-10)
+    # a constant group has all its energy in the block's first coefficient
+    c = orc.block_hadamard_cols(np.full((1, 64), 3.0), 64)
+    assert np.isclose(c[0, 0], 3.0 * 8.0) and np.allclose(c[0, 1:], 0.0, atol=1e-12)
+
+
+def test_decomposition_is_exact_for_any_projection():
+    rng = np.random.default_rng(1)
+    K, N, r, G, M = 256, 48, 32, 64, 33
+    W = rng.standard_normal((K, N)) * 0.02
+    x_bits = orc.bf16_round(rng.standard_normal((M, K)) * rng.choice([0.1, 1.0, 20.0], size=(1, K)))
+    x = _bf(x_bits)
+    for Uh in (np.linalg.qr(rng.standard_normal((K, r)))[0], rng.standard_normal((K, r)) * 0.3):   # orthonormal or not
+        lay = orc.prepare_layer_ph(W, Uh, G)
+        out = orc.linear_deployed_ph(x_bits, lay)
+        Uhb = _bf(lay["Uhb"])
+        assert np.allclose(_bf(out["xh"]) @ Uhb.T + out["d"], x, rtol=0, atol=1e-12 * np.abs(x).max())
+        # unquantized: x~_h (U_hb^T W) + (d H)(H^T W) = x W
+        ideal = _bf(out["xh"]) @ (Uhb.T @ W) + out["xl"] @ orc.block_hadamard_rows(W, G)
+        assert np.allclose(ideal, x @ W, rtol=1e-10, atol=1e-10)
+        # the high rows of the prepared weight are bf16(U_hb^T W), the low rows the K transformed rows
+        assert np.array_equal(lay["Wh"], orc.bf16_round(Uhb.T @ W))
+        assert lay["wcodes"].shape == (K, N) and out["codes"].shape == (M, K)
+
+
+def test_integer_path_equals_dequantize_then_multiply():
+    spec = synth.LayerSpec(K=256, N=80, r=32, G=64, model=synth.PIXART, seed=3, calib_tokens=1024)
+    inp = synth.make_layer_inputs(spec, 24, with_bias=True)
+    Q = np.asarray(inp["Q"], dtype=np.float64)
+    lay = orc.prepare_layer_ph(inp["W"], Q[:, :spec.r], spec.G)
+    out = orc.linear_deployed_ph(inp["x"], lay, bias=inp["bias"])
+    sx = np.repeat(_bf(out["scales"]), spec.G, axis=1)
+    sw = np.repeat(_bf(lay["wscales"]), spec.G, axis=0)
+    ref = (sx * out["codes"]) @ (sw * lay["wcodes"]) + _bf(out["xh"]) @ _bf(lay["Wh"]) + _bf(inp["bias"])[None, :]
+    assert np.allclose(out["y64"], ref, rtol=1e-12, atol=1e-12)
+    assert np.array_equal(out["y"], orc.bf16_round(out["y64"]))
+
+
+def test_without_projection_it_is_group_rounding_of_the_hadamard_rotated_operands():
+    rng = np.random.default_rng(4)
+    K, N, G, M = 128, 16, 64, 9
+    W = rng.standard_normal((K, N)) * 0.02
+    x_bits = orc.bf16_round(rng.standard_normal((M, K)))
+    lay = orc.prepare_layer_ph(W, np.zeros((K, 16)), G)          # sixteen null directions: x~_h = 0, d = x
+    out = orc.linear_deployed_ph(x_bits, lay)
+    assert not out["xh"].any() and np.array_equal(out["d"], _bf(x_bits))
+    xr = orc.block_hadamard_cols(_bf(x_bits), G)
+    for m in range(M):
+        for g in range(K // G):
+            sb, codes, _ = orc.quantize_group(xr[m, g * G:(g + 1) * G])
+            assert sb == out["scales"][m, g] and np.array_equal(codes, out["codes"][m, g * G:(g + 1) * G])
+    rtn = orc.prepare_weights(orc.block_hadamard_rows(W, G), 0, G)
+    assert np.array_equal(lay["wcodes"], rtn["wcodes"]) and np.array_equal(lay["wscales"], rtn["wscales"])
+
+
+def test_error_matches_the_dense_rotation_and_the_projection_is_what_removes_the_outliers():
+    spec = synth.LayerSpec(K=512, N=96, r=32, G=64, model=synth.PIXART, seed=5, calib_tokens=2048)
+    inp = synth.make_layer_inputs(spec, 160, with_bias=False)
+    Q = np.asarray(inp["Q"], dtype=np.float64)
+    x = _bf(inp["x"])
+    ideal = x @ np.asarray(inp["W"], dtype=np.float64)
+
+    def err(y):
+        return float(np.sqrt(np.mean((y - ideal) ** 2) / np.mean(ideal ** 2)))
+
+    e_paper = err(orc.linear_deployed(inp["x"], orc.prepare_layer(inp["W"], inp["Q"], spec.r, spec.G))["y64"])
+    e_proj = err(orc.linear_deployed_ph(inp["x"], orc.prepare_layer_ph(inp["W"], Q[:, :spec.r], spec.G))["y64"])
+    e_none = err(orc.linear_deployed_ph(inp["x"], orc.prepare_layer_ph(inp["W"], np.zeros((spec.K, spec.r)), spec.G))["y64"])
+    print(e_paper, e_proj, e_none)
+    assert 0.8 < e_proj / e_paper < 1.25          # same error as the paper's dense rotation on these activations
+    assert e_none > 3.0 * e_proj                  # a Hadamard alone does not remove the planted outlier directions
