@@ -224,6 +224,29 @@ DIROTQ_API dirotq_status_t dirotq_prepare_layer_sibling(const void* W, int w_dty
                                                         void* blob, size_t blob_bytes, void* scratch, size_t scratch_bytes,
                                                         dirotq_stream_t stream, dirotq_layer_t** layer_out);
 
+/* ---- projection form: a cheaper first stage (NOT the paper's Eq. 5; the formulation its remarks on the cost of the
+ * online rotation point towards: paper Sec. 4.2 keeps only the leading r directions in 16 bits, App. E notes that the
+ * rotation's cost and memory grow with the layer width) ----
+ *
+ *     x~_h = bf16(x U_hb)           U_hb = bf16(U_h), U_h [K,r] the leading principal directions
+ *     d    = x - x~_h U_hb^T        residual of the ROUNDED projection, so x = x~_h U_hb^T + d exactly
+ *     x~_l = d H                    H block-diagonal: one orthonormal Hadamard block per quantization group
+ *     y    = bf16( x~_h (U_hb^T W) + Q4(x~_l) Q4(H^T W) + bias )      Q4 as in dirotq_prepare_layer, over all K columns
+ *
+ * 4 M K r flops instead of 2 M K^2 in the first stage, and no K x K matrix in the layer.  Uh: DEVICE, row-major [K,r],
+ * uh_dtype DIROTQ_DTYPE_F64 or _F32; scratch: dirotq_prepare_scratch_bytes_ph bytes.  Such a layer is accepted by
+ * dirotq_workspace_bytes, dirotq_linear, dirotq_linear_host, dirotq_rotate_quantize (xrot_f32 must be NULL),
+ * dirotq_w4a4_gemm, dirotq_workspace_export (codes [M,K]), dirotq_int_gemm_debug, dirotq_layer_export (wcodes [K,N],
+ * q_bf16 must be NULL), dirotq_layer_info (K_lp = K, n_g = K / group) and dirotq_layer_destroy. */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes_ph(int K, int N, int r, int group, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_scratch_bytes_ph(int K, int N, int r, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                                   const void* bias, int K, int N, int r, int group, void* blob,
+                                                   size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                                   dirotq_stream_t stream, dirotq_layer_t** layer_out);
+/* uh_bf16 [K,r]: the rounded projection the layer applies. */
+DIROTQ_API dirotq_status_t dirotq_layer_export_uh(const dirotq_layer_t* layer, void* uh_bf16, dirotq_stream_t stream);
+
 /* ---- asymmetric activation codes (paper Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the 4-bit INT setting
  * quantizes the activations asymmetrically) ---- */
 

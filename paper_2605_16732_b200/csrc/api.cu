@@ -275,6 +275,100 @@ dirotq_status_t dirotq_prepare_layer_sibling(const void* W, int w_dtype, int w_l
                         blob_bytes, scratch, scratch_bytes, stream, layer_out);
 }
 
+// ---- projection form (fmt 4): U_h only, block-Hadamard residual ----
+
+static dirotq_status_t ph_geometry(int K, int N, int r, int group, Geometry* out) {
+    dirotq_status_t st = check_shape(K, N, r, group);
+    if (st != DIROTQ_OK) return st;
+    Geometry g = make_geometry(K, N, r, group);
+    make_ph(g);
+    *out = g;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_layer_bytes_ph(int K, int N, int r, int group, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    Geometry g;
+    dirotq_status_t st = ph_geometry(K, N, r, group, &g);
+    if (st != DIROTQ_OK) return st;
+    *bytes = make_blob_layout(g).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_scratch_bytes_ph(int K, int N, int r, size_t* bytes) {
+    if (!bytes || K <= 0 || N <= 0 || r <= 0) return DIROTQ_ERR_INVALID_ARG;
+    *bytes = (static_cast<size_t>(K) + r) * N * sizeof(double);
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                        const void* bias, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                        void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                        dirotq_layer_t** layer_out) {
+    if (!W || !Uh || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
+    if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
+    if (uh_dtype != DIROTQ_DTYPE_F64 && uh_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
+    if (w_layout != DIROTQ_LAYOUT_KN && w_layout != DIROTQ_LAYOUT_NK) return DIROTQ_ERR_INVALID_ARG;
+    Geometry g;
+    dirotq_status_t st = ph_geometry(K, N, r, group, &g);
+    if (st != DIROTQ_OK) return st;
+    if (!aligned16(W) || !aligned16(Uh) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
+    const BlobLayout lay = make_blob_layout(g);
+    if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (scratch_bytes < (static_cast<size_t>(K) + r) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    int dev = 0;
+    st = check_device(&dev);
+    if (st != DIROTQ_OK) return st;
+    dirotq_layer* L = new (std::nothrow) dirotq_layer;
+    if (!L) return DIROTQ_ERR_INVALID_ARG;
+    memset(L, 0, sizeof *L);
+    L->magic = kLayerMagic;
+    L->device = dev;
+    L->geo = g;
+    L->lay = lay;
+    L->blob = static_cast<char*>(blob);
+    // first stage, step 1: x [M,K] times U_hb^T stored as [r_pad][K] (a 128-row box reads zeros past r_pad);
+    // step 2: x~_h [M,r_pad] times U_hb stored as [K][r_pad]
+    st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K,
+                        (uint64_t)g.r_pad, (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_uh, (uint64_t)g.r_pad,
+                            (uint64_t)K, (uint64_t)g.r_pad * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
+                            (uint64_t)g.n_g, (uint64_t)N * 4, kGemmBN, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked128, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                            (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wscale128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
+                            (uint64_t)g.n_g, (uint64_t)N * 4, 128, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = launch_prepare_ph(L, W, w_dtype, w_layout, Uh, uh_dtype, bias, static_cast<double*>(scratch),
+                               static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) {
+        delete L;
+        return st;
+    }
+    *layer_out = L;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_layer_export_uh(const dirotq_layer_t* layer, void* uh_bf16, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || layer->geo.fmt != 4 || !uh_bf16) return DIROTQ_ERR_INVALID_ARG;
+    return launch_uh_export(layer, static_cast<uint16_t*>(uh_bf16), static_cast<cudaStream_t>(stream));
+}
+
 dirotq_status_t dirotq_layer_bytes_w4a8(int K, int N, int r, size_t* bytes) {
     if (!bytes) return DIROTQ_ERR_INVALID_ARG;
     dirotq_status_t st = check_shape(K, N, r, 64);
@@ -419,6 +513,7 @@ static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M,
 // First kernel(s): rotation + split + quantization.  W4A8 needs the token's whole row before it can quantize: the rotation
 // kernel writes fp32 coefficients and the row maxima, a second small kernel quantizes.
 static dirotq_status_t first_kernel(const dirotq_layer_t* layer, const RotateArgs& ra, int M, cudaStream_t s) {
+    if (layer->geo.fmt == 4) return launch_project_quantize(layer, ra, s);
     if (layer->geo.fmt == 3) {
         if (cudaMemsetAsync(ra.rowmax, 0, static_cast<size_t>(M) * 4, s) != cudaSuccess) return DIROTQ_ERR_CUDA;
         dirotq_status_t st = launch_rotate_quantize(layer, ra, s);
@@ -599,7 +694,7 @@ dirotq_status_t dirotq_workspace_wait_counters(const void* workspace, dirotq_str
 
 dirotq_status_t dirotq_workspace_export(const dirotq_layer_t* layer, int M, const void* workspace, void* xh_bf16,
                                         int8_t* codes, void* scales_bf16, dirotq_stream_t stream) {
-    if (!valid_layer(layer) || layer->geo.fmt != 0 || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
+    if (!valid_layer(layer) || (layer->geo.fmt != 0 && layer->geo.fmt != 4) || !workspace || M < 1 || M > 65535) return DIROTQ_ERR_INVALID_ARG;
     return launch_workspace_export(layer, M, static_cast<const char*>(workspace), static_cast<uint16_t*>(xh_bf16), codes,
                                    static_cast<uint16_t*>(scales_bf16), static_cast<cudaStream_t>(stream));
 }
@@ -637,7 +732,7 @@ dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M, const diro
 dirotq_status_t dirotq_layer_export(const dirotq_layer_t* layer, int8_t* wcodes, void* wscales_bf16, void* wh_bf16,
                                     void* q_bf16, dirotq_stream_t stream) {
     if (!valid_layer(layer) || layer->geo.fmt == 1) return DIROTQ_ERR_INVALID_ARG;
-    if (q_bf16 && layer->geo.no_rot) return DIROTQ_ERR_INVALID_ARG;  // a sibling layer holds no rotation
+    if (q_bf16 && (layer->geo.no_rot || layer->geo.fmt == 4)) return DIROTQ_ERR_INVALID_ARG;  // no K x K rotation in the blob
     return launch_layer_export(layer, wcodes, static_cast<uint16_t*>(wscales_bf16), static_cast<uint16_t*>(wh_bf16),
                                static_cast<uint16_t*>(q_bf16), static_cast<cudaStream_t>(stream));
 }

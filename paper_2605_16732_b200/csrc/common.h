@@ -28,6 +28,8 @@ struct Geometry {
     int fmt;     // 0 = INT4 groups with bf16 scales, 1 = NVFP4 (E2M1 elements, E4M3 block scales),
                  // 2 = INT4 with asymmetric activation codes (0..15, bf16 scale and zero-point per group),
                  // 3 = W4A8: INT8 activations with one scale per token, INT4 weights with one scale per output column
+                 // 4 = projection form: only U_h [K, r] is applied densely, the residual (all K columns) is rotated by a
+                 //     block Hadamard per group and quantized like fmt 0; then K_l = K_lp = K and there is no K x K rotation
                  //     (G = 128 is then only the packing granularity: K_lp = K_l rounded up to 128, n_g = K_lp / 128)
     int K4;      // K_l rounded up to 64 (<= K): width of the packed E2M1 rows
     int nkb64;   // K4 / 64: scale-factor atoms (128 rows x 4 scales) per row block
@@ -54,6 +56,14 @@ inline Geometry make_geometry(int K, int N, int r, int G) {
 constexpr size_t kAlign = 1024;
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
+// Projection form (fmt 4): every one of the K residual coefficients is low-precision.
+inline void make_ph(Geometry& g) {
+    g.fmt = 4;
+    g.K_l = g.K;
+    g.n_g = g.K / g.G;
+    g.K_lp = g.K;
+}
+
 // Sections of the device blob that holds a prepared layer.
 // Asymmetric activations (fmt 2): x^ = s u + z per group.  The zero-point term sum_g z[m,g] * (s_w[g,n] sum_{j in g} q_w[j,n])
 // is a rank-n_g product; it rides on the bf16 rank-r branch as 3 n_g extra columns: the activation side holds z (bf16,
@@ -72,13 +82,15 @@ struct BlobLayout {
     // NVFP4 variant: off_wpacked = E2M1 codes u8 [N][K4/2] (even k in the low nibble); off_wscale = E4M3 scale
     // atoms u8 [ceil(N/128)][nkb64p][512]; off_meta = {float out_scale = 2^(ex+ew), int ew, int ex, uint amax bits}
     size_t off_meta;
+    size_t off_uh;       // fmt 4 only: bf16 [K][r_pad], U_hb row-major (off_qt then holds its transpose, bf16 [r_pad][K])
     size_t total;
 };
 
 inline BlobLayout make_blob_layout(const Geometry& g) {
     BlobLayout b;
     size_t o = 0;
-    b.off_qt = o;      o = align_up(o + (g.no_rot ? 0 : (size_t)g.K * g.K * 2));
+    b.off_qt = o;      o = align_up(o + (g.fmt == 4 ? (size_t)g.r_pad * g.K * 2 : g.no_rot ? 0 : (size_t)g.K * g.K * 2));
+    b.off_uh = o;      o = align_up(o + (g.fmt == 4 ? (size_t)g.K * g.r_pad * 2 : 0));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K_lp / 2));
     b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * g.N * 4);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
@@ -92,6 +104,7 @@ inline BlobLayout make_blob_layout_nvfp4(const Geometry& g) {
     BlobLayout b;
     size_t o = 0;
     b.off_qt = o;      o = align_up(o + (size_t)g.K * g.K * 2);
+    b.off_uh = o;
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K4 / 2));
     b.off_wscale = o;  o = align_up(o + (size_t)((g.N + 127) / 128) * g.nkb64p * 512);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
@@ -250,6 +263,10 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
 dirotq_status_t set_nvfp4_tile_columns(int columns);
 dirotq_status_t set_w4a8_tile_columns(int columns);
 dirotq_status_t set_rotation_plan(int plan);
+dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                  const void* bias, double* scratch, cudaStream_t stream);
+dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, cudaStream_t stream);
+dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
 struct Nvfp4GemmArgs {
     int M;
     const uint8_t* codes;  // [M][K4/2]

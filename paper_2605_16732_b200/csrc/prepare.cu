@@ -560,6 +560,91 @@ dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype
     return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------ projection form (fmt 4)
+
+namespace {
+
+__device__ __forceinline__ double load_uh(const void* Uh, int dtype, int r, int k, int i) {
+    const size_t e = static_cast<size_t>(k) * r + i;
+    return dtype == DIROTQ_DTYPE_F64 ? static_cast<const double*>(Uh)[e] : static_cast<double>(static_cast<const float*>(Uh)[e]);
+}
+
+// uht[i][k] = uh[k][i] = bf16(Uh[k][i]), zero for i >= r
+__global__ void ph_round_uh_kernel(const void* Uh, int dtype, uint16_t* uht, uint16_t* uh, Geometry g) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= g.K) return;
+    for (int i = 0; i < g.r_pad; ++i) {
+        const uint16_t v = i < g.r ? f64_to_bf16(load_uh(Uh, dtype, g.r, k, i)) : 0;
+        uht[static_cast<size_t>(i) * g.K + k] = v;
+        uh[static_cast<size_t>(k) * g.r_pad + i] = v;
+    }
+}
+
+// Wt[i][n] = sum_k U_hb[k][i] W[k][n] for i < r (fp64 sums of the ROUNDED projection times the weights)
+__global__ void ph_fold_high_kernel(const uint16_t* uh, const void* W, int w_dtype, int w_layout, double* Wt, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = blockIdx.y;
+    if (n >= g.N) return;
+    double acc = 0.0;
+    for (int k = 0; k < g.K; ++k)
+        acc = fma(bf16_to_f64(uh[static_cast<size_t>(k) * g.r_pad + i]), load_w(W, w_dtype, w_layout, g.K, g.N, k, n), acc);
+    Wt[static_cast<size_t>(i) * g.N + n] = acc;
+}
+
+// Wt[r + b G + i][n] = (1 / sqrt(G)) sum_j (-1)^popc(i & j) W[b G + j][n]: the block Hadamard applied to the rows of W
+__global__ void ph_fold_low_kernel(const void* W, int w_dtype, int w_layout, double* Wt, Geometry g) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int row = blockIdx.y;  // 0 .. K-1
+    if (n >= g.N) return;
+    const int b = row / g.G, i = row % g.G;
+    double acc = 0.0;
+    for (int j = 0; j < g.G; ++j) {
+        const double w = load_w(W, w_dtype, w_layout, g.K, g.N, b * g.G + j, n);
+        acc += (__popc(i & j) & 1) ? -w : w;
+    }
+    Wt[static_cast<size_t>(g.r + row) * g.N + n] = acc / sqrt(static_cast<double>(g.G));
+}
+
+__global__ void ph_export_uh_kernel(const uint16_t* uh, uint16_t* out, Geometry g) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= g.K) return;
+    for (int i = 0; i < g.r; ++i) out[static_cast<size_t>(k) * g.r + i] = uh[static_cast<size_t>(k) * g.r_pad + i];
+}
+
+}  // namespace
+
+dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                  const void* bias, double* scratch, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    char* blob = L->blob;
+    uint16_t* uht = reinterpret_cast<uint16_t*>(blob + L->lay.off_qt);
+    uint16_t* uh = reinterpret_cast<uint16_t*>(blob + L->lay.off_uh);
+    ph_round_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(Uh, uh_dtype, uht, uh, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_fold_high_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(uh, W, w_dtype, w_layout, scratch, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_fold_low_kernel<<<dim3((g.N + 127) / 128, g.K), 128, 0, stream>>>(W, w_dtype, w_layout, scratch, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    if (cudaMemsetAsync(blob + L->lay.off_wpacked, 0, static_cast<size_t>(g.N) * (g.K_lp / 2), stream) != cudaSuccess)
+        return DIROTQ_ERR_CUDA;
+    // scratch now holds [r + K][N]: the same shape the INT4 pipeline quantizes (rows < r in 16 bits, the rest in groups)
+    high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale),
+        reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                       reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    ph_export_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(reinterpret_cast<const uint16_t*>(L->blob + L->lay.off_uh), uh, g);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
 dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint16_t* wscales, uint16_t* wh,
                                     uint16_t* qb, cudaStream_t stream) {
     const Geometry& g = L->geo;

@@ -42,6 +42,8 @@ constexpr int SMEM_BYTES = STAGES_WIDE * STAGE_BYTES_WIDE + 1024 /*alignment sla
 
 struct RotKernelParams {
     int M, K, K_l, K_lp, r, r_pad, r_pad0, ldm, n_g;
+    int n_out, k_red;      // output columns and reduction length of the GEMM (both K for the rotation x Q)
+    const uint16_t* xsub;  // FMT 4: bf16 [M][K], the accumulator is subtracted from it (residual of the projection)
     int8_t* codes;
     float* xscale;
     uint16_t* xh;
@@ -183,9 +185,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const int lane = threadIdx.x & 31;
 
     const int num_m_blocks = (p.M + BM - 1) / BM;
-    const int num_n_blocks = (p.K + BN - 1) / BN;
+    const int num_n_blocks = (p.n_out + BN - 1) / BN;
     const int num_tiles = num_m_blocks * num_n_blocks;
-    const int num_kb = p.K / BK;
+    const int num_kb = p.k_red / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -298,7 +300,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll 1
             for (int chunk = (BM == 256 ? 0 : half * CPH); chunk < min(CHUNKS, (BM == 256 ? 1 : half + 1) * CPH); ++chunk) {
                 const int col0 = n0 + chunk * G;  // permuted column of v[0]
-                if (col0 >= p.K) break;
+                if (col0 >= p.n_out) break;
                 float v[G];
 #pragma unroll
                 for (int c = 0; c < G / 32; ++c) {
@@ -319,6 +321,36 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                             dst[j] = make_float4(v[16 * b + 4 * j], v[16 * b + 4 * j + 1], v[16 * b + 4 * j + 2],
                                                  v[16 * b + 4 * j + 3]);
                     }
+                }
+                if constexpr (FMT == 4) {
+                    // projection form: v = x - x~_h U_hb^T (the accumulator holds the product), then the group's
+                    // Hadamard block in registers; what follows quantizes it like any other group
+                    if (row_ok) {
+                        const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + col0);
+#pragma unroll
+                        for (int b = 0; b < G / 8; ++b) {
+                            const uint4 w = __ldg(xs + b);
+                            const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                v[8 * b + 2 * e] = __uint_as_float(ws[e] << 16) - v[8 * b + 2 * e];
+                                v[8 * b + 2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u) - v[8 * b + 2 * e + 1];
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int h = 1; h < G; h <<= 1)
+#pragma unroll
+                        for (int i = 0; i < G; i += 2 * h)
+#pragma unroll
+                            for (int j = i; j < i + h; ++j) {
+                                const float a0 = v[j], a1 = v[j + h];
+                                v[j] = a0 + a1;
+                                v[j + h] = a0 - a1;
+                            }
+                    constexpr float kNorm = G == 64 ? 0.125f : 0.08838834764831845f;  // 1 / sqrt(G)
+#pragma unroll
+                    for (int j = 0; j < G; ++j) v[j] *= kNorm;
                 }
                 // number of low-precision values among v[] (a multiple of 16)
                 const int nlow = min(G, max(0, p.K_l - col0));
@@ -432,7 +464,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll
                     for (int b = 0; b < G / 16; ++b) {
                         const int pc = col0 + 16 * b;
-                        if (16 * b >= nlow && pc < p.K) {
+                        if (16 * b >= nlow && pc < p.n_out) {
                             uint4 lo = make_uint4(pack_bf16x2(v[16 * b + 0], v[16 * b + 1]), pack_bf16x2(v[16 * b + 2], v[16 * b + 3]),
                                                   pack_bf16x2(v[16 * b + 4], v[16 * b + 5]), pack_bf16x2(v[16 * b + 6], v[16 * b + 7]));
                             uint4 hi = make_uint4(pack_bf16x2(v[16 * b + 8], v[16 * b + 9]), pack_bf16x2(v[16 * b + 10], v[16 * b + 11]),
@@ -452,7 +484,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
-            if (n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
+            if (FMT != 4 && n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
                 for (int c = p.r; c < p.r_pad0; c += 8)
                     *reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + c) = make_uint4(0, 0, 0, 0);
                 if constexpr (FMT == 2) {  // behind the 3 n_g zero-point columns
@@ -484,6 +516,7 @@ dirotq_status_t set_rotation_plan(int plan) {
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     RotKernelParams p;
+    p.n_out = g.K; p.k_red = g.K; p.xsub = nullptr;
     p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
@@ -536,6 +569,59 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
                          p) == cudaSuccess
                ? DIROTQ_OK
                : DIROTQ_ERR_CUDA;
+}
+
+// Projection form (fmt 4): x~_h = bf16(x U_hb) with the rotation kernel on r_pad output columns, then the residual
+// x - x~_h U_hb^T, its block Hadamard and the group quantizer with the same kernel on a reduction of length r_pad.
+dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    if (a.xrot != nullptr) return DIROTQ_ERR_INVALID_ARG;  // there is no K-wide rotated activation in this form
+    const int sms = sm_count(L->device);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const RotKernelParams);
+    RotKernelParams p;
+    p.M = a.M; p.K = g.K; p.K_lp = g.K_lp; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
+    p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = nullptr; p.status = a.status;
+    p.xsf = nullptr; p.K4 = 0; p.nkb64p = 0; p.ex = 0; p.xtilde = nullptr; p.rowmax = nullptr;
+    dirotq_status_t st;
+    {
+        // step 1: all r_pad output columns are "high" (K_l = 0): the epilogue only rounds them to bf16 into xh
+        CUtensorMap tmap_x;
+        st = encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M, (uint64_t)g.K * 2, BK,
+                            128, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (st != DIROTQ_OK) return st;
+        RotKernelParams p1 = p;
+        p1.n_out = g.r_pad; p1.k_red = g.K; p1.K_l = 0; p1.r = g.r_pad; p1.xsub = nullptr;
+        const KernelFn k1 = rotate_quant_kernel<64, 0, 128, 128>;
+        static bool attr1 = false;
+        if (!attr1) {
+            if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return DIROTQ_ERR_CUDA;
+            attr1 = true;
+        }
+        const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.r_pad + 127) / 128);
+        if (launch_kernel(k1, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_x,
+                          L->tmap_qt128, p1) != cudaSuccess)
+            return DIROTQ_ERR_CUDA;
+    }
+    {
+        // step 2: A = x~_h [M][r_pad], B = U_hb [K][r_pad]; every output column is low-precision (K_l = K)
+        CUtensorMap tmap_xh;
+        st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,
+                            (uint64_t)g.r_pad * 2, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (st != DIROTQ_OK) return st;
+        RotKernelParams p2 = p;
+        p2.n_out = g.K; p2.k_red = g.r_pad; p2.K_l = g.K; p2.r = g.r; p2.xsub = static_cast<const uint16_t*>(a.x);
+        const KernelFn k2 = g.G == 64 ? rotate_quant_kernel<64, 4, 256, 128> : rotate_quant_kernel<128, 4, 256, 128>;
+        static bool attr2[2] = {false, false};
+        if (!attr2[g.G == 64 ? 0 : 1]) {
+            if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return DIROTQ_ERR_CUDA;
+            attr2[g.G == 64 ? 0 : 1] = true;
+        }
+        const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.K + 255) / 256);
+        if (launch_kernel(k2, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_xh, L->tmap_qt,
+                          p2) != cudaSuccess)
+            return DIROTQ_ERR_CUDA;
+    }
+    return DIROTQ_OK;
 }
 
 }  // namespace dirotq

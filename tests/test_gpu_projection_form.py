@@ -1,0 +1,105 @@
+"""Parity of the projection form (U_h only + block-Hadamard residual, a cheaper first stage that is NOT the paper's
+Eq. 5) against its CPU reference, stage by stage: prepared weights, x~_h, codes and scales of the rotated residual,
+integer group sums, output."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dirotq_oracle as orc
+from paper_2605_16732_b200 import binding as dq
+from paper_2605_16732_b200 import synth
+
+from parity_utils import bf16_tensor_to_bits, bits_to_bf16_tensor, check_activation_side, check_layer_output
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_case(spec: synth.LayerSpec, M: int, with_bias=True):
+    inp = synth.make_layer_inputs(spec, M, with_bias=with_bias)
+    Uh = np.ascontiguousarray(np.asarray(inp["Q"], dtype=np.float64)[:, :spec.r])
+    lo = orc.prepare_layer_ph(inp["W"], Uh, spec.G)
+    oo = orc.linear_deployed_ph(inp["x"], lo, bias=inp["bias"])
+
+    dev = "cuda"
+    W = torch.from_numpy(inp["W"]).to(dev)
+    bias = bits_to_bf16_tensor(inp["bias"]) if with_bias else None
+    layer = dq.dirotq_prepare_layer_ph(W, torch.from_numpy(Uh).to(dev), spec.G, bias=bias)
+    assert (layer.K_l, layer.n_g) == (spec.K, spec.K // spec.G)
+
+    # weight side: the rounded projection, the 16-bit rows U_hb^T W, scales and codes of H^T W (exact ties may differ)
+    assert np.array_equal(bf16_tensor_to_bits(dq.dirotq_layer_export_uh(layer)), lo["Uhb"])
+    wcodes = torch.empty((spec.K, spec.N), dtype=torch.int8, device=dev)
+    wscales = torch.empty((layer.n_g, spec.N), dtype=torch.bfloat16, device=dev)
+    wh = torch.empty((spec.r, spec.N), dtype=torch.bfloat16, device=dev)
+    dq._check(dq.lib().dirotq_layer_export(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(), None, None),
+              "dirotq_layer_export")
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_tensor_to_bits(wh), lo["Wh"])
+    assert np.array_equal(bf16_tensor_to_bits(wscales), lo["wscales"])
+    bad = wcodes.cpu().numpy() != lo["wcodes"]
+    if bad.any():
+        t = lo["wt"][bad]
+        assert bad.sum() <= 4 and np.all(np.abs(np.abs(t - np.floor(t)) - 0.5) < 1e-9)
+    lo_gpu = dict(lo)
+    lo_gpu["wcodes"] = wcodes.cpu().numpy()
+
+    x = bits_to_bf16_tensor(inp["x"])
+    ws = dq.alloc_workspace(layer, M)
+    dq.dirotq_rotate_quantize(x, layer, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, scales = dq.dirotq_workspace_export(layer, M, ws)
+    xh_b, codes_n, scales_b = bf16_tensor_to_bits(xh), codes.cpu().numpy(), bf16_tensor_to_bits(scales)
+    assert codes_n.shape == (M, spec.K)
+    # x~_h: within one bf16 step of the reference where the fp32 sum lands on a rounding boundary
+    xh_g, xh_o = orc.bf16_to_f64(xh_b), orc.bf16_to_f64(oo["xh"])
+    xnorm = np.linalg.norm(orc.bf16_to_f64(inp["x"]), axis=1, keepdims=True)
+    assert np.all(np.abs(xh_g - xh_o) <= np.maximum(np.abs(xh_o), 2.0 ** -126) * 2.0 ** -7 + 1e-5 * xnorm)
+    # The residual is DEFINED through the rounded x~_h, so a token whose x~_h differs in one element has a different
+    # (equally valid) residual: codes and scales are held to the reference's second step run on the library's own x~_h,
+    # with the same protocol as for the rotation (equal except at rounding boundaries).
+    Uhb = orc.bf16_to_f64(lo["Uhb"])
+    xl_ref = orc.block_hadamard_cols(orc.bf16_to_f64(inp["x"]) - xh_g @ Uhb.T, spec.G)
+    sq_ref = orc.split_quantize(xl_ref, 0, spec.G, want_t=True)
+    same_xh = np.all(xh_b == oo["xh"], axis=1)
+    assert np.array_equal(sq_ref["codes"][same_xh], oo["codes"][same_xh])      # consistency of the re-run
+    prot = {"xt": np.concatenate([xh_g, xl_ref], axis=1), "xh": xh_b, "scales": sq_ref["scales"], "codes": sq_ref["codes"]}
+    stats = check_activation_side(None, xh_b, codes_n, scales_b, prot, spec.r, spec.G)
+    stats["xh_exact_frac"] = float(np.mean(xh_b == oo["xh"]))
+
+    padded = np.ascontiguousarray(oo["codes"])
+    P = dq.dirotq_int_gemm_debug(torch.from_numpy(padded).to(dev), layer, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    assert np.array_equal(P.cpu().numpy(), orc.int_gemm(oo["codes"], lo_gpu["wcodes"], spec.G)), "int32 group sums differ"
+
+    y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    stats.update(check_layer_output(bf16_tensor_to_bits(y), xh_b, codes_n, scales_b, lo_gpu, oo, inp["bias"]))
+    y2 = torch.zeros_like(y)
+    dq.dirotq_linear(x, layer, y2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    with pytest.raises(dq.DirotqError):
+        dq.dirotq_layer_export(layer)          # asks for the K x K rotation, which this form does not have
+    layer.close()
+    return stats
+
+
+def test_projection_form_small():
+    spec = synth.LayerSpec(K=256, N=256, r=32, G=64, model=synth.PIXART, seed=101, calib_tokens=512)
+    print(_run_case(spec, M=100))
+
+
+def test_projection_form_pixart_projection():
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=102)
+    print(_run_case(spec, M=256))
+
+
+def test_projection_form_ragged_rows_columns_group128():
+    spec = synth.LayerSpec(K=512, N=400, r=16, G=128, model=synth.FLUX, seed=103, calib_tokens=1024)
+    print(_run_case(spec, M=300))
+
+
+def test_projection_form_rank_112_no_bias():
+    spec = synth.LayerSpec(K=1152, N=384, r=112, G=64, model=synth.PIXART, seed=104)
+    print(_run_case(spec, M=257, with_bias=False))
