@@ -126,6 +126,8 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
         elif fmt == "nvfp4":
             lo = orc.nvfp4_prepare_layer(W, Q, RANK)
             lo["ex"] = orc.nvfp4_global_exponent(float(np.abs(orc.rotate(x, lo["Qb"])[:, RANK:]).max()))
+        elif fmt == "int4_ph":
+            lo = orc.prepare_layer_ph(W, np.ascontiguousarray(Q[:, :RANK]), GROUP)
         else:
             lo = orc.prepare_layer(W, Q, RANK, GROUP)
         layers.append((lo, x, K, cols))
@@ -139,6 +141,8 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
                 orc.linear_deployed_asym(x, lo, bias=None, want_t=False)
             elif fmt == "w4a8":
                 orc.linear_deployed_w4a8(x, lo, bias=None, want_t=False)
+            elif fmt == "int4_ph":
+                orc.linear_deployed_ph(x, lo, bias=None, want_t=False)
             else:
                 orc.linear_deployed(x, lo, bias=None, want_t=False)
         times.append(time.perf_counter() - t0)
@@ -163,7 +167,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64 (oracle; nvfp4 codes)" if args.fmt == "nvfp4" else "f64 + int32 (oracle; int4 codes)",
-        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else ""),
+        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else "_projection_form" if args.fmt == "int4_ph" else ""),
                                         "format": args.fmt,
                                         "sample": res["sample"]},
         "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
@@ -222,6 +226,8 @@ def run_ours(args):
             layer = dq.dirotq_prepare_layer_w4a8(torch.from_numpy(W).to(dev), Q, RANK, bias=bf(bias))
         elif args.fmt == "int4_asym":
             layer = dq.dirotq_prepare_layer_asym(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
+        elif args.fmt == "int4_ph":
+            layer = dq.dirotq_prepare_layer_ph(torch.from_numpy(W).to(dev), Q[:, :RANK].contiguous(), GROUP, bias=bf(bias))
         else:
             layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         del Q
@@ -342,8 +348,10 @@ def run_ours(args):
     rot_ms = {n: float(np.mean(v["rotate_ms"])) for n, v in per.items()}
     gemm_ms = {n: float(np.mean(v["gemm_ms"])) for n, v in per.items()}
     rot_total, gemm_total = sum(rot_ms.values()), sum(gemm_ms.values())
-    rot_flops = {n: 2.0 * M * K * K for n, K, _ in FLUX_SHAPES}
-    gemm_ops = {n: 2.0 * M * (K - RANK) * N for n, K, N in FLUX_SHAPES}
+    ph = args.fmt == "int4_ph"
+    # projection form: two skinny GEMMs on a 64-wide padded rank instead of the K x K rotation; all K columns are 4-bit
+    rot_flops = {n: (4.0 * M * K * 64 if ph else 2.0 * M * K * K) for n, K, _ in FLUX_SHAPES}
+    gemm_ops = {n: 2.0 * M * (K if ph else K - RANK) * N for n, K, N in FLUX_SHAPES}
     nv = args.fmt == "nvfp4"
     # nominal ratios of the part: 8-bit (int8 / fp8) 2x and fp4 4x the dense bf16 rate (4.5 and 9 : 2.25 PFLOP/s)
     int8_peak = (4.0 if nv else 2.0) * peaks["bf16_sustained"]
@@ -366,7 +374,7 @@ def run_ours(args):
                     "frac": ach / int8_peak, "traffic": NCU_TRAFFIC_QKV.get(gname),
                     "traffic_note": "ncu dram read+write of one qkv-shaped launch (algorithmic bytes of that launch: 117.5e6)",
                     "peak_source": f"{'4' if nv else '2'} x {peaks['source']} bf16 sustained (nominal {'fp4' if nv else '8-bit'}:bf16 ratio)"}
-        if args.fmt in ("int4", "int4_asym"):
+        if args.fmt in ("int4", "int4_asym", "int4_ph"):
             roofline["alu"] = {"bound": "alu", "achieved": ach_alu / 1e9, "peak": alu_peak / 1e9, "unit": "G element-steps/s",
                                "frac": ach_alu / alu_peak,
                                "note": "per-group rescale: 2 fp32 fused multiply-adds per output element and K-group; "
@@ -394,7 +402,7 @@ def run_ours(args):
         "dtype": ("nvfp4 (e2m1 x e2m1, e4m3 block scales) + bf16" if nv else "int8xint4->int32 + bf16" if args.fmt == "w4a8"
                   else "int4xint4 (exact group sums on the e4m3 tensor path) + bf16"),
         "data": "synthetic",
-        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
+        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else "_projection_form" if args.fmt == "int4_ph" else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
                    "group": 16 if nv else ("per-token / per-channel" if args.fmt == "w4a8" else GROUP), "format": args.fmt,
                    "l2": "inputs_exceed_l2 (each step streams > 500 MB of rotations, codes and outputs)",
                    "parallelism": f"token rows x{world}, no collective"},
@@ -419,10 +427,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shapes", default="", help="comma-separated subset of qkv,out,mlp_up,mlp_down (profiling runs)")
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8"],
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8", "int4_ph"],
                     help="int4: the headline format (groups of 64, bf16 scales, symmetric); nvfp4: E2M1 blocks of 16 with E4M3 "
                          "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group); w4a8: per-token int8 "
-                         "activations, per-channel int4 weights")
+                         "activations, per-channel int4 weights; int4_ph: the projection form (U_h only + block-Hadamard residual), "
+                         "a cheaper first stage that is not the paper's Eq. 5")
     ap.add_argument("--gemm-tile", type=int, default=0, choices=[0, 128, 256],
                     help="output columns per tile of the second kernel (int4 / int4_asym / nvfp4): 0 = chosen per call")
     ap.add_argument("--lite", action="store_true", help="skip the cuBLAS, end-to-end and CPU-baseline legs (profiling runs)")

@@ -50,7 +50,7 @@ FMT = "int4"  # set from --fmt: "int4" (groups of G, bf16 scales) or "nvfp4" (bl
 class Case:
     def __init__(self, M, K, N, r, G, model):
         self.M, self.K, self.N, self.r, self.G = M, K, N, r, G
-        spec = synth.LayerSpec(K=K, N=N, r=r, G=G if FMT in ("int4", "int4_asym") else 64, model=model, seed=7)
+        spec = synth.LayerSpec(K=K, N=N, r=r, G=G if FMT in ("int4", "int4_asym", "int4_ph") else 64, model=model, seed=7)
         W, bias = synth.make_weights(spec)
         self.x = _bf(synth.make_tokens(spec, M, batch_seed=11))
         Wd, Q = torch.from_numpy(W).cuda(), _householder(K, K + r)
@@ -68,6 +68,8 @@ class Case:
             self.layer = dq.dirotq_prepare_layer_w4a8(Wd, Q, r, bias=_bf(bias))
         elif FMT == "int4_asym":
             self.layer = dq.dirotq_prepare_layer_asym(Wd, Q, r, G, bias=_bf(bias))
+        elif FMT == "int4_ph":
+            self.layer = dq.dirotq_prepare_layer_ph(Wd, Q[:, :r].contiguous(), G, bias=_bf(bias))
         else:
             self.layer = dq.dirotq_prepare_layer(Wd, Q, r, G, bias=_bf(bias))
         self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
@@ -131,11 +133,12 @@ class Case:
     def report(self, tag, iters, p_bf16, hbm, graphs=False):
         rot, gem, cb = self.time_kernels(iters)
         M, K, N, r, G = self.M, self.K, self.N, self.r, self.G
-        K_l = K - r
+        K_l = K if FMT == "int4_ph" else K - r
         n_g = -(-K_l // G) if G else 1
         tot = rot + gem
         p_i8 = (4.0 if FMT == "nvfp4" else 2.0) * p_bf16  # nominal ratio of the 4-bit / 8-bit tensor peak to bf16
-        t_roof = (2.0 * M * K_l * N / p_i8 + (2.0 * M * K * K + 2.0 * M * r * N) / p_bf16) / 1e12 * 1e3
+        first_flops = 4.0 * M * K * max(64, -(-r // 64) * 64) if FMT == "int4_ph" else 2.0 * M * K * K
+        t_roof = (2.0 * M * K_l * N / p_i8 + (first_flops + 2.0 * M * r * N) / p_bf16) / 1e12 * 1e3
         if FMT == "w4a8":
             bytes_alg = 2 * M * K + 2 * K * K + K_l * N / 2 + 4 * N + 2 * 64 * N + 2 * (M * K_l * 5 + 8 * M + 2 * M * 64) + 2 * M * N
         elif FMT == "nvfp4":
@@ -179,7 +182,7 @@ def main():
     ap.add_argument("--memory", action="store_true", help="print the layer sizes (no GPU needed) and exit")
     ap.add_argument("--configs", default="1,2,4,5", help="comma-separated subset of 1,2,3p,4,5")
     ap.add_argument("--iters", type=int, default=20)
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8"])
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8", "int4_ph"])
     ap.add_argument("--ranks", default="16,32,64,128", help="ranks swept by config 4")
     args = ap.parse_args()
     if args.memory:
@@ -235,7 +238,7 @@ def main():
     if "4" in todo:
         for K, N in [(3072, 9216), (12288, 3072)]:
             for r in [int(v) for v in args.ranks.split(",")]:
-                for G in ((64, 128) if FMT in ("int4", "int4_asym") else (16,) if FMT == "nvfp4" else (0,)):
+                for G in ((64, 128) if FMT in ("int4", "int4_asym", "int4_ph") else (16,) if FMT == "nvfp4" else (0,)):
                     c = Case(18432, K, N, r, G, synth.FLUX)
                     c.report("4: FLUX batch 4 (M=18432) rank/group sweep", max(5, args.iters // 2), p_bf16, hbm)
                     c.close()

@@ -300,3 +300,63 @@ def _run_w4a8(M, K, N, r, model, n_rows=24, n_cols=96, seed=0):
 @pytest.mark.parametrize("K,N", [(3072, 9216), (12288, 3072)])
 def test_w4a8_flux_linears(K, N):
     print(_run_w4a8(4608, K, N, 32, synth.FLUX))
+
+
+# ------------------------------------------------------------------ projection form at the benchmark's sizes
+
+def _run_ph(M, K, N, r, G, model, n_rows=24, n_cols=96, seed=0):
+    """Sampled parity of the projection form: the reference's steps on a sample of token rows (all K columns, since the
+    Hadamard blocks and the groups need them) and a sample of output columns."""
+    from parity_utils import check_activation_side, check_output
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=model, seed=seed)
+    rng = np.random.default_rng(1234 + seed)
+    rows = np.sort(rng.choice(M, size=n_rows, replace=False))
+    cols = np.sort(rng.choice(N, size=n_cols, replace=False))
+    Q = synth.make_rotation(spec, device="cuda")
+    Uh = np.ascontiguousarray(np.asarray(Q, dtype=np.float64)[:, :r])
+    W, bias = synth.make_weights(spec)
+    x_bits = synth.make_tokens(spec, M, batch_seed=7)
+    dev = "cuda"
+    layer = dq.dirotq_prepare_layer_ph(torch.from_numpy(W).to(dev), torch.from_numpy(Uh).to(dev), G, bias=bits_to_bf16_tensor(bias))
+    x = bits_to_bf16_tensor(x_bits)
+    ws = dq.alloc_workspace(layer, M)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device=dev)
+    dq.dirotq_linear(x, layer, y, ws)
+    torch.cuda.synchronize()
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, scales = dq.dirotq_workspace_export(layer, M, ws)
+    xh_b = bf16_tensor_to_bits(xh)[rows]
+    codes_n, scales_b = codes.cpu().numpy()[rows], bf16_tensor_to_bits(scales)[rows]
+    lo = orc.prepare_layer_ph(np.ascontiguousarray(W[:, cols]), Uh, G)
+    oo = orc.linear_deployed_ph(np.ascontiguousarray(x_bits[rows]), lo, bias=np.ascontiguousarray(bias[cols]))
+    Uhb = orc.bf16_to_f64(lo["Uhb"])
+    xh_g = orc.bf16_to_f64(xh_b)
+    xl_ref = orc.block_hadamard_cols(orc.bf16_to_f64(x_bits[rows]) - xh_g @ Uhb.T, G)
+    sq_ref = orc.split_quantize(xl_ref, 0, G, want_t=True)
+    prot = {"xt": np.concatenate([xh_g, xl_ref], axis=1), "xh": xh_b, "scales": sq_ref["scales"], "codes": sq_ref["codes"]}
+    stats = check_activation_side(None, xh_b, codes_n, scales_b, prot, r, G)
+    xnorm = np.linalg.norm(orc.bf16_to_f64(x_bits[rows]), axis=1, keepdims=True)
+    xh_o = orc.bf16_to_f64(oo["xh"])
+    assert np.all(np.abs(xh_g - xh_o) <= np.maximum(np.abs(xh_o), 2.0 ** -126) * 2.0 ** -7 + 1e-5 * xnorm)
+    # output on the sample: the reference's last steps on the library's own codes, scales and x~_h
+    wcodes = torch.empty((K, N), dtype=torch.int8, device=dev)
+    dq._check(dq.lib().dirotq_layer_export(layer.handle, wcodes.data_ptr(), None, None, None, None), "dirotq_layer_export")
+    torch.cuda.synchronize()
+    wc = wcodes.cpu().numpy()[:, cols]
+    bad = wc != lo["wcodes"]
+    assert bad.sum() <= 4
+    P = orc.int_gemm(codes_n, np.ascontiguousarray(wc), G)
+    y_ref, _ = orc.combine(P, scales_b, lo["wscales"], xh_b, lo["Wh"], np.ascontiguousarray(bias[cols]))
+    y_s = bf16_tensor_to_bits(y)[np.ix_(rows, cols)]
+    stats.update(check_output(y_s, y_ref))
+    layer.close()
+    return stats
+
+
+@pytest.mark.parametrize("K,N", [(3072, 9216), (12288, 3072)])
+def test_projection_form_flux_linears(K, N):
+    print(_run_ph(4608, K, N, 32, 64, synth.FLUX))
+
+
+def test_projection_form_batch4_group128_rank128():
+    print(_run_ph(18432, 3072, 3072, 128, 128, synth.FLUX))
