@@ -103,3 +103,68 @@ def test_projection_form_ragged_rows_columns_group128():
 def test_projection_form_rank_112_no_bias():
     spec = synth.LayerSpec(K=1152, N=384, r=112, G=64, model=synth.PIXART, seed=104)
     print(_run_case(spec, M=257, with_bias=False))
+
+
+def test_projection_form_through_the_other_entry_points():
+    # host entry (pipelined copies, M >= 2048 so that it cuts the rows into chunks), the built-in workspace, the two
+    # kernels called separately, a CUDA graph and every tile knob: all give the bits of dirotq_linear
+    spec = synth.LayerSpec(K=512, N=384, r=32, G=64, model=synth.PIXART, seed=105, calib_tokens=1024)
+    M, dev = 2300, "cuda"
+    inp = synth.make_layer_inputs(spec, M, with_bias=True)
+    Uh = np.ascontiguousarray(np.asarray(inp["Q"], dtype=np.float64)[:, :spec.r])
+    layer = dq.dirotq_prepare_layer_ph(torch.from_numpy(inp["W"]).to(dev), torch.from_numpy(Uh).to(dev), spec.G,
+                                       bias=bits_to_bf16_tensor(inp["bias"]))
+    x = bits_to_bf16_tensor(inp["x"])
+    ws = dq.alloc_workspace(layer, M)
+    y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
+    dq.dirotq_linear(x, layer, y, ws)
+    torch.cuda.synchronize()
+    ref = y.view(torch.int16).clone()
+
+    x_host = x.cpu().pin_memory()
+    y_host = torch.zeros((M, spec.N), dtype=torch.bfloat16).pin_memory()
+    xd, yd = torch.empty_like(x), torch.empty_like(y)
+    dq.dirotq_linear_host(x_host, layer, y_host, xd, yd, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y_host.view(torch.int16), ref.cpu())
+
+    m_small = 200                                    # the built-in workspace is small
+    y_small = torch.zeros((m_small, spec.N), dtype=torch.bfloat16, device=dev)
+    dq.dirotq_linear_noalloc(x[:m_small].contiguous(), layer, y_small)
+    torch.cuda.synchronize()
+    assert torch.equal(y_small.view(torch.int16), ref[:m_small])
+
+    y.zero_()
+    dq.dirotq_rotate_quantize(x, layer, ws)
+    dq.dirotq_w4a4_gemm(M, layer, ws, y)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), ref)
+
+    try:
+        for tile, plan, pdl in [(128, 1, False), (256, 3, True), (0, 2, True)]:
+            dq.dirotq_set_gemm_tile(tile)
+            dq.dirotq_set_rotation_tile(plan)       # the projection form has its own fixed plans: must be unaffected
+            dq.dirotq_set_dependent_launch(pdl)
+            y.zero_()
+            dq.dirotq_linear(x, layer, y, ws)
+            torch.cuda.synchronize()
+            assert torch.equal(y.view(torch.int16), ref)
+    finally:
+        dq.dirotq_set_gemm_tile(0)
+        dq.dirotq_set_rotation_tile(0)
+        dq.dirotq_set_dependent_launch(True)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            dq.dirotq_linear(x, layer, y, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    y.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), ref) and dq.dirotq_workspace_status(ws) == 0
+    with pytest.raises(dq.DirotqError):
+        dq.dirotq_rotate_quantize(x, layer, ws, torch.empty((M, spec.K), dtype=torch.float32, device=dev))
+    layer.close()
