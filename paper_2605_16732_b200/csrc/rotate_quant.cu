@@ -290,10 +290,21 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const int n0 = n_blk * BN;
             const uint32_t acc = tcount % ACC_BUFS;
             const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
-            if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
-            tc_fence_after_sync();
             const int row = m0 + (BM == 256 ? half * 128 : 0) + q * 32 + lane;
             const bool row_ok = row < p.M;
+            // FMT 4: this thread's 128 or 256 bytes of x for the chunk it handles next; requested a chunk ahead (the
+            // first one before the accumulator wait) so that the load's latency is not paid per chunk
+            [[maybe_unused]] uint4 xq[G / 8];
+            [[maybe_unused]] const int chunk_first = BM == 256 ? 0 : half * CPH;
+            if constexpr (FMT == 4) {
+                if (row_ok && n0 + chunk_first * G < p.n_out) {
+                    const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + n0 + chunk_first * G);
+#pragma unroll
+                    for (int b = 0; b < G / 8; ++b) xq[b] = __ldg(xs + b);
+                }
+            }
+            if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
+            tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (BM == 256 ? half * 256 : acc * BN);
 
             float tile_amax = 0.f;  // W4A8: this thread's row, this tile's columns
@@ -326,16 +337,20 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     // projection form: v = x - x~_h U_hb^T (the accumulator holds the product), then the group's
                     // Hadamard block in registers; what follows quantizes it like any other group
                     if (row_ok) {
-                        const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + col0);
 #pragma unroll
                         for (int b = 0; b < G / 8; ++b) {
-                            const uint4 w = __ldg(xs + b);
+                            const uint4 w = xq[b];
                             const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 v[8 * b + 2 * e] = __uint_as_float(ws[e] << 16) - v[8 * b + 2 * e];
                                 v[8 * b + 2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u) - v[8 * b + 2 * e + 1];
                             }
+                        }
+                        if (CPH > 1 && col0 + G < p.n_out && chunk + 1 < min(CHUNKS, (BM == 256 ? 1 : half + 1) * CPH)) {
+                            const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + col0 + G);
+#pragma unroll
+                            for (int b = 0; b < G / 8; ++b) xq[b] = __ldg(xs + b);
                         }
                     }
 #pragma unroll
