@@ -11,13 +11,14 @@ from paper_2605_16732_b200 import synth
 import test_gpu_asym
 import test_gpu_nvfp4
 import test_gpu_parity
+import test_gpu_projection_form
 import test_gpu_w4a8
 
 pytestmark = pytest.mark.gpu
 
 
 def _one(rng, big):
-    fmt = rng.choice(["int4", "int4", "asym", "nvfp4", "w4a8"])
+    fmt = rng.choice(["int4", "int4", "asym", "nvfp4", "w4a8", "ph"])
     if big:
         M = rng.choice([19000, 20001, 25000])
         K = 64 * rng.randint(2, 4)
@@ -38,7 +39,7 @@ def _one(rng, big):
         r = 16 * rng.randint(1, max(1, K // 32))      # up to half of K in 16 bits
     bias = rng.random() < 0.7
     model = rng.choice([synth.PIXART, synth.FLUX])
-    spec = synth.LayerSpec(K=K, N=N, r=r, G=G if fmt in ("int4", "asym") else 64, model=model, seed=rng.randint(1, 10 ** 6),
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=G if fmt in ("int4", "asym", "ph") else 64, model=model, seed=rng.randint(1, 10 ** 6),
                            calib_tokens=max(512, 2 * K))
     desc = dict(fmt=fmt, M=M, K=K, N=N, r=r, G=spec.G, tile=tile, pdl=pdl, bias=bias, plan=plan)
     dq.dirotq_set_gemm_tile(tile)
@@ -49,6 +50,8 @@ def _one(rng, big):
             test_gpu_parity._run_case(spec, M=M, with_bias=bias, check_rot=not big)
         elif fmt == "asym":
             test_gpu_asym._run_case(spec, M=M, with_bias=bias, shift=rng.choice([0.0, 1.5]), check_rot=not big)
+        elif fmt == "ph":
+            test_gpu_projection_form._run_case(spec, M=M, with_bias=bias)
         elif fmt == "nvfp4":
             test_gpu_nvfp4._run_case(spec, M=M, with_bias=bias, check_rot=not big)
         else:
