@@ -276,6 +276,47 @@ def linear_deployed_ph(x_bits, layer, bias=None, want_t: bool = True):
             "y64": y64, "y": yb}
 
 
+def nvfp4_prepare_layer_ph(W, Uh, want_t: bool = False):
+    """Projection form with NVFP4 operands: rows U_hb^T W in 16 bits, the rows of H^T W (Hadamard blocks of 64) as E2M1
+    codes with E4M3 block scales and a per-tensor power of two, exactly as nvfp4_prepare_layer quantizes its low rows."""
+    W = _c(W, np.float64)
+    Uh = _c(Uh, np.float64)
+    K, N = W.shape
+    r = Uh.shape[1]
+    assert Uh.shape[0] == K and K % 64 == 0
+    Uhb = bf16_round(Uh)
+    Wt = np.ascontiguousarray(np.concatenate([matmul(np.ascontiguousarray(bf16_to_f64(Uhb).T), W), block_hadamard_rows(W, 64)],
+                                             axis=0))
+    nb = K // 16
+    Wh = np.empty((r, N), dtype=np.uint16)
+    wcodes = np.empty((K, N), dtype=np.uint8)
+    wsf = np.empty((nb, N), dtype=np.uint8)
+    wt = np.empty((K, N), dtype=np.float64) if want_t else None
+    ew = _load().dq_nvfp4_prepare_weights(_p(Wt), ctypes.c_int(K + r), ctypes.c_int(N), ctypes.c_int(r), _p(Wh), _p(wcodes),
+                                          _p(wsf), _p(wt))
+    return {"Wh": Wh, "wcodes": wcodes, "wsf": wsf, "ew": int(ew), "wt": wt, "Uhb": Uhb, "r": r, "K": K}
+
+
+def nvfp4_residual(x_bits, layer, xh_bits=None):
+    """x~_h (bf16 bits) and x~_l = (x - x~_h U_hb^T) H for the projection form; xh_bits overrides the reference's own x~_h."""
+    x = bf16_to_f64(_c(x_bits, np.uint16))
+    Uhb = bf16_to_f64(layer["Uhb"])
+    if xh_bits is None:
+        xh_bits = bf16_round(matmul(x, Uhb))
+    d = x - matmul(bf16_to_f64(xh_bits), np.ascontiguousarray(Uhb.T))
+    return xh_bits, block_hadamard_cols(d, 64)
+
+
+def nvfp4_linear_deployed_ph(x_bits, layer, ex: int, bias=None, want_t: bool = True):
+    r = layer["r"]
+    xh_bits, xl = nvfp4_residual(x_bits, layer)
+    xt = np.ascontiguousarray(np.concatenate([bf16_to_f64(xh_bits), xl], axis=1))
+    sq = nvfp4_split_quantize(xt, r, ex, want_t=want_t)
+    assert np.array_equal(sq["xh"], xh_bits)
+    y64, yb = nvfp4_combine(sq["codes"], sq["sf"], ex, layer, sq["xh"], bias)
+    return {"xt": xt, "xh": sq["xh"], "xl": xl, "codes": sq["codes"], "sf": sq["sf"], "t": sq["t"], "y64": y64, "y": yb}
+
+
 # ---------------------------------------------------------------------------------------------
 # GPTQ rounding of the residual weight (Sec. 4.1: the rounding minimises ||X W - X W^||_F^2 rather than the
 # layer-wise surrogate; App. F.1: damping 0.01, block size 128).  The steps are those of the published GPTQ

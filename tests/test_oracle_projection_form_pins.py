@@ -92,3 +92,31 @@ def test_error_matches_the_dense_rotation_and_the_projection_is_what_removes_the
     print(e_paper, e_proj, e_none)
     assert 0.8 < e_proj / e_paper < 1.25          # same error as the paper's dense rotation on these activations
     assert e_none > 3.0 * e_proj                  # a Hadamard alone does not remove the planted outlier directions
+
+
+def test_nvfp4_projection_form_shares_the_decomposition_and_matches_the_dense_form():
+    spec = synth.LayerSpec(K=256, N=64, r=32, G=64, model=synth.PIXART, seed=6, calib_tokens=1024)
+    inp = synth.make_layer_inputs(spec, 48, with_bias=True)
+    Q = np.asarray(inp["Q"], dtype=np.float64)
+    x = _bf(inp["x"])
+    lay = orc.nvfp4_prepare_layer_ph(inp["W"], np.ascontiguousarray(Q[:, :spec.r]), want_t=True)
+    xh_bits, xl = orc.nvfp4_residual(inp["x"], lay)
+    Uhb = _bf(lay["Uhb"])
+    # same exact decomposition as the INT4 projection form, Hadamard blocks of 64
+    assert np.allclose(_bf(xh_bits) @ Uhb.T + orc.block_hadamard_cols(xl, 64), x, atol=1e-12 * np.abs(x).max())
+    ex = orc.nvfp4_global_exponent(float(np.abs(xl).max()))
+    out = orc.nvfp4_linear_deployed_ph(inp["x"], lay, ex, bias=inp["bias"])
+    # block-scaled product = dequantize-then-multiply of the codes it returns
+    mag = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float64)
+    deq = lambda c: np.where(c & 8, -1.0, 1.0) * mag[c & 7]
+    xs = np.repeat(orc.e4m3_to_f64(out["sf"]), 16, axis=1) * 2.0 ** ex * deq(out["codes"])
+    ws = np.repeat(orc.e4m3_to_f64(lay["wsf"]), 16, axis=0) * 2.0 ** lay["ew"] * deq(lay["wcodes"])
+    ref = xs @ ws + _bf(out["xh"]) @ _bf(lay["Wh"]) + _bf(inp["bias"])[None, :]
+    assert np.allclose(out["y64"], ref, rtol=1e-9, atol=1e-9)
+    # and its error is that of the dense NVFP4 form on these activations
+    ideal = x @ np.asarray(inp["W"], dtype=np.float64) + _bf(inp["bias"])[None, :]
+    lo = orc.nvfp4_prepare_layer(inp["W"], inp["Q"], spec.r)
+    ex2 = orc.nvfp4_global_exponent(float(np.abs(orc.rotate(inp["x"], lo["Qb"])[:, spec.r:]).max()))
+    dense = orc.nvfp4_linear_deployed(inp["x"], lo, ex2, bias=inp["bias"])
+    e = lambda y: float(np.sqrt(np.mean((y - ideal) ** 2) / np.mean(ideal ** 2)))
+    assert 0.8 < e(out["y64"]) / e(dense["y64"]) < 1.25
