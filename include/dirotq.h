@@ -244,6 +244,15 @@ DIROTQ_API dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, i
                                                    const void* bias, int K, int N, int r, int group, void* blob,
                                                    size_t blob_bytes, void* scratch, size_t scratch_bytes,
                                                    dirotq_stream_t stream, dirotq_layer_t** layer_out);
+/* The projection form with NVFP4 operands (as dirotq_prepare_layer_nvfp4, with Uh in place of Q; Hadamard blocks of 64,
+ * E2M1 blocks of 16).  Accepted by the same calls as an NVFP4 layer; q_bf16 of dirotq_layer_export_nvfp4 and xrot_f32 of
+ * dirotq_rotate_quantize must be NULL; scratch: dirotq_prepare_scratch_bytes_ph bytes. */
+DIROTQ_API dirotq_status_t dirotq_layer_bytes_nvfp4_ph(int K, int N, int r, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_nvfp4_ph(const void* W, int w_dtype, int w_layout, const void* Uh,
+                                                         int uh_dtype, const void* bias, int K, int N, int r,
+                                                         int act_scale_log2, void* blob, size_t blob_bytes, void* scratch,
+                                                         size_t scratch_bytes, dirotq_stream_t stream,
+                                                         dirotq_layer_t** layer_out);
 /* uh_bf16 [K,r]: the rounded projection the layer applies. */
 DIROTQ_API dirotq_status_t dirotq_layer_export_uh(const dirotq_layer_t* layer, void* uh_bf16, dirotq_stream_t stream);
 

@@ -30,7 +30,7 @@ EXPORTED = [
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
     "dirotq_prepare_layer_codes", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
-    "dirotq_layer_export_uh", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_layer_export_uh", "dirotq_layer_bytes_nvfp4_ph", "dirotq_prepare_layer_nvfp4_ph", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.dirotq_prepare_scratch_bytes_ph.argtypes = [i, i, i, ctypes.POINTER(sz)]
         L.dirotq_prepare_layer_ph.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_layer_export_uh.argtypes = [vp, vp, vp]
+        L.dirotq_layer_bytes_nvfp4_ph.argtypes = [i, i, i, ctypes.POINTER(sz)]
+        L.dirotq_prepare_layer_nvfp4_ph.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_set_gemm_tile.argtypes = [i]
         L.dirotq_set_dependent_launch.argtypes = [i]
         L.dirotq_set_rotation_tile.argtypes = [i]
@@ -135,7 +137,7 @@ class Layer:
         self.handle, self.blob = handle, blob
         self.K, self.N, self.r, self.group = K, N, r, group
         self.fmt = fmt
-        self.K_l = K if fmt == "int4_ph" else K - r      # projection form: all K residual coefficients are low-precision
+        self.K_l = K if fmt in ("int4_ph", "nvfp4_ph") else K - r      # projection form: all K residual coefficients are low-precision
         self.n_g = -(-self.K_l // group)
         self.K_lp = self.n_g * group
 
@@ -330,10 +332,13 @@ def dirotq_layer_export_nvfp4(layer: Layer, stream=None):
     wcodes = torch.empty((layer.K_l, layer.N), dtype=torch.uint8, device=dev)
     wscales = torch.empty((nb, layer.N), dtype=torch.uint8, device=dev)
     wh = torch.empty((layer.r, layer.N), dtype=torch.bfloat16, device=dev)
-    qb = torch.empty((layer.K, layer.K), dtype=torch.bfloat16, device=dev)
+    # the projection form holds U_hb instead of a K x K rotation: returned in the rotation's place
+    qb = None if layer.fmt == "nvfp4_ph" else torch.empty((layer.K, layer.K), dtype=torch.bfloat16, device=dev)
     ew = torch.zeros(1, dtype=torch.int32, device=dev)
     _check(lib().dirotq_layer_export_nvfp4(layer.handle, wcodes.data_ptr(), wscales.data_ptr(), wh.data_ptr(),
-                                           qb.data_ptr(), ew.data_ptr(), _stream(stream)), "dirotq_layer_export_nvfp4")
+                                           _ptr(qb), ew.data_ptr(), _stream(stream)), "dirotq_layer_export_nvfp4")
+    if qb is None:
+        qb = dirotq_layer_export_uh(layer, stream)
     return wcodes, wscales, wh, qb, int(ew.item())
 
 
@@ -411,6 +416,28 @@ def dirotq_prepare_layer_ph(W: torch.Tensor, Uh: torch.Tensor, group: int, bias:
     _check(st, "dirotq_prepare_layer_ph")
     torch.cuda.current_stream().synchronize()
     return Layer(handle.value, blob, K, N, r, group, fmt="int4_ph")
+
+
+def dirotq_prepare_layer_nvfp4_ph(W: torch.Tensor, Uh: torch.Tensor, act_scale_log2: int, bias: torch.Tensor | None = None,
+                                  w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """Projection form with NVFP4 operands."""
+    assert W.is_cuda and Uh.is_cuda and W.is_contiguous() and Uh.is_contiguous()
+    K, r = Uh.shape
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    uh_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Uh.dtype]
+    nb, ns = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(lib().dirotq_layer_bytes_nvfp4_ph(K, N, r, ctypes.byref(nb)), "dirotq_layer_bytes_nvfp4_ph")
+    _check(lib().dirotq_prepare_scratch_bytes_ph(K, N, r, ctypes.byref(ns)), "dirotq_prepare_scratch_bytes_ph")
+    blob = _alloc_bytes(nb.value, W.device)
+    scratch = _alloc_bytes(ns.value, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_nvfp4_ph(_ptr(W), w_dtype, w_layout, _ptr(Uh), uh_dtype, _ptr(bias), K, N, r,
+                                             int(act_scale_log2), blob.data_ptr(), blob.numel(), scratch.data_ptr(), ns.value,
+                                             _stream(stream), ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_nvfp4_ph")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, 16, fmt="nvfp4_ph")
 
 
 def dirotq_layer_export_uh(layer: Layer, stream=None) -> torch.Tensor:

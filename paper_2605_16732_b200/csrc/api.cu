@@ -365,7 +365,7 @@ dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout
 }
 
 dirotq_status_t dirotq_layer_export_uh(const dirotq_layer_t* layer, void* uh_bf16, dirotq_stream_t stream) {
-    if (!valid_layer(layer) || layer->geo.fmt != 4 || !uh_bf16) return DIROTQ_ERR_INVALID_ARG;
+    if (!valid_layer(layer) || !layer->geo.ph || !uh_bf16) return DIROTQ_ERR_INVALID_ARG;
     return launch_uh_export(layer, static_cast<uint16_t*>(uh_bf16), static_cast<cudaStream_t>(stream));
 }
 
@@ -513,7 +513,7 @@ static RotateArgs rotate_args(const dirotq_layer_t* layer, const void* x, int M,
 // First kernel(s): rotation + split + quantization.  W4A8 needs the token's whole row before it can quantize: the rotation
 // kernel writes fp32 coefficients and the row maxima, a second small kernel quantizes.
 static dirotq_status_t first_kernel(const dirotq_layer_t* layer, const RotateArgs& ra, int M, cudaStream_t s) {
-    if (layer->geo.fmt == 4) return launch_project_quantize(layer, ra, s);
+    if (layer->geo.ph) return launch_project_quantize(layer, ra, s);
     if (layer->geo.fmt == 3) {
         if (cudaMemsetAsync(ra.rowmax, 0, static_cast<size_t>(M) * 4, s) != cudaSuccess) return DIROTQ_ERR_CUDA;
         dirotq_status_t st = launch_rotate_quantize(layer, ra, s);
@@ -806,9 +806,72 @@ dirotq_status_t dirotq_workspace_export_nvfp4(const dirotq_layer_t* layer, int M
                                          scales_e4m3, static_cast<cudaStream_t>(stream));
 }
 
+dirotq_status_t dirotq_layer_bytes_nvfp4_ph(int K, int N, int r, size_t* bytes) {
+    if (!bytes) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, 64);
+    if (st != DIROTQ_OK) return st;
+    Geometry g = make_geometry(K, N, r, 64);
+    make_ph_nvfp4(g);
+    *bytes = make_blob_layout_nvfp4(g).total;
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_nvfp4_ph(const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                              const void* bias, int K, int N, int r, int act_scale_log2, void* blob,
+                                              size_t blob_bytes, void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                              dirotq_layer_t** layer_out) {
+    if (!W || !Uh || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
+    if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
+    if (uh_dtype != DIROTQ_DTYPE_F64 && uh_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
+    if (w_layout != DIROTQ_LAYOUT_KN && w_layout != DIROTQ_LAYOUT_NK) return DIROTQ_ERR_INVALID_ARG;
+    if (act_scale_log2 < -100 || act_scale_log2 > 100) return DIROTQ_ERR_INVALID_ARG;
+    dirotq_status_t st = check_shape(K, N, r, 64);
+    if (st != DIROTQ_OK) return st;
+    if (!aligned16(W) || !aligned16(Uh) || !aligned16(scratch) || (bias && !aligned16(bias))) return DIROTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blob) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
+    Geometry g = make_geometry(K, N, r, 64);
+    make_ph_nvfp4(g);
+    const BlobLayout lay = make_blob_layout_nvfp4(g);
+    if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (scratch_bytes < (static_cast<size_t>(K) + r) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    int dev = 0;
+    st = check_device(&dev);
+    if (st != DIROTQ_OK) return st;
+    dirotq_layer* L = new (std::nothrow) dirotq_layer;
+    if (!L) return DIROTQ_ERR_INVALID_ARG;
+    memset(L, 0, sizeof *L);
+    L->magic = kLayerMagic;
+    L->device = dev;
+    L->geo = g;
+    L->lay = lay;
+    L->blob = static_cast<char*>(blob);
+    L->act_scale_log2 = act_scale_log2;
+    st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K,
+                        (uint64_t)g.r_pad, (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_uh, (uint64_t)g.r_pad,
+                            (uint64_t)K, (uint64_t)g.r_pad * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked, (uint64_t)g.K4 / 2,
+                            (uint64_t)N, (uint64_t)g.K4 / 2, 128, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = launch_prepare_nvfp4_ph(L, W, w_dtype, w_layout, Uh, uh_dtype, bias, static_cast<double*>(scratch),
+                                     static_cast<cudaStream_t>(stream));
+    if (st != DIROTQ_OK) {
+        delete L;
+        return st;
+    }
+    *layer_out = L;
+    return DIROTQ_OK;
+}
+
 dirotq_status_t dirotq_layer_export_nvfp4(const dirotq_layer_t* layer, uint8_t* wcodes, uint8_t* wscales_e4m3, void* wh_bf16,
                                           void* q_bf16, int* weight_scale_log2, dirotq_stream_t stream) {
     if (!valid_layer(layer) || layer->geo.fmt != 1) return DIROTQ_ERR_INVALID_ARG;
+    if (q_bf16 && layer->geo.ph) return DIROTQ_ERR_INVALID_ARG;  // no K x K rotation in the blob
     return launch_layer_export_nvfp4(layer, wcodes, wscales_e4m3, static_cast<uint16_t*>(wh_bf16),
                                      static_cast<uint16_t*>(q_bf16), weight_scale_log2, static_cast<cudaStream_t>(stream));
 }

@@ -34,6 +34,7 @@ struct Geometry {
     int K4;      // K_l rounded up to 64 (<= K): width of the packed E2M1 rows
     int nkb64;   // K4 / 64: scale-factor atoms (128 rows x 4 scales) per row block
     int nkb64p;  // nkb64 rounded up to 4: one TMA k-block = 256 elements = 4 atoms
+    int ph;      // 1: projection form in front of the format's quantizer (fmt 4 is ph with the INT4 quantizer; fmt 1 + ph is NVFP4)
     int no_rot;  // 1: the blob holds no rotation (a layer that only consumes a workspace rotated through a sibling layer)
 };
 
@@ -50,6 +51,7 @@ inline Geometry make_geometry(int K, int N, int r, int G) {
     g.nkb64 = g.K4 / 64;
     g.nkb64p = (g.nkb64 + 3) / 4 * 4;
     g.no_rot = 0;
+    g.ph = 0;
     return g;
 }
 
@@ -59,9 +61,18 @@ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a
 // Projection form (fmt 4): every one of the K residual coefficients is low-precision.
 inline void make_ph(Geometry& g) {
     g.fmt = 4;
+    g.ph = 1;
     g.K_l = g.K;
     g.n_g = g.K / g.G;
     g.K_lp = g.K;
+}
+// ... and with NVFP4 operands (G = 64 is then the Hadamard block and the epilogue's chunk)
+inline void make_ph_nvfp4(Geometry& g) {
+    make_ph(g);
+    g.fmt = 1;
+    g.K4 = g.K;
+    g.nkb64 = g.K / 64;
+    g.nkb64p = (g.nkb64 + 3) / 4 * 4;
 }
 
 // Sections of the device blob that holds a prepared layer.
@@ -103,8 +114,8 @@ inline BlobLayout make_blob_layout(const Geometry& g) {
 inline BlobLayout make_blob_layout_nvfp4(const Geometry& g) {
     BlobLayout b;
     size_t o = 0;
-    b.off_qt = o;      o = align_up(o + (size_t)g.K * g.K * 2);
-    b.off_uh = o;
+    b.off_qt = o;      o = align_up(o + (g.ph ? (size_t)g.r_pad * g.K * 2 : (size_t)g.K * g.K * 2));
+    b.off_uh = o;      o = align_up(o + (g.ph ? (size_t)g.K * g.r_pad * 2 : 0));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K4 / 2));
     b.off_wscale = o;  o = align_up(o + (size_t)((g.N + 127) / 128) * g.nkb64p * 512);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
@@ -266,6 +277,8 @@ dirotq_status_t set_rotation_plan(int plan);
 dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
                                   const void* bias, double* scratch, cudaStream_t stream);
 dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, cudaStream_t stream);
+dirotq_status_t launch_prepare_nvfp4_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                        const void* bias, double* scratch, cudaStream_t stream);
 dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);
 struct Nvfp4GemmArgs {
     int M;

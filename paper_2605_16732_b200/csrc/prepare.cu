@@ -415,7 +415,7 @@ struct Nvfp4Meta {
 
 __global__ void nvfp4_amax_kernel(const double* Wt, Geometry g, Nvfp4Meta* meta) {
     double a = 0.0;
-    const size_t lo = static_cast<size_t>(g.r) * g.N, hi = static_cast<size_t>(g.K) * g.N;
+    const size_t lo = static_cast<size_t>(g.r) * g.N, hi = static_cast<size_t>(g.r + g.K_l) * g.N;  // the low rows of the scratch
     for (size_t i = lo + blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < hi;
          i += static_cast<size_t>(gridDim.x) * blockDim.x)
         a = fmax(a, fabs(Wt[i]));
@@ -775,6 +775,40 @@ dirotq_status_t launch_prepare_nvfp4(const dirotq_layer* L, const void* W, int w
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     rotation_kernel<<<dim3((g.K + 31) / 32, (g.K + 31) / 32), dim3(32, 8), 0, stream>>>(
         Q, q_dtype, reinterpret_cast<uint16_t*>(blob + L->lay.off_qt), g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                       reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
+dirotq_status_t launch_prepare_nvfp4_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
+                                        const void* bias, double* scratch, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    char* blob = L->blob;
+    Nvfp4Meta* meta = reinterpret_cast<Nvfp4Meta*>(blob + L->lay.off_meta);
+    uint16_t* uht = reinterpret_cast<uint16_t*>(blob + L->lay.off_qt);
+    uint16_t* uh = reinterpret_cast<uint16_t*>(blob + L->lay.off_uh);
+    ph_round_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(Uh, uh_dtype, uht, uh, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_fold_high_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(uh, W, w_dtype, w_layout, scratch, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_fold_low_kernel<<<dim3((g.N + 127) / 128, g.K), 128, 0, stream>>>(W, w_dtype, w_layout, scratch, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    // the scratch now holds [r + K][N]: quantized exactly like the dense form's folded weight
+    if (cudaMemsetAsync(meta, 0, 64, stream) != cudaSuccess) return DIROTQ_ERR_CUDA;
+    if (cudaMemsetAsync(blob + L->lay.off_wscale, 0, static_cast<size_t>((g.N + 127) / 128) * g.nkb64p * 512, stream) !=
+        cudaSuccess)
+        return DIROTQ_ERR_CUDA;
+    nvfp4_amax_kernel<<<592, 256, 0, stream>>>(scratch, g, meta);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    nvfp4_meta_kernel<<<1, 1, 0, stream>>>(meta, L->act_scale_log2);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    nvfp4_quantize_weights_kernel<<<dim3((g.N + 127) / 128, g.nkb64), 128, 0, stream>>>(
+        scratch, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<uint8_t*>(blob + L->lay.off_wscale),
+        meta, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    nvfp4_high_rows_kernel<<<(g.N + 127) / 128, 128, 0, stream>>>(scratch, reinterpret_cast<uint16_t*>(blob + L->lay.off_wh),
+                                                                  meta, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     bias_kernel<<<(g.N + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
                                                        reinterpret_cast<float*>(blob + L->lay.off_bias), g.N);

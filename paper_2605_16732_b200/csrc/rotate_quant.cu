@@ -154,7 +154,8 @@ __device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float ex_inv, 
     return sb;
 }
 
-template <int G, int FMT, int BN, int BM>
+// PH: the epilogue first forms the projection form's residual (FMT 4 is PH with the INT4 quantizer of FMT 0).
+template <int G, int FMT, int BN, int BM, bool PH = (FMT == 4)>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
                     const RotKernelParams p) {
@@ -296,7 +297,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             // first one before the accumulator wait) so that the load's latency is not paid per chunk
             [[maybe_unused]] uint4 xq[G / 8];
             [[maybe_unused]] const int chunk_first = BM == 256 ? 0 : half * CPH;
-            if constexpr (FMT == 4) {
+            if constexpr (PH) {
                 if (row_ok && n0 + chunk_first * G < p.n_out) {
                     const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + n0 + chunk_first * G);
 #pragma unroll
@@ -333,7 +334,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                                                  v[16 * b + 4 * j + 3]);
                     }
                 }
-                if constexpr (FMT == 4) {
+                if constexpr (PH) {
                     // projection form: v = x - x~_h U_hb^T (the accumulator holds the product), then the group's
                     // Hadamard block in registers; what follows quantizes it like any other group
                     if (row_ok) {
@@ -499,7 +500,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
-            if (FMT != 4 && n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
+            if (!PH && n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
                 for (int c = p.r; c < p.r_pad0; c += 8)
                     *reinterpret_cast<uint4*>(p.xh + static_cast<size_t>(row) * p.r_pad + c) = make_uint4(0, 0, 0, 0);
                 if constexpr (FMT == 2) {  // behind the 3 n_g zero-point columns
@@ -625,11 +626,15 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
         if (st != DIROTQ_OK) return st;
         RotKernelParams p2 = p;
         p2.n_out = g.K; p2.k_red = g.r_pad; p2.K_l = g.K; p2.r = g.r; p2.xsub = static_cast<const uint16_t*>(a.x);
-        const KernelFn k2 = g.G == 64 ? rotate_quant_kernel<64, 4, 256, 128> : rotate_quant_kernel<128, 4, 256, 128>;
-        static bool attr2[2] = {false, false};
-        if (!attr2[g.G == 64 ? 0 : 1]) {
+        const int vi = g.fmt == 1 ? 2 : (g.G == 64 ? 0 : 1);
+        static const KernelFn k2s[3] = {rotate_quant_kernel<64, 4, 256, 128>, rotate_quant_kernel<128, 4, 256, 128>,
+                                        rotate_quant_kernel<64, 1, 256, 128, true>};
+        const KernelFn k2 = k2s[vi];
+        if (g.fmt == 1) { p2.xsf = a.xsf; p2.K4 = g.K4; p2.nkb64p = g.nkb64p; p2.ex = L->act_scale_log2; }
+        static bool attr2[3] = {false, false, false};
+        if (!attr2[vi]) {
             if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return DIROTQ_ERR_CUDA;
-            attr2[g.G == 64 ? 0 : 1] = true;
+            attr2[vi] = true;
         }
         const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.K + 255) / 256);
         if (launch_kernel(k2, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_xh, L->tmap_qt,

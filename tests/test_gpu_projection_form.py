@@ -168,3 +168,65 @@ def test_projection_form_through_the_other_entry_points():
     with pytest.raises(dq.DirotqError):
         dq.dirotq_rotate_quantize(x, layer, ws, torch.empty((M, spec.K), dtype=torch.float32, device=dev))
     layer.close()
+
+
+# ------------------------------------------------------------------ NVFP4 operands behind the projection form
+
+from parity_utils import check_activation_side_nvfp4, check_layer_output_nvfp4, check_weight_side_nvfp4
+
+
+def _run_case_nvfp4(spec: synth.LayerSpec, M: int, with_bias=True):
+    inp = synth.make_layer_inputs(spec, M, with_bias=with_bias)
+    Uh = np.ascontiguousarray(np.asarray(inp["Q"], dtype=np.float64)[:, :spec.r])
+    lo = orc.nvfp4_prepare_layer_ph(inp["W"], Uh, want_t=True)
+    _, xl = orc.nvfp4_residual(inp["x"], lo)
+    ex = orc.nvfp4_global_exponent(float(np.abs(xl).max()))          # calibration of the power-of-two scale: this batch
+    oo = orc.nvfp4_linear_deployed_ph(inp["x"], lo, ex, bias=inp["bias"])
+
+    dev = "cuda"
+    bias = bits_to_bf16_tensor(inp["bias"]) if with_bias else None
+    layer = dq.dirotq_prepare_layer_nvfp4_ph(torch.from_numpy(inp["W"]).to(dev), torch.from_numpy(Uh).to(dev), ex, bias=bias)
+    lo_chk = dict(lo)
+    lo_chk["Qb"] = lo["Uhb"]                 # the export returns U_hb in the rotation's place
+    stats = check_weight_side_nvfp4(dq.dirotq_layer_export_nvfp4(layer), lo_chk)
+
+    x = bits_to_bf16_tensor(inp["x"])
+    ws = dq.alloc_workspace(layer, M)
+    y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, sf = dq.dirotq_workspace_export_nvfp4(layer, M, ws)
+    xh_b, codes_n, sf_n = bf16_tensor_to_bits(xh), codes.cpu().numpy(), sf.cpu().numpy()
+    assert codes_n.shape == (M, spec.K)
+    # codes and block scales against the reference's second step on the library's own x~_h (the residual is defined
+    # through the rounded x~_h), with the NVFP4 protocol
+    _, xl_ref = orc.nvfp4_residual(inp["x"], lo, xh_bits=xh_b)
+    xt_ref = np.ascontiguousarray(np.concatenate([orc.bf16_to_f64(xh_b), xl_ref], axis=1))
+    sq_ref = orc.nvfp4_split_quantize(xt_ref, spec.r, ex, want_t=True)
+    prot = {"xt": xt_ref, "xh": sq_ref["xh"], "codes": sq_ref["codes"], "sf": sq_ref["sf"], "t": sq_ref["t"]}
+    stats.update(check_activation_side_nvfp4(None, xh_b, codes_n, sf_n, prot, spec.r, ex))
+    xh_g, xh_o = orc.bf16_to_f64(xh_b), orc.bf16_to_f64(oo["xh"])
+    xnorm = np.linalg.norm(orc.bf16_to_f64(inp["x"]), axis=1, keepdims=True)
+    assert np.all(np.abs(xh_g - xh_o) <= np.maximum(np.abs(xh_o), 2.0 ** -126) * 2.0 ** -7 + 1e-5 * xnorm)
+    stats.update(check_layer_output_nvfp4(bf16_tensor_to_bits(y), xh_b, codes_n, sf_n, ex, lo, oo, inp["bias"]))
+    y2 = torch.zeros_like(y)
+    dq.dirotq_linear(x, layer, y2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    layer.close()
+    return stats
+
+
+def test_nvfp4_projection_form_small():
+    spec = synth.LayerSpec(K=256, N=256, r=32, G=64, model=synth.PIXART, seed=111, calib_tokens=512)
+    print(_run_case_nvfp4(spec, M=100))
+
+
+def test_nvfp4_projection_form_pixart_projection():
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=112)
+    print(_run_case_nvfp4(spec, M=256))
+
+
+def test_nvfp4_projection_form_ragged_rank64_no_bias():
+    spec = synth.LayerSpec(K=768, N=400, r=64, G=64, model=synth.FLUX, seed=113, calib_tokens=1024)
+    print(_run_case_nvfp4(spec, M=300, with_bias=False))
