@@ -128,6 +128,9 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
             lo["ex"] = orc.nvfp4_global_exponent(float(np.abs(orc.rotate(x, lo["Qb"])[:, RANK:]).max()))
         elif fmt == "int4_ph":
             lo = orc.prepare_layer_ph(W, np.ascontiguousarray(Q[:, :RANK]), GROUP)
+        elif fmt == "nvfp4_ph":
+            lo = orc.nvfp4_prepare_layer_ph(W, np.ascontiguousarray(Q[:, :RANK]))
+            lo["ex"] = orc.nvfp4_global_exponent(float(np.abs(orc.nvfp4_residual(x, lo)[1]).max()))
         else:
             lo = orc.prepare_layer(W, Q, RANK, GROUP)
         layers.append((lo, x, K, cols))
@@ -143,6 +146,8 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
                 orc.linear_deployed_w4a8(x, lo, bias=None, want_t=False)
             elif fmt == "int4_ph":
                 orc.linear_deployed_ph(x, lo, bias=None, want_t=False)
+            elif fmt == "nvfp4_ph":
+                orc.nvfp4_linear_deployed_ph(x, lo, lo["ex"], bias=None, want_t=False)
             else:
                 orc.linear_deployed(x, lo, bias=None, want_t=False)
         times.append(time.perf_counter() - t0)
@@ -150,8 +155,13 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
     t = float(np.mean(times))
     return {"value": ops / t / 1e12, "unit": "TOPS", "cores": orc.num_threads(), "kind": "oracle",
             "sample": f"{rows} token rows x {cols} output columns of each of the 4 linears, online steps only "
-                      f"(rotation, quantize, {'block-scaled products' if fmt == 'nvfp4' else 'int GEMM'}, combine); Householder rotation",
+                      f"(rotation, quantize, {'block-scaled products' if fmt in ('nvfp4', 'nvfp4_ph') else 'int GEMM'}, combine); Householder rotation",
             "seconds_per_step": t}
+
+
+def _suffix(fmt):
+    return {"nvfp4": "_nvfp4", "int4_asym": "_asym", "w4a8": "_w4a8", "int4_ph": "_projection_form",
+            "nvfp4_ph": "_projection_form_nvfp4"}.get(fmt, "")
 
 
 def run_reference(args):
@@ -166,8 +176,8 @@ def run_reference(args):
         "impl": "reference", "metric": "dirotq_w4a4_linear_effective_tops", "value": res["value"], "unit": "TOPS",
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64 (oracle; nvfp4 codes)" if args.fmt == "nvfp4" else "f64 + int32 (oracle; int4 codes)",
-        "data": "synthetic", "config": {"workload": WORKLOAD + ("_nvfp4" if args.fmt == "nvfp4" else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else "_projection_form" if args.fmt == "int4_ph" else ""),
+        "dtype": "f64 (oracle; nvfp4 codes)" if args.fmt in ("nvfp4", "nvfp4_ph") else "f64 + int32 (oracle; int4 codes)",
+        "data": "synthetic", "config": {"workload": WORKLOAD + _suffix(args.fmt),
                                         "format": args.fmt,
                                         "sample": res["sample"]},
         "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
@@ -184,6 +194,7 @@ def run_reference(args):
 def run_ours(args):
     import torch
     from paper_2605_16732_b200 import binding as dq
+    from paper_2605_16732_b200.suite import residual_exponent
     from paper_2605_16732_b200 import synth
     from paper_2605_16732_b200.shard import aggregate_throughput, max_over_ranks
 
@@ -228,6 +239,9 @@ def run_ours(args):
             layer = dq.dirotq_prepare_layer_asym(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         elif args.fmt == "int4_ph":
             layer = dq.dirotq_prepare_layer_ph(torch.from_numpy(W).to(dev), Q[:, :RANK].contiguous(), GROUP, bias=bf(bias))
+        elif args.fmt == "nvfp4_ph":
+            Uh = Q[:, :RANK].contiguous()
+            layer = dq.dirotq_prepare_layer_nvfp4_ph(torch.from_numpy(W).to(dev), Uh, residual_exponent(x, Uh), bias=bf(bias))
         else:
             layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         del Q
@@ -348,11 +362,11 @@ def run_ours(args):
     rot_ms = {n: float(np.mean(v["rotate_ms"])) for n, v in per.items()}
     gemm_ms = {n: float(np.mean(v["gemm_ms"])) for n, v in per.items()}
     rot_total, gemm_total = sum(rot_ms.values()), sum(gemm_ms.values())
-    ph = args.fmt == "int4_ph"
+    ph = args.fmt in ("int4_ph", "nvfp4_ph")
     # projection form: two skinny GEMMs on a 64-wide padded rank instead of the K x K rotation; all K columns are 4-bit
     rot_flops = {n: (4.0 * M * K * 64 if ph else 2.0 * M * K * K) for n, K, _ in FLUX_SHAPES}
     gemm_ops = {n: 2.0 * M * (K if ph else K - RANK) * N for n, K, N in FLUX_SHAPES}
-    nv = args.fmt == "nvfp4"
+    nv = args.fmt in ("nvfp4", "nvfp4_ph")
     # nominal ratios of the part: 8-bit (int8 / fp8) 2x and fp4 4x the dense bf16 rate (4.5 and 9 : 2.25 PFLOP/s)
     int8_peak = (4.0 if nv else 2.0) * peaks["bf16_sustained"]
     # DRAM bytes of one launch of the dominant kernel, from the ncu capture summarised under profiles/
@@ -402,14 +416,14 @@ def run_ours(args):
         "dtype": ("nvfp4 (e2m1 x e2m1, e4m3 block scales) + bf16" if nv else "int8xint4->int32 + bf16" if args.fmt == "w4a8"
                   else "int4xint4 (exact group sums on the e4m3 tensor path) + bf16"),
         "data": "synthetic",
-        "config": {"workload": WORKLOAD + ("_nvfp4" if nv else "_asym" if args.fmt == "int4_asym" else "_w4a8" if args.fmt == "w4a8" else "_projection_form" if args.fmt == "int4_ph" else ""), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
+        "config": {"workload": WORKLOAD + _suffix(args.fmt), "M": M, "shapes": [[K, N] for _, K, N in FLUX_SHAPES], "r": RANK,
                    "group": 16 if nv else ("per-token / per-channel" if args.fmt == "w4a8" else GROUP), "format": args.fmt,
                    "l2": "inputs_exceed_l2 (each step streams > 500 MB of rotations, codes and outputs)",
                    "parallelism": f"token rows x{world}, no collective"},
         "clocks": clocks,
         "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-        "gpu_launches": (3 if args.fmt == "w4a8" else 2) * len(layers) * args.steps,
+        "gpu_launches": (3 if args.fmt == "w4a8" or ph else 2) * len(layers) * args.steps,
         "roofline": roofline,
         "kernels": kernels,
         "frac_int8_peak_effective": value / world / int8_peak,
@@ -427,7 +441,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shapes", default="", help="comma-separated subset of qkv,out,mlp_up,mlp_down (profiling runs)")
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8", "int4_ph"],
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8", "int4_ph", "nvfp4_ph"],
                     help="int4: the headline format (groups of 64, bf16 scales, symmetric); nvfp4: E2M1 blocks of 16 with E4M3 "
                          "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group); w4a8: per-token int8 "
                          "activations, per-channel int4 weights; int4_ph: the projection form (U_h only + block-Hadamard residual), "

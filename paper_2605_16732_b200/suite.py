@@ -47,6 +47,19 @@ def _householder(K: int, seed: int) -> torch.Tensor:
 FMT = "int4"  # set from --fmt: "int4" (groups of G, bf16 scales) or "nvfp4" (blocks of 16, E4M3 scales)
 
 
+def residual_exponent(x, Uh, rows=1024):
+    """Offline calibration of the NVFP4 projection form's power-of-two activation scale (App. E): the largest
+    Hadamard-rotated residual coefficient of the first `rows` tokens, taken with plain torch ops."""
+    xs = x[:rows].float()
+    Ub = Uh.to(torch.bfloat16).float()
+    d = xs - (xs @ Ub).to(torch.bfloat16).float() @ Ub.t()
+    H = torch.ones((1, 1), device=x.device)
+    while H.shape[0] < 64:
+        H = torch.cat([torch.cat([H, H], 1), torch.cat([H, -H], 1)], 0)
+    amax = float(((d.view(d.shape[0], -1, 64) @ H) / 8.0).abs().max().item())
+    return int(np.ceil(np.log2(amax / 1536.0)))
+
+
 class Case:
     def __init__(self, M, K, N, r, G, model):
         self.M, self.K, self.N, self.r, self.G = M, K, N, r, G
@@ -70,6 +83,9 @@ class Case:
             self.layer = dq.dirotq_prepare_layer_asym(Wd, Q, r, G, bias=_bf(bias))
         elif FMT == "int4_ph":
             self.layer = dq.dirotq_prepare_layer_ph(Wd, Q[:, :r].contiguous(), G, bias=_bf(bias))
+        elif FMT == "nvfp4_ph":
+            Uh = Q[:, :r].contiguous()
+            self.layer = dq.dirotq_prepare_layer_nvfp4_ph(Wd, Uh, residual_exponent(self.x, Uh), bias=_bf(bias))
         else:
             self.layer = dq.dirotq_prepare_layer(Wd, Q, r, G, bias=_bf(bias))
         self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
@@ -133,15 +149,16 @@ class Case:
     def report(self, tag, iters, p_bf16, hbm, graphs=False):
         rot, gem, cb = self.time_kernels(iters)
         M, K, N, r, G = self.M, self.K, self.N, self.r, self.G
-        K_l = K if FMT == "int4_ph" else K - r
+        PH, NV = FMT in ("int4_ph", "nvfp4_ph"), FMT in ("nvfp4", "nvfp4_ph")
+        K_l = K if PH else K - r
         n_g = -(-K_l // G) if G else 1
         tot = rot + gem
-        p_i8 = (4.0 if FMT == "nvfp4" else 2.0) * p_bf16  # nominal ratio of the 4-bit / 8-bit tensor peak to bf16
-        first_flops = 4.0 * M * K * max(64, -(-r // 64) * 64) if FMT == "int4_ph" else 2.0 * M * K * K
+        p_i8 = (4.0 if NV else 2.0) * p_bf16  # nominal ratio of the 4-bit / 8-bit tensor peak to bf16
+        first_flops = 4.0 * M * K * max(64, -(-r // 64) * 64) if PH else 2.0 * M * K * K
         t_roof = (2.0 * M * K_l * N / p_i8 + (first_flops + 2.0 * M * r * N) / p_bf16) / 1e12 * 1e3
         if FMT == "w4a8":
             bytes_alg = 2 * M * K + 2 * K * K + K_l * N / 2 + 4 * N + 2 * 64 * N + 2 * (M * K_l * 5 + 8 * M + 2 * M * 64) + 2 * M * N
-        elif FMT == "nvfp4":
+        elif NV:
             bytes_alg = 2 * M * K + 2 * K * K + K_l * N / 2 + K_l / 16 * N + 2 * 64 * N + 2 * (M * K_l / 2 + M * K_l / 16 + 2 * M * 64) + 2 * M * N
         else:
             bytes_alg = 2 * M * K + 2 * K * K + n_g * G * N / 2 + 4 * n_g * N + 2 * 64 * N + 2 * (M * n_g * G + 4 * M * n_g + 2 * M * 64) + 2 * M * N
@@ -182,7 +199,7 @@ def main():
     ap.add_argument("--memory", action="store_true", help="print the layer sizes (no GPU needed) and exit")
     ap.add_argument("--configs", default="1,2,4,5", help="comma-separated subset of 1,2,3p,4,5")
     ap.add_argument("--iters", type=int, default=20)
-    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8", "int4_ph"])
+    ap.add_argument("--fmt", default="int4", choices=["int4", "nvfp4", "int4_asym", "w4a8", "int4_ph", "nvfp4_ph"])
     ap.add_argument("--ranks", default="16,32,64,128", help="ranks swept by config 4")
     args = ap.parse_args()
     if args.memory:
@@ -238,7 +255,7 @@ def main():
     if "4" in todo:
         for K, N in [(3072, 9216), (12288, 3072)]:
             for r in [int(v) for v in args.ranks.split(",")]:
-                for G in ((64, 128) if FMT in ("int4", "int4_asym", "int4_ph") else (16,) if FMT == "nvfp4" else (0,)):
+                for G in ((64, 128) if FMT in ("int4", "int4_asym", "int4_ph") else (16,) if FMT in ("nvfp4", "nvfp4_ph") else (0,)):
                     c = Case(18432, K, N, r, G, synth.FLUX)
                     c.report("4: FLUX batch 4 (M=18432) rank/group sweep", max(5, args.iters // 2), p_bf16, hbm)
                     c.close()

@@ -360,3 +360,69 @@ def test_projection_form_flux_linears(K, N):
 
 def test_projection_form_batch4_group128_rank128():
     print(_run_ph(18432, 3072, 3072, 128, 128, synth.FLUX))
+
+
+# ------------------------------------------------------------------ NVFP4 operands behind the projection form, full size
+
+def _run_nvfp4_ph(M, K, N, r, model, n_rows=24, n_cols=96, seed=0):
+    from parity_utils import check_activation_side_nvfp4, check_layer_output_nvfp4, _codes_equal_mod_zero
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=64, model=model, seed=seed)
+    Uh = np.ascontiguousarray(np.asarray(synth.make_rotation(spec, device="cuda"), dtype=np.float64)[:, :r])
+    W, bias = synth.make_weights(spec)
+    x_bits = synth.make_tokens(spec, M, batch_seed=3)
+    g = np.random.default_rng(K * 7 + N + 2)
+    rows = np.sort(g.choice(M, size=min(n_rows, M), replace=False))
+    rows[-1] = M - 1
+    cols = np.sort(g.choice(N, size=n_cols, replace=False))
+    cols[-1] = N - 1
+
+    # the weights' per-tensor exponent depends on all columns: the reference folds the whole weight
+    lo_full = orc.nvfp4_prepare_layer_ph(W, Uh, want_t=True)
+    lo = dict(lo_full)
+    lo["wcodes"], lo["wsf"], lo["Wh"] = lo_full["wcodes"][:, cols], lo_full["wsf"][:, cols], lo_full["Wh"][:, cols]
+    if lo_full["wt"] is not None:
+        lo["wt"] = lo_full["wt"][:, cols]
+    bias_s = np.ascontiguousarray(bias[cols])
+    xs = np.ascontiguousarray(x_bits[rows])
+    ex = orc.nvfp4_global_exponent(float(np.abs(orc.nvfp4_residual(xs, lo)[1]).max()))
+    oo = orc.nvfp4_linear_deployed_ph(xs, lo, ex, bias=bias_s)
+
+    layer = dq.dirotq_prepare_layer_nvfp4_ph(torch.from_numpy(W).cuda(), torch.from_numpy(Uh).cuda(), ex,
+                                             bias=bits_to_bf16_tensor(bias))
+    wcodes, wsf, wh, uhb, ew = dq.dirotq_layer_export_nvfp4(layer)
+    assert ew == lo_full["ew"]
+    assert np.array_equal(bf16_tensor_to_bits(uhb), lo["Uhb"])
+    cols_t = torch.from_numpy(cols).cuda()
+    assert np.array_equal(wsf[:, cols_t].cpu().numpy(), lo["wsf"])
+    assert np.array_equal(bf16_tensor_to_bits(wh[:, cols_t]), lo["Wh"])
+    bad = ~_codes_equal_mod_zero(wcodes[:, cols_t].cpu().numpy(), lo["wcodes"])
+    assert bad.sum() <= 2
+    del wcodes, wsf, wh
+
+    x = bits_to_bf16_tensor(x_bits)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = dq.alloc_workspace(layer, M)
+    dq.dirotq_linear(x, layer, y, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    xh, codes, sf = dq.dirotq_workspace_export_nvfp4(layer, M, ws)
+    rows_t = torch.from_numpy(rows).cuda()
+    xh_b = bf16_tensor_to_bits(xh[rows_t])
+    codes_n, sf_n = codes[rows_t].cpu().numpy(), sf[rows_t].cpu().numpy()
+    _, xl_ref = orc.nvfp4_residual(xs, lo, xh_bits=xh_b)
+    xt_ref = np.ascontiguousarray(np.concatenate([orc.bf16_to_f64(xh_b), xl_ref], axis=1))
+    sq_ref = orc.nvfp4_split_quantize(xt_ref, r, ex, want_t=True)
+    prot = {"xt": xt_ref, "xh": sq_ref["xh"], "codes": sq_ref["codes"], "sf": sq_ref["sf"], "t": sq_ref["t"]}
+    stats = check_activation_side_nvfp4(None, xh_b, codes_n, sf_n, prot, r, ex)
+    y_s = bf16_tensor_to_bits(y[rows_t][:, cols_t])
+    stats.update(check_layer_output_nvfp4(y_s, xh_b, codes_n, sf_n, ex, lo, oo, bias_s))
+    layer.close()
+    return stats
+
+
+@pytest.mark.parametrize("K,N", [(3072, 9216), (12288, 3072)])
+def test_nvfp4_projection_form_flux_linears(K, N):
+    print(_run_nvfp4_ph(4608, K, N, 32, synth.FLUX))
+
+
+def test_nvfp4_projection_form_batch4_rank128():
+    print(_run_nvfp4_ph(18432, 3072, 3072, 128, synth.FLUX))

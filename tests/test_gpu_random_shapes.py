@@ -17,8 +17,8 @@ import test_gpu_w4a8
 pytestmark = pytest.mark.gpu
 
 
-def _one(rng, big):
-    fmt = rng.choice(["int4", "int4", "asym", "nvfp4", "w4a8", "ph"])
+def _one(rng, big, fmt=None):
+    fmt = fmt or rng.choice(["int4", "int4", "asym", "nvfp4", "w4a8", "ph"])
     if big:
         M = rng.choice([19000, 20001, 25000])
         K = 64 * rng.randint(2, 4)
@@ -52,6 +52,8 @@ def _one(rng, big):
             test_gpu_asym._run_case(spec, M=M, with_bias=bias, shift=rng.choice([0.0, 1.5]), check_rot=not big)
         elif fmt == "ph":
             test_gpu_projection_form._run_case(spec, M=M, with_bias=bias)
+        elif fmt == "nvfp4_ph":
+            test_gpu_projection_form._run_case_nvfp4(spec, M=M, with_bias=bias)
         elif fmt == "nvfp4":
             test_gpu_nvfp4._run_case(spec, M=M, with_bias=bias, check_rot=not big)
         else:
@@ -74,3 +76,11 @@ def test_random_large_m_shapes():
     rng = random.Random(20252)
     for _ in range(6):
         _one(rng, big=True)
+
+
+def test_random_nvfp4_projection_form_shapes():
+    rng = random.Random(20253)
+    for _ in range(25):
+        _one(rng, big=False, fmt="nvfp4_ph")
+    for _ in range(2):
+        _one(rng, big=True, fmt="nvfp4_ph")
