@@ -30,7 +30,7 @@ EXPORTED = [
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
     "dirotq_prepare_layer_codes", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
-    "dirotq_layer_export_uh", "dirotq_layer_bytes_nvfp4_ph", "dirotq_prepare_layer_nvfp4_ph", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_layer_export_uh", "dirotq_layer_bytes_nvfp4_ph", "dirotq_prepare_layer_nvfp4_ph", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_set_first_step_split", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -93,6 +93,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_set_gemm_tile.argtypes = [i]
         L.dirotq_set_dependent_launch.argtypes = [i]
         L.dirotq_set_rotation_tile.argtypes = [i]
+        L.dirotq_set_first_step_split.argtypes = [i]
         L.dirotq_prepare_layer_codes.argtypes = [vp, i, i, vp, i, vp, vp, vp, i, i, i, i, i, vp, sz, vp, sz, vp,
                                                  ctypes.POINTER(vp)]
         L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -454,6 +455,11 @@ def dirotq_set_gemm_tile(columns: int) -> None:
 def dirotq_set_rotation_tile(plan: int) -> None:
     """Tile plan of the rotation kernel: 0 automatic, 1 = 128x128, 2 = 128x256, 3 = 256x256 (process-wide)."""
     _check(lib().dirotq_set_rotation_tile(int(plan)), "dirotq_set_rotation_tile")
+
+
+def dirotq_set_first_step_split(enabled: bool) -> None:
+    """Projection form: split the first step's reduction over K into ranges when there are few row tiles (default on)."""
+    _check(lib().dirotq_set_first_step_split(int(bool(enabled))), "dirotq_set_first_step_split")
 
 
 def dirotq_set_dependent_launch(enabled: bool) -> None:

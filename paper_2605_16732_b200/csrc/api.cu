@@ -544,6 +544,11 @@ static dirotq_status_t second_kernel(const dirotq_layer_t* layer, const RotateAr
 
 dirotq_status_t dirotq_set_rotation_tile(int plan) { return set_rotation_plan(plan); }
 
+dirotq_status_t dirotq_set_first_step_split(int enabled) {
+    dirotq::set_first_step_split(enabled != 0);
+    return DIROTQ_OK;
+}
+
 dirotq_status_t dirotq_set_dependent_launch(int enabled) {
     dirotq::set_dependent_launch(enabled != 0);
     return DIROTQ_OK;

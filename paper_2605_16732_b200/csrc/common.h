@@ -274,6 +274,7 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
 dirotq_status_t set_nvfp4_tile_columns(int columns);
 dirotq_status_t set_w4a8_tile_columns(int columns);
 dirotq_status_t set_rotation_plan(int plan);
+void set_first_step_split(bool on);
 dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
                                   const void* bias, double* scratch, cudaStream_t stream);
 dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, cudaStream_t stream);

@@ -25,6 +25,7 @@
 
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <atomic>
 
 namespace dirotq {
@@ -56,6 +57,10 @@ struct RotKernelParams {
     // W4A8 variant: first pass only (the token's scale needs its whole row)
     float* xtilde;          // fp32 [M][K_lp]
     unsigned int* rowmax;   // per-token max |x~_l| as a bit pattern, atomic max (zeroed by the host before the launch)
+    // Split reduction (first step of the projection form with few row tiles): the k-blocks are cut into `ksplit` ranges,
+    // one tile each, and every range's fp32 accumulators go to partial[range][M][n_out]; nothing else is written.
+    int ksplit = 1;
+    float* partial = nullptr;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -187,7 +192,8 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     const int num_m_blocks = (p.M + BM - 1) / BM;
     const int num_n_blocks = (p.n_out + BN - 1) / BN;
-    const int num_tiles = num_m_blocks * num_n_blocks;
+    const int num_mn = num_m_blocks * num_n_blocks;
+    const int num_tiles = num_mn * p.ksplit;
     const int num_kb = p.k_red / BK;
 
     if (threadIdx.x == 0) {
@@ -223,9 +229,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile % num_m_blocks) * BM;
-                const int n0 = (tile / num_m_blocks) * BN;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int mn = tile % num_mn, sp = tile / num_mn;
+                const int m0 = (mn % num_m_blocks) * BM;
+                const int n0 = (mn / num_m_blocks) * BN;
+                const int kb_end = static_cast<int>(static_cast<long>(sp + 1) * num_kb / p.ksplit);
+                for (int kb = static_cast<int>(static_cast<long>(sp) * num_kb / p.ksplit); kb < kb_end; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
@@ -257,7 +265,10 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int sp = tile / num_mn;
+                const int kb_begin = static_cast<int>(static_cast<long>(sp) * num_kb / p.ksplit);
+                const int kb_end = static_cast<int>(static_cast<long>(sp + 1) * num_kb / p.ksplit);
+                for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
@@ -267,9 +278,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
-                        umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
                         if constexpr (BM == 256)  // token rows 128..255: next 16 KB of the x tile, columns 256..511 of TMEM
-                            umma_bf16(d + 256, adesc + (A_BYTES_128 >> 4) + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                            umma_bf16(d + 256, adesc + (A_BYTES_128 >> 4) + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
                     }
                     umma_commit(empty_bar(s));
                 }
@@ -286,8 +297,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-            const int m0 = (tile % num_m_blocks) * BM;
-            const int n_blk = tile / num_m_blocks;
+            const int mn = tile % num_mn;
+            const int m0 = (mn % num_m_blocks) * BM;
+            const int n_blk = mn / num_m_blocks;
             const int n0 = n_blk * BN;
             const uint32_t acc = tcount % ACC_BUFS;
             const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
@@ -321,6 +333,17 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[c * 32 + j] = __uint_as_float(raw[j]);
+                }
+                if (p.partial != nullptr) {
+                    // split reduction: this range's accumulators, as they are
+                    if (row_ok) {
+                        float4* dst = reinterpret_cast<float4*>(
+                            p.partial + (static_cast<size_t>(tile / num_mn) * p.M + row) * p.n_out + col0);
+#pragma unroll
+                        for (int j = 0; j < G / 4; ++j)
+                            if (col0 + 4 * j < p.n_out) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    }
+                    continue;
                 }
                 if (p.xrot != nullptr && row_ok) {
 #pragma unroll
@@ -519,9 +542,32 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     }
 }
 
+// Sums the ranges of a split reduction in range order and rounds to bf16: xh[row][c] = bf16(sum_s partial[s][row][c]).
+// One thread per 8 consecutive columns.
+__global__ void __launch_bounds__(256) reduce_partials_kernel(const float* __restrict__ partial, int ksplit, int M, int n_out,
+                                                              uint16_t* __restrict__ xh) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const long idx = static_cast<long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long total = static_cast<long>(M) * n_out / 8;
+    if (idx >= total) return;
+    float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int s = 0; s < ksplit; ++s) {
+        const float4* src = reinterpret_cast<const float4*>(partial + static_cast<size_t>(s) * M * n_out) + 2 * idx;
+        const float4 u = src[0], w = src[1];
+        a[0] += u.x; a[1] += u.y; a[2] += u.z; a[3] += u.w;
+        a[4] += w.x; a[5] += w.y; a[6] += w.z; a[7] += w.w;
+    }
+    reinterpret_cast<uint4*>(xh)[idx] = make_uint4(pack_bf16x2(a[0], a[1]), pack_bf16x2(a[2], a[3]), pack_bf16x2(a[4], a[5]),
+                                                   pack_bf16x2(a[6], a[7]));
+}
+
+static std::atomic<int> g_first_step_split{1};  // projection form: 0 keeps the first step's reduction in one piece
 static std::atomic<int> g_rotation_plan{0};  // 0: chosen per call; 1: 128 x 128, 2: 128 x 256, 3: 256 x 256 tiles
 
 }  // namespace
+
+void set_first_step_split(bool on) { g_first_step_split.store(on ? 1 : 0); }
 
 dirotq_status_t set_rotation_plan(int plan) {
     if (plan < 0 || plan > 3) return DIROTQ_ERR_INVALID_ARG;
@@ -613,10 +659,27 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
             if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return DIROTQ_ERR_CUDA;
             attr1 = true;
         }
-        const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.r_pad + 127) / 128);
+        long tiles = static_cast<long>((a.M + 127) / 128) * ((g.r_pad + 127) / 128);
+        // Few row tiles leave most SMs idle while x streams through: cut the reduction into ranges, one tile each.  The
+        // ranges' fp32 sums are parked in the (still unused) code region of the workspace and added up in range order.
+        int ksplit = static_cast<int>(sms / tiles);
+        ksplit = std::min(ksplit, std::min(8, (g.K / BK) / 8));
+        const size_t code_bytes = static_cast<size_t>(a.M) * (g.fmt == 1 ? g.K4 / 2 : g.K_lp);
+        while (ksplit > 1 && static_cast<size_t>(ksplit) * a.M * g.r_pad * 4 > code_bytes) --ksplit;
+        if (ksplit > 1 && g_first_step_split.load() != 0) {
+            p1.ksplit = ksplit;
+            p1.partial = reinterpret_cast<float*>(a.codes);
+            tiles *= ksplit;
+        }
         if (launch_kernel(k1, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_x,
                           L->tmap_qt128, p1) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
+        if (p1.partial != nullptr) {
+            const long threads = static_cast<long>(a.M) * g.r_pad / 8;
+            if (launch_kernel(reduce_partials_kernel, static_cast<int>((threads + 255) / 256), 256, 0, stream, true,
+                              static_cast<const float*>(p1.partial), p1.ksplit, a.M, g.r_pad, a.xh) != cudaSuccess)
+                return DIROTQ_ERR_CUDA;
+        }
     }
     {
         // step 2: A = x~_h [M][r_pad], B = U_hb [K][r_pad]; every output column is low-precision (K_l = K)

@@ -77,6 +77,7 @@ def test_knobs_validate_their_argument_without_a_gpu(L):
     for bad in (-1, 64, 192, 512):
         assert L.dirotq_set_gemm_tile(bad) == 1
     assert L.dirotq_set_dependent_launch(0) == 0 and L.dirotq_set_dependent_launch(1) == 0
+    assert L.dirotq_set_first_step_split(0) == 0 and L.dirotq_set_first_step_split(1) == 0
 
 
 def test_prepare_from_codes_rejects_null_arguments(L):

@@ -230,3 +230,15 @@ def test_nvfp4_projection_form_pixart_projection():
 def test_nvfp4_projection_form_ragged_rank64_no_bias():
     spec = synth.LayerSpec(K=768, N=400, r=64, G=64, model=synth.FLUX, seed=113, calib_tokens=1024)
     print(_run_case_nvfp4(spec, M=300, with_bias=False))
+
+
+@pytest.mark.parametrize("split", [False, True])
+def test_first_step_split_on_and_off(split):
+    # M = 300: 3 row tiles, so the reduction is split when the knob is on; both settings must satisfy the same checks
+    dq.dirotq_set_first_step_split(split)
+    try:
+        spec = synth.LayerSpec(K=2048, N=512, r=32, G=64, model=synth.FLUX, seed=114, calib_tokens=4096)
+        print(_run_case(spec, M=300))
+        print(_run_case_nvfp4(spec, M=300))
+    finally:
+        dq.dirotq_set_first_step_split(True)
