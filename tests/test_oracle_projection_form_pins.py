@@ -1,10 +1,11 @@
 """Pins of the oracle's projection form (only U_h applied densely, the residual rotated by a block Hadamard): the
-reference for a cheaper first stage that no CUDA kernel computes yet.  What the construction fixes: the Hadamard blocks
+reference for the cheaper first stage.  What the construction fixes: the Hadamard blocks
 are orthonormal; the decomposition x = x~_h U_hb^T + d is exact for ANY U_h because d is the residual of the rounded
 projection, so without quantization the layer is x W; the integer path equals dequantize-then-multiply; with no
 projection it reduces to group-wise rounding of the Hadamard-rotated operands; and on activations with outlier
 directions the projection is what keeps the error down."""
 import numpy as np
+import pytest
 
 from oracle import dirotq_oracle as orc
 from paper_2605_16732_b200 import synth
@@ -120,3 +121,32 @@ def test_nvfp4_projection_form_shares_the_decomposition_and_matches_the_dense_fo
     dense = orc.nvfp4_linear_deployed(inp["x"], lo, ex2, bias=inp["bias"])
     e = lambda y: float(np.sqrt(np.mean((y - ideal) ** 2) / np.mean(ideal ** 2)))
     assert 0.8 < e(out["y64"]) / e(dense["y64"]) < 1.25
+
+
+@pytest.mark.parametrize("n_outlier,magnitude,spread", [(0, 1.0, 0.0), (48, 30.0, 0.0), (48, 30.0, 1.0), (96, 100.0, 1.0)])
+def test_residuals_that_are_not_white(n_outlier, magnitude, spread):
+    """The synthetic layer generator leaves a white residual.  Here the residual is far from white: log-normal channel
+    scales and more axis-aligned outlier channels than the r directions U_h can take (PCA of calibration tokens picks
+    the largest).  A per-group Hadamard spreads a leftover outlier over its 64 neighbours only, the dense random
+    rotation over all K - r coefficients; with one scale per group of 64 the output errors come out alike."""
+    K, N, r, G, T, M = 512, 96, 32, 64, 2048, 160
+    g = np.random.default_rng(40 + n_outlier)
+    sig = np.exp(spread * g.standard_normal(K))
+    idx = g.choice(K, n_outlier, replace=False)
+    sig[idx] *= magnitude * g.uniform(0.3, 1.0, n_outlier)
+    calib = np.random.default_rng(1).standard_normal((T, K)) * sig
+    _, V = np.linalg.eigh(calib.T @ calib)
+    V = V[:, ::-1]                                                  # PCA directions, largest first (Sec. 4.1)
+    R, _ = np.linalg.qr(g.standard_normal((K - r, K - r)))         # the random rotation of the residual (Eq. 5)
+    Q = np.concatenate([V[:, :r], V[:, r:] @ R], axis=1)
+    W = 0.02 * g.standard_normal((K, N))
+    xb = orc.bf16_round(np.random.default_rng(2).standard_normal((M, K)) * sig)
+    ideal = _bf(xb) @ W
+
+    def err(y):
+        return float(np.sqrt(np.mean((y - ideal) ** 2) / np.mean(ideal ** 2)))
+
+    e_paper = err(orc.linear_deployed(xb, orc.prepare_layer(W, Q, r, G))["y64"])
+    e_proj = err(orc.linear_deployed_ph(xb, orc.prepare_layer_ph(W, np.ascontiguousarray(Q[:, :r]), G))["y64"])
+    print(n_outlier, magnitude, spread, e_paper, e_proj)
+    assert e_proj < 1.15 * e_paper
