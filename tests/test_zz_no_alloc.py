@@ -67,3 +67,35 @@ def test_noalloc_rejects_what_does_not_fit():
     assert dq.lib().dirotq_linear_noalloc(None, 8, layer.handle, y.data_ptr(), None, None) == 1
     torch.cuda.synchronize()
     layer.close()
+
+
+def test_noalloc_matches_linear_for_every_layer_format():
+    K, N, r, G, M = 512, 400, 32, 64, 260
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=synth.FLUX, seed=24, calib_tokens=1024)
+    W, bias = synth.make_weights(spec)
+    g = np.random.default_rng(24)
+    v = g.standard_normal(K)
+    v /= np.linalg.norm(v)
+    Q = torch.from_numpy(np.eye(K) - 2.0 * np.outer(v, v)).cuda()
+    Wd, Uh, b = torch.from_numpy(W).cuda(), Q[:, :r].contiguous(), _bf(bias)
+    x = _bf(synth.make_tokens(spec, M, batch_seed=5))
+    layers = {
+        "int4_asym": dq.dirotq_prepare_layer_asym(Wd, Q, r, G, bias=b),
+        "w4a8": dq.dirotq_prepare_layer_w4a8(Wd, Q, r, bias=b),
+        "nvfp4": dq.dirotq_prepare_layer_nvfp4(Wd, Q, r, -8, bias=b),
+        "int4_ph": dq.dirotq_prepare_layer_ph(Wd, Uh, G, bias=b),
+        "nvfp4_ph": dq.dirotq_prepare_layer_nvfp4_ph(Wd, Uh, -8, bias=b),
+    }
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    for name, ly in layers.items():
+        ref = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = dq.alloc_workspace(ly, M)
+        dq.dirotq_linear(x, ly, ref, ws)
+        assert dq.dirotq_workspace_status(ws) == 0
+        out = torch.zeros_like(ref)
+        dq.dirotq_linear_noalloc(x, ly, out, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, name
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), name
+        assert float(ref.float().abs().max()) > 0
+        ly.close()
