@@ -183,7 +183,7 @@ DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
  * K = 12288 at M = 4608).  Process-wide; results do not depend on it.  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_rotation_tile(int plan);
 
-/* Projection form, first step (x~_h = x U_hb): with few token-row tiles (M / 128 well below the number of SMs) the
+/* Projection form, first step (x~_h = x U_hb): with few token-row tiles (M / 128 at most half the number of SMs) and K >= 2048 the
  * reduction over K is cut into up to 8 ranges that run as tiles of their own; their fp32 sums are parked in the
  * workspace's code region (not yet in use at that point) and a small kernel adds them in range order and rounds to
  * bf16.  On (default) or off, process-wide.  x~_h may differ in the last bf16 digit between the two settings (another

@@ -664,6 +664,7 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
         // ranges' fp32 sums are parked in the (still unused) code region of the workspace and added up in range order.
         int ksplit = static_cast<int>(sms / tiles);
         ksplit = std::min(ksplit, std::min(8, (g.K / BK) / 8));
+        if (g.K / BK < 32) ksplit = 1;  // short reductions gain nothing (K = 1152 measured the same either way): one launch fewer
         const size_t code_bytes = static_cast<size_t>(a.M) * (g.fmt == 1 ? g.K4 / 2 : g.K_lp);
         while (ksplit > 1 && static_cast<size_t>(ksplit) * a.M * g.r_pad * 4 > code_bytes) --ksplit;
         if (ksplit > 1 && g_first_step_split.load() != 0) {
