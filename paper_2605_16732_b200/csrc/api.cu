@@ -196,8 +196,9 @@ static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int 
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
-        st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
-                            (uint64_t)g.n_g, (uint64_t)N * 4, kGemmBN, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+        st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale,
+                            (uint64_t)wscale_row_len(N), (uint64_t)g.n_g, (uint64_t)wscale_row_len(N) * 4, kGemmBN, 128 / group,
+                            CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -205,8 +206,9 @@ static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int 
         st = encode_tmap_2d(&L->tmap_wpacked128, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
-        st = encode_tmap_2d(&L->tmap_wscale128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
-                            (uint64_t)g.n_g, (uint64_t)N * 4, 128, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+        st = encode_tmap_2d(&L->tmap_wscale128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale,
+                            (uint64_t)wscale_row_len(N), (uint64_t)g.n_g, (uint64_t)wscale_row_len(N) * 4, 128, 128 / group,
+                            CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -339,8 +341,9 @@ dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
-        st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
-                            (uint64_t)g.n_g, (uint64_t)N * 4, kGemmBN, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+        st = encode_tmap_2d(&L->tmap_wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale,
+                            (uint64_t)wscale_row_len(N), (uint64_t)g.n_g, (uint64_t)wscale_row_len(N) * 4, kGemmBN, 128 / group,
+                            CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -348,8 +351,9 @@ dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout
         st = encode_tmap_2d(&L->tmap_wpacked128, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
-        st = encode_tmap_2d(&L->tmap_wscale128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale, (uint64_t)N,
-                            (uint64_t)g.n_g, (uint64_t)N * 4, 128, 128 / group, CU_TENSOR_MAP_SWIZZLE_NONE);
+        st = encode_tmap_2d(&L->tmap_wscale128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale,
+                            (uint64_t)wscale_row_len(N), (uint64_t)g.n_g, (uint64_t)wscale_row_len(N) * 4, 128, 128 / group,
+                            CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);

@@ -55,6 +55,39 @@ inline Geometry make_geometry(int K, int N, int r, int G) {
     return g;
 }
 
+// ------------------------------------------------------------------ weight-side layouts of the grouped INT4 formats
+//
+// Group scales of the weight codes, f32 [n_g][N32] (N32 = N rounded up to 32).  Two things are folded in offline:
+//   * the value stored is 2^18 s_w (exact): the second kernel's accumulators hold 2^-18 times the integer group sums;
+//   * inside every aligned run of 32 output columns the scales are permuted so that the 8 a thread of the second
+//     kernel's epilogue needs (columns 8 b + 2 p + e, b = 0..3, e = 0..1, for its p = lane % 4) lie side by side:
+//     column 8 b + 2 p + e of the run is stored at position 8 p + 2 b + e.
+// (W4A8 layers keep one plain scale per output column: f32 [N].)
+constexpr float kWScaleFold = 262144.0f;  // 2^18
+__host__ __device__ inline int wscale_row_len(int N) { return (N + 31) / 32 * 32; }
+__host__ __device__ inline size_t wscale_index(int N, int grp, int n) {
+    const int c = n & 31;
+    return static_cast<size_t>(grp) * wscale_row_len(N) + (n & ~31) + ((c >> 1) & 3) * 8 + (c >> 3) * 2 + (c & 1);
+}
+
+// Packed weight codes of the grouped INT4 formats: a 32-bit word holds eight codes as sign + 3-bit magnitude.  Code t < 4
+// sits in byte t with its magnitude in bits 2..0 and its sign in bit 7; code t >= 4 is the same picture rotated left
+// by four bit positions (magnitude in bits 6..4 of byte t - 4, sign in bit 3 of the next byte, wrapping around), so that
+//     w & 0x87878787  and  rotate_right(w, 4) & 0x87878787
+// are codes 0..3 and 4..7 as one byte each, s0000mmm: read as E4M3 that byte is q * 2^-9 exactly.
+__host__ __device__ inline uint32_t signmag_nibble_bits(int t, int q) {  // bits of code t (0..7), q in [-7, 7]
+    const uint32_t mag = static_cast<uint32_t>(q < 0 ? -q : q), sign = q < 0 ? 1u : 0u;
+    const uint32_t v = mag | (sign << 7);                 // s0000mmm in byte 0
+    const uint32_t placed = v << (8 * (t & 3));
+    return t < 4 ? placed : ((placed << 4) | (placed >> 28));
+}
+__host__ __device__ inline int signmag_nibble_decode(uint32_t word, int t) {
+    const uint32_t w = t < 4 ? word : ((word >> 4) | (word << 28));
+    const uint32_t v = (w >> (8 * (t & 3))) & 0x87u;
+    const int mag = static_cast<int>(v & 7u);
+    return (v & 0x80u) ? -mag : mag;
+}
+
 constexpr size_t kAlign = 1024;
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
@@ -87,7 +120,7 @@ inline void make_asym(Geometry& g) {
 struct BlobLayout {
     size_t off_qt;       // bf16 [K][K]: row c' = permuted output column, K-major over the input channel
     size_t off_wpacked;  // u8   [N][K_lp/2]: two INT4 codes per byte, K-major, see prepare.cu for the nibble order
-    size_t off_wscale;   // f32  [n_g][N]: bf16-valued group scales of the weight codes
+    size_t off_wscale;   // f32  [n_g][N32]: bf16-valued group scales of the weight codes times 2^18, see wscale_index
     size_t off_wh;       // bf16 [N][r_pad]: high-precision rows of the folded weight, K-major, zero padded
     size_t off_bias;     // f32  [N]
     // NVFP4 variant: off_wpacked = E2M1 codes u8 [N][K4/2] (even k in the low nibble); off_wscale = E4M3 scale
@@ -103,7 +136,7 @@ inline BlobLayout make_blob_layout(const Geometry& g) {
     b.off_qt = o;      o = align_up(o + (g.fmt == 4 ? (size_t)g.r_pad * g.K * 2 : g.no_rot ? 0 : (size_t)g.K * g.K * 2));
     b.off_uh = o;      o = align_up(o + (g.fmt == 4 ? (size_t)g.K * g.r_pad * 2 : 0));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K_lp / 2));
-    b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * g.N * 4);
+    b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * wscale_row_len(g.N) * 4);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
     b.off_bias = o;    o = align_up(o + (size_t)g.N * 4);
     b.off_meta = o;    o = align_up(o + 64);
@@ -130,8 +163,7 @@ struct WorkspaceLayout {
     int ldm;            // leading dimension (tokens) of the transposed activation-scale array
     size_t off_status;  // int32[64]: word 0 = device status
     size_t off_codes;   // u8  [M][K_lp]: activation codes, one per byte, sign-magnitude (bit 7 = sign, bits 2..0 = |q|)
-    size_t off_xscale;  // f32 [2 n_g][ldm]: rows 0..n_g-1 the bf16-valued activation scales s (group-major),
-                        //                   rows n_g..2 n_g-1 the offset corrections -8 * s * sum_k q (see w4a4_gemm.cu)
+    size_t off_xscale;  // f32 [n_g][ldm]: the bf16-valued activation scales s, group-major
     size_t off_xh;      // bf16 [M][r_pad]
     // NVFP4 variant: off_codes = E2M1 codes u8 [M][K4/2]; off_xscale = E4M3 scale atoms u8 [ceil(M/128)][nkb64p][512]
     size_t total;
@@ -143,7 +175,7 @@ inline WorkspaceLayout make_workspace_layout(const Geometry& g, int M) {
     size_t o = 0;
     w.off_status = o;  o = align_up(o + 256);
     w.off_codes = o;   o = align_up(o + (size_t)M * g.K_lp);
-    w.off_xscale = o;  o = align_up(o + (size_t)2 * g.n_g * w.ldm * 4);
+    w.off_xscale = o;  o = align_up(o + (size_t)g.n_g * w.ldm * 4);
     w.off_xh = o;      o = align_up(o + (size_t)M * g.r_pad * 2);
     w.total = o;
     return w;
@@ -190,8 +222,8 @@ struct dirotq_layer {
     char* blob;  // device
     CUtensorMap tmap_qt;       // bf16 [K][K], box 64 x 256, 128B swizzle
     CUtensorMap tmap_qt128;    // the same tensor with box 64 x 128 (narrow tiles of the rotation kernel)
-    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2] (nibble = q + 8), box 64 x kGemmBN, no swizzle
-    CUtensorMap tmap_wscale;   // f32 [n_g][N], box kGemmBN x (128/G)
+    CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2] (two codes per byte), box 64 x kGemmBN, no swizzle
+    CUtensorMap tmap_wscale;   // f32 [n_g][N32], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
     CUtensorMap tmap_wpacked128, tmap_wscale128, tmap_wh128;  // the same three with 128-row boxes (narrow W4A4 tiles)
     int act_scale_log2;        // NVFP4 variant: exponent of the activations' per-tensor power-of-two scale

@@ -4,11 +4,12 @@
 // per layer and is not on the timed path.
 //
 // Packed weight-code layout, row n of u8 [N][K_lp/2] (K-major): codes are taken 32 at a time
-// (16 bytes); inside such a piece, byte 4*j + b (j, b in 0..3) holds code 8*j + b in its low
-// nibble and code 8*j + 4 + b in its high nibble; a nibble holds u = q + 8 (1..15).  With this order the
-// online unpack of a 32-bit word is two logic ops per four codes:
-//   w & 0x0F0F0F0F  ->  codes 8j..8j+3 as bytes 0000uuuu,      (w >> 4) & 0x0F0F0F0F  ->  codes 8j+4..8j+7,
-// and a byte 0000uuuu read as E4M3 is u * 2^-9 exactly (see w4a4_gemm.cu).
+// (16 bytes, four 32-bit words); word j of such a piece holds codes 8*j .. 8*j + 7.  In the grouped INT4
+// formats a code is stored as sign + 3-bit magnitude, codes 8j..8j+3 in bits 7, 2..0 of the word's bytes and
+// codes 8j+4..8j+7 four bit positions further up (signmag_nibble_bits in common.h), so that the online unpack of a
+// word is a mask, a rotate and a mask, and the resulting byte s0000mmm read as E4M3 is q * 2^-9 exactly (see
+// w4a4_gemm.cu).  The W4A8 format keeps the nibble u = q + 8 (code 8j + b in the low, 8j + 4 + b in the high nibble
+// of byte 4j + b), which its own kernel turns into the int8 value 16 q.
 #include "common.h"
 
 #include <cuda_bf16.h>
@@ -94,7 +95,7 @@ __global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, floa
     for (int j = 0; j < len; ++j) a = fmax(a, fabs(col[static_cast<size_t>(j) * g.N]));
     const uint16_t sb = (a == 0.0) ? 0 : f64_to_bf16(a / 7.0);
     const double s = bf16_to_f64(sb);
-    wscale[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(s);
+    wscale[wscale_index(g.N, grp, n)] = static_cast<float>(s) * kWScaleFold;  // a power of two times a bf16 value: exact
     uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
     int csum = 0;
     for (int jb = 0; jb < g.G; jb += 8) {
@@ -109,9 +110,7 @@ __global__ void quantize_weights_kernel(const double* Wt, uint8_t* wpacked, floa
                 q = static_cast<int>(qq);
             }
             csum += q;
-            // stored with an offset of 8: the nibble u = q + 8 in 1..15, read as an E4M3 byte, is u * 2^-9 exactly
-            const uint32_t nib = static_cast<uint32_t>(q + 8) & 0xFu;
-            word |= nib << (8 * (t & 3) + 4 * (t >> 2));
+            word |= signmag_nibble_bits(t, q);
         }
         *reinterpret_cast<uint32_t*>(row + packed_byte_index(j0 + jb)) = word;
     }
@@ -138,7 +137,7 @@ __global__ void pack_codes_kernel(const int8_t* codes, const uint16_t* scales, u
     const int j0 = grp * g.G;
     const int len = min(g.G, g.K_l - j0);
     const double s = bf16_to_f64(scales[static_cast<size_t>(grp) * g.N + n]);
-    wscale[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(s);
+    wscale[wscale_index(g.N, grp, n)] = static_cast<float>(s) * kWScaleFold;
     const int8_t* col = codes + static_cast<size_t>(j0) * g.N + n;
     uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
     int csum = 0;
@@ -148,7 +147,7 @@ __global__ void pack_codes_kernel(const int8_t* codes, const uint16_t* scales, u
             const int j = jb + t;
             const int q = j < len ? max(-7, min(7, static_cast<int>(col[static_cast<size_t>(j) * g.N]))) : 0;
             csum += q;
-            word |= (static_cast<uint32_t>(q + 8) & 0xFu) << (8 * (t & 3) + 4 * (t >> 2));
+            word |= signmag_nibble_bits(t, q);
         }
         *reinterpret_cast<uint32_t*>(row + packed_byte_index(j0 + jb)) = word;
     }
@@ -200,14 +199,24 @@ __global__ void export_wcodes_kernel(const uint8_t* wpacked, int8_t* wcodes, Geo
     const int n = blockIdx.x * blockDim.x + threadIdx.x;
     const int j = blockIdx.y;
     if (n >= g.N || j >= g.K_l) return;
-    const uint8_t byte = wpacked[static_cast<size_t>(n) * (g.K_lp / 2) + packed_byte_index(j)];
-    const int nib = packed_is_high(j) ? (byte >> 4) : (byte & 0xF);
-    wcodes[static_cast<size_t>(j) * g.N + n] = static_cast<int8_t>(nib - 8);  // stored with an offset of 8
+    const uint8_t* row = wpacked + static_cast<size_t>(n) * (g.K_lp / 2);
+    if (g.fmt == 3) {  // W4A8: nibble = q + 8
+        const uint8_t byte = row[packed_byte_index(j)];
+        const int nib = packed_is_high(j) ? (byte >> 4) : (byte & 0xF);
+        wcodes[static_cast<size_t>(j) * g.N + n] = static_cast<int8_t>(nib - 8);
+    } else {           // grouped formats: sign + magnitude, see signmag_nibble_bits
+        const uint32_t word = *reinterpret_cast<const uint32_t*>(row + packed_byte_index(j & ~7));
+        wcodes[static_cast<size_t>(j) * g.N + n] = static_cast<int8_t>(signmag_nibble_decode(word, j & 7));
+    }
 }
 
-__global__ void export_wscales_kernel(const float* wscale, uint16_t* out, size_t count) {
-    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i < count) out[i] = static_cast<uint16_t>(__float_as_uint(wscale[i]) >> 16);  // values are bf16-exact
+// Group scales back in plain order as bf16: [rows][N].  `grouped`: stored permuted and times 2^18 (wscale_index).
+__global__ void export_wscales_kernel(const float* wscale, uint16_t* out, int rows, int N, bool grouped) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int grp = blockIdx.y;
+    if (n >= N || grp >= rows) return;
+    const float v = grouped ? wscale[wscale_index(N, grp, n)] * (1.0f / kWScaleFold) : wscale[static_cast<size_t>(grp) * N + n];
+    out[static_cast<size_t>(grp) * N + n] = static_cast<uint16_t>(__float_as_uint(v) >> 16);  // values are bf16-exact
 }
 
 __global__ void export_wh_kernel(const uint16_t* wh, uint16_t* out, Geometry g) {
@@ -279,21 +288,18 @@ __global__ void export_zero_term_kernel(const uint16_t* wh, float* d, Geometry g
     d[static_cast<size_t>(grp) * g.N + n] = static_cast<float>(v);  // 17 significant bits: exact
 }
 
-// Debug entry of the group GEMM: two's-complement codes [M][K_lp] -> the sign-magnitude bytes the kernel reads,
-// unit scales and the offset corrections -8 sum(q) (one thread per token and group).
+// Debug entry of the group GEMM: two's-complement codes [M][K_lp] -> the sign-magnitude bytes the kernel reads, and
+// unit scales (one thread per token and group).
 __global__ void debug_codes_kernel(const int8_t* in, uint8_t* out, float* xscale, int M, int ldm, Geometry g) {
     const int m = blockIdx.x * blockDim.x + threadIdx.x;
     const int grp = blockIdx.y;
     if (m >= M) return;
-    int sum = 0;
     for (int j = 0; j < g.G; ++j) {
         const size_t idx = static_cast<size_t>(m) * g.K_lp + grp * g.G + j;
         const int q = in[idx];
-        sum += q;
         out[idx] = static_cast<uint8_t>((q < 0 ? 0x80 : 0) | (q < 0 ? -q : q));
     }
     xscale[static_cast<size_t>(grp) * ldm + m] = 1.0f;
-    xscale[static_cast<size_t>(g.n_g + grp) * ldm + m] = -8.0f * static_cast<float>(sum);
 }
 
 // ================================================================ W4A8 (paper Sec. 5.1: per-channel 4-bit weights, per-token 8-bit activations)
@@ -655,9 +661,9 @@ dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint1
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
     }
     if (wscales) {
-        const size_t count = static_cast<size_t>(g.fmt == 3 ? 1 : g.n_g) * g.N;  // W4A8: one scale per output column
-        export_wscales_kernel<<<static_cast<unsigned>((count + 255) / 256), 256, 0, stream>>>(
-            reinterpret_cast<const float*>(blob + L->lay.off_wscale), wscales, count);
+        const int rows = g.fmt == 3 ? 1 : g.n_g;  // W4A8: one scale per output column
+        export_wscales_kernel<<<dim3((g.N + 255) / 256, rows), 256, 0, stream>>>(
+            reinterpret_cast<const float*>(blob + L->lay.off_wscale), wscales, rows, g.N, g.fmt != 3);
         if (!launch_ok()) return DIROTQ_ERR_CUDA;
     }
     if (wh) {

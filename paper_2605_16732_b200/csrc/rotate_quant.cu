@@ -3,8 +3,7 @@
 //   x~ = x Q_b                      bf16 x bf16 -> fp32 on tcgen05 (kind::f16), operands by TMA
 //   x~_h = bf16(x~[:, high])        the r high-precision coefficients          (paper Sec. 4.2)
 //   per token, per group of G low-precision coefficients:                      (paper Eq. 1, z = 0)
-//       s = bf16(max|x~| / 7),  q = clip(rint(x~ / s), -7, 7)   stored as a sign-magnitude byte,
-//       plus the offset correction -8 s sum(q) that the second kernel needs
+//       s = bf16(max|x~| / 7),  q = clip(rint(x~ / s), -7, 7)   stored as a sign-magnitude byte
 //
 // The rotated activations never reach HBM: the fp32 accumulators are read from tensor memory by
 // the epilogue warps, where each thread owns one token row, so the group maximum is a
@@ -70,8 +69,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // Quantizes 16 consecutive values with the reciprocal scale and packs them one code per byte in
 // sign-magnitude form (bit 7 = sign, bits 2..0 = |q|): read as E4M3 that byte is q * 2^-9 exactly, which
-// is how the second kernel's tensor-core instruction consumes it.  The codes are also added to `sum`.
-__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, bool slow, int& sum) {
+// is how the second kernel's tensor-core instruction consumes it.
+__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, bool slow) {
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -85,7 +84,6 @@ __device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, 
             f[j] = __float_as_uint(t + 12582912.0f);
         }
         const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
-        sum = __dp4a(static_cast<int>(tw), 0x01010101, sum);
         const uint32_t sg = (tw >> 7) & 0x01010101u;           // 1 where the code is negative
         const uint32_t mag = (tw ^ (sg * 0xFFu)) + sg;         // |q| per byte (at most 7: no carry between bytes)
         w[i] = mag | (tw & 0x80808080u);
@@ -94,8 +92,8 @@ __device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, 
 }
 
 // Asymmetric variant (Eq. 1 with z = min X): 16 values -> 16 bytes u = clip(rint((v - z) / s), 0, 15); as E4M3 the byte
-// 0000uuuu is u * 2^-9 exactly.  The codes are also added to `sum`.
-__device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float inv, float s, bool slow, int& sum) {
+// 0000uuuu is u * 2^-9 exactly.
+__device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float inv, float s, bool slow) {
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -108,7 +106,6 @@ __device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float 
             f[j] = __float_as_uint(t + 12582912.0f);  // nearest integer, ties to even, in the low byte
         }
         const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
-        sum = __dp4a(tw, 0x01010101u, static_cast<unsigned>(sum));
         w[i] = tw;
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
@@ -454,16 +451,14 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         const bool slow = !(s >= 1e-30f);
                         const float inv = slow ? 0.f : __frcp_rn(s);
                         int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
-                        int usum = 0;
 #pragma unroll
                         for (int b = 0; b < G / 16; ++b) {
                             uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
-                            if (16 * b < nlow) packed = quantize16_asym(v + 16 * b, z, inv, s, slow, usum);
+                            if (16 * b < nlow) packed = quantize16_asym(v + 16 * b, z, inv, s, slow);
                             *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
                         }
                         const int grp = col0 / G;
                         p.xscale[static_cast<size_t>(grp) * p.ldm + row] = s;
-                        p.xscale[static_cast<size_t>(p.n_g + grp) * p.ldm + row] = -8.0f * static_cast<float>(usum) * s;
                         // the zero-point, three times, in the extra columns of the bf16 rank-r operand
                         uint16_t* zrow = p.xh + static_cast<size_t>(row) * p.r_pad + p.r_pad0 + grp;
                         const uint16_t zbits = *reinterpret_cast<const uint16_t*>(&zb);
@@ -485,17 +480,13 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const float inv = slow ? 0.f : __frcp_rn(s);
                     if (row_ok) {
                         int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
-                        int qsum = 0;
 #pragma unroll
                         for (int b = 0; b < G / 16; ++b) {
                             uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
-                            if (16 * b < nlow) packed = quantize16(v + 16 * b, inv, s, slow, qsum);
+                            if (16 * b < nlow) packed = quantize16(v + 16 * b, inv, s, slow);
                             *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
                         }
                         p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
-                        // the weights reach the tensor core as q_w + 8: -8 s sum(q_x) takes the offset out again
-                        // (exact in fp32: |sum| <= 7 G and s has 8 significant bits)
-                        p.xscale[static_cast<size_t>(p.n_g + col0 / G) * p.ldm + row] = -8.0f * static_cast<float>(qsum) * s;
                     }
                 }
                 if (nlow < G && row_ok) {

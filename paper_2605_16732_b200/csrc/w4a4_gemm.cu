@@ -6,18 +6,19 @@
 // sm_100a has no INT4 MMA, and an int32 accumulator costs a conversion per element and group before it
 // can be scaled.  The integer products are therefore computed EXACTLY on the 8-bit float path
 // (tcgen05.mma kind::f8f6f4, E4M3 operands, fp32 accumulation):
-//   * an E4M3 byte 0000mmmm is m * 2^-9 for m = 0..15 (the subnormals 0..7 and the first binade 8..15
-//     lie on one line), and bit 7 is the sign;
-//   * activation codes arrive from kernel (a) one per byte in sign-magnitude form: q_x * 2^-9;
-//   * weight codes stay packed (two per byte) in HBM and in the TMA staging buffer with an offset of 8
-//     (u_w = q_w + 8 in 1..15); two "unpack" warps split every byte into two bytes 0000uuuu = u_w * 2^-9
-//     in the 128-byte-swizzled layout the MMA reads;
+//   * an E4M3 byte s0000mmm is (-1)^s m * 2^-9 for m = 0..7 (subnormals; with a fourth magnitude bit, 0..15: the
+//     first binade continues the same line), so a code stored as sign + magnitude IS an E4M3 number;
+//   * activation codes arrive from kernel (a) one per byte in that form: q_x * 2^-9 (the asymmetric variant
+//     stores u = 0..15 as 0000uuuu = u * 2^-9);
+//   * weight codes stay packed (two per byte: sign + 3-bit magnitude each) in HBM and in the TMA staging
+//     buffer; two "unpack" warps split every 32-bit word of eight codes into two words of four bytes
+//     s0000mmm = q_w * 2^-9 (one mask, one rotate and one mask: the nibble order of prepare.cu is chosen for
+//     that) in the 128-byte-swizzled layout the MMA reads;
 //   * every product is an integer times 2^-18 and a group's sum is below 2^24 in magnitude, so the fp32
-//     accumulator holds S_g = 2^-18 sum_j q_x u_w without rounding, and
-//         P_g = 2^18 S_g - 8 sum_j q_x[m,j];
-//     kernel (a) stores e[m,g] = -8 s_x sum_j q_x (exact in fp32), so that
-//         s_x P_g = fma(S_g, 2^18 s_x, e)        -- one rounding, that of the product s_x P_g itself --
-//     and the group is folded in with two fused multiply-adds per element and no integer conversion.
+//     accumulator holds S_g = 2^-18 P_g without rounding.  The weight scales are stored as 2^18 s_w (exact), so
+//         t = S_g * s_x                   -- one rounding, that of the product s_x P_g itself --
+//         acc = fma(t, 2^18 s_w, acc)
+//     folds a group in with one multiply and one fused multiply-add per element and no integer conversion.
 // The exactness of the accumulation is a property of the tensor core that the parity tests pin: the
 // group sums exported by the debug entry equal the CPU checker's int32 sums bit for bit, on random
 // codes and on patterns built to lose low bits (long runs of +-49 followed by +-1).
@@ -47,6 +48,13 @@ constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_
 constexpr int SC_SLOTS = 8;
 constexpr int NUM_THREADS = 384;
 constexpr int NUM_EPI_WARPS = 8;
+constexpr uint32_t kSignMag = 0x87878787u;  // sign and 3-bit magnitude of four one-byte codes
+#ifndef W4A4_EPI_REGS
+#define W4A4_EPI_REGS 216
+#endif
+#ifndef W4A4_AUX_REGS
+#define W4A4_AUX_REGS 64
+#endif
 
 // Shared-memory plan for tiles of BN output columns.  256 columns is the default; 128-column tiles (with more
 // pipeline stages) are used when the wide ones would leave most SMs idle in the last wave, see the launcher.
@@ -57,8 +65,8 @@ struct Plan {
     static constexpr int BP_BYTES = BN * BKC / 2;     // packed weight codes (TMA staging)
     static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB / 40 KB
     static constexpr int SC_SW_BYTES = 2 * BN * 4;    // up to two groups per k-block
-    static constexpr int SC_SX_BYTES = 2 * 2 * BM * 4;  // scales of up to two groups, then their offset corrections
-    static constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 4 KB / 3 KB
+    static constexpr int SC_SX_BYTES = 2 * BM * 4;    // activation scales of up to two groups
+    static constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 3 KB / 2 KB
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
     static constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024;
 };
@@ -91,6 +99,25 @@ __device__ __forceinline__ void flush_wait(int* status, int slot, long long cycl
     atomicAdd(reinterpret_cast<unsigned long long*>(status) + slot, static_cast<unsigned long long>(cycles));
 }
 
+// Two fp32 values in one 64-bit register pair (sm_100 has packed fp32 arithmetic on such pairs).
+__device__ __forceinline__ uint64_t pack_u32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) { return pack_u32x2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {  // round to nearest even, per element
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -106,23 +133,24 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     constexpr int STAGES = P::STAGES, STAGE_BYTES = P::STAGE_BYTES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES;
     constexpr int SC_SW_BYTES = P::SC_SW_BYTES, SC_BYTES = P::SC_BYTES, BAR_OFFSET = P::BAR_OFFSET;
     constexpr int HB = BN / 2;         // columns per epilogue warp: the warpgroup selects the half of the tile
-    constexpr int CHUNKS = HB / 16;    // 16-column chunks per epilogue warp and accumulator tile
+    constexpr int CHUNKS = HB / 32;    // 32-column chunks per epilogue warp and accumulator tile
     constexpr int GPK = BKC / G;       // groups per k-block: 2 (G = 64) or 1 (G = 128)
     constexpr int MMA_PER_G = G / 32;  // 8-bit MMA instructions (K = 32) per group
+    constexpr int NBUF = 512 / BN;     // accumulator tiles in tensor memory: 2 of 256 columns or 4 of 128
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t sc_base = smem_base + STAGES * STAGE_BYTES;
     const uint32_t bar_base = smem_base + BAR_OFFSET;
-    // barriers: full[S], unpacked[S], empty[S], sc_full[SC], sc_empty[SC], tmem_full[2], tmem_empty[2]
+    // barriers: full[S], unpacked[S], empty[S], sc_full[SC], sc_empty[SC], tmem_full[NBUF], tmem_empty[NBUF]
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto unp_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto empty_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
     auto scfull_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + s); };
     auto scempty_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + SC_SLOTS + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + a); };
-    auto tempty_bar = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 2 + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 4 + a); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 400);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 404);
 
@@ -136,16 +164,16 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
-            mbar_init(unp_bar(s), 2);  // one arrival per unpack warp
+            mbar_init(unp_bar(s), 64);  // every thread of the two unpack warps arrives for itself
             mbar_init(empty_bar(s), 1);
         }
         for (int s = 0; s < SC_SLOTS; ++s) {
             mbar_init(scfull_bar(s), 1);
-            mbar_init(scempty_bar(s), NUM_EPI_WARPS);
+            mbar_init(scempty_bar(s), NUM_EPI_WARPS * 32);
         }
-        for (int a = 0; a < 2; ++a) {
+        for (int a = 0; a < NBUF; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), NUM_EPI_WARPS);
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -170,7 +198,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     grid_launch_dependents();
 
     if (warp < 4) {
-        reg_dealloc<72>();
+        reg_dealloc<W4A4_AUX_REGS>();
+
         if (warp == 0) {
             // -------------------------------------------------------- TMA producer
             if (lane == 0) {
@@ -190,10 +219,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         const int slot = sc_it % SC_SLOTS;
                         if (!mbar_wait(scempty_bar(slot), ((sc_it / SC_SLOTS) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                         const uint32_t sc = sc_base + slot * SC_BYTES;
-                        mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + 2 * BM) * 4);
+                        mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + BM) * 4);
                         tma_load_2d(sc, &tmap_wscale, scfull_bar(slot), n0, kb * GPK);
                         tma_load_2d(sc + SC_SW_BYTES, &tmap_xscale, scfull_bar(slot), m0, kb * GPK);
-                        tma_load_2d(sc + SC_SW_BYTES + 2 * BM * 4, &tmap_xscale, scfull_bar(slot), m0, p.n_g + kb * GPK);
                     }
                     if (!ok) break;
                     for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
@@ -223,59 +251,65 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             }
         } else if (warp == 1) {
             // -------------------------------------------------------- MMA issuer
+            // One thread, and every instruction it executes waits its turn behind the two epilogue warps of its
+            // scheduler, so its loop is kept short: stage index, parities and the operand descriptors are carried
+            // along instead of recomputed (a descriptor differs between stages only in the address field of its low
+            // word, which cannot overflow: shared-memory addresses have 18 bits, the field holds address / 16).
             if (lane == 0) {
                 constexpr uint32_t idesc_f8 = umma_idesc(1 /*f32*/, 0 /*E4M3*/, BM, BN);
                 constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
-                uint32_t it = 0, git = 0;
+                const uint64_t desc0 = umma_desc_sw128(smem_base);
+                const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32), desc_lo0 = static_cast<uint32_t>(desc0);
+                auto desc = [&](uint32_t lo) { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
+                uint32_t s = 0, ph = 0;        // stage of the operand ring and its parity
+                uint32_t b = 0, bph = 1;       // accumulator tile and the parity its "empty" barrier is waited with
                 long long w_ops = 0, w_tempty = 0;
                 const long long t_kernel = clock64();
                 bool ok = true;
                 for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                    for (int kb = 0; ok && kb < p.num_kb; ++kb, ++it) {
-                        const int s = it % STAGES;
-                        const uint32_t ph = (it / STAGES) & 1;
-                        if (!timed_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops) ||
-                            !timed_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
+                    int groups_left = p.n_g;
+                    for (int kb = 0; ok && kb < p.num_kb; ++kb) {
+                        if (!timed_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
+                        if (!timed_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
                         tc_fence_after_sync();
-                        const uint32_t st = smem_base + s * STAGE_BYTES;
-                        const uint64_t adesc = umma_desc_sw128(st);
-                        const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
-                        const int ng_here = min(GPK, p.n_g - kb * GPK);
-                        for (int gi = 0; gi < ng_here; ++gi, ++git) {
-                            const uint32_t b = git & 1;
-                            if (!timed_wait(tempty_bar(b), ((git >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA, w_tempty)) { ok = false; break; }
-                            tc_fence_after_sync();
+                        const uint32_t a_lo = desc_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
-                            for (int k = 0; k < MMA_PER_G; ++k) {
-                                const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
-                                umma_f8f6f4(tmem_base + b * BN, adesc + 2 * kk, bdesc + 2 * kk, idesc_f8, k != 0);
+                        for (int gi = 0; gi < GPK; ++gi) {
+                            if (gi < groups_left) {
+                                if (!timed_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_tempty)) { ok = false; break; }
+                                tc_fence_after_sync();
+#pragma unroll
+                                for (int k = 0; k < MMA_PER_G; ++k) {
+                                    const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
+                                    umma_f8f6f4(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_f8, k != 0);
+                                }
+                                umma_commit(tfull_bar(b));
+                                if (++b == NBUF) { b = 0; bph ^= 1; }
                             }
-                            umma_commit(tfull_bar(b));
                         }
+                        if (!ok) break;
+                        groups_left -= GPK;
                         umma_commit(empty_bar(s));
+                        if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (!ok) break;
                     // rank-r bf16 branch: one more accumulator tile, fp32
-                    const uint32_t b = git & 1;
-                    if (!mbar_wait(tempty_bar(b), ((git >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    if (!mbar_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
-                    for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
-                        const int s = it % STAGES;
-                        const uint32_t ph = (it / STAGES) & 1;
+                    for (int lr = 0; lr < p.lr_chunks; ++lr) {
                         if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
                             !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                         tc_fence_after_sync();
-                        const uint32_t st = smem_base + s * STAGE_BYTES;
-                        const uint64_t adesc = umma_desc_sw128(st);
-                        const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+                        const uint32_t a_lo = desc_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem_base + b * BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, (lr | k) != 0);
+                            umma_bf16(tmem_base + b * BN, desc(a_lo + 2 * k), desc(b_lo + 2 * k), idesc_bf, (lr | k) != 0);
                         umma_commit(empty_bar(s));
+                        if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (!ok) break;
                     umma_commit(tfull_bar(b));
-                    ++git;
+                    if (++b == NBUF) { b = 0; bph ^= 1; }
                 }
                 flush_wait(p.status, WS_MMA_OPERANDS, w_ops);
                 flush_wait(p.status, WS_MMA_TEMPTY, w_tempty);
@@ -292,7 +326,6 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
                     ok = timed_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK, w_full);
-                    ok = __any_sync(0xffffffffu, ok);
                     if (!ok) break;
                     if (i < p.num_kb) {
                         // 16-byte piece idx = u + 64 j of the packed tile: row = idx/4 = u/4 + 16 j, piece c = u%4.
@@ -313,191 +346,200 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                             for (int j = 0; j < 8; ++j) pk[j] = src[64 * (jb + j)];
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
-                                // low nibbles of a word are codes k..k+3, high nibbles k+4..k+7 (see prepare.cu)
+                                // a word holds codes k..k+3 in bits 7, 2..0 of its bytes and codes k+4..k+7 four bit
+                                // positions further up, wrapping around (see prepare.cu): mask, rotate, mask
                                 uint4 o0, o1;
-                                o0.x = pk[j].x & 0x0F0F0F0Fu; o0.y = (pk[j].x >> 4) & 0x0F0F0F0Fu;
-                                o0.z = pk[j].y & 0x0F0F0F0Fu; o0.w = (pk[j].y >> 4) & 0x0F0F0F0Fu;
-                                o1.x = pk[j].z & 0x0F0F0F0Fu; o1.y = (pk[j].z >> 4) & 0x0F0F0F0Fu;
-                                o1.z = pk[j].w & 0x0F0F0F0Fu; o1.w = (pk[j].w >> 4) & 0x0F0F0F0Fu;
+                                o0.x = pk[j].x & kSignMag; o0.y = __funnelshift_r(pk[j].x, pk[j].x, 4) & kSignMag;
+                                o0.z = pk[j].y & kSignMag; o0.w = __funnelshift_r(pk[j].y, pk[j].y, 4) & kSignMag;
+                                o1.x = pk[j].z & kSignMag; o1.y = __funnelshift_r(pk[j].z, pk[j].z, 4) & kSignMag;
+                                o1.z = pk[j].w & kSignMag; o1.w = __funnelshift_r(pk[j].w, pk[j].w, 4) & kSignMag;
                                 *reinterpret_cast<uint4*>(d0 + (jb + j) * 2048) = o0;  // 16 rows of 128 bytes further down
                                 *reinterpret_cast<uint4*>(d1 + (jb + j) * 2048) = o1;
                             }
                         }
                         fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(unp_bar(s));
+                    // each thread signs off its own writes (a warp-wide barrier followed by one lane's arrival costs about
+                    // a hundred cycles more on this part than 32 arrivals)
+                    mbar_arrive(unp_bar(s));
                 }
             }
             if (u == 0) flush_wait(p.status, WS_UNPACK_FULL, w_full);
         }
     } else {
-        reg_alloc<208>();
+        reg_alloc<W4A4_EPI_REGS>();
         // ------------------------------------------------------------ epilogue (warps 4..11)
         // A warp owns 32 token rows (its TMEM lane quadrant) x BN/2 columns.  The accumulators are read with the
         // 16x256b shape: a thread then holds 4 rows (l/4 + 8 i) x the column pairs 2 (l%4) + {0, 1} of every block
-        // of 8 columns, so one 8-byte load of weight scales serves four rows (with the 32x32b shape, one row per
-        // thread, every thread would need all 128 column scales of every group and the shared-memory pipe, not the
-        // FMA pipe, would bound the kernel).
+        // of 8 columns, so one load of weight scales serves four rows (with the 32x32b shape, one row per thread,
+        // every thread would need all 128 column scales of every group and the shared-memory pipe, not the FMA
+        // pipe, would bound the kernel).  A chunk is 32 columns: two .x4 loads (TMEM lanes 0..15 and 16..31 of the
+        // quadrant), 32 values per thread, and the 8 weight scales of the thread's columns, which the layer stores
+        // side by side (see wscale_index in common.h), in two 16-byte loads.
+        //
+        // The accumulator tiles of an output tile (one per K-group, then the rank-r one) are one stream: while the
+        // last chunk of a tile is folded in, the next tile's barrier is tested (not waited for) and, if it has
+        // completed, its first chunk is requested, so that in the steady state neither the hand-over nor the first
+        // tensor-memory round trip is paid between groups.
         const int q = warp & 3;
         const int half = (warp - 4) >> 2;
         const int lr4 = lane >> 2;        // row inside a group of 8
         const int lc2 = (lane & 3) * 2;   // first of this thread's two columns inside a block of 8
-        uint32_t git = 0, sc_it = 0;
+        uint32_t b = 0, bph = 0;          // accumulator tile read next, parity its "full" barrier is waited with
+        uint32_t slot = 0, sph = 0;       // scale slot of the current k-block, parity of its "full" barrier
         long long w_tfull = 0, w_sc = 0;
         const long long t_epi = clock64();
+        const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * HB;
+        const float* sc0 = reinterpret_cast<const float*>(smem_gen + STAGES * STAGE_BYTES);
+        // No vote after a wait: the warp is converged there, so the barrier test, the abort flag and the clock are read
+        // by one instruction for all lanes and every lane gets the same answer.
         bool ok = true;
+        uint32_t raw[2][32];  // [0..15]: TMEM lanes 0..15 of the quadrant (rows i = 0, 1), [16..31]: lanes 16..31
+        auto request_chunk = [&](uint32_t buf, int c, uint32_t* dst) {
+            tmem_ld_16x256b_x4(taddr0 + buf * BN + c * 32, dst);
+            tmem_ld_16x256b_x4(taddr0 + buf * BN + (16u << 16) + c * 32, dst + 16);
+        };
+        auto release_tile = [&](uint32_t buf) {  // every tcgen05.ld of this thread on the tile has completed
+            tc_fence_before_sync();
+            mbar_arrive(tempty_bar(buf));  // all lanes arrive (see the unpack warps' note on the cost of electing one)
+        };
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
             const int rbase = m0 + q * 32 + lr4;  // this thread's rows: rbase + 8 i, i = 0..3
             const int colbase = n0 + half * HB;
-            float accf[HB];  // [((chunk c) * 2 + (block cb)) * 4 + row i] * 2 + {0, 1}
+            __align__(8) float accf[HB];  // [(block of 8 columns) * 4 + row i] * 2 + {0, 1}
 #pragma unroll
             for (int j = 0; j < HB; ++j) accf[j] = 0.f;
 
-            for (int kb = 0; ok && kb < p.num_kb; ++kb, ++sc_it) {
-                const int slot = sc_it % SC_SLOTS;
-                ok = timed_wait(scfull_bar(slot), (sc_it / SC_SLOTS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc);
-                ok = __any_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const float* s_sw = reinterpret_cast<const float*>(smem_gen + STAGES * STAGE_BYTES + slot * SC_BYTES);
-                const float* s_sx = s_sw + 2 * BN;
-                const int ng_here = min(GPK, p.n_g - kb * GPK);
-                for (int gi = 0; gi < ng_here; ++gi, ++git) {
-                    const uint32_t b = git & 1;
-                    ok = timed_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
-                    ok = __any_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    // the accumulator holds S = 2^-18 sum q_x (q_w + 8):  s_x P = fma(S, 2^18 s_x, e),  e = -8 s_x sum q_x
-                    float sxv[4], ev[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        sxv[i] = s_sx[gi * BM + q * 32 + lr4 + 8 * i] * 262144.0f;
-                        ev[i] = s_sx[(2 + gi) * BM + q * 32 + lr4 + 8 * i];
-                    }
-                    const float* swp = s_sw + gi * BN + half * HB + lc2;
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * HB;
-                    // software pipeline over the 16-column chunks: the loads of chunk c+1 are in flight while
-                    // chunk c is folded in (tcgen05.wait::ld waits for every outstanding load, hence depth one)
-                    uint32_t raw[2][16];  // [0..7]: TMEM lanes 0..15 of the quadrant (rows i = 0, 1), [8..15]: lanes 16..31
-                    tmem_ld_16x256b_x2(taddr, raw[0]);
-                    tmem_ld_16x256b_x2(taddr + (16u << 16), raw[0] + 8);
-#pragma unroll
-                    for (int c = 0; c < CHUNKS; ++c) {
-                        uint32_t (&cur)[16] = raw[c & 1];
-                        // this chunk's weight scales: requested before the wait so that their latency hides behind it
-                        float2 w[2];
-                        if constexpr (!kPartials) {
-                            w[0] = *reinterpret_cast<const float2*>(swp + c * 16);
-                            w[1] = *reinterpret_cast<const float2*>(swp + c * 16 + 8);
-                        }
-                        tmem_ld_wait();
-                        tmem_ld_fence(cur);
-                        if (c < CHUNKS - 1) {
-                            tmem_ld_16x256b_x2(taddr + (c + 1) * 16, raw[(c + 1) & 1]);
-                            tmem_ld_16x256b_x2(taddr + (16u << 16) + (c + 1) * 16, raw[(c + 1) & 1] + 8);
-                        } else {
-                            // the whole tile is in registers: hand it back to the MMA warp
-                            tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(tempty_bar(b));
-                        }
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                            for (int cb = 0; cb < 2; ++cb) {
-#pragma unroll
-                                for (int rr = 0; rr < 2; ++rr) {
-                                    const int i = 2 * h + rr;
-                                    const int pidx = 8 * h + 4 * cb + 2 * rr;
-                                    if constexpr (kPartials) {
-                                        // unit scales here: fma(S, 2^18, -8 sum q_x) = P, an integer
-                                        const float sxs = sxv[i], e = ev[i];
-                                        const int row = rbase + 8 * i;
-                                        const int col = colbase + c * 16 + cb * 8 + lc2;
-                                        if (row < p.M && col < p.N) {
-                                            const int g = kb * GPK + gi;
-                                            *reinterpret_cast<int2*>(p.partials + (static_cast<size_t>(g) * p.M + row) * p.N + col) =
-                                                make_int2(__float2int_rn(fmaf(__uint_as_float(cur[pidx]), sxs, e)),
-                                                          __float2int_rn(fmaf(__uint_as_float(cur[pidx + 1]), sxs, e)));
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                        if constexpr (!kPartials) {
-                            // two passes, each ordered so that consecutive instructions share operands (the token's scale
-                            // and correction in the first, the column's weight scale in the second): shared operands come
-                            // from the operand-reuse latches instead of the register banks
-                            float t[16];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                                for (int cb = 0; cb < 2; ++cb)
-#pragma unroll
-                                    for (int bit = 0; bit < 2; ++bit) {
-                                        const int pidx = 8 * (i >> 1) + 4 * cb + 2 * (i & 1) + bit;
-                                        t[pidx] = fmaf(__uint_as_float(cur[pidx]), sxv[i], ev[i]);
-                                    }
-#pragma unroll
-                            for (int cb = 0; cb < 2; ++cb)
-#pragma unroll
-                                for (int bit = 0; bit < 2; ++bit)
-#pragma unroll
-                                    for (int i = 0; i < 4; ++i) {
-                                        const int pidx = 8 * (i >> 1) + 4 * cb + 2 * (i & 1) + bit;
-                                        const int a = ((c * 2 + cb) * 4 + i) * 2 + bit;
-                                        accf[a] = fmaf(t[pidx], bit ? w[cb].y : w[cb].x, accf[a]);
-                                    }
-                        }
-                    }
-                }
-                if (!ok) break;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(scempty_bar(slot));
-            }
+            // first scales and first accumulator tile of this output tile
+            ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc) &&
+                 timed_wait(tfull_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
             if (!ok) break;
-            // rank-r branch: fp32 tile
-            {
-                const uint32_t b = git & 1;
-                ok = timed_wait(tfull_bar(b), (git >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
-                ok = __any_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + half * HB;
+            tc_fence_after_sync();
+            request_chunk(b, 0, raw[0]);
+
+            for (int g = 0; g < p.n_g; ++g) {
+                const int gi = g & (GPK - 1);
+                const bool last_of_kb = gi == GPK - 1 || g == p.n_g - 1;
+                const float* s_sw = sc0 + slot * (SC_BYTES / 4);
+                // the accumulator holds S = 2^-18 P
+                float sxv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sxv[i] = s_sw[2 * BN + gi * BM + q * 32 + lr4 + 8 * i];
+                const float4* swp = reinterpret_cast<const float4*>(s_sw + gi * BN + half * HB + 4 * lc2);
+                // what comes after this tile: the next group's, or the rank-r tile
+                const uint32_t nb = b + 1 == NBUF ? 0 : b + 1, nbph = b + 1 == NBUF ? bph ^ 1 : bph;
+                const uint32_t nslot = slot + 1 == SC_SLOTS ? 0 : slot + 1, nsph = slot + 1 == SC_SLOTS ? sph ^ 1 : sph;
+                const bool new_scales = last_of_kb && g + 1 < p.n_g;
+                bool ahead = false;
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
-                    uint32_t raw[16];
-                    tmem_ld_16x256b_x2(taddr + c * 16, raw);
-                    tmem_ld_16x256b_x2(taddr + (16u << 16) + c * 16, raw + 8);
-                    tmem_ld_wait();
-                    tmem_ld_fence(raw);
+                    uint32_t (&cur)[32] = raw[c & 1];
+                    // this chunk's weight scales: requested before the wait so that their latency hides behind it
+                    float w[8];
+                    if constexpr (!kPartials) {
+                        const float4 wa = swp[c * 8], wb = swp[c * 8 + 1];
+                        w[0] = wa.x; w[1] = wa.y; w[2] = wa.z; w[3] = wa.w;
+                        w[4] = wb.x; w[5] = wb.y; w[6] = wb.z; w[7] = wb.w;
+                    }
+                    tmem_ld_wait();  // waits for every outstanding load, hence a look-ahead of one chunk
+                    tmem_ld_fence(cur);
+                    if (c < CHUNKS - 1) {
+                        request_chunk(b, c + 1, raw[(c + 1) & 1]);
+                    } else {
+                        // the whole tile is in registers: hand it back to the MMA warp, and look at the next one
+                        release_tile(b);
+                        ahead = mbar_test_wait(tfull_bar(nb), nbph) && (!new_scales || mbar_test_wait(scfull_bar(nslot), nsph));
+                        if (ahead) {
+                            tc_fence_after_sync();
+                            request_chunk(nb, 0, raw[0]);  // CHUNKS is even: the last chunk sits in raw[1]
+                        }
+                    }
+                    if constexpr (kPartials) {
+                        // unit scales here: 2^18 S = P, an integer
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                        for (int i = 0; i < 4; ++i)
 #pragma unroll
-                        for (int cb = 0; cb < 2; ++cb)
-#pragma unroll
-                            for (int rr = 0; rr < 2; ++rr) {
-                                const int pidx = 8 * h + 4 * cb + 2 * rr;
-                                const int a = ((c * 2 + cb) * 4 + 2 * h + rr) * 2;
-                                accf[a] += __uint_as_float(raw[pidx]);
-                                accf[a + 1] += __uint_as_float(raw[pidx + 1]);
+                            for (int cb = 0; cb < 4; ++cb) {
+                                const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
+                                const int row = rbase + 8 * i;
+                                const int col = colbase + c * 32 + cb * 8 + lc2;
+                                if (row < p.M && col < p.N)
+                                    *reinterpret_cast<int2*>(p.partials + (static_cast<size_t>(g) * p.M + row) * p.N + col) =
+                                        make_int2(__float2int_rn(__uint_as_float(cur[pidx]) * 262144.0f),
+                                                  __float2int_rn(__uint_as_float(cur[pidx + 1]) * 262144.0f));
                             }
+                    } else {
+                        // t = S s_x for two adjacent columns at a time (one packed multiply: half the issue slots of two
+                        // scalar ones), then acc = fma(t, 2^18 s_w, acc); both passes ordered so that consecutive
+                        // instructions share an operand (the token's scale in the first, the column's in the second)
+                        uint64_t t2[16];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint64_t sx2 = pack_f32x2(sxv[i], sxv[i]);
+#pragma unroll
+                            for (int cb = 0; cb < 4; ++cb) {
+                                const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
+                                t2[pidx >> 1] = mul_f32x2(pack_u32x2(cur[pidx], cur[pidx + 1]), sx2);
+                            }
+                        }
+#pragma unroll
+                        for (int cb = 0; cb < 4; ++cb)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
+                                const int a = ((c * 4 + cb) * 4 + i) * 2;
+                                float t_lo, t_hi;
+                                unpack_f32x2(t2[pidx >> 1], t_lo, t_hi);
+                                accf[a] = fmaf(t_lo, w[2 * cb], accf[a]);
+                                accf[a + 1] = fmaf(t_hi, w[2 * cb + 1], accf[a + 1]);
+                            }
+                    }
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(b));
-                ++git;
+                if (last_of_kb) {
+                    // this k-block's scales have all been read (the multiply-adds that consumed them were issued above)
+                    mbar_arrive(scempty_bar(slot));
+                    slot = nslot;
+                    sph = nsph;
+                }
+                b = nb;
+                bph = nbph;
+                if (!ahead) {
+                    if (new_scales) ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc);
+                    ok = ok && timed_wait(tfull_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    request_chunk(b, 0, raw[0]);
+                }
             }
+            if (!ok) break;
+            // rank-r branch: an fp32 tile whose first chunk is already on its way
+#pragma unroll
+            for (int c = 0; c < CHUNKS; ++c) {
+                uint32_t (&cur)[32] = raw[c & 1];
+                tmem_ld_wait();
+                tmem_ld_fence(cur);
+                if (c < CHUNKS - 1) request_chunk(b, c + 1, raw[(c + 1) & 1]);
+                else release_tile(b);
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int cb = 0; cb < 4; ++cb) {
+                        const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
+                        const int a = ((c * 4 + cb) * 4 + i) * 2;
+                        accf[a] += __uint_as_float(cur[pidx]);
+                        accf[a + 1] += __uint_as_float(cur[pidx + 1]);
+                    }
+            }
+            if (++b == NBUF) { b = 0; bph ^= 1; }
             if constexpr (!kPartials) {
                 // A lane holds 2 of the 8 columns of every block; four blocks are transposed inside the quad of lanes
                 // (two exchange steps) so that each lane ends up with all 8 columns = 16 bytes of one block and the
                 // warp writes 64 contiguous bytes per row.
                 const int j = lane & 3;
 #pragma unroll
-                for (int m = 0; m < CHUNKS / 2; ++m) {
+                for (int m = 0; m < CHUNKS; ++m) {
                     float2 bv[4];
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
@@ -564,7 +606,7 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
     st = encode_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K_lp, (uint64_t)a.M,
                         (uint64_t)g.K_lp, BKC, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != DIROTQ_OK) return st;
-    st = encode_tmap_2d(&tmap_xscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xscale, (uint64_t)a.ldm, (uint64_t)2 * g.n_g,
+    st = encode_tmap_2d(&tmap_xscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xscale, (uint64_t)a.ldm, (uint64_t)g.n_g,
                         (uint64_t)a.ldm * 4, BM, BKC / g.G, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != DIROTQ_OK) return st;
     st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,
