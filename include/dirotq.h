@@ -375,6 +375,19 @@ DIROTQ_API dirotq_status_t dirotq_linear_noalloc(const void* x, int M, const dir
 DIROTQ_API dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* status_word, float* tera_ops_per_s,
                                                  dirotq_stream_t stream);
 
+/* ---- failure-path check (no counterpart in the paper) ---------------------------------------- */
+
+/* Every wait on a barrier inside the library's kernels is bounded: when its time runs out the
+ * waiting role records a code in the workspace's status word and the kernel returns, so that a
+ * logic error shows up as DIROTQ_ERR_DEVICE_TIMEOUT from dirotq_workspace_status and not as a hung
+ * GPU.  This entry point runs that give-up path on purpose and harmlessly: one warp of one small
+ * kernel waits, with the same wait routine, on a barrier in its own shared memory that nothing
+ * arrives on, gives up after limit_us microseconds (1..100000), writes code 5 to the status word
+ * at the start of `workspace` (a device buffer of at least 256 bytes whose first word is zero) and
+ * exits normally.  It touches no other memory, no TMA and no tensor memory.  Enqueues on `stream`,
+ * does not synchronise.  Zero the status word (256 bytes) before reusing the workspace. */
+DIROTQ_API dirotq_status_t dirotq_wait_selftest(void* workspace, unsigned int limit_us, dirotq_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

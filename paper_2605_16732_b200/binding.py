@@ -26,7 +26,7 @@ EXPORTED = [
     "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_wait_counters", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
-    "dirotq_mma_rate_probe", "dirotq_linear_noalloc",
+    "dirotq_mma_rate_probe", "dirotq_linear_noalloc", "dirotq_wait_selftest",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
     "dirotq_prepare_layer_codes", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_layer_export.argtypes = [vp, vp, vp, vp, vp, vp]
         L.dirotq_linear_noalloc.argtypes = [vp, i, vp, vp, vp, vp]
         L.dirotq_mma_rate_probe.argtypes = [i, i, vp, ctypes.POINTER(ctypes.c_float), vp]
+        L.dirotq_wait_selftest.argtypes = [vp, ctypes.c_uint, vp]
         L.dirotq_layer_bytes_nvfp4.argtypes = [i, i, i, psz]
         L.dirotq_prepare_layer_nvfp4.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_workspace_export_nvfp4.argtypes = [vp, i, vp, vp, vp, vp, vp]
@@ -277,6 +278,11 @@ def dirotq_mma_rate_probe(kind: int, iters: int = 20000, stream=None) -> float:
     if int(status[0].item()) != 0:
         raise DirotqError(6, "dirotq_mma_rate_probe")
     return float(out.value)
+
+
+def dirotq_wait_selftest(workspace: torch.Tensor, limit_us: int = 1000, stream=None) -> None:
+    """Runs the bounded-wait give-up path on purpose (see the header); the status word of `workspace` then reads 5."""
+    _check(lib().dirotq_wait_selftest(workspace.data_ptr(), int(limit_us), _stream(stream)), "dirotq_wait_selftest")
 
 
 def dirotq_linear_noalloc(x: torch.Tensor, layer: Layer, y: torch.Tensor, device_status: torch.Tensor | None = None,

@@ -482,6 +482,10 @@ static dirotq_status_t check_call(const dirotq_layer_t* layer, int M, const void
     if (rotates && layer->geo.no_rot) return DIROTQ_ERR_INVALID_ARG;  // a sibling layer holds no rotation
     if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return DIROTQ_ERR_INVALID_ARG;
     if (workspace_bytes < workspace_need(layer, M)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    // the layer's blob and tensor maps belong to the device it was prepared on: that device must be current
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DIROTQ_ERR_CUDA;
+    if (dev != layer->device) return DIROTQ_ERR_INVALID_ARG;
     return DIROTQ_OK;
 }
 

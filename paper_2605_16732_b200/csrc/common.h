@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <utility>
 #include <stddef.h>
 #include <stdint.h>
@@ -302,6 +303,22 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
     cfg.numAttrs = pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
+
+// Raising a kernel's dynamic shared-memory limit (cudaFuncSetAttribute) applies to the CURRENT device only, so what has been
+// done is remembered per device: one table of flags per launch site, indexed by device and kernel variant.  Safe to
+// call from several host threads (the attribute call is idempotent; the flag only saves repeating it).
+template <int VARIANTS>
+struct SmemOptIn {
+    std::atomic<bool> done[64][VARIANTS];
+    template <typename Kernel>
+    bool ensure(Kernel kern, int variant, int device, int bytes) {
+        const bool cached = device >= 0 && device < 64;
+        if (cached && done[device][variant].load(std::memory_order_acquire)) return true;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+        if (cached) done[device][variant].store(true, std::memory_order_release);
+        return true;
+    }
+};
 
 dirotq_status_t set_nvfp4_tile_columns(int columns);
 dirotq_status_t set_w4a8_tile_columns(int columns);

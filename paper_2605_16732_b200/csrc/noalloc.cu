@@ -11,6 +11,7 @@
 // calls share it.
 #include "common.h"
 
+#include <atomic>
 #include <stdio.h>
 
 namespace dirotq {
@@ -21,8 +22,8 @@ constexpr size_t kStaticWorkspaceBytes = 16u << 20;
 static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes + 1024];
 
 struct PerDevice {
-    bool ready;
-    char* base;  // DEVICE address of the aligned window
+    std::atomic<bool> ready;   // set (release) after `base` is written, read (acquire) before it is used
+    std::atomic<char*> base;   // DEVICE address of the aligned window
 };
 PerDevice g_dev[64];
 
@@ -30,15 +31,16 @@ PerDevice g_dev[64];
 // device address has to be asked for, once per device, with that device current.
 dirotq_status_t static_workspace(int device, char** out) {
     if (device < 0 || device >= 64) return DIROTQ_ERR_INVALID_ARG;
-    if (!g_dev[device].ready) {
+    if (!g_dev[device].ready.load(std::memory_order_acquire)) {
+        // two threads racing here both ask and both get the same address
         void* p = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(&p, g_static_workspace);
         if (e != cudaSuccess || p == nullptr) return DIROTQ_ERR_CUDA;
         const uintptr_t a = (reinterpret_cast<uintptr_t>(p) + 1023u) & ~static_cast<uintptr_t>(1023u);
-        g_dev[device].base = reinterpret_cast<char*>(a);
-        g_dev[device].ready = true;
+        g_dev[device].base.store(reinterpret_cast<char*>(a), std::memory_order_relaxed);
+        g_dev[device].ready.store(true, std::memory_order_release);
     }
-    *out = g_dev[device].base;
+    *out = g_dev[device].base.load(std::memory_order_relaxed);
     return DIROTQ_OK;
 }
 

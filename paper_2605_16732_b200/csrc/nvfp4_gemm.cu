@@ -149,8 +149,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), NUM_EPI_WARPS);
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
         }
+        mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_codes);
@@ -343,8 +344,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             for (int c = 0; c < HB / 32; ++c) tmem_ld_32x32b_x32(taddr + c * 32, raw[c]);
             tmem_ld_wait();
             tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            mbar_arrive(tempty_bar(acc));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             if (row < p.M) {
                 const float* bq = s_b + half * HB;
                 uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + n0 + half * HB;
@@ -368,6 +368,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         }
     }
 
+    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -399,13 +400,8 @@ static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4Ge
     p.y = a.y; p.status = a.status;
     const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(nvfp4_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<BN>::SMEM_BYTES) !=
-            cudaSuccess)
-            return DIROTQ_ERR_CUDA;
-        attr_set = true;
-    }
+    static SmemOptIn<1> opt_in;
+    if (!opt_in.ensure(nvfp4_gemm_kernel<BN>, 0, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand
     const cudaError_t err = launch_kernel(nvfp4_gemm_kernel<BN>, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true,
                                           tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);

@@ -62,10 +62,32 @@ __global__ void __launch_bounds__(PEAK_THREADS, 1) mma_peak_kernel(int kind, int
     }
 }
 
+// One warp waits, with the same bounded wait every kernel of the library uses, on a barrier nobody will ever arrive on:
+// the wait gives up after `limit_ns`, records its code in the status word and the kernel returns normally.
+__global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, DEV_TIMEOUT_SELFTEST, limit_ns);
+    (void)ok;  // false: either this thread's clock ran out or it saw another thread's abort flag
+}
+
 }  // namespace
 }  // namespace dirotq
 
 using namespace dirotq;
+
+extern "C" dirotq_status_t dirotq_wait_selftest(void* workspace, unsigned int limit_us, dirotq_stream_t stream) {
+    if (!workspace || limit_us < 1 || limit_us > 100000) return DIROTQ_ERR_INVALID_ARG;
+    wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<int*>(workspace),
+                                                                         static_cast<unsigned long long>(limit_us) * 1000ull);
+    return cudaGetLastError() == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
 
 extern "C" dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* status_word, float* tera_ops_per_s,
                                                 dirotq_stream_t stream) {
@@ -76,12 +98,8 @@ extern "C" dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* stat
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DIROTQ_ERR_CUDA;
     if (major != 10) return DIROTQ_ERR_ARCH;
-    static bool attr = false;
-    if (!attr) {
-        if (cudaFuncSetAttribute(mma_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PEAK_SMEM) != cudaSuccess)
-            return DIROTQ_ERR_CUDA;
-        attr = true;
-    }
+    static SmemOptIn<1> opt_in;
+    if (!opt_in.ensure(mma_peak_kernel, 0, dev, PEAK_SMEM)) return DIROTQ_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaEvent_t e0, e1;
     if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return DIROTQ_ERR_CUDA;

@@ -14,6 +14,7 @@ enum : int {
     DEV_TIMEOUT_MMA = 2,
     DEV_TIMEOUT_UNPACK = 3,
     DEV_TIMEOUT_EPILOGUE = 4,
+    DEV_TIMEOUT_SELFTEST = 5,  // written by the wait self-test only
 };
 
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
@@ -79,7 +80,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // caller then leaves its loops and goes to the common teardown.  `abort_flag` is a word in
 // shared memory, `status` a word in global memory that the host reads.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+                                          int code, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
 #pragma unroll 1
@@ -89,7 +90,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag != 0) return false;
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = code;
                 atomicCAS(status, 0, code);
                 return false;
@@ -204,6 +205,15 @@ __device__ __forceinline__ void umma_f8f6f4(uint32_t d_tmem, uint64_t adesc, uin
 // All MMAs issued so far by this thread arrive on `bar` when they have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Error path only.  After a bounded wait gave up, MMAs that were already issued may still be running: the issuing
+// thread waits (again with a limit) for them on a spare barrier (count 1, never used otherwise) before the tensor
+// memory they write into is freed.
+__device__ __forceinline__ void umma_drain(uint32_t spare_bar) {
+    umma_commit(spare_bar);
+    const unsigned long long t0 = globaltimer_ns();
+    while (!mbar_try_wait(spare_bar, 0) && globaltimer_ns() - t0 < 100000000ull) {}
 }
 
 // ---------------------------------------------------------------- programmatic dependent launch

@@ -200,8 +200,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 8);  // one arrival per epilogue warp
+            mbar_init(tempty_bar(a), 8 * 32);  // every thread of the eight epilogue warps arrives
         }
+        mbar_init(bar_base + 136u, 1);  // spare: see umma_drain
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
@@ -511,8 +512,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             }
             // release the accumulator: every tcgen05.ld of this warp has completed
             tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            mbar_arrive(tempty_bar(acc));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
             if (!PH && n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
                 for (int c = p.r; c < p.r_pad0; c += 8)
@@ -525,6 +525,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     }
 
     // ---------------------------------------------------------------- teardown
+    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 136u);  // a wait gave up: let issued MMAs finish first
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -610,14 +611,11 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         {rotate_quant_kernel<64, 0, 256, 256>, rotate_quant_kernel<128, 0, 256, 256>, rotate_quant_kernel<64, 1, 256, 256>,
          rotate_quant_kernel<64, 2, 256, 256>, rotate_quant_kernel<128, 2, 256, 256>, rotate_quant_kernel<64, 3, 256, 256>}};
     const KernelFn kern = table[plan - 1][vi];
-    // a dependent launch needs a kernel as the previous operation of the stream: the W4A8 path puts a memset there
+    // the W4A8 path puts a memset in front of this kernel; programmatic serialization only relaxes the wait for a
+    // preceding KERNEL, so nothing would be gained there and the launch is a plain one
     const bool dependent = g.fmt != 3;
-    static bool attr_set[3][6] = {};
-    if (!attr_set[plan - 1][vi]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-            return DIROTQ_ERR_CUDA;
-        attr_set[plan - 1][vi] = true;
-    }
+    static SmemOptIn<18> opt_in;
+    if (!opt_in.ensure(kern, (plan - 1) * 6 + vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, plan == 1 ? L->tmap_qt128 : L->tmap_qt,
                          p) == cudaSuccess
                ? DIROTQ_OK
@@ -645,11 +643,8 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
         RotKernelParams p1 = p;
         p1.n_out = g.r_pad; p1.k_red = g.K; p1.K_l = 0; p1.r = g.r_pad; p1.xsub = nullptr;
         const KernelFn k1 = rotate_quant_kernel<64, 0, 128, 128>;
-        static bool attr1 = false;
-        if (!attr1) {
-            if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return DIROTQ_ERR_CUDA;
-            attr1 = true;
-        }
+        static SmemOptIn<1> opt_in1;
+        if (!opt_in1.ensure(k1, 0, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
         long tiles = static_cast<long>((a.M + 127) / 128) * ((g.r_pad + 127) / 128);
         // Few row tiles leave most SMs idle while x streams through: cut the reduction into ranges, one tile each.  The
         // ranges' fp32 sums are parked in the (still unused) code region of the workspace and added up in range order.
@@ -686,11 +681,8 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
                                         rotate_quant_kernel<64, 1, 256, 128, true>};
         const KernelFn k2 = k2s[vi];
         if (g.fmt == 1) { p2.xsf = a.xsf; p2.K4 = g.K4; p2.nkb64p = g.nkb64p; p2.ex = L->act_scale_log2; }
-        static bool attr2[3] = {false, false, false};
-        if (!attr2[vi]) {
-            if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return DIROTQ_ERR_CUDA;
-            attr2[vi] = true;
-        }
+        static SmemOptIn<3> opt_in2;
+        if (!opt_in2.ensure(k2, vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
         const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.K + 255) / 256);
         if (launch_kernel(k2, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_xh, L->tmap_qt,
                           p2) != cudaSuccess)

@@ -175,6 +175,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             mbar_init(tfull_bar(a), 1);
             mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
         }
+        mbar_init(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 8), 1);  // spare: see umma_drain
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_codes);
@@ -578,6 +579,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     }
 
     // ---------------------------------------------------------------- teardown
+    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 8));  // a wait gave up: let issued MMAs finish first
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -628,13 +630,9 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
     const bool dbg = a.partials != nullptr;
     if (g.G == 64) kern = dbg ? w4a4_gemm_kernel<64, true, BN> : w4a4_gemm_kernel<64, false, BN>;
     else           kern = dbg ? w4a4_gemm_kernel<128, true, BN> : w4a4_gemm_kernel<128, false, BN>;
-    static bool attr_set[4] = {false, false, false, false};
+    static SmemOptIn<4> opt_in;  // one per instantiation of this launcher, i.e. per tile width
     const int vi = (g.G == 64 ? 0 : 2) + (dbg ? 1 : 0);
-    if (!attr_set[vi]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<BN>::SMEM_BYTES) != cudaSuccess)
-            return DIROTQ_ERR_CUDA;
-        attr_set[vi] = true;
-    }
+    if (!opt_in.ensure(kern, vi, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     const bool narrow = BN == 128;
     const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
                                           narrow ? L->tmap_wpacked128 : L->tmap_wpacked,

@@ -100,11 +100,12 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
-            mbar_init(unp_bar(s), NUM_UNPACK_WARPS);
+            mbar_init(unp_bar(s), NUM_UNPACK_WARPS * 32);
             mbar_init(empty_bar(s), 1);
         }
         mbar_init(tfull_bar, 1);
-        mbar_init(tempty_bar, NUM_EPI_WARPS);
+        mbar_init(tempty_bar, NUM_EPI_WARPS * 32);
+        mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_codes);
@@ -241,8 +242,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                     fence_proxy_async_smem();
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(unp_bar(s));
+                mbar_arrive(unp_bar(s));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             }
         }
     } else {
@@ -301,8 +301,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 tmem_ld_fence32(lr);
                 if (c == (half + 1) * CPH - 1) {
                     tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar);
+                    mbar_arrive(tempty_bar);
                 }
                 const int col = n0 + c * 32;
                 if (row < p.M) {
@@ -342,6 +341,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         }
     }
 
+    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -373,12 +373,8 @@ static dirotq_status_t launch_w4a8_gemm_bn(const dirotq_layer* L, const A8GemmAr
     const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
     const bool dbg = a.partials != nullptr;
     auto kern = dbg ? w4a8_gemm_kernel<true, BN> : w4a8_gemm_kernel<false, BN>;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[dbg]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<BN>::SMEM_BYTES) != cudaSuccess)
-            return DIROTQ_ERR_CUDA;
-        attr_set[dbg] = true;
-    }
+    static SmemOptIn<2> opt_in;
+    if (!opt_in.ensure(kern, dbg ? 1 : 0, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     const bool narrow = BN == 128;
     const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
                                           narrow ? L->tmap_wpacked128 : L->tmap_wpacked, tmap_xh,

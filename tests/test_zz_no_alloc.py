@@ -99,3 +99,38 @@ def test_noalloc_matches_linear_for_every_layer_format():
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), name
         assert float(ref.float().abs().max()) > 0
         ly.close()
+
+
+@pytest.mark.parametrize("fmt", ["int4_ph", "nvfp4_ph"])
+def test_noalloc_with_the_split_first_step_of_the_projection_form(fmt):
+    """K = 2048 with few token rows: the projection form's first step splits its reduction and parks the ranges' partial
+    sums in the code region of the workspace, which the second pass then overwrites -- here that region is the shared
+    array, still holding what another layer's call left there."""
+    K, N, r, G, M = 2048, 256, 32, 64, 512
+    spec = synth.LayerSpec(K=K, N=N, r=r, G=G, model=synth.FLUX, seed=41, calib_tokens=512)
+    W, bias = synth.make_weights(spec)
+    g = np.random.default_rng(41)
+    Uh = torch.from_numpy(np.linalg.qr(g.standard_normal((K, r)))[0]).cuda().contiguous()
+    Wd, b = torch.from_numpy(W).cuda(), _bf(bias)
+    layer = (dq.dirotq_prepare_layer_ph(Wd, Uh, G, bias=b) if fmt == "int4_ph"
+             else dq.dirotq_prepare_layer_nvfp4_ph(Wd, Uh, -6, bias=b))
+    _, other = _layer(512, 768, 32, 64, seed=42)
+    spec_o = synth.LayerSpec(K=512, N=768, r=32, G=64, model=synth.PIXART, seed=42, calib_tokens=512)
+    x = _bf(synth.make_tokens(spec, M, batch_seed=6))
+    xo = _bf(synth.make_tokens(spec_o, 300, batch_seed=7))
+    ref = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = dq.alloc_workspace(layer, M)
+    assert ws.numel() <= 16 << 20
+    dq.dirotq_linear(x, layer, ref, ws)
+    assert dq.dirotq_workspace_status(ws) == 0
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    yo = torch.zeros((300, 768), dtype=torch.bfloat16, device="cuda")
+    for call in range(2):
+        dq.dirotq_linear_noalloc(xo, other, yo, status)  # leaves its own codes and scales in the shared array
+        out = torch.zeros_like(ref)
+        dq.dirotq_linear_noalloc(x, layer, out, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), f"{fmt} call {call}"
+    layer.close()
+    other.close()
