@@ -18,7 +18,7 @@
  *   - the r high-precision coefficients and the r high rows of W~ are bf16,
  *   - every scale is a bf16 value and the rounded scale is used to divide,
  *   - the output is bf16.
- * Readings taken where the paper is silent (listed again in the design notes):
+ * Readings taken where the paper is silent:
  *   groups are counted from the first low-precision column; the last group may be
  *   ragged; rounding is half-to-even; codes are clipped to [-7, 7]; a group whose
  *   absmax is zero has scale 0 and codes 0; bias is added before the final rounding.

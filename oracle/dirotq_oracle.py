@@ -220,7 +220,7 @@ def linear_deployed(x_bits, layer, bias=None, want_t: bool = True):
 #     x~_h = bf16(x U_hb),   d = x - x~_h U_hb^T,   x~_l = d H,   y = x~_h (U_hb^T W) + Q4(x~_l) Q4(H^T W) + bias
 # with U_hb = bf16(U_h) and H block-diagonal, one orthonormal Hadamard block per quantization group.  Because d is the
 # residual of the ROUNDED projection, x = x~_h U_hb^T + d holds exactly, so the layer equals x W when nothing is
-# quantized, for any U_h.  No CUDA path computes this form yet; these functions are the reference it will be held to.
+# quantized, for any U_h.  These functions are the reference the library's projection-form layers are held to.
 
 def hadamard(n: int) -> np.ndarray:
     """Orthonormal Sylvester-Hadamard matrix of order n (a power of two): entries +-1/sqrt(n), symmetric."""

@@ -1,4 +1,4 @@
-"""Timing sweep over the task's other configurations (bench.py keeps to its one-line contract).
+"""Timing sweep over the configurations bench.py does not time (bench.py keeps to its one-line contract).
 
     python -m paper_2605_16732_b200.suite [--configs 1,2,4,5] [--iters 20]
 

@@ -1,4 +1,4 @@
-"""Parity at the full sizes of the task's configurations, in the launch configuration bench.py times
+"""Parity at the full sizes of the benchmarked configurations (PixArt- and FLUX-shaped layers), in the launch configuration bench.py times
 (persistent 148-CTA grids, many tiles per CTA), on sampled outputs the oracle can compute one by one.
 
 Token rows are independent (per-token scales, row-wise GEMM) and so are output columns of the weight
