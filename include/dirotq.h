@@ -217,6 +217,27 @@ DIROTQ_API dirotq_status_t dirotq_prepare_layer_codes(const void* W, int w_dtype
                                                       size_t blob_bytes, void* scratch, size_t scratch_bytes,
                                                       dirotq_stream_t stream, dirotq_layer_t** layer_out);
 
+/* ---- residual weights rounded with GPTQ inside the library (paper Sec. 4.1: the residual weight is rounded so as
+ * to minimise ||X W - X W^||^2 on calibration tokens rather than value by value; App. "Quantization details":
+ * damping 0.01, block size 128) ----
+ *
+ * As dirotq_prepare_layer (asym == 0) or dirotq_prepare_layer_asym (asym != 0), except that the folded rows
+ * r..K-1 are rounded by the GPTQ algorithm: the Hessian is X~_l^T X~_l of the calibration tokens calib_x (bf16
+ * [calib_tokens, K], DEVICE, row-major) rotated by the layer's own bf16 rotation; damp * mean(diag) is added to
+ * its diagonal (the paper uses damp = 0.01); rows are rounded in order, each row's rounding error is spread over
+ * the rows not yet rounded (weights from the upper Cholesky factor of the inverse Hessian), the rows behind the
+ * current block of `block` rows (a multiple of `group`, at most 128; the paper uses 128) are corrected once per
+ * block; a group's scale bf16(max|w|/7) is taken from its rows as they stand when the group starts.  Everything
+ * runs on the device in fp64, offline; the factorisation is an unblocked one whose cost grows with (K-r)^3, which
+ * is seconds at K = 3072.  scratch: DEVICE, dirotq_prepare_scratch_bytes_gptq bytes, free again when the call's
+ * work on `stream` has completed.  The online path and every export are those of the round-to-nearest layer. */
+DIROTQ_API dirotq_status_t dirotq_prepare_scratch_bytes_gptq(int K, int N, int r, int calib_tokens, size_t* bytes);
+DIROTQ_API dirotq_status_t dirotq_prepare_layer_gptq(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                                     const void* bias, const void* calib_x, int calib_tokens, double damp,
+                                                     int block, int asym, int K, int N, int r, int group, void* blob,
+                                                     size_t blob_bytes, void* scratch, size_t scratch_bytes,
+                                                     dirotq_stream_t stream, dirotq_layer_t** layer_out);
+
 /* ---- layers that share one rotation (paper Sec. 4.2: the rotation belongs to a layer's INPUT, so linears that read
  * the same activations, e.g. the q, k and v projections of a block, are rotated by the same Q) ----
  *

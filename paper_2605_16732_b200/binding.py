@@ -29,7 +29,7 @@ EXPORTED = [
     "dirotq_mma_rate_probe", "dirotq_linear_noalloc", "dirotq_wait_selftest",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
-    "dirotq_prepare_layer_codes", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
+    "dirotq_prepare_layer_codes", "dirotq_prepare_scratch_bytes_gptq", "dirotq_prepare_layer_gptq", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
     "dirotq_layer_export_uh", "dirotq_layer_bytes_nvfp4_ph", "dirotq_prepare_layer_nvfp4_ph", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_set_first_step_split", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
@@ -95,6 +95,9 @@ def lib() -> ctypes.CDLL:
         L.dirotq_set_dependent_launch.argtypes = [i]
         L.dirotq_set_rotation_tile.argtypes = [i]
         L.dirotq_set_first_step_split.argtypes = [i]
+        L.dirotq_prepare_scratch_bytes_gptq.argtypes = [i, i, i, i, psz]
+        L.dirotq_prepare_layer_gptq.argtypes = [vp, i, i, vp, i, vp, vp, i, ctypes.c_double, i, i, i, i, i, i, vp, sz, vp, sz,
+                                                vp, ctypes.POINTER(vp)]
         L.dirotq_prepare_layer_codes.argtypes = [vp, i, i, vp, i, vp, vp, vp, i, i, i, i, i, vp, sz, vp, sz, vp,
                                                  ctypes.POINTER(vp)]
         L.dirotq_workspace_export_asym.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -494,6 +497,30 @@ def dirotq_prepare_layer_codes(W: torch.Tensor, Q: torch.Tensor, wcodes: torch.T
                                           wscales.data_ptr(), int(asym), K, N, r, group, blob.data_ptr(), blob.numel(),
                                           scratch.data_ptr(), scratch_bytes, _stream(stream), ctypes.byref(handle))
     _check(st, "dirotq_prepare_layer_codes")
+    torch.cuda.current_stream().synchronize()
+    return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym" if asym else "int4")
+
+
+def dirotq_prepare_layer_gptq(W: torch.Tensor, Q: torch.Tensor, calib_x: torch.Tensor, r: int, group: int,
+                              bias: torch.Tensor | None = None, asym: bool = False, damp: float = 0.01, block: int = 128,
+                              w_layout: int = LAYOUT_KN, stream=None) -> Layer:
+    """As dirotq_prepare_layer(_asym), with the residual rows rounded by GPTQ on the calibration tokens calib_x (bf16 [T,K])."""
+    assert W.is_cuda and Q.is_cuda and W.is_contiguous() and Q.is_contiguous()
+    K = Q.shape[0]
+    N = W.shape[1] if w_layout == LAYOUT_KN else W.shape[0]
+    assert calib_x.is_cuda and calib_x.is_contiguous() and calib_x.dtype == torch.bfloat16 and calib_x.shape[1] == K
+    w_dtype = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    q_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Q.dtype]
+    nbytes = dirotq_layer_bytes_asym(K, N, r, group) if asym else dirotq_layer_bytes(K, N, r, group)
+    blob = _alloc_bytes(nbytes, W.device)
+    need = ctypes.c_size_t(0)
+    _check(lib().dirotq_prepare_scratch_bytes_gptq(K, N, r, calib_x.shape[0], ctypes.byref(need)), "dirotq_prepare_scratch_bytes_gptq")
+    scratch = _alloc_bytes(need.value, W.device)
+    handle = ctypes.c_void_p(0)
+    st = lib().dirotq_prepare_layer_gptq(_ptr(W), w_dtype, w_layout, _ptr(Q), q_dtype, _ptr(bias), calib_x.data_ptr(),
+                                         calib_x.shape[0], float(damp), int(block), int(asym), K, N, r, group, blob.data_ptr(),
+                                         blob.numel(), scratch.data_ptr(), need.value, _stream(stream), ctypes.byref(handle))
+    _check(st, "dirotq_prepare_layer_gptq")
     torch.cuda.current_stream().synchronize()
     return Layer(handle.value, blob, K, N, r, group, fmt="int4_asym" if asym else "int4")
 

@@ -151,11 +151,18 @@ dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_
     return DIROTQ_OK;
 }
 
+struct GptqArgs {
+    const void* calib;  // bf16 [T][K] calibration tokens (device); NULL: round to nearest
+    int T;
+    double damp;
+    int block;
+};
+
 static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
                                     const void* bias, const int8_t* wcodes, const void* wscales, int K, int N, int r,
                                     int group, void* blob, size_t blob_bytes,
                                     void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
-                                    dirotq_layer_t** layer_out) {
+                                    dirotq_layer_t** layer_out, const GptqArgs* gptq = nullptr) {
     if (!W || !Q || !blob || !scratch || !layer_out) return DIROTQ_ERR_INVALID_ARG;
     if (w_dtype != DIROTQ_DTYPE_F32 && w_dtype != DIROTQ_DTYPE_BF16) return DIROTQ_ERR_INVALID_ARG;
     if (q_dtype != DIROTQ_DTYPE_F64 && q_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
@@ -171,6 +178,12 @@ static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int 
     const BlobLayout lay = make_blob_layout(g);
     if (blob_bytes < lay.total) return DIROTQ_ERR_BUFFER_TOO_SMALL;
     if (scratch_bytes < static_cast<size_t>(K) * N * sizeof(double)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    if (gptq) {
+        if (!gptq->calib || !aligned16(gptq->calib) || gptq->T < 1 || !(gptq->damp > 0.0) || gptq->block < group ||
+            gptq->block > 128 || gptq->block % group != 0)
+            return DIROTQ_ERR_INVALID_ARG;
+        if (scratch_bytes < gptq_scratch_bytes(K, N, r, gptq->T)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    }
     int dev = 0;
     st = check_device(&dev);
     if (st != DIROTQ_OK) return st;
@@ -215,12 +228,37 @@ static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int 
     if (st == DIROTQ_OK)
         st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, static_cast<double*>(scratch),
                             static_cast<cudaStream_t>(stream));
+    if (st == DIROTQ_OK && gptq) {
+        // the round-to-nearest layer above left the folded weight in the scratch and the bf16 rotation in the blob: round
+        // the residual rows again with error feedback and put those codes and scales in place of the first ones
+        const int8_t* codes = nullptr;
+        const uint16_t* scales = nullptr;
+        st = launch_gptq_round(L, gptq->calib, gptq->T, gptq->damp, gptq->block, static_cast<char*>(scratch),
+                               static_cast<cudaStream_t>(stream), &codes, &scales);
+        if (st == DIROTQ_OK) st = launch_pack_codes(L, codes, scales, static_cast<cudaStream_t>(stream));
+    }
     if (st != DIROTQ_OK) {
         delete L;
         return st;
     }
     *layer_out = L;
     return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_scratch_bytes_gptq(int K, int N, int r, int calib_tokens, size_t* bytes) {
+    if (!bytes || K <= 0 || N <= 0 || r <= 0 || r >= K || calib_tokens < 1) return DIROTQ_ERR_INVALID_ARG;
+    *bytes = gptq_scratch_bytes(K, N, r, calib_tokens);
+    return DIROTQ_OK;
+}
+
+dirotq_status_t dirotq_prepare_layer_gptq(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,
+                                          const void* bias, const void* calib_x, int calib_tokens, double damp, int block,
+                                          int asym, int K, int N, int r, int group, void* blob, size_t blob_bytes,
+                                          void* scratch, size_t scratch_bytes, dirotq_stream_t stream,
+                                          dirotq_layer_t** layer_out) {
+    const GptqArgs ga = {calib_x, calib_tokens, damp, block};
+    return prepare_int4(asym != 0, false, W, w_dtype, w_layout, Q, q_dtype, bias, nullptr, nullptr, K, N, r, group, blob,
+                        blob_bytes, scratch, scratch_bytes, stream, layer_out, &ga);
 }
 
 dirotq_status_t dirotq_prepare_layer(const void* W, int w_dtype, int w_layout, const void* Q, int q_dtype,

@@ -348,6 +348,10 @@ dirotq_status_t launch_workspace_export_nvfp4(const dirotq_layer* L, int M, cons
 dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Q,
                                int q_dtype, const void* bias, const int8_t* wcodes, const void* wscales, double* scratch,
                                cudaStream_t stream);
+dirotq_status_t launch_pack_codes(const dirotq_layer* L, const int8_t* wcodes, const uint16_t* wscales, cudaStream_t stream);
+size_t gptq_scratch_bytes(int K, int N, int r, int T);
+dirotq_status_t launch_gptq_round(const dirotq_layer* L, const void* calib_bf16, int T, double damp, int block, char* scratch,
+                                  cudaStream_t stream, const int8_t** codes_out, const uint16_t** scales_out);
 dirotq_status_t launch_layer_export(const dirotq_layer* L, int8_t* wcodes, uint16_t* wscales, uint16_t* wh,
                                     uint16_t* qb, cudaStream_t stream);
 dirotq_status_t launch_workspace_export(const dirotq_layer* L, int M, const char* workspace, uint16_t* xh,

@@ -566,6 +566,18 @@ dirotq_status_t launch_prepare(const dirotq_layer* L, const void* W, int w_dtype
     return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
+// Replaces the residual codes and scales of a prepared grouped-INT4 layer (codes int8 [K_l][N], bf16 scales [n_g][N], device).
+dirotq_status_t launch_pack_codes(const dirotq_layer* L, const int8_t* wcodes, const uint16_t* wscales, cudaStream_t stream) {
+    const Geometry& g = L->geo;
+    char* blob = L->blob;
+    if (cudaMemsetAsync(blob + L->lay.off_wpacked, 0, static_cast<size_t>(g.N) * (g.K_lp / 2), stream) != cudaSuccess)
+        return DIROTQ_ERR_CUDA;
+    pack_codes_kernel<<<dim3((g.N + 127) / 128, g.n_g), 128, 0, stream>>>(
+        wcodes, wscales, reinterpret_cast<uint8_t*>(blob + L->lay.off_wpacked), reinterpret_cast<float*>(blob + L->lay.off_wscale),
+        reinterpret_cast<uint16_t*>(blob + L->lay.off_wh), g);
+    return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------ projection form (fmt 4)
 
 namespace {

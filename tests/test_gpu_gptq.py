@@ -1,6 +1,7 @@
-"""Layers whose residual weights were rounded with GPTQ (Sec. 4.1, App. F.1) by the CPU oracle and handed to the
-library as codes: the deployed layer must carry exactly those codes, and the online path must agree with the
-oracle's deployed layer element by element."""
+"""Layers whose residual weights are rounded with GPTQ (Sec. 4.1, App. F.1).  The library rounds them itself
+(dirotq_prepare_layer_gptq): its codes and scales must equal the CPU oracle's GPTQ, and the online path must agree with
+the oracle's deployed layer element by element.  Codes rounded elsewhere can be deployed too (dirotq_prepare_layer_codes):
+such a layer must carry exactly the codes it was given."""
 import numpy as np
 import pytest
 import torch
@@ -15,7 +16,7 @@ from parity_utils import (bf16_tensor_to_bits, bits_to_bf16_tensor, check_activa
 pytestmark = pytest.mark.gpu
 
 
-def _run_case(spec: synth.LayerSpec, M: int, asym: bool, calib: int = 512):
+def _run_case(spec: synth.LayerSpec, M: int, asym: bool, calib: int = 512, own_rounding: bool = True):
     inp = synth.make_layer_inputs(spec, M, with_bias=True)
     calib_bits = synth.make_tokens(spec, calib, batch_seed=99)
     lo = orc.prepare_layer_gptq(inp["W"], inp["Q"], calib_bits, spec.r, spec.G)
@@ -26,8 +27,13 @@ def _run_case(spec: synth.LayerSpec, M: int, asym: bool, calib: int = 512):
     W = torch.from_numpy(inp["W"]).to(dev)
     Q = torch.from_numpy(inp["Q"]).to(dev)
     bias = bits_to_bf16_tensor(inp["bias"])
-    layer = dq.dirotq_prepare_layer_codes(W, Q, torch.from_numpy(lo["wcodes"]).to(dev),
-                                          bits_to_bf16_tensor(lo["wscales"]), spec.r, spec.G, bias=bias, asym=asym)
+    if own_rounding:
+        # the library's own GPTQ: same steps in fp64 on the device; equal codes and scales unless a quotient of the
+        # error-feedback chain falls within rounding error of a tie (then the two chains part and this check fails)
+        layer = dq.dirotq_prepare_layer_gptq(W, Q, bits_to_bf16_tensor(calib_bits), spec.r, spec.G, bias=bias, asym=asym)
+    else:
+        layer = dq.dirotq_prepare_layer_codes(W, Q, torch.from_numpy(lo["wcodes"]).to(dev),
+                                              bits_to_bf16_tensor(lo["wscales"]), spec.r, spec.G, bias=bias, asym=asym)
     check_weight_side(dq.dirotq_layer_export(layer), lo)            # exact: lo carries no tie information
     if asym:
         csum = np.stack([lo["wcodes"][g * spec.G:(g + 1) * spec.G].astype(np.int64).sum(axis=0)
@@ -88,6 +94,28 @@ def test_gptq_codes_symmetric_activations():
 def test_gptq_codes_asymmetric_activations_group128_ragged():
     spec = synth.LayerSpec(K=640, N=400, r=16, G=128, model=synth.FLUX, seed=22, calib_tokens=1024)
     print(_run_case(spec, M=150, asym=True))
+
+
+def test_gptq_rounding_at_pixart_width():
+    spec = synth.LayerSpec(K=1152, N=384, r=32, G=64, model=synth.PIXART, seed=23, calib_tokens=2048)
+    print(_run_case(spec, M=160, asym=False, calib=1024))
+
+
+def test_codes_rounded_elsewhere_are_deployed_as_given():
+    spec = synth.LayerSpec(K=512, N=256, r=32, G=64, model=synth.PIXART, seed=21, calib_tokens=1024)
+    print(_run_case(spec, M=200, asym=False, own_rounding=False))
+
+
+def test_prepare_layer_gptq_rejects_bad_arguments():
+    spec = synth.LayerSpec(K=256, N=256, r=32, G=64, model=synth.PIXART, seed=1, calib_tokens=512)
+    inp = synth.make_layer_inputs(spec, 8, with_bias=False)
+    W, Q = torch.from_numpy(inp["W"]).cuda(), torch.from_numpy(inp["Q"]).cuda()
+    calib = bits_to_bf16_tensor(synth.make_tokens(spec, 64, batch_seed=3))
+    with pytest.raises(dq.DirotqError):
+        dq.dirotq_prepare_layer_gptq(W, Q, calib, spec.r, spec.G, block=96)    # not a multiple of the group
+    with pytest.raises(dq.DirotqError):
+        dq.dirotq_prepare_layer_gptq(W, Q, calib, spec.r, spec.G, damp=0.0)
+    torch.cuda.synchronize()
 
 
 def test_prepare_layer_codes_rejects_missing_codes():
