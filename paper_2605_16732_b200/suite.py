@@ -178,6 +178,64 @@ class Case:
         self.layer.close()
 
 
+def small_m_summary(M=256, K=1152, N=1152, r=32, G=64, hbm_gbs=None):
+    """The memory-bound small layer (PixArt attention projection at M = 256): device time per layer replayed from a CUDA
+    graph, the bytes the method must move (activations, rotation, weight codes and scales, intermediates, output) and
+    the bandwidth that amounts to."""
+    c = Case(M, K, N, r, G, synth.PIXART)
+    K_l = K - r
+    n_g = -(-K_l // G)
+    bytes_alg = 2 * M * K + 2 * K * K + n_g * G * N / 2 + 4 * n_g * N + 2 * 64 * N + 2 * (M * n_g * G + 4 * M * n_g + 2 * M * 64) + 2 * M * N
+    us = c.graph_ms(c.run) * 1e3
+    us_cublas = c.graph_ms(lambda: torch.matmul(c.x, c.Wb)) * 1e3
+    assert dq.dirotq_workspace_status(c.ws) == 0
+    c.close()
+    gbs = bytes_alg / (us * 1e-6) / 1e9
+    return {"workload": f"pixart_attention_projection_M{M}_K{K}_N{N}_r{r}_g{G}", "linear_graph_us": us, "cublas_bf16_graph_us": us_cublas,
+            "algorithmic_bytes": bytes_alg, "algorithmic_gbs": gbs, "frac_hbm_peak": gbs / hbm_gbs if hbm_gbs else None}
+
+
+def pixart_block_summary(M=4096, iters=10):
+    """Config 2: the PixArt-shaped block linears at M = 4096, per shape: both kernels' device times and cuBLAS bf16."""
+    out = {}
+    for K, N in [(1152, 1152), (1152, 4608), (4608, 1152)]:
+        c = Case(M, K, N, 32, 64, synth.PIXART)
+        rot, gem, cb = c.time_kernels(iters)
+        out[f"{K}x{N}"] = {"rotate_ms": rot, "gemm_ms": gem, "cublas_bf16_ms": cb, "effective_tops": 2.0 * M * N * K / ((rot + gem) * 1e-3) / 1e12}
+        c.close()
+    return out
+
+
+def flux_step_summary(run_by_name, cublas_by_name, status_check, M=4608, reps=3):
+    """Config 5: the 152 linears of one FLUX.1-dev-shaped denoising step in sequence (19 double-stream blocks of four
+    linears, 38 single-stream blocks of two), device-timed, against the same chain of cuBLAS bf16 GEMMs.  `run_by_name`
+    and `cublas_by_name` map a shape name to a callable that enqueues that layer once."""
+    shapes = {"qkv": (3072, 9216), "out": (3072, 3072), "mlp_up": (3072, 12288), "mlp_down": (12288, 3072),
+              "single_in": (3072, 21504), "single_out": (15360, 3072)}
+    chain = ["qkv", "out", "mlp_up", "mlp_down"] * 19 + ["single_in", "single_out"] * 38
+    res = {}
+    for name, table in (("dirotq", run_by_name), ("cublas_bf16", cublas_by_name)):
+        def fn():
+            for n in chain:
+                table[n]()
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        res[name] = float(np.median(ts))
+    status_check()
+    ops = sum(2.0 * M * shapes[n][0] * shapes[n][1] for n in chain)
+    return {"linears": len(chain), "dirotq_chain_ms": res["dirotq"], "cublas_bf16_chain_ms": res["cublas_bf16"],
+            "effective_tops": ops / (res["dirotq"] * 1e-3) / 1e12, "speedup_vs_cublas_bf16": res["cublas_bf16"] / res["dirotq"],
+            "note": "one prepared layer per distinct shape is reused for every block of that shape"}
+
+
 def memory_report():
     """Bytes of a prepared layer (`dirotq_layer_bytes*`, no GPU needed) against its bf16 weights, for the layer shapes of
     the configurations, at the benchmark's rank and at about a tenth of K."""
