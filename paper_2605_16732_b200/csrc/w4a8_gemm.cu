@@ -12,8 +12,9 @@
 //
 // Roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2..5 unpack,
 // warps 6..13 epilogue (one token row per thread, two warps per lane quadrant).  TMEM: columns 0..255 the int32 tile, 256..511 the
-// fp32 tile of the bf16 rank-r branch (kind::f16 cannot accumulate into the integer tile); single
-// buffered, so the epilogue of a tile (one pass) is not overlapped with the next tile's MMAs.
+// fp32 tile of the bf16 rank-r branch (kind::f16 cannot accumulate into the integer tile); with 256-column tiles that
+// pair fills tensor memory and a tile's epilogue (one pass) is not overlapped with the next tile's MMAs; with 128-column
+// tiles two pairs alternate and it is.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -43,7 +44,8 @@ struct Plan {
     static constexpr int SCALE_OFFSET = BAR_OFFSET + 256;  // two buffers of {weight scales, bias} for a tile's columns
     static constexpr int SCALE_BYTES = 2 * 2 * BN * 4;
     static constexpr int SMEM_BYTES = SCALE_OFFSET + SCALE_BYTES + 1024;
-    static_assert(8 * (3 * STAGES + 2) <= 192, "barriers must end below the two words at +192");
+    static constexpr int NACC = 512 / (2 * BN);  // {int32 tile, fp32 tile} pairs in tensor memory: 1 (wide) or 2 (narrow tiles)
+    static_assert(8 * (3 * STAGES + 4) <= 192, "barriers must end below the two words at +192");
     static_assert(SMEM_BYTES <= 232448 && STAGE_BYTES % 1024 == 0, "shared memory plan");
 };
 
@@ -86,8 +88,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto unp_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto empty_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
-    const uint32_t tfull_bar = bar_base + 8u * (3 * STAGES);
-    const uint32_t tempty_bar = bar_base + 8u * (3 * STAGES + 1);
+    constexpr int NACC = P::NACC;
+    auto tfull_bar = [&](uint32_t a) { return bar_base + 8u * (3 * STAGES + a); };
+    auto tempty_bar = [&](uint32_t a) { return bar_base + 8u * (3 * STAGES + 2 + a); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 192);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 196);
 
@@ -103,8 +106,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             mbar_init(unp_bar(s), NUM_UNPACK_WARPS * 32);
             mbar_init(empty_bar(s), 1);
         }
-        mbar_init(tfull_bar, 1);
-        mbar_init(tempty_bar, NUM_EPI_WARPS * 32);
+        for (int a = 0; a < NACC; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
+        }
         mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
         fence_mbar_init();
@@ -166,7 +171,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-                if (!mbar_wait(tempty_bar, (tcount & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                // with narrow tiles two accumulator pairs alternate: a tile's epilogue runs under the next tile's MMAs
+                const uint32_t acc = tcount % NACC, tacc = tmem_base + acc * 2 * BN;
+                if (!mbar_wait(tempty_bar(acc), ((tcount / NACC) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                 tc_fence_after_sync();
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
@@ -179,15 +186,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
                     if (i < p.num_kb) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_i8(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
+                        for (int k = 0; k < 4; ++k) umma_i8(tacc, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
                     } else {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem_base + BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, ((i - p.num_kb) | k) != 0);
+                            umma_bf16(tacc + BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, ((i - p.num_kb) | k) != 0);
                     }
                     umma_commit(empty_bar(s));
                 }
-                if (ok) umma_commit(tfull_bar);
+                if (ok) umma_commit(tfull_bar(acc));
             }
         }
     } else if (warp < 2 + NUM_UNPACK_WARPS) {
@@ -273,7 +280,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     *reinterpret_cast<float2*>(s_b + 2 * e) = b2;
                 }
             }
-            const bool mine = mbar_wait(tfull_bar, tcount & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+            const uint32_t acc_i = tcount % NACC;
+            const bool mine = mbar_wait(tfull_bar(acc_i), (tcount / NACC) & 1, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
             uint32_t any_failed;
             asm volatile(
                 "{\n\t"
@@ -290,7 +298,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             tc_fence_after_sync();
             const int row = m0 + q * 32 + lane;
             const float sx = row < p.M ? __ldg(p.xscale + row) : 0.f;
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc_i * 2 * BN;
 #pragma unroll 1
             for (int c = half * CPH; c < (half + 1) * CPH; ++c) {
                 uint32_t acc[32], lr[32];
@@ -301,7 +309,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 tmem_ld_fence32(lr);
                 if (c == (half + 1) * CPH - 1) {
                     tc_fence_before_sync();
-                    mbar_arrive(tempty_bar);
+                    mbar_arrive(tempty_bar(acc_i));
                 }
                 const int col = n0 + c * 32;
                 if (row < p.M) {
