@@ -173,7 +173,9 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 /* Tuning knob of the second kernels (all four formats): output columns per tile.
  * 0 (default): chosen per call from M, N and the number of SMs (INT4: 256 columns unless 128-column tiles fill the
  * SMs so much better that they win although a narrow tile costs about 0.73 of a wide one; NVFP4 likewise with 0.6);
- * 128 or 256: forced.  Process-wide; results do not depend on it (each output element is accumulated in the same
+ * 128 or 256: forced; 192: the grouped INT4 kernel's plan with three epilogue warpgroups (64 columns per thread; the
+ * other formats' kernels then choose for themselves), never chosen automatically: on the FLUX shapes it measured
+ * between the other two.  Process-wide; results do not depend on it (each output element is accumulated in the same
  * order).  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
 

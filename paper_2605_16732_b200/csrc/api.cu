@@ -151,6 +151,22 @@ dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_
     return DIROTQ_OK;
 }
 
+// Weight-side tensor maps with 192-row boxes (the 192-column tile plan of the grouped INT4 second kernel).
+static dirotq_status_t encode_tmaps_192(dirotq_layer* L, int N, int group) {
+    const Geometry& g = L->geo;
+    const BlobLayout& lay = L->lay;
+    dirotq_status_t st = encode_tmap_2d(&L->tmap_wpacked192, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                                        (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, 192, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wscale192, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale,
+                            (uint64_t)wscale_row_len(N), (uint64_t)g.n_g, (uint64_t)wscale_row_len(N) * 4, 192, 128 / group,
+                            CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_wh192, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 192, CU_TENSOR_MAP_SWIZZLE_128B);
+    return st;
+}
+
 struct GptqArgs {
     const void* calib;  // bf16 [T][K] calibration tokens (device); NULL: round to nearest
     int T;
@@ -225,6 +241,7 @@ static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int 
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK) st = encode_tmaps_192(L, N, group);
     if (st == DIROTQ_OK)
         st = launch_prepare(L, W, w_dtype, w_layout, Q, q_dtype, bias, wcodes, wscales, static_cast<double*>(scratch),
                             static_cast<cudaStream_t>(stream));
@@ -395,6 +412,7 @@ dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wh128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
                             (uint64_t)N, (uint64_t)g.r_pad * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK) st = encode_tmaps_192(L, N, group);
     if (st == DIROTQ_OK)
         st = launch_prepare_ph(L, W, w_dtype, w_layout, Uh, uh_dtype, bias, static_cast<double*>(scratch),
                                static_cast<cudaStream_t>(stream));
@@ -602,8 +620,9 @@ dirotq_status_t dirotq_set_dependent_launch(int enabled) {
 
 dirotq_status_t dirotq_set_gemm_tile(int columns) {
     dirotq_status_t st = set_w4a4_tile_columns(columns);
-    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(columns);
-    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(columns);
+    const int others = columns == 192 ? 0 : columns;  // the 192-column plan exists for the grouped INT4 second kernel only
+    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(others);
+    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(others);
 }
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,

@@ -227,6 +227,7 @@ struct dirotq_layer {
     CUtensorMap tmap_wscale;   // f32 [n_g][N32], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
     CUtensorMap tmap_wpacked128, tmap_wscale128, tmap_wh128;  // the same three with 128-row boxes (narrow W4A4 tiles)
+    CUtensorMap tmap_wpacked192, tmap_wscale192, tmap_wh192;  // ... and with 192-row boxes (grouped INT4 formats)
     int act_scale_log2;        // NVFP4 variant: exponent of the activations' per-tensor power-of-two scale
 };
 

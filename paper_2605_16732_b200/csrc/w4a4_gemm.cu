@@ -45,22 +45,24 @@ namespace {
 constexpr int BM = 128;
 constexpr int BKC = 128;  // one-byte codes per k-block (128-byte rows)
 constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_h chunk
-constexpr int SC_SLOTS = 8;
-constexpr int NUM_THREADS = 384;
-constexpr int NUM_EPI_WARPS = 8;
 constexpr uint32_t kSignMag = 0x87878787u;  // sign and 3-bit magnitude of four one-byte codes
-#ifndef W4A4_EPI_REGS
-#define W4A4_EPI_REGS 216
-#endif
-#ifndef W4A4_AUX_REGS
-#define W4A4_AUX_REGS 64
-#endif
 
-// Shared-memory plan for tiles of BN output columns.  256 columns is the default; 128-column tiles (with more
-// pipeline stages) are used when the wide ones would leave most SMs idle in the last wave, see the launcher.
+// Plan for tiles of BN output columns.
+//   256: two epilogue warpgroups, 128 columns (128 fp32 accumulators) per thread; an accumulator tile can only be read in
+//        pieces between the arithmetic and is held for three quarters of a group.
+//   192: three epilogue warpgroups, 64 columns per thread: a thread's share of an accumulator tile fits its two chunk
+//        buffers, so the tile goes back to the tensor core after the first quarter of a group, and three warps per scheduler
+//        hide each other's waits.  16 warps: 152 registers for the epilogue threads, 56 for the others.
+//   128: two warpgroups, 64 columns per thread, four accumulator tiles; for layers whose wider tiles would leave SMs idle.
 template <int BN>
 struct Plan {
-    static constexpr int STAGES = BN == 256 ? 3 : 5;
+    static constexpr int EPI_WG = BN == 192 ? 3 : 2;          // epilogue warpgroups
+    static constexpr int EPI_WARPS = 4 * EPI_WG;
+    static constexpr int THREADS = 128 + 128 * EPI_WG;
+    static constexpr int EPI_REGS = EPI_WG == 3 ? 152 : 216;  // setmaxnreg budgets: 128 * AUX + 128 * EPI_WG * EPI <= 65536
+    static constexpr int AUX_REGS = EPI_WG == 3 ? 56 : 64;
+    static constexpr int SC_SLOTS = BN == 192 ? 6 : 8;
+    static constexpr int STAGES = BN == 256 ? 3 : BN == 192 ? 4 : 5;
     static constexpr int BU_BYTES = BN * BKC;         // unpacked weight codes / bf16 W~_h chunk (32 KB at BN = 256)
     static constexpr int BP_BYTES = BN * BKC / 2;     // packed weight codes (TMA staging)
     static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB / 40 KB
@@ -70,8 +72,10 @@ struct Plan {
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
     static constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024;
 };
-static_assert(Plan<256>::SMEM_BYTES <= 232448 && Plan<128>::SMEM_BYTES <= 232448, "shared memory plan too large");
+static_assert(Plan<256>::SMEM_BYTES <= 232448 && Plan<192>::SMEM_BYTES <= 232448 && Plan<128>::SMEM_BYTES <= 232448, "shared memory plan too large");
 static_assert(Plan<128>::STAGE_BYTES % 1024 == 0 && Plan<128>::SC_BYTES % 128 == 0, "tile alignment");
+static_assert(Plan<192>::STAGE_BYTES % 1024 == 0 && Plan<192>::SC_BYTES % 128 == 0, "tile alignment");
+static_assert(8 * (3 * Plan<128>::STAGES + 2 * 8 + 9) <= 400 && 8 * (3 * Plan<192>::STAGES + 2 * 6 + 9) <= 400, "barriers end below the words at +400");
 
 struct GemmKernelParams {
     int M, N, n_g, num_kb, lr_chunks;
@@ -124,7 +128,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 template <int G, bool kPartials, int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(Plan<BN>::THREADS, 1)
 w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
                  const __grid_constant__ CUtensorMap tmap_wscale, const __grid_constant__ CUtensorMap tmap_xscale,
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
@@ -132,7 +136,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     using P = Plan<BN>;
     constexpr int STAGES = P::STAGES, STAGE_BYTES = P::STAGE_BYTES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES;
     constexpr int SC_SW_BYTES = P::SC_SW_BYTES, SC_BYTES = P::SC_BYTES, BAR_OFFSET = P::BAR_OFFSET;
-    constexpr int HB = BN / 2;         // columns per epilogue warp: the warpgroup selects the half of the tile
+    constexpr int SC_SLOTS = P::SC_SLOTS, NUM_EPI_WARPS = P::EPI_WARPS;
+    constexpr int HB = BN / P::EPI_WG;  // columns per epilogue warp: the warpgroup selects the slice of the tile
     constexpr int CHUNKS = HB / 32;    // 32-column chunks per epilogue warp and accumulator tile
     constexpr int GPK = BKC / G;       // groups per k-block: 2 (G = 64) or 1 (G = 128)
     constexpr int MMA_PER_G = G / 32;  // 8-bit MMA instructions (K = 32) per group
@@ -199,7 +204,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     grid_launch_dependents();
 
     if (warp < 4) {
-        reg_dealloc<W4A4_AUX_REGS>();
+        reg_dealloc<P::AUX_REGS>();
 
         if (warp == 0) {
             // -------------------------------------------------------- TMA producer
@@ -341,12 +346,14 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         // staging buffer and the operand tile do not overlap, so a load written after a store would wait
                         // for it and the whole unpack would run as one dependent chain.
 #pragma unroll
-                        for (int jb = 0; jb < (BN * 4) / 64; jb += 8) {
-                            uint4 pk[8];
+                        constexpr int PIECES = (BN * 4) / 64, BATCH = PIECES % 8 == 0 ? 8 : 4;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) pk[j] = src[64 * (jb + j)];
+                        for (int jb = 0; jb < PIECES; jb += BATCH) {
+                            uint4 pk[BATCH];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
+                            for (int j = 0; j < BATCH; ++j) pk[j] = src[64 * (jb + j)];
+#pragma unroll
+                            for (int j = 0; j < BATCH; ++j) {
                                 // a word holds codes k..k+3 in bits 7, 2..0 of its bytes and codes k+4..k+7 four bit
                                 // positions further up, wrapping around (see prepare.cu): mask, rotate, mask
                                 uint4 o0, o1;
@@ -368,7 +375,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             if (u == 0) flush_wait(p.status, WS_UNPACK_FULL, w_full);
         }
     } else {
-        reg_alloc<W4A4_EPI_REGS>();
+        reg_alloc<P::EPI_REGS>();
         // ------------------------------------------------------------ epilogue (warps 4..11)
         // A warp owns 32 token rows (its TMEM lane quadrant) x BN/2 columns.  The accumulators are read with the
         // 16x256b shape: a thread then holds 4 rows (l/4 + 8 i) x the column pairs 2 (l%4) + {0, 1} of every block
@@ -633,26 +640,27 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
     static SmemOptIn<4> opt_in;  // one per instantiation of this launcher, i.e. per tile width
     const int vi = (g.G == 64 ? 0 : 2) + (dbg ? 1 : 0);
     if (!opt_in.ensure(kern, vi, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
-    const bool narrow = BN == 128;
-    const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
-                                          narrow ? L->tmap_wpacked128 : L->tmap_wpacked,
-                                          narrow ? L->tmap_wscale128 : L->tmap_wscale, tmap_xscale, tmap_xh,
-                                          narrow ? L->tmap_wh128 : L->tmap_wh, p);
+    const cudaError_t err = launch_kernel(kern, grid, Plan<BN>::THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
+                                          BN == 128 ? L->tmap_wpacked128 : BN == 192 ? L->tmap_wpacked192 : L->tmap_wpacked,
+                                          BN == 128 ? L->tmap_wscale128 : BN == 192 ? L->tmap_wscale192 : L->tmap_wscale,
+                                          tmap_xscale, tmap_xh,
+                                          BN == 128 ? L->tmap_wh128 : BN == 192 ? L->tmap_wh192 : L->tmap_wh, p);
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 }  // namespace
 
-static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 128 / 256: forced
+static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 128 / 192 / 256: forced
 
 dirotq_status_t set_w4a4_tile_columns(int columns) {
-    if (columns != 0 && columns != 128 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+    if (columns != 0 && columns != 128 && columns != 192 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
     g_tile_columns.store(columns);
     return DIROTQ_OK;
 }
 
 dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
     const int forced = g_tile_columns.load();
+    if (forced == 192) return launch_w4a4_gemm_bn<192>(L, a, stream);
     const bool narrow = forced ? forced == 128 : narrow_tiles_pay(a.M, L->geo.N, sm_count(L->device));
     return narrow ? launch_w4a4_gemm_bn<128>(L, a, stream) : launch_w4a4_gemm_bn<256>(L, a, stream);
 }

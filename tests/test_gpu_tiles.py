@@ -1,4 +1,4 @@
-"""The INT4 second kernel with 128- and 256-column tiles: both forced through dirotq_set_gemm_tile, on shapes the
+"""The INT4 second kernel with 128-, 192- (three epilogue warpgroups) and 256-column tiles: both forced through dirotq_set_gemm_tile, on shapes the
 automatic choice would send one way only.  Parity with the oracle under each setting, and bit-equal outputs and
 integer group sums between the two (every output element is accumulated in the same order)."""
 import numpy as np
@@ -22,20 +22,20 @@ def tile(request):
     dq.dirotq_set_gemm_tile(0)
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
 def test_parity_group64_ragged_everything(tile):
     # N = 400: ragged in both tile widths; M = 300: ragged rows; K_l = 496: ragged last group
     spec = synth.LayerSpec(K=512, N=400, r=16, G=64, model=synth.FLUX, seed=31, calib_tokens=1024)
     print(tile, test_gpu_parity._run_case(spec, M=300))
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
 def test_parity_group128_rank128(tile):
     spec = synth.LayerSpec(K=768, N=640, r=128, G=128, model=synth.FLUX, seed=32, calib_tokens=1024)
     print(tile, test_gpu_parity._run_case(spec, M=257, with_bias=False))
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
 def test_parity_pixart_projection_many_tiles(tile):
     # 8 row blocks x 9 (or 5) column blocks: several tiles per CTA are not reached on one GPU with 148 SMs, but the
     # tile -> (row block, column block) mapping and the ring phases across k-blocks are
@@ -43,7 +43,7 @@ def test_parity_pixart_projection_many_tiles(tile):
     print(tile, test_gpu_parity._run_case(spec, M=1024, check_rot=False))
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
 def test_parity_asymmetric_codes(tile):
     spec = synth.LayerSpec(K=640, N=400, r=32, G=64, model=synth.PIXART, seed=34, calib_tokens=1024)
     print(tile, test_gpu_asym._run_case(spec, M=200, shift=1.5))
@@ -60,7 +60,7 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
     ws = dq.alloc_workspace(layer, M)
     outs = {}
     try:
-        for cols in (0, 128, 256):
+        for cols in (0, 128, 192, 256):
             dq.dirotq_set_gemm_tile(cols)
             y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
             dq.dirotq_linear(x, layer, y, ws)
@@ -68,7 +68,7 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
             assert dq.dirotq_workspace_status(ws) == 0
             outs[cols] = y.view(torch.int16).clone()
         # several tiles per CTA here (33 row blocks x 9 column blocks on 148 SMs)
-        assert torch.equal(outs[128], outs[256]) and torch.equal(outs[0], outs[128])
+        assert torch.equal(outs[128], outs[256]) and torch.equal(outs[192], outs[256]) and torch.equal(outs[0], outs[128])
         with pytest.raises(dq.DirotqError):
             dq.dirotq_set_gemm_tile(64)
     finally:
