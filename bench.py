@@ -169,9 +169,11 @@ def run_reference(args):
     if rank != 0:
         return
     steps = max(1, args.steps)
+    # the sample shrinks with the number of steps so that the whole run stays within a few minutes of CPU time
+    rows, cols = (128, 512) if steps <= 5 else (64, 256) if steps <= 30 else (32, 128)
     for _ in range(min(args.warmup, 1)):
-        oracle_sample_run(1, fmt=args.fmt)
-    res = oracle_sample_run(steps, fmt=args.fmt)
+        oracle_sample_run(1, rows=rows, cols=cols, fmt=args.fmt)
+    res = oracle_sample_run(steps, rows=rows, cols=cols, fmt=args.fmt)
     line = {
         "impl": "reference", "metric": "dirotq_w4a4_linear_effective_tops", "value": res["value"], "unit": "TOPS",
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step"] * 1e3,
@@ -486,7 +488,8 @@ def run_ours(args):
                 c.close()
             del wbs
 
-    cpu = oracle_sample_run(1, fmt=args.fmt) if not args.lite else {"value": None, "unit": "TOPS", "cores": None, "kind": "oracle",
+    # about 10 s of CPU work: 128 token rows x 512 output columns of each of the four linears
+    cpu = oracle_sample_run(1, rows=128, cols=512, fmt=args.fmt) if not args.lite else {"value": None, "unit": "TOPS", "cores": None, "kind": "oracle",
                                                       "sample": "skipped (--lite)"}
     line = {
         "metric": "dirotq_w4a4_linear_effective_tops", "value": value, "unit": "TOPS", "n_gpus": world,
