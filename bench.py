@@ -196,7 +196,6 @@ def run_reference(args):
 def run_ours(args):
     import torch
     from paper_2605_16732_b200 import binding as dq
-    from paper_2605_16732_b200.suite import residual_exponent
     from paper_2605_16732_b200 import synth
     from paper_2605_16732_b200.shard import aggregate_throughput, max_over_ranks
 
@@ -230,11 +229,10 @@ def run_ours(args):
             probe = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, 0, bias=bf(bias))
             xrot = torch.empty((1024, K), dtype=torch.float32, device=dev)
             dq.dirotq_rotate_quantize(x[:1024], probe, dq.alloc_workspace(probe, 1024), xrot)
-            amax = float(xrot[:, RANK:].abs().max().item())
+            ex = dq.dirotq_act_scale_log2_from_rotated(xrot, RANK)
             probe.close()
             del xrot
-            layer = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, int(np.ceil(np.log2(amax / 1536.0))),
-                                                  bias=bf(bias))
+            layer = dq.dirotq_prepare_layer_nvfp4(torch.from_numpy(W).to(dev), Q, RANK, ex, bias=bf(bias))
         elif args.fmt == "w4a8":
             layer = dq.dirotq_prepare_layer_w4a8(torch.from_numpy(W).to(dev), Q, RANK, bias=bf(bias))
         elif args.fmt == "int4_asym":
@@ -243,7 +241,7 @@ def run_ours(args):
             layer = dq.dirotq_prepare_layer_ph(torch.from_numpy(W).to(dev), Q[:, :RANK].contiguous(), GROUP, bias=bf(bias))
         elif args.fmt == "nvfp4_ph":
             Uh = Q[:, :RANK].contiguous()
-            layer = dq.dirotq_prepare_layer_nvfp4_ph(torch.from_numpy(W).to(dev), Uh, residual_exponent(x, Uh), bias=bf(bias))
+            layer = dq.dirotq_prepare_layer_nvfp4_ph(torch.from_numpy(W).to(dev), Uh, dq.dirotq_act_scale_log2_ph(x[:1024].contiguous(), Uh), bias=bf(bias))
         else:
             layer = dq.dirotq_prepare_layer(torch.from_numpy(W).to(dev), Q, RANK, GROUP, bias=bf(bias))
         del Q

@@ -398,6 +398,21 @@ DIROTQ_API dirotq_status_t dirotq_linear_noalloc(const void* x, int M, const dir
 DIROTQ_API dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* status_word, float* tera_ops_per_s,
                                                  dirotq_stream_t stream);
 
+/* ---- calibration of the NVFP4 activations' power-of-two scale (paper Sec. 5.1 / App. E: FP8 block scales need a
+ * second-level scale; here 2^e with e = ceil(log2(max|X| / (6 * 256))), an argument of the NVFP4 layers' preparation) ----
+ *
+ * Both calls find the largest low-precision coefficient of a batch of calibration tokens on the device, SYNCHRONISE
+ * `stream` and return e in *act_scale_log2 (HOST).  device_word: 4 bytes of DEVICE scratch.
+ * dirotq_act_scale_log2_from_rotated: from fp32 rotated activations [M,K] in the column order of Q (what
+ * dirotq_rotate_quantize exports; the first r columns are the 16-bit ones and are skipped).
+ * dirotq_act_scale_log2_ph: projection form, from the tokens x (bf16 [M,K]) and U_h ([K,r] row-major, f64 or f32)
+ * alone: x~_h = bf16(x U_hb), d = x - x~_h U_hb^T, Hadamard blocks of 64, largest |coefficient| (fp32 arithmetic: the
+ * exponent only needs the maximum to within a few per cent).  K + r <= 51200. */
+DIROTQ_API dirotq_status_t dirotq_act_scale_log2_from_rotated(const float* xrot_f32, int M, int K, int r, void* device_word,
+                                                              int* act_scale_log2, dirotq_stream_t stream);
+DIROTQ_API dirotq_status_t dirotq_act_scale_log2_ph(const void* x, int M, const void* Uh, int uh_dtype, int K, int r,
+                                                    void* device_word, int* act_scale_log2, dirotq_stream_t stream);
+
 /* ---- failure-path check (no counterpart in the paper) ---------------------------------------- */
 
 /* Every wait on a barrier inside the library's kernels is bounded: when its time runs out the

@@ -26,7 +26,7 @@ EXPORTED = [
     "dirotq_prepare_scratch_bytes", "dirotq_workspace_bytes", "dirotq_prepare_layer", "dirotq_layer_destroy",
     "dirotq_layer_info", "dirotq_linear", "dirotq_linear_host", "dirotq_workspace_status",
     "dirotq_rotate_quantize", "dirotq_w4a4_gemm", "dirotq_workspace_wait_counters", "dirotq_workspace_export", "dirotq_int_gemm_debug", "dirotq_layer_export",
-    "dirotq_mma_rate_probe", "dirotq_linear_noalloc", "dirotq_wait_selftest",
+    "dirotq_mma_rate_probe", "dirotq_linear_noalloc", "dirotq_wait_selftest", "dirotq_act_scale_log2_from_rotated", "dirotq_act_scale_log2_ph",
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
     "dirotq_prepare_layer_codes", "dirotq_prepare_scratch_bytes_gptq", "dirotq_prepare_layer_gptq", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.dirotq_linear_noalloc.argtypes = [vp, i, vp, vp, vp, vp]
         L.dirotq_mma_rate_probe.argtypes = [i, i, vp, ctypes.POINTER(ctypes.c_float), vp]
         L.dirotq_wait_selftest.argtypes = [vp, ctypes.c_uint, vp]
+        L.dirotq_act_scale_log2_from_rotated.argtypes = [vp, i, i, i, vp, pi, vp]
+        L.dirotq_act_scale_log2_ph.argtypes = [vp, i, vp, i, i, i, vp, pi, vp]
         L.dirotq_layer_bytes_nvfp4.argtypes = [i, i, i, psz]
         L.dirotq_prepare_layer_nvfp4.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_workspace_export_nvfp4.argtypes = [vp, i, vp, vp, vp, vp, vp]
@@ -281,6 +283,27 @@ def dirotq_mma_rate_probe(kind: int, iters: int = 20000, stream=None) -> float:
     if int(status[0].item()) != 0:
         raise DirotqError(6, "dirotq_mma_rate_probe")
     return float(out.value)
+
+
+def dirotq_act_scale_log2_from_rotated(xrot: torch.Tensor, r: int, stream=None) -> int:
+    """Exponent of the NVFP4 activations' power-of-two scale from fp32 rotated calibration activations [M, K]."""
+    assert xrot.is_cuda and xrot.is_contiguous() and xrot.dtype == torch.float32
+    word = torch.zeros(1, dtype=torch.int32, device=xrot.device)
+    out = ctypes.c_int(0)
+    _check(lib().dirotq_act_scale_log2_from_rotated(xrot.data_ptr(), xrot.shape[0], xrot.shape[1], int(r), word.data_ptr(),
+                                                    ctypes.byref(out), _stream(stream)), "dirotq_act_scale_log2_from_rotated")
+    return out.value
+
+
+def dirotq_act_scale_log2_ph(x: torch.Tensor, Uh: torch.Tensor, stream=None) -> int:
+    """Projection form: the same exponent from calibration tokens x (bf16 [M, K]) and U_h ([K, r], f64 or f32)."""
+    assert x.is_cuda and x.is_contiguous() and x.dtype == torch.bfloat16 and Uh.is_cuda and Uh.is_contiguous()
+    uh_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Uh.dtype]
+    word = torch.zeros(1, dtype=torch.int32, device=x.device)
+    out = ctypes.c_int(0)
+    _check(lib().dirotq_act_scale_log2_ph(x.data_ptr(), x.shape[0], Uh.data_ptr(), uh_dtype, Uh.shape[0], Uh.shape[1],
+                                          word.data_ptr(), ctypes.byref(out), _stream(stream)), "dirotq_act_scale_log2_ph")
+    return out.value
 
 
 def dirotq_wait_selftest(workspace: torch.Tensor, limit_us: int = 1000, stream=None) -> None:

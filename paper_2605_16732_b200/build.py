@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdirotq.so")
-SOURCES = ["api.cu", "prepare.cu", "rotate_quant.cu", "w4a4_gemm.cu", "peak.cu", "noalloc.cu", "nvfp4_gemm.cu", "w4a8_gemm.cu", "gptq.cu"]
+SOURCES = ["api.cu", "prepare.cu", "rotate_quant.cu", "w4a4_gemm.cu", "peak.cu", "noalloc.cu", "nvfp4_gemm.cu", "w4a8_gemm.cu", "gptq.cu", "calib.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",

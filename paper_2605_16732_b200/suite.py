@@ -47,19 +47,6 @@ def _householder(K: int, seed: int) -> torch.Tensor:
 FMT = "int4"  # set from --fmt: "int4" (groups of G, bf16 scales) or "nvfp4" (blocks of 16, E4M3 scales)
 
 
-def residual_exponent(x, Uh, rows=1024):
-    """Offline calibration of the NVFP4 projection form's power-of-two activation scale (App. E): the largest
-    Hadamard-rotated residual coefficient of the first `rows` tokens, taken with plain torch ops."""
-    xs = x[:rows].float()
-    Ub = Uh.to(torch.bfloat16).float()
-    d = xs - (xs @ Ub).to(torch.bfloat16).float() @ Ub.t()
-    H = torch.ones((1, 1), device=x.device)
-    while H.shape[0] < 64:
-        H = torch.cat([torch.cat([H, H], 1), torch.cat([H, -H], 1)], 0)
-    amax = float(((d.view(d.shape[0], -1, 64) @ H) / 8.0).abs().max().item())
-    return int(np.ceil(np.log2(amax / 1536.0)))
-
-
 class Case:
     def __init__(self, M, K, N, r, G, model):
         self.M, self.K, self.N, self.r, self.G = M, K, N, r, G
@@ -73,9 +60,8 @@ class Case:
             rows = min(M, 1024)
             xrot = torch.empty((rows, K), dtype=torch.float32, device="cuda")
             dq.dirotq_rotate_quantize(self.x[:rows], probe, dq.alloc_workspace(probe, rows), xrot)
-            amax = float(xrot[:, r:].abs().max().item())
+            ex = dq.dirotq_act_scale_log2_from_rotated(xrot, r)
             probe.close()
-            ex = int(np.ceil(np.log2(amax / 1536.0)))
             self.layer = dq.dirotq_prepare_layer_nvfp4(Wd, Q, r, ex, bias=_bf(bias))
         elif FMT == "w4a8":
             self.layer = dq.dirotq_prepare_layer_w4a8(Wd, Q, r, bias=_bf(bias))
@@ -85,7 +71,7 @@ class Case:
             self.layer = dq.dirotq_prepare_layer_ph(Wd, Q[:, :r].contiguous(), G, bias=_bf(bias))
         elif FMT == "nvfp4_ph":
             Uh = Q[:, :r].contiguous()
-            self.layer = dq.dirotq_prepare_layer_nvfp4_ph(Wd, Uh, residual_exponent(self.x, Uh), bias=_bf(bias))
+            self.layer = dq.dirotq_prepare_layer_nvfp4_ph(Wd, Uh, dq.dirotq_act_scale_log2_ph(self.x[:1024].contiguous(), Uh), bias=_bf(bias))
         else:
             self.layer = dq.dirotq_prepare_layer(Wd, Q, r, G, bias=_bf(bias))
         self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
