@@ -13,7 +13,8 @@ import torch
 
 from . import build as _build
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdirotq.so")
+# DIROTQ_LIBRARY: another build of the same library to load instead (the integer-path fallback, build.build_i8())
+_LIB_PATH = os.environ.get("DIROTQ_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdirotq.so")
 
 DIROTQ_OK = 0
 STATUS_NAMES = {0: "ok", 1: "invalid argument", 2: "unsupported shape", 3: "buffer too small",

@@ -20,24 +20,28 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+# The fallback build: the W4A4 group sums on the integer tensor-core path (see kI8Path in csrc/common.h).  Same sources,
+# same interface; the binding loads it instead of libdirotq.so when DIROTQ_LIBRARY names it.
+LIB_I8 = os.path.join(HERE, "libdirotq_i8.so")
+
+
+def needs_build(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "dirotq.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB
+def _build(lib: str, build_dir: str, defines: list[str], force: bool, verbose: bool) -> str:
+    if not force and not needs_build(lib):
+        return lib
     objs = []
     procs = []
-    build_dir = os.path.join(HERE, "_build")
     os.makedirs(build_dir, exist_ok=True)
     for src in SOURCES:
         obj = os.path.join(build_dir, src.replace(".cu", ".o"))
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [_nvcc(), *NVCC_FLAGS, *defines, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
@@ -51,12 +55,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB + f".{os.getpid()}.tmp"
+    tmp = lib + f".{os.getpid()}.tmp"
     subprocess.check_call([_nvcc(), "-Wno-deprecated-gpu-targets", "-shared", "-o", tmp, *objs, "-cudart", "static", "-Xlinker", "--no-undefined",
                            "-lpthread", "-ldl", "-lrt"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    return _build(LIB, os.path.join(HERE, "_build"), [], force, verbose)
+
+
+def build_i8(force: bool = False, verbose: bool = False) -> str:
+    return _build(LIB_I8, os.path.join(HERE, "_build_i8"), ["-DDIROTQ_I8_PATH"], force, verbose)
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    fn = build_i8 if "--i8" in sys.argv else build
+    print(fn(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -89,6 +89,18 @@ __host__ __device__ inline int signmag_nibble_decode(uint32_t word, int t) {
     return (v & 0x80u) ? -mag : mag;
 }
 
+// Fallback build of the library (-DDIROTQ_I8_PATH): the W4A4 group sums run on the integer tensor-core path
+// (tcgen05.mma kind::i8, int32 accumulators) instead of the 8-bit float one, whose exact integer accumulation is a
+// measured property of the hardware rather than a documented one.  The activation codes in the workspace are then
+// two's-complement bytes, the unpack warps turn the weights' sign-magnitude bytes into two's complement, and the
+// epilogue converts every group sum to fp32 before it is scaled (2^18 s_w is stored either way, so the token scale
+// is multiplied by 2^-18 once per group instead).  Same blob, same interface, bit-identical results; slower.
+#ifdef DIROTQ_I8_PATH
+constexpr bool kI8Path = true;
+#else
+constexpr bool kI8Path = false;
+#endif
+
 constexpr size_t kAlign = 1024;
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 

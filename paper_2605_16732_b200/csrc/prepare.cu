@@ -248,7 +248,8 @@ __global__ void export_workspace_kernel(const int8_t* codes, const float* xscale
     for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < g.K_l; c += gridDim.x * blockDim.x)
         if (codes_out) {
             const int sm = static_cast<uint8_t>(codes[static_cast<size_t>(m) * g.K_lp + c]);  // sign-magnitude byte
-            codes_out[static_cast<size_t>(m) * g.K_l + c] = static_cast<int8_t>((sm & 0x80) ? -(sm & 7) : (sm & 7));
+            codes_out[static_cast<size_t>(m) * g.K_l + c] =
+                kI8Path ? static_cast<int8_t>(sm) : static_cast<int8_t>((sm & 0x80) ? -(sm & 7) : (sm & 7));
         }
     if (blockIdx.x == 0) {
         for (int i = threadIdx.x; i < g.r; i += blockDim.x)
@@ -297,7 +298,7 @@ __global__ void debug_codes_kernel(const int8_t* in, uint8_t* out, float* xscale
     for (int j = 0; j < g.G; ++j) {
         const size_t idx = static_cast<size_t>(m) * g.K_lp + grp * g.G + j;
         const int q = in[idx];
-        out[idx] = static_cast<uint8_t>((q < 0 ? 0x80 : 0) | (q < 0 ? -q : q));
+        out[idx] = kI8Path ? static_cast<uint8_t>(q) : static_cast<uint8_t>((q < 0 ? 0x80 : 0) | (q < 0 ? -q : q));
     }
     xscale[static_cast<size_t>(grp) * ldm + m] = 1.0f;
 }

@@ -86,7 +86,7 @@ __device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, 
         const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
         const uint32_t sg = (tw >> 7) & 0x01010101u;           // 1 where the code is negative
         const uint32_t mag = (tw ^ (sg * 0xFFu)) + sg;         // |q| per byte (at most 7: no carry between bytes)
-        w[i] = mag | (tw & 0x80808080u);
+        w[i] = kI8Path ? tw : (mag | (tw & 0x80808080u));  // the integer-path build keeps two's complement
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }

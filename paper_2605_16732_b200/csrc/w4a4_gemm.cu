@@ -46,6 +46,7 @@ constexpr int BM = 128;
 constexpr int BKC = 128;  // one-byte codes per k-block (128-byte rows)
 constexpr int A_BYTES = BM * BKC;          // 16 KB  activation codes / bf16 x~_h chunk
 constexpr uint32_t kSignMag = 0x87878787u;  // sign and 3-bit magnitude of four one-byte codes
+constexpr float kAccUnit = kI8Path ? 1.0f : kWScaleFold;  // integer group sum = accumulator value x this
 
 // Plan for tiles of BN output columns.
 //   256: two epilogue warpgroups, 128 columns (128 fp32 accumulators) per thread; an accumulator tile can only be read in
@@ -120,6 +121,17 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {  // roun
     uint64_t r;
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
+}
+
+// Four weight codes as the bytes the MMA reads: the sign-magnitude bytes themselves (E4M3 path) or, in the integer-path
+// build, their two's complement (per byte: (m ^ s) - s with s = 0xFF where the sign bit is set).
+__device__ __forceinline__ uint32_t code_bytes(uint32_t v) {
+    if constexpr (!kI8Path) {
+        return v;
+    } else {
+        const uint32_t sg = ((v >> 7) & 0x01010101u) * 0xFFu;
+        return __vsub4((v & 0x07070707u) ^ sg, sg);
+    }
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -263,6 +275,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             // word, which cannot overflow: shared-memory addresses have 18 bits, the field holds address / 16).
             if (lane == 0) {
                 constexpr uint32_t idesc_f8 = umma_idesc(1 /*f32*/, 0 /*E4M3*/, BM, BN);
+                constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);  // integer-path build only
                 constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
                 const uint64_t desc0 = umma_desc_sw128(smem_base);
                 const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32), desc_lo0 = static_cast<uint32_t>(desc0);
@@ -287,7 +300,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
                                 for (int k = 0; k < MMA_PER_G; ++k) {
                                     const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
-                                    umma_f8f6f4(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_f8, k != 0);
+                                    if constexpr (kI8Path)
+                                        umma_i8(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_i8, k != 0);
+                                    else
+                                        umma_f8f6f4(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_f8, k != 0);
                                 }
                                 umma_commit(tfull_bar(b));
                                 if (++b == NBUF) { b = 0; bph ^= 1; }
@@ -345,7 +361,6 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         // The loads of a batch are issued before any of its stores: the compiler cannot prove that the
                         // staging buffer and the operand tile do not overlap, so a load written after a store would wait
                         // for it and the whole unpack would run as one dependent chain.
-#pragma unroll
                         constexpr int PIECES = (BN * 4) / 64, BATCH = PIECES % 8 == 0 ? 8 : 4;
 #pragma unroll
                         for (int jb = 0; jb < PIECES; jb += BATCH) {
@@ -357,10 +372,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                 // a word holds codes k..k+3 in bits 7, 2..0 of its bytes and codes k+4..k+7 four bit
                                 // positions further up, wrapping around (see prepare.cu): mask, rotate, mask
                                 uint4 o0, o1;
-                                o0.x = pk[j].x & kSignMag; o0.y = __funnelshift_r(pk[j].x, pk[j].x, 4) & kSignMag;
-                                o0.z = pk[j].y & kSignMag; o0.w = __funnelshift_r(pk[j].y, pk[j].y, 4) & kSignMag;
-                                o1.x = pk[j].z & kSignMag; o1.y = __funnelshift_r(pk[j].z, pk[j].z, 4) & kSignMag;
-                                o1.z = pk[j].w & kSignMag; o1.w = __funnelshift_r(pk[j].w, pk[j].w, 4) & kSignMag;
+                                o0.x = code_bytes(pk[j].x & kSignMag); o0.y = code_bytes(__funnelshift_r(pk[j].x, pk[j].x, 4) & kSignMag);
+                                o0.z = code_bytes(pk[j].y & kSignMag); o0.w = code_bytes(__funnelshift_r(pk[j].y, pk[j].y, 4) & kSignMag);
+                                o1.x = code_bytes(pk[j].z & kSignMag); o1.y = code_bytes(__funnelshift_r(pk[j].z, pk[j].z, 4) & kSignMag);
+                                o1.z = code_bytes(pk[j].w & kSignMag); o1.w = code_bytes(__funnelshift_r(pk[j].w, pk[j].w, 4) & kSignMag);
                                 *reinterpret_cast<uint4*>(d0 + (jb + j) * 2048) = o0;  // 16 rows of 128 bytes further down
                                 *reinterpret_cast<uint4*>(d1 + (jb + j) * 2048) = o1;
                             }
@@ -431,10 +446,11 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 const int gi = g & (GPK - 1);
                 const bool last_of_kb = gi == GPK - 1 || g == p.n_g - 1;
                 const float* s_sw = sc0 + slot * (SC_BYTES / 4);
-                // the accumulator holds S = 2^-18 P
+                // the accumulator holds S = 2^-18 P (integer-path build: P as int32, and 2^-18 goes into the token scale)
                 float sxv[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sxv[i] = s_sw[2 * BN + gi * BM + q * 32 + lr4 + 8 * i];
+                for (int i = 0; i < 4; ++i)
+                    sxv[i] = s_sw[2 * BN + gi * BM + q * 32 + lr4 + 8 * i] * (kI8Path ? 1.0f / kWScaleFold : 1.0f);
                 const float4* swp = reinterpret_cast<const float4*>(s_sw + gi * BN + half * HB + 4 * lc2);
                 // what comes after this tile: the next group's, or the rank-r tile
                 const uint32_t nb = b + 1 == NBUF ? 0 : b + 1, nbph = b + 1 == NBUF ? bph ^ 1 : bph;
@@ -453,6 +469,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                     tmem_ld_wait();  // waits for every outstanding load, hence a look-ahead of one chunk
                     tmem_ld_fence(cur);
+                    if constexpr (kI8Path) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) cur[i] = __float_as_uint(__int2float_rn(static_cast<int>(cur[i])));  // |P| < 2^24: exact
+                    }
                     if (c < CHUNKS - 1) {
                         request_chunk(b, c + 1, raw[(c + 1) & 1]);
                     } else {
@@ -475,8 +495,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                 const int col = colbase + c * 32 + cb * 8 + lc2;
                                 if (row < p.M && col < p.N)
                                     *reinterpret_cast<int2*>(p.partials + (static_cast<size_t>(g) * p.M + row) * p.N + col) =
-                                        make_int2(__float2int_rn(__uint_as_float(cur[pidx]) * 262144.0f),
-                                                  __float2int_rn(__uint_as_float(cur[pidx + 1]) * 262144.0f));
+                                        make_int2(__float2int_rn(__uint_as_float(cur[pidx]) * kAccUnit),
+                                                  __float2int_rn(__uint_as_float(cur[pidx + 1]) * kAccUnit));
                             }
                     } else {
                         // t = S s_x for two adjacent columns at a time (one packed multiply: half the issue slots of two
