@@ -216,19 +216,39 @@ def linear_deployed(x_bits, layer, bias=None, want_t: bool = True):
 # ---------------------------------------------------------------------------------------------
 # Projection form with a structured rotation: NOT the paper's Eq. 5 but the cheaper formulation its remarks on the cost
 # of the online rotation point towards (Sec. 4.2 keeps only the top-r directions in 16 bits; App. E notes that the
-# rotation's cost and memory grow with the layer width).  Only U_h is applied densely:
-#     x~_h = bf16(x U_hb),   d = x - x~_h U_hb^T,   x~_l = d H,   y = x~_h (U_hb^T W) + Q4(x~_l) Q4(H^T W) + bias
-# with U_hb = bf16(U_h) and H block-diagonal, one orthonormal Hadamard block per quantization group.  Because d is the
-# residual of the ROUNDED projection, x = x~_h U_hb^T + d holds exactly, so the layer equals x W when nothing is
-# quantized, for any U_h.  These functions are the reference the library's projection-form layers are held to.
+# rotation's cost and memory grow with the layer width).  Only U_h is applied densely, and the residual is taken in
+# the Hadamard domain so that both of its terms are plain matrix products:
+#     U_hb = bf16(U_h),   V = bf16(U_hb^T H+-)            [r, K]   (H+- = sqrt(G) H: block-diagonal, entries +-1)
+#     x~_h = bf16(x U_hb)
+#     x~_l = (x H+-  -  x~_h V) / sqrt(G)
+#     y    = x~_h ((V H+-^T / G) W)  +  Q4(x~_l) Q4(H^T W)  +  bias
+# with H block-diagonal, one orthonormal Hadamard block per quantization group.  x H+- = sqrt(G) x~_l + x~_h V holds by
+# construction, and H+- H+-^T = G I, so x = x~_l H^T + x~_h (V H+-^T / G): the layer equals x W when nothing is
+# quantized, for any U_h and whatever the rounding of V.  (With V unrounded, x~_l is the block-Hadamard transform of the
+# residual x - x~_h U_hb^T of the rounded projection.)  These functions are the reference the library's projection-form
+# layers are held to.
 
-def hadamard(n: int) -> np.ndarray:
-    """Orthonormal Sylvester-Hadamard matrix of order n (a power of two): entries +-1/sqrt(n), symmetric."""
+def hadamard_signs(n: int) -> np.ndarray:
+    """Sylvester-Hadamard matrix of order n (a power of two) with entries +-1: symmetric, H+- H+-^T = n I."""
     assert n >= 1 and n & (n - 1) == 0
     H = np.ones((1, 1), dtype=np.float64)
     while H.shape[0] < n:
         H = np.block([[H, H], [H, -H]])
-    return H / np.sqrt(float(n))
+    return H
+
+
+def hadamard(n: int) -> np.ndarray:
+    """Orthonormal Sylvester-Hadamard matrix of order n: entries +-1/sqrt(n), symmetric."""
+    return hadamard_signs(n) / np.sqrt(float(n))
+
+
+def block_signs_cols(A, G: int) -> np.ndarray:
+    """A H+-: every group of G consecutive COLUMNS of A multiplied by the +-1 Hadamard block (sums only: exact in fp64
+    for operands of a few significant bits)."""
+    A = _c(A, np.float64)
+    M, K = A.shape
+    assert K % G == 0
+    return (A.reshape(M, K // G, G) @ hadamard_signs(G)).reshape(M, K)
 
 
 def block_hadamard_rows(A, G: int) -> np.ndarray:
@@ -246,6 +266,29 @@ def block_hadamard_cols(A, G: int) -> np.ndarray:
     return block_hadamard_rows(np.ascontiguousarray(A.T), G).T.copy()
 
 
+def projection_operands_ph(Uh, G: int):
+    """U_hb = bf16(U_h) [K, r] and V = bf16(U_hb^T H+-) [r, K], both as bf16 bit patterns."""
+    Uh = _c(Uh, np.float64)
+    Uhb = bf16_round(Uh)
+    V = bf16_round(block_signs_cols(np.ascontiguousarray(bf16_to_f64(Uhb).T), G))
+    return Uhb, V
+
+
+def folded_high_rows_ph(V_bits, W, G: int) -> np.ndarray:
+    """(V H+-^T / G) W [r, N] in fp64: the weight the 16-bit coefficients x~_h multiply."""
+    back = block_signs_cols(bf16_to_f64(V_bits), G) / float(G)      # V H+-^T / G (H+- is symmetric); exact
+    return matmul(np.ascontiguousarray(back), _c(W, np.float64))
+
+
+def residual_ph(x_bits, layer, G: int, xh_bits=None):
+    """x~_h (bf16 bits) and x~_l = (x H+- - x~_h V) / sqrt(G); xh_bits overrides the reference's own x~_h."""
+    x = bf16_to_f64(_c(x_bits, np.uint16))
+    if xh_bits is None:
+        xh_bits = bf16_round(matmul(x, bf16_to_f64(layer["Uhb"])))
+    xl = (block_signs_cols(x, G) - matmul(bf16_to_f64(xh_bits), bf16_to_f64(layer["V"]))) / np.sqrt(float(G))
+    return xh_bits, xl
+
+
 def prepare_layer_ph(W, Uh, G: int):
     """Offline part of the projection form.  W [K, N]; Uh [K, r] (the leading principal directions, unrounded)."""
     W = _c(W, np.float64)
@@ -253,40 +296,35 @@ def prepare_layer_ph(W, Uh, G: int):
     K, N = W.shape
     r = Uh.shape[1]
     assert Uh.shape[0] == K and K % G == 0
-    Uhb = bf16_round(Uh)                                        # the projection that runs online
-    Wt = np.concatenate([matmul(np.ascontiguousarray(bf16_to_f64(Uhb).T), W), block_hadamard_rows(W, G)], axis=0)
+    Uhb, V = projection_operands_ph(Uh, G)                      # what runs online
+    Wt = np.concatenate([folded_high_rows_ph(V, W, G), block_hadamard_rows(W, G)], axis=0)
     out = prepare_weights(Wt, r, G, want_t=True)               # rows < r -> bf16, the K transformed rows -> INT4 groups
-    out["Uhb"] = Uhb
+    out["Uhb"], out["V"] = Uhb, V
     out["r"], out["G"], out["K"] = r, G, K
     return out
 
 
 def linear_deployed_ph(x_bits, layer, bias=None, want_t: bool = True):
     """Online part of the projection form on bf16 inputs; every intermediate is returned."""
-    r, G, K = layer["r"], layer["G"], layer["K"]
-    x = bf16_to_f64(_c(x_bits, np.uint16))
-    Uhb = bf16_to_f64(layer["Uhb"])
-    xh_bits = bf16_round(matmul(x, Uhb))
-    d = x - matmul(bf16_to_f64(xh_bits), np.ascontiguousarray(Uhb.T))
-    xl = block_hadamard_cols(d, G)
-    sq = split_quantize(np.concatenate([np.zeros((x.shape[0], 0)), xl], axis=1), 0, G, want_t=want_t)
+    G = layer["G"]
+    xh_bits, xl = residual_ph(x_bits, layer, G)
+    sq = split_quantize(np.concatenate([np.zeros((xl.shape[0], 0)), xl], axis=1), 0, G, want_t=want_t)
     P = int_gemm(sq["codes"], layer["wcodes"], G)
     y64, yb = combine(P, sq["scales"], layer["wscales"], xh_bits, layer["Wh"], bias)
-    return {"xh": xh_bits, "d": d, "xl": xl, "codes": sq["codes"], "scales": sq["scales"], "t": sq["t"], "P": P,
+    return {"xh": xh_bits, "xl": xl, "codes": sq["codes"], "scales": sq["scales"], "t": sq["t"], "P": P,
             "y64": y64, "y": yb}
 
 
 def nvfp4_prepare_layer_ph(W, Uh, want_t: bool = False):
-    """Projection form with NVFP4 operands: rows U_hb^T W in 16 bits, the rows of H^T W (Hadamard blocks of 64) as E2M1
-    codes with E4M3 block scales and a per-tensor power of two, exactly as nvfp4_prepare_layer quantizes its low rows."""
+    """Projection form with NVFP4 operands: rows (V H+-^T / G) W in 16 bits, the rows of H^T W (Hadamard blocks of 64) as
+    E2M1 codes with E4M3 block scales and a per-tensor power of two, exactly as nvfp4_prepare_layer quantizes its low rows."""
     W = _c(W, np.float64)
     Uh = _c(Uh, np.float64)
     K, N = W.shape
     r = Uh.shape[1]
     assert Uh.shape[0] == K and K % 64 == 0
-    Uhb = bf16_round(Uh)
-    Wt = np.ascontiguousarray(np.concatenate([matmul(np.ascontiguousarray(bf16_to_f64(Uhb).T), W), block_hadamard_rows(W, 64)],
-                                             axis=0))
+    Uhb, V = projection_operands_ph(Uh, 64)
+    Wt = np.ascontiguousarray(np.concatenate([folded_high_rows_ph(V, W, 64), block_hadamard_rows(W, 64)], axis=0))
     nb = K // 16
     Wh = np.empty((r, N), dtype=np.uint16)
     wcodes = np.empty((K, N), dtype=np.uint8)
@@ -294,17 +332,12 @@ def nvfp4_prepare_layer_ph(W, Uh, want_t: bool = False):
     wt = np.empty((K, N), dtype=np.float64) if want_t else None
     ew = _load().dq_nvfp4_prepare_weights(_p(Wt), ctypes.c_int(K + r), ctypes.c_int(N), ctypes.c_int(r), _p(Wh), _p(wcodes),
                                           _p(wsf), _p(wt))
-    return {"Wh": Wh, "wcodes": wcodes, "wsf": wsf, "ew": int(ew), "wt": wt, "Uhb": Uhb, "r": r, "K": K}
+    return {"Wh": Wh, "wcodes": wcodes, "wsf": wsf, "ew": int(ew), "wt": wt, "Uhb": Uhb, "V": V, "r": r, "K": K}
 
 
 def nvfp4_residual(x_bits, layer, xh_bits=None):
-    """x~_h (bf16 bits) and x~_l = (x - x~_h U_hb^T) H for the projection form; xh_bits overrides the reference's own x~_h."""
-    x = bf16_to_f64(_c(x_bits, np.uint16))
-    Uhb = bf16_to_f64(layer["Uhb"])
-    if xh_bits is None:
-        xh_bits = bf16_round(matmul(x, Uhb))
-    d = x - matmul(bf16_to_f64(xh_bits), np.ascontiguousarray(Uhb.T))
-    return xh_bits, block_hadamard_cols(d, 64)
+    """residual_ph with the NVFP4 form's Hadamard blocks of 64."""
+    return residual_ph(x_bits, layer, 64, xh_bits=xh_bits)
 
 
 def nvfp4_linear_deployed_ph(x_bits, layer, ex: int, bias=None, want_t: bool = True):

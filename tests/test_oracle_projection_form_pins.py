@@ -1,7 +1,9 @@
 """Pins of the oracle's projection form (only U_h applied densely, the residual rotated by a block Hadamard): the
 reference for the cheaper first stage.  What the construction fixes: the Hadamard blocks
-are orthonormal; the decomposition x = x~_h U_hb^T + d is exact for ANY U_h because d is the residual of the rounded
-projection, so without quantization the layer is x W; the integer path equals dequantize-then-multiply; with no
+are orthonormal; the decomposition x H+- = sqrt(G) x~_l + x~_h V is exact for ANY U_h and any rounding of V because
+x~_l is defined as that difference, so without quantization the layer is x W; up to the rounding of V the low-precision
+coefficients are the block-Hadamard transform of the rounded projection's residual; the integer path equals
+dequantize-then-multiply; with no
 projection it reduces to group-wise rounding of the Hadamard-rotated operands; and on activations with outlier
 directions the projection is what keeps the error down."""
 import numpy as np
@@ -26,24 +28,42 @@ def test_hadamard_blocks_are_orthonormal_and_the_two_transforms_cancel():
     # a constant group has all its energy in the block's first coefficient
     c = orc.block_hadamard_cols(np.full((1, 64), 3.0), 64)
     assert np.isclose(c[0, 0], 3.0 * 8.0) and np.allclose(c[0, 1:], 0.0, atol=1e-12)
+    # the +-1 form: entry (i, j) is (-1)^popcount(i & j); the block product is that matrix applied group by group
+    for n in (4, 64, 128):
+        S = orc.hadamard_signs(n)
+        assert all(S[i, j] == (-1.0) ** bin(i & j).count("1") for i in range(n) for j in range(0, n, 7))
+        assert np.array_equal(S @ S.T, n * np.eye(n))
+    A = np.round(rng.standard_normal((3, 128)) * 64.0)
+    ref = np.array([[sum(A[m, 64 * b + j] * (-1.0) ** bin(j & c).count("1") for j in range(64)) for b in range(2) for c in range(64)]
+                    for m in range(3)])
+    assert np.array_equal(orc.block_signs_cols(A, 64), ref)
 
 
-def test_decomposition_is_exact_for_any_projection():
+@pytest.mark.parametrize("G", [64, 128])
+def test_decomposition_is_exact_for_any_projection(G):
     rng = np.random.default_rng(1)
-    K, N, r, G, M = 256, 48, 32, 64, 33
+    K, N, r, M = 256, 48, 32, 33
     W = rng.standard_normal((K, N)) * 0.02
     x_bits = orc.bf16_round(rng.standard_normal((M, K)) * rng.choice([0.1, 1.0, 20.0], size=(1, K)))
     x = _bf(x_bits)
     for Uh in (np.linalg.qr(rng.standard_normal((K, r)))[0], rng.standard_normal((K, r)) * 0.3):   # orthonormal or not
         lay = orc.prepare_layer_ph(W, Uh, G)
         out = orc.linear_deployed_ph(x_bits, lay)
-        Uhb = _bf(lay["Uhb"])
-        assert np.allclose(_bf(out["xh"]) @ Uhb.T + out["d"], x, rtol=0, atol=1e-12 * np.abs(x).max())
-        # unquantized: x~_h (U_hb^T W) + (d H)(H^T W) = x W
-        ideal = _bf(out["xh"]) @ (Uhb.T @ W) + out["xl"] @ orc.block_hadamard_rows(W, G)
+        Uhb, V, xh = _bf(lay["Uhb"]), _bf(lay["V"]), _bf(out["xh"])
+        S = np.kron(np.eye(K // G), orc.hadamard_signs(G))             # H+- written out
+        assert np.array_equal(lay["Uhb"], orc.bf16_round(Uh)) and np.array_equal(lay["V"], orc.bf16_round(Uhb.T @ S))
+        assert np.array_equal(out["xh"], orc.bf16_round(x @ Uhb))
+        assert np.allclose(np.sqrt(G) * out["xl"] + xh @ V, x @ S, rtol=0, atol=1e-12 * np.abs(x @ S).max())
+        # unquantized: x~_h ((V H+-^T / G) W) + x~_l (H^T W) = x W
+        back = V @ S.T / G
+        ideal = xh @ (back @ W) + out["xl"] @ orc.block_hadamard_rows(W, G)
         assert np.allclose(ideal, x @ W, rtol=1e-10, atol=1e-10)
-        # the high rows of the prepared weight are bf16(U_hb^T W), the low rows the K transformed rows
-        assert np.array_equal(lay["Wh"], orc.bf16_round(Uhb.T @ W))
+        # up to the rounding of V (2^-9 relative per entry), x~_l is the transformed residual of the rounded projection
+        plain = orc.block_hadamard_cols(x - xh @ Uhb.T, G)
+        bound = (np.abs(xh) @ (np.abs(V) * 2.0 ** -9)) / np.sqrt(G)
+        assert np.all(np.abs(out["xl"] - plain) <= bound + 1e-12) and np.abs(out["xl"] - plain).max() > 0
+        # the high rows of the prepared weight are bf16((V H+-^T / G) W), the low rows the K transformed rows
+        assert np.array_equal(lay["Wh"], orc.bf16_round(back @ W))
         assert lay["wcodes"].shape == (K, N) and out["codes"].shape == (M, K)
 
 
@@ -67,7 +87,7 @@ def test_without_projection_it_is_group_rounding_of_the_hadamard_rotated_operand
     x_bits = orc.bf16_round(rng.standard_normal((M, K)))
     lay = orc.prepare_layer_ph(W, np.zeros((K, 16)), G)          # sixteen null directions: x~_h = 0, d = x
     out = orc.linear_deployed_ph(x_bits, lay)
-    assert not out["xh"].any() and np.array_equal(out["d"], _bf(x_bits))
+    assert not out["xh"].any() and not lay["V"].any()
     xr = orc.block_hadamard_cols(_bf(x_bits), G)
     for m in range(M):
         for g in range(K // G):
@@ -102,9 +122,11 @@ def test_nvfp4_projection_form_shares_the_decomposition_and_matches_the_dense_fo
     x = _bf(inp["x"])
     lay = orc.nvfp4_prepare_layer_ph(inp["W"], np.ascontiguousarray(Q[:, :spec.r]), want_t=True)
     xh_bits, xl = orc.nvfp4_residual(inp["x"], lay)
-    Uhb = _bf(lay["Uhb"])
     # same exact decomposition as the INT4 projection form, Hadamard blocks of 64
-    assert np.allclose(_bf(xh_bits) @ Uhb.T + orc.block_hadamard_cols(xl, 64), x, atol=1e-12 * np.abs(x).max())
+    S = np.kron(np.eye(spec.K // 64), orc.hadamard_signs(64))
+    assert np.allclose(8.0 * xl + _bf(xh_bits) @ _bf(lay["V"]), x @ S, rtol=0, atol=1e-12 * np.abs(x @ S).max())
+    ref = orc.prepare_layer_ph(inp["W"], np.ascontiguousarray(Q[:, :spec.r]), 64)
+    assert np.array_equal(lay["V"], ref["V"]) and np.array_equal(lay["Uhb"], ref["Uhb"]) and np.array_equal(lay["Wh"], ref["Wh"])
     ex = orc.nvfp4_global_exponent(float(np.abs(xl).max()))
     out = orc.nvfp4_linear_deployed_ph(inp["x"], lay, ex, bias=inp["bias"])
     # block-scaled product = dequantize-then-multiply of the codes it returns
