@@ -258,12 +258,15 @@ DIROTQ_API dirotq_status_t dirotq_prepare_layer_sibling(const void* W, int w_dty
  * online rotation point towards: paper Sec. 4.2 keeps only the leading r directions in 16 bits, App. E notes that the
  * rotation's cost and memory grow with the layer width) ----
  *
- *     x~_h = bf16(x U_hb)           U_hb = bf16(U_h), U_h [K,r] the leading principal directions
- *     d    = x - x~_h U_hb^T        residual of the ROUNDED projection, so x = x~_h U_hb^T + d exactly
- *     x~_l = d H                    H block-diagonal: one orthonormal Hadamard block per quantization group
- *     y    = bf16( x~_h (U_hb^T W) + Q4(x~_l) Q4(H^T W) + bias )      Q4 as in dirotq_prepare_layer, over all K columns
+ *     x~_h = bf16(x U_hb)                       U_hb = bf16(U_h), U_h [K,r] the leading principal directions
+ *     x~_l = (x H+- - x~_h V) / sqrt(group)     H+- block-diagonal, one Hadamard block of entries +-1 per quantization
+ *                                               group (H = H+- / sqrt(group) is orthonormal); V = bf16(U_hb^T H+-) [r,K]
+ *     y    = bf16( x~_h ((V H+-^T / group) W) + Q4(x~_l) Q4(H^T W) + bias )   Q4 as in dirotq_prepare_layer, over all K columns
  *
- * 4 M K r flops instead of 2 M K^2 in the first stage, and no K x K matrix in the layer.  Uh: DEVICE, row-major [K,r],
+ * x H+- = sqrt(group) x~_l + x~_h V holds by construction and H+- H+-^T = group I, so the layer is x W exactly when
+ * nothing is quantized, for any U_h; with V unrounded, x~_l is the block-Hadamard transform of the rounded projection's
+ * residual x - x~_h U_hb^T.  Both terms of x~_l are matrix products (they run on the tensor core).
+ * 4 M K r + 2 M K group flops instead of 2 M K^2 in the first stage, and no K x K matrix in the layer.  Uh: DEVICE, row-major [K,r],
  * uh_dtype DIROTQ_DTYPE_F64 or _F32; scratch: dirotq_prepare_scratch_bytes_ph bytes.  Such a layer is accepted by
  * dirotq_workspace_bytes, dirotq_linear, dirotq_linear_host, dirotq_rotate_quantize (xrot_f32 must be NULL),
  * dirotq_w4a4_gemm, dirotq_workspace_export (codes [M,K]), dirotq_int_gemm_debug, dirotq_layer_export (wcodes [K,N],
@@ -283,8 +286,10 @@ DIROTQ_API dirotq_status_t dirotq_prepare_layer_nvfp4_ph(const void* W, int w_dt
                                                          int act_scale_log2, void* blob, size_t blob_bytes, void* scratch,
                                                          size_t scratch_bytes, dirotq_stream_t stream,
                                                          dirotq_layer_t** layer_out);
-/* uh_bf16 [K,r]: the rounded projection the layer applies. */
+/* uh_bf16 [K,r]: the rounded projection the layer applies (U_hb); v_bf16 [r,K]: V = bf16(U_hb^T H+-).  DEVICE outputs,
+ * row-major; projection-form layers only (DIROTQ_ERR_INVALID_ARG otherwise). */
 DIROTQ_API dirotq_status_t dirotq_layer_export_uh(const dirotq_layer_t* layer, void* uh_bf16, dirotq_stream_t stream);
+DIROTQ_API dirotq_status_t dirotq_layer_export_v(const dirotq_layer_t* layer, void* v_bf16, dirotq_stream_t stream);
 
 /* ---- asymmetric activation codes (paper Sec. 3, Eq. 1 with z = min X; Sec. 5.1: the 4-bit INT setting
  * quantizes the activations asymmetrically) ---- */
@@ -402,16 +407,18 @@ DIROTQ_API dirotq_status_t dirotq_mma_rate_probe(int kind, int iters, void* stat
  * second-level scale; here 2^e with e = ceil(log2(max|X| / (6 * 256))), an argument of the NVFP4 layers' preparation) ----
  *
  * Both calls find the largest low-precision coefficient of a batch of calibration tokens on the device, SYNCHRONISE
- * `stream` and return e in *act_scale_log2 (HOST).  device_word: 4 bytes of DEVICE scratch.
+ * `stream` and return e in *act_scale_log2 (HOST).  device_word: 4 bytes of DEVICE scratch; scratch: DEVICE, at least
+ * 16 + 4 r K bytes, 16-byte aligned (DIROTQ_ERR_BUFFER_TOO_SMALL otherwise).
  * dirotq_act_scale_log2_from_rotated: from fp32 rotated activations [M,K] in the column order of Q (what
  * dirotq_rotate_quantize exports; the first r columns are the 16-bit ones and are skipped).
  * dirotq_act_scale_log2_ph: projection form, from the tokens x (bf16 [M,K]) and U_h ([K,r] row-major, f64 or f32)
- * alone: x~_h = bf16(x U_hb), d = x - x~_h U_hb^T, Hadamard blocks of 64, largest |coefficient| (fp32 arithmetic: the
- * exponent only needs the maximum to within a few per cent).  K + r <= 51200. */
+ * alone: x~_h = bf16(x U_hb), V = bf16(U_hb^T H+-) with Hadamard blocks of 64, largest |(x H+- - x~_h V) / 8| (fp32
+ * arithmetic).  K + r <= 51200. */
 DIROTQ_API dirotq_status_t dirotq_act_scale_log2_from_rotated(const float* xrot_f32, int M, int K, int r, void* device_word,
                                                               int* act_scale_log2, dirotq_stream_t stream);
 DIROTQ_API dirotq_status_t dirotq_act_scale_log2_ph(const void* x, int M, const void* Uh, int uh_dtype, int K, int r,
-                                                    void* device_word, int* act_scale_log2, dirotq_stream_t stream);
+                                                    void* scratch, size_t scratch_bytes, int* act_scale_log2,
+                                                    dirotq_stream_t stream);
 
 /* ---- failure-path check (no counterpart in the paper) ---------------------------------------- */
 

@@ -31,7 +31,7 @@ EXPORTED = [
     "dirotq_layer_bytes_nvfp4", "dirotq_prepare_layer_nvfp4", "dirotq_workspace_export_nvfp4", "dirotq_layer_export_nvfp4",
     "dirotq_layer_bytes_w4a8", "dirotq_prepare_layer_w4a8", "dirotq_workspace_export_w4a8",
     "dirotq_prepare_layer_codes", "dirotq_prepare_scratch_bytes_gptq", "dirotq_prepare_layer_gptq", "dirotq_layer_bytes_ph", "dirotq_prepare_scratch_bytes_ph", "dirotq_prepare_layer_ph",
-    "dirotq_layer_export_uh", "dirotq_layer_bytes_nvfp4_ph", "dirotq_prepare_layer_nvfp4_ph", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_set_first_step_split", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
+    "dirotq_layer_export_uh", "dirotq_layer_export_v", "dirotq_layer_bytes_nvfp4_ph", "dirotq_prepare_layer_nvfp4_ph", "dirotq_layer_bytes_sibling", "dirotq_prepare_layer_sibling", "dirotq_set_gemm_tile", "dirotq_set_dependent_launch", "dirotq_set_rotation_tile", "dirotq_set_first_step_split", "dirotq_layer_bytes_asym", "dirotq_prepare_layer_asym", "dirotq_workspace_export_asym", "dirotq_layer_export_zero_term",
 ]
 
 
@@ -76,7 +76,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_mma_rate_probe.argtypes = [i, i, vp, ctypes.POINTER(ctypes.c_float), vp]
         L.dirotq_wait_selftest.argtypes = [vp, ctypes.c_uint, vp]
         L.dirotq_act_scale_log2_from_rotated.argtypes = [vp, i, i, i, vp, pi, vp]
-        L.dirotq_act_scale_log2_ph.argtypes = [vp, i, vp, i, i, i, vp, pi, vp]
+        L.dirotq_act_scale_log2_ph.argtypes = [vp, i, vp, i, i, i, vp, sz, pi, vp]
         L.dirotq_layer_bytes_nvfp4.argtypes = [i, i, i, psz]
         L.dirotq_prepare_layer_nvfp4.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_workspace_export_nvfp4.argtypes = [vp, i, vp, vp, vp, vp, vp]
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.dirotq_prepare_scratch_bytes_ph.argtypes = [i, i, i, ctypes.POINTER(sz)]
         L.dirotq_prepare_layer_ph.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_layer_export_uh.argtypes = [vp, vp, vp]
+        L.dirotq_layer_export_v.argtypes = [vp, vp, vp]
         L.dirotq_layer_bytes_nvfp4_ph.argtypes = [i, i, i, ctypes.POINTER(sz)]
         L.dirotq_prepare_layer_nvfp4_ph.argtypes = [vp, i, i, vp, i, vp, i, i, i, i, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         L.dirotq_set_gemm_tile.argtypes = [i]
@@ -300,10 +301,11 @@ def dirotq_act_scale_log2_ph(x: torch.Tensor, Uh: torch.Tensor, stream=None) -> 
     """Projection form: the same exponent from calibration tokens x (bf16 [M, K]) and U_h ([K, r], f64 or f32)."""
     assert x.is_cuda and x.is_contiguous() and x.dtype == torch.bfloat16 and Uh.is_cuda and Uh.is_contiguous()
     uh_dtype = {torch.float64: DTYPE_F64, torch.float32: DTYPE_F32}[Uh.dtype]
-    word = torch.zeros(1, dtype=torch.int32, device=x.device)
+    K, r = Uh.shape
+    scratch = torch.empty(16 + 4 * r * K, dtype=torch.uint8, device=x.device)
     out = ctypes.c_int(0)
-    _check(lib().dirotq_act_scale_log2_ph(x.data_ptr(), x.shape[0], Uh.data_ptr(), uh_dtype, Uh.shape[0], Uh.shape[1],
-                                          word.data_ptr(), ctypes.byref(out), _stream(stream)), "dirotq_act_scale_log2_ph")
+    _check(lib().dirotq_act_scale_log2_ph(x.data_ptr(), x.shape[0], Uh.data_ptr(), uh_dtype, K, r, scratch.data_ptr(),
+                                          scratch.numel(), ctypes.byref(out), _stream(stream)), "dirotq_act_scale_log2_ph")
     return out.value
 
 
@@ -478,6 +480,13 @@ def dirotq_layer_export_uh(layer: Layer, stream=None) -> torch.Tensor:
     uh = torch.empty((layer.K, layer.r), dtype=torch.bfloat16, device=layer.blob.device)
     _check(lib().dirotq_layer_export_uh(layer.handle, uh.data_ptr(), _stream(stream)), "dirotq_layer_export_uh")
     return uh
+
+
+def dirotq_layer_export_v(layer: Layer, stream=None) -> torch.Tensor:
+    """V = bf16(U_hb^T H+-) [r, K] of a projection-form layer."""
+    v = torch.empty((layer.r, layer.K), dtype=torch.bfloat16, device=layer.blob.device)
+    _check(lib().dirotq_layer_export_v(layer.handle, v.data_ptr(), _stream(stream)), "dirotq_layer_export_v")
+    return v
 
 
 def dirotq_set_gemm_tile(columns: int) -> None:

@@ -386,12 +386,15 @@ dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout
     L->lay = lay;
     L->blob = static_cast<char*>(blob);
     // first stage, step 1: x [M,K] times U_hb^T stored as [r_pad][K] (a 128-row box reads zeros past r_pad);
-    // step 2: x~_h [M,r_pad] times U_hb stored as [K][r_pad]
+    // step 2: x~_h [M,r_pad] times -V^T stored as [K][r_pad], then x times the +-1 Hadamard block, group by group
     st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K,
                         (uint64_t)g.r_pad, (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_uh, (uint64_t)g.r_pad,
                             (uint64_t)K, (uint64_t)g.r_pad * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_had, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_had, (uint64_t)g.G,
+                            (uint64_t)g.G, (uint64_t)g.G * 2, 64, g.G, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -426,7 +429,12 @@ dirotq_status_t dirotq_prepare_layer_ph(const void* W, int w_dtype, int w_layout
 
 dirotq_status_t dirotq_layer_export_uh(const dirotq_layer_t* layer, void* uh_bf16, dirotq_stream_t stream) {
     if (!valid_layer(layer) || !layer->geo.ph || !uh_bf16) return DIROTQ_ERR_INVALID_ARG;
-    return launch_uh_export(layer, static_cast<uint16_t*>(uh_bf16), static_cast<cudaStream_t>(stream));
+    return launch_uh_export(layer, static_cast<uint16_t*>(uh_bf16), nullptr, static_cast<cudaStream_t>(stream));
+}
+
+dirotq_status_t dirotq_layer_export_v(const dirotq_layer_t* layer, void* v_bf16, dirotq_stream_t stream) {
+    if (!valid_layer(layer) || !layer->geo.ph || !v_bf16) return DIROTQ_ERR_INVALID_ARG;
+    return launch_uh_export(layer, nullptr, static_cast<uint16_t*>(v_bf16), static_cast<cudaStream_t>(stream));
 }
 
 dirotq_status_t dirotq_layer_bytes_w4a8(int K, int N, int r, size_t* bytes) {
@@ -921,6 +929,9 @@ dirotq_status_t dirotq_prepare_layer_nvfp4_ph(const void* W, int w_dtype, int w_
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_qt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_uh, (uint64_t)g.r_pad,
                             (uint64_t)K, (uint64_t)g.r_pad * 2, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_had, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_had, (uint64_t)g.G,
+                            (uint64_t)g.G, (uint64_t)g.G * 2, 64, g.G, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked, (uint64_t)g.K4 / 2,
                             (uint64_t)N, (uint64_t)g.K4 / 2, 128, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);

@@ -3,8 +3,9 @@
 // the largest block scale lands in (128, 256] of E4M3's range).  Offline, outside the timed path: the largest
 // low-precision coefficient of a batch of calibration tokens is found on the device and turned into e on the host.
 //   * dense rotation: from the fp32 rotated activations that dirotq_rotate_quantize exports;
-//   * projection form: x~_h = bf16(x U_hb), d = x - x~_h U_hb^T, x~_l = d H (orthonormal Hadamard blocks of 64), from x
-//     and U_h alone (no layer exists yet: the exponent is an argument of the layer's preparation).
+//   * projection form: x~_h = bf16(x U_hb), x~_l = (x H+- - x~_h V) / 8 with V = bf16(U_hb^T H+-) and H+- the +-1
+//     Hadamard blocks of 64, from x and U_h alone (no layer exists yet: the exponent is an argument of the layer's
+//     preparation).
 #include "common.h"
 
 #include <math.h>
@@ -52,9 +53,27 @@ __global__ void __launch_bounds__(256) absmax_low_kernel(const float* xrot, int 
     block_max_to(out, v, red);
 }
 
-// One CTA per token row.  Dynamic shared memory: K floats (the residual) after r_max floats (x~_h).
+// V[i][k] = bf16(sum_j (-1)^popc(j & c) U_hb[64 b + j][i]) for k = 64 b + c, as fp32 (the sum is exact in fp64)
+__global__ void __launch_bounds__(128) projection_v_kernel(const void* Uh, int uh_dtype, int K, int r, float* V) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const int b = k / 64, c = k % 64;
+    for (int i = 0; i < r; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < 64; ++j) {
+            const double u = static_cast<double>(load_uh_bf16(Uh, uh_dtype, static_cast<size_t>(64 * b + j) * r + i));
+            acc += (__popc(j & c) & 1) ? -u : u;
+        }
+        float f = __double2float_rz(acc);  // one rounding into bf16: round to odd into fp32 first
+        uint32_t u = __float_as_uint(f);
+        if (static_cast<double>(f) != acc) u |= 1u;
+        V[static_cast<size_t>(i) * K + k] = bf16_round_f32(__uint_as_float(u));
+    }
+}
+
+// One CTA per token row.  Dynamic shared memory: K floats (x H+-, then the residual) after r floats (x~_h).
 __global__ void __launch_bounds__(256) residual_absmax_kernel(const uint16_t* x, int M, int K, int r, const void* Uh, int uh_dtype,
-                                                              unsigned int* out) {
+                                                              const float* V, unsigned int* out) {
     extern __shared__ float sm[];
     __shared__ float red[8];
     float* xh = sm;       // [r]
@@ -68,13 +87,9 @@ __global__ void __launch_bounds__(256) residual_absmax_kernel(const uint16_t* x,
         xh[i] = bf16_round_f32(acc);
     }
     __syncthreads();
-    for (int k = threadIdx.x; k < K; k += blockDim.x) {
-        float acc = 0.f;
-        for (int i = 0; i < r; ++i) acc = fmaf(xh[i], load_uh_bf16(Uh, uh_dtype, static_cast<size_t>(k) * r + i), acc);
-        d[k] = __uint_as_float(static_cast<uint32_t>(xr[k]) << 16) - acc;
-    }
+    for (int k = threadIdx.x; k < K; k += blockDim.x) d[k] = __uint_as_float(static_cast<uint32_t>(xr[k]) << 16);
     __syncthreads();
-    // Hadamard blocks of 64: six butterfly stages in place
+    // x H+-, Hadamard blocks of 64: six butterfly stages in place
     for (int h = 1; h < 64; h <<= 1) {
         for (int p = threadIdx.x; p < K / 2; p += blockDim.x) {
             const int blk = p / 32, q = p % 32;              // pair q of block blk
@@ -87,7 +102,11 @@ __global__ void __launch_bounds__(256) residual_absmax_kernel(const uint16_t* x,
         __syncthreads();
     }
     float v = 0.f;
-    for (int k = threadIdx.x; k < K; k += blockDim.x) v = fmaxf(v, fabsf(d[k]) * 0.125f);
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float acc = 0.f;
+        for (int i = 0; i < r; ++i) acc = fmaf(xh[i], V[static_cast<size_t>(i) * K + k], acc);
+        v = fmaxf(v, fabsf(d[k] - acc) * 0.125f);
+    }
     block_max_to(out, v, red);
 }
 
@@ -119,9 +138,13 @@ extern "C" dirotq_status_t dirotq_act_scale_log2_from_rotated(const float* xrot_
 }
 
 extern "C" dirotq_status_t dirotq_act_scale_log2_ph(const void* x, int M, const void* Uh, int uh_dtype, int K, int r,
-                                                   void* device_word, int* act_scale_log2, dirotq_stream_t stream) {
-    if (!x || !Uh || !device_word || !act_scale_log2 || M < 1 || K < 64 || K % 64 != 0 || r < 1 || r >= K)
+                                                   void* scratch, size_t scratch_bytes, int* act_scale_log2,
+                                                   dirotq_stream_t stream) {
+    if (!x || !Uh || !scratch || !act_scale_log2 || M < 1 || K < 64 || K % 64 != 0 || r < 1 || r >= K)
         return DIROTQ_ERR_INVALID_ARG;
+    if (scratch_bytes < 16 + static_cast<size_t>(r) * K * sizeof(float)) return DIROTQ_ERR_BUFFER_TOO_SMALL;
+    void* device_word = scratch;
+    float* V = reinterpret_cast<float*>(static_cast<char*>(scratch) + 16);
     if (uh_dtype != DIROTQ_DTYPE_F64 && uh_dtype != DIROTQ_DTYPE_F32) return DIROTQ_ERR_INVALID_ARG;
     const size_t smem = static_cast<size_t>(K + r) * sizeof(float);
     if (smem > 200 * 1024) return DIROTQ_ERR_UNSUPPORTED_SHAPE;
@@ -131,7 +154,9 @@ extern "C" dirotq_status_t dirotq_act_scale_log2_ph(const void* x, int M, const 
     if (!opt_in.ensure(residual_absmax_kernel, 0, dev, 200 * 1024)) return DIROTQ_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(device_word, 0, 4, s) != cudaSuccess) return DIROTQ_ERR_CUDA;
-    residual_absmax_kernel<<<M, 256, smem, s>>>(static_cast<const uint16_t*>(x), M, K, r, Uh, uh_dtype,
+    projection_v_kernel<<<(K + 127) / 128, 128, 0, s>>>(Uh, uh_dtype, K, r, V);
+    if (cudaGetLastError() != cudaSuccess) return DIROTQ_ERR_CUDA;
+    residual_absmax_kernel<<<M, 256, smem, s>>>(static_cast<const uint16_t*>(x), M, K, r, Uh, uh_dtype, V,
                                                 static_cast<unsigned int*>(device_word));
     if (cudaGetLastError() != cudaSuccess) return DIROTQ_ERR_CUDA;
     return finish(static_cast<unsigned int*>(device_word), s, act_scale_log2);

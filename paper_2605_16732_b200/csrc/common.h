@@ -139,7 +139,10 @@ struct BlobLayout {
     // NVFP4 variant: off_wpacked = E2M1 codes u8 [N][K4/2] (even k in the low nibble); off_wscale = E4M3 scale
     // atoms u8 [ceil(N/128)][nkb64p][512]; off_meta = {float out_scale = 2^(ex+ew), int ew, int ex, uint amax bits}
     size_t off_meta;
-    size_t off_uh;       // fmt 4 only: bf16 [K][r_pad], U_hb row-major (off_qt then holds its transpose, bf16 [r_pad][K])
+    // projection form only: off_qt holds U_hb^T, bf16 [r_pad][K]; off_uh holds -V^T, bf16 [K][r_pad], with
+    // V = bf16(U_hb^T H+-); off_had holds one +-1 Hadamard block, bf16 [G][G] (G = 64 for NVFP4 layers)
+    size_t off_uh;
+    size_t off_had;
     size_t total;
 };
 
@@ -148,6 +151,7 @@ inline BlobLayout make_blob_layout(const Geometry& g) {
     size_t o = 0;
     b.off_qt = o;      o = align_up(o + (g.fmt == 4 ? (size_t)g.r_pad * g.K * 2 : g.no_rot ? 0 : (size_t)g.K * g.K * 2));
     b.off_uh = o;      o = align_up(o + (g.fmt == 4 ? (size_t)g.K * g.r_pad * 2 : 0));
+    b.off_had = o;     o = align_up(o + (g.fmt == 4 ? (size_t)g.G * g.G * 2 : 0));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K_lp / 2));
     b.off_wscale = o;  o = align_up(o + (size_t)g.n_g * wscale_row_len(g.N) * 4);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
@@ -162,6 +166,7 @@ inline BlobLayout make_blob_layout_nvfp4(const Geometry& g) {
     size_t o = 0;
     b.off_qt = o;      o = align_up(o + (g.ph ? (size_t)g.r_pad * g.K * 2 : (size_t)g.K * g.K * 2));
     b.off_uh = o;      o = align_up(o + (g.ph ? (size_t)g.K * g.r_pad * 2 : 0));
+    b.off_had = o;     o = align_up(o + (g.ph ? (size_t)64 * 64 * 2 : 0));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K4 / 2));
     b.off_wscale = o;  o = align_up(o + (size_t)((g.N + 127) / 128) * g.nkb64p * 512);
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
@@ -235,6 +240,7 @@ struct dirotq_layer {
     char* blob;  // device
     CUtensorMap tmap_qt;       // bf16 [K][K], box 64 x 256, 128B swizzle
     CUtensorMap tmap_qt128;    // the same tensor with box 64 x 128 (narrow tiles of the rotation kernel)
+    CUtensorMap tmap_had;      // projection form: the +-1 Hadamard block, bf16 [G][G], box 64 x G, 128B swizzle
     CUtensorMap tmap_wpacked;  // u8 [N][K_lp/2] (two codes per byte), box 64 x kGemmBN, no swizzle
     CUtensorMap tmap_wscale;   // f32 [n_g][N32], box kGemmBN x (128/G)
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
@@ -339,7 +345,7 @@ dirotq_status_t set_rotation_plan(int plan);
 void set_first_step_split(bool on);
 dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
                                   const void* bias, double* scratch, cudaStream_t stream);
-dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, cudaStream_t stream);
+dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, uint16_t* v, cudaStream_t stream);
 dirotq_status_t launch_prepare_nvfp4_ph(const dirotq_layer* L, const void* W, int w_dtype, int w_layout, const void* Uh, int uh_dtype,
                                         const void* bias, double* scratch, cudaStream_t stream);
 dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream);

@@ -588,26 +588,66 @@ __device__ __forceinline__ double load_uh(const void* Uh, int dtype, int r, int 
     return dtype == DIROTQ_DTYPE_F64 ? static_cast<const double*>(Uh)[e] : static_cast<double>(static_cast<const float*>(Uh)[e]);
 }
 
-// uht[i][k] = uh[k][i] = bf16(Uh[k][i]), zero for i >= r
-__global__ void ph_round_uh_kernel(const void* Uh, int dtype, uint16_t* uht, uint16_t* uh, Geometry g) {
+// uht[i][k] = bf16(Uh[k][i]) = U_hb^T, zero for i >= r
+__global__ void ph_round_uh_kernel(const void* Uh, int dtype, uint16_t* uht, Geometry g) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= g.K) return;
+    for (int i = 0; i < g.r_pad; ++i)
+        uht[static_cast<size_t>(i) * g.K + k] = i < g.r ? f64_to_bf16(load_uh(Uh, dtype, g.r, k, i)) : 0;
+}
+
+// V = bf16(U_hb^T H+-): V[i][b hg + c] = bf16(sum_j (-1)^popc(j & c) U_hb[b hg + j][i]) (an exact fp64 sum of bf16 values,
+// rounded once).  Stored negated and transposed, negvt[k][i] = -V[i][k], the B operand of the online residual's
+// projection term; zero for i >= r.  hg: order of the Hadamard blocks.
+__global__ void ph_v_kernel(const uint16_t* uht, uint16_t* negvt, int hg, Geometry g) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= g.K) return;
+    const int b = k / hg, c = k % hg;
     for (int i = 0; i < g.r_pad; ++i) {
-        const uint16_t v = i < g.r ? f64_to_bf16(load_uh(Uh, dtype, g.r, k, i)) : 0;
-        uht[static_cast<size_t>(i) * g.K + k] = v;
-        uh[static_cast<size_t>(k) * g.r_pad + i] = v;
+        uint16_t out = 0;
+        if (i < g.r) {
+            double acc = 0.0;
+            for (int j = 0; j < hg; ++j) {
+                const double u = bf16_to_f64(uht[static_cast<size_t>(i) * g.K + b * hg + j]);
+                acc += (__popc(j & c) & 1) ? -u : u;
+            }
+            out = f64_to_bf16(-acc);
+        }
+        negvt[static_cast<size_t>(k) * g.r_pad + i] = out;
     }
 }
 
-// Wt[i][n] = sum_k U_hb[k][i] W[k][n] for i < r (fp64 sums of the ROUNDED projection times the weights)
-__global__ void ph_fold_high_kernel(const uint16_t* uh, const void* W, int w_dtype, int w_layout, double* Wt, Geometry g) {
+// had[c][j] = (-1)^popc(c & j) as bf16
+__global__ void ph_hadamard_kernel(uint16_t* had, int hg) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= hg * hg) return;
+    had[idx] = (__popc((idx / hg) & (idx % hg)) & 1) ? 0xBF80 : 0x3F80;
+}
+
+// Wt[i][n] = sum_k back[k][i] W[k][n] for i < r, with back = H+- V^T / hg, i.e. back[b hg + j][i] =
+// (1 / hg) sum_c (-1)^popc(j & c) V[i][b hg + c] (exact in fp64): the weight the 16-bit coefficients multiply.
+// One CTA per (128 output columns, i); a block's hg values of `back` are shared through shared memory.
+__global__ void __launch_bounds__(128) ph_fold_high_kernel(const uint16_t* negvt, const void* W, int w_dtype, int w_layout,
+                                                           double* Wt, int hg, Geometry g) {
+    __shared__ double back[128];
     const int n = blockIdx.x * blockDim.x + threadIdx.x;
     const int i = blockIdx.y;
-    if (n >= g.N) return;
     double acc = 0.0;
-    for (int k = 0; k < g.K; ++k)
-        acc = fma(bf16_to_f64(uh[static_cast<size_t>(k) * g.r_pad + i]), load_w(W, w_dtype, w_layout, g.K, g.N, k, n), acc);
-    Wt[static_cast<size_t>(i) * g.N + n] = acc;
+    for (int b = 0; b < g.K / hg; ++b) {
+        __syncthreads();
+        for (int j = threadIdx.x; j < hg; j += blockDim.x) {
+            double t = 0.0;
+            for (int c = 0; c < hg; ++c) {
+                const double v = -bf16_to_f64(negvt[static_cast<size_t>(b * hg + c) * g.r_pad + i]);
+                t += (__popc(j & c) & 1) ? -v : v;
+            }
+            back[j] = t / static_cast<double>(hg);
+        }
+        __syncthreads();
+        if (n < g.N)
+            for (int j = 0; j < hg; ++j) acc = fma(back[j], load_w(W, w_dtype, w_layout, g.K, g.N, b * hg + j, n), acc);
+    }
+    if (n < g.N) Wt[static_cast<size_t>(i) * g.N + n] = acc;
 }
 
 // Wt[r + b G + i][n] = (1 / sqrt(G)) sum_j (-1)^popc(i & j) W[b G + j][n]: the block Hadamard applied to the rows of W
@@ -624,10 +664,17 @@ __global__ void ph_fold_low_kernel(const void* W, int w_dtype, int w_layout, dou
     Wt[static_cast<size_t>(g.r + row) * g.N + n] = acc / sqrt(static_cast<double>(g.G));
 }
 
-__global__ void ph_export_uh_kernel(const uint16_t* uh, uint16_t* out, Geometry g) {
+// out_uh[k][i] = U_hb[k][i] (K x r) and/or out_v[i][k] = V[i][k] (r x K)
+__global__ void ph_export_uh_kernel(const uint16_t* uht, const uint16_t* negvt, uint16_t* out_uh, uint16_t* out_v, Geometry g) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= g.K) return;
-    for (int i = 0; i < g.r; ++i) out[static_cast<size_t>(k) * g.r + i] = uh[static_cast<size_t>(k) * g.r_pad + i];
+    for (int i = 0; i < g.r; ++i) {
+        if (out_uh) out_uh[static_cast<size_t>(k) * g.r + i] = uht[static_cast<size_t>(i) * g.K + k];
+        if (out_v) {
+            const uint16_t nv = negvt[static_cast<size_t>(k) * g.r_pad + i];
+            out_v[static_cast<size_t>(i) * g.K + k] = (nv & 0x7FFF) ? (nv ^ 0x8000) : 0;
+        }
+    }
 }
 
 }  // namespace
@@ -637,10 +684,15 @@ dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dt
     const Geometry& g = L->geo;
     char* blob = L->blob;
     uint16_t* uht = reinterpret_cast<uint16_t*>(blob + L->lay.off_qt);
-    uint16_t* uh = reinterpret_cast<uint16_t*>(blob + L->lay.off_uh);
-    ph_round_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(Uh, uh_dtype, uht, uh, g);
+    uint16_t* negvt = reinterpret_cast<uint16_t*>(blob + L->lay.off_uh);
+    const int hg = g.fmt == 1 ? 64 : g.G;  // order of the Hadamard blocks
+    ph_round_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(Uh, uh_dtype, uht, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
-    ph_fold_high_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(uh, W, w_dtype, w_layout, scratch, g);
+    ph_v_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(uht, negvt, hg, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_hadamard_kernel<<<(hg * hg + 255) / 256, 256, 0, stream>>>(reinterpret_cast<uint16_t*>(blob + L->lay.off_had), hg);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_fold_high_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(negvt, W, w_dtype, w_layout, scratch, hg, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     ph_fold_low_kernel<<<dim3((g.N + 127) / 128, g.K), 128, 0, stream>>>(W, w_dtype, w_layout, scratch, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
@@ -658,9 +710,10 @@ dirotq_status_t launch_prepare_ph(const dirotq_layer* L, const void* W, int w_dt
     return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
-dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, cudaStream_t stream) {
+dirotq_status_t launch_uh_export(const dirotq_layer* L, uint16_t* uh, uint16_t* v, cudaStream_t stream) {
     const Geometry& g = L->geo;
-    ph_export_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(reinterpret_cast<const uint16_t*>(L->blob + L->lay.off_uh), uh, g);
+    ph_export_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(reinterpret_cast<const uint16_t*>(L->blob + L->lay.off_qt),
+                                                              reinterpret_cast<const uint16_t*>(L->blob + L->lay.off_uh), uh, v, g);
     return launch_ok() ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
@@ -806,10 +859,15 @@ dirotq_status_t launch_prepare_nvfp4_ph(const dirotq_layer* L, const void* W, in
     char* blob = L->blob;
     Nvfp4Meta* meta = reinterpret_cast<Nvfp4Meta*>(blob + L->lay.off_meta);
     uint16_t* uht = reinterpret_cast<uint16_t*>(blob + L->lay.off_qt);
-    uint16_t* uh = reinterpret_cast<uint16_t*>(blob + L->lay.off_uh);
-    ph_round_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(Uh, uh_dtype, uht, uh, g);
+    uint16_t* negvt = reinterpret_cast<uint16_t*>(blob + L->lay.off_uh);
+    const int hg = g.fmt == 1 ? 64 : g.G;  // order of the Hadamard blocks
+    ph_round_uh_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(Uh, uh_dtype, uht, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
-    ph_fold_high_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(uh, W, w_dtype, w_layout, scratch, g);
+    ph_v_kernel<<<(g.K + 127) / 128, 128, 0, stream>>>(uht, negvt, hg, g);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_hadamard_kernel<<<(hg * hg + 255) / 256, 256, 0, stream>>>(reinterpret_cast<uint16_t*>(blob + L->lay.off_had), hg);
+    if (!launch_ok()) return DIROTQ_ERR_CUDA;
+    ph_fold_high_kernel<<<dim3((g.N + 127) / 128, g.r), 128, 0, stream>>>(negvt, W, w_dtype, w_layout, scratch, hg, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     ph_fold_low_kernel<<<dim3((g.N + 127) / 128, g.K), 128, 0, stream>>>(W, w_dtype, w_layout, scratch, g);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;

@@ -43,7 +43,6 @@ constexpr int SMEM_BYTES = STAGES_WIDE * STAGE_BYTES_WIDE + 1024 /*alignment sla
 struct RotKernelParams {
     int M, K, K_l, K_lp, r, r_pad, r_pad0, ldm, n_g;
     int n_out, k_red;      // output columns and reduction length of the GEMM (both K for the rotation x Q)
-    const uint16_t* xsub;  // FMT 4: bf16 [M][K], the accumulator is subtracted from it (residual of the projection)
     int8_t* codes;
     float* xscale;
     uint16_t* xh;
@@ -67,33 +66,59 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Quantizes 16 consecutive values with the reciprocal scale and packs them one code per byte in
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    // byte permute; a selector nibble with bit 3 set replicates the sign bit of the selected byte
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Quantizes 16 consecutive values, q = clip(rint(pre * v / s), -7, 7), and packs them one code per byte in
 // sign-magnitude form (bit 7 = sign, bits 2..0 = |q|): read as E4M3 that byte is q * 2^-9 exactly, which
 // is how the second kernel's tensor-core instruction consumes it.
-__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, bool slow) {
+// Common path (SLOW = false): t = v * inv with inv = pre / s.  The scale is bf16(max|pre v| / 7) >= max|pre v| / 7 *
+// (1 - 2^-9), so |t| <= 7.02 for finite inputs and rounds to at most 7: no clamp is needed.  |t| + 1.5 * 2^23 leaves
+// |q| (nearest, ties to even) in the low byte of the sum's bit pattern; the signs come from the top bytes of t.
+// SLOW: the scale is zero or too small for its reciprocal: divide (rare, kept out of the common path's code).
+template <bool SLOW>
+__device__ __forceinline__ uint4 quantize16(const float* v, float inv, float s, float pre) {
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        uint32_t f[4];
+        if constexpr (SLOW || kI8Path) {
+            uint32_t f[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float t = slow ? (s != 0.f ? v[4 * i + j] / s : 0.f) : v[4 * i + j] * inv;
-            t = fminf(fmaxf(t, -7.0f), 7.0f);
-            // adding 1.5 * 2^23 rounds to the nearest integer, ties to even, and leaves the two's-complement code
-            // in the low byte of the bit pattern
-            f[j] = __float_as_uint(t + 12582912.0f);
+            for (int j = 0; j < 4; ++j) {
+                float t = SLOW ? (s != 0.f ? (v[4 * i + j] * pre) / s : 0.f) : v[4 * i + j] * inv;
+                t = fminf(fmaxf(t, -7.0f), 7.0f);
+                // adding 1.5 * 2^23 rounds to the nearest integer, ties to even, and leaves the two's-complement code
+                // in the low byte of the bit pattern
+                f[j] = __float_as_uint(t + 12582912.0f);
+            }
+            const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
+            const uint32_t sg = (tw >> 7) & 0x01010101u;           // 1 where the code is negative
+            const uint32_t mag = (tw ^ (sg * 0xFFu)) + sg;         // |q| per byte (at most 7: no carry between bytes)
+            w[i] = kI8Path ? tw : (mag | (tw & 0x80808080u));  // the integer-path build keeps two's complement
+        } else {
+            uint32_t t[4], m[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float tj = v[4 * i + j] * inv;
+                t[j] = __float_as_uint(tj);
+                m[j] = __float_as_uint(fabsf(tj) + 12582912.0f);
+            }
+            const uint32_t mag = prmt(prmt(m[0], m[1], 0x0040u), prmt(m[2], m[3], 0x0040u), 0x5410u);
+            const uint32_t sgn = prmt(prmt(t[0], t[1], 0x00FBu), prmt(t[2], t[3], 0x00FBu), 0x5410u);  // 0xFF where t < 0
+            w[i] = (sgn & 0x80808080u) | mag;
         }
-        const uint32_t tw = __byte_perm(__byte_perm(f[0], f[1], 0x0040), __byte_perm(f[2], f[3], 0x0040), 0x5410);
-        const uint32_t sg = (tw >> 7) & 0x01010101u;           // 1 where the code is negative
-        const uint32_t mag = (tw ^ (sg * 0xFFu)) + sg;         // |q| per byte (at most 7: no carry between bytes)
-        w[i] = kI8Path ? tw : (mag | (tw & 0x80808080u));  // the integer-path build keeps two's complement
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // Asymmetric variant (Eq. 1 with z = min X): 16 values -> 16 bytes u = clip(rint((v - z) / s), 0, 15); as E4M3 the byte
 // 0000uuuu is u * 2^-9 exactly.
-__device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float inv, float s, bool slow) {
+template <bool SLOW>
+__device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float inv, float s) {
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -101,7 +126,7 @@ __device__ __forceinline__ uint4 quantize16_asym(const float* v, float z, float 
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float d = v[4 * i + j] - z;
-            float t = slow ? (s != 0.f ? d / s : 0.f) : d * inv;
+            float t = SLOW ? (s != 0.f ? d / s : 0.f) : d * inv;
             t = fminf(fmaxf(t, 0.0f), 15.0f);
             f[j] = __float_as_uint(t + 12582912.0f);  // nearest integer, ties to even, in the low byte
         }
@@ -139,13 +164,16 @@ __device__ __forceinline__ uint32_t f32x2_to_e2m1x2(float lo, float hi) {
 }
 
 // One block of 16 values: returns the E4M3 scale byte and writes the 8 code bytes (two 32-bit words).
-__device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float ex_inv, float ex_scale, uint32_t& w0, uint32_t& w1) {
-    float amax = 0.f;
+// The values quantized are pre * v[j], pre a power of two (so that scaling the maximum and the reciprocal instead of
+// every value gives the same bits).
+__device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float pre, float ex_inv, float ex_scale, uint32_t& w0, uint32_t& w1) {
+    float am[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[j]));
+    for (int j = 0; j < 16; ++j) am[j & 3] = fmaxf(am[j & 3], fabsf(v[j]));
+    const float amax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * pre;
     const uint32_t sb = f32_to_e4m3(__fdiv_rn(amax, 6.0f) * ex_inv);
     const float s = e4m3_to_f32(sb) * ex_scale;
-    const float inv = s > 0.f ? __frcp_rn(s) : 0.f;
+    const float inv = s > 0.f ? __frcp_rn(s) * pre : 0.f;
     w0 = 0;
     w1 = 0;
 #pragma unroll
@@ -156,10 +184,21 @@ __device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float ex_inv, 
     return sb;
 }
 
-// PH: the epilogue first forms the projection form's residual (FMT 4 is PH with the INT4 quantizer of FMT 0).
-template <int G, int FMT, int BN, int BM, bool PH = (FMT == 4)>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// PH: second step of the projection form (FMT 4 is PH with the INT4 quantizer of FMT 0).  The accumulator of a tile is
+//     x H+- - x~_h V  =  [x~_h | x] [-V ; H+-]
+// built from k_red / 64 k-blocks of x~_h (tmap_x) against -V^T (tmap_qt) over all BN columns, followed, for every group of
+// G columns under the tile, by G / 64 k-blocks of that group's columns of x (tmap_x2) against the +-1 Hadamard block
+// (tmap_had) into the group's own column slice of the accumulator (MMAs with N = G).  The epilogue scales by
+// 1 / sqrt(G) and quantizes.  Without PH the last two tensor maps are not used.  (Cutting the projection term into
+// per-group k-blocks too, for a ring of eight 24 KB stages that holds a whole tile ahead of the MMAs, measured slower:
+// 87 against 79 us for the whole first stage at M = 4608, K = 12288.)
+// EPI_WARPS: 8, or 16 for the PH mode with groups of 64 (four warps per lane quadrant, one 64-column chunk each): that
+// mode has no long main loop to hide the epilogue under, and its epilogue is a chain of dependent instructions per
+// thread that only more warps per scheduler speed up.
+template <int G, int FMT, int BN, int BM, bool PH = (FMT == 4), int EPI_WARPS = 8>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
+                    const __grid_constant__ CUtensorMap tmap_x2, const __grid_constant__ CUtensorMap tmap_had,
                     const RotKernelParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -175,14 +214,16 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     constexpr int ACC_BUFS = BM == 256 ? 1 : 2;
     static_assert(STAGES * STAGE_BYTES == STAGES_WIDE * STAGE_BYTES_WIDE && STAGE_BYTES % 1024 == 0, "ring layout");
     const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
-    // barrier map (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+    // barrier map (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2] (at most 20 of them); the
+    // tensor-memory slot, the abort flag and the spare barrier follow at +192, +196 and +200
+    static_assert(8 * (2 * STAGES + 4) <= 192, "barriers end below the words at +192");
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + STAGES * STAGE_BYTES + 128);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + STAGES * STAGE_BYTES + 132);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + STAGES * STAGE_BYTES + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + STAGES * STAGE_BYTES + 196);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -200,13 +241,17 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 8 * 32);  // every thread of the eight epilogue warps arrives
+            mbar_init(tempty_bar(a), EPI_WARPS * 32);  // every thread of the epilogue warps arrives
         }
-        mbar_init(bar_base + 136u, 1);  // spare: see umma_drain
+        mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
         tma_prefetch_desc(&tmap_qt);
+        if constexpr (PH) {
+            tma_prefetch_desc(&tmap_x2);
+            tma_prefetch_desc(&tmap_had);
+        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
@@ -230,6 +275,27 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 const int mn = tile % num_mn, sp = tile / num_mn;
                 const int m0 = (mn % num_m_blocks) * BM;
                 const int n0 = (mn / num_m_blocks) * BN;
+                if constexpr (PH) {
+                    const int nv = num_kb;                            // k-blocks of the projection term
+                    const int nx = min(BN, p.n_out - n0) / BK;        // 64-column pieces of x under this tile
+                    for (int i = 0; i < nv + nx; ++i, ++it) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                        const uint32_t sa = smem_base + s * STAGE_BYTES;
+                        if (i < nv) {
+                            mbar_arrive_expect_tx(full_bar(s), A_BYTES + BN * BK * 2);
+                            tma_load_2d(sa, &tmap_x, full_bar(s), i * BK, m0);
+                            tma_load_2d(sa + A_BYTES, &tmap_qt, full_bar(s), i * BK, n0);
+                        } else {
+                            const int j = i - nv;
+                            mbar_arrive_expect_tx(full_bar(s), A_BYTES + G * BK * 2);
+                            tma_load_2d(sa, &tmap_x2, full_bar(s), n0 + j * BK, m0);
+                            tma_load_2d(sa + A_BYTES, &tmap_had, full_bar(s), (j % (G / BK)) * BK, 0);
+                        }
+                    }
+                    continue;
+                }
                 const int kb_end = static_cast<int>(static_cast<long>(sp + 1) * num_kb / p.ksplit);
                 for (int kb = static_cast<int>(static_cast<long>(sp) * num_kb / p.ksplit); kb < kb_end; ++kb, ++it) {
                     const int s = it % STAGES;
@@ -263,6 +329,31 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + acc * BN;
+                if constexpr (PH) {
+                    constexpr uint32_t idesc_g = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM_MMA, G);
+                    const int n0 = ((tile % num_mn) / num_m_blocks) * BN;
+                    const int nv = num_kb, nx = min(BN, p.n_out - n0) / BK;
+                    for (int i = 0; i < nv + nx; ++i, ++it) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t sa = smem_base + s * STAGE_BYTES;
+                        const uint64_t adesc = umma_desc_sw128(sa);
+                        const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
+                        if (i < nv) {
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k) umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k) != 0);
+                        } else {
+                            const uint32_t dg = d + ((i - nv) / (G / BK)) * G;  // the group's columns of the accumulator
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k) umma_bf16(dg, adesc + 2 * k, bdesc + 2 * k, idesc_g, 1);
+                        }
+                        umma_commit(empty_bar(s));
+                    }
+                    if (ok) umma_commit(tfull_bar(acc));
+                    continue;
+                }
                 const int sp = tile / num_mn;
                 const int kb_begin = static_cast<int>(static_cast<long>(sp) * num_kb / p.ksplit);
                 const int kb_end = static_cast<int>(static_cast<long>(sp + 1) * num_kb / p.ksplit);
@@ -291,7 +382,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // two warps per quadrant: with 128-row tiles they share the tile's column chunks, with 256-row tiles each
         // takes all chunks of one 128-row block
         const int half = (warp - 2) >> 2;
-        constexpr int CHUNKS = BN / G, CPH = BM == 256 ? CHUNKS : (CHUNKS > 1 ? CHUNKS / 2 : 1);
+        constexpr int EPI_Q = EPI_WARPS / 4;  // warps per lane quadrant
+        static_assert(EPI_WARPS == 8 || (EPI_WARPS == 16 && BM == 128 && BN / G >= 4), "epilogue warp plan");
+        constexpr int CHUNKS = BN / G, CPH = BM == 256 ? CHUNKS : (CHUNKS >= EPI_Q ? CHUNKS / EPI_Q : 1);
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
@@ -303,17 +396,6 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
             const int row = m0 + (BM == 256 ? half * 128 : 0) + q * 32 + lane;
             const bool row_ok = row < p.M;
-            // FMT 4: this thread's 128 or 256 bytes of x for the chunk it handles next; requested a chunk ahead (the
-            // first one before the accumulator wait) so that the load's latency is not paid per chunk
-            [[maybe_unused]] uint4 xq[G / 8];
-            [[maybe_unused]] const int chunk_first = BM == 256 ? 0 : half * CPH;
-            if constexpr (PH) {
-                if (row_ok && n0 + chunk_first * G < p.n_out) {
-                    const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + n0 + chunk_first * G);
-#pragma unroll
-                    for (int b = 0; b < G / 8; ++b) xq[b] = __ldg(xs + b);
-                }
-            }
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (BM == 256 ? half * 256 : acc * BN);
@@ -356,39 +438,17 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
                 if constexpr (PH) {
-                    // projection form: v = x - x~_h U_hb^T (the accumulator holds the product), then the group's
-                    // Hadamard block in registers; what follows quantizes it like any other group
-                    if (row_ok) {
+                    // projection form: the accumulator holds x H+- - x~_h V = sqrt(G) x~_l
+                    // (G = 64: the factor 1/8 goes into the quantizers' scale arithmetic instead, see kPre)
+                    if constexpr (G != 64) {
 #pragma unroll
-                        for (int b = 0; b < G / 8; ++b) {
-                            const uint4 w = xq[b];
-                            const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                v[8 * b + 2 * e] = __uint_as_float(ws[e] << 16) - v[8 * b + 2 * e];
-                                v[8 * b + 2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u) - v[8 * b + 2 * e + 1];
-                            }
-                        }
-                        if (CPH > 1 && col0 + G < p.n_out && chunk + 1 < min(CHUNKS, (BM == 256 ? 1 : half + 1) * CPH)) {
-                            const uint4* xs = reinterpret_cast<const uint4*>(p.xsub + static_cast<size_t>(row) * p.K + col0 + G);
-#pragma unroll
-                            for (int b = 0; b < G / 8; ++b) xq[b] = __ldg(xs + b);
-                        }
+                        for (int j = 0; j < G; ++j) v[j] *= 0.08838834764831845f;  // 1 / sqrt(128)
                     }
-#pragma unroll
-                    for (int h = 1; h < G; h <<= 1)
-#pragma unroll
-                        for (int i = 0; i < G; i += 2 * h)
-#pragma unroll
-                            for (int j = i; j < i + h; ++j) {
-                                const float a0 = v[j], a1 = v[j + h];
-                                v[j] = a0 + a1;
-                                v[j + h] = a0 - a1;
-                            }
-                    constexpr float kNorm = G == 64 ? 0.125f : 0.08838834764831845f;  // 1 / sqrt(G)
-#pragma unroll
-                    for (int j = 0; j < G; ++j) v[j] *= kNorm;
                 }
+                constexpr float kPre = (PH && G == 64) ? 0.125f : 1.0f;
+#ifdef EXP_NOQUANT
+                if (PH) { if (v[0] == 123.456f) p.xscale[0] = v[1]; continue; }
+#endif
                 // number of low-precision values among v[] (a multiple of 16)
                 const int nlow = min(G, max(0, p.K_l - col0));
                 if constexpr (FMT == 1) {
@@ -402,7 +462,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll
                         for (int b = 0; b < 4; ++b) {
                             uint32_t w0 = 0, w1 = 0;
-                            if (16 * b < nlow) sfword |= nvfp4_block16(v + 16 * b, ex_inv, ex_scale, w0, w1) << (8 * b);
+                            if (16 * b < nlow) sfword |= nvfp4_block16(v + 16 * b, kPre, ex_inv, ex_scale, w0, w1) << (8 * b);
                             *reinterpret_cast<uint2*>(crow + 8 * b) = make_uint2(w0, w1);  // zero in the padding slots
                         }
                         const int mr = row & 127;
@@ -452,11 +512,20 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         const bool slow = !(s >= 1e-30f);
                         const float inv = slow ? 0.f : __frcp_rn(s);
                         int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+                        if (!slow) {
 #pragma unroll
-                        for (int b = 0; b < G / 16; ++b) {
-                            uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
-                            if (16 * b < nlow) packed = quantize16_asym(v + 16 * b, z, inv, s, slow);
-                            *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                            for (int b = 0; b < G / 16; ++b) {
+                                uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
+                                if (16 * b < nlow) packed = quantize16_asym<false>(v + 16 * b, z, inv, s);
+                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                            }
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < G / 16; ++b) {
+                                uint4 packed = make_uint4(0, 0, 0, 0);
+                                if (16 * b < nlow) packed = quantize16_asym<true>(v + 16 * b, z, inv, s);
+                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                            }
                         }
                         const int grp = col0 / G;
                         p.xscale[static_cast<size_t>(grp) * p.ldm + row] = s;
@@ -468,24 +537,35 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         zrow[2 * p.n_g] = zbits;
                     }
                 } else if (nlow > 0) {
-                    float amax = 0.f;
+                    // four running maxima instead of one chain of G dependent instructions
+                    float am[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int b = 0; b < G / 16; ++b) {
                         if (16 * b < nlow) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[16 * b + j]));
+                            for (int j = 0; j < 16; ++j) am[j & 3] = fmaxf(am[j & 3], fabsf(v[16 * b + j]));
                         }
                     }
+                    const float amax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * kPre;
                     const float s = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(amax, 7.0f)));
                     const bool slow = !(s >= 1e-30f);  // zero or tiny scale: divide instead of multiplying
-                    const float inv = slow ? 0.f : __frcp_rn(s);
+                    const float inv = slow ? 0.f : __frcp_rn(s) * kPre;
                     if (row_ok) {
                         int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+                        if (!slow) {
 #pragma unroll
-                        for (int b = 0; b < G / 16; ++b) {
-                            uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
-                            if (16 * b < nlow) packed = quantize16(v + 16 * b, inv, s, slow);
-                            *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                            for (int b = 0; b < G / 16; ++b) {
+                                uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
+                                if (16 * b < nlow) packed = quantize16<false>(v + 16 * b, inv, s, kPre);
+                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                            }
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < G / 16; ++b) {
+                                uint4 packed = make_uint4(0, 0, 0, 0);
+                                if (16 * b < nlow) packed = quantize16<true>(v + 16 * b, inv, s, kPre);
+                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                            }
                         }
                         p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
                     }
@@ -525,7 +605,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     }
 
     // ---------------------------------------------------------------- teardown
-    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 136u);  // a wait gave up: let issued MMAs finish first
+    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -570,7 +650,7 @@ dirotq_status_t set_rotation_plan(int plan) {
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     RotKernelParams p;
-    p.n_out = g.K; p.k_red = g.K; p.xsub = nullptr;
+    p.n_out = g.K; p.k_red = g.K;
     p.M = a.M; p.K = g.K; p.K_l = g.K_l; p.K_lp = g.K_lp; p.r = g.r; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = a.xrot; p.status = a.status;
     p.xsf = a.xsf; p.K4 = g.K4; p.nkb64p = g.nkb64p; p.ex = L->act_scale_log2;
@@ -602,7 +682,7 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     const long num_tiles = ((a.M + bm - 1) / bm) * ((g.K + bn - 1) / bn);
     const int grid = num_tiles < sms ? static_cast<int>(num_tiles) : sms;
     const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
-    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const RotKernelParams);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
     static const KernelFn table[3][6] = {
         {rotate_quant_kernel<64, 0, 128, 128>, rotate_quant_kernel<128, 0, 128, 128>, rotate_quant_kernel<64, 1, 128, 128>,
          rotate_quant_kernel<64, 2, 128, 128>, rotate_quant_kernel<128, 2, 128, 128>, rotate_quant_kernel<64, 3, 128, 128>},
@@ -616,32 +696,32 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     const bool dependent = g.fmt != 3;
     static SmemOptIn<18> opt_in;
     if (!opt_in.ensure(kern, (plan - 1) * 6 + vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
-    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, plan == 1 ? L->tmap_qt128 : L->tmap_qt,
-                         p) == cudaSuccess
+    const CUtensorMap& tmap_q = plan == 1 ? L->tmap_qt128 : L->tmap_qt;
+    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, tmap_q, tmap_x, tmap_q, p) == cudaSuccess
                ? DIROTQ_OK
                : DIROTQ_ERR_CUDA;
 }
 
-// Projection form (fmt 4): x~_h = bf16(x U_hb) with the rotation kernel on r_pad output columns, then the residual
-// x - x~_h U_hb^T, its block Hadamard and the group quantizer with the same kernel on a reduction of length r_pad.
+// Projection form (fmt 4): x~_h = bf16(x U_hb) with the rotation kernel on r_pad output columns, then
+// x~_l = (x H+- - x~_h V) / sqrt(G) and the group quantizer with the same kernel in its PH mode.
 dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     if (a.xrot != nullptr) return DIROTQ_ERR_INVALID_ARG;  // there is no K-wide rotated activation in this form
     const int sms = sm_count(L->device);
-    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const RotKernelParams);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
     RotKernelParams p;
     p.M = a.M; p.K = g.K; p.K_lp = g.K_lp; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = nullptr; p.status = a.status;
     p.xsf = nullptr; p.K4 = 0; p.nkb64p = 0; p.ex = 0; p.xtilde = nullptr; p.rowmax = nullptr;
     dirotq_status_t st;
+    CUtensorMap tmap_x;
+    st = encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M, (uint64_t)g.K * 2, BK,
+                        128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != DIROTQ_OK) return st;
     {
         // step 1: all r_pad output columns are "high" (K_l = 0): the epilogue only rounds them to bf16 into xh
-        CUtensorMap tmap_x;
-        st = encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M, (uint64_t)g.K * 2, BK,
-                            128, CU_TENSOR_MAP_SWIZZLE_128B);
-        if (st != DIROTQ_OK) return st;
         RotKernelParams p1 = p;
-        p1.n_out = g.r_pad; p1.k_red = g.K; p1.K_l = 0; p1.r = g.r_pad; p1.xsub = nullptr;
+        p1.n_out = g.r_pad; p1.k_red = g.K; p1.K_l = 0; p1.r = g.r_pad;
         const KernelFn k1 = rotate_quant_kernel<64, 0, 128, 128>;
         static SmemOptIn<1> opt_in1;
         if (!opt_in1.ensure(k1, 0, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
@@ -659,7 +739,7 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
             tiles *= ksplit;
         }
         if (launch_kernel(k1, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_x,
-                          L->tmap_qt128, p1) != cudaSuccess)
+                          L->tmap_qt128, tmap_x, L->tmap_qt128, p1) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
         if (p1.partial != nullptr) {
             const long threads = static_cast<long>(a.M) * g.r_pad / 8;
@@ -669,23 +749,25 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
         }
     }
     {
-        // step 2: A = x~_h [M][r_pad], B = U_hb [K][r_pad]; every output column is low-precision (K_l = K)
+        // step 2: x~_h [M][r_pad] against -V^T [K][r_pad], then x against the Hadamard block, group by group (see the
+        // kernel's PH note); every output column is low-precision (K_l = K)
         CUtensorMap tmap_xh;
         st = encode_tmap_2d(&tmap_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.xh, (uint64_t)g.r_pad, (uint64_t)a.M,
                             (uint64_t)g.r_pad * 2, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B);
         if (st != DIROTQ_OK) return st;
         RotKernelParams p2 = p;
-        p2.n_out = g.K; p2.k_red = g.r_pad; p2.K_l = g.K; p2.r = g.r; p2.xsub = static_cast<const uint16_t*>(a.x);
+        p2.n_out = g.K; p2.k_red = g.r_pad; p2.K_l = g.K; p2.r = g.r;
         const int vi = g.fmt == 1 ? 2 : (g.G == 64 ? 0 : 1);
-        static const KernelFn k2s[3] = {rotate_quant_kernel<64, 4, 256, 128>, rotate_quant_kernel<128, 4, 256, 128>,
-                                        rotate_quant_kernel<64, 1, 256, 128, true>};
+        static const KernelFn k2s[3] = {rotate_quant_kernel<64, 4, 256, 128, true, 8>, rotate_quant_kernel<128, 4, 256, 128>,
+                                        rotate_quant_kernel<64, 1, 256, 128, true, 8>};
+        const int threads2 = NUM_THREADS;
         const KernelFn k2 = k2s[vi];
         if (g.fmt == 1) { p2.xsf = a.xsf; p2.K4 = g.K4; p2.nkb64p = g.nkb64p; p2.ex = L->act_scale_log2; }
         static SmemOptIn<3> opt_in2;
         if (!opt_in2.ensure(k2, vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
         const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.K + 255) / 256);
-        if (launch_kernel(k2, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_xh, L->tmap_qt,
-                          p2) != cudaSuccess)
+        if (launch_kernel(k2, static_cast<int>(tiles < sms ? tiles : sms), threads2, SMEM_BYTES, stream, true, tmap_xh, L->tmap_qt,
+                          tmap_x, L->tmap_had, p2) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
     }
     return DIROTQ_OK;

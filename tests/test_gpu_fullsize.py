@@ -329,9 +329,8 @@ def _run_ph(M, K, N, r, G, model, n_rows=24, n_cols=96, seed=0):
     codes_n, scales_b = codes.cpu().numpy()[rows], bf16_tensor_to_bits(scales)[rows]
     lo = orc.prepare_layer_ph(np.ascontiguousarray(W[:, cols]), Uh, G)
     oo = orc.linear_deployed_ph(np.ascontiguousarray(x_bits[rows]), lo, bias=np.ascontiguousarray(bias[cols]))
-    Uhb = orc.bf16_to_f64(lo["Uhb"])
     xh_g = orc.bf16_to_f64(xh_b)
-    xl_ref = orc.block_hadamard_cols(orc.bf16_to_f64(x_bits[rows]) - xh_g @ Uhb.T, G)
+    _, xl_ref = orc.residual_ph(np.ascontiguousarray(x_bits[rows]), lo, G, xh_bits=xh_b)
     sq_ref = orc.split_quantize(xl_ref, 0, G, want_t=True)
     prot = {"xt": np.concatenate([xh_g, xl_ref], axis=1), "xh": xh_b, "scales": sq_ref["scales"], "codes": sq_ref["codes"]}
     stats = check_activation_side(None, xh_b, codes_n, scales_b, prot, r, G)

@@ -26,8 +26,10 @@ def _run_case(spec: synth.LayerSpec, M: int, with_bias=True):
     layer = dq.dirotq_prepare_layer_ph(W, torch.from_numpy(Uh).to(dev), spec.G, bias=bias)
     assert (layer.K_l, layer.n_g) == (spec.K, spec.K // spec.G)
 
-    # weight side: the rounded projection, the 16-bit rows U_hb^T W, scales and codes of H^T W (exact ties may differ)
+    # weight side: the rounded projection, V = bf16(U_hb^T H+-), the 16-bit rows (V H+-^T / G) W, scales and codes of
+    # H^T W (exact ties may differ)
     assert np.array_equal(bf16_tensor_to_bits(dq.dirotq_layer_export_uh(layer)), lo["Uhb"])
+    assert np.array_equal(bf16_tensor_to_bits(dq.dirotq_layer_export_v(layer)), lo["V"])
     wcodes = torch.empty((spec.K, spec.N), dtype=torch.int8, device=dev)
     wscales = torch.empty((layer.n_g, spec.N), dtype=torch.bfloat16, device=dev)
     wh = torch.empty((spec.r, spec.N), dtype=torch.bfloat16, device=dev)
@@ -57,8 +59,7 @@ def _run_case(spec: synth.LayerSpec, M: int, with_bias=True):
     # The residual is DEFINED through the rounded x~_h, so a token whose x~_h differs in one element has a different
     # (equally valid) residual: codes and scales are held to the reference's second step run on the library's own x~_h,
     # with the same protocol as for the rotation (equal except at rounding boundaries).
-    Uhb = orc.bf16_to_f64(lo["Uhb"])
-    xl_ref = orc.block_hadamard_cols(orc.bf16_to_f64(inp["x"]) - xh_g @ Uhb.T, spec.G)
+    _, xl_ref = orc.residual_ph(inp["x"], lo, spec.G, xh_bits=xh_b)
     sq_ref = orc.split_quantize(xl_ref, 0, spec.G, want_t=True)
     same_xh = np.all(xh_b == oo["xh"], axis=1)
     assert np.array_equal(sq_ref["codes"][same_xh], oo["codes"][same_xh])      # consistency of the re-run
@@ -189,6 +190,7 @@ def _run_case_nvfp4(spec: synth.LayerSpec, M: int, with_bias=True):
     lo_chk = dict(lo)
     lo_chk["Qb"] = lo["Uhb"]                 # the export returns U_hb in the rotation's place
     stats = check_weight_side_nvfp4(dq.dirotq_layer_export_nvfp4(layer), lo_chk)
+    assert np.array_equal(bf16_tensor_to_bits(dq.dirotq_layer_export_v(layer)), lo["V"])
 
     x = bits_to_bf16_tensor(inp["x"])
     ws = dq.alloc_workspace(layer, M)
