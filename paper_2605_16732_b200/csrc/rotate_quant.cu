@@ -296,8 +296,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                     continue;
                 }
-                const int kb_end = static_cast<int>(static_cast<long>(sp + 1) * num_kb / p.ksplit);
-                for (int kb = static_cast<int>(static_cast<long>(sp) * num_kb / p.ksplit); kb < kb_end; ++kb, ++it) {
+                // a split reduction is dealt out k-block by k-block: range sp takes k-blocks sp, sp + ksplit, ... (measured the
+                // same as contiguous ranges)
+                for (int kb = sp; kb < num_kb; kb += p.ksplit, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
@@ -355,9 +356,8 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     continue;
                 }
                 const int sp = tile / num_mn;
-                const int kb_begin = static_cast<int>(static_cast<long>(sp) * num_kb / p.ksplit);
-                const int kb_end = static_cast<int>(static_cast<long>(sp + 1) * num_kb / p.ksplit);
-                for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+                const int kb_begin = sp;
+                for (int kb = kb_begin; kb < num_kb; kb += p.ksplit, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
@@ -446,9 +446,6 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
                 constexpr float kPre = (PH && G == 64) ? 0.125f : 1.0f;
-#ifdef EXP_NOQUANT
-                if (PH) { if (v[0] == 123.456f) p.xscale[0] = v[1]; continue; }
-#endif
                 // number of low-precision values among v[] (a multiple of 16)
                 const int nlow = min(G, max(0, p.K_l - col0));
                 if constexpr (FMT == 1) {
