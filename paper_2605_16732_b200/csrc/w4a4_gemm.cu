@@ -16,9 +16,10 @@
 //     that) in the 128-byte-swizzled layout the MMA reads;
 //   * every product is an integer times 2^-18 and a group's sum is below 2^24 in magnitude, so the fp32
 //     accumulator holds S_g = 2^-18 P_g without rounding.  The weight scales are stored as 2^18 s_w (exact), so
-//         t = S_g * s_x                   -- one rounding, that of the product s_x P_g itself --
-//         acc = fma(t, 2^18 s_w, acc)
-//     folds a group in with one multiply and one fused multiply-add per element and no integer conversion.
+//         t = s_x * (2^18 s_w)            -- exact: two bf16-valued factors and a power of two --
+//         acc = fma(S_g, t, acc)          -- one rounding per element and group --
+//     folds a group in with one (packed, two columns at a time) multiply and one fused multiply-add per element and
+//     no integer conversion.
 // The exactness of the accumulation is a property of the tensor core that the parity tests pin: the
 // group sums exported by the debug entry equal the CPU checker's int32 sums bit for bit, on random
 // codes and on patterns built to lose low bits (long runs of +-49 followed by +-1).
@@ -451,7 +452,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     sxv[i] = s_sw[2 * BN + gi * BM + q * 32 + lr4 + 8 * i] * (kI8Path ? 1.0f / kWScaleFold : 1.0f);
-                const float4* swp = reinterpret_cast<const float4*>(s_sw + gi * BN + half * HB + 4 * lc2);
+                uint64_t sx2[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sx2[i] = pack_f32x2(sxv[i], sxv[i]);
+                const ulonglong2* swp = reinterpret_cast<const ulonglong2*>(s_sw + gi * BN + half * HB + 4 * lc2);
                 // what comes after this tile: the next group's, or the rank-r tile
                 const uint32_t nb = b + 1 == NBUF ? 0 : b + 1, nbph = b + 1 == NBUF ? bph ^ 1 : bph;
                 const uint32_t nslot = slot + 1 == SC_SLOTS ? 0 : slot + 1, nsph = slot + 1 == SC_SLOTS ? sph ^ 1 : sph;
@@ -460,12 +464,12 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
                     uint32_t (&cur)[32] = raw[c & 1];
-                    // this chunk's weight scales: requested before the wait so that their latency hides behind it
-                    float w[8];
+                    // this chunk's weight scales, two adjacent columns per 64-bit register: requested before the wait so
+                    // that their latency hides behind it
+                    uint64_t w2[4];
                     if constexpr (!kPartials) {
-                        const float4 wa = swp[c * 8], wb = swp[c * 8 + 1];
-                        w[0] = wa.x; w[1] = wa.y; w[2] = wa.z; w[3] = wa.w;
-                        w[4] = wb.x; w[5] = wb.y; w[6] = wb.z; w[7] = wb.w;
+                        const ulonglong2 wa = swp[c * 8], wb = swp[c * 8 + 1];
+                        w2[0] = wa.x; w2[1] = wa.y; w2[2] = wb.x; w2[3] = wb.y;
                     }
                     tmem_ld_wait();  // waits for every outstanding load, hence a look-ahead of one chunk
                     tmem_ld_fence(cur);
@@ -499,19 +503,11 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                                   __float2int_rn(__uint_as_float(cur[pidx + 1]) * kAccUnit));
                             }
                     } else {
-                        // t = S s_x for two adjacent columns at a time (one packed multiply: half the issue slots of two
-                        // scalar ones), then acc = fma(t, 2^18 s_w, acc); both passes ordered so that consecutive
-                        // instructions share an operand (the token's scale in the first, the column's in the second)
-                        uint64_t t2[16];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint64_t sx2 = pack_f32x2(sxv[i], sxv[i]);
-#pragma unroll
-                            for (int cb = 0; cb < 4; ++cb) {
-                                const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
-                                t2[pidx >> 1] = mul_f32x2(pack_u32x2(cur[pidx], cur[pidx + 1]), sx2);
-                            }
-                        }
+                        // The scale of an element is t = s_x * (2^18 s_w): two bf16-valued factors (and a power of two), so
+                        // the fp32 product is EXACT.  It is formed for two adjacent columns at a time with one packed
+                        // multiply whose operands are 64-bit registers as they come (the pair of column scales straight
+                        // from a shared-memory load, the token's scale duplicated once per group), so no register moves
+                        // are spent on packing; then acc = fma(S, t, acc): one rounding per element and group.
 #pragma unroll
                         for (int cb = 0; cb < 4; ++cb)
 #pragma unroll
@@ -519,9 +515,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                 const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
                                 const int a = ((c * 4 + cb) * 4 + i) * 2;
                                 float t_lo, t_hi;
-                                unpack_f32x2(t2[pidx >> 1], t_lo, t_hi);
-                                accf[a] = fmaf(t_lo, w[2 * cb], accf[a]);
-                                accf[a + 1] = fmaf(t_hi, w[2 * cb + 1], accf[a + 1]);
+                                unpack_f32x2(mul_f32x2(w2[cb], sx2[i]), t_lo, t_hi);
+                                accf[a] = fmaf(__uint_as_float(cur[pidx]), t_lo, accf[a]);
+                                accf[a + 1] = fmaf(__uint_as_float(cur[pidx + 1]), t_hi, accf[a + 1]);
                             }
                     }
                 }
