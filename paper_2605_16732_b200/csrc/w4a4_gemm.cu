@@ -443,9 +443,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             const int n0 = (tile / num_m_blocks) * BN;
             const int rbase = m0 + q * 32 + lr4;  // this thread's rows: rbase + 8 i, i = 0..3
             const int colbase = n0 + half * HB;
-            __align__(8) float accf[HB];  // [(block of 8 columns) * 4 + row i] * 2 + {0, 1}
+            uint64_t acc2[HB / 2];  // two adjacent columns per 64-bit register: [(block of 8 columns) * 4 + row i]
 #pragma unroll
-            for (int j = 0; j < HB; ++j) accf[j] = 0.f;
+            for (int j = 0; j < HB / 2; ++j) acc2[j] = 0ull;
 
             // first scales and first accumulator tile of this output tile
             ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc) &&
@@ -518,17 +518,16 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         // the fp32 product is EXACT.  It is formed for two adjacent columns at a time with one packed
                         // multiply whose operands are 64-bit registers as they come (the pair of column scales straight
                         // from a shared-memory load, the token's scale duplicated once per group), so no register moves
-                        // are spent on packing; then acc = fma(S, t, acc): one rounding per element and group.
+                        // are spent on packing; then acc = fma(S, t, acc), again packed (the accumulator's two adjacent
+                        // columns are consecutive registers of the tensor-memory load): one rounding per element and group,
+                        // two instructions per two elements.
 #pragma unroll
                         for (int cb = 0; cb < 4; ++cb)
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
-                                const int a = ((c * 4 + cb) * 4 + i) * 2;
-                                float t_lo, t_hi;
-                                unpack_f32x2(mul_f32x2(w2[cb], sx2[i]), t_lo, t_hi);
-                                accf[a] = fmaf(__uint_as_float(cur[pidx]), t_lo, accf[a]);
-                                accf[a + 1] = fmaf(__uint_as_float(cur[pidx + 1]), t_hi, accf[a + 1]);
+                                const int a = (c * 4 + cb) * 4 + i;
+                                acc2[a] = fma_f32x2(pack_u32x2(cur[pidx], cur[pidx + 1]), mul_f32x2(w2[cb], sx2[i]), acc2[a]);
                             }
                     }
                 }
@@ -562,9 +561,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
                     for (int cb = 0; cb < 4; ++cb) {
                         const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
-                        const int a = ((c * 4 + cb) * 4 + i) * 2;
-                        accf[a] += __uint_as_float(cur[pidx]);
-                        accf[a + 1] += __uint_as_float(cur[pidx + 1]);
+                        const int a = (c * 4 + cb) * 4 + i;
+                        acc2[a] = add_f32x2(acc2[a], pack_u32x2(cur[pidx], cur[pidx + 1]));
                     }
             }
             if (++b == NBUF) { b = 0; bph ^= 1; }
@@ -586,8 +584,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         uint32_t v[4];
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
-                            const int a = ((4 * m + t) * 4 + i) * 2;
-                            v[t] = pack_bf16x2(accf[a] + bv[t].x, accf[a + 1] + bv[t].y);
+                            float y_lo, y_hi;
+                            unpack_f32x2(acc2[(4 * m + t) * 4 + i], y_lo, y_hi);
+                            v[t] = pack_bf16x2(y_lo + bv[t].x, y_hi + bv[t].y);
                         }
                         const bool odd = (j & 1) != 0, upper = (j & 2) != 0;
                         const uint32_t r01 = __shfl_xor_sync(0xffffffffu, odd ? v[0] : v[1], 1);
