@@ -159,6 +159,25 @@ def oracle_sample_run(steps: int, rows: int = 32, cols: int = 128, seed: int = 0
             "seconds_per_step": t}
 
 
+def oracle_config1_full():
+    """The oracle on the whole PixArt attention-projection layer (M = 256, K = N = 1152, r = 32, groups of 64, PCA rotation of a
+    seeded calibration batch): nothing sampled, nothing extrapolated.  Online steps only, best of two runs."""
+    from oracle import dirotq_oracle as orc
+    from paper_2605_16732_b200 import synth
+
+    spec = synth.LayerSpec(K=1152, N=1152, r=RANK, G=GROUP, model=synth.PIXART, seed=2)
+    inp = synth.make_layer_inputs(spec, 256)
+    lo = orc.prepare_layer(inp["W"], inp["Q"], RANK, GROUP)
+    best = None
+    for _ in range(2):
+        t0 = time.perf_counter()
+        orc.linear_deployed(inp["x"], lo, bias=inp["bias"], want_t=False)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return {"workload": "pixart_attention_projection_M256_K1152_N1152_r32_g64", "seconds": best,
+            "value": 2.0 * 256 * 1152 * 1152 / best / 1e12, "unit": "TOPS", "cores": orc.num_threads()}
+
+
 def _suffix(fmt):
     return {"nvfp4": "_nvfp4", "int4_asym": "_asym", "w4a8": "_w4a8", "int4_ph": "_projection_form",
             "nvfp4_ph": "_projection_form_nvfp4"}.get(fmt, "")
@@ -512,6 +531,8 @@ def run_ours(args):
         "frac_int8_peak_effective": value / world / int8_peak,
         "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
     }
+    if not args.lite and args.fmt == "int4":
+        line["cpu_baseline"]["config1_full"] = oracle_config1_full()  # a whole layer, not a sample (a fraction of a second)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
