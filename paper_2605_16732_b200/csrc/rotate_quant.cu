@@ -272,7 +272,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int mn = tile % num_mn, sp = tile / num_mn;
+                const int mn = PH ? num_mn - 1 - tile : tile % num_mn, sp = tile / num_mn;
                 const int m0 = (mn % num_m_blocks) * BM;
                 const int n0 = (mn / num_m_blocks) * BN;
                 if constexpr (PH) {
@@ -332,7 +332,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 const uint32_t d = tmem_base + acc * BN;
                 if constexpr (PH) {
                     constexpr uint32_t idesc_g = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM_MMA, G);
-                    const int n0 = ((tile % num_mn) / num_m_blocks) * BN;
+                    const int n0 = ((num_mn - 1 - tile) / num_m_blocks) * BN;
                     const int nv = num_kb, nx = min(BN, p.n_out - n0) / BK;
                     for (int i = 0; i < nv + nx; ++i, ++it) {
                         const int s = it % STAGES;
@@ -388,7 +388,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-            const int mn = tile % num_mn;
+            // PH: the tiles are walked from the last columns to the first, i.e. starting with the part of x that the step
+            // before this one read last and that is most likely still in L2
+            const int mn = PH ? num_mn - 1 - tile : tile % num_mn;
             const int m0 = (mn % num_m_blocks) * BM;
             const int n_blk = mn / num_m_blocks;
             const int n0 = n_blk * BN;
