@@ -323,6 +323,28 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
+// The same launch as clusters of two CTAs (`grid` must be even).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_pairs(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, bool dependent,
+                                       Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    const bool pdl = dependent && dependent_launch_enabled();
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 // Raising a kernel's dynamic shared-memory limit (cudaFuncSetAttribute) applies to the CURRENT device only, so what has been
 // done is remembered per device: one table of flags per launch site, indexed by device and kernel variant.  Safe to
 // call from several host threads (the attribute call is idempotent; the flag only saves repeating it).

@@ -195,7 +195,13 @@ __device__ __forceinline__ uint32_t nvfp4_block16(const float* v, float pre, flo
 // EPI_WARPS: 8, or 16 for the PH mode with groups of 64 (four warps per lane quadrant, one 64-column chunk each): that
 // mode has no long main loop to hide the epilogue under, and its epilogue is a chain of dependent instructions per
 // thread that only more warps per scheduler speed up.
-template <int G, int FMT, int BN, int BM, bool PH = (FMT == 4), int EPI_WARPS = 8>
+// PAIR: launched as clusters of two CTAs that share every MMA (tcgen05.mma.cta_group::2, M = 256): a pair owns 256
+// token rows x BN columns, each CTA loads its own 128 rows of x and HALF of the rotation tile (BN / 2 rows of Q^T), so a
+// third fewer operand bytes travel from L2 per flop than with 128 x 256 tiles, and both accumulator buffers stay free
+// for overlapping the epilogue (which the single-CTA 256 x 256 plan gives up).  The even CTA (rank 0) issues the MMAs
+// and owns the "stage full" and "accumulator drained" barriers both CTAs' loads and epilogue warps report to; completion
+// of the MMAs is signalled to both CTAs' "stage empty" / "accumulator full" barriers.
+template <int G, int FMT, int BN, int BM, bool PH = (FMT == 4), int EPI_WARPS = 8, bool PAIR = false>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
                     const __grid_constant__ CUtensorMap tmap_x2, const __grid_constant__ CUtensorMap tmap_had,
@@ -209,8 +215,10 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // where a tile's main loop is long and there are many tiles per SM.
     static_assert(BM == 128 || (BM == 256 && BN == 256), "256-row tiles are 256 columns wide");
     constexpr int A_BYTES = BM * BK * 2;
-    constexpr int STAGES = BM == 256 ? 3 : (BN == 256 ? STAGES_WIDE : 6);
-    constexpr int STAGE_BYTES = A_BYTES + BN * BK * 2;
+    static_assert(!PAIR || (BM == 128 && BN == 256 && !PH), "pairs: 128 rows per CTA, 256 columns per pair");
+    constexpr int B_ROWS = PAIR ? BN / 2 : BN;  // rows of the rotation tile this CTA holds
+    constexpr int STAGES = BM == 256 ? 3 : (B_ROWS == 256 ? STAGES_WIDE : 6);
+    constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;
     constexpr int ACC_BUFS = BM == 256 ? 1 : 2;
     static_assert(STAGES * STAGE_BYTES == STAGES_WIDE * STAGE_BYTES_WIDE && STAGE_BYTES % 1024 == 0, "ring layout");
     const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
@@ -228,7 +236,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    const int num_m_blocks = (p.M + BM - 1) / BM;
+    const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
+    constexpr int TILE_ROWS = PAIR ? 2 * BM : BM;  // token rows of a tile (of the pair's tile)
+    const int tile_first = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+    const int num_m_blocks = (p.M + TILE_ROWS - 1) / TILE_ROWS;
     const int num_n_blocks = (p.n_out + BN - 1) / BN;
     const int num_mn = num_m_blocks * num_n_blocks;
     const int num_tiles = num_mn * p.ksplit;
@@ -241,7 +253,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), EPI_WARPS * 32);  // every thread of the epilogue warps arrives
+            mbar_init(tempty_bar(a), EPI_WARPS * 32 * (PAIR ? 2 : 1));  // every thread of the epilogue warps (of both CTAs) arrives
         }
         mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
@@ -254,11 +266,17 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
-        tmem_relinquish();
+        if constexpr (PAIR) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+            tmem_relinquish();
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     grid_dependency_wait();
@@ -271,9 +289,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
                 const int mn = PH ? num_mn - 1 - tile : tile % num_mn, sp = tile / num_mn;
-                const int m0 = (mn % num_m_blocks) * BM;
+                const int m0 = (mn % num_m_blocks) * TILE_ROWS + static_cast<int>(cta_rank) * BM * (PAIR ? 1 : 0);
                 const int n0 = (mn / num_m_blocks) * BN;
                 if constexpr (PH) {
                     const int nv = num_kb;                            // k-blocks of the projection term
@@ -302,13 +320,25 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(s), A_BYTES + BN * BK * 2);
                     const uint32_t sa = smem_base + s * STAGE_BYTES;
-                    tma_load_2d(sa, &tmap_x, full_bar(s), kb * BK, m0);
-                    tma_load_2d(sa + A_BYTES, &tmap_qt, full_bar(s), kb * BK, n0);
+                    if constexpr (PAIR) {
+                        // both CTAs' bytes are counted on the leader's barrier, which expects the sum
+                        const uint32_t full_leader = map_to_cta(full_bar(s), 0);
+                        if (cta_rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+                        tma_load_2d_pair(sa, &tmap_x, full_leader, kb * BK, m0);
+                        tma_load_2d_pair(sa + A_BYTES, &tmap_qt, full_leader, kb * BK, n0 + static_cast<int>(cta_rank) * B_ROWS);
+                    } else {
+                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BN * BK * 2);
+                        tma_load_2d(sa, &tmap_x, full_bar(s), kb * BK, m0);
+                        tma_load_2d(sa + A_BYTES, &tmap_qt, full_bar(s), kb * BK, n0);
+                    }
                 }
             }
-            if (!ok) {
+            if (!ok && PAIR && cta_rank != 0) {
+                // this CTA's loads report to the leader's barriers: give them a fixed time instead
+                const unsigned long long t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 1000000ull) {}
+            } else if (!ok) {
                 // leave no bulk copy in flight: wait (bounded) for the loads already issued
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
                 for (uint32_t j = first; j < it; ++j) {
@@ -320,11 +350,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM_MMA, BN);
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc = umma_idesc(1 /*f32*/, 1 /*bf16*/, PAIR ? 2 * BM_MMA : BM_MMA, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step, ++tcount) {
                 const uint32_t acc = tcount % ACC_BUFS;
                 const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
                 if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
@@ -367,13 +397,21 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
-                        umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
-                        if constexpr (BM == 256)  // token rows 128..255: next 16 KB of the x tile, columns 256..511 of TMEM
-                            umma_bf16(d + 256, adesc + (A_BYTES_128 >> 4) + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
+                        if constexpr (PAIR) {
+                            umma_bf16_pair(d, adesc + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
+                        } else {
+                            umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
+                            if constexpr (BM == 256)  // token rows 128..255: next 16 KB of the x tile, columns 256..511 of TMEM
+                                umma_bf16(d + 256, adesc + (A_BYTES_128 >> 4) + 2 * k, bdesc + 2 * k, idesc, kb != kb_begin || k != 0);
+                        }
                     }
-                    umma_commit(empty_bar(s));
+                    if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);  // both CTAs' producers may refill the stage
+                    else umma_commit(empty_bar(s));
                 }
-                if (ok) umma_commit(tfull_bar(acc));
+                if (ok) {
+                    if constexpr (PAIR) umma_commit_pair(tfull_bar(acc), 3);  // both CTAs' epilogue warps
+                    else umma_commit(tfull_bar(acc));
+                }
             }
         }
     } else {
@@ -387,11 +425,11 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         constexpr int CHUNKS = BN / G, CPH = BM == 256 ? CHUNKS : (CHUNKS >= EPI_Q ? CHUNKS / EPI_Q : 1);
         uint32_t tcount = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+        for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step, ++tcount) {
             // PH: the tiles are walked from the last columns to the first, i.e. starting with the part of x that the step
             // before this one read last and that is most likely still in L2
             const int mn = PH ? num_mn - 1 - tile : tile % num_mn;
-            const int m0 = (mn % num_m_blocks) * BM;
+            const int m0 = (mn % num_m_blocks) * TILE_ROWS + static_cast<int>(cta_rank) * BM * (PAIR ? 1 : 0);
             const int n_blk = mn / num_m_blocks;
             const int n0 = n_blk * BN;
             const uint32_t acc = tcount % ACC_BUFS;
@@ -591,7 +629,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             }
             // release the accumulator: every tcgen05.ld of this warp has completed
             tc_fence_before_sync();
-            mbar_arrive(tempty_bar(acc));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
+            // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
+            if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
+            else mbar_arrive(tempty_bar(acc));
             // zero padding of the bf16 rank-r operand (written once, by the tile that holds column K-1)
             if (!PH && n_blk == num_n_blocks - 1 && row_ok && (BM == 256 || half == 0)) {
                 for (int c = p.r; c < p.r_pad0; c += 8)
@@ -604,12 +644,26 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     }
 
     // ---------------------------------------------------------------- teardown
-    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
+    if constexpr (PAIR) {
+        if (warp == 1 && lane == 0 && cta_rank == 0 && *abort_flag != 0) {  // a wait gave up: let issued MMAs finish first
+            umma_commit_pair(bar_base + 200u, 1);
+            const unsigned long long t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar_base + 200u, 0) && globaltimer_ns() - t0 < 100000000ull) {}
+        }
+        tc_fence_before_sync();
+        cluster_sync_all();  // neither CTA leaves while the other may still read its operands or signal its barriers
+        if (warp == 1) {
+            tc_fence_after_sync();
+            tmem_dealloc_pair(tmem_base, 512);
+        }
+    } else {
+        if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
+        tc_fence_before_sync();
+        __syncthreads();
+        if (warp == 1) {
+            tc_fence_after_sync();
+            tmem_dealloc(tmem_base, 512);
+        }
     }
 }
 
@@ -641,7 +695,7 @@ static std::atomic<int> g_rotation_plan{0};  // 0: chosen per call; 1: 128 x 128
 void set_first_step_split(bool on) { g_first_step_split.store(on ? 1 : 0); }
 
 dirotq_status_t set_rotation_plan(int plan) {
-    if (plan < 0 || plan > 3) return DIROTQ_ERR_INVALID_ARG;
+    if (plan < 0 || plan > 4) return DIROTQ_ERR_INVALID_ARG;
     g_rotation_plan.store(plan);
     return DIROTQ_OK;
 }
@@ -672,6 +726,27 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         if (mb128 * nb256 < 2 * sms) plan = 1;
         else if ((g.K >= 8192 || x_exceeds_l2) && cost256 * static_cast<double>(waves256) < 0.98 * static_cast<double>(waves128)) plan = 3;
         else plan = 2;
+    }
+    if (plan == 4) {
+        // CTA pairs: 256 rows x 256 columns per pair, 128 rows of x and half of the rotation tile per CTA
+        CUtensorMap tmap_xp;
+        dirotq_status_t stp = encode_tmap_2d(&tmap_xp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M,
+                                             (uint64_t)g.K * 2, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (stp != DIROTQ_OK) return stp;
+        const long pair_tiles = ((a.M + 255) / 256) * nb256;
+        const int pairs = static_cast<int>(pair_tiles < sms / 2 ? pair_tiles : sms / 2);
+        const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
+        using PairFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
+        static const PairFn pair_table[6] = {
+            rotate_quant_kernel<64, 0, 256, 128, false, 8, true>, rotate_quant_kernel<128, 0, 256, 128, false, 8, true>,
+            rotate_quant_kernel<64, 1, 256, 128, false, 8, true>, rotate_quant_kernel<64, 2, 256, 128, false, 8, true>,
+            rotate_quant_kernel<128, 2, 256, 128, false, 8, true>, rotate_quant_kernel<64, 3, 256, 128, false, 8, true>};
+        static SmemOptIn<6> opt_in_pair;
+        if (!opt_in_pair.ensure(pair_table[vi], vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+        return launch_kernel_pairs(pair_table[vi], 2 * pairs, NUM_THREADS, SMEM_BYTES, stream, g.fmt != 3, tmap_xp, L->tmap_qt128,
+                                   tmap_xp, L->tmap_qt128, p) == cudaSuccess
+                   ? DIROTQ_OK
+                   : DIROTQ_ERR_CUDA;
     }
     const int bm = plan == 3 ? 256 : 128, bn = plan == 1 ? 128 : 256;
     CUtensorMap tmap_x;
