@@ -182,7 +182,9 @@ DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
 /* Tuning knob of the first kernel (rotation): tile plan.  0 (default): chosen per call from M, K and the number of
  * SMs; 1: 128 tokens x 128 rotated columns; 2: 128 x 256; 3: 256 x 256 (two MMAs share one tile of the rotation: a
  * third fewer operand bytes per flop, no overlap of the epilogue; pays where a layer has many tiles per SM, e.g.
- * K = 12288 at M = 4608).  Process-wide; results do not depend on it.  Other values: DIROTQ_ERR_INVALID_ARG. */
+ * K = 12288 at M = 4608); 4: 256 x 256 per PAIR of CTAs (clusters of two: tcgen05.mma.cta_group::2, each CTA loads its
+ * own 128 rows of x and half of the rotation tile; the epilogue stays overlapped).  Process-wide; results do not depend
+ * on it.  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_rotation_tile(int plan);
 
 /* Projection form, first step (x~_h = x U_hb): with few token-row tiles (M / 128 at most half the number of SMs) and K >= 2048 the

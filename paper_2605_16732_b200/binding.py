@@ -495,7 +495,8 @@ def dirotq_set_gemm_tile(columns: int) -> None:
 
 
 def dirotq_set_rotation_tile(plan: int) -> None:
-    """Tile plan of the rotation kernel: 0 automatic, 1 = 128x128, 2 = 128x256, 3 = 256x256 (process-wide)."""
+    """Tile plan of the rotation kernel: 0 automatic, 1 = 128x128, 2 = 128x256, 3 = 256x256, 4 = 256x256 per pair of CTAs sharing
+    every MMA (process-wide)."""
     _check(lib().dirotq_set_rotation_tile(int(plan)), "dirotq_set_rotation_tile")
 
 

@@ -717,14 +717,24 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     const long mb128 = (a.M + 127) / 128, mb256 = (a.M + 255) / 256, nb256 = (g.K + 255) / 256;
     int plan = g_rotation_plan.load();
     if (plan == 0) {
+        const long nb128 = (g.K + 127) / 128;
         const long waves128 = (mb128 * nb256 + sms - 1) / sms, waves256 = (mb256 * nb256 + sms - 1) / sms;
+        const long waves_narrow = (mb128 * nb128 + sms - 1) / sms;
         const double kb = static_cast<double>(g.K / BK);
         // a 256-row tile in units of a 128-row tile; once x no longer fits the L2 beside the rotation the 128-row plan
         // re-reads it from HBM and the ratio falls to 1.9 (measured at M = 18432, K = 3072: 0.304 -> 0.288 ms)
         const bool x_exceeds_l2 = static_cast<double>(a.M) * g.K * 2.0 > 96e6;
         const double cost256 = x_exceeds_l2 ? 1.9 : 1.86 + 11.0 / kb;
-        if (mb128 * nb256 < 2 * sms) plan = 1;
+        // a 128-column tile costs about 0.62 of a 256-column one: narrow tiles when that shortens the schedule (few
+        // tiles: M = 256, K = 1152 runs on 18 instead of 10 SMs; M = 4096, K = 1152: 288 tiles in two waves instead of
+        // 160 in two), not otherwise (M = 1024, K = 3072: 96 wide tiles in one wave, 30 us, against 192 narrow ones in
+        // two, 45 us)
+        if (0.62 * static_cast<double>(waves_narrow) < static_cast<double>(waves128)) plan = 1;
         else if ((g.K >= 8192 || x_exceeds_l2) && cost256 * static_cast<double>(waves256) < 0.98 * static_cast<double>(waves128)) plan = 3;
+        // CTA pairs where there are a few waves of tiles and the main loop is not long enough for the operand traffic
+        // to hide behind the MMAs anyway (measured against 128 x 256 tiles: M = 4608, K = 3072 68.4 -> 67.3 us; M = 9216,
+        // K = 3072 122 -> 114; M = 4096, K = 4608 124 -> 111; at K = 12288 and 15360 the 256-row plan stays ahead)
+        else if (mb128 * nb256 >= 5 * sms / 2 && g.K < 8192) plan = 4;
         else plan = 2;
     }
     if (plan == 4) {

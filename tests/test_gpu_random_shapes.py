@@ -34,7 +34,7 @@ def _one(rng, big, fmt=None):
         G = 64
     tile = rng.choice([0, 0, 128, 256])
     pdl = rng.choice([True, True, False])
-    plan = rng.choice([0, 0, 1, 2, 3])     # tile plan of the rotation kernel
+    plan = rng.choice([0, 0, 1, 2, 3, 4])  # tile plan of the rotation kernel (4: CTA pairs)
     if not big and rng.random() < 0.3:
         r = 16 * rng.randint(1, max(1, K // 32))      # up to half of K in 16 bits
     bias = rng.random() < 0.7

@@ -149,7 +149,7 @@ def test_w4a8_pixart_projection_many_tiles(tile):
     print(tile, test_gpu_w4a8._run_case(spec, M=1024, check_rot=False))
 
 
-# ------------------------------------------------------------------ rotation kernel: the three tile plans
+# ------------------------------------------------------------------ rotation kernel: the tile plans (4 = CTA pairs)
 
 @pytest.fixture
 def rot_plan(request):
@@ -158,20 +158,20 @@ def rot_plan(request):
     dq.dirotq_set_rotation_tile(0)
 
 
-@pytest.mark.parametrize("rot_plan", [1, 2, 3], indirect=True)
+@pytest.mark.parametrize("rot_plan", [1, 2, 3, 4], indirect=True)
 def test_rotation_plans_int4_ragged(rot_plan):
     # M = 300: the second 128-row block of a 256-row tile is ragged; K_l = 496: ragged last group
     spec = synth.LayerSpec(K=512, N=256, r=16, G=64, model=synth.FLUX, seed=91, calib_tokens=1024)
     print(rot_plan, test_gpu_parity._run_case(spec, M=300))
 
 
-@pytest.mark.parametrize("rot_plan", [1, 2, 3], indirect=True)
+@pytest.mark.parametrize("rot_plan", [1, 2, 3, 4], indirect=True)
 def test_rotation_plans_group128_many_row_blocks(rot_plan):
     spec = synth.LayerSpec(K=768, N=128, r=128, G=128, model=synth.PIXART, seed=92, calib_tokens=1024)
     print(rot_plan, test_gpu_parity._run_case(spec, M=1100, with_bias=False))
 
 
-@pytest.mark.parametrize("rot_plan", [3], indirect=True)
+@pytest.mark.parametrize("rot_plan", [3, 4], indirect=True)
 def test_rotation_256_row_tiles_other_formats(rot_plan):
     spec = synth.LayerSpec(K=640, N=256, r=32, G=64, model=synth.FLUX, seed=93, calib_tokens=1024)
     print(test_gpu_asym._run_case(spec, M=385, shift=1.0))
@@ -190,7 +190,7 @@ def test_rotation_plans_give_the_same_codes_and_outputs():
     ws = dq.alloc_workspace(layer, M)
     outs = {}
     try:
-        for plan in (0, 1, 2, 3):
+        for plan in (0, 1, 2, 3, 4):
             dq.dirotq_set_rotation_tile(plan)
             y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
             dq.dirotq_linear(x, layer, y, ws)
@@ -198,11 +198,11 @@ def test_rotation_plans_give_the_same_codes_and_outputs():
             assert dq.dirotq_workspace_status(ws) == 0
             xh, codes, scales = dq.dirotq_workspace_export(layer, M, ws)
             outs[plan] = (y.view(torch.int16).clone(), codes.clone(), scales.view(torch.int16).clone(), xh.view(torch.int16).clone())
-        for plan in (0, 1, 3):
+        for plan in (0, 1, 3, 4):
             for a, b in zip(outs[plan], outs[2]):
                 assert torch.equal(a, b)
         with pytest.raises(dq.DirotqError):
-            dq.dirotq_set_rotation_tile(4)
+            dq.dirotq_set_rotation_tile(5)
     finally:
         dq.dirotq_set_rotation_tile(0)
     layer.close()
