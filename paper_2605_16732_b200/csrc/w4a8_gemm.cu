@@ -33,17 +33,11 @@ constexpr int NUM_UNPACK_WARPS = 4;
 constexpr int NUM_EPI_WARPS = 8;  // two per TMEM lane quadrant, half of the tile's columns each
 
 // Shared-memory plan for tiles of BN output columns (256, or 128 where wide tiles would leave SMs idle).
-// PAIR: clusters of two CTAs share every MMA (tcgen05.mma.cta_group::2, M = 256): a pair owns 256 token rows x BN columns,
-// each CTA holds its own 128 rows of activation codes and HALF of the weight tile (BN / 2 output columns: half the TMA
-// bytes, half the unpack work and half the tensor core's operand reads per CTA and flop), and each CTA's tensor memory
-// receives its 128 rows x BN columns.  Every CTA's loads complete on its own "stage full" barrier; its unpack warps then
-// report to the leader's "stage unpacked" barrier, which is what the MMA thread (rank 0 only) waits for.
-template <int BN, bool PAIR = false>
+template <int BN>
 struct Plan {
-    static constexpr int BCOLS = PAIR ? BN / 2 : BN;  // output columns whose weights this CTA holds
-    static constexpr int STAGES = BCOLS == 256 ? 4 : 6;
-    static constexpr int BU_BYTES = BCOLS * BKC;      // unpacked weight codes / bf16 W~_h chunk (32 KB for 256 columns)
-    static constexpr int BP_BYTES = BCOLS * BKC / 2;  // packed weight codes: TMA puts them into the UPPER HALF of the
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int BU_BYTES = BN * BKC;      // unpacked weight codes / bf16 W~_h chunk (32 KB at BN = 256)
+    static constexpr int BP_BYTES = BN * BKC / 2;  // packed weight codes: TMA puts them into the UPPER HALF of the
     static constexpr int BP_OFFSET = A_BYTES + BU_BYTES - BP_BYTES;  // operand buffer and the unpack expands them in place
     static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES;           // 48 KB x 4 or 32 KB x 6
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
@@ -78,17 +72,15 @@ __device__ __forceinline__ void tmem_ld_fence32(uint32_t (&v)[32]) {
                  :: "memory");
 }
 
-template <bool kPartials, int BN, bool PAIR = false>
+template <bool kPartials, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                  const A8KernelParams p) {
-    using P = Plan<BN, PAIR>;
-    static_assert(!PAIR || BN == 256, "pairs: 256 columns per pair");
+    using P = Plan<BN>;
     constexpr int STAGES = P::STAGES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES, BP_OFFSET = P::BP_OFFSET;
     constexpr int STAGE_BYTES = P::STAGE_BYTES, BAR_OFFSET = P::BAR_OFFSET, SCALE_OFFSET = P::SCALE_OFFSET;
-    constexpr int BCOLS = P::BCOLS;
-    constexpr int PIECES = BCOLS * 4 / (NUM_UNPACK_WARPS * 32);  // 16-byte pieces of the packed tile per unpack thread
+    constexpr int PIECES = BN * 4 / (NUM_UNPACK_WARPS * 32);  // 16-byte pieces of the packed tile per unpack thread
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -104,25 +96,19 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
-    constexpr int TILE_ROWS = PAIR ? 2 * BM : BM;  // token rows of a tile (of the pair's tile)
-    const int tile_first = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
-    const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
-    const int row_off = PAIR ? static_cast<int>(cta_rank) * BM : 0;        // this CTA's rows inside the tile
-    const int col_off = PAIR ? static_cast<int>(cta_rank) * BCOLS : 0;     // this CTA's share of the weight tile
-    const int num_m_blocks = (p.M + TILE_ROWS - 1) / TILE_ROWS;
+    const int num_m_blocks = (p.M + BM - 1) / BM;
     const int num_n_blocks = (p.N + BN - 1) / BN;
     const int num_tiles = num_m_blocks * num_n_blocks;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
-            mbar_init(unp_bar(s), NUM_UNPACK_WARPS * 32 * (PAIR ? 2 : 1));
+            mbar_init(unp_bar(s), NUM_UNPACK_WARPS * 32);
             mbar_init(empty_bar(s), 1);
         }
         for (int a = 0; a < NACC; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32 * (PAIR ? 2 : 1));
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
         }
         mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
@@ -133,17 +119,11 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         tma_prefetch_desc(&tmap_wh);
     }
     if (warp == 1) {
-        if constexpr (PAIR) {
-            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
-            tmem_relinquish_pair();
-        } else {
-            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
-            tmem_relinquish();
-        }
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+        tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
-    if constexpr (PAIR) cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
@@ -157,9 +137,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
-                const int m0 = (tile % num_m_blocks) * TILE_ROWS + row_off;
-                const int n0 = (tile / num_m_blocks) * BN + col_off;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m0 = (tile % num_m_blocks) * BM;
+                const int n0 = (tile / num_m_blocks) * BN;
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
@@ -185,12 +165,12 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && cta_rank == 0) {
-            constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, TILE_ROWS, BN);
-            constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, TILE_ROWS, BN);
+        if (lane == 0) {
+            constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);
+            constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step, ++tcount) {
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
                 // with narrow tiles two accumulator pairs alternate: a tile's epilogue runs under the next tile's MMAs
                 const uint32_t acc = tcount % NACC, tacc = tmem_base + acc * 2 * BN;
                 if (!mbar_wait(tempty_bar(acc), ((tcount / NACC) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
@@ -206,24 +186,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
                     if (i < p.num_kb) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            if constexpr (PAIR) umma_i8_pair(tacc, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
-                            else umma_i8(tacc, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
-                        }
+                        for (int k = 0; k < 4; ++k) umma_i8(tacc, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
                     } else {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            if constexpr (PAIR) umma_bf16_pair(tacc + BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, ((i - p.num_kb) | k) != 0);
-                            else umma_bf16(tacc + BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, ((i - p.num_kb) | k) != 0);
-                        }
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16(tacc + BN, adesc + 2 * k, bdesc + 2 * k, idesc_bf, ((i - p.num_kb) | k) != 0);
                     }
-                    if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);  // both CTAs' producers may refill the stage
-                    else umma_commit(empty_bar(s));
+                    umma_commit(empty_bar(s));
                 }
-                if (ok) {
-                    if constexpr (PAIR) umma_commit_pair(tfull_bar(acc), 3);  // both CTAs' epilogue warps
-                    else umma_commit(tfull_bar(acc));
-                }
+                if (ok) umma_commit(tfull_bar(acc));
             }
         }
     } else if (warp < 2 + NUM_UNPACK_WARPS) {
@@ -231,7 +202,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         const int u = threadIdx.x - 64;  // 0..127
         uint32_t it = 0;
         bool ok = true;
-        for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int i = 0; i < items; ++i, ++it) {
                 const int s = it % STAGES;
                 // The four unpack warps meet at a hardware barrier below, which has no time limit: they must all go on or
@@ -276,12 +247,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         *reinterpret_cast<uint4*>(d0 + j * 4096) = o0;  // 32 rows of 128 bytes further down
                         *reinterpret_cast<uint4*>(d1 + j * 4096) = o1;
                     }
-                    if constexpr (PAIR) fence_proxy_async_all();
-                    else fence_proxy_async_smem();
+                    fence_proxy_async_smem();
                 }
-                // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
-                if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(unp_bar(s), 0));  // this CTA's stage has landed and is unpacked
-                else mbar_arrive(unp_bar(s));
+                mbar_arrive(unp_bar(s));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             }
         }
     } else {
@@ -291,8 +259,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         constexpr int CPH = BN / 32 / 2;  // 32-column chunks per warp
         uint32_t tcount = 0;
         bool ok = true;
-        for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step, ++tcount) {
-            const int m0 = (tile % num_m_blocks) * TILE_ROWS + row_off;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
             // This tile's column scales and bias go to shared memory while the MMAs are still running (two buffers: a warp
             // can be one tile ahead of the others).  The reducing barrier orders these stores before the reads below and
@@ -341,8 +309,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 tmem_ld_fence32(lr);
                 if (c == (half + 1) * CPH - 1) {
                     tc_fence_before_sync();
-                    if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc_i), 0));  // the leader's barrier
-                    else mbar_arrive(tempty_bar(acc_i));
+                    mbar_arrive(tempty_bar(acc_i));
                 }
                 const int col = n0 + c * 32;
                 if (row < p.M) {
@@ -382,30 +349,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         }
     }
 
-    if constexpr (PAIR) {
-        if (warp == 1 && lane == 0 && cta_rank == 0 && *abort_flag != 0) {  // a wait gave up: let issued MMAs finish first
-            umma_commit_pair(bar_base + 200u, 1);
-            const unsigned long long t0 = globaltimer_ns();
-            while (!mbar_try_wait(bar_base + 200u, 0) && globaltimer_ns() - t0 < 100000000ull) {}
-        }
-        tc_fence_before_sync();
-        cluster_sync_all();  // neither CTA leaves while the other may still read its operands or signal its barriers
-        if (warp == 1) {
-            tc_fence_after_sync();
-            tmem_dealloc_pair(tmem_base, 512);
-        }
-    } else {
-        if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
-        tc_fence_before_sync();
-        __syncthreads();
-        if (warp == 1) {
-            tc_fence_after_sync();
-            tmem_dealloc(tmem_base, 512);
-        }
+    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
-template <int BN, bool PAIR = false>
+template <int BN>
 static dirotq_status_t launch_w4a8_gemm_bn(const dirotq_layer* L, const A8GemmArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     CUtensorMap tmap_codes, tmap_xh;
@@ -424,24 +377,16 @@ static dirotq_status_t launch_w4a8_gemm_bn(const dirotq_layer* L, const A8GemmAr
     p.wscale = reinterpret_cast<const float*>(L->blob + L->lay.off_wscale);
     p.bias = reinterpret_cast<const float*>(L->blob + L->lay.off_bias);
     p.y = a.y; p.partials = a.partials; p.status = a.status;
+    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
     const bool dbg = a.partials != nullptr;
-    auto kern = dbg ? w4a8_gemm_kernel<true, BN, PAIR> : w4a8_gemm_kernel<false, BN, PAIR>;
-    static SmemOptIn<2> opt_in;  // one per instantiation of this launcher
-    if (!opt_in.ensure(kern, dbg ? 1 : 0, L->device, Plan<BN, PAIR>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
-    const bool narrow = BN == 128 || PAIR;  // 128 weight columns per CTA: the 128-row boxes
-    const int sms = sm_count(L->device);
-    cudaError_t err;
-    if constexpr (PAIR) {
-        const int pair_tiles = ((a.M + 2 * BM - 1) / (2 * BM)) * ((g.N + BN - 1) / BN);
-        const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
-        err = launch_kernel_pairs(kern, 2 * pairs, NUM_THREADS, Plan<BN, PAIR>::SMEM_BYTES, stream, true, tmap_codes,
-                                  L->tmap_wpacked128, tmap_xh, L->tmap_wh128, p);
-    } else {
-        const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
-        const int grid = num_tiles < sms ? num_tiles : sms;
-        err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
-                            narrow ? L->tmap_wpacked128 : L->tmap_wpacked, tmap_xh, narrow ? L->tmap_wh128 : L->tmap_wh, p);
-    }
+    auto kern = dbg ? w4a8_gemm_kernel<true, BN> : w4a8_gemm_kernel<false, BN>;
+    static SmemOptIn<2> opt_in;
+    if (!opt_in.ensure(kern, dbg ? 1 : 0, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+    const bool narrow = BN == 128;
+    const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
+                                          narrow ? L->tmap_wpacked128 : L->tmap_wpacked, tmap_xh,
+                                          narrow ? L->tmap_wh128 : L->tmap_wh, p);
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
@@ -449,8 +394,8 @@ static std::atomic<int> g_a8_tile_columns{0};  // 0: chosen per call; 128 / 256:
 
 }  // namespace
 
-dirotq_status_t set_w4a8_tile_columns(int columns) {  // 512: 256 columns per pair of CTAs
-    if (columns != 0 && columns != 128 && columns != 256 && columns != 512) return DIROTQ_ERR_INVALID_ARG;
+dirotq_status_t set_w4a8_tile_columns(int columns) {
+    if (columns != 0 && columns != 128 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
     g_a8_tile_columns.store(columns);
     return DIROTQ_OK;
 }
@@ -464,7 +409,6 @@ dirotq_status_t launch_w4a8_gemm(const dirotq_layer* L, const A8GemmArgs& a, cud
     const long t_wide = m_blocks * ((L->geo.N + 255) / 256), t_narrow = m_blocks * ((L->geo.N + 127) / 128);
     const bool narrow_pays =
         NARROW_COST * static_cast<double>((t_narrow + sms - 1) / sms) < 0.98 * static_cast<double>((t_wide + sms - 1) / sms);
-    if (forced == 512) return launch_w4a8_gemm_bn<256, true>(L, a, stream);
     const bool narrow = forced ? forced == 128 : narrow_pays;
     return narrow ? launch_w4a8_gemm_bn<128>(L, a, stream) : launch_w4a8_gemm_bn<256>(L, a, stream);
 }
