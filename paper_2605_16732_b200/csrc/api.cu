@@ -627,10 +627,10 @@ dirotq_status_t dirotq_set_dependent_launch(int enabled) {
 }
 
 dirotq_status_t dirotq_set_gemm_tile(int columns) {
-    dirotq_status_t st = set_w4a4_tile_columns(columns);
-    const int others = columns == 192 ? 0 : columns;  // the 192-column plan exists for the grouped INT4 second kernel only
-    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(others);
-    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(others);
+    // 192: a plan of the grouped INT4 second kernel only; 512: 256 columns per pair of CTAs, NVFP4 second kernel only
+    dirotq_status_t st = set_w4a4_tile_columns(columns == 512 ? 0 : columns);
+    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(columns == 192 ? 0 : columns);
+    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(columns == 192 || columns == 512 ? 0 : columns);
 }
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,

@@ -41,19 +41,27 @@ constexpr int NUM_EPI_WARPS = 8;
 // layers with few tiles.  With 256 columns one accumulator (256 of the 512 tensor-memory columns) is all that fits
 // beside the scale factors: the epilogue of a tile then does not overlap the MMAs of the next, but the producer keeps
 // filling the stages meanwhile, and the MMAs catch up on a full pipeline.
-template <int BN>
+// PAIR (BN = 256): clusters of two CTAs share every MMA (cta_group::2, M = 256): a pair owns 256 token rows x 256 columns;
+// each CTA loads its own 128 rows of activation codes with their scale atoms, ONE of the tile's two 128-column blocks of
+// weight codes, and the scale atoms of both blocks (every CTA's tensor core scales all 256 columns of its rows): 38
+// instead of 54 KB per k-block and CTA.  All loads complete on the CTA's own "stage full" barrier; the second CTA's first
+// copier thread then tells the leader (one arrival per stage on the leader's "peer landed" barrier), whose copier threads
+// issue the pair-wide scale copies and whose MMA thread issues the pair-wide MMAs.
+template <int BN, bool PAIR = false>
 struct Plan {
     static constexpr int NB = BN / 128;               // 128-column blocks per tile
-    static constexpr int STAGES = BN == 128 ? 6 : 4;
+    static constexpr int NB_DATA = PAIR ? 1 : NB;     // ... whose weight codes this CTA holds
+    static constexpr int STAGES = PAIR ? 5 : (BN == 128 ? 6 : 4);
     static constexpr int ACC_BUFS = BN == 128 ? 2 : 1;
-    static constexpr int B_BYTES = BN * 128;          // 16 / 32 KB
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + (1 + NB) * SF_BYTES;  // 36 / 54 KB
+    static constexpr int B_BYTES = NB_DATA * 128 * 128;  // 16 / 32 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + (1 + NB) * SF_BYTES;  // 36 / 54 KB (pairs: 38 KB)
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int BIAS_OFFSET = BAR_OFFSET + 256;  // two buffers of a tile's bias values
     static constexpr int SMEM_BYTES = BIAS_OFFSET + 2 * BN * 4 + 1024;
     static constexpr int TMEM_SF_BASE = ACC_BUFS * BN;    // columns 256.. hold the scale factors
     static constexpr int SF_COLS = 16 * (1 + NB);         // per stage: 16 columns for the tokens, 16 per 128 output columns
     static_assert(TMEM_SF_BASE + STAGES * SF_COLS <= 512, "tensor memory plan");
+    static_assert(8 * ((PAIR ? 4 : 3) * STAGES + 4) <= 192, "barriers end below the words at +192");
     static_assert(SMEM_BYTES <= 232448, "shared memory plan");
     static_assert(STAGE_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
 };
@@ -95,6 +103,10 @@ __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
 __device__ __forceinline__ void tmem_cp_32x128b_warpx4(uint32_t taddr, uint64_t desc) {
     asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
 }
+// The same over a CTA pair: each CTA's shared memory (same offset) into its own tensor memory (same address).
+__device__ __forceinline__ void tmem_cp_32x128b_warpx4_pair(uint32_t taddr, uint64_t desc) {
+    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+}
 
 // Block-scaled instruction descriptor: E2M1 x E2M1 -> fp32, UE4M3 scales, both operands K-major.
 __host__ __device__ constexpr uint32_t nvfp4_idesc(uint32_t M, uint32_t N) {
@@ -114,13 +126,26 @@ __device__ __forceinline__ void umma_nvfp4(uint32_t d_tmem, uint64_t adesc, uint
         : "memory");
 }
 
-template <int BN>
+__device__ __forceinline__ void umma_nvfp4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t tsfa,
+                                                uint32_t tsfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+        : "memory");
+}
+
+template <int BN, bool PAIR = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wcodes,
                   const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                   const NvKernelParams p) {
-    using P = Plan<BN>;
-    constexpr int NB = P::NB, STAGES = P::STAGES, ACC_BUFS = P::ACC_BUFS, B_BYTES = P::B_BYTES;
+    using P = Plan<BN, PAIR>;
+    static_assert(!PAIR || BN == 256, "pairs: 256 columns per pair");
+    constexpr int NB = P::NB, NB_DATA = P::NB_DATA, STAGES = P::STAGES, ACC_BUFS = P::ACC_BUFS, B_BYTES = P::B_BYTES;
     constexpr int STAGE_BYTES = P::STAGE_BYTES, BAR_OFFSET = P::BAR_OFFSET, BIAS_OFFSET = P::BIAS_OFFSET;
     constexpr int TMEM_SF_BASE = P::TMEM_SF_BASE, SF_COLS = P::SF_COLS;
     extern __shared__ uint8_t smem_raw[];
@@ -132,12 +157,17 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     auto sfready_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + 4 + s); };
+    auto peer_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + 4 + s); };  // pairs, leader: the other CTA's stage has landed
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BAR_OFFSET + 192);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BAR_OFFSET + 196);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int num_m_blocks = (p.M + BM - 1) / BM;
+    const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
+    constexpr int TILE_ROWS = PAIR ? 2 * BM : BM;  // token rows of a tile (of the pair's tile)
+    const int tile_first = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+    const int num_m_blocks = (p.M + TILE_ROWS - 1) / TILE_ROWS;
     const int num_n_blocks = (p.N + BN - 1) / BN;
     const int num_tiles = num_m_blocks * num_n_blocks;
 
@@ -146,10 +176,11 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
             mbar_init(sfready_bar(s), 2);  // one arrival per copier warp
+            if constexpr (PAIR) mbar_init(peer_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
+            mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32 * (PAIR ? 2 : 1));
         }
         mbar_init(bar_base + 200u, 1);  // spare: see umma_drain
         *abort_flag = 0;
@@ -160,11 +191,17 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         tma_prefetch_desc(&tmap_wh);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
-        tmem_relinquish();
+        if constexpr (PAIR) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+            tmem_relinquish();
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
@@ -177,23 +214,29 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m_blk = tile % num_m_blocks, n_blk = tile / num_m_blocks;
+            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
+                // m_blk: this CTA's block of 128 token rows
+                const int m_blk = (tile % num_m_blocks) * (PAIR ? 2 : 1) + static_cast<int>(cta_rank), n_blk = tile / num_m_blocks;
                 const int m0 = m_blk * BM, n0 = n_blk * BN;
                 // 128-column blocks of this tile that exist (the scale atoms of a missing one are not fetched; its
                 // outputs are never stored)
                 const int nb_here = min(NB, (p.N + 127) / 128 - n_blk * NB);
+                // pairs: the second CTA's block of rows may lie past M (odd number of row blocks): it has no scale atoms
+                // (its codes are read as zeros, its outputs never stored)
+                const int sfa_here = m0 < p.M ? 1 : 0;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t st = smem_base + s * STAGE_BYTES;
-                    mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES + (1 + nb_here) * SF_BYTES);
+                    mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES + (sfa_here + nb_here) * SF_BYTES);
                     tma_load_2d(st, &tmap_codes, full_bar(s), kb * 128, m0);             // byte coordinates
 #pragma unroll
-                    for (int b = 0; b < NB; ++b)  // rows past N are filled with zeros (and still counted)
-                        tma_load_2d(st + A_BYTES + b * 16384, &tmap_wcodes, full_bar(s), kb * 128, n0 + b * 128);
-                    bulk_load(st + A_BYTES + B_BYTES, p.xsf + (static_cast<size_t>(m_blk) * p.nkb64p + kb * 4) * 512, SF_BYTES,
-                              full_bar(s));
+                    for (int b = 0; b < NB_DATA; ++b)  // rows past N are filled with zeros (and still counted)
+                        tma_load_2d(st + A_BYTES + b * 16384, &tmap_wcodes, full_bar(s), kb * 128,
+                                    n0 + (PAIR ? static_cast<int>(cta_rank) : b) * 128);
+                    if (sfa_here)
+                        bulk_load(st + A_BYTES + B_BYTES, p.xsf + (static_cast<size_t>(m_blk) * p.nkb64p + kb * 4) * 512, SF_BYTES,
+                                  full_bar(s));
                     for (int b = 0; b < nb_here; ++b)
                         bulk_load(st + A_BYTES + B_BYTES + (1 + b) * SF_BYTES,
                                   p.wsf + (static_cast<size_t>(n_blk * NB + b) * p.nkb64p + kb * 4) * 512, SF_BYTES, full_bar(s));
@@ -206,8 +249,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
                     tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
 #pragma unroll
-                    for (int b = 0; b < NB; ++b)
-                        tma_load_2d(st + A_BYTES + b * 16384, &tmap_wh, full_bar(s), lr * 64, n0 + b * 128);
+                    for (int b = 0; b < NB_DATA; ++b)
+                        tma_load_2d(st + A_BYTES + b * 16384, &tmap_wh, full_bar(s), lr * 64,
+                                    n0 + (PAIR ? static_cast<int>(cta_rank) : b) * 128);
                 }
             }
             if (!ok) {
@@ -220,12 +264,12 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_nv = nvfp4_idesc(BM, BN);
-            constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc_nv = nvfp4_idesc(TILE_ROWS, BN);
+            constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, TILE_ROWS, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step, ++tcount) {
                 const uint32_t acc = tcount % ACC_BUFS;
                 if (!mbar_wait(tempty_bar(acc), ((tcount / ACC_BUFS) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                 tc_fence_after_sync();
@@ -242,9 +286,14 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)  // K = 64 elements = 32 bytes per instruction
-                        umma_nvfp4(d, adesc + 2 * k, bdesc + 2 * k, idesc_nv, tsf + 4 * k, tsf + 16 + 4 * NB * k, (kb | k) != 0);
-                    umma_commit(empty_bar(s));
+                    for (int k = 0; k < 4; ++k) {  // K = 64 elements = 32 bytes per instruction
+                        if constexpr (PAIR)
+                            umma_nvfp4_pair(d, adesc + 2 * k, bdesc + 2 * k, idesc_nv, tsf + 4 * k, tsf + 16 + 4 * NB * k, (kb | k) != 0);
+                        else
+                            umma_nvfp4(d, adesc + 2 * k, bdesc + 2 * k, idesc_nv, tsf + 4 * k, tsf + 16 + 4 * NB * k, (kb | k) != 0);
+                    }
+                    if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);  // both CTAs' producers may refill the stage
+                    else umma_commit(empty_bar(s));
                 }
                 if (!ok) break;
                 for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
@@ -256,10 +305,17 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc_bf, 1u);
-                    umma_commit(empty_bar(s));
+                    for (int k = 0; k < 4; ++k) {
+                        if constexpr (PAIR) umma_bf16_pair(d, adesc + 2 * k, bdesc + 2 * k, idesc_bf, 1u);
+                        else umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc_bf, 1u);
+                    }
+                    if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);
+                    else umma_commit(empty_bar(s));
                 }
-                if (ok) umma_commit(tfull_bar(acc));
+                if (ok) {
+                    if constexpr (PAIR) umma_commit_pair(tfull_bar(acc), 3);  // both CTAs' epilogue warps
+                    else umma_commit(tfull_bar(acc));
+                }
             }
         }
     } else if (warp < 4) {
@@ -271,11 +327,19 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
                 const int items = p.num_kb + p.lr_chunks;
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK)) { ok = false; break; }
+                    if constexpr (PAIR) {
+                        if (cta_rank != 0) {
+                            // this CTA's stage has landed: one word to the leader, whose copiers and MMA thread act for both
+                            if (warp == 2) mbar_arrive_cluster(map_to_cta(peer_bar(s), 0));
+                            continue;
+                        }
+                        if (!mbar_wait(peer_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK)) { ok = false; break; }
+                    }
                     if (i < p.num_kb) {
                         tc_fence_after_sync();
                         const uint32_t sf = smem_base + s * STAGE_BYTES + A_BYTES + B_BYTES;
@@ -283,16 +347,24 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                         if (warp == 2) {
                             // activation scales: the four K = 64 steps of the k-block, 4 columns each
 #pragma unroll
-                            for (int a = 0; a < 4; ++a) tmem_cp_32x128b_warpx4(tsf + 4 * a, sf_desc(sf + a * 512));
+                            for (int a = 0; a < 4; ++a) {
+                                if constexpr (PAIR) tmem_cp_32x128b_warpx4_pair(tsf + 4 * a, sf_desc(sf + a * 512));
+                                else tmem_cp_32x128b_warpx4(tsf + 4 * a, sf_desc(sf + a * 512));
+                            }
                         } else {
                             // weight scales: per K step, the tile's 128-column blocks side by side (4 columns each)
 #pragma unroll
                             for (int a = 0; a < 4; ++a)
 #pragma unroll
-                                for (int b = 0; b < NB; ++b)
-                                    tmem_cp_32x128b_warpx4(tsf + 16 + 4 * NB * a + 4 * b, sf_desc(sf + (1 + b) * SF_BYTES + a * 512));
+                                for (int b = 0; b < NB; ++b) {
+                                    if constexpr (PAIR)
+                                        tmem_cp_32x128b_warpx4_pair(tsf + 16 + 4 * NB * a + 4 * b, sf_desc(sf + (1 + b) * SF_BYTES + a * 512));
+                                    else
+                                        tmem_cp_32x128b_warpx4(tsf + 16 + 4 * NB * a + 4 * b, sf_desc(sf + (1 + b) * SF_BYTES + a * 512));
+                                }
                         }
-                        umma_commit(sfready_bar(s));
+                        if constexpr (PAIR) umma_commit_pair(sfready_bar(s), 1);  // the leader's barrier only
+                        else umma_commit(sfready_bar(s));
                     } else {
                         mbar_arrive(sfready_bar(s));  // a rank-r chunk: nothing to copy
                     }
@@ -310,8 +382,8 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         uint32_t tcount = 0;
         bool ok = true;
         const float out_scale = __ldg(p.out_scale);
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-            const int m0 = (tile % num_m_blocks) * BM;
+        for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step, ++tcount) {
+            const int m0 = (tile % num_m_blocks) * TILE_ROWS + (PAIR ? static_cast<int>(cta_rank) * BM : 0);
             const int n0 = (tile / num_m_blocks) * BN;
             const uint32_t acc = tcount % ACC_BUFS;
             // The tile's bias goes to shared memory while its MMAs are still running (two buffers: a warp can be one tile
@@ -344,7 +416,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             for (int c = 0; c < HB / 32; ++c) tmem_ld_32x32b_x32(taddr + c * 32, raw[c]);
             tmem_ld_wait();
             tc_fence_before_sync();
-            mbar_arrive(tempty_bar(acc));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
+            // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
+            if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
+            else mbar_arrive(tempty_bar(acc));
             if (row < p.M) {
                 const float* bq = s_b + half * HB;
                 uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + n0 + half * HB;
@@ -368,16 +442,30 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         }
     }
 
-    if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
+    if constexpr (PAIR) {
+        if (warp == 1 && lane == 0 && cta_rank == 0 && *abort_flag != 0) {  // a wait gave up: let issued MMAs finish first
+            umma_commit_pair(bar_base + 200u, 1);
+            const unsigned long long t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar_base + 200u, 0) && globaltimer_ns() - t0 < 100000000ull) {}
+        }
+        tc_fence_before_sync();
+        cluster_sync_all();  // neither CTA leaves while the other may still read its operands or signal its barriers
+        if (warp == 1) {
+            tc_fence_after_sync();
+            tmem_dealloc_pair(tmem_base, 512);
+        }
+    } else {
+        if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 200u);  // a wait gave up: let issued MMAs finish first
+        tc_fence_before_sync();
+        __syncthreads();
+        if (warp == 1) {
+            tc_fence_after_sync();
+            tmem_dealloc(tmem_base, 512);
+        }
     }
 }
 
-template <int BN>
+template <int BN, bool PAIR = false>
 static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4GemmArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     CUtensorMap tmap_codes, tmap_xh;
@@ -398,13 +486,22 @@ static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4Ge
     p.bias = reinterpret_cast<const float*>(L->blob + L->lay.off_bias);
     p.out_scale = reinterpret_cast<const float*>(L->blob + L->lay.off_meta);
     p.y = a.y; p.status = a.status;
-    const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
-    const int grid = num_tiles < sm_count(L->device) ? num_tiles : sm_count(L->device);
-    static SmemOptIn<1> opt_in;
-    if (!opt_in.ensure(nvfp4_gemm_kernel<BN>, 0, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
-    // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand
-    const cudaError_t err = launch_kernel(nvfp4_gemm_kernel<BN>, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true,
-                                          tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    const int sms = sm_count(L->device);
+    static SmemOptIn<1> opt_in;  // one per instantiation of this launcher
+    if (!opt_in.ensure(nvfp4_gemm_kernel<BN, PAIR>, 0, L->device, Plan<BN, PAIR>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+    // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand (one per CTA of a pair)
+    cudaError_t err;
+    if constexpr (PAIR) {
+        const int pair_tiles = ((a.M + 2 * BM - 1) / (2 * BM)) * ((g.N + BN - 1) / BN);
+        const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
+        err = launch_kernel_pairs(nvfp4_gemm_kernel<BN, PAIR>, 2 * pairs, NUM_THREADS, Plan<BN, PAIR>::SMEM_BYTES, stream, true,
+                                  tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    } else {
+        const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+        const int grid = num_tiles < sms ? num_tiles : sms;
+        err = launch_kernel(nvfp4_gemm_kernel<BN>, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true,
+                            tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+    }
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
@@ -412,8 +509,8 @@ static std::atomic<int> g_nv_tile_columns{0};  // 0: chosen per call; 128 / 256:
 
 }  // namespace
 
-dirotq_status_t set_nvfp4_tile_columns(int columns) {
-    if (columns != 0 && columns != 128 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+dirotq_status_t set_nvfp4_tile_columns(int columns) {  // 512: 256 columns per pair of CTAs
+    if (columns != 0 && columns != 128 && columns != 256 && columns != 512) return DIROTQ_ERR_INVALID_ARG;
     g_nv_tile_columns.store(columns);
     return DIROTQ_OK;
 }
@@ -426,6 +523,7 @@ dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a,
     const long m_blocks = (a.M + BM - 1) / BM;
     const long t_wide = m_blocks * ((L->geo.N + 255) / 256), t_narrow = m_blocks * ((L->geo.N + 127) / 128);
     const bool narrow_pays = 0.6 * static_cast<double>((t_narrow + sms - 1) / sms) < 0.98 * static_cast<double>((t_wide + sms - 1) / sms);
+    if (forced == 512) return launch_nvfp4_gemm_bn<256, true>(L, a, stream);
     const bool wide = forced ? forced == 256 : !narrow_pays;
     return wide ? launch_nvfp4_gemm_bn<256>(L, a, stream) : launch_nvfp4_gemm_bn<128>(L, a, stream);
 }

@@ -281,6 +281,11 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, 
         : "memory");
 }
 
+// Generic-proxy writes of this thread -> visible to the tensor core, whichever CTA of the pair issues the MMA.
+__device__ __forceinline__ void fence_proxy_async_all() {
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 // Arrival, on completion of all MMAs issued so far by this thread, on the barrier at `bar`'s offset in the shared memory
 // of every CTA named in cta_mask (bit 0: rank 0, bit 1: rank 1).  A barrier arrival, not a data transfer.
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask) {
