@@ -151,8 +151,27 @@ dirotq_status_t dirotq_workspace_bytes(const dirotq_layer_t* layer, int M, size_
     return DIROTQ_OK;
 }
 
-// Weight-side tensor maps with 192-row boxes (the 192-column tile plan of the grouped INT4 second kernel).
+// Weight-side tensor maps with 192-row boxes (the 192-column tile plan of the grouped INT4 second kernel) and with 64-row
+// boxes (its plan for calls with few token rows).
+static dirotq_status_t encode_tmaps_rows(dirotq_layer* L, int N, int group, int rows, CUtensorMap* wpacked, CUtensorMap* wscale,
+                                         CUtensorMap* wh) {
+    const Geometry& g = L->geo;
+    const BlobLayout& lay = L->lay;
+    dirotq_status_t st = encode_tmap_2d(wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
+                                        (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, rows, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(wscale, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, L->blob + lay.off_wscale,
+                            (uint64_t)wscale_row_len(N), (uint64_t)g.n_g, (uint64_t)wscale_row_len(N) * 4, rows, 128 / group,
+                            CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(wh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_wh, (uint64_t)g.r_pad,
+                            (uint64_t)N, (uint64_t)g.r_pad * 2, 64, rows, CU_TENSOR_MAP_SWIZZLE_128B);
+    return st;
+}
+
 static dirotq_status_t encode_tmaps_192(dirotq_layer* L, int N, int group) {
+    dirotq_status_t st64 = encode_tmaps_rows(L, N, group, 64, &L->tmap_wpacked64, &L->tmap_wscale64, &L->tmap_wh64);
+    if (st64 != DIROTQ_OK) return st64;
     const Geometry& g = L->geo;
     const BlobLayout& lay = L->lay;
     dirotq_status_t st = encode_tmap_2d(&L->tmap_wpacked192, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
@@ -220,6 +239,9 @@ static dirotq_status_t prepare_int4(bool asym, bool sibling, const void* W, int 
         if (st == DIROTQ_OK)
             st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K,
                                 (uint64_t)K, (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (st == DIROTQ_OK)
+            st = encode_tmap_2d(&L->tmap_qt64, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K,
+                                (uint64_t)K, (uint64_t)K * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
     }
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
@@ -480,6 +502,9 @@ dirotq_status_t dirotq_prepare_layer_w4a8(const void* W, int w_dtype, int w_layo
         st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
                             (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt64, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                            (uint64_t)K * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked,
                             (uint64_t)g.K_lp / 2, (uint64_t)N, (uint64_t)g.K_lp / 2, 64, kGemmBN, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st == DIROTQ_OK)
@@ -627,10 +652,11 @@ dirotq_status_t dirotq_set_dependent_launch(int enabled) {
 }
 
 dirotq_status_t dirotq_set_gemm_tile(int columns) {
-    // 192: a plan of the grouped INT4 second kernel only; 512: 256 columns per pair of CTAs, NVFP4 second kernel only
+    // 64 and 192: plans of the grouped INT4 second kernel only; 512: 256 columns per pair of CTAs, NVFP4 second kernel only
+    const bool int4_only = columns == 64 || columns == 192;
     dirotq_status_t st = set_w4a4_tile_columns(columns == 512 ? 0 : columns);
-    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(columns == 192 ? 0 : columns);
-    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(columns == 192 || columns == 512 ? 0 : columns);
+    if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(int4_only ? 0 : columns);
+    return st != DIROTQ_OK ? st : set_w4a8_tile_columns(int4_only || columns == 512 ? 0 : columns);
 }
 
 dirotq_status_t dirotq_rotate_quantize(const void* x, int M, const dirotq_layer_t* layer, void* workspace,
@@ -860,6 +886,9 @@ dirotq_status_t dirotq_prepare_layer_nvfp4(const void* W, int w_dtype, int w_lay
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_qt128, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
                             (uint64_t)K * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st == DIROTQ_OK)
+        st = encode_tmap_2d(&L->tmap_qt64, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L->blob + lay.off_qt, (uint64_t)K, (uint64_t)K,
+                            (uint64_t)K * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st == DIROTQ_OK)
         st = encode_tmap_2d(&L->tmap_wpacked, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, L->blob + lay.off_wpacked, (uint64_t)g.K4 / 2,
                             (uint64_t)N, (uint64_t)g.K4 / 2, 128, kNvfp4BN, CU_TENSOR_MAP_SWIZZLE_128B);

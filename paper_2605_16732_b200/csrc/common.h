@@ -246,6 +246,8 @@ struct dirotq_layer {
     CUtensorMap tmap_wh;       // bf16 [N][r_pad], box 64 x kGemmBN, 128B swizzle
     CUtensorMap tmap_wpacked128, tmap_wscale128, tmap_wh128;  // the same three with 128-row boxes (narrow W4A4 tiles)
     CUtensorMap tmap_wpacked192, tmap_wscale192, tmap_wh192;  // ... and with 192-row boxes (grouped INT4 formats)
+    CUtensorMap tmap_wpacked64, tmap_wscale64, tmap_wh64;     // ... and with 64-row boxes (calls with few token rows)
+    CUtensorMap tmap_qt64;     // the rotation with box 64 x 64 (calls with few token rows, groups of 64)
     int act_scale_log2;        // NVFP4 variant: exponent of the activations' per-tensor power-of-two scale
 };
 

@@ -217,7 +217,8 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     constexpr int A_BYTES = BM * BK * 2;
     static_assert(!PAIR || (BM == 128 && BN == 256 && !PH), "pairs: 128 rows per CTA, 256 columns per pair");
     constexpr int B_ROWS = PAIR ? BN / 2 : BN;  // rows of the rotation tile this CTA holds
-    constexpr int STAGES = BM == 256 ? 3 : (B_ROWS == 256 ? STAGES_WIDE : 6);
+    static_assert(BN >= G, "a tile holds whole groups");
+    constexpr int STAGES = BM == 256 ? 3 : (B_ROWS == 256 ? STAGES_WIDE : B_ROWS == 128 ? 6 : 8);
     constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;
     constexpr int ACC_BUFS = BM == 256 ? 1 : 2;
     static_assert(STAGES * STAGE_BYTES == STAGES_WIDE * STAGE_BYTES_WIDE && STAGE_BYTES % 1024 == 0, "ring layout");
@@ -688,14 +689,14 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const float* __res
 }
 
 static std::atomic<int> g_first_step_split{1};  // projection form: 0 keeps the first step's reduction in one piece
-static std::atomic<int> g_rotation_plan{0};  // 0: chosen per call; 1: 128 x 128, 2: 128 x 256, 3: 256 x 256 tiles
+static std::atomic<int> g_rotation_plan{0};  // 0: chosen per call; 1: 128 x 128, 2: 128 x 256, 3: 256 x 256 tiles, 4: CTA pairs, 5: 128 x 64
 
 }  // namespace
 
 void set_first_step_split(bool on) { g_first_step_split.store(on ? 1 : 0); }
 
 dirotq_status_t set_rotation_plan(int plan) {
-    if (plan < 0 || plan > 4) return DIROTQ_ERR_INVALID_ARG;
+    if (plan < 0 || plan > 5) return DIROTQ_ERR_INVALID_ARG;
     g_rotation_plan.store(plan);
     return DIROTQ_OK;
 }
@@ -729,7 +730,11 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         // tiles: M = 256, K = 1152 runs on 18 instead of 10 SMs; M = 4096, K = 1152: 288 tiles in two waves instead of
         // 160 in two), not otherwise (M = 1024, K = 3072: 96 wide tiles in one wave, 30 us, against 192 narrow ones in
         // two, 45 us)
-        if (0.62 * static_cast<double>(waves_narrow) < static_cast<double>(waves128)) plan = 1;
+        // few token rows: when even the 128-column tiles would keep fewer than half of the SMs busy, 64-column tiles (eight
+        // 24 KB stages) on twice as many: every CTA streams all of x's row block and its own columns of the rotation through
+        // one SM's port to L2, so the time of a call this small falls with the bytes per CTA
+        if (2 * mb128 * nb128 <= sms && g.G == 64) plan = 5;
+        else if (0.62 * static_cast<double>(waves_narrow) < static_cast<double>(waves128)) plan = 1;
         else if ((g.K >= 8192 || x_exceeds_l2) && cost256 * static_cast<double>(waves256) < 0.98 * static_cast<double>(waves128)) plan = 3;
         // CTA pairs where there are a few waves of tiles and the main loop is not long enough for the operand traffic
         // to hide behind the MMAs anyway (measured against 128 x 256 tiles: M = 4608, K = 3072 68.4 -> 67.3 us; M = 9216,
@@ -755,6 +760,24 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         if (!opt_in_pair.ensure(pair_table[vi], vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
         return launch_kernel_pairs(pair_table[vi], 2 * pairs, NUM_THREADS, SMEM_BYTES, stream, g.fmt != 3, tmap_xp, L->tmap_qt128,
                                    tmap_xp, L->tmap_qt128, p) == cudaSuccess
+                   ? DIROTQ_OK
+                   : DIROTQ_ERR_CUDA;
+    }
+    if (plan == 5 && g.G != 64) plan = 1;  // a tile holds whole groups
+    if (plan == 5) {
+        CUtensorMap tmap_x5;
+        dirotq_status_t st5 = encode_tmap_2d(&tmap_x5, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)g.K, (uint64_t)a.M,
+                                             (uint64_t)g.K * 2, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (st5 != DIROTQ_OK) return st5;
+        const long tiles5 = mb128 * ((g.K + 63) / 64);
+        const int vi5 = g.fmt == 1 ? 1 : g.fmt == 2 ? 2 : g.fmt == 3 ? 3 : 0;
+        using Fn5 = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
+        static const Fn5 table5[4] = {rotate_quant_kernel<64, 0, 64, 128>, rotate_quant_kernel<64, 1, 64, 128>,
+                                      rotate_quant_kernel<64, 2, 64, 128>, rotate_quant_kernel<64, 3, 64, 128>};
+        static SmemOptIn<4> opt_in5;
+        if (!opt_in5.ensure(table5[vi5], vi5, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+        return launch_kernel(table5[vi5], static_cast<int>(tiles5 < sms ? tiles5 : sms), NUM_THREADS, SMEM_BYTES, stream, g.fmt != 3,
+                             tmap_x5, L->tmap_qt64, tmap_x5, L->tmap_qt64, p) == cudaSuccess
                    ? DIROTQ_OK
                    : DIROTQ_ERR_CUDA;
     }

@@ -56,15 +56,20 @@ constexpr float kAccUnit = kI8Path ? 1.0f : kWScaleFold;  // integer group sum =
 //        buffers, so the tile goes back to the tensor core after the first quarter of a group, and three warps per scheduler
 //        hide each other's waits.  16 warps: 152 registers for the epilogue threads, 56 for the others.
 //   128: two warpgroups, 64 columns per thread, four accumulator tiles; for layers whose wider tiles would leave SMs idle.
+//    64: one warpgroup, 64 columns per thread, four accumulator tiles, seven stages; for calls with so few token rows that
+//        even 128-column tiles occupy a fraction of the SMs: there a tile's K-groups are a chain of hand-overs between the
+//        tensor core and the epilogue, whose length does not depend on the tile's width, so more, narrower tiles on more SMs
+//        shorten the call.  256 threads, no register re-partitioning (every thread may use 255).
 template <int BN>
 struct Plan {
-    static constexpr int EPI_WG = BN == 192 ? 3 : 2;          // epilogue warpgroups
+    static constexpr int EPI_WG = BN == 192 ? 3 : BN == 64 ? 1 : 2;  // epilogue warpgroups
     static constexpr int EPI_WARPS = 4 * EPI_WG;
     static constexpr int THREADS = 128 + 128 * EPI_WG;
+    static constexpr bool REPARTITION = EPI_WG > 1;            // setmaxnreg after the role split
     static constexpr int EPI_REGS = EPI_WG == 3 ? 152 : 216;  // setmaxnreg budgets: 128 * AUX + 128 * EPI_WG * EPI <= 65536
     static constexpr int AUX_REGS = EPI_WG == 3 ? 56 : 64;
     static constexpr int SC_SLOTS = BN == 192 ? 6 : 8;
-    static constexpr int STAGES = BN == 256 ? 3 : BN == 192 ? 4 : 5;
+    static constexpr int STAGES = BN == 256 ? 3 : BN == 192 ? 4 : BN == 128 ? 5 : 7;
     static constexpr int BU_BYTES = BN * BKC;         // unpacked weight codes / bf16 W~_h chunk (32 KB at BN = 256)
     static constexpr int BP_BYTES = BN * BKC / 2;     // packed weight codes (TMA staging)
     static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB / 40 KB
@@ -77,7 +82,9 @@ struct Plan {
 static_assert(Plan<256>::SMEM_BYTES <= 232448 && Plan<192>::SMEM_BYTES <= 232448 && Plan<128>::SMEM_BYTES <= 232448, "shared memory plan too large");
 static_assert(Plan<128>::STAGE_BYTES % 1024 == 0 && Plan<128>::SC_BYTES % 128 == 0, "tile alignment");
 static_assert(Plan<192>::STAGE_BYTES % 1024 == 0 && Plan<192>::SC_BYTES % 128 == 0, "tile alignment");
-static_assert(8 * (3 * Plan<128>::STAGES + 2 * 8 + 9) <= 400 && 8 * (3 * Plan<192>::STAGES + 2 * 6 + 9) <= 400, "barriers end below the words at +400");
+static_assert(Plan<64>::SMEM_BYTES <= 232448 && Plan<64>::STAGE_BYTES % 1024 == 0 && Plan<64>::SC_BYTES % 128 == 0, "tile alignment");
+static_assert(8 * (3 * Plan<128>::STAGES + 2 * 8 + 9) <= 400 && 8 * (3 * Plan<192>::STAGES + 2 * 6 + 9) <= 400 &&
+              8 * (3 * Plan<64>::STAGES + 2 * 8 + 9) <= 400, "barriers end below the words at +400");
 
 struct GemmKernelParams {
     int M, N, n_g, num_kb, lr_chunks;
@@ -165,7 +172,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     constexpr int CHUNKS = HB / 32;    // 32-column chunks per epilogue warp and accumulator tile
     constexpr int GPK = BKC / G;       // groups per k-block: 2 (G = 64) or 1 (G = 128)
     constexpr int MMA_PER_G = G / 32;  // 8-bit MMA instructions (K = 32) per group
-    constexpr int NBUF = 512 / BN;     // accumulator tiles in tensor memory: 2 of 256 columns or 4 of 128
+    constexpr int NBUF = BN == 64 ? 4 : 512 / BN;  // accumulator tiles in tensor memory: 2 of 256 columns, 4 of 128 or of 64 (the barrier map has four slots)
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -228,7 +235,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     grid_launch_dependents();
 
     if (warp < 4) {
-        reg_dealloc<P::AUX_REGS>();
+        if constexpr (P::REPARTITION) reg_dealloc<P::AUX_REGS>();
 
         if (warp == 0) {
             // -------------------------------------------------------- TMA producer
@@ -402,7 +409,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             if (u == 0) flush_wait(p.status, WS_UNPACK_FULL, w_full);
         }
     } else {
-        reg_alloc<P::EPI_REGS>();
+        if constexpr (P::REPARTITION) reg_alloc<P::EPI_REGS>();
         // ------------------------------------------------------------ epilogue (warps 4..11)
         // A warp owns 32 token rows (its TMEM lane quadrant) x BN/2 columns.  The accumulators are read with the
         // 16x256b shape: a thread then holds 4 rows (l/4 + 8 i) x the column pairs 2 (l%4) + {0, 1} of every block
@@ -667,19 +674,19 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
     const int vi = (g.G == 64 ? 0 : 2) + (dbg ? 1 : 0);
     if (!opt_in.ensure(kern, vi, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     const cudaError_t err = launch_kernel(kern, grid, Plan<BN>::THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
-                                          BN == 128 ? L->tmap_wpacked128 : BN == 192 ? L->tmap_wpacked192 : L->tmap_wpacked,
-                                          BN == 128 ? L->tmap_wscale128 : BN == 192 ? L->tmap_wscale192 : L->tmap_wscale,
+                                          BN == 64 ? L->tmap_wpacked64 : BN == 128 ? L->tmap_wpacked128 : BN == 192 ? L->tmap_wpacked192 : L->tmap_wpacked,
+                                          BN == 64 ? L->tmap_wscale64 : BN == 128 ? L->tmap_wscale128 : BN == 192 ? L->tmap_wscale192 : L->tmap_wscale,
                                           tmap_xscale, tmap_xh,
-                                          BN == 128 ? L->tmap_wh128 : BN == 192 ? L->tmap_wh192 : L->tmap_wh, p);
+                                          BN == 64 ? L->tmap_wh64 : BN == 128 ? L->tmap_wh128 : BN == 192 ? L->tmap_wh192 : L->tmap_wh, p);
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
 }  // namespace
 
-static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 128 / 192 / 256: forced
+static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 64 / 128 / 192 / 256: forced
 
 dirotq_status_t set_w4a4_tile_columns(int columns) {
-    if (columns != 0 && columns != 128 && columns != 192 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+    if (columns != 0 && columns != 64 && columns != 128 && columns != 192 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
     g_tile_columns.store(columns);
     return DIROTQ_OK;
 }
@@ -687,6 +694,10 @@ dirotq_status_t set_w4a4_tile_columns(int columns) {
 dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
     const int forced = g_tile_columns.load();
     if (forced == 192) return launch_w4a4_gemm_bn<192>(L, a, stream);
+    // few token rows: when even 128-column tiles would keep fewer than half of the SMs busy, 64-column tiles on twice as many
+    const int sms = sm_count(L->device);
+    const long t128 = static_cast<long>((a.M + BM - 1) / BM) * ((L->geo.N + 127) / 128);
+    if (forced == 64 || (forced == 0 && 2 * t128 <= sms)) return launch_w4a4_gemm_bn<64>(L, a, stream);
     const bool narrow = forced ? forced == 128 : narrow_tiles_pay(a.M, L->geo.N, sm_count(L->device));
     return narrow ? launch_w4a4_gemm_bn<128>(L, a, stream) : launch_w4a4_gemm_bn<256>(L, a, stream);
 }

@@ -72,9 +72,9 @@ def test_null_and_bad_handles_are_rejected(L):
 
 
 def test_knobs_validate_their_argument_without_a_gpu(L):
-    for ok in (0, 128, 192, 256, 0):
+    for ok in (0, 64, 128, 192, 256, 512, 0):
         assert L.dirotq_set_gemm_tile(ok) == 0
-    for bad in (-1, 64, 160, 512):
+    for bad in (-1, 96, 160, 384, 1024):
         assert L.dirotq_set_gemm_tile(bad) == 1
     assert L.dirotq_set_dependent_launch(0) == 0 and L.dirotq_set_dependent_launch(1) == 0
     assert L.dirotq_set_first_step_split(0) == 0 and L.dirotq_set_first_step_split(1) == 0

@@ -1,4 +1,4 @@
-"""The INT4 second kernel with 128-, 192- (three epilogue warpgroups) and 256-column tiles: both forced through dirotq_set_gemm_tile, on shapes the
+"""The INT4 second kernel with 64- (one epilogue warpgroup, for calls with few token rows), 128-, 192- (three epilogue warpgroups) and 256-column tiles: both forced through dirotq_set_gemm_tile, on shapes the
 automatic choice would send one way only.  Parity with the oracle under each setting, and bit-equal outputs and
 integer group sums between the two (every output element is accumulated in the same order)."""
 import numpy as np
@@ -22,20 +22,20 @@ def tile(request):
     dq.dirotq_set_gemm_tile(0)
 
 
-@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
 def test_parity_group64_ragged_everything(tile):
     # N = 400: ragged in both tile widths; M = 300: ragged rows; K_l = 496: ragged last group
     spec = synth.LayerSpec(K=512, N=400, r=16, G=64, model=synth.FLUX, seed=31, calib_tokens=1024)
     print(tile, test_gpu_parity._run_case(spec, M=300))
 
 
-@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
 def test_parity_group128_rank128(tile):
     spec = synth.LayerSpec(K=768, N=640, r=128, G=128, model=synth.FLUX, seed=32, calib_tokens=1024)
     print(tile, test_gpu_parity._run_case(spec, M=257, with_bias=False))
 
 
-@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
 def test_parity_pixart_projection_many_tiles(tile):
     # 8 row blocks x 9 (or 5) column blocks: several tiles per CTA are not reached on one GPU with 148 SMs, but the
     # tile -> (row block, column block) mapping and the ring phases across k-blocks are
@@ -43,7 +43,7 @@ def test_parity_pixart_projection_many_tiles(tile):
     print(tile, test_gpu_parity._run_case(spec, M=1024, check_rot=False))
 
 
-@pytest.mark.parametrize("tile", [128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
 def test_parity_asymmetric_codes(tile):
     spec = synth.LayerSpec(K=640, N=400, r=32, G=64, model=synth.PIXART, seed=34, calib_tokens=1024)
     print(tile, test_gpu_asym._run_case(spec, M=200, shift=1.5))
@@ -60,7 +60,7 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
     ws = dq.alloc_workspace(layer, M)
     outs = {}
     try:
-        for cols in (0, 128, 192, 256):
+        for cols in (0, 64, 128, 192, 256):
             dq.dirotq_set_gemm_tile(cols)
             y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
             dq.dirotq_linear(x, layer, y, ws)
@@ -69,33 +69,35 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
             outs[cols] = y.view(torch.int16).clone()
         # several tiles per CTA here (33 row blocks x 9 column blocks on 148 SMs)
         assert torch.equal(outs[128], outs[256]) and torch.equal(outs[192], outs[256]) and torch.equal(outs[0], outs[128])
+        assert torch.equal(outs[64], outs[256])
         with pytest.raises(dq.DirotqError):
-            dq.dirotq_set_gemm_tile(64)
+            dq.dirotq_set_gemm_tile(96)
     finally:
         dq.dirotq_set_gemm_tile(0)
     layer.close()
 
 
-# ------------------------------------------------------------------ NVFP4 second kernel: 128- and 256-column tiles
+# ------------------------------------------------------------------ NVFP4 second kernel: 128- and 256-column tiles, and
+# 256 rows x 256 columns per pair of CTAs (knob value 512)
 
 import test_gpu_nvfp4
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 256, 512], indirect=True)
 def test_nvfp4_ragged_columns_two_blocks_in_last_tile(tile):
     # N = 400: four 128-column blocks, the last one ragged
     spec = synth.LayerSpec(K=512, N=400, r=16, G=64, model=synth.FLUX, seed=51, calib_tokens=1024)
     print(tile, test_gpu_nvfp4._run_case(spec, M=300))
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 256, 512], indirect=True)
 def test_nvfp4_odd_number_of_column_blocks(tile):
     # N = 384: three 128-column blocks, so the second 256-column tile has no second block (its scale atoms do not exist)
     spec = synth.LayerSpec(K=768, N=384, r=32, G=64, model=synth.PIXART, seed=52, calib_tokens=1024)
     print(tile, test_gpu_nvfp4._run_case(spec, M=257, with_bias=False))
 
 
-@pytest.mark.parametrize("tile", [128, 256], indirect=True)
+@pytest.mark.parametrize("tile", [128, 256, 512], indirect=True)
 def test_nvfp4_single_column_block_and_two_rank_chunks(tile):
     spec = synth.LayerSpec(K=640, N=128, r=128, G=64, model=synth.FLUX, seed=53, calib_tokens=1024)
     print(tile, test_gpu_nvfp4._run_case(spec, M=130))
@@ -118,7 +120,7 @@ def test_nvfp4_both_widths_give_the_same_bits():
     ws = dq.alloc_workspace(layer, M)
     outs = {}
     try:
-        for cols in (0, 128, 256):
+        for cols in (0, 128, 256, 512):
             dq.dirotq_set_gemm_tile(cols)
             y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
             dq.dirotq_linear(x, layer, y, ws)
@@ -126,7 +128,7 @@ def test_nvfp4_both_widths_give_the_same_bits():
             assert dq.dirotq_workspace_status(ws) == 0
             outs[cols] = y.view(torch.int16).clone()
         # the accumulation order inside the tensor core does not depend on the tile width: same bits
-        assert torch.equal(outs[128], outs[256]) and torch.equal(outs[0], outs[128])
+        assert torch.equal(outs[128], outs[256]) and torch.equal(outs[0], outs[128]) and torch.equal(outs[512], outs[256])
     finally:
         dq.dirotq_set_gemm_tile(0)
     layer.close()
@@ -149,7 +151,8 @@ def test_w4a8_pixart_projection_many_tiles(tile):
     print(tile, test_gpu_w4a8._run_case(spec, M=1024, check_rot=False))
 
 
-# ------------------------------------------------------------------ rotation kernel: the tile plans (4 = CTA pairs)
+# ------------------------------------------------------------------ rotation kernel: the tile plans (4 = CTA pairs, 5 = 64-column
+# tiles for calls with few token rows; with groups of 128 plan 5 falls back to plan 1)
 
 @pytest.fixture
 def rot_plan(request):
@@ -158,20 +161,20 @@ def rot_plan(request):
     dq.dirotq_set_rotation_tile(0)
 
 
-@pytest.mark.parametrize("rot_plan", [1, 2, 3, 4], indirect=True)
+@pytest.mark.parametrize("rot_plan", [1, 2, 3, 4, 5], indirect=True)
 def test_rotation_plans_int4_ragged(rot_plan):
     # M = 300: the second 128-row block of a 256-row tile is ragged; K_l = 496: ragged last group
     spec = synth.LayerSpec(K=512, N=256, r=16, G=64, model=synth.FLUX, seed=91, calib_tokens=1024)
     print(rot_plan, test_gpu_parity._run_case(spec, M=300))
 
 
-@pytest.mark.parametrize("rot_plan", [1, 2, 3, 4], indirect=True)
+@pytest.mark.parametrize("rot_plan", [1, 2, 3, 4, 5], indirect=True)
 def test_rotation_plans_group128_many_row_blocks(rot_plan):
     spec = synth.LayerSpec(K=768, N=128, r=128, G=128, model=synth.PIXART, seed=92, calib_tokens=1024)
     print(rot_plan, test_gpu_parity._run_case(spec, M=1100, with_bias=False))
 
 
-@pytest.mark.parametrize("rot_plan", [3, 4], indirect=True)
+@pytest.mark.parametrize("rot_plan", [3, 4, 5], indirect=True)
 def test_rotation_256_row_tiles_other_formats(rot_plan):
     spec = synth.LayerSpec(K=640, N=256, r=32, G=64, model=synth.FLUX, seed=93, calib_tokens=1024)
     print(test_gpu_asym._run_case(spec, M=385, shift=1.0))
@@ -190,7 +193,7 @@ def test_rotation_plans_give_the_same_codes_and_outputs():
     ws = dq.alloc_workspace(layer, M)
     outs = {}
     try:
-        for plan in (0, 1, 2, 3, 4):
+        for plan in (0, 1, 2, 3, 4, 5):
             dq.dirotq_set_rotation_tile(plan)
             y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
             dq.dirotq_linear(x, layer, y, ws)
@@ -198,11 +201,28 @@ def test_rotation_plans_give_the_same_codes_and_outputs():
             assert dq.dirotq_workspace_status(ws) == 0
             xh, codes, scales = dq.dirotq_workspace_export(layer, M, ws)
             outs[plan] = (y.view(torch.int16).clone(), codes.clone(), scales.view(torch.int16).clone(), xh.view(torch.int16).clone())
-        for plan in (0, 1, 3, 4):
+        for plan in (0, 1, 3, 4, 5):
             for a, b in zip(outs[plan], outs[2]):
                 assert torch.equal(a, b)
         with pytest.raises(dq.DirotqError):
-            dq.dirotq_set_rotation_tile(5)
+            dq.dirotq_set_rotation_tile(6)
     finally:
         dq.dirotq_set_rotation_tile(0)
     layer.close()
+
+
+# ------------------------------------------------------------------ few token rows: the automatic choice is the 64-column plans
+
+@pytest.mark.parametrize("M", [1, 100, 256, 300])
+def test_few_token_rows_take_the_narrow_plans(M):
+    # 1152 -> 1152: with up to three row blocks even 128-column tiles would use 27 of 148 SMs; both kernels then run with
+    # 64-column tiles (nothing forced here)
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=95)
+    print(M, test_gpu_parity._run_case(spec, M=M))
+
+
+def test_few_token_rows_other_formats():
+    spec = synth.LayerSpec(K=640, N=320, r=32, G=64, model=synth.FLUX, seed=96, calib_tokens=1024)
+    print(test_gpu_asym._run_case(spec, M=130, shift=1.0))
+    print(test_gpu_nvfp4._run_case(spec, M=130))
+    print(test_gpu_w4a8._run_case(spec, M=130))
