@@ -29,6 +29,14 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     return t;
 }
 
+// Diagnostic build (-DDIROTQ_TRACE): block 0 stamps the SM clock at marked points of each role into the 8-byte slots
+// 9..31 of the workspace's status block, for reading a small call's critical path off the device.
+#ifdef DIROTQ_TRACE
+#define TRACE_CLK(status, slot) do { if (blockIdx.x == 0) reinterpret_cast<volatile unsigned long long*>(status)[slot] = clock64(); } while (0)
+#else
+#define TRACE_CLK(status, slot) do {} while (0)
+#endif
+
 // ---------------------------------------------------------------- mbarrier
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -97,6 +105,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             }
         }
     }
+}
+
+// One lane of a converged warp (the same one every time).  A loop that the whole warp walks, with only the issue of an
+// instruction left to the elected lane, keeps its counters and addresses warp-uniform.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
 }
 
 // ---------------------------------------------------------------- proxies / fences

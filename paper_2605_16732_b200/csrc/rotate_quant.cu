@@ -287,7 +287,10 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // The whole warp walks the loops and waits; one elected lane issues.  Loop counters, addresses and coordinates
+        // then stay warp-uniform, which shortens the chain of instructions per stage (337 against 475 cycles per stage
+        // measured with 18 SMs busy, where that chain paces the kernel).
+        {
             uint32_t it = 0;
             bool ok = true;
             for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
@@ -302,6 +305,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         const uint32_t ph = (it / STAGES) & 1;
                         if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                         const uint32_t sa = smem_base + s * STAGE_BYTES;
+                        if (!elect_one()) continue;
                         if (i < nv) {
                             mbar_arrive_expect_tx(full_bar(s), A_BYTES + BN * BK * 2);
                             tma_load_2d(sa, &tmap_x, full_bar(s), i * BK, m0);
@@ -322,6 +326,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    if (!elect_one()) continue;
                     if constexpr (PAIR) {
                         // both CTAs' bytes are counted on the leader's barrier, which expects the sum
                         const uint32_t full_leader = map_to_cta(full_bar(s), 0);
@@ -335,7 +340,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
             }
-            if (!ok && PAIR && cta_rank != 0) {
+            if (lane != 0) {
+                // one lane looks after the loads in flight
+            } else if (!ok && PAIR && cta_rank != 0) {
                 // this CTA's loads report to the leader's barriers: give them a fixed time instead
                 const unsigned long long t0 = globaltimer_ns();
                 while (globaltimer_ns() - t0 < 1000000ull) {}
@@ -350,8 +357,8 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && cta_rank == 0) {
+        // ------------------------------------------------------------ MMA issuer (whole warp in the loops, one lane issues)
+        if (cta_rank == 0) {
             constexpr uint32_t idesc = umma_idesc(1 /*f32*/, 1 /*bf16*/, PAIR ? 2 * BM_MMA : BM_MMA, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
@@ -373,6 +380,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         const uint32_t sa = smem_base + s * STAGE_BYTES;
                         const uint64_t adesc = umma_desc_sw128(sa);
                         const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
+                        if (!elect_one()) continue;
                         if (i < nv) {
 #pragma unroll
                             for (int k = 0; k < BK / 16; ++k) umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k) != 0);
@@ -383,7 +391,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         }
                         umma_commit(empty_bar(s));
                     }
-                    if (ok) umma_commit(tfull_bar(acc));
+                    if (ok && elect_one()) umma_commit(tfull_bar(acc));
                     continue;
                 }
                 const int sp = tile / num_mn;
@@ -396,6 +404,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint32_t sa = smem_base + s * STAGE_BYTES;
                     const uint64_t adesc = umma_desc_sw128(sa);
                     const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
+                    if (!elect_one()) continue;
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
                         if constexpr (PAIR) {
@@ -409,7 +418,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);  // both CTAs' producers may refill the stage
                     else umma_commit(empty_bar(s));
                 }
-                if (ok) {
+                if (ok && elect_one()) {
                     if constexpr (PAIR) umma_commit_pair(tfull_bar(acc), 3);  // both CTAs' epilogue warps
                     else umma_commit(tfull_bar(acc));
                 }

@@ -64,7 +64,12 @@ template <int BN>
 struct Plan {
     static constexpr int EPI_WG = BN == 192 ? 3 : BN == 64 ? 1 : 2;  // epilogue warpgroups
     static constexpr int EPI_WARPS = 4 * EPI_WG;
-    static constexpr int THREADS = 128 + 128 * EPI_WG;
+    // MMA-issuing warps.  With few token rows a tile's K-groups are a chain of single-thread instructions (wait, fence, two
+    // MMAs, commit: each tens of cycles) that paces the kernel; two warps then issue alternate accumulator tiles (the second
+    // one is the block's last warp).
+    static constexpr int MMA_WARPS = 1;
+    static constexpr int MMA_B_WARP = 4 + 4 * EPI_WG;
+    static constexpr int THREADS = 128 + 128 * EPI_WG + (MMA_WARPS == 2 ? 32 : 0);
     static constexpr bool REPARTITION = EPI_WG > 1;            // setmaxnreg after the role split
     static constexpr int EPI_REGS = EPI_WG == 3 ? 152 : 216;  // setmaxnreg budgets: 128 * AUX + 128 * EPI_WG * EPI <= 65536
     static constexpr int AUX_REGS = EPI_WG == 3 ? 56 : 64;
@@ -84,7 +89,7 @@ static_assert(Plan<128>::STAGE_BYTES % 1024 == 0 && Plan<128>::SC_BYTES % 128 ==
 static_assert(Plan<192>::STAGE_BYTES % 1024 == 0 && Plan<192>::SC_BYTES % 128 == 0, "tile alignment");
 static_assert(Plan<64>::SMEM_BYTES <= 232448 && Plan<64>::STAGE_BYTES % 1024 == 0 && Plan<64>::SC_BYTES % 128 == 0, "tile alignment");
 static_assert(8 * (3 * Plan<128>::STAGES + 2 * 8 + 9) <= 400 && 8 * (3 * Plan<192>::STAGES + 2 * 6 + 9) <= 400 &&
-              8 * (3 * Plan<64>::STAGES + 2 * 8 + 9) <= 400, "barriers end below the words at +400");
+              8 * (3 * Plan<64>::STAGES + 2 * 8 + 10) <= 400, "barriers end below the words at +400");
 
 struct GemmKernelParams {
     int M, N, n_g, num_kb, lr_chunks;
@@ -192,6 +197,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 9);
 
     const int num_m_blocks = (p.M + BM - 1) / BM;
     const int num_n_blocks = (p.N + BN - 1) / BN;
@@ -201,7 +207,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(unp_bar(s), 64);  // every thread of the two unpack warps arrives for itself
-            mbar_init(empty_bar(s), 1);
+            mbar_init(empty_bar(s), P::MMA_WARPS);  // every MMA-issuing warp commits to it
         }
         for (int s = 0; s < SC_SLOTS; ++s) {
             mbar_init(scfull_bar(s), 1);
@@ -212,6 +218,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
         }
         mbar_init(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 8), 1);  // spare: see umma_drain
+        mbar_init(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 9), 1);  // ... of the second MMA-issuing warp
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_codes);
@@ -230,16 +237,21 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 10);
     grid_dependency_wait();
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 11);
     // the next layer's first kernel may be scheduled as this grid's CTAs leave their SMs (it waits for this whole grid)
     grid_launch_dependents();
 
-    if (warp < 4) {
+    const bool mma_b = P::MMA_WARPS == 2 && warp == P::MMA_B_WARP;
+    if (warp < 4 || mma_b) {
         if constexpr (P::REPARTITION) reg_dealloc<P::AUX_REGS>();
 
         if (warp == 0) {
             // -------------------------------------------------------- TMA producer
-            if (lane == 0) {
+            // (the whole warp walks the loops and waits, one elected lane issues: counters, addresses and coordinates stay
+            // warp-uniform, which shortens the chain of instructions per stage)
+            {
                 uint32_t it = 0, sc_it = 0;
                 long long w_empty = 0;
                 bool ok = true;
@@ -250,28 +262,36 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         const int s = it % STAGES;
                         if (!timed_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER, w_empty)) { ok = false; break; }
                         const uint32_t st = smem_base + s * STAGE_BYTES;
-                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
-                        tma_load_2d(st, &tmap_codes, full_bar(s), kb * BKC, m0);
-                        tma_load_2d(st + A_BYTES + BU_BYTES, &tmap_wpacked, full_bar(s), kb * (BKC / 2), n0);
+                        if (elect_one()) {
+                            mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
+                            tma_load_2d(st, &tmap_codes, full_bar(s), kb * BKC, m0);
+                            tma_load_2d(st + A_BYTES + BU_BYTES, &tmap_wpacked, full_bar(s), kb * (BKC / 2), n0);
+                        }
                         const int slot = sc_it % SC_SLOTS;
                         if (!mbar_wait(scempty_bar(slot), ((sc_it / SC_SLOTS) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                         const uint32_t sc = sc_base + slot * SC_BYTES;
-                        mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + BM) * 4);
-                        tma_load_2d(sc, &tmap_wscale, scfull_bar(slot), n0, kb * GPK);
-                        tma_load_2d(sc + SC_SW_BYTES, &tmap_xscale, scfull_bar(slot), m0, kb * GPK);
+                        if (elect_one()) {
+                            mbar_arrive_expect_tx(scfull_bar(slot), GPK * (BN + BM) * 4);
+                            tma_load_2d(sc, &tmap_wscale, scfull_bar(slot), n0, kb * GPK);
+                            tma_load_2d(sc + SC_SW_BYTES, &tmap_xscale, scfull_bar(slot), m0, kb * GPK);
+                            if (it == 0) TRACE_CLK(p.status, 12);
+                        }
                     }
                     if (!ok) break;
                     for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
                         const int s = it % STAGES;
                         if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                         const uint32_t st = smem_base + s * STAGE_BYTES;
-                        mbar_arrive_expect_tx(full_bar(s), A_BYTES + BU_BYTES);
-                        tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
-                        tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), lr * 64, n0);
+                        if (elect_one()) {
+                            mbar_arrive_expect_tx(full_bar(s), A_BYTES + BU_BYTES);
+                            tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
+                            tma_load_2d(st + A_BYTES, &tmap_wh, full_bar(s), lr * 64, n0);
+                        }
                     }
                 }
-                flush_wait(p.status, WS_PROD_EMPTY, w_empty);
-                if (!ok) {
+                if (lane == 0) TRACE_CLK(p.status, 13);
+                if (lane == 0) flush_wait(p.status, WS_PROD_EMPTY, w_empty);
+                if (!ok && lane == 0) {
                     const uint32_t first = it > STAGES ? it - STAGES : 0;
                     for (uint32_t j = first; j < it; ++j) {
                         const unsigned long long t0 = globaltimer_ns();
@@ -286,13 +306,14 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                 }
             }
-        } else if (warp == 1) {
+        } else if (warp == 1 || mma_b) {
             // -------------------------------------------------------- MMA issuer
             // One thread, and every instruction it executes waits its turn behind the two epilogue warps of its
             // scheduler, so its loop is kept short: stage index, parities and the operand descriptors are carried
             // along instead of recomputed (a descriptor differs between stages only in the address field of its low
             // word, which cannot overflow: shared-memory addresses have 18 bits, the field holds address / 16).
-            if (lane == 0) {
+            // (whole warp in the loops, one elected lane issues, as in the producer)
+            {
                 constexpr uint32_t idesc_f8 = umma_idesc(1 /*f32*/, 0 /*E4M3*/, BM, BN);
                 constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);  // integer-path build only
                 constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
@@ -301,60 +322,77 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 auto desc = [&](uint32_t lo) { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
                 uint32_t s = 0, ph = 0;        // stage of the operand ring and its parity
                 uint32_t b = 0, bph = 1;       // accumulator tile and the parity its "empty" barrier is waited with
+                // two issuing warps: this one takes the accumulator tiles of its parity (their number is even), follows
+                // every stage, and commits to every stage's "empty" barrier, which counts both warps
+                const uint32_t my = mma_b ? 1u : 0u;
+                auto mine = [&](uint32_t tile_idx) { return P::MMA_WARPS == 1 || (tile_idx & 1u) == my; };
                 long long w_ops = 0, w_tempty = 0;
                 const long long t_kernel = clock64();
                 bool ok = true;
                 for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                     int groups_left = p.n_g;
                     for (int kb = 0; ok && kb < p.num_kb; ++kb) {
-                        if (!timed_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
+                        // the unpack warps arrive after they have seen the stage's loads land (one barrier for both operands), so
+                        // their barrier covers the activation codes as well
                         if (!timed_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
+                        if (lane == 0) { if (kb == 0) TRACE_CLK(p.status, 16); if (kb == 4) TRACE_CLK(p.status, 17); if (kb == p.num_kb - 1) TRACE_CLK(p.status, 18); }
                         tc_fence_after_sync();
                         const uint32_t a_lo = desc_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
                         for (int gi = 0; gi < GPK; ++gi) {
                             if (gi < groups_left) {
+                              if (mine(b)) {
                                 if (!timed_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_tempty)) { ok = false; break; }
                                 tc_fence_after_sync();
+                                if (elect_one()) {
 #pragma unroll
-                                for (int k = 0; k < MMA_PER_G; ++k) {
-                                    const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
-                                    if constexpr (kI8Path)
-                                        umma_i8(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_i8, k != 0);
-                                    else
-                                        umma_f8f6f4(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_f8, k != 0);
+                                    for (int k = 0; k < MMA_PER_G; ++k) {
+                                        const int kk = gi * MMA_PER_G + k;  // 32-byte step inside the 128-byte row
+                                        if constexpr (kI8Path)
+                                            umma_i8(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_i8, k != 0);
+                                        else
+                                            umma_f8f6f4(tmem_base + b * BN, desc(a_lo + 2 * kk), desc(b_lo + 2 * kk), idesc_f8, k != 0);
+                                    }
+                                    umma_commit(tfull_bar(b));
                                 }
-                                umma_commit(tfull_bar(b));
+                              }
                                 if (++b == NBUF) { b = 0; bph ^= 1; }
                             }
                         }
                         if (!ok) break;
                         groups_left -= GPK;
-                        umma_commit(empty_bar(s));
+                        if (elect_one()) umma_commit(empty_bar(s));
                         if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (!ok) break;
                     // rank-r bf16 branch: one more accumulator tile, fp32
-                    if (!mbar_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    const bool rank_mine = mine(b);
+                    if (rank_mine && !mbar_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
                     for (int lr = 0; lr < p.lr_chunks; ++lr) {
-                        if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
-                            !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                        if (!mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                         tc_fence_after_sync();
                         const uint32_t a_lo = desc_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (A_BYTES >> 4);
+                        if (elect_one()) {
+                            if (rank_mine) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem_base + b * BN, desc(a_lo + 2 * k), desc(b_lo + 2 * k), idesc_bf, (lr | k) != 0);
-                        umma_commit(empty_bar(s));
+                                for (int k = 0; k < 4; ++k)
+                                    umma_bf16(tmem_base + b * BN, desc(a_lo + 2 * k), desc(b_lo + 2 * k), idesc_bf, (lr | k) != 0);
+                            }
+                            umma_commit(empty_bar(s));
+                        }
                         if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (!ok) break;
-                    umma_commit(tfull_bar(b));
+                    if (rank_mine && elect_one()) umma_commit(tfull_bar(b));
+                    if (lane == 0) TRACE_CLK(p.status, 19);
                     if (++b == NBUF) { b = 0; bph ^= 1; }
                 }
-                flush_wait(p.status, WS_MMA_OPERANDS, w_ops);
-                flush_wait(p.status, WS_MMA_TEMPTY, w_tempty);
-                flush_wait(p.status, WS_KERNEL, clock64() - t_kernel);
+                if (lane == 0 && !mma_b) {
+                    flush_wait(p.status, WS_MMA_OPERANDS, w_ops);
+                    flush_wait(p.status, WS_MMA_TEMPTY, w_tempty);
+                    flush_wait(p.status, WS_KERNEL, clock64() - t_kernel);
+                }
             }
         } else {
             // -------------------------------------------------------- nibble -> byte unpack (warps 2, 3)
@@ -368,6 +406,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     const int s = it % STAGES;
                     ok = timed_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK, w_full);
                     if (!ok) break;
+                    if (it == 0 && u == 0) TRACE_CLK(p.status, 14);
                     if (i < p.num_kb) {
                         // 16-byte piece idx = u + 64 j of the packed tile: row = idx/4 = u/4 + 16 j, piece c = u%4.
                         // The swizzle phase row%8 = (u/4)%8 and the piece do not depend on j, so every address is
@@ -404,6 +443,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     // each thread signs off its own writes (a warp-wide barrier followed by one lane's arrival costs about
                     // a hundred cycles more on this part than 32 arrivals)
                     mbar_arrive(unp_bar(s));
+                    if (it == 0 && u == 0) TRACE_CLK(p.status, 15);
                 }
             }
             if (u == 0) flush_wait(p.status, WS_UNPACK_FULL, w_full);
@@ -458,10 +498,12 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc) &&
                  timed_wait(tfull_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
             if (!ok) break;
+            if (warp == 4 && lane == 0) TRACE_CLK(p.status, 20);
             tc_fence_after_sync();
             request_chunk(b, 0, raw[0]);
 
             for (int g = 0; g < p.n_g; ++g) {
+                if (warp == 4 && lane == 0 && g == 8) TRACE_CLK(p.status, 21);
                 const int gi = g & (GPK - 1);
                 const bool last_of_kb = gi == GPK - 1 || g == p.n_g - 1;
                 const float* s_sw = sc0 + slot * (SC_BYTES / 4);
@@ -555,6 +597,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 }
             }
             if (!ok) break;
+            if (warp == 4 && lane == 0) TRACE_CLK(p.status, 22);
             // rank-r branch: an fp32 tile whose first chunk is already on its way
 #pragma unroll
             for (int c = 0; c < CHUNKS; ++c) {
@@ -573,6 +616,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
             }
             if (++b == NBUF) { b = 0; bph ^= 1; }
+            if (warp == 4 && lane == 0) TRACE_CLK(p.status, 23);
             if constexpr (!kPartials) {
                 // A lane holds 2 of the 8 columns of every block; four blocks are transposed inside the quad of lanes
                 // (two exchange steps) so that each lane ends up with all 8 columns = 16 bytes of one block and the
@@ -611,6 +655,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 }
             }
         }
+        if (warp == 4 && lane == 0) TRACE_CLK(p.status, 24);
         if (warp == 4 && lane == 0) {
             flush_wait(p.status, WS_EPI_TFULL, w_tfull);
             flush_wait(p.status, WS_EPI_SCALES, w_sc);
@@ -620,6 +665,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     // ---------------------------------------------------------------- teardown
     if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 8));  // a wait gave up: let issued MMAs finish first
+    if (mma_b && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 9));
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
