@@ -550,7 +550,7 @@ def main():
                          "scales; int4_asym: int4 with asymmetric activation codes (zero-point per group); w4a8: per-token int8 "
                          "activations, per-channel int4 weights; int4_ph: the projection form (U_h only + block-Hadamard residual), "
                          "a cheaper first stage that is not the paper's Eq. 5")
-    ap.add_argument("--gemm-tile", type=int, default=0, choices=[0, 64, 128, 192, 256, 512],
+    ap.add_argument("--gemm-tile", type=int, default=0, choices=[0, 64, 66, 128, 192, 256, 512],
                     help="output columns per tile of the second kernel (int4 / int4_asym / nvfp4): 0 = chosen per call")
     ap.add_argument("--configs", default="1,2,5",
                     help="other configurations summarised in the line (int4 format, one GPU): 1 = small memory-bound layer, "

@@ -172,19 +172,29 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
 
 /* Tuning knob of the second kernels (all four formats): output columns per tile.
  * 0 (default): chosen per call from M, N and the number of SMs (INT4: 256 columns unless 128-column tiles fill the
- * SMs so much better that they win although a narrow tile costs about 0.73 of a wide one; NVFP4 likewise with 0.6);
- * 128 or 256: forced; 192: the grouped INT4 kernel's plan with three epilogue warpgroups (64 columns per thread; the
- * other formats' kernels then choose for themselves), never chosen automatically: on the FLUX shapes it measured
- * between the other two.  Process-wide; results do not depend on it (each output element is accumulated in the same
- * order).  Other values: DIROTQ_ERR_INVALID_ARG. */
+ * SMs so much better that they win although a narrow tile costs about 0.73 of a wide one, and 64 columns when even
+ * 128-column tiles would keep under half of the SMs busy, i.e. for calls with few token rows; NVFP4 likewise with 0.6
+ * and no 64-column plan);
+ * 128 or 256: forced; 64: the grouped INT4 kernel's plan for few token rows, forced, one CTA per tile; 66: the same
+ * tiles with the K-groups of a tile cut over a cluster of up to four CTAs (partial tiles added in one of them through
+ * distributed shared memory) wherever every tile's cluster is resident at once and every CTA keeps two k-blocks; never
+ * chosen automatically, because its outputs differ from the other plans' in fp32 summation order (a bf16 step on a few
+ * values), and with 0 a token's output bits do not depend on how many tokens a call has; 192: the grouped INT4 kernel's plan
+ * with three epilogue warpgroups (64 columns per thread), never chosen automatically: on the FLUX shapes it measured
+ * between the other two; 512: the NVFP4 kernel in pairs of CTAs (clusters of two, tcgen05.mma.cta_group::2, 256 token
+ * rows x 256 columns per pair, each CTA loading its own rows and one half of the weight tile), never chosen
+ * automatically: 4-9 % faster alone on the widest FLUX layers, no change of a whole step.  A value that names a plan of
+ * one kernel leaves the other formats' kernels choosing for themselves.  Process-wide; results do not depend on it (each
+ * output element is accumulated in the same order).  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);
 
 /* Tuning knob of the first kernel (rotation): tile plan.  0 (default): chosen per call from M, K and the number of
  * SMs; 1: 128 tokens x 128 rotated columns; 2: 128 x 256; 3: 256 x 256 (two MMAs share one tile of the rotation: a
  * third fewer operand bytes per flop, no overlap of the epilogue; pays where a layer has many tiles per SM, e.g.
  * K = 12288 at M = 4608); 4: 256 x 256 per PAIR of CTAs (clusters of two: tcgen05.mma.cta_group::2, each CTA loads its
- * own 128 rows of x and half of the rotation tile; the epilogue stays overlapped).  Process-wide; results do not depend
- * on it.  Other values: DIROTQ_ERR_INVALID_ARG. */
+ * own 128 rows of x and half of the rotation tile; the epilogue stays overlapped); 5: 128 x 64 (groups of 64 only, else
+ * plan 1 is taken; for calls with few token rows, chosen when plan 1 would keep under half of the SMs busy).
+ * Process-wide; results do not depend on it.  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_rotation_tile(int plan);
 
 /* Projection form, first step (x~_h = x U_hb): with few token-row tiles (M / 128 at most half the number of SMs) and K >= 2048 the

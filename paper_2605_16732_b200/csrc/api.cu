@@ -653,7 +653,7 @@ dirotq_status_t dirotq_set_dependent_launch(int enabled) {
 
 dirotq_status_t dirotq_set_gemm_tile(int columns) {
     // 64 and 192: plans of the grouped INT4 second kernel only; 512: 256 columns per pair of CTAs, NVFP4 second kernel only
-    const bool int4_only = columns == 64 || columns == 192;
+    const bool int4_only = columns == 64 || columns == 66 || columns == 192;  // 66: 64 columns with the reduction split over a cluster
     dirotq_status_t st = set_w4a4_tile_columns(columns == 512 ? 0 : columns);
     if (st == DIROTQ_OK) st = set_nvfp4_tile_columns(int4_only ? 0 : columns);
     return st != DIROTQ_OK ? st : set_w4a8_tile_columns(int4_only || columns == 512 ? 0 : columns);

@@ -325,6 +325,47 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
+// The same launch as clusters of `cluster` CTAs (`grid` a multiple of it).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_clusters(void (*kern)(KArgs...), int grid, int cluster, int block, size_t smem, cudaStream_t stream,
+                                          bool dependent, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    const bool pdl = dependent && dependent_launch_enabled();
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
+// How many clusters of `cluster` CTAs of `kern` the current device holds at once (0 on error).
+template <typename... KArgs>
+inline int max_active_clusters(void (*kern)(KArgs...), int cluster, int block, size_t smem) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(cluster));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
 // The same launch as clusters of two CTAs (`grid` must be even).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel_pairs(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, bool dependent,

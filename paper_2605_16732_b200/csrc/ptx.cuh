@@ -29,10 +29,13 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     return t;
 }
 
-// Diagnostic build (-DDIROTQ_TRACE): block 0 stamps the SM clock at marked points of each role into the 8-byte slots
+// Diagnostic build (-DDIROTQ_TRACE, optionally -DDIROTQ_TRACE_BLOCK=n): block n (0) stamps the SM clock at marked points of each role into the 8-byte slots
 // 9..31 of the workspace's status block, for reading a small call's critical path off the device.
 #ifdef DIROTQ_TRACE
-#define TRACE_CLK(status, slot) do { if (blockIdx.x == 0) reinterpret_cast<volatile unsigned long long*>(status)[slot] = clock64(); } while (0)
+#ifndef DIROTQ_TRACE_BLOCK
+#define DIROTQ_TRACE_BLOCK 0
+#endif
+#define TRACE_CLK(status, slot) do { if (blockIdx.x == DIROTQ_TRACE_BLOCK) reinterpret_cast<volatile unsigned long long*>(status)[slot] = clock64(); } while (0)
 #else
 #define TRACE_CLK(status, slot) do {} while (0)
 #endif
@@ -266,6 +269,74 @@ __device__ __forceinline__ void cluster_sync_all() {
 // Arrival on a barrier given by its shared::cluster address (this CTA's or the other's).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+// The same with release ordering at cluster scope: what this thread wrote into another CTA's shared memory before the
+// arrival is visible to a thread of that CTA that then passes mbar_wait_cluster on the barrier.
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {  // acquire at cluster scope
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait like mbar_wait, for a barrier that threads of other CTAs of the cluster arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                                  unsigned long long limit_ns = kWaitLimitNs) {
+    unsigned long long t0 = 0;
+#pragma unroll 1
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((spins & 255u) == 0) {
+            if (*abort_flag != 0) return false;
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > limit_ns) {
+                *abort_flag = code;
+                atomicCAS(status, 0, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster (destination and barrier given by
+// their shared::cluster addresses); the bytes are counted on that barrier.  Addresses and size: multiples of 16.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t cluster_dst, uint32_t src, uint32_t bytes, uint32_t cluster_bar) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(cluster_dst),
+                 "r"(src), "r"(bytes), "r"(cluster_bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void st_shared_u64(uint32_t addr, uint64_t v) {
+    asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+
+// 8-byte store into the shared memory of a CTA of the cluster (address from map_to_cta) and 8-byte load from this CTA's own.
+__device__ __forceinline__ void st_cluster_u64(uint32_t cluster_addr, uint64_t v) {
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(cluster_addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint64_t ld_shared_u64(uint32_t addr) {
+    uint64_t v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+    return v;
 }
 
 // 2-D tiled load into THIS CTA's shared memory whose bytes are counted on a barrier given by its shared::cluster

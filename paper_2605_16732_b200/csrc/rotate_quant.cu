@@ -218,8 +218,13 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     static_assert(!PAIR || (BM == 128 && BN == 256 && !PH), "pairs: 128 rows per CTA, 256 columns per pair");
     constexpr int B_ROWS = PAIR ? BN / 2 : BN;  // rows of the rotation tile this CTA holds
     static_assert(BN >= G, "a tile holds whole groups");
-    constexpr int STAGES = BM == 256 ? 3 : (B_ROWS == 256 ? STAGES_WIDE : B_ROWS == 128 ? 6 : 8);
-    constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;
+    // 64-column tiles (few token rows) put TWO k-blocks into a stage: there the kernel is paced by the producer's and the MMA
+    // issuer's chains of single-thread instructions per stage (wait, expect, loads; wait, fence, MMAs, commit), so fewer, larger
+    // stages shorten it (the split reduction of the projection form's first step never runs with this plan)
+    constexpr int KSUB = BN == 64 ? 2 : 1;
+    constexpr int SUB_BYTES = A_BYTES + B_ROWS * BK * 2;  // one k-block's operands: [x tile | rotation tile]
+    constexpr int STAGES = BM == 256 ? 3 : (B_ROWS == 256 ? STAGES_WIDE : B_ROWS == 128 ? 6 : 4);
+    constexpr int STAGE_BYTES = KSUB * SUB_BYTES;
     constexpr int ACC_BUFS = BM == 256 ? 1 : 2;
     static_assert(STAGES * STAGE_BYTES == STAGES_WIDE * STAGE_BYTES_WIDE && STAGE_BYTES % 1024 == 0, "ring layout");
     const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
@@ -321,12 +326,21 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
                 // a split reduction is dealt out k-block by k-block: range sp takes k-blocks sp, sp + ksplit, ... (measured the
                 // same as contiguous ranges)
-                for (int kb = sp; kb < num_kb; kb += p.ksplit, ++it) {
+                for (int kb = sp; kb < num_kb; kb += p.ksplit * KSUB, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t sa = smem_base + s * STAGE_BYTES;
                     if (!elect_one()) continue;
+                    if constexpr (KSUB > 1) {
+                        const int nsub = min(KSUB, num_kb - kb);  // k-blocks in this stage
+                        mbar_arrive_expect_tx(full_bar(s), nsub * SUB_BYTES);
+                        for (int j = 0; j < nsub; ++j) {
+                            tma_load_2d(sa + j * SUB_BYTES, &tmap_x, full_bar(s), (kb + j) * BK, m0);
+                            tma_load_2d(sa + j * SUB_BYTES + A_BYTES, &tmap_qt, full_bar(s), (kb + j) * BK, n0);
+                        }
+                        continue;
+                    }
                     if constexpr (PAIR) {
                         // both CTAs' bytes are counted on the leader's barrier, which expects the sum
                         const uint32_t full_leader = map_to_cta(full_bar(s), 0);
@@ -396,7 +410,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
                 const int sp = tile / num_mn;
                 const int kb_begin = sp;
-                for (int kb = kb_begin; kb < num_kb; kb += p.ksplit, ++it) {
+                for (int kb = kb_begin; kb < num_kb; kb += p.ksplit * KSUB, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
@@ -405,6 +419,17 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint64_t adesc = umma_desc_sw128(sa);
                     const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
                     if (!elect_one()) continue;
+                    if constexpr (KSUB > 1) {
+                        const int nsub = min(KSUB, num_kb - kb);
+                        for (int j = 0; j < nsub; ++j) {
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                umma_bf16(d, adesc + j * (SUB_BYTES >> 4) + 2 * k, bdesc + j * (SUB_BYTES >> 4) + 2 * k, idesc,
+                                          kb != kb_begin || j != 0 || k != 0);
+                        }
+                        umma_commit(empty_bar(s));
+                        continue;
+                    }
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
                         if constexpr (PAIR) {

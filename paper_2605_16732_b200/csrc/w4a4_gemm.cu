@@ -60,21 +60,22 @@ constexpr float kAccUnit = kI8Path ? 1.0f : kWScaleFold;  // integer group sum =
 //        even 128-column tiles occupy a fraction of the SMs: there a tile's K-groups are a chain of hand-overs between the
 //        tensor core and the epilogue, whose length does not depend on the tile's width, so more, narrower tiles on more SMs
 //        shorten the call.  256 threads, no register re-partitioning (every thread may use 255).
-template <int BN>
+//    64 + SPLITK: clusters of up to four CTAs cut the K-groups of one 128 x 64 tile into contiguous ranges; each CTA rescales its
+//        range into its own fp32 accumulators, the others store theirs into the last CTA's shared memory (distributed shared
+//        memory, one cluster-scope barrier), and that CTA adds them in rank order, adds the rank-r branch and the bias, and
+//        stores.  For calls so small that the chain of K-groups per tile, not the number of tiles, sets the time.
+constexpr int SPLIT_MAX = 4;          // CTAs per cluster of the split plan
+constexpr int RED_BYTES = 128 * 64 * 4;  // one CTA's partial tile: 128 rows x 64 columns fp32
+template <int BN, bool SPLITK = false>
 struct Plan {
     static constexpr int EPI_WG = BN == 192 ? 3 : BN == 64 ? 1 : 2;  // epilogue warpgroups
     static constexpr int EPI_WARPS = 4 * EPI_WG;
-    // MMA-issuing warps.  With few token rows a tile's K-groups are a chain of single-thread instructions (wait, fence, two
-    // MMAs, commit: each tens of cycles) that paces the kernel; two warps then issue alternate accumulator tiles (the second
-    // one is the block's last warp).
-    static constexpr int MMA_WARPS = 1;
-    static constexpr int MMA_B_WARP = 4 + 4 * EPI_WG;
-    static constexpr int THREADS = 128 + 128 * EPI_WG + (MMA_WARPS == 2 ? 32 : 0);
+    static constexpr int THREADS = 128 + 128 * EPI_WG;
     static constexpr bool REPARTITION = EPI_WG > 1;            // setmaxnreg after the role split
     static constexpr int EPI_REGS = EPI_WG == 3 ? 152 : 216;  // setmaxnreg budgets: 128 * AUX + 128 * EPI_WG * EPI <= 65536
     static constexpr int AUX_REGS = EPI_WG == 3 ? 56 : 64;
     static constexpr int SC_SLOTS = BN == 192 ? 6 : 8;
-    static constexpr int STAGES = BN == 256 ? 3 : BN == 192 ? 4 : BN == 128 ? 5 : 7;
+    static constexpr int STAGES = BN == 256 ? 3 : BN == 192 ? 4 : BN == 128 ? 5 : SPLITK ? 3 : 7;
     static constexpr int BU_BYTES = BN * BKC;         // unpacked weight codes / bf16 W~_h chunk (32 KB at BN = 256)
     static constexpr int BP_BYTES = BN * BKC / 2;     // packed weight codes (TMA staging)
     static constexpr int STAGE_BYTES = A_BYTES + BU_BYTES + BP_BYTES;  // 64 KB / 40 KB
@@ -82,14 +83,17 @@ struct Plan {
     static constexpr int SC_SX_BYTES = 2 * BM * 4;    // activation scales of up to two groups
     static constexpr int SC_BYTES = SC_SW_BYTES + SC_SX_BYTES;  // 3 KB / 2 KB
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES + SC_SLOTS * SC_BYTES;
-    static constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024;
+    static constexpr int RED_OFFSET = BAR_OFFSET + 512;  // split plan: the other CTAs' partial tiles land here (last CTA)
+    static constexpr int SMEM_BYTES = BAR_OFFSET + 512 + 1024 + (SPLITK ? (SPLIT_MAX - 1) * RED_BYTES : 0);
+    static_assert(!SPLITK || BN == 64, "the split plan has 64-column tiles");
 };
+static_assert(Plan<64, true>::SMEM_BYTES <= 232448, "shared memory plan too large");
 static_assert(Plan<256>::SMEM_BYTES <= 232448 && Plan<192>::SMEM_BYTES <= 232448 && Plan<128>::SMEM_BYTES <= 232448, "shared memory plan too large");
 static_assert(Plan<128>::STAGE_BYTES % 1024 == 0 && Plan<128>::SC_BYTES % 128 == 0, "tile alignment");
 static_assert(Plan<192>::STAGE_BYTES % 1024 == 0 && Plan<192>::SC_BYTES % 128 == 0, "tile alignment");
 static_assert(Plan<64>::SMEM_BYTES <= 232448 && Plan<64>::STAGE_BYTES % 1024 == 0 && Plan<64>::SC_BYTES % 128 == 0, "tile alignment");
 static_assert(8 * (3 * Plan<128>::STAGES + 2 * 8 + 9) <= 400 && 8 * (3 * Plan<192>::STAGES + 2 * 6 + 9) <= 400 &&
-              8 * (3 * Plan<64>::STAGES + 2 * 8 + 10) <= 400, "barriers end below the words at +400");
+              8 * (3 * Plan<64>::STAGES + 2 * 8 + 9) <= 400, "barriers end below the words at +400");
 
 struct GemmKernelParams {
     int M, N, n_g, num_kb, lr_chunks;
@@ -163,13 +167,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int G, bool kPartials, int BN>
+template <int G, bool kPartials, int BN, bool SPLITK = false>
 __global__ void __launch_bounds__(Plan<BN>::THREADS, 1)
 w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
                  const __grid_constant__ CUtensorMap tmap_wscale, const __grid_constant__ CUtensorMap tmap_xscale,
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
                  const GemmKernelParams p) {
-    using P = Plan<BN>;
+    using P = Plan<BN, SPLITK>;
+    static_assert(!SPLITK || !kPartials, "the debug export runs unsplit");
     constexpr int STAGES = P::STAGES, STAGE_BYTES = P::STAGE_BYTES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES;
     constexpr int SC_SW_BYTES = P::SC_SW_BYTES, SC_BYTES = P::SC_BYTES, BAR_OFFSET = P::BAR_OFFSET;
     constexpr int SC_SLOTS = P::SC_SLOTS, NUM_EPI_WARPS = P::EPI_WARPS;
@@ -202,12 +207,27 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     const int num_m_blocks = (p.M + BM - 1) / BM;
     const int num_n_blocks = (p.N + BN - 1) / BN;
     const int num_tiles = num_m_blocks * num_n_blocks;
+    // Split plan: this CTA's range of k-blocks [kb0, kb1) and of K-groups [g0, g1) of the cluster's tile (the first ranks take
+    // one k-block more when the division leaves a rest); the LAST rank gathers the partial tiles and has the rank-r branch.
+    // (Without the split every one of these is the constant or the parameter it stands for.)
+    const uint32_t csize = SPLITK ? cluster_nctarank() : 1u, crank = SPLITK ? cluster_ctarank() : 0u;
+    const bool gathers = !SPLITK || crank == csize - 1;
+    const int split_base = SPLITK ? p.num_kb / static_cast<int>(csize) : 0, split_rest = SPLITK ? p.num_kb % static_cast<int>(csize) : 0;
+    const int kb0 = SPLITK ? static_cast<int>(crank) * split_base + min(static_cast<int>(crank), split_rest) : 0;
+    const int kb1 = SPLITK ? kb0 + split_base + (static_cast<int>(crank) < split_rest ? 1 : 0) : p.num_kb;
+    const int g0 = SPLITK ? kb0 * GPK : 0, g1 = SPLITK ? min(kb1 * GPK, p.n_g) : p.n_g;
+    const int lr_here = gathers ? p.lr_chunks : 0;
+    // (tile loops read these where they are needed, like blockIdx.x and gridDim.x themselves: held in registers across the
+    // roles' loops they cost the 256-column plan spills)
+    auto first_tile = [&]() { return SPLITK ? static_cast<int>(blockIdx.x / csize) : static_cast<int>(blockIdx.x); };
+    auto tile_stride = [&]() { return SPLITK ? static_cast<int>(gridDim.x / csize) : static_cast<int>(gridDim.x); };
+    const uint32_t red_bar = bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 9);  // split plan: "partial tiles landed" (last CTA)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(unp_bar(s), 64);  // every thread of the two unpack warps arrives for itself
-            mbar_init(empty_bar(s), P::MMA_WARPS);  // every MMA-issuing warp commits to it
+            mbar_init(empty_bar(s), 1);
         }
         for (int s = 0; s < SC_SLOTS; ++s) {
             mbar_init(scfull_bar(s), 1);
@@ -218,7 +238,11 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             mbar_init(tempty_bar(a), NUM_EPI_WARPS * 32);
         }
         mbar_init(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 8), 1);  // spare: see umma_drain
-        mbar_init(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 9), 1);  // ... of the second MMA-issuing warp
+        if constexpr (SPLITK) {
+            mbar_init(red_bar, 1);  // counts the bytes of the other CTAs' partial tiles
+            mbar_init(red_bar + 8u, 128);  // this CTA's partial tile is in its shared memory (every epilogue thread arrives)
+            if (gathers) mbar_arrive_expect_tx(red_bar, (csize - 1) * RED_BYTES);
+        }
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_codes);
@@ -234,6 +258,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     }
     tc_fence_before_sync();
     __syncthreads();
+    if constexpr (SPLITK) cluster_sync_all();  // the gathering CTA's barrier is initialised before anything arrives on it
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's own shared and tensor memory; what follows reads the first kernel's output
@@ -243,8 +268,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
     // the next layer's first kernel may be scheduled as this grid's CTAs leave their SMs (it waits for this whole grid)
     grid_launch_dependents();
 
-    const bool mma_b = P::MMA_WARPS == 2 && warp == P::MMA_B_WARP;
-    if (warp < 4 || mma_b) {
+    if (warp < 4) {
         if constexpr (P::REPARTITION) reg_dealloc<P::AUX_REGS>();
 
         if (warp == 0) {
@@ -255,10 +279,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 uint32_t it = 0, sc_it = 0;
                 long long w_empty = 0;
                 bool ok = true;
-                for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                for (int tile = first_tile(); ok && tile < num_tiles; tile += tile_stride()) {
                     const int m0 = (tile % num_m_blocks) * BM;
                     const int n0 = (tile / num_m_blocks) * BN;
-                    for (int kb = 0; kb < p.num_kb; ++kb, ++it, ++sc_it) {
+                    for (int kb = kb0; kb < kb1; ++kb, ++it, ++sc_it) {
                         const int s = it % STAGES;
                         if (!timed_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER, w_empty)) { ok = false; break; }
                         const uint32_t st = smem_base + s * STAGE_BYTES;
@@ -278,7 +302,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         }
                     }
                     if (!ok) break;
-                    for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
+                    for (int lr = 0; lr < lr_here; ++lr, ++it) {
                         const int s = it % STAGES;
                         if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                         const uint32_t st = smem_base + s * STAGE_BYTES;
@@ -306,7 +330,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                 }
             }
-        } else if (warp == 1 || mma_b) {
+        } else if (warp == 1) {
             // -------------------------------------------------------- MMA issuer
             // One thread, and every instruction it executes waits its turn behind the two epilogue warps of its
             // scheduler, so its loop is kept short: stage index, parities and the operand descriptors are carried
@@ -322,26 +346,21 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 auto desc = [&](uint32_t lo) { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
                 uint32_t s = 0, ph = 0;        // stage of the operand ring and its parity
                 uint32_t b = 0, bph = 1;       // accumulator tile and the parity its "empty" barrier is waited with
-                // two issuing warps: this one takes the accumulator tiles of its parity (their number is even), follows
-                // every stage, and commits to every stage's "empty" barrier, which counts both warps
-                const uint32_t my = mma_b ? 1u : 0u;
-                auto mine = [&](uint32_t tile_idx) { return P::MMA_WARPS == 1 || (tile_idx & 1u) == my; };
                 long long w_ops = 0, w_tempty = 0;
                 const long long t_kernel = clock64();
                 bool ok = true;
-                for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                    int groups_left = p.n_g;
-                    for (int kb = 0; ok && kb < p.num_kb; ++kb) {
+                for (int tile = first_tile(); ok && tile < num_tiles; tile += tile_stride()) {
+                    int groups_left = g1 - g0;
+                    for (int kb = kb0; ok && kb < kb1; ++kb) {
                         // the unpack warps arrive after they have seen the stage's loads land (one barrier for both operands), so
                         // their barrier covers the activation codes as well
                         if (!timed_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_ops)) { ok = false; break; }
-                        if (lane == 0) { if (kb == 0) TRACE_CLK(p.status, 16); if (kb == 4) TRACE_CLK(p.status, 17); if (kb == p.num_kb - 1) TRACE_CLK(p.status, 18); }
+                        if (lane == 0) { if (kb == kb0) TRACE_CLK(p.status, 16); if (kb == 4) TRACE_CLK(p.status, 17); if (kb == kb1 - 1) TRACE_CLK(p.status, 18); }
                         tc_fence_after_sync();
                         const uint32_t a_lo = desc_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
                         for (int gi = 0; gi < GPK; ++gi) {
                             if (gi < groups_left) {
-                              if (mine(b)) {
                                 if (!timed_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA, w_tempty)) { ok = false; break; }
                                 tc_fence_after_sync();
                                 if (elect_one()) {
@@ -355,7 +374,6 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                     }
                                     umma_commit(tfull_bar(b));
                                 }
-                              }
                                 if (++b == NBUF) { b = 0; bph ^= 1; }
                             }
                         }
@@ -365,30 +383,28 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (!ok) break;
+                    if (SPLITK && lr_here == 0) continue;  // split plan: only the gathering CTA has the rank-r branch
                     // rank-r bf16 branch: one more accumulator tile, fp32
-                    const bool rank_mine = mine(b);
-                    if (rank_mine && !mbar_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    if (!mbar_wait(tempty_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
-                    for (int lr = 0; lr < p.lr_chunks; ++lr) {
+                    for (int lr = 0; lr < lr_here; ++lr) {
                         if (!mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                         tc_fence_after_sync();
                         const uint32_t a_lo = desc_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (A_BYTES >> 4);
                         if (elect_one()) {
-                            if (rank_mine) {
 #pragma unroll
-                                for (int k = 0; k < 4; ++k)
-                                    umma_bf16(tmem_base + b * BN, desc(a_lo + 2 * k), desc(b_lo + 2 * k), idesc_bf, (lr | k) != 0);
-                            }
+                            for (int k = 0; k < 4; ++k)
+                                umma_bf16(tmem_base + b * BN, desc(a_lo + 2 * k), desc(b_lo + 2 * k), idesc_bf, (lr | k) != 0);
                             umma_commit(empty_bar(s));
                         }
                         if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (!ok) break;
-                    if (rank_mine && elect_one()) umma_commit(tfull_bar(b));
+                    if (elect_one()) umma_commit(tfull_bar(b));
                     if (lane == 0) TRACE_CLK(p.status, 19);
                     if (++b == NBUF) { b = 0; bph ^= 1; }
                 }
-                if (lane == 0 && !mma_b) {
+                if (lane == 0) {
                     flush_wait(p.status, WS_MMA_OPERANDS, w_ops);
                     flush_wait(p.status, WS_MMA_TEMPTY, w_tempty);
                     flush_wait(p.status, WS_KERNEL, clock64() - t_kernel);
@@ -400,14 +416,14 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             uint32_t it = 0;
             long long w_full = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int items = p.num_kb + p.lr_chunks;
+            for (int tile = first_tile(); ok && tile < num_tiles; tile += tile_stride()) {
+                const int items = (kb1 - kb0) + lr_here;
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
                     ok = timed_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK, w_full);
                     if (!ok) break;
                     if (it == 0 && u == 0) TRACE_CLK(p.status, 14);
-                    if (i < p.num_kb) {
+                    if (i < kb1 - kb0) {
                         // 16-byte piece idx = u + 64 j of the packed tile: row = idx/4 = u/4 + 16 j, piece c = u%4.
                         // The swizzle phase row%8 = (u/4)%8 and the piece do not depend on j, so every address is
                         // a per-thread base plus a compile-time offset.
@@ -485,7 +501,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             tc_fence_before_sync();
             mbar_arrive(tempty_bar(buf));  // all lanes arrive (see the unpack warps' note on the cost of electing one)
         };
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        for (int tile = first_tile(); ok && tile < num_tiles; tile += tile_stride()) {
             const int m0 = (tile % num_m_blocks) * BM;
             const int n0 = (tile / num_m_blocks) * BN;
             const int rbase = m0 + q * 32 + lr4;  // this thread's rows: rbase + 8 i, i = 0..3
@@ -494,15 +510,18 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 #pragma unroll
             for (int j = 0; j < HB / 2; ++j) acc2[j] = 0ull;
 
-            // first scales and first accumulator tile of this output tile
-            ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc) &&
-                 timed_wait(tfull_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
-            if (!ok) break;
-            if (warp == 4 && lane == 0) TRACE_CLK(p.status, 20);
-            tc_fence_after_sync();
-            request_chunk(b, 0, raw[0]);
+            // first scales and first accumulator tile of this output tile (split plan: of this CTA's range, which may be
+            // empty, and only the gathering CTA has a rank-r tile)
+            if (!SPLITK || g1 > g0) ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc);
+            if (!SPLITK || g1 > g0 || lr_here > 0) {
+                ok = ok && timed_wait(tfull_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
+                if (!ok) break;
+                if (warp == 4 && lane == 0) TRACE_CLK(p.status, 20);
+                tc_fence_after_sync();
+                request_chunk(b, 0, raw[0]);
+            }
 
-            for (int g = 0; g < p.n_g; ++g) {
+            for (int g = g0; g < g1; ++g) {
                 if (warp == 4 && lane == 0 && g == 8) TRACE_CLK(p.status, 21);
                 const int gi = g & (GPK - 1);
                 const bool last_of_kb = gi == GPK - 1 || g == p.n_g - 1;
@@ -519,7 +538,8 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 // what comes after this tile: the next group's, or the rank-r tile
                 const uint32_t nb = b + 1 == NBUF ? 0 : b + 1, nbph = b + 1 == NBUF ? bph ^ 1 : bph;
                 const uint32_t nslot = slot + 1 == SC_SLOTS ? 0 : slot + 1, nsph = slot + 1 == SC_SLOTS ? sph ^ 1 : sph;
-                const bool new_scales = last_of_kb && g + 1 < p.n_g;
+                const bool new_scales = last_of_kb && g + 1 < g1;
+                const bool more = !SPLITK || g + 1 < g1 || lr_here > 0;  // another accumulator tile follows (always, unless split)
                 bool ahead = false;
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
@@ -542,7 +562,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     } else {
                         // the whole tile is in registers: hand it back to the MMA warp, and look at the next one
                         release_tile(b);
-                        ahead = mbar_test_wait(tfull_bar(nb), nbph) && (!new_scales || mbar_test_wait(scfull_bar(nslot), nsph));
+                        ahead = more && mbar_test_wait(tfull_bar(nb), nbph) && (!new_scales || mbar_test_wait(scfull_bar(nslot), nsph));
                         if (ahead) {
                             tc_fence_after_sync();
                             request_chunk(nb, 0, raw[0]);  // CHUNKS is even: the last chunk sits in raw[1]
@@ -588,7 +608,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 }
                 b = nb;
                 bph = nbph;
-                if (!ahead) {
+                if (!ahead && more) {
                     if (new_scales) ok = timed_wait(scfull_bar(slot), sph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_sc);
                     ok = ok && timed_wait(tfull_bar(b), bph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE, w_tfull);
                     if (!ok) break;
@@ -599,24 +619,51 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             if (!ok) break;
             if (warp == 4 && lane == 0) TRACE_CLK(p.status, 22);
             // rank-r branch: an fp32 tile whose first chunk is already on its way
+            if (!SPLITK || lr_here > 0) {
 #pragma unroll
-            for (int c = 0; c < CHUNKS; ++c) {
-                uint32_t (&cur)[32] = raw[c & 1];
-                tmem_ld_wait();
-                tmem_ld_fence(cur);
-                if (c < CHUNKS - 1) request_chunk(b, c + 1, raw[(c + 1) & 1]);
-                else release_tile(b);
+                for (int c = 0; c < CHUNKS; ++c) {
+                    uint32_t (&cur)[32] = raw[c & 1];
+                    tmem_ld_wait();
+                    tmem_ld_fence(cur);
+                    if (c < CHUNKS - 1) request_chunk(b, c + 1, raw[(c + 1) & 1]);
+                    else release_tile(b);
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                    for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int cb = 0; cb < 4; ++cb) {
-                        const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
-                        const int a = (c * 4 + cb) * 4 + i;
-                        acc2[a] = add_f32x2(acc2[a], pack_u32x2(cur[pidx], cur[pidx + 1]));
-                    }
+                        for (int cb = 0; cb < 4; ++cb) {
+                            const int pidx = 16 * (i >> 1) + 4 * cb + 2 * (i & 1);
+                            const int a = (c * 4 + cb) * 4 + i;
+                            acc2[a] = add_f32x2(acc2[a], pack_u32x2(cur[pidx], cur[pidx + 1]));
+                        }
+                }
+                if (++b == NBUF) { b = 0; bph ^= 1; }
             }
-            if (++b == NBUF) { b = 0; bph ^= 1; }
             if (warp == 4 && lane == 0) TRACE_CLK(p.status, 23);
+            if constexpr (SPLITK) {
+                // The partial tiles meet in the last CTA of the cluster.  Every other CTA's epilogue threads put their 32
+                // register pairs into their own shared memory (the operand ring, idle by now: every MMA of this CTA has
+                // completed), word j of thread t at [j][t]; one thread then sends the 32 KB to the gathering CTA with a bulk
+                // copy that counts its bytes on that CTA's barrier.  The gathering thread t holds the same rows and columns
+                // in every CTA and adds the partial tiles in rank order.
+                const uint32_t et = threadIdx.x - 128u;
+                const uint32_t red_base = smem_base + P::RED_OFFSET;
+                if (!gathers) {
+#pragma unroll
+                    for (int j = 0; j < HB / 2; ++j) st_shared_u64(smem_base + j * 1024u + et * 8u, acc2[j]);
+                    fence_proxy_async_smem();       // these writes -> visible to the copy engine
+                    mbar_arrive(red_bar + 8u);
+                    if (et == 0 && mbar_wait(red_bar + 8u, 0, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE))  // a bounded wait, like all
+                        bulk_copy_to_cluster(map_to_cta(red_base + crank * RED_BYTES, csize - 1), smem_base, RED_BYTES,
+                                             map_to_cta(red_bar, csize - 1));
+                    continue;  // one tile per cluster: nothing else to do (the cluster meets once more before anyone leaves)
+                }
+                if (!mbar_wait(red_bar, 0, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
+                for (uint32_t r = 0; r + 1 < csize; ++r) {
+#pragma unroll
+                    for (int j = 0; j < HB / 2; ++j)
+                        acc2[j] = add_f32x2(acc2[j], ld_shared_u64(red_base + r * RED_BYTES + j * 1024u + et * 8u));
+                }
+            }
             if constexpr (!kPartials) {
                 // A lane holds 2 of the 8 columns of every block; four blocks are transposed inside the quad of lanes
                 // (two exchange steps) so that each lane ends up with all 8 columns = 16 bytes of one block and the
@@ -665,9 +712,9 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     // ---------------------------------------------------------------- teardown
     if (warp == 1 && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 8));  // a wait gave up: let issued MMAs finish first
-    if (mma_b && lane == 0 && *abort_flag != 0) umma_drain(bar_base + 8u * (3 * STAGES + 2 * SC_SLOTS + 9));
     tc_fence_before_sync();
     __syncthreads();
+    if constexpr (SPLITK) cluster_sync_all();  // no CTA of the cluster leaves while another may still write into it or signal it
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, 512);
@@ -686,8 +733,9 @@ static bool narrow_tiles_pay(int M, int N, int sms) {
     return cost_narrow < 0.98 * cost_wide;
 }
 
+// split: 0 = one CTA per tile; 2..SPLIT_MAX = the split plan with clusters of that many CTAs (BN = 64, no debug export)
 template <int BN>
-static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream) {
+static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs& a, cudaStream_t stream, int split = 0) {
     const Geometry& g = L->geo;
     CUtensorMap tmap_codes, tmap_xscale, tmap_xh;
     dirotq_status_t st;
@@ -718,6 +766,17 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
     else           kern = dbg ? w4a4_gemm_kernel<128, true, BN> : w4a4_gemm_kernel<128, false, BN>;
     static SmemOptIn<4> opt_in;  // one per instantiation of this launcher, i.e. per tile width
     const int vi = (g.G == 64 ? 0 : 2) + (dbg ? 1 : 0);
+    if constexpr (BN == 64) {
+        if (split >= 2 && !dbg) {
+            const KernelFn ks = g.G == 64 ? w4a4_gemm_kernel<64, false, 64, true> : w4a4_gemm_kernel<128, false, 64, true>;
+            static SmemOptIn<2> opt_in_split;
+            if (!opt_in_split.ensure(ks, g.G == 64 ? 0 : 1, L->device, Plan<64, true>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+            const cudaError_t es = launch_kernel_clusters(ks, num_tiles * split, split, Plan<64>::THREADS, Plan<64, true>::SMEM_BYTES,
+                                                          stream, true, tmap_codes, L->tmap_wpacked64, L->tmap_wscale64, tmap_xscale,
+                                                          tmap_xh, L->tmap_wh64, p);
+            return es == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
+        }
+    }
     if (!opt_in.ensure(kern, vi, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     const cudaError_t err = launch_kernel(kern, grid, Plan<BN>::THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
                                           BN == 64 ? L->tmap_wpacked64 : BN == 128 ? L->tmap_wpacked128 : BN == 192 ? L->tmap_wpacked192 : L->tmap_wpacked,
@@ -729,10 +788,10 @@ static dirotq_status_t launch_w4a4_gemm_bn(const dirotq_layer* L, const GemmArgs
 
 }  // namespace
 
-static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 64 / 128 / 192 / 256: forced
+static std::atomic<int> g_tile_columns{0};  // 0: chosen per call; 64 / 128 / 192 / 256: forced; 66: 64 columns, split plan where it applies
 
 dirotq_status_t set_w4a4_tile_columns(int columns) {
-    if (columns != 0 && columns != 64 && columns != 128 && columns != 192 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
+    if (columns != 0 && columns != 64 && columns != 66 && columns != 128 && columns != 192 && columns != 256) return DIROTQ_ERR_INVALID_ARG;
     g_tile_columns.store(columns);
     return DIROTQ_OK;
 }
@@ -743,7 +802,36 @@ dirotq_status_t launch_w4a4_gemm(const dirotq_layer* L, const GemmArgs& a, cudaS
     // few token rows: when even 128-column tiles would keep fewer than half of the SMs busy, 64-column tiles on twice as many
     const int sms = sm_count(L->device);
     const long t128 = static_cast<long>((a.M + BM - 1) / BM) * ((L->geo.N + 127) / 128);
-    if (forced == 64 || (forced == 0 && 2 * t128 <= sms)) return launch_w4a4_gemm_bn<64>(L, a, stream);
+    if (forced == 64 || forced == 66 || (forced == 0 && 2 * t128 <= sms)) {
+        // The split plan: the largest cluster (4, 3 or 2 CTAs over the k-blocks of a tile) that leaves every CTA at least two
+        // k-blocks and whose clusters, one per tile, are all resident at once (asked of the runtime once per device and size).
+        // Only on request (knob value 66): the partial tiles are added in another order than one CTA adds the groups, and by
+        // default a token's output bits do not depend on how many other tokens the call has.  Measured on the 1152 -> 1152 layer
+        // at M = 256: 14.5 against 15.1 us per layer in graph replay.
+        int split = 0;
+        if (forced == 66 && a.partials == nullptr) {
+            const long t64 = static_cast<long>((a.M + BM - 1) / BM) * ((L->geo.N + 63) / 64);
+            const int num_kb = (L->geo.K_lp + BKC - 1) / BKC;
+            static std::atomic<int> resident[64][SPLIT_MAX + 1];  // 0: not asked yet; else clusters resident at once + 1
+            for (int c = SPLIT_MAX; c >= 2 && split == 0; --c) {
+                if (num_kb / c < 2) continue;
+                const int dev = L->device;
+                int have = dev >= 0 && dev < 64 ? resident[dev][c].load() : 0;
+                if (have == 0) {
+                    // (the question needs the kernel's shared-memory limit raised first; both group sizes have the same footprint)
+                    if (cudaFuncSetAttribute(w4a4_gemm_kernel<64, false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Plan<64, true>::SMEM_BYTES) != cudaSuccess) {
+                        cudaGetLastError();
+                        break;
+                    }
+                    have = 1 + max_active_clusters(w4a4_gemm_kernel<64, false, 64, true>, c, Plan<64>::THREADS, Plan<64, true>::SMEM_BYTES);
+                    if (dev >= 0 && dev < 64) resident[dev][c].store(have);
+                }
+                if (t64 <= have - 1) split = c;
+            }
+        }
+        return launch_w4a4_gemm_bn<64>(L, a, stream, split);
+    }
     const bool narrow = forced ? forced == 128 : narrow_tiles_pay(a.M, L->geo.N, sm_count(L->device));
     return narrow ? launch_w4a4_gemm_bn<128>(L, a, stream) : launch_w4a4_gemm_bn<256>(L, a, stream);
 }

@@ -72,7 +72,7 @@ def test_null_and_bad_handles_are_rejected(L):
 
 
 def test_knobs_validate_their_argument_without_a_gpu(L):
-    for ok in (0, 64, 128, 192, 256, 512, 0):
+    for ok in (0, 64, 66, 128, 192, 256, 512, 0):
         assert L.dirotq_set_gemm_tile(ok) == 0
     for bad in (-1, 96, 160, 384, 1024):
         assert L.dirotq_set_gemm_tile(bad) == 1

@@ -22,20 +22,20 @@ def tile(request):
     dq.dirotq_set_gemm_tile(0)
 
 
-@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 66, 128, 192, 256], indirect=True)
 def test_parity_group64_ragged_everything(tile):
     # N = 400: ragged in both tile widths; M = 300: ragged rows; K_l = 496: ragged last group
     spec = synth.LayerSpec(K=512, N=400, r=16, G=64, model=synth.FLUX, seed=31, calib_tokens=1024)
     print(tile, test_gpu_parity._run_case(spec, M=300))
 
 
-@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 66, 128, 192, 256], indirect=True)
 def test_parity_group128_rank128(tile):
     spec = synth.LayerSpec(K=768, N=640, r=128, G=128, model=synth.FLUX, seed=32, calib_tokens=1024)
     print(tile, test_gpu_parity._run_case(spec, M=257, with_bias=False))
 
 
-@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 66, 128, 192, 256], indirect=True)
 def test_parity_pixart_projection_many_tiles(tile):
     # 8 row blocks x 9 (or 5) column blocks: several tiles per CTA are not reached on one GPU with 148 SMs, but the
     # tile -> (row block, column block) mapping and the ring phases across k-blocks are
@@ -43,7 +43,7 @@ def test_parity_pixart_projection_many_tiles(tile):
     print(tile, test_gpu_parity._run_case(spec, M=1024, check_rot=False))
 
 
-@pytest.mark.parametrize("tile", [64, 128, 192, 256], indirect=True)
+@pytest.mark.parametrize("tile", [64, 66, 128, 192, 256], indirect=True)
 def test_parity_asymmetric_codes(tile):
     spec = synth.LayerSpec(K=640, N=400, r=32, G=64, model=synth.PIXART, seed=34, calib_tokens=1024)
     print(tile, test_gpu_asym._run_case(spec, M=200, shift=1.5))
@@ -60,7 +60,7 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
     ws = dq.alloc_workspace(layer, M)
     outs = {}
     try:
-        for cols in (0, 64, 128, 192, 256):
+        for cols in (0, 64, 66, 128, 192, 256):
             dq.dirotq_set_gemm_tile(cols)
             y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
             dq.dirotq_linear(x, layer, y, ws)
@@ -69,7 +69,7 @@ def test_both_widths_give_the_same_bits_and_automatic_choice_is_one_of_them():
             outs[cols] = y.view(torch.int16).clone()
         # several tiles per CTA here (33 row blocks x 9 column blocks on 148 SMs)
         assert torch.equal(outs[128], outs[256]) and torch.equal(outs[192], outs[256]) and torch.equal(outs[0], outs[128])
-        assert torch.equal(outs[64], outs[256])
+        assert torch.equal(outs[64], outs[256]) and torch.equal(outs[66], outs[256])  # 66 applies to calls with few tiles only
         with pytest.raises(dq.DirotqError):
             dq.dirotq_set_gemm_tile(96)
     finally:
@@ -219,6 +219,37 @@ def test_few_token_rows_take_the_narrow_plans(M):
     # 64-column tiles (nothing forced here)
     spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=95)
     print(M, test_gpu_parity._run_case(spec, M=M))
+
+
+def test_split_reduction_against_one_cta_per_tile():
+    # knob 66: the K-groups of a 128 x 64 tile cut over a cluster of CTAs whose partial tiles meet in one of them through
+    # distributed shared memory.  The partial sums are added in another order than one CTA adds the groups, so the outputs
+    # agree to fp32 rounding (a bf16 step where a value sits on a rounding boundary), not bit for bit.
+    spec = synth.LayerSpec(K=1152, N=1152, r=32, G=64, model=synth.PIXART, seed=97)
+    for M in (256, 130):
+        inp = synth.make_layer_inputs(spec, M, with_bias=True)
+        dev = "cuda"
+        layer = dq.dirotq_prepare_layer(torch.from_numpy(inp["W"]).to(dev), torch.from_numpy(inp["Q"]).to(dev), spec.r, spec.G,
+                                        bias=bits_to_bf16_tensor(inp["bias"]))
+        x = bits_to_bf16_tensor(inp["x"])
+        ws = dq.alloc_workspace(layer, M)
+        outs = {}
+        try:
+            for cols in (64, 66):
+                dq.dirotq_set_gemm_tile(cols)
+                y = torch.zeros((M, spec.N), dtype=torch.bfloat16, device=dev)
+                for _ in range(3):  # consecutive calls: the barriers and the landing area start afresh every launch
+                    dq.dirotq_linear(x, layer, y, ws)
+                torch.cuda.synchronize()
+                assert dq.dirotq_workspace_status(ws) == 0
+                outs[cols] = y.float().clone()
+        finally:
+            dq.dirotq_set_gemm_tile(0)
+        a, b = outs[64], outs[66]
+        rms = float(a.pow(2).mean().sqrt())
+        assert float((a - b).abs().max()) <= 2.0 ** -7 * float(a.abs().max()) + 1e-6 * rms  # at most one bf16 step of the largest value
+        assert float((a != b).float().mean()) < 0.02
+        layer.close()
 
 
 def test_few_token_rows_other_formats():
