@@ -182,8 +182,9 @@ DIROTQ_API dirotq_status_t dirotq_int_gemm_debug(const int8_t* act_codes, int M,
  * values), and with 0 a token's output bits do not depend on how many tokens a call has; 192: the grouped INT4 kernel's plan
  * with three epilogue warpgroups (64 columns per thread), never chosen automatically: on the FLUX shapes it measured
  * between the other two; 512: the NVFP4 kernel in pairs of CTAs (clusters of two, tcgen05.mma.cta_group::2, 256 token
- * rows x 256 columns per pair, each CTA loading its own rows and one half of the weight tile), never chosen
- * automatically: 4-9 % faster alone on the widest FLUX layers, no change of a whole step.  A value that names a plan of
+ * rows x 256 columns per pair, each CTA loading its own rows and one half of the weight tile), forced; 0 takes it
+ * where its schedule is the shortest (a pair does two wide tiles' work in about 0.9 of a wide tile's time: every FLUX
+ * shape at M = 4608).  A value that names a plan of
  * one kernel leaves the other formats' kernels choosing for themselves.  Process-wide; results do not depend on it (each
  * output element is accumulated in the same order).  Other values: DIROTQ_ERR_INVALID_ARG. */
 DIROTQ_API dirotq_status_t dirotq_set_gemm_tile(int columns);

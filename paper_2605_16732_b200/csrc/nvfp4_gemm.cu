@@ -211,7 +211,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        if (lane == 0) {
+        // (the whole warp walks the loops and waits, one elected lane issues: counters, addresses and coordinates stay
+        // warp-uniform, which shortens the chain of instructions per stage; the same in the MMA and copier warps)
+        {
             uint32_t it = 0;
             bool ok = true;
             for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
@@ -228,6 +230,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const int s = it % STAGES;
                     if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t st = smem_base + s * STAGE_BYTES;
+                    if (!elect_one()) continue;
                     mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES + (sfa_here + nb_here) * SF_BYTES);
                     tma_load_2d(st, &tmap_codes, full_bar(s), kb * 128, m0);             // byte coordinates
 #pragma unroll
@@ -246,6 +249,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const int s = it % STAGES;
                     if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t st = smem_base + s * STAGE_BYTES;
+                    if (!elect_one()) continue;
                     mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
                     tma_load_2d(st, &tmap_xh, full_bar(s), lr * 64, m0);
 #pragma unroll
@@ -254,7 +258,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                                     n0 + (PAIR ? static_cast<int>(cta_rank) : b) * 128);
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
                 for (uint32_t j = first; j < it; ++j) {
                     const unsigned long long t0 = globaltimer_ns();
@@ -264,7 +268,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && cta_rank == 0) {
+        if (cta_rank == 0) {
             constexpr uint32_t idesc_nv = nvfp4_idesc(TILE_ROWS, BN);
             constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, TILE_ROWS, BN);
             uint32_t it = 0, tcount = 0;
@@ -285,6 +289,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     tc_fence_after_sync();
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+                    if (!elect_one()) continue;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {  // K = 64 elements = 32 bytes per instruction
                         if constexpr (PAIR)
@@ -304,6 +309,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+                    if (!elect_one()) continue;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         if constexpr (PAIR) umma_bf16_pair(d, adesc + 2 * k, bdesc + 2 * k, idesc_bf, 1u);
@@ -312,7 +318,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);
                     else umma_commit(empty_bar(s));
                 }
-                if (ok) {
+                if (ok && elect_one()) {
                     if constexpr (PAIR) umma_commit_pair(tfull_bar(acc), 3);  // both CTAs' epilogue warps
                     else umma_commit(tfull_bar(acc));
                 }
@@ -324,7 +330,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         // the MMA thread, that thread bounded the kernel (0.137 ms on the 4608 x 3072 -> 9216 layer; 0.112 ms with one
         // copier thread, itself the bound; 0.093 ms with two).  Each copier hands its half of a stage over through an
         // mbarrier that tcgen05.commit arrives on once the copies have landed in tensor memory.
-        if (lane == 0) {
+        {
             uint32_t it = 0;
             bool ok = true;
             for (int tile = tile_first; ok && tile < num_tiles; tile += tile_step) {
@@ -335,7 +341,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     if constexpr (PAIR) {
                         if (cta_rank != 0) {
                             // this CTA's stage has landed: one word to the leader, whose copiers and MMA thread act for both
-                            if (warp == 2) mbar_arrive_cluster(map_to_cta(peer_bar(s), 0));
+                            if (warp == 2 && elect_one()) mbar_arrive_cluster(map_to_cta(peer_bar(s), 0));
                             continue;
                         }
                         if (!mbar_wait(peer_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_UNPACK)) { ok = false; break; }
@@ -344,6 +350,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                         tc_fence_after_sync();
                         const uint32_t sf = smem_base + s * STAGE_BYTES + A_BYTES + B_BYTES;
                         const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * SF_COLS;
+                        if (!elect_one()) continue;
                         if (warp == 2) {
                             // activation scales: the four K = 64 steps of the k-block, 4 columns each
 #pragma unroll
@@ -365,7 +372,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                         }
                         if constexpr (PAIR) umma_commit_pair(sfready_bar(s), 1);  // the leader's barrier only
                         else umma_commit(sfready_bar(s));
-                    } else {
+                    } else if (elect_one()) {
                         mbar_arrive(sfready_bar(s));  // a rank-r chunk: nothing to copy
                     }
                 }
@@ -522,9 +529,17 @@ dirotq_status_t launch_nvfp4_gemm(const dirotq_layer* L, const Nvfp4GemmArgs& a,
     const int sms = sm_count(L->device);
     const long m_blocks = (a.M + BM - 1) / BM;
     const long t_wide = m_blocks * ((L->geo.N + 255) / 256), t_narrow = m_blocks * ((L->geo.N + 127) / 128);
-    const bool narrow_pays = 0.6 * static_cast<double>((t_narrow + sms - 1) / sms) < 0.98 * static_cast<double>((t_wide + sms - 1) / sms);
-    if (forced == 512) return launch_nvfp4_gemm_bn<256, true>(L, a, stream);
-    const bool wide = forced ? forced == 256 : !narrow_pays;
+    const double cost_wide = static_cast<double>((t_wide + sms - 1) / sms);
+    const double cost_narrow = 0.6 * static_cast<double>((t_narrow + sms - 1) / sms);
+    // CTA pairs (256 token rows x 256 columns per cluster of two) do two wide tiles' work in about 0.9 of a wide tile's
+    // time (measured on the FLUX shapes at M = 4608: 0.078 -> 0.071, 0.033 -> 0.031, 0.106 -> 0.094, 0.078 -> 0.070 ms), on
+    // half as many schedulable units; same bits as the other plans
+    const int pair_units = sms / 2;
+    const long t_pair = ((a.M + 2 * BM - 1) / (2 * BM)) * ((L->geo.N + 255) / 256);
+    const double cost_pair = a.M > BM ? 0.9 * static_cast<double>((t_pair + pair_units - 1) / pair_units) : 1e30;
+    if (forced == 512 || (forced == 0 && cost_pair < 0.98 * cost_wide && cost_pair < 0.98 * cost_narrow))
+        return launch_nvfp4_gemm_bn<256, true>(L, a, stream);
+    const bool wide = forced ? forced == 256 : !(cost_narrow < 0.98 * cost_wide);
     return wide ? launch_nvfp4_gemm_bn<256>(L, a, stream) : launch_nvfp4_gemm_bn<128>(L, a, stream);
 }
 

@@ -134,7 +134,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // (the whole warp walks the loops and waits, one elected lane issues: counters, addresses and coordinates stay
+        // warp-uniform, which shortens the chain of instructions per stage; the same in the MMA warp)
+        {
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
@@ -144,6 +146,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     const int s = it % STAGES;
                     if (!mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                     const uint32_t st = smem_base + s * STAGE_BYTES;
+                    if (!elect_one()) continue;
                     if (i < p.num_kb) {
                         mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
                         tma_load_2d(st, &tmap_codes, full_bar(s), i * BKC, m0);
@@ -155,7 +158,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                 }
             }
-            if (!ok) {  // let the copies in flight land before the CTA's shared memory goes away
+            if (!ok && lane == 0) {  // let the copies in flight land before the CTA's shared memory goes away
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
                 for (uint32_t j = first; j < it; ++j) {
                     const unsigned long long t0 = globaltimer_ns();
@@ -165,7 +168,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        {
             constexpr uint32_t idesc_i8 = umma_idesc(2 /*s32*/, 1 /*s8*/, BM, BN);
             constexpr uint32_t idesc_bf = umma_idesc(1 /*f32*/, 1 /*bf16*/, BM, BN);
             uint32_t it = 0, tcount = 0;
@@ -178,12 +181,14 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 for (int i = 0; i < items; ++i, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
-                        !mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    // (the unpack warps arrive after they have seen the stage's loads land, and one barrier counts both operands'
+                    // bytes: their barrier covers the activation codes as well)
+                    if (!mbar_wait(unp_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
+                    if (!elect_one()) continue;
                     if (i < p.num_kb) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k) umma_i8(tacc, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
@@ -194,7 +199,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                     umma_commit(empty_bar(s));
                 }
-                if (ok) umma_commit(tfull_bar(acc));
+                if (ok && elect_one()) umma_commit(tfull_bar(acc));
             }
         }
     } else if (warp < 2 + NUM_UNPACK_WARPS) {
