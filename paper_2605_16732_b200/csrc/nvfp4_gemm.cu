@@ -57,7 +57,10 @@ struct Plan {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + (1 + NB) * SF_BYTES;  // 36 / 54 KB (pairs: 38 KB)
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int BIAS_OFFSET = BAR_OFFSET + 256;  // two buffers of a tile's bias values
-    static constexpr int SMEM_BYTES = BIAS_OFFSET + 2 * BN * 4 + 1024;
+    // pairs: one 32-row x 128-byte staging tile per epilogue warp (1024-byte aligned: 128-byte swizzle), from which the outputs
+    // leave as TMA stores
+    static constexpr int STORE_OFFSET = (BIAS_OFFSET + 2 * BN * 4 + 1023) / 1024 * 1024;
+    static constexpr int SMEM_BYTES = PAIR ? STORE_OFFSET + NUM_EPI_WARPS * 4096 + 1024 : BIAS_OFFSET + 2 * BN * 4 + 1024;
     static constexpr int TMEM_SF_BASE = ACC_BUFS * BN;    // columns 256.. hold the scale factors
     static constexpr int SF_COLS = 16 * (1 + NB);         // per stage: 16 columns for the tokens, 16 per 128 output columns
     static_assert(TMEM_SF_BASE + STAGES * SF_COLS <= 512, "tensor memory plan");
@@ -142,7 +145,7 @@ template <int BN, bool PAIR = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wcodes,
                   const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
-                  const NvKernelParams p) {
+                  const __grid_constant__ CUtensorMap tmap_y, const NvKernelParams p) {
     using P = Plan<BN, PAIR>;
     static_assert(!PAIR || BN == 256, "pairs: 256 columns per pair");
     constexpr int NB = P::NB, NB_DATA = P::NB_DATA, STAGES = P::STAGES, ACC_BUFS = P::ACC_BUFS, B_BYTES = P::B_BYTES;
@@ -163,6 +166,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 30);
     const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
     constexpr int TILE_ROWS = PAIR ? 2 * BM : BM;  // token rows of a tile (of the pair's tile)
     const int tile_first = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
@@ -189,6 +193,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         tma_prefetch_desc(&tmap_wcodes);
         tma_prefetch_desc(&tmap_xh);
         tma_prefetch_desc(&tmap_wh);
+        if constexpr (PAIR) tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) {
         if constexpr (PAIR) {
@@ -243,6 +248,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     for (int b = 0; b < nb_here; ++b)
                         bulk_load(st + A_BYTES + B_BYTES + (1 + b) * SF_BYTES,
                                   p.wsf + (static_cast<size_t>(n_blk * NB + b) * p.nkb64p + kb * 4) * 512, SF_BYTES, full_bar(s));
+                    if (it >= 6 && it <= 8) TRACE_CLK(p.status, 3 + it);
                 }
                 if (!ok) break;
                 for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
@@ -280,16 +286,16 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                 const uint32_t d = tmem_base + acc * BN;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
-                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
-                    tc_fence_after_sync();
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * SF_COLS;
-                    // the scale factors of this stage are copied into tensor memory by the copier warp
+                    // the scale factors of this stage are copied into tensor memory by the copier warps, which have seen the
+                    // stage's loads land first (in both CTAs of a pair): their barrier covers the operands as well
                     if (!mbar_wait(sfready_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
                     if (!elect_one()) continue;
+                    if (it >= 6 && it <= 8) TRACE_CLK(p.status, 15 + it);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {  // K = 64 elements = 32 bytes per instruction
                         if constexpr (PAIR)
@@ -299,12 +305,12 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     }
                     if constexpr (PAIR) umma_commit_pair(empty_bar(s), 3);  // both CTAs' producers may refill the stage
                     else umma_commit(empty_bar(s));
+                    if (it >= 6 && it <= 8) TRACE_CLK(p.status, 18 + it);
                 }
                 if (!ok) break;
                 for (int lr = 0; lr < p.lr_chunks; ++lr, ++it) {
                     const int s = it % STAGES;
-                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA) ||
-                        !mbar_wait(sfready_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
+                    if (!mbar_wait(sfready_bar(s), (it / STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t st = smem_base + s * STAGE_BYTES;
                     const uint64_t adesc = umma_desc_sw128(st);
@@ -351,6 +357,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                         const uint32_t sf = smem_base + s * STAGE_BYTES + A_BYTES + B_BYTES;
                         const uint32_t tsf = tmem_base + TMEM_SF_BASE + s * SF_COLS;
                         if (!elect_one()) continue;
+                        if (warp == 2 && it >= 6 && it <= 8) TRACE_CLK(p.status, 6 + it);
                         if (warp == 2) {
                             // activation scales: the four K = 64 steps of the k-block, 4 columns each
 #pragma unroll
@@ -372,6 +379,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                         }
                         if constexpr (PAIR) umma_commit_pair(sfready_bar(s), 1);  // the leader's barrier only
                         else umma_commit(sfready_bar(s));
+                        if (it >= 6 && it <= 8) TRACE_CLK(p.status, (warp == 2 ? 9 : 12) + it);
                     } else if (elect_one()) {
                         mbar_arrive(sfready_bar(s));  // a rank-r chunk: nothing to copy
                     }
@@ -419,14 +427,52 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             const int row = m0 + q * 32 + lane;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + half * HB;
             uint32_t raw[HB / 32][32];
+            if (warp == 4 && lane == 0 && tcount == 0) TRACE_CLK(p.status, 27);
+            if (warp == 4 && lane == 0 && tcount >= 1 && tcount <= 2) TRACE_CLK(p.status, 3 * tcount - 2);
 #pragma unroll
             for (int c = 0; c < HB / 32; ++c) tmem_ld_32x32b_x32(taddr + c * 32, raw[c]);
             tmem_ld_wait();
             tc_fence_before_sync();
+            if (warp == 4 && lane == 0 && tcount == 0) TRACE_CLK(p.status, 28);
+            if (warp == 4 && lane == 0 && tcount >= 1 && tcount <= 2) TRACE_CLK(p.status, 3 * tcount - 1);
             // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
             else mbar_arrive(tempty_bar(acc));
-            if (row < p.M) {
+            if constexpr (PAIR) {
+                // Outputs leave through shared memory: a thread holds one token row, so direct stores would be 32 scattered
+                // 16-byte pieces per instruction, and a clock trace showed 7600-9500 cycles of them per tile, during which
+                // the next tile's operand loads ran at half their rate.  Each warp converts 64 columns of its 32 rows into
+                // its own staging tile (128-byte swizzle: a quarter-warp's pieces fall into different banks) and one lane
+                // hands the tile to a TMA store, which writes whole lines and clips at M and N.
+                const float* bq = s_b + half * HB;
+                const uint32_t sbuf = smem_base + P::STORE_OFFSET + static_cast<uint32_t>(warp - 4) * 4096u;
+                const int row0 = m0 + q * 32;
+#pragma unroll
+                for (int cc = 0; cc < HB / 64; ++cc) {
+                    if (lane == 0) bulk_wait_group_read_all();  // the tile's previous contents have been read
+                    __syncwarp();
+#pragma unroll
+                    for (int p8 = 0; p8 < 8; ++p8) {
+                        const int c = cc * 2 + (p8 >> 2), j = (p8 & 3) * 8;
+                        const float4 b0 = *reinterpret_cast<const float4*>(bq + c * 32 + j);
+                        const float4 b1 = *reinterpret_cast<const float4*>(bq + c * 32 + j + 4);
+                        uint4 o;
+                        o.x = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 0]), out_scale, b0.x), fmaf(__uint_as_float(raw[c][j + 1]), out_scale, b0.y));
+                        o.y = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 2]), out_scale, b0.z), fmaf(__uint_as_float(raw[c][j + 3]), out_scale, b0.w));
+                        o.z = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 4]), out_scale, b1.x), fmaf(__uint_as_float(raw[c][j + 5]), out_scale, b1.y));
+                        o.w = pack_bf16x2(fmaf(__uint_as_float(raw[c][j + 6]), out_scale, b1.z), fmaf(__uint_as_float(raw[c][j + 7]), out_scale, b1.w));
+                        const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 128u + (static_cast<uint32_t>(p8 ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+                    }
+                    fence_proxy_async_smem();  // these writes -> visible to the copy engine
+                    __syncwarp();
+                    const int col0 = n0 + half * HB + cc * 64;
+                    if (lane == 0 && row0 < p.M && col0 < p.N) {
+                        tma_store_2d(&tmap_y, sbuf, col0, row0);
+                        bulk_commit_group();
+                    }
+                }
+            } else if (row < p.M) {
                 const float* bq = s_b + half * HB;
                 uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + n0 + half * HB;
 #pragma unroll
@@ -446,6 +492,11 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     }
                 }
             }
+            if (warp == 4 && lane == 0 && tcount == 0) TRACE_CLK(p.status, 29);
+            if (warp == 4 && lane == 0 && tcount >= 1 && tcount <= 2) TRACE_CLK(p.status, 3 * tcount);
+        }
+        if constexpr (PAIR) {
+            if (lane == 0) bulk_wait_group_all();  // this warp's stores are performed before the CTA leaves
         }
     }
 
@@ -499,15 +550,20 @@ static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4Ge
     // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand (one per CTA of a pair)
     cudaError_t err;
     if constexpr (PAIR) {
+        // the outputs leave as TMA stores of 32 rows x 64 columns (128-byte swizzle in shared memory)
+        CUtensorMap tmap_y;
+        st = encode_tmap_2d(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.y, (uint64_t)g.N, (uint64_t)a.M, (uint64_t)g.N * 2, 64, 32,
+                            CU_TENSOR_MAP_SWIZZLE_128B);
+        if (st != DIROTQ_OK) return st;
         const int pair_tiles = ((a.M + 2 * BM - 1) / (2 * BM)) * ((g.N + BN - 1) / BN);
         const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
         err = launch_kernel_pairs(nvfp4_gemm_kernel<BN, PAIR>, 2 * pairs, NUM_THREADS, Plan<BN, PAIR>::SMEM_BYTES, stream, true,
-                                  tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+                                  tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, tmap_y, p);
     } else {
         const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
         const int grid = num_tiles < sms ? num_tiles : sms;
         err = launch_kernel(nvfp4_gemm_kernel<BN>, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true,
-                            tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, p);
+                            tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, tmap_xh /* unused without pairs */, p);
     }
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
