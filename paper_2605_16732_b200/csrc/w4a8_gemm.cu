@@ -43,7 +43,9 @@ struct Plan {
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int SCALE_OFFSET = BAR_OFFSET + 256;  // two buffers of {weight scales, bias} for a tile's columns
     static constexpr int SCALE_BYTES = 2 * 2 * BN * 4;
-    static constexpr int SMEM_BYTES = SCALE_OFFSET + SCALE_BYTES + 1024;
+    // one 32-row x 64-byte staging tile per epilogue warp (64-byte swizzle), from which the outputs leave as TMA stores
+    static constexpr int STORE_OFFSET = (SCALE_OFFSET + SCALE_BYTES + 1023) / 1024 * 1024;
+    static constexpr int SMEM_BYTES = STORE_OFFSET + NUM_EPI_WARPS * 2048 + 1024;
     static constexpr int NACC = 512 / (2 * BN);  // {int32 tile, fp32 tile} pairs in tensor memory: 1 (wide) or 2 (narrow tiles)
     static_assert(8 * (3 * STAGES + 4) <= 192, "barriers must end below the two words at +192");
     static_assert(SMEM_BYTES <= 232448 && STAGE_BYTES % 1024 == 0, "shared memory plan");
@@ -76,7 +78,7 @@ template <bool kPartials, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_wpacked,
                  const __grid_constant__ CUtensorMap tmap_xh, const __grid_constant__ CUtensorMap tmap_wh,
-                 const A8KernelParams p) {
+                 const __grid_constant__ CUtensorMap tmap_y, const A8KernelParams p) {
     using P = Plan<BN>;
     constexpr int STAGES = P::STAGES, BU_BYTES = P::BU_BYTES, BP_BYTES = P::BP_BYTES, BP_OFFSET = P::BP_OFFSET;
     constexpr int STAGE_BYTES = P::STAGE_BYTES, BAR_OFFSET = P::BAR_OFFSET, SCALE_OFFSET = P::SCALE_OFFSET;
@@ -117,6 +119,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
         tma_prefetch_desc(&tmap_wpacked);
         tma_prefetch_desc(&tmap_xh);
         tma_prefetch_desc(&tmap_wh);
+        if constexpr (!kPartials) tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
@@ -326,11 +329,21 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                 *reinterpret_cast<int4*>(dst + j) =
                                     make_int4(static_cast<int32_t>(acc[j]) >> 4, static_cast<int32_t>(acc[j + 1]) >> 4,
                                               static_cast<int32_t>(acc[j + 2]) >> 4, static_cast<int32_t>(acc[j + 3]) >> 4);
-                    } else {
-                        uint16_t* yrow = p.y + static_cast<size_t>(row) * p.N + col;
+                    }
+                }
+                if constexpr (!kPartials) {
+                    // Outputs leave through shared memory: a thread holds one token row, so direct stores would be 32 scattered
+                    // 16-byte pieces per instruction (in the NVFP4 kernel a clock trace showed such stores taking thousands of
+                    // cycles per tile and slowing the operand loads).  The warp converts 32 columns of its 32 rows into its
+                    // staging tile (64-byte swizzle: a quarter-warp's pieces fall into different banks) and one lane hands
+                    // it to a TMA store, which writes whole sectors and clips at M and N.
+                    const uint32_t sbuf = smem_base + P::STORE_OFFSET + static_cast<uint32_t>(warp - (2 + NUM_UNPACK_WARPS)) * 2048u;
+                    if (lane == 0) bulk_wait_group_read_all();  // the tile's previous contents have been read
+                    __syncwarp();
+                    {
 #pragma unroll
                         for (int j = 0; j < 32; j += 8) {
-                            if (col + j < p.N) {
+                            {
                                 float o[8];
 #pragma unroll
                                 for (int t = 0; t < 8; t += 4) {
@@ -344,13 +357,25 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                                         o[t + e] = fmaf(pf * sx, sws[e], __uint_as_float(lr[j + t + e])) + bs[e];
                                     }
                                 }
-                                *reinterpret_cast<uint4*>(yrow + j) = make_uint4(pack_bf16x2(o[0], o[1]), pack_bf16x2(o[2], o[3]),
-                                                                                 pack_bf16x2(o[4], o[5]), pack_bf16x2(o[6], o[7]));
+                                const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 64u +
+                                                     (static_cast<uint32_t>((j >> 3) ^ ((lane >> 1) & 3)) << 4);
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16x2(o[0], o[1])),
+                                             "r"(pack_bf16x2(o[2], o[3])), "r"(pack_bf16x2(o[4], o[5])), "r"(pack_bf16x2(o[6], o[7]))
+                                             : "memory");
                             }
                         }
                     }
+                    fence_proxy_async_smem();  // these writes -> visible to the copy engine
+                    __syncwarp();
+                    if (lane == 0 && m0 + q * 32 < p.M && col < p.N) {
+                        tma_store_2d(&tmap_y, sbuf, col, m0 + q * 32);
+                        bulk_commit_group();
+                    }
                 }
             }
+        }
+        if constexpr (!kPartials) {
+            if (lane == 0) bulk_wait_group_all();  // this warp's stores are performed before the CTA leaves
         }
     }
 
@@ -389,9 +414,17 @@ static dirotq_status_t launch_w4a8_gemm_bn(const dirotq_layer* L, const A8GemmAr
     static SmemOptIn<2> opt_in;
     if (!opt_in.ensure(kern, dbg ? 1 : 0, L->device, Plan<BN>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     const bool narrow = BN == 128;
+    // the outputs leave as TMA stores of 32 rows x 32 columns (64-byte swizzle in shared memory); the debug export of the
+    // integer sums stores directly and is given the activation map in its place
+    CUtensorMap tmap_y = tmap_xh;
+    if (!dbg) {
+        st = encode_tmap_2d(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.y, (uint64_t)g.N, (uint64_t)a.M, (uint64_t)g.N * 2, 32, 32,
+                            CU_TENSOR_MAP_SWIZZLE_64B);
+        if (st != DIROTQ_OK) return st;
+    }
     const cudaError_t err = launch_kernel(kern, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true, tmap_codes,
                                           narrow ? L->tmap_wpacked128 : L->tmap_wpacked, tmap_xh,
-                                          narrow ? L->tmap_wh128 : L->tmap_wh, p);
+                                          narrow ? L->tmap_wh128 : L->tmap_wh, tmap_y, p);
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
 
