@@ -38,7 +38,11 @@ constexpr int A_BYTES_128 = BM_MMA * BK * 2;  // 16 KB per 128 token rows
 constexpr int B_BYTES = BN_MAX * BK * 2;  // 32 KB (a 128-column tile uses half of it)
 constexpr int STAGE_BYTES_WIDE = A_BYTES_128 + B_BYTES;
 constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, eight epilogue warps
-constexpr int SMEM_BYTES = STAGES_WIDE * STAGE_BYTES_WIDE + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// Behind the ring: 1 KB for the barriers, then one 4 KB staging tile per epilogue warp (32 rows x up to 128 bytes, swizzled),
+// from which the activation codes (or the W4A8 path's fp32 coefficients) leave as TMA stores.
+constexpr int STORE_OFFSET = STAGES_WIDE * STAGE_BYTES_WIDE + 1024;
+constexpr int SMEM_BYTES = STORE_OFFSET + 8 * 4096 + 1024 /*alignment slack*/;
+static_assert(SMEM_BYTES <= 232448, "shared memory plan");
 
 struct RotKernelParams {
     int M, K, K_l, K_lp, r, r_pad, r_pad0, ldm, n_g;
@@ -205,7 +209,7 @@ template <int G, int FMT, int BN, int BM, bool PH = (FMT == 4), int EPI_WARPS = 
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_qt,
                     const __grid_constant__ CUtensorMap tmap_x2, const __grid_constant__ CUtensorMap tmap_had,
-                    const RotKernelParams p) {
+                    const __grid_constant__ CUtensorMap tmap_out, const RotKernelParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     // The ring holds 192 KB either way; with narrow tiles it is cut into more, smaller stages: the operand stream is
@@ -266,6 +270,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
         tma_prefetch_desc(&tmap_qt);
+        if constexpr (FMT == 0 || FMT == 2 || FMT == 3 || FMT == 4) tma_prefetch_desc(&tmap_out);
         if constexpr (PH) {
             tma_prefetch_desc(&tmap_x2);
             tma_prefetch_desc(&tmap_had);
@@ -471,6 +476,27 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const uint32_t acc_ph = (tcount / ACC_BUFS) & 1;
             const int row = m0 + (BM == 256 ? half * 128 : 0) + q * 32 + lane;
             const bool row_ok = row < p.M;
+            // A thread holds one token row, so direct stores of its codes would be 16-byte pieces of 32 different rows per
+            // instruction (in the NVFP4 second kernel a clock trace showed such stores taking thousands of cycles per tile
+            // and halving the rate of the operand loads).  The INT4 codes (one byte each: G bytes per row and chunk) and the
+            // W4A8 path's fp32 coefficients (128 bytes per row at a time) go into the warp's staging tile instead, swizzled
+            // so that a quarter-warp's pieces fall into different banks, and one lane hands the tile to a TMA store
+            // (tmap_out), which writes whole sectors and clips at M and at the row's width.
+            constexpr bool STAGED = EPI_WARPS == 8 && (FMT == 0 || FMT == 2 || FMT == 3 || FMT == 4);
+            const uint32_t sbuf = smem_base + STORE_OFFSET + static_cast<uint32_t>(warp - 2) * 4096u;
+            const int row0w = row - lane;  // the warp's first row
+            auto stage_piece128 = [&](int piece, uint4 val) {  // rows of 128 bytes, 128-byte swizzle
+                const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 128u + (static_cast<uint32_t>(piece ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+            };
+            auto stage_code_piece = [&](int piece, uint4 val) {  // G one-byte codes per row: 64-byte rows (64-byte swizzle) or 128
+                if constexpr (G == 64) {
+                    const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 64u + (static_cast<uint32_t>(piece ^ ((lane >> 1) & 3)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+                } else {
+                    stage_piece128(piece, val);
+                }
+            };
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (BM == 256 ? half * 256 : acc * BN);
@@ -548,24 +574,47 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 } else if constexpr (FMT == 3) {
                     // W4A8, first pass: the rotated low-precision coefficients go out as fp32 and the token's maximum is
-                    // gathered with an atomic max (non-negative floats order like their bit patterns)
-                    if (nlow > 0 && row_ok) {
-                        float4* dst = reinterpret_cast<float4*>(p.xtilde + static_cast<size_t>(row) * p.K_lp + col0);
+                    // gathered with an atomic max (non-negative floats order like their bit patterns).  Columns of the chunk
+                    // past K_l are written too where the chunk is staged (the quantizer pass reads none of them).
+                    if (nlow > 0) {
 #pragma unroll
                         for (int b = 0; b < G / 16; ++b) {
                             if (16 * b < nlow) {
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const float4 q4 = make_float4(v[16 * b + 4 * j], v[16 * b + 4 * j + 1], v[16 * b + 4 * j + 2],
-                                                                  v[16 * b + 4 * j + 3]);
-                                    dst[4 * b + j] = q4;
-                                    tile_amax = fmaxf(tile_amax, fmaxf(fmaxf(fabsf(q4.x), fabsf(q4.y)), fmaxf(fabsf(q4.z), fabsf(q4.w))));
+                                for (int j = 0; j < 16; ++j) tile_amax = fmaxf(tile_amax, fabsf(v[16 * b + j]));
+                            }
+                        }
+                        if constexpr (STAGED) {
+#pragma unroll
+                            for (int h = 0; h < G / 32; ++h) {  // 32 floats = 128 bytes per row at a time
+                                if (lane == 0) bulk_wait_group_read_all();  // the staging tile's previous contents have been read
+                                __syncwarp();
+#pragma unroll
+                                for (int f = 0; f < 8; ++f)
+                                    stage_piece128(f, make_uint4(__float_as_uint(v[32 * h + 4 * f]), __float_as_uint(v[32 * h + 4 * f + 1]),
+                                                                 __float_as_uint(v[32 * h + 4 * f + 2]), __float_as_uint(v[32 * h + 4 * f + 3])));
+                                fence_proxy_async_smem();  // these writes -> visible to the copy engine
+                                __syncwarp();
+                                if (lane == 0 && row0w < p.M && col0 + 32 * h < p.K_lp) {
+                                    tma_store_2d(&tmap_out, sbuf, col0 + 32 * h, row0w);
+                                    bulk_commit_group();
+                                }
+                            }
+                        } else if (row_ok) {
+                            float4* dst = reinterpret_cast<float4*>(p.xtilde + static_cast<size_t>(row) * p.K_lp + col0);
+#pragma unroll
+                            for (int b = 0; b < G / 16; ++b) {
+                                if (16 * b < nlow) {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j)
+                                        dst[4 * b + j] = make_float4(v[16 * b + 4 * j], v[16 * b + 4 * j + 1], v[16 * b + 4 * j + 2],
+                                                                     v[16 * b + 4 * j + 3]);
                                 }
                             }
                         }
                     }
                 } else if constexpr (FMT == 2) {
-                    if (nlow > 0 && row_ok) {
+                    if (nlow > 0) {
                         // asymmetric: z = bf16(min), s = bf16((max - min) / 15) over the group's real elements
                         float lo = v[0], hi = v[0];
 #pragma unroll
@@ -584,29 +633,45 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         const bool slow = !(s >= 1e-30f);
                         const float inv = slow ? 0.f : __frcp_rn(s);
                         int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+                        if constexpr (STAGED) {
+                            if (lane == 0) bulk_wait_group_read_all();
+                            __syncwarp();
+                        }
                         if (!slow) {
 #pragma unroll
                             for (int b = 0; b < G / 16; ++b) {
                                 uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
                                 if (16 * b < nlow) packed = quantize16_asym<false>(v + 16 * b, z, inv, s);
-                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                                if constexpr (STAGED) stage_code_piece(b, packed);
+                                else if (row_ok) *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
                             }
                         } else {
 #pragma unroll
                             for (int b = 0; b < G / 16; ++b) {
                                 uint4 packed = make_uint4(0, 0, 0, 0);
                                 if (16 * b < nlow) packed = quantize16_asym<true>(v + 16 * b, z, inv, s);
-                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                                if constexpr (STAGED) stage_code_piece(b, packed);
+                                else if (row_ok) *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
                             }
                         }
-                        const int grp = col0 / G;
-                        p.xscale[static_cast<size_t>(grp) * p.ldm + row] = s;
-                        // the zero-point, three times, in the extra columns of the bf16 rank-r operand
-                        uint16_t* zrow = p.xh + static_cast<size_t>(row) * p.r_pad + p.r_pad0 + grp;
-                        const uint16_t zbits = *reinterpret_cast<const uint16_t*>(&zb);
-                        zrow[0] = zbits;
-                        zrow[p.n_g] = zbits;
-                        zrow[2 * p.n_g] = zbits;
+                        if constexpr (STAGED) {
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0 && row0w < p.M) {
+                                tma_store_2d(&tmap_out, sbuf, col0, row0w);
+                                bulk_commit_group();
+                            }
+                        }
+                        if (row_ok) {
+                            const int grp = col0 / G;
+                            p.xscale[static_cast<size_t>(grp) * p.ldm + row] = s;
+                            // the zero-point, three times, in the extra columns of the bf16 rank-r operand
+                            uint16_t* zrow = p.xh + static_cast<size_t>(row) * p.r_pad + p.r_pad0 + grp;
+                            const uint16_t zbits = *reinterpret_cast<const uint16_t*>(&zb);
+                            zrow[0] = zbits;
+                            zrow[p.n_g] = zbits;
+                            zrow[2 * p.n_g] = zbits;
+                        }
                     }
                 } else if (nlow > 0) {
                     // four running maxima instead of one chain of G dependent instructions
@@ -622,25 +687,37 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const float s = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(amax, 7.0f)));
                     const bool slow = !(s >= 1e-30f);  // zero or tiny scale: divide instead of multiplying
                     const float inv = slow ? 0.f : __frcp_rn(s) * kPre;
-                    if (row_ok) {
-                        int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
-                        if (!slow) {
-#pragma unroll
-                            for (int b = 0; b < G / 16; ++b) {
-                                uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
-                                if (16 * b < nlow) packed = quantize16<false>(v + 16 * b, inv, s, kPre);
-                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
-                            }
-                        } else {
-#pragma unroll
-                            for (int b = 0; b < G / 16; ++b) {
-                                uint4 packed = make_uint4(0, 0, 0, 0);
-                                if (16 * b < nlow) packed = quantize16<true>(v + 16 * b, inv, s, kPre);
-                                *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
-                            }
-                        }
-                        p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
+                    int8_t* crow = p.codes + static_cast<size_t>(row) * p.K_lp + col0;
+                    if constexpr (STAGED) {
+                        if (lane == 0) bulk_wait_group_read_all();  // the staging tile's previous contents have been read
+                        __syncwarp();
                     }
+                    if (!slow) {
+#pragma unroll
+                        for (int b = 0; b < G / 16; ++b) {
+                            uint4 packed = make_uint4(0, 0, 0, 0);  // padding slots of a ragged group
+                            if (16 * b < nlow) packed = quantize16<false>(v + 16 * b, inv, s, kPre);
+                            if constexpr (STAGED) stage_code_piece(b, packed);
+                            else if (row_ok) *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                        }
+                    } else {
+#pragma unroll
+                        for (int b = 0; b < G / 16; ++b) {
+                            uint4 packed = make_uint4(0, 0, 0, 0);
+                            if (16 * b < nlow) packed = quantize16<true>(v + 16 * b, inv, s, kPre);
+                            if constexpr (STAGED) stage_code_piece(b, packed);
+                            else if (row_ok) *reinterpret_cast<uint4*>(crow + 16 * b) = packed;
+                        }
+                    }
+                    if constexpr (STAGED) {
+                        fence_proxy_async_smem();  // these writes -> visible to the copy engine
+                        __syncwarp();
+                        if (lane == 0 && row0w < p.M) {
+                            tma_store_2d(&tmap_out, sbuf, col0, row0w);
+                            bulk_commit_group();
+                        }
+                    }
+                    if (row_ok) p.xscale[static_cast<size_t>(col0 / G) * p.ldm + row] = s;
                 }
                 if (nlow < G && row_ok) {
                     // high-precision coefficients: permuted columns >= K_l
@@ -678,6 +755,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     }
 
+    if (warp >= 2 && lane == 0) bulk_wait_group_all();  // an epilogue warp's TMA stores are performed before the CTA leaves
     // ---------------------------------------------------------------- teardown
     if constexpr (PAIR) {
         if (warp == 1 && lane == 0 && cta_rank == 0 && *abort_flag != 0) {  // a wait gave up: let issued MMAs finish first
@@ -735,6 +813,21 @@ dirotq_status_t set_rotation_plan(int plan) {
     return DIROTQ_OK;
 }
 
+// The tensor map the epilogue's TMA stores go through: the INT4 activation codes (one byte each, [M][K_lp], boxes of 32 rows x
+// one group) or, on the W4A8 path, the fp32 coefficients ([M][K_lp], boxes of 32 rows x 32 values).  NVFP4 layers store
+// directly and get a copy of `unused` (any valid map).
+static dirotq_status_t encode_out_map(CUtensorMap* out, const Geometry& g, const RotateArgs& a, const CUtensorMap& unused) {
+    if (g.fmt == 3)
+        return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xtilde, (uint64_t)g.K_lp, (uint64_t)a.M, (uint64_t)g.K_lp * 4,
+                              32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (g.fmt == 1) {
+        *out = unused;
+        return DIROTQ_OK;
+    }
+    return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K_lp, (uint64_t)a.M, (uint64_t)g.K_lp, g.G, 32,
+                          g.G == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
 dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& a, cudaStream_t stream) {
     const Geometry& g = L->geo;
     RotKernelParams p;
@@ -785,15 +878,18 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         const long pair_tiles = ((a.M + 255) / 256) * nb256;
         const int pairs = static_cast<int>(pair_tiles < sms / 2 ? pair_tiles : sms / 2);
         const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
-        using PairFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
+        using PairFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
         static const PairFn pair_table[6] = {
             rotate_quant_kernel<64, 0, 256, 128, false, 8, true>, rotate_quant_kernel<128, 0, 256, 128, false, 8, true>,
             rotate_quant_kernel<64, 1, 256, 128, false, 8, true>, rotate_quant_kernel<64, 2, 256, 128, false, 8, true>,
             rotate_quant_kernel<128, 2, 256, 128, false, 8, true>, rotate_quant_kernel<64, 3, 256, 128, false, 8, true>};
         static SmemOptIn<6> opt_in_pair;
         if (!opt_in_pair.ensure(pair_table[vi], vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+        CUtensorMap tmap_out;
+        stp = encode_out_map(&tmap_out, g, a, tmap_xp);
+        if (stp != DIROTQ_OK) return stp;
         return launch_kernel_pairs(pair_table[vi], 2 * pairs, NUM_THREADS, SMEM_BYTES, stream, g.fmt != 3, tmap_xp, L->tmap_qt128,
-                                   tmap_xp, L->tmap_qt128, p) == cudaSuccess
+                                   tmap_xp, L->tmap_qt128, tmap_out, p) == cudaSuccess
                    ? DIROTQ_OK
                    : DIROTQ_ERR_CUDA;
     }
@@ -805,13 +901,16 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
         if (st5 != DIROTQ_OK) return st5;
         const long tiles5 = mb128 * ((g.K + 63) / 64);
         const int vi5 = g.fmt == 1 ? 1 : g.fmt == 2 ? 2 : g.fmt == 3 ? 3 : 0;
-        using Fn5 = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
+        using Fn5 = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
         static const Fn5 table5[4] = {rotate_quant_kernel<64, 0, 64, 128>, rotate_quant_kernel<64, 1, 64, 128>,
                                       rotate_quant_kernel<64, 2, 64, 128>, rotate_quant_kernel<64, 3, 64, 128>};
         static SmemOptIn<4> opt_in5;
         if (!opt_in5.ensure(table5[vi5], vi5, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
+        CUtensorMap tmap_out5;
+        st5 = encode_out_map(&tmap_out5, g, a, tmap_x5);
+        if (st5 != DIROTQ_OK) return st5;
         return launch_kernel(table5[vi5], static_cast<int>(tiles5 < sms ? tiles5 : sms), NUM_THREADS, SMEM_BYTES, stream, g.fmt != 3,
-                             tmap_x5, L->tmap_qt64, tmap_x5, L->tmap_qt64, p) == cudaSuccess
+                             tmap_x5, L->tmap_qt64, tmap_x5, L->tmap_qt64, tmap_out5, p) == cudaSuccess
                    ? DIROTQ_OK
                    : DIROTQ_ERR_CUDA;
     }
@@ -823,7 +922,7 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     const long num_tiles = ((a.M + bm - 1) / bm) * ((g.K + bn - 1) / bn);
     const int grid = num_tiles < sms ? static_cast<int>(num_tiles) : sms;
     const int vi = g.fmt == 1 ? 2 : g.fmt == 3 ? 5 : (g.fmt == 2 ? (g.G == 64 ? 3 : 4) : (g.G == 64 ? 0 : 1));
-    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
     static const KernelFn table[3][6] = {
         {rotate_quant_kernel<64, 0, 128, 128>, rotate_quant_kernel<128, 0, 128, 128>, rotate_quant_kernel<64, 1, 128, 128>,
          rotate_quant_kernel<64, 2, 128, 128>, rotate_quant_kernel<128, 2, 128, 128>, rotate_quant_kernel<64, 3, 128, 128>},
@@ -838,7 +937,10 @@ dirotq_status_t launch_rotate_quantize(const dirotq_layer* L, const RotateArgs& 
     static SmemOptIn<18> opt_in;
     if (!opt_in.ensure(kern, (plan - 1) * 6 + vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     const CUtensorMap& tmap_q = plan == 1 ? L->tmap_qt128 : L->tmap_qt;
-    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, tmap_q, tmap_x, tmap_q, p) == cudaSuccess
+    CUtensorMap tmap_out;
+    st = encode_out_map(&tmap_out, g, a, tmap_x);
+    if (st != DIROTQ_OK) return st;
+    return launch_kernel(kern, grid, NUM_THREADS, SMEM_BYTES, stream, dependent, tmap_x, tmap_q, tmap_x, tmap_q, tmap_out, p) == cudaSuccess
                ? DIROTQ_OK
                : DIROTQ_ERR_CUDA;
 }
@@ -849,7 +951,7 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
     const Geometry& g = L->geo;
     if (a.xrot != nullptr) return DIROTQ_ERR_INVALID_ARG;  // there is no K-wide rotated activation in this form
     const int sms = sm_count(L->device);
-    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const RotKernelParams);
     RotKernelParams p;
     p.M = a.M; p.K = g.K; p.K_lp = g.K_lp; p.r_pad = g.r_pad; p.r_pad0 = g.r_pad0; p.ldm = a.ldm; p.n_g = g.n_g;
     p.codes = a.codes; p.xscale = a.xscale; p.xh = a.xh; p.xrot = nullptr; p.status = a.status;
@@ -880,7 +982,7 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
             tiles *= ksplit;
         }
         if (launch_kernel(k1, static_cast<int>(tiles < sms ? tiles : sms), NUM_THREADS, SMEM_BYTES, stream, true, tmap_x,
-                          L->tmap_qt128, tmap_x, L->tmap_qt128, p1) != cudaSuccess)
+                          L->tmap_qt128, tmap_x, L->tmap_qt128, tmap_x /* no codes in this step */, p1) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
         if (p1.partial != nullptr) {
             const long threads = static_cast<long>(a.M) * g.r_pad / 8;
@@ -907,8 +1009,11 @@ dirotq_status_t launch_project_quantize(const dirotq_layer* L, const RotateArgs&
         static SmemOptIn<3> opt_in2;
         if (!opt_in2.ensure(k2, vi, L->device, SMEM_BYTES)) return DIROTQ_ERR_CUDA;
         const long tiles = static_cast<long>((a.M + 127) / 128) * ((g.K + 255) / 256);
+        CUtensorMap tmap_out;
+        st = encode_out_map(&tmap_out, g, a, tmap_x);
+        if (st != DIROTQ_OK) return st;
         if (launch_kernel(k2, static_cast<int>(tiles < sms ? tiles : sms), threads2, SMEM_BYTES, stream, true, tmap_xh, L->tmap_qt,
-                          tmap_x, L->tmap_had, p2) != cudaSuccess)
+                          tmap_x, L->tmap_had, tmap_out, p2) != cudaSuccess)
             return DIROTQ_ERR_CUDA;
     }
     return DIROTQ_OK;
