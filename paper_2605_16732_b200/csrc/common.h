@@ -130,6 +130,14 @@ inline void make_asym(Geometry& g) {
     g.r_pad = (g.r_pad0 + 3 * g.n_g + 63) / 64 * 64;
 }
 
+// NVFP4 weight scale atoms (512 bytes: 128 output columns x the 4 block scales of one 64-element MMA step).  Atom `ak` (index
+// along K) of 128-column block `nb` sits at [nb / 2][ak / 4][nb % 2][ak % 4]: the eight atoms a 256-column tile needs for one
+// k-block of 256 elements are contiguous (one bulk load), and so are the four of either of its 128-column blocks.
+__host__ __device__ inline size_t wsf_atom_offset(int nb, int ak, int nkb64p) {
+    return ((((static_cast<size_t>(nb >> 1) * (nkb64p >> 2) + (ak >> 2)) * 2 + (nb & 1)) * 4) + (ak & 3)) * 512;
+}
+inline size_t wsf_bytes(int N, int nkb64p) { return static_cast<size_t>((N + 255) / 256) * 2 * nkb64p * 512; }
+
 struct BlobLayout {
     size_t off_qt;       // bf16 [K][K]: row c' = permuted output column, K-major over the input channel
     size_t off_wpacked;  // u8   [N][K_lp/2]: two INT4 codes per byte, K-major, see prepare.cu for the nibble order
@@ -137,7 +145,7 @@ struct BlobLayout {
     size_t off_wh;       // bf16 [N][r_pad]: high-precision rows of the folded weight, K-major, zero padded
     size_t off_bias;     // f32  [N]
     // NVFP4 variant: off_wpacked = E2M1 codes u8 [N][K4/2] (even k in the low nibble); off_wscale = E4M3 scale
-    // atoms u8 [ceil(N/128)][nkb64p][512]; off_meta = {float out_scale = 2^(ex+ew), int ew, int ex, uint amax bits}
+    // atoms u8, ordered as wsf_atom_offset says; off_meta = {float out_scale = 2^(ex+ew), int ew, int ex, uint amax bits}
     size_t off_meta;
     // projection form only: off_qt holds U_hb^T, bf16 [r_pad][K]; off_uh holds -V^T, bf16 [K][r_pad], with
     // V = bf16(U_hb^T H+-); off_had holds one +-1 Hadamard block, bf16 [G][G] (G = 64 for NVFP4 layers)
@@ -168,7 +176,7 @@ inline BlobLayout make_blob_layout_nvfp4(const Geometry& g) {
     b.off_uh = o;      o = align_up(o + (g.ph ? (size_t)g.K * g.r_pad * 2 : 0));
     b.off_had = o;     o = align_up(o + (g.ph ? (size_t)64 * 64 * 2 : 0));
     b.off_wpacked = o; o = align_up(o + (size_t)g.N * (g.K4 / 2));
-    b.off_wscale = o;  o = align_up(o + (size_t)((g.N + 127) / 128) * g.nkb64p * 512);
+    b.off_wscale = o;  o = align_up(o + wsf_bytes(g.N, g.nkb64p));
     b.off_wh = o;      o = align_up(o + (size_t)g.N * g.r_pad * 2);
     b.off_bias = o;    o = align_up(o + (size_t)g.N * 4);
     b.off_meta = o;    o = align_up(o + 64);

@@ -72,7 +72,7 @@ struct Plan {
 struct NvKernelParams {
     int M, N, num_kb, nkb64p, lr_chunks;
     const uint8_t* xsf;   // activation scale atoms [ceil(M/128)][nkb64p][512]
-    const uint8_t* wsf;   // weight scale atoms [ceil(N/128)][nkb64p][512]
+    const uint8_t* wsf;   // weight scale atoms, see wsf_atom_offset
     const float* bias;
     const float* out_scale;  // 2^(ex+ew)
     uint16_t* y;
@@ -245,9 +245,9 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
                     if (sfa_here)
                         bulk_load(st + A_BYTES + B_BYTES, p.xsf + (static_cast<size_t>(m_blk) * p.nkb64p + kb * 4) * 512, SF_BYTES,
                                   full_bar(s));
-                    for (int b = 0; b < nb_here; ++b)
-                        bulk_load(st + A_BYTES + B_BYTES + (1 + b) * SF_BYTES,
-                                  p.wsf + (static_cast<size_t>(n_blk * NB + b) * p.nkb64p + kb * 4) * 512, SF_BYTES, full_bar(s));
+                    // the atoms of the tile's 128-column blocks for this k-block are contiguous: one copy
+                    bulk_load(st + A_BYTES + B_BYTES + SF_BYTES, p.wsf + wsf_atom_offset(n_blk * NB, kb * 4, p.nkb64p),
+                              nb_here * SF_BYTES, full_bar(s));
                     if (it >= 6 && it <= 8) TRACE_CLK(p.status, 3 + it);
                 }
                 if (!ok) break;

@@ -473,7 +473,7 @@ __global__ void nvfp4_quantize_weights_kernel(const double* Wt, uint8_t* wcodes,
         for (int j = 0; j < 16; j += 2) crow[b * 8 + j / 2] = static_cast<uint8_t>(codes[j] | (codes[j + 1] << 4));
     }
     const int nr = n & 127;
-    *reinterpret_cast<uint32_t*>(wsf + (static_cast<size_t>(n >> 7) * g.nkb64p + kb) * 512 + (nr & 31) * 16 + (nr >> 5) * 4) = sfword;
+    *reinterpret_cast<uint32_t*>(wsf + wsf_atom_offset(n >> 7, kb, g.nkb64p) + (nr & 31) * 16 + (nr >> 5) * 4) = sfword;
 }
 
 // wh[n][i] = bf16(Wt[i][n]) * 2^-(ex+ew)  (exact: a power of two), zero padded to r_pad.
@@ -502,7 +502,7 @@ __global__ void nvfp4_export_weights_kernel(const uint8_t* wcodes, const uint8_t
     if (j < nb && sf_out) {
         const int nr = n & 127;
         sf_out[static_cast<size_t>(j) * g.N + n] =
-            wsf[(static_cast<size_t>(n >> 7) * g.nkb64p + (j >> 2)) * 512 + (nr & 31) * 16 + (nr >> 5) * 4 + (j & 3)];
+            wsf[wsf_atom_offset(n >> 7, j >> 2, g.nkb64p) + (nr & 31) * 16 + (nr >> 5) * 4 + (j & 3)];
     }
     if (j < g.r && wh_out)
         wh_out[static_cast<size_t>(j) * g.N + n] =
@@ -831,7 +831,7 @@ dirotq_status_t launch_prepare_nvfp4(const dirotq_layer* L, const void* W, int w
                                                                           g.K, g.N);
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     if (cudaMemsetAsync(meta, 0, 64, stream) != cudaSuccess) return DIROTQ_ERR_CUDA;
-    if (cudaMemsetAsync(blob + L->lay.off_wscale, 0, static_cast<size_t>((g.N + 127) / 128) * g.nkb64p * 512, stream) !=
+    if (cudaMemsetAsync(blob + L->lay.off_wscale, 0, wsf_bytes(g.N, g.nkb64p), stream) !=
         cudaSuccess)
         return DIROTQ_ERR_CUDA;
     nvfp4_amax_kernel<<<592, 256, 0, stream>>>(scratch, g, meta);
@@ -873,7 +873,7 @@ dirotq_status_t launch_prepare_nvfp4_ph(const dirotq_layer* L, const void* W, in
     if (!launch_ok()) return DIROTQ_ERR_CUDA;
     // the scratch now holds [r + K][N]: quantized exactly like the dense form's folded weight
     if (cudaMemsetAsync(meta, 0, 64, stream) != cudaSuccess) return DIROTQ_ERR_CUDA;
-    if (cudaMemsetAsync(blob + L->lay.off_wscale, 0, static_cast<size_t>((g.N + 127) / 128) * g.nkb64p * 512, stream) !=
+    if (cudaMemsetAsync(blob + L->lay.off_wscale, 0, wsf_bytes(g.N, g.nkb64p), stream) !=
         cudaSuccess)
         return DIROTQ_ERR_CUDA;
     nvfp4_amax_kernel<<<592, 256, 0, stream>>>(scratch, g, meta);
