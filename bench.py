@@ -430,7 +430,7 @@ def run_ours(args):
     # DRAM bytes of one launch of the dominant kernel, from the ncu capture summarised under profiles/
     # (qkv shape; read + write).  Static: a profiler is never run inside the benchmark.
     # one launch each, on the qkv shape (3072 -> 9216, M = 4608); other shapes' launches were not captured
-    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 72.8e6, "rotate_quant_kernel": 48.5e6, "nvfp4_gemm_kernel": 60.5e6}
+    NCU_TRAFFIC_QKV = {"w4a4_gemm_kernel": 72.8e6, "rotate_quant_kernel": 48.5e6, "nvfp4_gemm_kernel": 57.0e6}
     sm_hz = (clocks or {}).get("sm_mhz") or 1850.0
     elem_steps = sum(M * N * (-(-(K - RANK) // GROUP)) for _, K, N in FLUX_SHAPES)
     alu_peak = 148 * (128.0 / 2.0) * sm_hz * 1e6  # element-steps/s: 2 fused multiply-adds each, 128 fp32 lanes per SM
