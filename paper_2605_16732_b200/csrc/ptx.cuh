@@ -285,46 +285,6 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 
-// The same with release ordering at cluster scope: what this thread wrote into another CTA's shared memory before the
-// arrival is visible to a thread of that CTA that then passes mbar_wait_cluster on the barrier.
-__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {  // acquire at cluster scope
-    uint32_t ok;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait like mbar_wait, for a barrier that threads of other CTAs of the cluster arrive on.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
-                                                  unsigned long long limit_ns = kWaitLimitNs) {
-    unsigned long long t0 = 0;
-#pragma unroll 1
-    for (uint32_t spins = 1;; ++spins) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((spins & 255u) == 0) {
-            if (*abort_flag != 0) return false;
-            const unsigned long long now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            if (now - t0 > limit_ns) {
-                *abort_flag = code;
-                atomicCAS(status, 0, code);
-                return false;
-            }
-        }
-    }
-}
-
 __device__ __forceinline__ uint32_t cluster_nctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
@@ -343,10 +303,7 @@ __device__ __forceinline__ void st_shared_u64(uint32_t addr, uint64_t v) {
     asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 
-// 8-byte store into the shared memory of a CTA of the cluster (address from map_to_cta) and 8-byte load from this CTA's own.
-__device__ __forceinline__ void st_cluster_u64(uint32_t cluster_addr, uint64_t v) {
-    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(cluster_addr), "l"(v) : "memory");
-}
+// 8-byte load from this CTA's shared memory.
 __device__ __forceinline__ uint64_t ld_shared_u64(uint32_t addr) {
     uint64_t v;
     asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
@@ -386,11 +343,6 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, 
         "}\n" ::"r"(d_tmem),
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
         : "memory");
-}
-
-// Generic-proxy writes of this thread -> visible to the tensor core, whichever CTA of the pair issues the MMA.
-__device__ __forceinline__ void fence_proxy_async_all() {
-    asm volatile("fence.proxy.async;" ::: "memory");
 }
 
 // Arrival, on completion of all MMAs issued so far by this thread, on the barrier at `bar`'s offset in the shared memory

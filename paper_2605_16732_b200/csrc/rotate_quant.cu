@@ -270,7 +270,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
         tma_prefetch_desc(&tmap_qt);
-        if constexpr (FMT == 0 || FMT == 2 || FMT == 3 || FMT == 4) tma_prefetch_desc(&tmap_out);
+        tma_prefetch_desc(&tmap_out);
         if constexpr (PH) {
             tma_prefetch_desc(&tmap_x2);
             tma_prefetch_desc(&tmap_had);
@@ -482,7 +482,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             // W4A8 path's fp32 coefficients (128 bytes per row at a time) go into the warp's staging tile instead, swizzled
             // so that a quarter-warp's pieces fall into different banks, and one lane hands the tile to a TMA store
             // (tmap_out), which writes whole sectors and clips at M and at the row's width.
-            constexpr bool STAGED = EPI_WARPS == 8 && (FMT == 0 || FMT == 2 || FMT == 3 || FMT == 4);
+            constexpr bool STAGED = EPI_WARPS == 8;
             const uint32_t sbuf = smem_base + STORE_OFFSET + static_cast<uint32_t>(warp - 2) * 4096u;
             const int row0w = row - lane;  // the warp's first row
             auto stage_piece128 = [&](int piece, uint4 val) {  // rows of 128 bytes, 128-byte swizzle
@@ -552,17 +552,37 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 if constexpr (FMT == 1) {
                     // NVFP4: four blocks of 16 per 64-column chunk; one 32-bit word of scale bytes per chunk
                     static_assert(FMT == 0 || G == 64, "the NVFP4 epilogue works on 64-column chunks");
-                    if (col0 < p.K4 && row_ok) {
+                    if (col0 < p.K4) {
                         const float ex_scale = __uint_as_float(static_cast<uint32_t>(127 + p.ex) << 23);
                         const float ex_inv = __uint_as_float(static_cast<uint32_t>(127 - p.ex) << 23);
                         uint32_t sfword = 0;
                         uint8_t* crow = reinterpret_cast<uint8_t*>(p.codes) + static_cast<size_t>(row) * (p.K4 / 2) + col0 / 2;
+                        if constexpr (STAGED) {
+                            if (lane == 0) bulk_wait_group_read_all();  // the staging tile's previous contents have been read
+                            __syncwarp();
+                        }
 #pragma unroll
                         for (int b = 0; b < 4; ++b) {
                             uint32_t w0 = 0, w1 = 0;
                             if (16 * b < nlow) sfword |= nvfp4_block16(v + 16 * b, kPre, ex_inv, ex_scale, w0, w1) << (8 * b);
-                            *reinterpret_cast<uint2*>(crow + 8 * b) = make_uint2(w0, w1);  // zero in the padding slots
+                            if constexpr (STAGED) {
+                                // 32 bytes of codes per row: rows of 32 bytes, 32-byte swizzle (16-byte piece b / 2)
+                                const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 32u +
+                                                     (static_cast<uint32_t>((b >> 1) ^ ((lane >> 2) & 1)) << 4) + (b & 1) * 8u;
+                                asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst), "r"(w0), "r"(w1) : "memory");
+                            } else if (row_ok) {
+                                *reinterpret_cast<uint2*>(crow + 8 * b) = make_uint2(w0, w1);  // zero in the padding slots
+                            }
                         }
+                        if constexpr (STAGED) {
+                            fence_proxy_async_smem();  // these writes -> visible to the copy engine
+                            __syncwarp();
+                            if (lane == 0 && row0w < p.M) {
+                                tma_store_2d(&tmap_out, sbuf, col0 / 2, row0w);
+                                bulk_commit_group();
+                            }
+                        }
+                      if (row_ok) {
                         const int mr = row & 127;
                         *reinterpret_cast<uint32_t*>(p.xsf + (static_cast<size_t>(row >> 7) * p.nkb64p + (col0 >> 6)) * 512 +
                                                      (mr & 31) * 16 + (mr >> 5) * 4) = sfword;
@@ -571,6 +591,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                             for (int a = (col0 >> 6) + 1; a < p.nkb64p; ++a)
                                 *reinterpret_cast<uint32_t*>(p.xsf + (static_cast<size_t>(row >> 7) * p.nkb64p + a) * 512 +
                                                              (mr & 31) * 16 + (mr >> 5) * 4) = 0u;
+                      }
                     }
                 } else if constexpr (FMT == 3) {
                     // W4A8, first pass: the rotated low-precision coefficients go out as fp32 and the token's maximum is
@@ -814,16 +835,16 @@ dirotq_status_t set_rotation_plan(int plan) {
 }
 
 // The tensor map the epilogue's TMA stores go through: the INT4 activation codes (one byte each, [M][K_lp], boxes of 32 rows x
-// one group) or, on the W4A8 path, the fp32 coefficients ([M][K_lp], boxes of 32 rows x 32 values).  NVFP4 layers store
-// directly and get a copy of `unused` (any valid map).
+// one group), the NVFP4 codes (two per byte, [M][K4/2], boxes of 32 rows x 32 bytes) or, on the W4A8 path, the fp32 coefficients
+// ([M][K_lp], boxes of 32 rows x 32 values).
 static dirotq_status_t encode_out_map(CUtensorMap* out, const Geometry& g, const RotateArgs& a, const CUtensorMap& unused) {
     if (g.fmt == 3)
         return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.xtilde, (uint64_t)g.K_lp, (uint64_t)a.M, (uint64_t)g.K_lp * 4,
                               32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (g.fmt == 1) {
-        *out = unused;
-        return DIROTQ_OK;
-    }
+    (void)unused;
+    if (g.fmt == 1)  // NVFP4: two codes per byte, 32 bytes per row and 64-column chunk
+        return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K4 / 2, (uint64_t)a.M, (uint64_t)g.K4 / 2, 32, 32,
+                              CU_TENSOR_MAP_SWIZZLE_32B);
     return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.codes, (uint64_t)g.K_lp, (uint64_t)a.M, (uint64_t)g.K_lp, g.G, 32,
                           g.G == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
 }
