@@ -51,7 +51,10 @@ template <int BN, bool PAIR = false>
 struct Plan {
     static constexpr int NB = BN / 128;               // 128-column blocks per tile
     static constexpr int NB_DATA = PAIR ? 1 : NB;     // ... whose weight codes this CTA holds
-    static constexpr int STAGES = PAIR ? 5 : (BN == 128 ? 6 : 4);
+    // outputs through per-warp staging tiles and TMA stores where the shared memory allows it: the pair plan, and the
+    // 128-column plan with five stages instead of six
+    static constexpr bool STAGED_OUT = PAIR || BN == 128;
+    static constexpr int STAGES = PAIR ? 5 : (BN == 128 ? 5 : 4);
     static constexpr int ACC_BUFS = BN == 128 ? 2 : 1;
     static constexpr int B_BYTES = NB_DATA * 128 * 128;  // 16 / 32 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + (1 + NB) * SF_BYTES;  // 36 / 54 KB (pairs: 38 KB)
@@ -60,7 +63,7 @@ struct Plan {
     // pairs: one 32-row x 128-byte staging tile per epilogue warp (1024-byte aligned: 128-byte swizzle), from which the outputs
     // leave as TMA stores
     static constexpr int STORE_OFFSET = (BIAS_OFFSET + 2 * BN * 4 + 1023) / 1024 * 1024;
-    static constexpr int SMEM_BYTES = PAIR ? STORE_OFFSET + NUM_EPI_WARPS * 4096 + 1024 : BIAS_OFFSET + 2 * BN * 4 + 1024;
+    static constexpr int SMEM_BYTES = STAGED_OUT ? STORE_OFFSET + NUM_EPI_WARPS * 4096 + 1024 : BIAS_OFFSET + 2 * BN * 4 + 1024;
     static constexpr int TMEM_SF_BASE = ACC_BUFS * BN;    // columns 256.. hold the scale factors
     static constexpr int SF_COLS = 16 * (1 + NB);         // per stage: 16 columns for the tokens, 16 per 128 output columns
     static_assert(TMEM_SF_BASE + STAGES * SF_COLS <= 512, "tensor memory plan");
@@ -193,7 +196,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
         tma_prefetch_desc(&tmap_wcodes);
         tma_prefetch_desc(&tmap_xh);
         tma_prefetch_desc(&tmap_wh);
-        if constexpr (PAIR) tma_prefetch_desc(&tmap_y);
+        if constexpr (P::STAGED_OUT) tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) {
         if constexpr (PAIR) {
@@ -438,7 +441,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
             else mbar_arrive(tempty_bar(acc));
-            if constexpr (PAIR) {
+            if constexpr (P::STAGED_OUT) {
                 // Outputs leave through shared memory: a thread holds one token row, so direct stores would be 32 scattered
                 // 16-byte pieces per instruction, and a clock trace showed 7600-9500 cycles of them per tile, during which
                 // the next tile's operand loads ran at half their rate.  Each warp converts 64 columns of its 32 rows into
@@ -495,7 +498,7 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
             if (warp == 4 && lane == 0 && tcount == 0) TRACE_CLK(p.status, 29);
             if (warp == 4 && lane == 0 && tcount >= 1 && tcount <= 2) TRACE_CLK(p.status, 3 * tcount);
         }
-        if constexpr (PAIR) {
+        if constexpr (P::STAGED_OUT) {
             if (lane == 0) bulk_wait_group_all();  // this warp's stores are performed before the CTA leaves
         }
     }
@@ -549,12 +552,14 @@ static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4Ge
     if (!opt_in.ensure(nvfp4_gemm_kernel<BN, PAIR>, 0, L->device, Plan<BN, PAIR>::SMEM_BYTES)) return DIROTQ_ERR_CUDA;
     // the weight-side tensor maps have 128-row boxes: a 256-column tile fetches two of them per operand (one per CTA of a pair)
     cudaError_t err;
-    if constexpr (PAIR) {
-        // the outputs leave as TMA stores of 32 rows x 64 columns (128-byte swizzle in shared memory)
-        CUtensorMap tmap_y;
+    // where the outputs leave as TMA stores: boxes of 32 rows x 64 columns (128-byte swizzle in shared memory)
+    CUtensorMap tmap_y = tmap_xh;  // (unused by the plan that stores directly)
+    if constexpr (Plan<BN, PAIR>::STAGED_OUT) {
         st = encode_tmap_2d(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.y, (uint64_t)g.N, (uint64_t)a.M, (uint64_t)g.N * 2, 64, 32,
                             CU_TENSOR_MAP_SWIZZLE_128B);
         if (st != DIROTQ_OK) return st;
+    }
+    if constexpr (PAIR) {
         const int pair_tiles = ((a.M + 2 * BM - 1) / (2 * BM)) * ((g.N + BN - 1) / BN);
         const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
         err = launch_kernel_pairs(nvfp4_gemm_kernel<BN, PAIR>, 2 * pairs, NUM_THREADS, Plan<BN, PAIR>::SMEM_BYTES, stream, true,
@@ -563,7 +568,7 @@ static dirotq_status_t launch_nvfp4_gemm_bn(const dirotq_layer* L, const Nvfp4Ge
         const int num_tiles = ((a.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
         const int grid = num_tiles < sms ? num_tiles : sms;
         err = launch_kernel(nvfp4_gemm_kernel<BN>, grid, NUM_THREADS, Plan<BN>::SMEM_BYTES, stream, true,
-                            tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, tmap_xh /* unused without pairs */, p);
+                            tmap_codes, L->tmap_wpacked, tmap_xh, L->tmap_wh, tmap_y, p);
     }
     return err == cudaSuccess ? DIROTQ_OK : DIROTQ_ERR_CUDA;
 }
