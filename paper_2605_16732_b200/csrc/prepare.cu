@@ -346,19 +346,32 @@ __global__ void a8_quantize_kernel(const float* xtilde, const unsigned int* rowm
     if (lane == 0) xscale[m] = s;
     const float* xr = xtilde + static_cast<size_t>(m) * g.K_lp;
     int8_t* cr = codes + static_cast<size_t>(m) * g.K_lp;
-    for (int j = lane * 4; j < g.K_lp; j += 128) {
-        uint32_t word = 0;
-        if (j < g.K_l) {  // K_l is a multiple of 16: the four values are all real or all padding
-            const float4 v = *reinterpret_cast<const float4*>(xr + j);
-            const float vv[4] = {v.x, v.y, v.z, v.w};
+    // four independent 16-byte loads in flight per thread (a warp covers 2 KB of its row per step): with one load per
+    // step the pass ran at the latency of a load, not at the rate of the memory
+    constexpr int UNROLL = 4;
+    for (int j0 = lane * 4; j0 < g.K_lp; j0 += 128 * UNROLL) {
+        float4 v[UNROLL];
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                float q = slow ? (s != 0.f ? vv[t] / s : 0.f) : vv[t] * inv;
-                q = fminf(fmaxf(q, -127.0f), 127.0f);
-                word |= (static_cast<uint32_t>(__float2int_rn(q)) & 0xFFu) << (8 * t);
-            }
+        for (int u = 0; u < UNROLL; ++u) {
+            const int j = j0 + 128 * u;
+            v[u] = j < g.K_l ? __ldcs(reinterpret_cast<const float4*>(xr + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        *reinterpret_cast<uint32_t*>(cr + j) = word;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int j = j0 + 128 * u;
+            if (j >= g.K_lp) break;
+            uint32_t word = 0;
+            if (j < g.K_l) {  // K_l is a multiple of 16: the four values are all real or all padding
+                const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    float q = slow ? (s != 0.f ? vv[t] / s : 0.f) : vv[t] * inv;
+                    q = fminf(fmaxf(q, -127.0f), 127.0f);
+                    word |= (static_cast<uint32_t>(__float2int_rn(q)) & 0xFFu) << (8 * t);
+                }
+            }
+            *reinterpret_cast<uint32_t*>(cr + j) = word;
+        }
     }
 }
 
