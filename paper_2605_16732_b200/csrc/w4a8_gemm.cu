@@ -98,6 +98,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 30);
     const int num_m_blocks = (p.M + BM - 1) / BM;
     const int num_n_blocks = (p.N + BN - 1) / BN;
     const int num_tiles = num_m_blocks * num_n_blocks;
@@ -154,6 +155,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                         mbar_arrive_expect_tx(full_bar(s), A_BYTES + BP_BYTES);
                         tma_load_2d(st, &tmap_codes, full_bar(s), i * BKC, m0);
                         tma_load_2d(st + BP_OFFSET, &tmap_wpacked, full_bar(s), i * (BKC / 2), n0);
+                        if (it >= 10 && it <= 12) TRACE_CLK(p.status, it - 1);
                     } else {
                         mbar_arrive_expect_tx(full_bar(s), A_BYTES + BU_BYTES);
                         tma_load_2d(st, &tmap_xh, full_bar(s), (i - p.num_kb) * 64, m0);
@@ -192,6 +194,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     const uint64_t adesc = umma_desc_sw128(st);
                     const uint64_t bdesc = umma_desc_sw128(st + A_BYTES);
                     if (!elect_one()) continue;
+                    if (it >= 10 && it <= 12) TRACE_CLK(p.status, it + 8);
                     if (i < p.num_kb) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k) umma_i8(tacc, adesc + 2 * k, bdesc + 2 * k, idesc_i8, (i | k) != 0);
@@ -229,6 +232,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     : "memory");
                 ok = any_failed == 0;
                 if (!ok) break;
+                if (u == 0 && it >= 10 && it <= 12) TRACE_CLK(p.status, it + 2);
                 if (i < p.num_kb) {
                     // 16-byte piece idx = u + 128 j of the packed tile: row = idx / 4 = u / 4 + 32 j, piece c = u % 4; the
                     // swizzle phase row % 8 and the piece do not depend on j
@@ -257,6 +261,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                     fence_proxy_async_smem();
                 }
+                if (u == 0 && it >= 10 && it <= 12) TRACE_CLK(p.status, it + 5);
                 mbar_arrive(unp_bar(s));  // every lane arrives for itself: a warp barrier followed by one elected lane's arrival costs about a hundred cycles more
             }
         }
@@ -304,6 +309,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
             ok = any_failed == 0;
             if (!ok) break;
             tc_fence_after_sync();
+            if (warp == 2 + NUM_UNPACK_WARPS && lane == 0 && tcount < 3) TRACE_CLK(p.status, 21 + 3 * tcount);
             const int row = m0 + q * 32 + lane;
             const float sx = row < p.M ? __ldg(p.xscale + row) : 0.f;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc_i * 2 * BN;
@@ -318,6 +324,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                 if (c == (half + 1) * CPH - 1) {
                     tc_fence_before_sync();
                     mbar_arrive(tempty_bar(acc_i));
+                    if (warp == 2 + NUM_UNPACK_WARPS && lane == 0 && tcount < 3) TRACE_CLK(p.status, 22 + 3 * tcount);
                 }
                 const int col = n0 + c * 32;
                 if (row < p.M) {
@@ -338,32 +345,37 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     // staging tile (64-byte swizzle: a quarter-warp's pieces fall into different banks) and one lane hands
                     // it to a TMA store, which writes whole sectors and clips at M and N.
                     const uint32_t sbuf = smem_base + P::STORE_OFFSET + static_cast<uint32_t>(warp - (2 + NUM_UNPACK_WARPS)) * 2048u;
-                    if (lane == 0) bulk_wait_group_read_all();  // the tile's previous contents have been read
-                    __syncwarp();
-                    {
+                    // the chunk is converted first; only then does the warp wait for the copy engine to have read the staging
+                    // tile's previous contents (this epilogue is exposed: nothing else hides that read)
+                    uint32_t packed[16];
 #pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            {
-                                float o[8];
+                    for (int j = 0; j < 32; j += 8) {
+                        float o[8];
 #pragma unroll
-                                for (int t = 0; t < 8; t += 4) {
-                                    const float4 sw = *reinterpret_cast<const float4*>(s_sw + c * 32 + j + t);
-                                    const float4 b = *reinterpret_cast<const float4*>(s_b + c * 32 + j + t);
-                                    const float sws[4] = {sw.x, sw.y, sw.z, sw.w}, bs[4] = {b.x, b.y, b.z, b.w};
+                        for (int t = 0; t < 8; t += 4) {
+                            const float4 sw = *reinterpret_cast<const float4*>(s_sw + c * 32 + j + t);
+                            const float4 b = *reinterpret_cast<const float4*>(s_b + c * 32 + j + t);
+                            const float sws[4] = {sw.x, sw.y, sw.z, sw.w}, bs[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-                                    for (int e = 0; e < 4; ++e) {
-                                        // the accumulator holds 16 P (exact); |P| < 2^24, so the conversion is exact too
-                                        const float pf = static_cast<float>(static_cast<int32_t>(acc[j + t + e]) >> 4);
-                                        o[t + e] = fmaf(pf * sx, sws[e], __uint_as_float(lr[j + t + e])) + bs[e];
-                                    }
-                                }
-                                const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 64u +
-                                                     (static_cast<uint32_t>((j >> 3) ^ ((lane >> 1) & 3)) << 4);
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16x2(o[0], o[1])),
-                                             "r"(pack_bf16x2(o[2], o[3])), "r"(pack_bf16x2(o[4], o[5])), "r"(pack_bf16x2(o[6], o[7]))
-                                             : "memory");
+                            for (int e = 0; e < 4; ++e) {
+                                // the accumulator holds 16 P (exact); |P| < 2^24, so the conversion is exact too
+                                const float pf = static_cast<float>(static_cast<int32_t>(acc[j + t + e]) >> 4);
+                                o[t + e] = fmaf(pf * sx, sws[e], __uint_as_float(lr[j + t + e])) + bs[e];
                             }
                         }
+                        packed[(j >> 1) + 0] = pack_bf16x2(o[0], o[1]);
+                        packed[(j >> 1) + 1] = pack_bf16x2(o[2], o[3]);
+                        packed[(j >> 1) + 2] = pack_bf16x2(o[4], o[5]);
+                        packed[(j >> 1) + 3] = pack_bf16x2(o[6], o[7]);
+                    }
+                    if (lane == 0) bulk_wait_group_read_all();  // the tile's previous contents have been read
+                    __syncwarp();
+#pragma unroll
+                    for (int pc = 0; pc < 4; ++pc) {
+                        const uint32_t dst = sbuf + static_cast<uint32_t>(lane) * 64u + (static_cast<uint32_t>(pc ^ ((lane >> 1) & 3)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[4 * pc]), "r"(packed[4 * pc + 1]),
+                                     "r"(packed[4 * pc + 2]), "r"(packed[4 * pc + 3])
+                                     : "memory");
                     }
                     fence_proxy_async_smem();  // these writes -> visible to the copy engine
                     __syncwarp();
@@ -373,6 +385,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
                     }
                 }
             }
+            if (warp == 2 + NUM_UNPACK_WARPS && lane == 0 && tcount < 3) TRACE_CLK(p.status, 23 + 3 * tcount);
         }
         if constexpr (!kPartials) {
             if (lane == 0) bulk_wait_group_all();  // this warp's stores are performed before the CTA leaves
