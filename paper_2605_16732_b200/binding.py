@@ -44,6 +44,15 @@ class DirotqError(RuntimeError):
 _lib = None
 
 
+def use_library(path: str) -> None:
+    """Makes the binding load another build of the library (before its first use): the integer-path fallback or the
+    diagnostic build of paper_2605_16732_b200.build."""
+    global _LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("a library is loaded already")
+    _LIB_PATH = path
+
+
 def lib() -> ctypes.CDLL:
     """Loads libdirotq.so (must have been built: ``python -m paper_2605_16732_b200.build``)."""
     global _lib

@@ -70,6 +70,15 @@ def build_i8(force: bool = False, verbose: bool = False) -> str:
     return _build(LIB_I8, os.path.join(HERE, "_build_i8"), ["-DDIROTQ_I8_PATH"], force, verbose)
 
 
+# The diagnostic build: block 0 of every kernel stamps the SM clock at marked points of its roles into spare slots of the workspace's
+# status block (TRACE_CLK in csrc/ptx.cuh; the slot map is at each kernel's first stamp).  paper_2605_16732_b200/trace.py reads it.
+LIB_TRACE = os.path.join(HERE, "libdirotq_trace.so")
+
+
+def build_trace(force: bool = False, verbose: bool = False) -> str:
+    return _build(LIB_TRACE, os.path.join(HERE, "_build_trace"), ["-DDIROTQ_TRACE"], force, verbose)
+
+
 if __name__ == "__main__":
-    fn = build_i8 if "--i8" in sys.argv else build
+    fn = build_i8 if "--i8" in sys.argv else build_trace if "--trace" in sys.argv else build
     print(fn(force="--force" in sys.argv, verbose="-v" in sys.argv))

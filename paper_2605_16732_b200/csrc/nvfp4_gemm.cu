@@ -169,6 +169,10 @@ nvfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_c
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // Trace build (TRACE_CLK), stages 6..8 of the block's first tile: slots 9..11 producer has issued the stage, 12..14 first copier warp
+    // sees it landed, 15..17 / 18..20 first / second copier warp has committed its scale copies, 21..23 MMA warp sees the scales
+    // ready, 24..26 it has committed the stage's MMAs; tiles 0, 1, 2 of the first epilogue warp: accumulator seen / released / outputs
+    // handed over in slots 27..29, 1..3, 4..6; slot 30 entry.
     if (threadIdx.x == 0) TRACE_CLK(p.status, 30);
     const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
     constexpr int TILE_ROWS = PAIR ? 2 * BM : BM;  // token rows of a tile (of the pair's tile)

@@ -245,6 +245,10 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // Trace build (TRACE_CLK): slot 9 entry, 10 set-up done, 11 previous grid ended, 12 producer has filled the ring once, 13 producer has
+    // issued everything, 14 / 15 MMA warp sees the first / ninth stage, 16 MMA warp has committed its last tile, 17 first epilogue
+    // warp sees its first accumulator, 18 that warp has finished its last tile.
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 9);
 
     const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
     constexpr int TILE_ROWS = PAIR ? 2 * BM : BM;  // token rows of a tile (of the pair's tile)
@@ -290,7 +294,9 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     if constexpr (PAIR) cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 10);
     grid_dependency_wait();
+    if (threadIdx.x == 0) TRACE_CLK(p.status, 11);
     // the second kernel of the layer may be scheduled onto SMs as this grid's CTAs leave them (it waits for the whole
     // grid before it reads anything)
     grid_launch_dependents();
@@ -344,6 +350,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                             tma_load_2d(sa + j * SUB_BYTES, &tmap_x, full_bar(s), (kb + j) * BK, m0);
                             tma_load_2d(sa + j * SUB_BYTES + A_BYTES, &tmap_qt, full_bar(s), (kb + j) * BK, n0);
                         }
+                        if (it == STAGES - 1) TRACE_CLK(p.status, 12);
                         continue;
                     }
                     if constexpr (PAIR) {
@@ -357,8 +364,10 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         tma_load_2d(sa, &tmap_x, full_bar(s), kb * BK, m0);
                         tma_load_2d(sa + A_BYTES, &tmap_qt, full_bar(s), kb * BK, n0);
                     }
+                    if (it == STAGES - 1) TRACE_CLK(p.status, 12);
                 }
             }
+            if (lane == 0) TRACE_CLK(p.status, 13);
             if (lane != 0) {
                 // one lane looks after the loads in flight
             } else if (!ok && PAIR && cta_rank != 0) {
@@ -424,6 +433,8 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint64_t adesc = umma_desc_sw128(sa);
                     const uint64_t bdesc = umma_desc_sw128(sa + A_BYTES);
                     if (!elect_one()) continue;
+                    if (it == 0) TRACE_CLK(p.status, 14);
+                    if (it == 8) TRACE_CLK(p.status, 15);
                     if constexpr (KSUB > 1) {
                         const int nsub = min(KSUB, num_kb - kb);
                         for (int j = 0; j < nsub; ++j) {
@@ -451,6 +462,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 if (ok && elect_one()) {
                     if constexpr (PAIR) umma_commit_pair(tfull_bar(acc), 3);  // both CTAs' epilogue warps
                     else umma_commit(tfull_bar(acc));
+                    TRACE_CLK(p.status, 16);
                 }
             }
         }
@@ -498,6 +510,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             };
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE)) { ok = false; break; }
+            if (warp == 2 && lane == 0 && tcount == 0) TRACE_CLK(p.status, 17);
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (BM == 256 ? half * 256 : acc * BN);
 
@@ -777,6 +790,7 @@ rotate_quant_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     }
 
     if (warp >= 2 && lane == 0) bulk_wait_group_all();  // an epilogue warp's TMA stores are performed before the CTA leaves
+    if (warp == 2 && lane == 0) TRACE_CLK(p.status, 18);
     // ---------------------------------------------------------------- teardown
     if constexpr (PAIR) {
         if (warp == 1 && lane == 0 && cta_rank == 0 && *abort_flag != 0) {  // a wait gave up: let issued MMAs finish first

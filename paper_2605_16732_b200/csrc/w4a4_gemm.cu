@@ -202,6 +202,10 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // Trace build (TRACE_CLK): slot 9 entry, 10 set-up done, 11 previous grid ended, 12 / 13 producer has issued its first k-block /
+    // everything, 14 / 15 first unpack warp sees / has expanded the first stage, 16 / 17 / 18 MMA warp starts the first / fifth / last
+    // k-block, 19 it has committed the last tile, 20 first epilogue warp sees its first accumulator, 21 starts its ninth K-group, 22 has
+    // folded in the last group, 23 the rank-r tile, 24 has stored its last outputs.
     if (threadIdx.x == 0) TRACE_CLK(p.status, 9);
 
     const int num_m_blocks = (p.M + BM - 1) / BM;

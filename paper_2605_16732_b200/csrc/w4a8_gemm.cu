@@ -98,6 +98,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_codes, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // Trace build (TRACE_CLK), stages 10..12 of the block's first tile: slots 9..11 producer has issued the stage, 12..14 first unpack warp
+    // sees it landed, 15..17 it has expanded it, 18..20 MMA warp starts on it; tiles 0, 1, 2 of the first epilogue warp: accumulators
+    // seen / released / outputs handed over in slots 21..23, 24..26, 27..29; slot 30 entry.
     if (threadIdx.x == 0) TRACE_CLK(p.status, 30);
     const int num_m_blocks = (p.M + BM - 1) / BM;
     const int num_n_blocks = (p.N + BN - 1) / BN;
