@@ -107,3 +107,14 @@ def test_memory_report_runs_without_a_gpu(capsys):
     for row in rows:
         assert row["layer_bytes"] - row["layer_bytes_without_rotation"] >= 2 * row["K"] ** 2
         assert 2.5 < row["x_smaller_than_bf16_without_rotation"] < 3.6
+
+
+def test_the_other_builds_export_the_same_interface():
+    # the integer-path fallback and the diagnostic build are the same sources with one definition each: same symbols
+    from paper_2605_16732_b200 import build
+    for path in (build.build_i8(), build.build_trace()):
+        other = ctypes.CDLL(path)
+        for name in binding.EXPORTED:
+            assert getattr(other, name) is not None, (path, name)
+        other.dirotq_version.restype = ctypes.c_int
+        assert other.dirotq_version() >= 100
